@@ -1,0 +1,280 @@
+"""CPU oracle, part 2: the residual networks the paper trains, cut into units.
+
+TEST INFRASTRUCTURE ONLY (see oracle/layers.py).
+
+The paper splits the layer indices {1..L} into K contiguous groups q(k)
+(Section 3.1, first paragraph).  Here the network is an ordered list of units
+-- stem, residual blocks 1..3n, head -- and a split point is a block index, so
+module 1 owns the stem and module K owns the head.  Each unit offers a forward
+that returns what its backward will need (the "saved computation graph" of
+Fig. 1(b)) and a backward that is the chain rule of Eq. 8 / Eq. 9 through its
+layers.
+
+The paper defines no architecture; these are the standard definitions of the
+networks it cites (Tables 3-6):
+  * "resnet6n2": post-activation basic blocks, 3 stages of n blocks,
+       block(x) = ReLU( BN(conv3x3(ReLU(BN(conv3x3_s(x))))) + sc(x) ),
+       sc = identity, or BN(conv1x1_s(x)) when the shape changes;
+       stem = ReLU(BN(conv3x3(image))); head = GAP -> FC -> softmax-CE.
+  * "wrn": pre-activation basic blocks,
+       o = ReLU(BN(x)); block(x) = conv3x3(ReLU(BN(conv3x3_s(o)))) + sc,
+       sc = x, or conv1x1_s(o) when the shape changes;
+       stem = conv3x3(image); head = ReLU(BN(.)) -> GAP -> FC -> softmax-CE.
+
+Parameter order inside a unit (and therefore inside a module's flat vector) is
+the order of `param_spec()`; convolution weights are [C_out, R, S, C_in].
+"""
+from dataclasses import dataclass, field
+from typing import Tuple
+import numpy as np
+
+from . import layers as L
+
+
+@dataclass
+class Arch:
+    family: str = "resnet6n2"          # "resnet6n2" | "wrn"
+    n_per_stage: int = 1
+    widths: Tuple[int, int, int] = (16, 32, 64)
+    stem_width: int = 16
+    in_h: int = 32
+    in_w: int = 32
+    in_c: int = 3
+    num_classes: int = 10
+    batch: int = 128
+    bn_eps: float = 1e-5
+
+
+# ----------------------------------------------------------------------------
+# units
+# ----------------------------------------------------------------------------
+class Stem:
+    def __init__(self, arch):
+        self.ci, self.co, self.eps = arch.in_c, arch.stem_width, arch.bn_eps
+        self.with_bn = arch.family == "resnet6n2"
+        self.name = "stem"
+
+    def param_spec(self):
+        spec = [("conv.w", "conv", (self.co, 3, 3, self.ci))]
+        if self.with_bn:
+            spec += [("bn.g", "bn_gamma", (self.co,)), ("bn.b", "bn_beta", (self.co,))]
+        return spec
+
+    def forward(self, x, p):
+        c = L.conv2d_forward(x, p["conv.w"], 1, 1)
+        if not self.with_bn:
+            return c, dict(x=x)
+        b, sv = L.batchnorm_forward(c, p["bn.g"], p["bn.b"], self.eps)
+        y = L.relu_forward(b)
+        return y, dict(x=x, sv=sv, y=y)
+
+    def backward(self, dy, ctx, p):
+        g = {}
+        if self.with_bn:
+            db = L.relu_backward(dy, ctx["y"])
+            dc, g["bn.g"], g["bn.b"] = L.batchnorm_backward(db, ctx["sv"], p["bn.g"])
+        else:
+            dc = dy
+        dx, g["conv.w"] = L.conv2d_backward(dc, ctx["x"], p["conv.w"], 1, 1)
+        return dx, g
+
+
+class BasicBlock:
+    """Post-activation block of the 6n+2 networks."""
+
+    def __init__(self, arch, ci, co, stride, index):
+        self.ci, self.co, self.stride, self.eps = ci, co, stride, arch.bn_eps
+        self.proj = (ci != co) or (stride != 1)
+        self.name = "block%d" % index
+
+    def param_spec(self):
+        spec = [("conv1.w", "conv", (self.co, 3, 3, self.ci)),
+                ("bn1.g", "bn_gamma", (self.co,)), ("bn1.b", "bn_beta", (self.co,)),
+                ("conv2.w", "conv", (self.co, 3, 3, self.co)),
+                ("bn2.g", "bn_gamma", (self.co,)), ("bn2.b", "bn_beta", (self.co,))]
+        if self.proj:
+            spec += [("sc.w", "conv", (self.co, 1, 1, self.ci)),
+                     ("scbn.g", "bn_gamma", (self.co,)), ("scbn.b", "bn_beta", (self.co,))]
+        return spec
+
+    def forward(self, x, p):
+        c1 = L.conv2d_forward(x, p["conv1.w"], self.stride, 1)
+        b1, sv1 = L.batchnorm_forward(c1, p["bn1.g"], p["bn1.b"], self.eps)
+        a1 = L.relu_forward(b1)
+        c2 = L.conv2d_forward(a1, p["conv2.w"], 1, 1)
+        b2, sv2 = L.batchnorm_forward(c2, p["bn2.g"], p["bn2.b"], self.eps)
+        ctx = dict(x=x, sv1=sv1, a1=a1, sv2=sv2)
+        if self.proj:
+            cs = L.conv2d_forward(x, p["sc.w"], self.stride, 0)
+            sc, ctx["svs"] = L.batchnorm_forward(cs, p["scbn.g"], p["scbn.b"], self.eps)
+        else:
+            sc = x
+        y = L.relu_forward(b2 + sc)
+        ctx["y"] = y
+        return y, ctx
+
+    def backward(self, dy, ctx, p):
+        g = {}
+        dsum = L.relu_backward(dy, ctx["y"])          # gradient of b2 + sc
+        dc2, g["bn2.g"], g["bn2.b"] = L.batchnorm_backward(dsum, ctx["sv2"], p["bn2.g"])
+        da1, g["conv2.w"] = L.conv2d_backward(dc2, ctx["a1"], p["conv2.w"], 1, 1)
+        db1 = L.relu_backward(da1, ctx["a1"])
+        dc1, g["bn1.g"], g["bn1.b"] = L.batchnorm_backward(db1, ctx["sv1"], p["bn1.g"])
+        dx, g["conv1.w"] = L.conv2d_backward(dc1, ctx["x"], p["conv1.w"], self.stride, 1)
+        if self.proj:
+            dcs, g["scbn.g"], g["scbn.b"] = L.batchnorm_backward(dsum, ctx["svs"], p["scbn.g"])
+            dxs, g["sc.w"] = L.conv2d_backward(dcs, ctx["x"], p["sc.w"], self.stride, 0)
+            dx = dx + dxs
+        else:
+            dx = dx + dsum
+        return dx, g
+
+
+class PreActBlock:
+    """Pre-activation block of the wide residual networks."""
+
+    def __init__(self, arch, ci, co, stride, index):
+        self.ci, self.co, self.stride, self.eps = ci, co, stride, arch.bn_eps
+        self.proj = (ci != co) or (stride != 1)
+        self.name = "block%d" % index
+
+    def param_spec(self):
+        spec = [("bn1.g", "bn_gamma", (self.ci,)), ("bn1.b", "bn_beta", (self.ci,)),
+                ("conv1.w", "conv", (self.co, 3, 3, self.ci)),
+                ("bn2.g", "bn_gamma", (self.co,)), ("bn2.b", "bn_beta", (self.co,)),
+                ("conv2.w", "conv", (self.co, 3, 3, self.co))]
+        if self.proj:
+            spec += [("sc.w", "conv", (self.co, 1, 1, self.ci))]
+        return spec
+
+    def forward(self, x, p):
+        b1, sv1 = L.batchnorm_forward(x, p["bn1.g"], p["bn1.b"], self.eps)
+        o = L.relu_forward(b1)
+        c1 = L.conv2d_forward(o, p["conv1.w"], self.stride, 1)
+        b2, sv2 = L.batchnorm_forward(c1, p["bn2.g"], p["bn2.b"], self.eps)
+        a2 = L.relu_forward(b2)
+        c2 = L.conv2d_forward(a2, p["conv2.w"], 1, 1)
+        if self.proj:
+            sc = L.conv2d_forward(o, p["sc.w"], self.stride, 0)
+        else:
+            sc = x
+        y = c2 + sc
+        return y, dict(sv1=sv1, o=o, sv2=sv2, a2=a2)
+
+    def backward(self, dy, ctx, p):
+        g = {}
+        da2, g["conv2.w"] = L.conv2d_backward(dy, ctx["a2"], p["conv2.w"], 1, 1)
+        db2 = L.relu_backward(da2, ctx["a2"])
+        dc1, g["bn2.g"], g["bn2.b"] = L.batchnorm_backward(db2, ctx["sv2"], p["bn2.g"])
+        do, g["conv1.w"] = L.conv2d_backward(dc1, ctx["o"], p["conv1.w"], self.stride, 1)
+        if self.proj:
+            dos, g["sc.w"] = L.conv2d_backward(dy, ctx["o"], p["sc.w"], self.stride, 0)
+            do = do + dos
+        db1 = L.relu_backward(do, ctx["o"])
+        dx, g["bn1.g"], g["bn1.b"] = L.batchnorm_backward(db1, ctx["sv1"], p["bn1.g"])
+        if not self.proj:
+            dx = dx + dy
+        return dx, g
+
+
+class Head:
+    """Classifier and loss.  The paper's f is abstract (Eq. 1); the task is
+    classification, so f is the mean softmax cross-entropy over the batch."""
+
+    def __init__(self, arch, feat):
+        self.feat, self.classes, self.eps = feat, arch.num_classes, arch.bn_eps
+        self.with_bn = arch.family == "wrn"
+        self.name = "head"
+
+    def param_spec(self):
+        spec = []
+        if self.with_bn:
+            spec += [("bn.g", "bn_gamma", (self.feat,)), ("bn.b", "bn_beta", (self.feat,))]
+        spec += [("fc.w", "fc_w", (self.classes, self.feat)), ("fc.b", "fc_b", (self.classes,))]
+        return spec
+
+    def forward_loss(self, x, labels, p):
+        ctx = dict(shape=x.shape)
+        if self.with_bn:
+            b, ctx["sv"] = L.batchnorm_forward(x, p["bn.g"], p["bn.b"], self.eps)
+            x = L.relu_forward(b)
+            ctx["a"] = x
+        pooled = L.gap_forward(x)
+        logits = L.fc_forward(pooled, p["fc.w"], p["fc.b"])
+        loss, probs = L.softmax_xent_forward(logits, labels)
+        ctx.update(pooled=pooled, probs=probs, labels=labels, logits=logits)
+        return loss, ctx
+
+    def backward(self, ctx, p):
+        g = {}
+        dlogits = L.softmax_xent_backward(ctx["probs"], ctx["labels"])
+        dpooled, g["fc.w"], g["fc.b"] = L.fc_backward(dlogits, ctx["pooled"], p["fc.w"])
+        dx = L.gap_backward(dpooled, ctx["shape"])
+        if self.with_bn:
+            db = L.relu_backward(dx, ctx["a"])
+            dx, g["bn.g"], g["bn.b"] = L.batchnorm_backward(db, ctx["sv"], p["bn.g"])
+        return dx, g
+
+
+# ----------------------------------------------------------------------------
+# network = stem + 3n blocks + head, and its partition into K modules
+# ----------------------------------------------------------------------------
+def build_units(arch):
+    units = [Stem(arch)]
+    block_cls = BasicBlock if arch.family == "resnet6n2" else PreActBlock
+    ci = arch.stem_width
+    index = 0
+    for stage in range(3):
+        for j in range(arch.n_per_stage):
+            index += 1
+            stride = 2 if (stage > 0 and j == 0) else 1
+            units.append(block_cls(arch, ci, arch.widths[stage], stride, index))
+            ci = arch.widths[stage]
+    units.append(Head(arch, ci))
+    return units
+
+
+def split_units(units, split_after_block):
+    """Partition [stem, block1..blockN, head] at the given block indices
+    (ascending, 1-based): the paper's q(1)..q(K) with module 1 holding the stem
+    and module K the head."""
+    n_blocks = len(units) - 2
+    cuts = list(split_after_block)
+    assert all(1 <= c < n_blocks for c in cuts) and cuts == sorted(set(cuts)), cuts
+    bounds = [0] + [c + 1 for c in cuts] + [len(units)]
+    return [units[bounds[k]:bounds[k + 1]] for k in range(len(bounds) - 1)]
+
+
+def module_param_spec(module_units):
+    """[(qualified name, kind, shape)] in flat-vector order."""
+    spec = []
+    for u in module_units:
+        for name, kind, shape in u.param_spec():
+            spec.append((u.name + "." + name, kind, shape))
+    return spec
+
+
+def spec_size(spec):
+    return int(sum(int(np.prod(s)) for _, _, s in spec))
+
+
+def unflatten(flat, spec):
+    """Views into `flat`, keyed by qualified name."""
+    out, off = {}, 0
+    for name, _, shape in spec:
+        n = int(np.prod(shape))
+        out[name] = flat[off:off + n].reshape(shape)
+        off += n
+    assert off == flat.size
+    return out
+
+
+def flatten(named, spec, dtype):
+    return np.concatenate([np.asarray(named[name], dtype=dtype).reshape(-1) for name, _, _ in spec]) \
+        if spec else np.zeros(0, dtype=dtype)
+
+
+def unit_params(named, unit):
+    """The sub-dictionary of one unit with the unit prefix stripped."""
+    pre = unit.name + "."
+    return {k[len(pre):]: v for k, v in named.items() if k.startswith(pre)}

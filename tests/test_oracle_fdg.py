@@ -1,0 +1,304 @@
+"""Pins for oracle/fdg.py and oracle/nets.py: what the paper and the
+mathematics fix about the FDG iteration, checked against independent code
+(torch autograd / torch.optim in tests/torch_ref.py, closed forms, the paper's
+printed values)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import fdg_synth as S
+from oracle import fdg, nets
+from tests import torch_ref
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def tiny_arch(family="resnet6n2", n=1, batch=4, hw=8, classes=5):
+    if family == "wrn":
+        return nets.Arch(family="wrn", n_per_stage=n, widths=(8, 12, 16), stem_width=4,
+                         in_h=hw, in_w=hw, num_classes=classes, batch=batch)
+    return nets.Arch(n_per_stage=n, widths=(4, 8, 12), stem_width=4, in_h=hw, in_w=hw,
+                     num_classes=classes, batch=batch)
+
+
+def make(arch, K, splits, **kw):
+    cfg = fdg.FDGConfig(K=K, split_after_block=tuple(splits), **kw)
+    o = fdg.FDGOracle(arch, cfg)
+    for k in range(1, K + 1):
+        o.set_params(k, S.init_params(3, k, o.param_spec(k), jitter=True))
+    return o
+
+
+def batch(arch, t):
+    return (S.images(5, t, arch.batch, arch.in_h, arch.in_w, arch.in_c).astype(np.float64),
+            S.labels(5, t, arch.batch, arch.num_classes))
+
+
+def all_params(o):
+    return np.concatenate([o.get_params(k) for k in range(1, o.K + 1)])
+
+
+def relerr(a, b):
+    return np.abs(a - b).max() / max(np.abs(b).max(), 1e-300)
+
+
+# ---------------------------------------------------------------- schedule --
+def test_schedule_printed_example():
+    for line in open(os.path.join(GOLD, "schedule_k3_fig1.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        K, k, b, tf, tb = map(int, line.split())
+        assert fdg.forward_batch(tf, k) == b
+        assert fdg.backward_batch(tb, k, K) == b
+        assert tb - tf == 2 * (K - k)
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 4])
+@pytest.mark.parametrize("order", [fdg.BACKWARD_FIRST, fdg.FORWARD_FIRST])
+def test_schedule_log_matches_closed_forms(K, order):
+    """Forward of batch b in module k at iteration b+k-1, backward at b+2K-k-1
+    (Section 3.1); the top module has no delay; nothing runs for batches < 1."""
+    arch = tiny_arch(n=2)
+    o = make(arch, K, [2, 3, 4][:K - 1], order=order, beta=0.5)
+    T = 12
+    for t in range(1, T + 1):
+        o.step(*batch(arch, t))
+    rows = {(r["t"], r["k"]): r for r in o.log}
+    assert len(rows) == T * K
+    for t in range(1, T + 1):
+        for k in range(1, K + 1):
+            r = rows[(t, k)]
+            ef, eb = t - k + 1, t - 2 * K + k + 1
+            assert r["tau_f"] == (ef if ef >= 1 else -1)
+            assert r["tau_b"] == (eb if eb >= 1 else -1)
+    # delay between forward and backward of one batch is 2(K-k)
+    fwd_at = {(r["k"], r["tau_f"]): r["t"] for r in o.log if r["tau_f"] > 0}
+    bwd_at = {(r["k"], r["tau_b"]): r["t"] for r in o.log if r["tau_b"] > 0}
+    for (k, b), tb in bwd_at.items():
+        assert tb - fwd_at[(k, b)] == 2 * (K - k)
+    # stashed reading: the backward of a batch sees the version its forward saw
+    ver_f = {(r["k"], r["tau_f"]): r["ver_f"] for r in o.log if r["tau_f"] > 0}
+    for r in o.log:
+        if r["tau_b"] > 0:
+            assert r["ver_b"] == ver_f[(r["k"], r["tau_b"])]
+    # live contexts never exceed 2(K-k) (+1 when the forward runs first)
+    for k in range(1, K):
+        assert len(o.modules[k - 1].saved) == 2 * (K - k)
+    assert len(o.modules[K - 1].saved) == 0
+
+
+# ------------------------------------------------------- K = 1 is BP + SGD --
+@pytest.mark.parametrize("family", ["resnet6n2", "wrn"])
+def test_k1_equals_backprop_sgd(family):
+    """With K=1 the delay 2(K-k) is zero and Eq. 14 is Eq. 6: FDG must follow
+    torch autograd + torch.optim.SGD(momentum, weight_decay) step for step."""
+    arch = tiny_arch(family, n=1)
+    o = make(arch, 1, [], beta=0.3, lr=0.05, momentum=0.9, weight_decay=5e-4)
+    theta = torch.tensor(all_params(o), requires_grad=True)
+    opt = torch.optim.SGD([theta], lr=0.05, momentum=0.9, weight_decay=5e-4)
+    for t in range(1, 6):
+        x, y = batch(arch, t)
+        loss_o = o.step(x, y)
+        opt.zero_grad()
+        loss_t = torch_ref.network_loss(arch, theta, torch.tensor(x), torch.tensor(y))
+        loss_t.backward()
+        assert relerr(o.get_grads(1), theta.grad.numpy()) < 1e-9
+        opt.step()
+        assert abs(loss_o - float(loss_t.detach())) < 1e-10
+        assert relerr(o.get_params(1), theta.detach().numpy()) < 1e-10
+
+
+# ------------------------------------------------------ gradient shrinking --
+@pytest.mark.parametrize("family,K,splits,order", [
+    ("resnet6n2", 2, [2], fdg.BACKWARD_FIRST), ("resnet6n2", 3, [1, 2], fdg.BACKWARD_FIRST),
+    ("resnet6n2", 4, [1, 3, 5], fdg.FORWARD_FIRST), ("wrn", 3, [1, 3], fdg.BACKWARD_FIRST)])
+def test_lr0_shrunk_gradient_is_beta_power_times_bp(family, K, splits, order):
+    """Eq. 16 / Eq. 17: with the weights frozen (lr = 0) module k's gradient for
+    batch b is beta^(K-k) times the back-propagation gradient of batch b, and
+    the gradient it hands down carries the same factor."""
+    beta = 0.6
+    arch = tiny_arch(family, n=2)
+    o = make(arch, K, splits, beta=beta, lr=0.0, order=order)
+    theta = all_params(o)
+    sizes = [o.param_count(k) for k in range(1, K + 1)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    bp = {}
+    checked = 0
+    for t in range(1, 2 * K + 4):
+        x, y = batch(arch, t)
+        xt = torch.tensor(x, requires_grad=True)
+        th = torch.tensor(theta, requires_grad=True)
+        loss = torch_ref.network_loss(arch, th, xt, torch.tensor(y))
+        gth, gx = torch.autograd.grad(loss, [th, xt])
+        bp[t] = (gth.numpy(), gx.numpy(), float(loss.detach()))
+        loss_o = o.step(x, y)
+        if loss_o is not None:
+            assert abs(loss_o - bp[t - K + 1][2]) < 1e-10
+        for r in o.log[-K:]:
+            if r["tau_b"] < 1:
+                continue
+            k, b = r["k"], r["tau_b"]
+            ref = beta ** (K - k) * bp[b][0][offs[k - 1]:offs[k]]
+            assert relerr(o.get_grads(k), ref) < 1e-9
+            checked += 1
+            if k == 1:
+                bb, gin = o.input_grad[1]
+                assert bb == b and relerr(gin, beta ** (K - 1) * bp[b][1]) < 1e-9
+    assert checked >= K * 3
+    assert np.array_equal(all_params(o), theta)          # lr = 0: nothing moved
+
+
+def test_beta_one_is_unshrunk():
+    """beta = 1: "the GS process is not used"; and beta only enters through the
+    received gradient, so the top module's first update is beta-independent."""
+    arch = tiny_arch(n=1)
+    outs = []
+    for beta in (1.0, 0.5):
+        o = make(arch, 2, [1], beta=beta, lr=0.1)
+        for t in range(1, 3):
+            o.step(*batch(arch, t))
+        outs.append((o.get_params(1), o.get_params(2), o.input_grad[2][1]))
+    # t=2: module 2 did its first forward/backward/update: no beta anywhere
+    assert np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][2], outs[1][2])
+    # module 1 has not been updated yet (first update at t = 2K-k = 3)
+    assert np.array_equal(outs[0][0], outs[1][0])
+
+
+# ------------------------------------- delayed gradient with stale weights --
+@pytest.mark.parametrize("reading", [fdg.STASHED, fdg.CURRENT])
+@pytest.mark.parametrize("order", [fdg.BACKWARD_FIRST, fdg.FORWARD_FIRST])
+def test_delayed_gradient_identity(reading, order):
+    """Eq. 13 with shrinking (Eq. 17): in the stashed reading module k's gradient
+    for batch b equals beta^(K-k) * d f_b / d theta_k of the network in which
+    every module j carries the weights it had when it forwarded batch b.  The
+    right-hand side is recomputed by autograd from recorded snapshots.  In the
+    "current" reading the identity must fail once the weights have moved."""
+    K, beta = 3, 0.7
+    arch = tiny_arch(n=1, batch=3)
+    o = make(arch, K, [1, 2], beta=beta, lr=0.05, order=order, weight_reading=reading)
+    sizes = [o.param_count(k) for k in range(1, K + 1)]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    snaps, data = {}, {}
+    inner = o._forward
+
+    def recording_forward(k, tau, x):
+        snaps[(k, tau)] = o.modules[k - 1].theta.copy()
+        return inner(k, tau, x)
+
+    o._forward = recording_forward
+    worst = 0.0
+    n = 0
+    for t in range(1, 14):
+        data[t] = batch(arch, t)
+        o.step(*data[t])
+        for r in o.log[-K:]:
+            b, k = r["tau_b"], r["k"]
+            if b < 1:
+                continue
+            theta = np.concatenate([snaps[(j, b)] for j in range(1, K + 1)])
+            _, g = torch_ref.loss_and_grad(arch, theta, *data[b])
+            err = relerr(o.get_grads(k), beta ** (K - k) * g[offs[k - 1]:offs[k]])
+            if k < K and r["t"] > 2 * K:          # delayed modules after weights have moved
+                worst = max(worst, err); n += 1
+            if reading == fdg.STASHED or k == K:
+                assert err < 1e-8, (t, k, err)
+    assert n > 0
+    if reading == fdg.CURRENT:
+        assert worst > 1e-4          # a different (inexact) gradient, as expected
+    else:
+        assert worst < 1e-8
+
+
+def test_orders_differ_only_in_weights_seen_by_forward():
+    """Appendix A's forward-first variant: the forward of iteration t runs before
+    the update of iteration t, so it sees one update fewer."""
+    arch = tiny_arch(n=1)
+    logs = {}
+    for order in (fdg.BACKWARD_FIRST, fdg.FORWARD_FIRST):
+        o = make(arch, 2, [1], beta=0.5, order=order)
+        for t in range(1, 8):
+            o.step(*batch(arch, t))
+        logs[order] = {(r["t"], r["k"]): r for r in o.log}
+    for key, rb in logs[fdg.BACKWARD_FIRST].items():
+        rf = logs[fdg.FORWARD_FIRST][key]
+        assert (rb["tau_f"], rb["tau_b"]) == (rf["tau_f"], rf["tau_b"])
+        if key[1] == 1 and rb["tau_b"] >= 1:
+            assert rb["ver_f"] == rf["ver_f"] + 1
+        else:
+            assert rb["ver_f"] == rf["ver_f"]
+
+
+# ------------------------------------------------------------- optimiser ----
+def test_sgd_closed_forms():
+    """Constant gradient g, no weight decay: v_n = g (1-mu^n)/(1-mu).
+    Zero gradient, no momentum: theta_n = theta_0 (1 - lr*wd)^n."""
+    arch = tiny_arch(n=1)
+    o = make(arch, 1, [], lr=0.1, momentum=0.9, weight_decay=0.0)
+    g = np.linspace(-1, 1, o.param_count(1))
+    th0 = o.get_params(1)
+    for n in range(1, 6):
+        o._update(1, g)
+        assert relerr(o.get_momentum(1), g * (1 - 0.9 ** n) / (1 - 0.9)) < 1e-13
+    total = sum((1 - 0.9 ** n) / (1 - 0.9) for n in range(1, 6))
+    assert relerr(o.get_params(1) - th0, -0.1 * total * g) < 1e-12
+    o = make(arch, 1, [], lr=0.1, momentum=0.0, weight_decay=0.01)
+    th0 = o.get_params(1)
+    for n in range(4):
+        o._update(1, np.zeros_like(th0))
+    assert relerr(o.get_params(1), th0 * (1 - 0.1 * 0.01) ** 4) < 1e-13
+
+
+# ---------------------------------------------------------- architectures ---
+def test_param_counts_printed_in_paper():
+    for line in open(os.path.join(GOLD, "param_counts_table3.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        fam, n, widths, stem, printed = line.split()
+        arch = nets.Arch(family=fam, n_per_stage=int(n), stem_width=int(stem),
+                         widths=tuple(int(w) for w in widths.split(",")))
+        units = nets.build_units(arch)
+        total = sum(nets.spec_size(nets.module_param_spec([u])) for u in units)
+        # the table rounds loosely (1.73M is printed as 1.70M): agree within 2 %
+        assert abs(total / 1e6 - float(printed)) <= 0.02 * float(printed), (line, total)
+
+
+def test_split_and_flat_layout():
+    arch = tiny_arch(n=2)
+    units = nets.build_units(arch)
+    parts = nets.split_units(units, (2, 4))
+    assert [len(p) for p in parts] == [3, 2, 3]
+    assert parts[0][0].name == "stem" and parts[-1][-1].name == "head"
+    whole = nets.module_param_spec(units)
+    assert [s for p in parts for s in nets.module_param_spec(p)] == whole
+    with pytest.raises(AssertionError):
+        nets.split_units(units, (4, 2))
+    with pytest.raises(AssertionError):
+        nets.split_units(units, (6,))
+
+
+def test_planted_mistakes_are_caught(monkeypatch):
+    """The pins above must notice a dropped shortcut gradient and a transposed
+    dgrad operand; this guards the guards."""
+    from oracle import layers as L
+    arch = tiny_arch(n=1)
+
+    def run():
+        o = make(arch, 1, [], lr=0.05)
+        x, y = batch(arch, 1)
+        o.step(x, y)
+        _, g = torch_ref.loss_and_grad(arch, all_params(make(arch, 1, [])), x, y)
+        return relerr(o.get_grads(1), g)
+
+    assert run() < 1e-9
+    real = L.conv2d_backward
+    monkeypatch.setattr(L, "conv2d_backward",
+                        lambda dy, x, w, s, p: (lambda dx, dw: (dx, dw[:, ::-1]))(*real(dy, x, w, s, p)))
+    assert run() > 1e-3
+    monkeypatch.setattr(L, "conv2d_backward", real)
+    real_relu = L.relu_backward
+    monkeypatch.setattr(L, "relu_backward", lambda dy, y: dy)
+    assert run() > 1e-3
+    monkeypatch.setattr(L, "relu_backward", real_relu)
+    assert run() < 1e-9
