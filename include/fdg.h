@@ -1,0 +1,207 @@
+/*
+ * libfdg -- fully decoupled training with delayed gradients (FDG) on one B200.
+ *
+ * The network (a residual CNN) is split into K modules; each module is a worker
+ * on its own CUDA stream.  One call of fdg_step() is one iteration t of
+ * Algorithm I of the FDG paper for every module k = 1..K:
+ *
+ *   forward   (Section 3.1 "forward")   module k forwards batch t-k+1, the output
+ *                                       module k-1 produced in iteration t-1;
+ *   backward  (Section 3.1 "backward",  module k back-propagates batch t-2K+k+1 from
+ *              Eq. 10, Eq. 15)          the gradient module k+1 produced in iteration
+ *                                       t-1, multiplied by the shrinking factor beta
+ *                                       (modules k < K only), through the activations
+ *                                       saved by the forward of that same batch;
+ *   update    (Eq. 11)                  SGD with momentum and weight decay on the
+ *                                       module's own parameters;
+ *   handoff   (Section 3.1              output activation -> module k+1, input gradient
+ *              "communication")         -> module k-1, both consumed in iteration t+1.
+ *
+ * Conventions
+ *   - Every function returns an fdg_status; none throws, aborts or exits.
+ *   - "dev" pointers are device pointers on the device that was current at
+ *     fdg_create(); "host or device" pointers may be either (unified addressing).
+ *   - The library allocates no device memory: the caller passes one workspace of
+ *     fdg_workspace_bytes() bytes (256-byte aligned) that the context owns until
+ *     fdg_destroy().
+ *   - Activations are NHWC; convolution weights are [C_out][R][S][C_in].
+ *   - Modules and blocks are numbered from 1 as in the paper.
+ *
+ * Flat parameter layout of a module (fp32), the order fdg_param_layout() reports:
+ *   units in network order: stem (module 1), residual blocks, head (module K);
+ *   FDG_RESNET_6N2: stem  = conv.w, bn.gamma, bn.beta
+ *                   block = conv1.w, bn1.gamma, bn1.beta, conv2.w, bn2.gamma, bn2.beta
+ *                           [, sc.w (1x1), scbn.gamma, scbn.beta  when the shape changes]
+ *                   head  = fc.w [classes][features], fc.b
+ *   FDG_WRN:        stem  = conv.w
+ *                   block = bn1.gamma, bn1.beta, conv1.w, bn2.gamma, bn2.beta, conv2.w
+ *                           [, sc.w (1x1)  when the shape changes]
+ *                   head  = bn.gamma, bn.beta, fc.w, fc.b
+ */
+#ifndef FDG_H_
+#define FDG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fdg_ctx fdg_ctx;            /* opaque; created by fdg_create, freed by fdg_destroy */
+typedef void* fdg_stream;                  /* a cudaStream_t, passed as a plain pointer (NULL = default stream) */
+
+typedef enum {
+  FDG_OK = 0,
+  FDG_ERR_INVALID_ARG = 1,
+  FDG_ERR_WORKSPACE_TOO_SMALL = 2,
+  FDG_ERR_CUDA = 3,
+  FDG_ERR_STATE = 4,
+  FDG_ERR_UNSUPPORTED = 5,
+  FDG_ERR_NONFINITE = 6,
+  FDG_ERR_TIMEOUT = 7
+} fdg_status;
+
+enum { FDG_RESNET_6N2 = 0, FDG_WRN = 1 };                 /* fdg_arch.family   */
+enum { FDG_BACKWARD_FIRST = 0, FDG_FORWARD_FIRST = 1 };   /* fdg_config.order  */
+enum { FDG_STASHED = 0, FDG_CURRENT = 1 };                /* fdg_config.weight_reading */
+enum { FDG_FP32_CUDACORE = 0, FDG_BF16_TC = 1 };          /* fdg_config.precision */
+enum { FDG_PARAM_CONV = 0, FDG_PARAM_BN_GAMMA = 1, FDG_PARAM_BN_BETA = 2,
+       FDG_PARAM_FC_W = 3, FDG_PARAM_FC_B = 4 };          /* fdg_param_entry.kind */
+
+/* The network: a stem convolution, three stages of n_per_stage residual blocks
+ * (stride 2 at the first block of stages 2 and 3), a classifier.  The paper
+ * defines no architecture of its own; these are the networks of its tables. */
+typedef struct {
+  int family;            /* FDG_RESNET_6N2 (post-activation blocks) | FDG_WRN (pre-activation blocks) */
+  int n_per_stage;       /* blocks per stage (ResNet-110: 18, WRN-28-10: 4) */
+  int widths[3];         /* channels of the three stages */
+  int stem_width;        /* output channels of the stem convolution */
+  int in_h, in_w, in_c;  /* image size */
+  int num_classes;
+  int batch;
+  float bn_eps;
+} fdg_arch;
+
+/* "Required: learning rate, number of split modules K, gradient shrinking factor
+ * beta" (Algorithm I), plus the optimiser constants of the experiments section. */
+typedef struct {
+  int K;                          /* number of modules, >= 1 */
+  const int* split_after_block;   /* K-1 ascending block indices in [1, 3n-1]: module k ends after that block */
+  float beta;                     /* shrinking factor, 0 < beta <= 1 (Eq. 15) */
+  float lr, momentum, weight_decay;
+  int order;                      /* FDG_BACKWARD_FIRST = Algorithm I; FDG_FORWARD_FIRST = Appendix A variant */
+  int weight_reading;             /* FDG_STASHED: delayed backward uses the weights of that batch's forward (Eq. 10) */
+  int precision;                  /* FDG_FP32_CUDACORE: fp32 storage and arithmetic;
+                                     FDG_BF16_TC: bf16 activations/weights for the convolutions, fp32 accumulation,
+                                     fp32 master weights, statistics and loss */
+  int serial;                     /* 1 = run all modules on the caller's stream in order (debug) */
+} fdg_config;
+
+typedef struct {            /* one tensor of a module's flat parameter vector */
+  int kind;                 /* FDG_PARAM_* */
+  int unit;                 /* 0 = stem, b = residual block b (1-based), -1 = head */
+  int dims[4];              /* conv: C_out,R,S,C_in; fc_w: classes,features,1,1; vectors: n,1,1,1 */
+  size_t offset;            /* first element in the flat vector */
+  size_t count;             /* number of elements */
+} fdg_param_entry;
+
+typedef struct {            /* one row of the schedule log: what module k did in iteration t */
+  int64_t t;                /* iteration, from 1 */
+  int32_t k;                /* module, from 1 */
+  int64_t tau_f;            /* batch forwarded (t-k+1), or -1 while the pipeline fills */
+  int64_t tau_b;            /* batch back-propagated (t-2K+k+1), or -1 */
+  int64_t ver_f;            /* number of updates the weights used by the forward had received, or -1 */
+  int64_t ver_b;            /* same for the weights used by the backward, or -1 */
+  int32_t slot_f;           /* activation-FIFO slot written by the forward, or -1 */
+  int32_t slot_b;           /* activation-FIFO slot read by the backward, or -1 */
+} fdg_sched_entry;
+
+/* Bytes of device workspace fdg_create() needs for this network and configuration.
+ * Errors: FDG_ERR_INVALID_ARG (null pointer, bad sizes or split points),
+ * FDG_ERR_UNSUPPORTED (a shape the kernels do not cover). */
+fdg_status fdg_workspace_bytes(const fdg_arch* arch, const fdg_config* cfg, size_t* out_bytes);
+
+/* Builds a context in `dev_workspace` (caller-owned, 256-byte aligned, `bytes` >=
+ * fdg_workspace_bytes; must outlive the context).  `streams` is an array of K
+ * cudaStream_t owned by the caller, or NULL to let the library create its own.
+ * Parameters start at zero: call fdg_set_params for every module before stepping.
+ * The iteration counter starts at t = 0 with an empty pipeline.  Blocks the host
+ * until the workspace has been cleared. */
+fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_workspace, size_t bytes,
+                      const fdg_stream* streams, fdg_ctx** out_ctx);
+
+/* Waits for all enqueued work, releases streams/events the library created, frees the
+ * host-side context.  The workspace returns to the caller. */
+fdg_status fdg_destroy(fdg_ctx* ctx);
+
+/* Number of fp32 parameters of module `module` (1..K). */
+fdg_status fdg_param_count(const fdg_ctx* ctx, int module, size_t* out_n);
+
+/* Table of the module's parameter tensors in flat order.  Writes at most `cap` entries
+ * to `dst` (may be NULL with cap = 0) and the total number to *out_n. */
+fdg_status fdg_param_layout(const fdg_ctx* ctx, int module, fdg_param_entry* dst, size_t cap, size_t* out_n);
+
+/* Copies n = fdg_param_count floats from `src` (host or device) into the module's
+ * master weights and refreshes the copies the kernels compute with; momentum is left
+ * as it is.  Blocks the host.  Meant for initialisation or a cold restart: batches
+ * in flight keep their saved activations but lose their stashed weight versions. */
+fdg_status fdg_set_params(fdg_ctx* ctx, int module, const float* src, size_t n);
+/* Same for the momentum buffer (checkpoint restore). */
+fdg_status fdg_set_momentum(fdg_ctx* ctx, int module, const float* src, size_t n);
+
+/* Copy out (to host or device memory; blocks the host until the module's stream has
+ * drained): fp32 master weights; the last shrunk delayed gradient ghat_theta of Eq. 15
+ * before weight decay is added (zeros before the module's first backward); momentum. */
+fdg_status fdg_get_params(fdg_ctx* ctx, int module, float* dst, size_t n);
+fdg_status fdg_get_grads(fdg_ctx* ctx, int module, float* dst, size_t n);
+fdg_status fdg_get_momentum(fdg_ctx* ctx, int module, float* dst, size_t n);
+
+/* Learning rate gamma_t used by every update enqueued from the next fdg_step on
+ * (Algorithm I takes gamma_t per iteration). */
+fdg_status fdg_set_lr(fdg_ctx* ctx, float lr);
+
+/* One iteration of Algorithm I.  `images_dev` is batch t, fp32 [batch][in_h][in_w][in_c];
+ * `labels_dev` int32 [batch] in [0, num_classes).  Both are read only by work enqueued
+ * behind `stream` inside this call, so the caller may overwrite them as soon as `stream`
+ * has passed the step.  `loss_dev` (nullable, device) receives the mean cross-entropy of
+ * batch t-K+1 computed in this iteration; it is written on a module stream, so read it
+ * after fdg_sync; it is left untouched while t < K.  Does not block the host.
+ * Errors: FDG_ERR_INVALID_ARG (null ctx/images/labels), FDG_ERR_CUDA (a launch failed;
+ * the context is then unusable), a latched asynchronous error. */
+fdg_status fdg_step(fdg_ctx* ctx, fdg_stream stream, const float* images_dev, const int32_t* labels_dev,
+                    float* loss_dev);
+
+/* Makes `stream` wait for every module stream, then blocks the host until `stream` is idle.
+ * Returns FDG_ERR_NONFINITE if any loss computed since the last call was NaN/Inf,
+ * FDG_ERR_CUDA on an asynchronous CUDA error. */
+fdg_status fdg_sync(fdg_ctx* ctx, fdg_stream stream);
+
+/* The most recent output activation of module k (1..K-1), and the most recent gradient
+ * with respect to the input of module k (2..K; the gradient with respect to the images
+ * is never formed, so k = 1 is FDG_ERR_INVALID_ARG), as fp32 NHWC to host or device memory.  `n` must equal the tensor's element
+ * count, which fdg_boundary_elems reports.  *batch_index receives the batch the tensor
+ * belongs to, or -1 (and nothing is copied) while the pipeline has not produced one.
+ * The input gradient is returned as produced, i.e. before the receiver applies beta.
+ * Both block the host. */
+fdg_status fdg_get_module_output(fdg_ctx* ctx, int module, float* dst, size_t n, int64_t* batch_index);
+fdg_status fdg_get_input_grad(fdg_ctx* ctx, int module, float* dst, size_t n, int64_t* batch_index);
+/* Element counts of those two tensors: the output of module k (0 for k = K) and its input. */
+fdg_status fdg_boundary_elems(const fdg_ctx* ctx, int module, size_t* out_elems, size_t* in_elems);
+
+/* Copies at most `cap` rows of the schedule log (oldest first) and writes the number
+ * of rows recorded so far to *out_n.  The log keeps every row of the last 4096 iterations. */
+fdg_status fdg_get_schedule_log(const fdg_ctx* ctx, fdg_sched_entry* dst, size_t cap, size_t* out_n);
+
+/* Number of kernel launches the library has enqueued since fdg_create. */
+fdg_status fdg_launch_count(const fdg_ctx* ctx, uint64_t* out_n);
+
+const char* fdg_status_string(fdg_status s);
+/* Human-readable description of the last error on this context ("" if none).  The
+ * pointer stays valid until the next call on the context. */
+const char* fdg_last_error(const fdg_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FDG_H_ */

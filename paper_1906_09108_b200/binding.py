@@ -1,0 +1,233 @@
+"""ctypes binding of libfdg: the same entry points as include/fdg.h, argument
+marshalling only.  Every step of the FDG path runs inside the CUDA library; there
+is no fallback -- if the library is missing or fails to load, importing raises.
+
+PyTorch appears here only as the owner of device memory and streams.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfdg.so")
+
+FDG_OK = 0
+STATUS_NAMES = {0: "FDG_OK", 1: "FDG_ERR_INVALID_ARG", 2: "FDG_ERR_WORKSPACE_TOO_SMALL", 3: "FDG_ERR_CUDA",
+                4: "FDG_ERR_STATE", 5: "FDG_ERR_UNSUPPORTED", 6: "FDG_ERR_NONFINITE", 7: "FDG_ERR_TIMEOUT"}
+FDG_RESNET_6N2, FDG_WRN = 0, 1
+FDG_BACKWARD_FIRST, FDG_FORWARD_FIRST = 0, 1
+FDG_STASHED, FDG_CURRENT = 0, 1
+FDG_FP32_CUDACORE, FDG_BF16_TC = 0, 1
+PARAM_KINDS = {0: "conv", 1: "bn_gamma", 2: "bn_beta", 3: "fc_w", 4: "fc_b"}
+
+EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count", "fdg_param_layout",
+           "fdg_set_params", "fdg_set_momentum", "fdg_get_params", "fdg_get_grads", "fdg_get_momentum",
+           "fdg_set_lr", "fdg_step", "fdg_sync", "fdg_get_module_output", "fdg_get_input_grad",
+           "fdg_boundary_elems", "fdg_get_schedule_log", "fdg_launch_count", "fdg_status_string",
+           "fdg_last_error"]
+
+
+class fdg_arch(C.Structure):
+    _fields_ = [("family", C.c_int), ("n_per_stage", C.c_int), ("widths", C.c_int * 3), ("stem_width", C.c_int),
+                ("in_h", C.c_int), ("in_w", C.c_int), ("in_c", C.c_int), ("num_classes", C.c_int),
+                ("batch", C.c_int), ("bn_eps", C.c_float)]
+
+
+class fdg_config(C.Structure):
+    _fields_ = [("K", C.c_int), ("split_after_block", C.POINTER(C.c_int)), ("beta", C.c_float), ("lr", C.c_float),
+                ("momentum", C.c_float), ("weight_decay", C.c_float), ("order", C.c_int),
+                ("weight_reading", C.c_int), ("precision", C.c_int), ("serial", C.c_int)]
+
+
+class fdg_param_entry(C.Structure):
+    _fields_ = [("kind", C.c_int), ("unit", C.c_int), ("dims", C.c_int * 4), ("offset", C.c_size_t),
+                ("count", C.c_size_t)]
+
+
+class fdg_sched_entry(C.Structure):
+    _fields_ = [("t", C.c_int64), ("k", C.c_int32), ("tau_f", C.c_int64), ("tau_b", C.c_int64),
+                ("ver_f", C.c_int64), ("ver_b", C.c_int64), ("slot_f", C.c_int32), ("slot_b", C.c_int32)]
+
+
+def load_library(path=LIB_PATH):
+    if not os.path.exists(path):
+        raise ImportError("libfdg.so is not built (%s); run `python -m paper_1906_09108_b200.build`" % path)
+    lib = C.CDLL(path)
+    vp, sz, i64 = C.c_void_p, C.c_size_t, C.c_int64
+    P = C.POINTER
+    sig = {
+        "fdg_workspace_bytes": [P(fdg_arch), P(fdg_config), P(sz)],
+        "fdg_create": [P(fdg_arch), P(fdg_config), vp, sz, P(vp), P(vp)],
+        "fdg_destroy": [vp],
+        "fdg_param_count": [vp, C.c_int, P(sz)],
+        "fdg_param_layout": [vp, C.c_int, P(fdg_param_entry), sz, P(sz)],
+        "fdg_set_params": [vp, C.c_int, vp, sz],
+        "fdg_set_momentum": [vp, C.c_int, vp, sz],
+        "fdg_get_params": [vp, C.c_int, vp, sz],
+        "fdg_get_grads": [vp, C.c_int, vp, sz],
+        "fdg_get_momentum": [vp, C.c_int, vp, sz],
+        "fdg_set_lr": [vp, C.c_float],
+        "fdg_step": [vp, vp, vp, vp, vp],
+        "fdg_sync": [vp, vp],
+        "fdg_get_module_output": [vp, C.c_int, vp, sz, P(i64)],
+        "fdg_get_input_grad": [vp, C.c_int, vp, sz, P(i64)],
+        "fdg_boundary_elems": [vp, C.c_int, P(sz), P(sz)],
+        "fdg_get_schedule_log": [vp, P(fdg_sched_entry), sz, P(sz)],
+        "fdg_launch_count": [vp, P(C.c_uint64)],
+    }
+    for name, args in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = C.c_int
+    lib.fdg_status_string.argtypes = [C.c_int]
+    lib.fdg_status_string.restype = C.c_char_p
+    lib.fdg_last_error.argtypes = [vp]
+    lib.fdg_last_error.restype = C.c_char_p
+    return lib
+
+
+class FDGError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__("%s: %s" % (STATUS_NAMES.get(status, status), message))
+        self.status = status
+
+
+def make_arch(family="resnet6n2", n_per_stage=1, widths=(16, 32, 64), stem_width=16, in_h=32, in_w=32, in_c=3,
+              num_classes=10, batch=128, bn_eps=1e-5):
+    fam = {"resnet6n2": FDG_RESNET_6N2, "wrn": FDG_WRN}[family]
+    return fdg_arch(fam, n_per_stage, (C.c_int * 3)(*widths), stem_width, in_h, in_w, in_c, num_classes, batch,
+                    bn_eps)
+
+
+class FDG:
+    """Owner of one fdg_ctx and of the torch tensor that backs its workspace.  Each
+    method is one C-ABI call (plus host<->device staging of its arguments)."""
+
+    def __init__(self, arch, K=2, split_after_block=(1,), beta=1.0, lr=0.1, momentum=0.9, weight_decay=5e-4,
+                 order=FDG_BACKWARD_FIRST, weight_reading=FDG_STASHED, precision=FDG_FP32_CUDACORE, serial=False,
+                 device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.lib = load_library()
+        self.arch = arch
+        self.K = K
+        self._splits = (C.c_int * max(len(split_after_block), 1))(*split_after_block)
+        self.cfg = fdg_config(K, C.cast(self._splits, C.POINTER(C.c_int)), beta, lr, momentum, weight_decay, order,
+                              weight_reading, precision, int(serial))
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        n = C.c_size_t()
+        self._check(self.lib.fdg_workspace_bytes(C.byref(self.arch), C.byref(self.cfg), C.byref(n)), None)
+        self.workspace_bytes = n.value
+        self.workspace = torch.empty(n.value + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        ctx = C.c_void_p()
+        self._check(self.lib.fdg_create(C.byref(self.arch), C.byref(self.cfg), base, n.value, None, C.byref(ctx)), None)
+        self.ctx = ctx
+
+    def _check(self, status, ctx):
+        if status != FDG_OK:
+            msg = self.lib.fdg_last_error(ctx).decode() if ctx else self.lib.fdg_status_string(status).decode()
+            raise FDGError(status, msg)
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            self.lib.fdg_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- parameters -----------------------------------------------------------
+    def param_count(self, k):
+        n = C.c_size_t()
+        self._check(self.lib.fdg_param_count(self.ctx, k, C.byref(n)), self.ctx)
+        return n.value
+
+    def param_layout(self, k):
+        """[(name, kind, shape)] in flat order, the same table the oracle builds."""
+        n = C.c_size_t()
+        self._check(self.lib.fdg_param_layout(self.ctx, k, None, 0, C.byref(n)), self.ctx)
+        arr = (fdg_param_entry * n.value)()
+        self._check(self.lib.fdg_param_layout(self.ctx, k, arr, n.value, C.byref(n)), self.ctx)
+        out = []
+        for e in arr:
+            kind = PARAM_KINDS[e.kind]
+            dims = tuple(e.dims)
+            shape = dims if kind == "conv" else (dims[:2] if kind == "fc_w" else dims[:1])
+            unit = "stem" if e.unit == 0 else ("head" if e.unit < 0 else "block%d" % e.unit)
+            out.append(("%s@%d" % (unit, e.offset), kind, shape))
+        return out
+
+    def _host_vec(self, fn, k):
+        out = np.empty(self.param_count(k), dtype=np.float32)
+        self._check(fn(self.ctx, k, out.ctypes.data, out.size), self.ctx)
+        return out
+
+    def set_params(self, k, flat):
+        flat = np.ascontiguousarray(flat, dtype=np.float32)
+        self._check(self.lib.fdg_set_params(self.ctx, k, flat.ctypes.data, flat.size), self.ctx)
+
+    def set_momentum(self, k, flat):
+        flat = np.ascontiguousarray(flat, dtype=np.float32)
+        self._check(self.lib.fdg_set_momentum(self.ctx, k, flat.ctypes.data, flat.size), self.ctx)
+
+    def get_params(self, k):
+        return self._host_vec(self.lib.fdg_get_params, k)
+
+    def get_grads(self, k):
+        return self._host_vec(self.lib.fdg_get_grads, k)
+
+    def get_momentum(self, k):
+        return self._host_vec(self.lib.fdg_get_momentum, k)
+
+    def set_lr(self, lr):
+        self._check(self.lib.fdg_set_lr(self.ctx, lr), self.ctx)
+
+    # ---- stepping -------------------------------------------------------------
+    def step(self, images_dev, labels_dev, loss_dev=None, stream=None):
+        """images_dev: float32 CUDA tensor [B,H,W,C]; labels_dev: int32 CUDA tensor [B]."""
+        st = self.torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self._check(self.lib.fdg_step(self.ctx, st, images_dev.data_ptr(), labels_dev.data_ptr(),
+                                      loss_dev.data_ptr() if loss_dev is not None else None), self.ctx)
+
+    def sync(self, stream=None):
+        st = self.torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self._check(self.lib.fdg_sync(self.ctx, st), self.ctx)
+
+    # ---- inspection -----------------------------------------------------------
+    def boundary_elems(self, k):
+        a, b = C.c_size_t(), C.c_size_t()
+        self._check(self.lib.fdg_boundary_elems(self.ctx, k, C.byref(a), C.byref(b)), self.ctx)
+        return a.value, b.value
+
+    def module_output(self, k):
+        n = self.boundary_elems(k)[0]
+        out = np.empty(n, dtype=np.float32)
+        b = C.c_int64()
+        self._check(self.lib.fdg_get_module_output(self.ctx, k, out.ctypes.data, n, C.byref(b)), self.ctx)
+        return b.value, out
+
+    def input_grad(self, k):
+        n = self.boundary_elems(k)[1]
+        out = np.empty(n, dtype=np.float32)
+        b = C.c_int64()
+        self._check(self.lib.fdg_get_input_grad(self.ctx, k, out.ctypes.data, n, C.byref(b)), self.ctx)
+        return b.value, out
+
+    def schedule_log(self):
+        n = C.c_size_t()
+        self._check(self.lib.fdg_get_schedule_log(self.ctx, None, 0, C.byref(n)), self.ctx)
+        arr = (fdg_sched_entry * max(n.value, 1))()
+        self._check(self.lib.fdg_get_schedule_log(self.ctx, arr, n.value, C.byref(n)), self.ctx)
+        return [dict(t=e.t, k=e.k, tau_f=e.tau_f, tau_b=e.tau_b, ver_f=e.ver_f, ver_b=e.ver_b, slot_f=e.slot_f,
+                     slot_b=e.slot_b) for e in arr[:n.value]]
+
+    def launch_count(self):
+        n = C.c_uint64()
+        self._check(self.lib.fdg_launch_count(self.ctx, C.byref(n)), self.ctx)
+        return n.value

@@ -1,0 +1,277 @@
+// Convolution forward, data gradient and weight gradient on the CUDA cores, fp32
+// accumulation: the exact-arithmetic mode of the library and the fallback for
+// shapes the tensor-core kernels do not take (3-channel stem, strided and 1x1
+// convolutions, channel counts that are not multiples of 16).
+//
+// All three are one tiled GEMM  C[m][n] = sum_k A(m,k) * B(k,n)  whose operands are
+// gathered on the fly (implicit GEMM, nothing is materialised):
+//   FPROP  m = output pixel (n,p,q)  n = c_out        k = (r,s,c_in)
+//          A = x[n, p*st+r-pad, q*st+s-pad, c_in]     B = w[c_out][r][s][c_in]
+//   DGRAD  m = input pixel (n,h,w)   n = c_in         k = (r,s,c_out)
+//          A = dy[n, (h+pad-r)/st, (w+pad-s)/st, c_out] where divisible and in range
+//          B = w[c_out][r][s][c_in]
+//   FPROP and DGRAD may add a residual tensor (optionally gated by [mask > 0]) to C.
+//   WGRAD  m = (r,s,c_in)            n = c_out        k = output pixel, split over gridDim.z
+//          A = x[n, p*st+r-pad, q*st+s-pad, c_in]     B = dy[pixel][c_out]
+//          C -> partial[z][c_out][r][s][c_in], summed over z in a fixed order afterwards
+#pragma once
+#include <type_traits>
+
+#include "elementwise.cuh"
+
+namespace fdg {
+
+struct ConvGeom {
+  int N, H, W, Ci;      // input  tensor [N][H][W][Ci]
+  int P, Q, Co;         // output tensor [N][P][Q][Co]
+  int R, S, stride, pad;
+};
+
+enum { CONV_FPROP = 0, CONV_DGRAD = 1, CONV_WGRAD = 2 };
+constexpr int kSimtBK = 16;
+constexpr int kSimtThreads = 256;
+
+template <typename T, int MODE, int BM, int BN, int TM, int TN>
+__global__ void __launch_bounds__(kSimtThreads)
+conv_simt_kernel(ConvGeom g, const T* __restrict__ act,      // FPROP/WGRAD: x ; DGRAD: dy
+                 const T* __restrict__ wgt,                  // FPROP/DGRAD: w ; WGRAD: dy
+                 T* __restrict__ out,                        // FPROP: y ; DGRAD: dx ; WGRAD: unused
+                 float* __restrict__ wpartial,               // WGRAD: [gridDim.z][Co*R*S*Ci]
+                 const T* __restrict__ res,                  // FPROP/DGRAD: optional addend, same shape as the output
+                 const T* __restrict__ res_mask,             // optional: the addend counts only where mask > 0
+                 int k_chunk) {                              // WGRAD: pixels per z-slice (multiple of BK)
+  static_assert((BM / TM) * (BN / TN) == kSimtThreads, "tile/thread mismatch");
+  constexpr int BK = kSimtBK;
+  __shared__ float As[BK][BM + 1];
+  __shared__ float Bs[BK][BN + 1];
+
+  const int tid = threadIdx.x;
+  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+  int Mdim, Ndim, Kdim;
+  if (MODE == CONV_FPROP) { Mdim = g.N * g.P * g.Q; Ndim = g.Co; Kdim = g.R * g.S * g.Ci; }
+  else if (MODE == CONV_DGRAD) { Mdim = g.N * g.H * g.W; Ndim = g.Ci; Kdim = g.R * g.S * g.Co; }
+  else { Mdim = g.R * g.S * g.Ci; Ndim = g.Co; Kdim = g.N * g.P * g.Q; }
+  int kbeg = 0, kend = Kdim;
+  if (MODE == CONV_WGRAD) { kbeg = blockIdx.z * k_chunk; kend = min(kbeg + k_chunk, Kdim); }
+
+  const int tx = tid % (BN / TN), ty = tid / (BN / TN);
+  float acc[TM][TN];
+#pragma unroll
+  for (int i = 0; i < TM; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+
+  // ---- loader geometry -------------------------------------------------------
+  // FPROP/DGRAD: A is contiguous along k -> thread owns column kk = tid%BK and rows tid/BK + j*16.
+  // WGRAD:       A is contiguous along m -> thread owns row   mm = tid%BM and columns tid/BM + j*(256/BM).
+  constexpr int A_PER = BM * BK / kSimtThreads;
+  constexpr int B_PER = (BN * BK + kSimtThreads - 1) / kSimtThreads;
+  int a_n[A_PER], a_h[A_PER], a_w[A_PER];       // decoded pixel of each owned row (FPROP/DGRAD)
+  if (MODE != CONV_WGRAD) {
+#pragma unroll
+    for (int j = 0; j < A_PER; ++j) {
+      int m = m0 + tid / BK + j * (kSimtThreads / BK);
+      if (m < Mdim) {
+        int hw = (MODE == CONV_FPROP) ? g.P * g.Q : g.H * g.W;
+        int wd = (MODE == CONV_FPROP) ? g.Q : g.W;
+        int n = m / hw, rem = m - n * hw;
+        a_n[j] = n; a_h[j] = rem / wd; a_w[j] = rem - a_h[j] * wd;
+      } else {
+        a_n[j] = -1; a_h[j] = 0; a_w[j] = 0;
+      }
+    }
+  }
+  int wm_r = 0, wm_s = 0, wm_c = 0;             // decoded (r,s,ci) of the owned row (WGRAD)
+  bool wm_ok = false;
+  if (MODE == CONV_WGRAD) {
+    int m = m0 + tid % BM;
+    wm_ok = m < Mdim;
+    if (wm_ok) { wm_r = m / (g.S * g.Ci); int rem = m - wm_r * g.S * g.Ci; wm_s = rem / g.Ci; wm_c = rem - wm_s * g.Ci; }
+  }
+
+  for (int k0 = kbeg; k0 < kend; k0 += BK) {
+    // ---- A tile ---------------------------------------------------------------
+    if (MODE == CONV_FPROP) {
+      const int kk = tid % BK, k = k0 + kk;
+      int r = 0, s = 0, c = 0;
+      const bool kok = k < kend;
+      if (kok) { r = k / (g.S * g.Ci); int rem = k - r * g.S * g.Ci; s = rem / g.Ci; c = rem - s * g.Ci; }
+#pragma unroll
+      for (int j = 0; j < A_PER; ++j) {
+        float v = 0.f;
+        if (kok && a_n[j] >= 0) {
+          int h = a_h[j] * g.stride + r - g.pad, w = a_w[j] * g.stride + s - g.pad;
+          if (h >= 0 && h < g.H && w >= 0 && w < g.W)
+            v = to_f(act[(((size_t)a_n[j] * g.H + h) * g.W + w) * g.Ci + c]);
+        }
+        As[kk][tid / BK + j * (kSimtThreads / BK)] = v;
+      }
+    } else if (MODE == CONV_DGRAD) {
+      const int kk = tid % BK, k = k0 + kk;
+      int r = 0, s = 0, c = 0;
+      const bool kok = k < kend;
+      if (kok) { r = k / (g.S * g.Co); int rem = k - r * g.S * g.Co; s = rem / g.Co; c = rem - s * g.Co; }
+#pragma unroll
+      for (int j = 0; j < A_PER; ++j) {
+        float v = 0.f;
+        if (kok && a_n[j] >= 0) {
+          int hp = a_h[j] + g.pad - r, wq = a_w[j] + g.pad - s;
+          if (hp >= 0 && wq >= 0 && hp % g.stride == 0 && wq % g.stride == 0) {
+            int p = hp / g.stride, q = wq / g.stride;
+            if (p < g.P && q < g.Q) v = to_f(act[(((size_t)a_n[j] * g.P + p) * g.Q + q) * g.Co + c]);
+          }
+        }
+        As[kk][tid / BK + j * (kSimtThreads / BK)] = v;
+      }
+    } else {
+      const int mm = tid % BM;
+#pragma unroll
+      for (int j = 0; j < A_PER; ++j) {
+        const int kk = tid / BM + j * (kSimtThreads / BM);
+        const int k = k0 + kk;
+        float v = 0.f;
+        if (wm_ok && k < kend) {
+          int n = k / (g.P * g.Q), rem = k - n * g.P * g.Q;
+          int p = rem / g.Q, q = rem - p * g.Q;
+          int h = p * g.stride + wm_r - g.pad, w = q * g.stride + wm_s - g.pad;
+          if (h >= 0 && h < g.H && w >= 0 && w < g.W) v = to_f(act[(((size_t)n * g.H + h) * g.W + w) * g.Ci + wm_c]);
+        }
+        As[kk][mm] = v;
+      }
+    }
+    // ---- B tile ---------------------------------------------------------------
+#pragma unroll
+    for (int j = 0; j < B_PER; ++j) {
+      const int e = tid + j * kSimtThreads;
+      if (e < BN * BK) {
+        float v = 0.f;
+        if (MODE == CONV_FPROP) {
+          const int kk = e % BK, nn = e / BK;
+          const int k = k0 + kk, n = n0 + nn;
+          if (k < kend && n < Ndim) v = to_f(wgt[(size_t)n * Kdim + k]);
+          Bs[kk][nn] = v;
+        } else if (MODE == CONV_DGRAD) {
+          const int nn = e % BN, kk = e / BN;
+          const int k = k0 + kk, n = n0 + nn;
+          if (k < kend && n < Ndim) {
+            int r = k / (g.S * g.Co), rem = k - r * g.S * g.Co;
+            int s = rem / g.Co, co = rem - s * g.Co;
+            v = to_f(wgt[(((size_t)co * g.R + r) * g.S + s) * g.Ci + n]);
+          }
+          Bs[kk][nn] = v;
+        } else {
+          const int nn = e % BN, kk = e / BN;
+          const int k = k0 + kk, n = n0 + nn;
+          if (k < kend && n < Ndim) v = to_f(wgt[(size_t)k * g.Co + n]);
+          Bs[kk][nn] = v;
+        }
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a[TM], b[TN];
+#pragma unroll
+      for (int i = 0; i < TM; ++i) a[i] = As[kk][ty * TM + i];
+#pragma unroll
+      for (int j = 0; j < TN; ++j) b[j] = Bs[kk][tx * TN + j];
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+
+  // ---- epilogue ---------------------------------------------------------------
+#pragma unroll
+  for (int i = 0; i < TM; ++i) {
+    const int m = m0 + ty * TM + i;
+    if (m >= Mdim) continue;
+#pragma unroll
+    for (int j = 0; j < TN; ++j) {
+      const int n = n0 + tx * TN + j;
+      if (n >= Ndim) continue;
+      if (MODE == CONV_WGRAD) {
+        wpartial[(size_t)blockIdx.z * Mdim * Ndim + (size_t)n * Mdim + m] = acc[i][j];
+      } else {
+        const size_t idx = (size_t)m * Ndim + n;
+        float v = acc[i][j];
+        if (res) {
+          float r = to_f(res[idx]);
+          if (res_mask && !(to_f(res_mask[idx]) > 0.f)) r = 0.f;
+          v += r;
+        }
+        out[idx] = from_f<T>(v);
+      }
+    }
+  }
+}
+
+// grad[i] = sum_z partial[z][i], z ascending.
+__global__ void wgrad_reduce_kernel(const float* __restrict__ partial, float* __restrict__ grad, size_t n, int splits) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    float a = 0.f;
+    for (int z = 0; z < splits; ++z) a += partial[(size_t)z * n + i];
+    grad[i] = a;
+  }
+}
+
+// Number of pixel slices the weight-gradient GEMM is split into, and the slice length.
+inline void wgrad_split(const ConvGeom& g, int bm, int bn, int* splits, int* k_chunk) {
+  const long M = (long)g.R * g.S * g.Ci, N = g.Co, K = (long)g.N * g.P * g.Q;
+  long tiles = ((M + bm - 1) / bm) * ((N + bn - 1) / bn);
+  long want = (2 * 148 + tiles - 1) / tiles;
+  long maxs = (K + 4 * kSimtBK - 1) / (4 * kSimtBK);
+  long s = want < 1 ? 1 : (want > maxs ? maxs : want);
+  long chunk = (K + s - 1) / s;
+  chunk = (chunk + kSimtBK - 1) / kSimtBK * kSimtBK;
+  *splits = (int)((K + chunk - 1) / chunk);
+  *k_chunk = (int)chunk;
+}
+
+// Tile choice by GEMM-N (c_out for FPROP/WGRAD, c_in for DGRAD).
+template <typename T, int MODE>
+inline cudaError_t launch_conv_simt(cudaStream_t st, const ConvGeom& g, const T* act, const T* wgt, T* out,
+                                    float* wpartial, float* wgrad_out, const T* res, const T* res_mask,
+                                    uint64_t* launches) {
+  long Mdim, Ndim;
+  if (MODE == CONV_FPROP) { Mdim = (long)g.N * g.P * g.Q; Ndim = g.Co; }
+  else if (MODE == CONV_DGRAD) { Mdim = (long)g.N * g.H * g.W; Ndim = g.Ci; }
+  else { Mdim = (long)g.R * g.S * g.Ci; Ndim = g.Co; }
+  int splits = 1, k_chunk = 0;
+  auto go = [&](auto bm_c, auto bn_c, auto tm_c, auto tn_c) {
+    constexpr int BM = decltype(bm_c)::value, BN = decltype(bn_c)::value;
+    constexpr int TM = decltype(tm_c)::value, TN = decltype(tn_c)::value;
+    if (MODE == CONV_WGRAD) wgrad_split(g, BM, BN, &splits, &k_chunk);
+    dim3 grid((unsigned)((Mdim + BM - 1) / BM), (unsigned)((Ndim + BN - 1) / BN), (unsigned)splits);
+    float* part = (MODE == CONV_WGRAD && splits == 1) ? wgrad_out : wpartial;
+    conv_simt_kernel<T, MODE, BM, BN, TM, TN><<<grid, kSimtThreads, 0, st>>>(g, act, wgt, out, part, res, res_mask, k_chunk);
+  };
+  using std::integral_constant;
+  if (Ndim <= 16) go(integral_constant<int, 128>{}, integral_constant<int, 16>{}, integral_constant<int, 4>{}, integral_constant<int, 2>{});
+  else if (Ndim <= 32) go(integral_constant<int, 128>{}, integral_constant<int, 32>{}, integral_constant<int, 4>{}, integral_constant<int, 4>{});
+  else go(integral_constant<int, 64>{}, integral_constant<int, 64>{}, integral_constant<int, 4>{}, integral_constant<int, 4>{});
+  ++*launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (MODE == CONV_WGRAD && splits > 1) {
+    ++*launches;
+    size_t n = (size_t)Mdim * Ndim;
+    int blocks = (int)((n + 255) / 256); if (blocks > 1184) blocks = 1184;
+    wgrad_reduce_kernel<<<blocks, 256, 0, st>>>(wpartial, wgrad_out, n, splits);
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+// Upper bound of the fp32 scratch elements a weight-gradient launch may need.
+inline size_t wgrad_scratch_elems(const ConvGeom& g) {
+  long Ndim = g.Co;
+  int bm = Ndim <= 32 ? 128 : 64, bn = Ndim <= 16 ? 16 : (Ndim <= 32 ? 32 : 64);
+  int splits, chunk;
+  wgrad_split(g, bm, bn, &splits, &chunk);
+  return (size_t)splits * g.R * g.S * g.Ci * g.Co;
+}
+
+}  // namespace fdg

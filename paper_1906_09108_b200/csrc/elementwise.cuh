@@ -1,0 +1,447 @@
+// Memory-bound kernels of the FDG module-step: batch-norm statistics / apply /
+// backward, the classifier head, the shrink of the received delayed gradient
+// (Eq. 15), the SGD-momentum update (Eq. 11), image ingest and dtype conversion.
+//
+// All tensors are NHWC, seen here as [rows = N*H*W][C].  T is the storage type
+// (float or __nv_bfloat16); arithmetic, statistics and reductions are fp32 (final
+// combination of per-block partial sums in fp64).  Every reduction has a fixed
+// order, so results do not depend on scheduling.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fdg {
+
+// ---------------------------------------------------------------- helpers ---
+template <typename T> struct Vec;   // 16-byte vector of T
+template <> struct Vec<float> {
+  static constexpr int N = 4;
+  float v[4];
+};
+template <> struct Vec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __nv_bfloat16 v[8];
+};
+
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f(float x);
+template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Loads VEC consecutive elements (VEC == 1 or a full 16-byte vector) as floats.
+template <typename T, int VEC>
+__device__ __forceinline__ void load_vec(const T* __restrict__ p, float (&out)[VEC]) {
+  if constexpr (VEC == 1) {
+    out[0] = to_f(p[0]);
+  } else {
+    static_assert(VEC * sizeof(T) == 16, "vector must be 16 bytes");
+    uint4 raw = *reinterpret_cast<const uint4*>(p);
+    const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) out[i] = to_f(e[i]);
+  }
+}
+template <typename T, int VEC>
+__device__ __forceinline__ void store_vec(T* __restrict__ p, const float (&in)[VEC]) {
+  if constexpr (VEC == 1) {
+    p[0] = from_f<T>(in[0]);
+  } else {
+    uint4 raw;
+    T* e = reinterpret_cast<T*>(&raw);
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) e[i] = from_f<T>(in[i]);
+    *reinterpret_cast<uint4*>(p) = raw;
+  }
+}
+
+constexpr int kRedThreads = 256;      // threads per block of the channel-reduction kernels
+constexpr int kRedMaxBlocks = 592;    // 4 blocks per SM on 148 SMs
+constexpr int kRedMaxSums = 3;
+
+// Per-channel statistics record written by the forward and read by the backward.
+// stats[0..C) = mean, stats[C..2C) = 1/sqrt(var+eps).
+
+// Geometry shared by the channel-reduction kernels: a block owns a contiguous range
+// of rows; thread (r, cv) walks rows r, r+RP, ... of channel vector cv.
+struct RedGeom {
+  int rows, C, cv, rp, blocks, rows_per_block;
+};
+inline RedGeom red_geom(int rows, int C, int vec) {
+  RedGeom g;
+  g.rows = rows; g.C = C; g.cv = C / vec;
+  g.rp = kRedThreads / g.cv; if (g.rp < 1) g.rp = 1;
+  int want = (rows + g.rp * 4 - 1) / (g.rp * 4);           // >= 4 passes per block
+  g.blocks = want < 1 ? 1 : (want > kRedMaxBlocks ? kRedMaxBlocks : want);
+  g.rows_per_block = (rows + g.blocks - 1) / g.blocks;
+  return g;
+}
+
+// Block-level part: NS sums per channel -> partial[block][NS][C]; the last block to
+// finish adds the partials in block order (fp64) and calls `fin(c, sums[NS])`.
+template <int NS, int VEC, typename Acc, typename Fin>
+__device__ __forceinline__ void channel_reduce(const RedGeom g, float* __restrict__ partial,
+                                               unsigned int* __restrict__ counter, Acc acc, Fin fin) {
+  extern __shared__ float red_smem[];                        // [rp][NS][C]
+  __shared__ bool is_last;
+  const int tid = threadIdx.x;
+  const int cvi = tid % g.cv, r = tid / g.cv;
+  const int C = g.C;
+  float sums[NS][VEC];
+#pragma unroll
+  for (int s = 0; s < NS; ++s)
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) sums[s][i] = 0.f;
+  const int row0 = blockIdx.x * g.rows_per_block;
+  const int row1 = min(row0 + g.rows_per_block, g.rows);
+  if (r < g.rp)
+    for (int row = row0 + r; row < row1; row += g.rp) acc(row, cvi * VEC, sums);
+  if (r < g.rp) {
+#pragma unroll
+    for (int s = 0; s < NS; ++s)
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) red_smem[(r * NS + s) * C + cvi * VEC + i] = sums[s][i];
+  }
+  __syncthreads();
+  for (int j = tid; j < NS * C; j += blockDim.x) {
+    float a = 0.f;
+    for (int rr = 0; rr < g.rp; ++rr) a += red_smem[rr * NS * C + j];
+    partial[(size_t)blockIdx.x * NS * C + j] = a;
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = (atomicInc(counter, gridDim.x - 1) == gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (int c = tid; c < C; c += blockDim.x) {
+    double tot[NS];
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+      double a = 0.0;
+      for (unsigned b = 0; b < gridDim.x; ++b) a += (double)__ldcg(&partial[(size_t)b * NS * C + s * C + c]);
+      tot[s] = a;
+    }
+    fin(c, tot);
+  }
+}
+
+// ------------------------------------------------- batch norm, forward ------
+// mean and 1/sqrt(var+eps) of each channel over all rows (biased variance).
+template <typename T, int VEC>
+__global__ void __launch_bounds__(kRedThreads)
+bn_stats_kernel(const T* __restrict__ x, RedGeom g, float eps, float* __restrict__ stats,
+                float* __restrict__ partial, unsigned int* __restrict__ counter) {
+  const int C = g.C;
+  const double inv_m = 1.0 / (double)g.rows;
+  channel_reduce<2, VEC>(
+      g, partial, counter,
+      [&](int row, int c0, float (&s)[2][VEC]) {
+        float v[VEC];
+        load_vec<T, VEC>(x + (size_t)row * C + c0, v);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) { s[0][i] += v[i]; s[1][i] += v[i] * v[i]; }
+      },
+      [&](int c, double (&tot)[2]) {
+        double mean = tot[0] * inv_m;
+        double var = tot[1] * inv_m - mean * mean;
+        if (var < 0.0) var = 0.0;
+        stats[c] = (float)mean;
+        stats[C + c] = (float)(1.0 / sqrt(var + (double)eps));
+      });
+}
+
+// y = [relu]( gamma*(x-mean)*invstd + beta + residual ), residual = none | r | BN_r(r).
+template <typename T, int VEC>
+__global__ void bn_apply_kernel(const T* __restrict__ x, const float* __restrict__ stats,
+                                const float* __restrict__ gamma, const float* __restrict__ beta,
+                                const T* __restrict__ res, const float* __restrict__ res_stats,
+                                const float* __restrict__ res_gamma, const float* __restrict__ res_beta,
+                                int relu, T* __restrict__ y, size_t nvec, int C) {
+  const int cv = C / VEC;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
+    const int c0 = (int)(i % cv) * VEC;
+    float v[VEC], r[VEC], o[VEC];
+    load_vec<T, VEC>(x + i * VEC, v);
+    if (res) load_vec<T, VEC>(res + i * VEC, r);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+      const int c = c0 + j;
+      float t = gamma[c] * ((v[j] - stats[c]) * stats[C + c]) + beta[c];
+      if (res) {
+        float rr = r[j];
+        if (res_stats) rr = res_gamma[c] * ((rr - res_stats[c]) * res_stats[C + c]) + res_beta[c];
+        t += rr;
+      }
+      o[j] = relu ? fmaxf(t, 0.f) : t;
+    }
+    store_vec<T, VEC>(y + i * VEC, o);
+  }
+}
+
+// ------------------------------------------------- batch norm, backward -----
+// dz = dy * [mask > 0];  s0 = sum dz, s1 = sum dz*xhat (xhat from x, stats),
+// s2 = sum dz*xhat2 (second normalised tensor sharing dz: the projection shortcut).
+// The sums are the parameter gradients: dbeta = s0, dgamma = s1 (dgamma2 = s2, dbeta2 = s0).
+template <typename T, int VEC, int NS>
+__global__ void __launch_bounds__(kRedThreads)
+bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ mask, const T* __restrict__ x,
+                     const float* __restrict__ stats, const T* __restrict__ x2, const float* __restrict__ stats2,
+                     RedGeom g, float* __restrict__ sums, float* __restrict__ dgamma, float* __restrict__ dbeta,
+                     float* __restrict__ dgamma2, float* __restrict__ dbeta2, float* __restrict__ partial,
+                     unsigned int* __restrict__ counter) {
+  const int C = g.C;
+  channel_reduce<NS, VEC>(
+      g, partial, counter,
+      [&](int row, int c0, float (&s)[NS][VEC]) {
+        const size_t off = (size_t)row * C + c0;
+        float d[VEC], m[VEC], v[VEC], v2[VEC];
+        load_vec<T, VEC>(dy + off, d);
+        if (mask) load_vec<T, VEC>(mask + off, m);
+        load_vec<T, VEC>(x + off, v);
+        if (NS == 3) load_vec<T, VEC>(x2 + off, v2);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+          const int c = c0 + i;
+          float dz = (mask && !(m[i] > 0.f)) ? 0.f : d[i];
+          s[0][i] += dz;
+          s[1][i] += dz * ((v[i] - stats[c]) * stats[C + c]);
+          if (NS == 3) s[2][i] += dz * ((v2[i] - stats2[c]) * stats2[C + c]);
+        }
+      },
+      [&](int c, double (&tot)[NS]) {
+        sums[c] = (float)tot[0];
+        sums[C + c] = (float)tot[1];
+        dbeta[c] = (float)tot[0];
+        dgamma[c] = (float)tot[1];
+        if (NS == 3) {
+          sums[2 * C + c] = (float)tot[2];
+          dbeta2[c] = (float)tot[0];
+          dgamma2[c] = (float)tot[2];
+        }
+      });
+}
+
+// dx = gamma*invstd*(dz - s0/M - xhat*s1/M) [+ res];  optionally the same for the second
+// normalised tensor (dx2) and/or the masked gradient itself (dz_out).
+template <typename T, int VEC>
+__global__ void bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ mask, const T* __restrict__ x,
+                                    const float* __restrict__ stats, const float* __restrict__ gamma,
+                                    const float* __restrict__ sums, const T* __restrict__ x2,
+                                    const float* __restrict__ stats2, const float* __restrict__ gamma2,
+                                    const T* __restrict__ res, T* __restrict__ dx, T* __restrict__ dx2,
+                                    T* __restrict__ dz_out, size_t nvec, int C, float inv_m) {
+  const int cv = C / VEC;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
+    const int c0 = (int)(i % cv) * VEC;
+    float d[VEC], m[VEC], v[VEC], v2[VEC], r[VEC], o[VEC], o2[VEC], oz[VEC];
+    load_vec<T, VEC>(dy + i * VEC, d);
+    if (mask) load_vec<T, VEC>(mask + i * VEC, m);
+    load_vec<T, VEC>(x + i * VEC, v);
+    if (dx2) load_vec<T, VEC>(x2 + i * VEC, v2);
+    if (res) load_vec<T, VEC>(res + i * VEC, r);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+      const int c = c0 + j;
+      float dz = (mask && !(m[j] > 0.f)) ? 0.f : d[j];
+      oz[j] = dz;
+      float xh = (v[j] - stats[c]) * stats[C + c];
+      float t = gamma[c] * stats[C + c] * (dz - sums[c] * inv_m - xh * (sums[C + c] * inv_m));
+      o[j] = res ? t + r[j] : t;
+      if (dx2) {
+        float xh2 = (v2[j] - stats2[c]) * stats2[C + c];
+        o2[j] = gamma2[c] * stats2[C + c] * (dz - sums[c] * inv_m - xh2 * (sums[2 * C + c] * inv_m));
+      }
+    }
+    store_vec<T, VEC>(dx + i * VEC, o);
+    if (dx2) store_vec<T, VEC>(dx2 + i * VEC, o2);
+    if (dz_out) store_vec<T, VEC>(dz_out + i * VEC, oz);
+  }
+}
+
+// -------------------------------------------------------- small elementwise -
+// out = scale * in  (the gradient-shrinking step, Eq. 15).
+template <typename T, int VEC>
+__global__ void scale_kernel(const T* __restrict__ in, T* __restrict__ out, float scale, size_t nvec) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
+    float v[VEC];
+    load_vec<T, VEC>(in + i * VEC, v);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) v[j] *= scale;
+    store_vec<T, VEC>(out + i * VEC, v);
+  }
+}
+
+// out = a + b
+template <typename T, int VEC>
+__global__ void add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* __restrict__ out, size_t nvec) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
+    float x[VEC], y[VEC];
+    load_vec<T, VEC>(a + i * VEC, x);
+    load_vec<T, VEC>(b + i * VEC, y);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) x[j] += y[j];
+    store_vec<T, VEC>(out + i * VEC, x);
+  }
+}
+
+// fp32 [rows][c_in] -> T [rows][c_out], channels c_in..c_out-1 zero (image ingest); labels copied alongside.
+template <typename T>
+__global__ void ingest_kernel(const float* __restrict__ img, T* __restrict__ out, size_t rows, int c_in, int c_out,
+                              const int32_t* __restrict__ labels_in, int32_t* __restrict__ labels_out, int batch) {
+  const size_t n = rows * (size_t)c_out;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t row = i / c_out;
+    const int c = (int)(i % c_out);
+    out[i] = from_f<T>(c < c_in ? img[row * c_in + c] : 0.f);
+  }
+  if (blockIdx.x == 0)
+    for (int i = threadIdx.x; i < batch; i += blockDim.x) labels_out[i] = labels_in[i];
+}
+
+// T [rows][c_src] -> fp32 [rows][c_dst] keeping the first c_dst channels (getters).
+template <typename T>
+__global__ void export_kernel(const T* __restrict__ in, float* __restrict__ out, size_t rows, int c_src, int c_dst) {
+  const size_t n = rows * (size_t)c_dst;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t row = i / c_dst;
+    out[i] = to_f(in[row * c_src + (i % c_dst)]);
+  }
+}
+
+// ------------------------------------------------------------------ head ----
+// One block per sample: global average pool -> FC -> softmax cross-entropy, and the
+// backward of all three down to the gradient of the pooled tensor's source.
+//   x [B][HW][F] (T)   w [classes][F], b [classes] (fp32)
+//   pooled [B][F], dlogits [B][classes], loss_n [B] (fp32 scratch for head_param_grad)
+//   dx [B][HW][F] (T) = dpooled[f] / HW
+// A label outside [0, classes) sets *bad_label and is treated as class 0.
+template <typename T>
+__global__ void head_fwd_bwd_kernel(const T* __restrict__ x, const float* __restrict__ w, const float* __restrict__ b,
+                                    const int32_t* __restrict__ labels, int HW, int F, int classes, int batch,
+                                    float* __restrict__ pooled, float* __restrict__ dlogits,
+                                    float* __restrict__ loss_n, T* __restrict__ dx, int* __restrict__ bad_label) {
+  extern __shared__ float hs[];            // pooled[F] | logits[classes] | dpooled[F]
+  float* s_pool = hs;
+  float* s_logit = hs + F;
+  float* s_dpool = s_logit + classes;
+  const int n = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+  const T* xn = x + (size_t)n * HW * F;
+  for (int f = tid; f < F; f += nt) {
+    float a = 0.f;
+    for (int p = 0; p < HW; ++p) a += to_f(xn[(size_t)p * F + f]);
+    a /= (float)HW;
+    s_pool[f] = a;
+    pooled[(size_t)n * F + f] = a;
+  }
+  __syncthreads();
+  const int warp = tid >> 5, lane = tid & 31, nwarps = nt >> 5;
+  for (int c = warp; c < classes; c += nwarps) {
+    float a = 0.f;
+    for (int f = lane; f < F; f += 32) a += w[(size_t)c * F + f] * s_pool[f];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) s_logit[c] = a + b[c];
+  }
+  __syncthreads();
+  __shared__ float s_max, s_sum;
+  int label = labels[n];
+  if (label < 0 || label >= classes) { if (tid == 0) atomicExch(bad_label, 1); label = 0; }
+  if (tid == 0) {
+    float m = s_logit[0];
+    for (int c = 1; c < classes; ++c) m = fmaxf(m, s_logit[c]);
+    float s = 0.f;
+    for (int c = 0; c < classes; ++c) s += expf(s_logit[c] - m);
+    s_max = m; s_sum = s;
+    loss_n[n] = -(s_logit[label] - m - logf(s));
+  }
+  __syncthreads();
+  for (int c = tid; c < classes; c += nt) {
+    float p = expf(s_logit[c] - s_max) / s_sum;
+    float d = (p - (c == label ? 1.f : 0.f)) / (float)batch;
+    s_logit[c] = d;
+    dlogits[(size_t)n * classes + c] = d;
+  }
+  __syncthreads();
+  for (int f = tid; f < F; f += nt) {
+    float a = 0.f;
+    for (int c = 0; c < classes; ++c) a += w[(size_t)c * F + f] * s_logit[c];
+    s_dpool[f] = a / (float)HW;
+  }
+  __syncthreads();
+  T* dxn = dx + (size_t)n * HW * F;
+  for (int i = tid; i < HW * F; i += nt) dxn[i] = from_f<T>(s_dpool[i % F]);
+}
+
+// One block per class: dW[c][f] = sum_n dlogits[n][c]*pooled[n][f], db[c] = sum_n dlogits[n][c];
+// block 0 also reduces the loss (mean over the batch) and raises *nonfinite if it is NaN/Inf.
+__global__ void head_param_grad_kernel(const float* __restrict__ pooled, const float* __restrict__ dlogits,
+                                       const float* __restrict__ loss_n, int F, int classes, int batch,
+                                       float* __restrict__ dW, float* __restrict__ db, float* __restrict__ loss,
+                                       int* __restrict__ nonfinite) {
+  const int c = blockIdx.x;
+  for (int f = threadIdx.x; f < F; f += blockDim.x) {
+    float a = 0.f;
+    for (int n = 0; n < batch; ++n) a += dlogits[(size_t)n * classes + c] * pooled[(size_t)n * F + f];
+    dW[(size_t)c * F + f] = a;
+  }
+  if (threadIdx.x == 0) {
+    float a = 0.f;
+    for (int n = 0; n < batch; ++n) a += dlogits[(size_t)n * classes + c];
+    db[c] = a;
+    if (c == 0) {
+      double l = 0.0;
+      for (int n = 0; n < batch; ++n) l += (double)loss_n[n];
+      float lf = (float)(l / (double)batch);
+      *loss = lf;
+      if (!isfinite(lf)) atomicExch(nonfinite, 1);
+    }
+  }
+}
+
+// ------------------------------------------------------------------- SGD ----
+// g' = g + wd*theta ; v = mu*v + g' ; theta -= lr*v   (v starts at 0, so the first
+// update gives v = g').  Also writes the copies of theta the kernels compute with into
+// the next weight-version slot: fp32 always, bf16 when next16 is given.  g is left untouched.
+__global__ void sgd_kernel(float* __restrict__ theta, float* __restrict__ v, const float* __restrict__ g,
+                           float* __restrict__ next32, __nv_bfloat16* __restrict__ next16, size_t n, float lr,
+                           float mu, float wd) {
+  const size_t n4 = n / 4;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    float4 th = reinterpret_cast<float4*>(theta)[i];
+    float4 vv = reinterpret_cast<float4*>(v)[i];
+    const float4 gg = reinterpret_cast<const float4*>(g)[i];
+    vv.x = mu * vv.x + (gg.x + wd * th.x); th.x -= lr * vv.x;
+    vv.y = mu * vv.y + (gg.y + wd * th.y); th.y -= lr * vv.y;
+    vv.z = mu * vv.z + (gg.z + wd * th.z); th.z -= lr * vv.z;
+    vv.w = mu * vv.w + (gg.w + wd * th.w); th.w -= lr * vv.w;
+    reinterpret_cast<float4*>(theta)[i] = th;
+    reinterpret_cast<float4*>(v)[i] = vv;
+    reinterpret_cast<float4*>(next32)[i] = th;
+    if (next16) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(th.x, th.y), hi = __floats2bfloat162_rn(th.z, th.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<unsigned int*>(&lo);
+      pk.y = *reinterpret_cast<unsigned int*>(&hi);
+      reinterpret_cast<uint2*>(next16)[i] = pk;
+    }
+  }
+  if (blockIdx.x == 0)
+    for (size_t i = n4 * 4 + threadIdx.x; i < n; i += blockDim.x) {
+      float vv = mu * v[i] + (g[i] + wd * theta[i]);
+      float th = theta[i] - lr * vv;
+      v[i] = vv; theta[i] = th;
+      next32[i] = th;
+      if (next16) next16[i] = __float2bfloat16_rn(th);
+    }
+}
+
+// fp32 -> T copy (refreshing the compute copies after fdg_set_params).
+template <typename T>
+__global__ void cast_kernel(const float* __restrict__ in, T* __restrict__ out, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    out[i] = from_f<T>(in[i]);
+}
+
+}  // namespace fdg

@@ -1,0 +1,1013 @@
+// libfdg: the module runtime and the C ABI (see include/fdg.h for the contract).
+//
+// One context holds K modules.  Each module owns, inside the caller's workspace:
+//   * fp32 master parameters, momentum and the last gradient (flat vectors);
+//   * a ring of weight versions: the copy of the parameters the kernels compute with,
+//     written by the update kernel, so that the delayed backward of a batch can read
+//     the weights its forward used (superscripts of Eq. 10);
+//   * an activation FIFO: one slot per batch in flight holding everything the backward
+//     of that batch needs (Fig. 1(b): "the previously saved computation graph");
+//   * a gradient mailbox (ring of 3) that receives the gradient of the module input
+//     and is read by the upstream module in the next iteration (Section 3.1,
+//     "communication");
+//   * private temporaries.
+// A module reads its input straight from the upstream module's FIFO slot, so the
+// "send" of an activation is the producer's own store and the "receive" is a stream
+// event.  Nothing is copied between modules.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/fdg.h"
+#include "conv_simt.cuh"
+#include "elementwise.cuh"
+
+namespace fdg {
+
+typedef __nv_bfloat16 bf16;
+constexpr int kEventRing = 4;
+constexpr int kMailRing = 3;
+constexpr size_t kLogIterations = 4096;
+
+enum UnitType { U_STEM, U_BASIC, U_PREACT, U_HEAD };
+
+struct Unit {
+  UnitType type;
+  int index;                 // 0 stem, b block, -1 head
+  int ci, co, stride;
+  bool proj;
+  bool bn;                   // stem: has BN+ReLU (6n+2); head: has BN+ReLU (WRN)
+  int H, W, P, Q;            // input / output spatial size
+  // offsets into the module's flat parameter vector
+  size_t w1, g1, b1, w2, g2, b2, ws, gs, bs;
+  // offsets (elements of T) of saved tensors inside an activation-FIFO slot; y is the unit output
+  size_t t_a, t_b, t_c, t_y, t_s;
+  // offsets (floats) of saved statistics inside the slot's fp32 region
+  size_t st1, st2, sts;
+};
+
+struct Module {
+  int k;                                   // 1-based
+  std::vector<Unit> units;
+  std::vector<fdg_param_entry> layout;
+  size_t n_params = 0;
+  int D = 1;                               // activation-FIFO depth
+  int Dw = 1;                              // weight versions kept
+  int Din = 0;                             // image ring depth (module 1 only)
+  size_t slot_elems = 0, slot_floats = 0;  // per FIFO slot
+  size_t in_elems = 0, out_elems = 0;      // module input / output tensor sizes (stored channels)
+  int in_h = 0, in_w = 0, in_c = 0, in_c_logical = 0, out_c = 0;
+  size_t max_act = 0;                      // largest activation tensor (elements)
+  size_t scratch_floats = 0;               // reduction partials / weight-gradient slices
+  // device pointers
+  float *theta = nullptr, *mom = nullptr, *grad = nullptr, *wver = nullptr;
+  bf16* wver16 = nullptr;
+  char* fifo = nullptr;                    // D slots of slot_elems*sizeof(T)
+  float* fifo_f = nullptr;                 // D slots of slot_floats
+  char* in_ring = nullptr;                 // module 1: Din image slots
+  char* mail = nullptr;                    // kMailRing slots of in_elems (k >= 2)
+  char* temps[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  float *scratch = nullptr, *bnsums = nullptr;
+  unsigned int* counter = nullptr;
+  float *pooled = nullptr, *dlogits = nullptr, *loss_n = nullptr, *loss = nullptr;   // head
+  // host state
+  int64_t updates = 0;
+  std::vector<int64_t> slot_version, slot_batch;
+  int64_t last_out_batch = -1, last_grad_batch = -1;
+  int last_out_slot = -1, last_grad_slot = -1;
+  cudaStream_t stream = nullptr;
+  cudaEvent_t ev_act[kEventRing], ev_grad[kEventRing];
+};
+
+}  // namespace fdg
+
+using namespace fdg;
+
+struct fdg_ctx {
+  fdg_arch arch;
+  fdg_config cfg;
+  std::vector<int> splits;
+  int K = 0;
+  bool bf16_mode = false;
+  size_t esize = 4;
+  std::vector<Module> mods;
+  bool own_streams = false;
+  cudaEvent_t ev_in[kEventRing];
+  cudaEvent_t ev_join;
+  int32_t* labels = nullptr;          // ring of label_ring batches
+  int label_ring = 0;
+  int* flags = nullptr;               // [0] non-finite loss, [1] label out of range
+  float* staging = nullptr;           // fp32 staging for getters
+  size_t staging_elems = 0;
+  int64_t t = 0;
+  float lr = 0.f;
+  uint64_t launches = 0;
+  std::vector<fdg_sched_entry> log;
+  mutable std::string err;
+  fdg_status latched = FDG_OK;
+  int device = 0;
+  cudaStream_t last_stream = nullptr;   // stream of the most recent fdg_step
+  bool stepped = false;
+};
+
+namespace fdg {
+
+// ------------------------------------------------------------------ planning --
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+  char* base;
+  size_t off = 0;
+  explicit Carver(char* b) : base(b) {}
+  template <typename P> P* take(size_t bytes) {
+    off = align_up(off, 256);
+    P* p = base ? reinterpret_cast<P*>(base + off) : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+static int conv_out(int n, int r, int stride, int pad) { return (n + 2 * pad - r) / stride + 1; }
+
+static fdg_status validate(const fdg_arch* a, const fdg_config* c, std::string* why) {
+  if (!a || !c) { *why = "null arch or config"; return FDG_ERR_INVALID_ARG; }
+  if (a->family != FDG_RESNET_6N2 && a->family != FDG_WRN) { *why = "unknown family"; return FDG_ERR_INVALID_ARG; }
+  if (a->n_per_stage < 1 || a->stem_width < 1 || a->in_h < 4 || a->in_w < 4 || a->in_c < 1 || a->num_classes < 2 ||
+      a->batch < 1 || !(a->bn_eps > 0.f)) { *why = "bad architecture sizes"; return FDG_ERR_INVALID_ARG; }
+  for (int i = 0; i < 3; ++i) if (a->widths[i] < 1) { *why = "bad stage width"; return FDG_ERR_INVALID_ARG; }
+  if (a->in_h % 4 || a->in_w % 4) { *why = "image size must be a multiple of 4"; return FDG_ERR_INVALID_ARG; }
+  if (c->K < 1 || c->K > 64) { *why = "K out of range"; return FDG_ERR_INVALID_ARG; }
+  if (c->K > 1 && !c->split_after_block) { *why = "split_after_block is null"; return FDG_ERR_INVALID_ARG; }
+  const int nblocks = 3 * a->n_per_stage;
+  int prev = 0;
+  for (int i = 0; i + 1 < c->K; ++i) {
+    int s = c->split_after_block[i];
+    if (s <= prev || s >= nblocks) { *why = "split points must ascend inside [1, 3n-1]"; return FDG_ERR_INVALID_ARG; }
+    prev = s;
+  }
+  if (!(c->beta > 0.f && c->beta <= 1.f)) { *why = "beta must be in (0, 1]"; return FDG_ERR_INVALID_ARG; }
+  if (!(c->lr >= 0.f) || !(c->momentum >= 0.f && c->momentum < 1.f) || !(c->weight_decay >= 0.f)) {
+    *why = "bad optimiser constants"; return FDG_ERR_INVALID_ARG; }
+  if ((c->order != FDG_BACKWARD_FIRST && c->order != FDG_FORWARD_FIRST) ||
+      (c->weight_reading != FDG_STASHED && c->weight_reading != FDG_CURRENT) ||
+      (c->precision != FDG_FP32_CUDACORE && c->precision != FDG_BF16_TC)) { *why = "bad enum value"; return FDG_ERR_INVALID_ARG; }
+  // channel counts the vectorised kernels can address
+  const int vec = c->precision == FDG_BF16_TC ? 8 : 4;
+  int chans[4] = {a->stem_width, a->widths[0], a->widths[1], a->widths[2]};
+  for (int ch : chans) {
+    if ((ch % vec != 0 && ch > kRedThreads) || ch / vec > kRedThreads) { *why = "channel count not addressable by the reduction kernels"; return FDG_ERR_UNSUPPORTED; }
+    if (c->precision == FDG_BF16_TC && ch % 8 != 0) { *why = "bf16 mode needs channel counts that are multiples of 8"; return FDG_ERR_UNSUPPORTED; }
+  }
+  if ((size_t)a->batch * a->in_h * a->in_w * (size_t)std::max({chans[0], chans[1], chans[2], chans[3]}) > (size_t)1 << 31) {
+    *why = "activation tensor exceeds 2^31 elements"; return FDG_ERR_UNSUPPORTED; }
+  return FDG_OK;
+}
+
+static void add_param(Module& m, int kind, int unit, int d0, int d1, int d2, int d3, size_t* off_out) {
+  fdg_param_entry e;
+  e.kind = kind; e.unit = unit; e.dims[0] = d0; e.dims[1] = d1; e.dims[2] = d2; e.dims[3] = d3;
+  e.offset = m.n_params; e.count = (size_t)d0 * d1 * d2 * d3;
+  *off_out = e.offset;
+  m.n_params += e.count;
+  m.layout.push_back(e);
+}
+
+// Builds the unit lists, parameter tables and slot layouts of all modules (no pointers yet).
+static void plan_modules(fdg_ctx* c) {
+  const fdg_arch& a = c->arch;
+  const int K = c->K;
+  const bool wrn = a.family == FDG_WRN;
+  const int nblocks = 3 * a.n_per_stage;
+  c->mods.assign(K, Module());
+  std::vector<int> last_block(K);
+  for (int k = 0; k < K; ++k) last_block[k] = (k + 1 < K) ? c->splits[k] : nblocks;
+
+  int k = 0;
+  int H = a.in_h, W = a.in_w, ci = a.stem_width;
+  const int in_c_store = a.in_c;
+  for (int kk = 0; kk < K; ++kk) c->mods[kk].k = kk + 1;
+  {   // stem
+    Module& m = c->mods[0];
+    Unit u{}; u.type = U_STEM; u.index = 0; u.ci = in_c_store; u.co = a.stem_width; u.stride = 1; u.bn = !wrn;
+    u.H = H; u.W = W; u.P = H; u.Q = W;
+    add_param(m, FDG_PARAM_CONV, 0, u.co, 3, 3, a.in_c, &u.w1);
+    if (u.bn) { add_param(m, FDG_PARAM_BN_GAMMA, 0, u.co, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, 0, u.co, 1, 1, 1, &u.b1); }
+    m.units.push_back(u);
+    m.in_h = H; m.in_w = W; m.in_c = in_c_store; m.in_c_logical = a.in_c;
+  }
+  for (int b = 1; b <= nblocks; ++b) {
+    while (b > last_block[k]) ++k;
+    Module& m = c->mods[k];
+    const int stage = (b - 1) / a.n_per_stage, j = (b - 1) % a.n_per_stage;
+    Unit u{}; u.type = wrn ? U_PREACT : U_BASIC; u.index = b; u.ci = ci; u.co = a.widths[stage];
+    u.stride = (stage > 0 && j == 0) ? 2 : 1;
+    u.proj = (u.ci != u.co) || u.stride != 1;
+    u.H = H; u.W = W; u.P = conv_out(H, 3, u.stride, 1); u.Q = conv_out(W, 3, u.stride, 1);
+    if (m.units.empty()) { m.in_h = H; m.in_w = W; m.in_c = ci; m.in_c_logical = ci; }
+    if (!wrn) {
+      add_param(m, FDG_PARAM_CONV, b, u.co, 3, 3, u.ci, &u.w1);
+      add_param(m, FDG_PARAM_BN_GAMMA, b, u.co, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, b, u.co, 1, 1, 1, &u.b1);
+      add_param(m, FDG_PARAM_CONV, b, u.co, 3, 3, u.co, &u.w2);
+      add_param(m, FDG_PARAM_BN_GAMMA, b, u.co, 1, 1, 1, &u.g2); add_param(m, FDG_PARAM_BN_BETA, b, u.co, 1, 1, 1, &u.b2);
+      if (u.proj) {
+        add_param(m, FDG_PARAM_CONV, b, u.co, 1, 1, u.ci, &u.ws);
+        add_param(m, FDG_PARAM_BN_GAMMA, b, u.co, 1, 1, 1, &u.gs); add_param(m, FDG_PARAM_BN_BETA, b, u.co, 1, 1, 1, &u.bs);
+      }
+    } else {
+      add_param(m, FDG_PARAM_BN_GAMMA, b, u.ci, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, b, u.ci, 1, 1, 1, &u.b1);
+      add_param(m, FDG_PARAM_CONV, b, u.co, 3, 3, u.ci, &u.w1);
+      add_param(m, FDG_PARAM_BN_GAMMA, b, u.co, 1, 1, 1, &u.g2); add_param(m, FDG_PARAM_BN_BETA, b, u.co, 1, 1, 1, &u.b2);
+      add_param(m, FDG_PARAM_CONV, b, u.co, 3, 3, u.co, &u.w2);
+      if (u.proj) add_param(m, FDG_PARAM_CONV, b, u.co, 1, 1, u.ci, &u.ws);
+    }
+    m.units.push_back(u);
+    H = u.P; W = u.Q; ci = u.co;
+  }
+  {   // head
+    Module& m = c->mods[K - 1];
+    Unit u{}; u.type = U_HEAD; u.index = -1; u.ci = ci; u.co = a.num_classes; u.bn = wrn; u.H = H; u.W = W; u.P = 1; u.Q = 1; u.stride = 1;
+    if (u.bn) { add_param(m, FDG_PARAM_BN_GAMMA, -1, ci, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, -1, ci, 1, 1, 1, &u.b1); }
+    add_param(m, FDG_PARAM_FC_W, -1, a.num_classes, ci, 1, 1, &u.w1);
+    add_param(m, FDG_PARAM_FC_B, -1, a.num_classes, 1, 1, 1, &u.w2);
+    m.units.push_back(u);
+  }
+  // per-module slot layouts, depths and scratch sizes
+  const size_t B = a.batch;
+  for (int kk = 0; kk < K; ++kk) {
+    Module& m = c->mods[kk];
+    const int kp = kk + 1;
+    m.D = (kp == K) ? 1 : 2 * (K - kp) + (c->cfg.order == FDG_FORWARD_FIRST ? 1 : 0);
+    m.Dw = (kp == K) ? 1 : 2 * (K - kp) + 1;
+    m.Din = (kp == 1) ? m.D + 2 : 0;
+    m.in_elems = B * m.in_h * m.in_w * m.in_c;
+    size_t te = 0, tf = 0, maxa = m.in_elems, scr = 0;
+    auto tens = [&](size_t e) { size_t o = te; te += align_up(e, 128); maxa = std::max(maxa, e); return o; };
+    auto stat = [&](int ch) { size_t o = tf; tf += align_up((size_t)2 * ch, 64); return o; };
+    auto red_scratch = [&](size_t rows, int ch) { scr = std::max(scr, (size_t)kRedMaxBlocks * kRedMaxSums * ch); (void)rows; };
+    auto wg_scratch = [&](int n, int h, int w, int cin, int p, int q, int cout, int r, int stride, int pad) {
+      ConvGeom g{n, h, w, cin, p, q, cout, r, r, stride, pad};
+      scr = std::max(scr, wgrad_scratch_elems(g));
+    };
+    for (Unit& u : m.units) {
+      const size_t in_e = B * u.H * u.W * u.ci, out_e = B * u.P * u.Q * u.co;
+      maxa = std::max(maxa, std::max(in_e, out_e));
+      switch (u.type) {
+        case U_STEM:
+          if (u.bn) { u.t_a = tens(out_e); u.st1 = stat(u.co); red_scratch(B * u.P * u.Q, u.co); }
+          u.t_y = tens(out_e);
+          wg_scratch(a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
+          break;
+        case U_BASIC:
+          u.t_a = tens(out_e); u.t_b = tens(out_e); u.t_c = tens(out_e); u.t_y = tens(out_e);
+          u.st1 = stat(u.co); u.st2 = stat(u.co);
+          if (u.proj) { u.t_s = tens(out_e); u.sts = stat(u.co); }
+          red_scratch(B * u.P * u.Q, u.co);
+          wg_scratch(a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
+          wg_scratch(a.batch, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
+          if (u.proj) wg_scratch(a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
+          break;
+        case U_PREACT:
+          u.t_a = tens(in_e); u.t_b = tens(out_e); u.t_c = tens(out_e); u.t_y = tens(out_e);
+          u.st1 = stat(u.ci); u.st2 = stat(u.co);
+          red_scratch(B * u.H * u.W, std::max(u.ci, u.co));
+          wg_scratch(a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
+          wg_scratch(a.batch, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
+          if (u.proj) wg_scratch(a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
+          break;
+        case U_HEAD:
+          if (u.bn) { u.t_a = tens(in_e); u.st1 = stat(u.ci); red_scratch(B * u.H * u.W, u.ci); }
+          break;
+      }
+    }
+    m.slot_elems = te; m.slot_floats = tf; m.max_act = maxa; m.scratch_floats = scr;
+    const Unit& last = m.units.back();
+    if (kp < K) { m.out_elems = B * last.P * last.Q * last.co; m.out_c = last.co; }
+    m.slot_version.assign(m.D, -1);
+    m.slot_batch.assign(m.D, -1);
+  }
+}
+
+// Assigns every device pointer; with base == nullptr only measures.
+static size_t carve(fdg_ctx* c, char* base) {
+  Carver cv(base);
+  const size_t es = c->esize;
+  c->flags = cv.take<int>(256);
+  c->label_ring = 2 * c->K + 2;
+  c->labels = cv.take<int32_t>((size_t)c->label_ring * c->arch.batch * sizeof(int32_t));
+  size_t stage = 0;
+  for (Module& m : c->mods) {
+    m.theta = cv.take<float>(m.n_params * 4);
+    m.mom = cv.take<float>(m.n_params * 4);
+    m.grad = cv.take<float>(m.n_params * 4);
+    m.wver = cv.take<float>((size_t)m.Dw * align_up(m.n_params, 64) * 4);
+    m.wver16 = c->bf16_mode ? cv.take<bf16>((size_t)m.Dw * align_up(m.n_params, 64) * 2) : nullptr;
+    m.fifo = cv.take<char>((size_t)m.D * m.slot_elems * es);
+    m.fifo_f = cv.take<float>((size_t)m.D * std::max<size_t>(m.slot_floats, 64) * 4);
+    m.in_ring = m.Din ? cv.take<char>((size_t)m.Din * align_up(m.in_elems, 128) * es) : nullptr;
+    m.mail = m.k >= 2 ? cv.take<char>((size_t)kMailRing * align_up(m.in_elems, 128) * es) : nullptr;
+    for (int i = 0; i < 5; ++i) m.temps[i] = cv.take<char>(align_up(m.max_act, 128) * es);
+    m.scratch = cv.take<float>(std::max<size_t>(m.scratch_floats, 64) * 4);
+    int maxc = 1;
+    for (const Unit& u : m.units) maxc = std::max(maxc, std::max(u.ci, u.co));
+    m.bnsums = cv.take<float>((size_t)kRedMaxSums * maxc * 4);
+    m.counter = cv.take<unsigned int>(256);
+    if (m.k == c->K) {
+      const Unit& h = m.units.back();
+      m.pooled = cv.take<float>((size_t)c->arch.batch * h.ci * 4);
+      m.dlogits = cv.take<float>((size_t)c->arch.batch * h.co * 4);
+      m.loss_n = cv.take<float>((size_t)c->arch.batch * 4);
+      m.loss = cv.take<float>(256);
+    }
+    stage = std::max(stage, std::max(m.in_elems, m.out_elems));
+  }
+  c->staging_elems = stage;
+  c->staging = cv.take<float>(stage * 4);
+  return align_up(cv.off, 256);
+}
+
+// ------------------------------------------------------------------ launching --
+struct Launch {
+  fdg_ctx* c;
+  cudaStream_t st;
+  cudaError_t err = cudaSuccess;
+  void check() { if (err == cudaSuccess) err = cudaGetLastError(); ++c->launches; }
+  void note(cudaError_t e) { if (err == cudaSuccess) err = e; }
+};
+
+static int ew_blocks(size_t nvec) {
+  size_t b = (nvec + 255) / 256;
+  return (int)std::min<size_t>(std::max<size_t>(b, 1), 148 * 8);
+}
+
+template <typename T> constexpr int full_vec() { return 16 / sizeof(T); }
+
+template <typename T>
+static void bn_stats(Launch& L, Module& m, const T* x, size_t rows, int C, float eps, float* stats) {
+  constexpr int V = full_vec<T>();
+  if (C % V == 0) {
+    RedGeom g = red_geom((int)rows, C, V);
+    bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)g.rp * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
+  } else {
+    RedGeom g = red_geom((int)rows, C, 1);
+    bn_stats_kernel<T, 1><<<g.blocks, kRedThreads, (size_t)g.rp * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
+  }
+  L.check();
+}
+
+template <typename T>
+static void bn_apply(Launch& L, const T* x, const float* stats, const float* gamma, const float* beta, const T* res,
+                     const float* res_stats, const float* res_gamma, const float* res_beta, bool relu, T* y,
+                     size_t rows, int C) {
+  constexpr int V = full_vec<T>();
+  const size_t n = rows * C;
+  if (C % V == 0)
+    bn_apply_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C);
+  else
+    bn_apply_kernel<T, 1><<<ew_blocks(n), 256, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C);
+  L.check();
+}
+
+// Backward of y = BN(x) (and optionally y2 = BN2(x2) sharing the same upstream gradient):
+// dz = dy*[mask>0]; parameter gradients into dgamma/dbeta; dx (+res) and dx2.
+template <typename T>
+static void bn_backward(Launch& L, Module& m, const T* dy, const T* mask, const T* x, const float* stats,
+                        const float* gamma, float* dgamma, float* dbeta, const T* x2, const float* stats2,
+                        const float* gamma2, float* dgamma2, float* dbeta2, const T* res, T* dx, T* dx2,
+                        size_t rows, int C) {
+  constexpr int V = full_vec<T>();
+  const bool two = x2 != nullptr;
+  const int ns = two ? 3 : 2;
+  const bool vec = C % V == 0;
+  RedGeom g = red_geom((int)rows, C, vec ? V : 1);
+  const size_t smem = (size_t)g.rp * ns * C * 4;
+#define FDG_RED(VV, NS) bn_bwd_reduce_kernel<T, VV, NS><<<g.blocks, kRedThreads, smem, L.st>>>( \
+      dy, mask, x, stats, x2, stats2, g, m.bnsums, dgamma, dbeta, dgamma2, dbeta2, m.scratch, m.counter)
+  if (vec) { if (two) FDG_RED(V, 3); else FDG_RED(V, 2); }
+  else     { if (two) FDG_RED(1, 3); else FDG_RED(1, 2); }
+#undef FDG_RED
+  L.check();
+  const size_t n = rows * C;
+  const float inv_m = 1.f / (float)rows;
+  if (vec)
+    bn_bwd_apply_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n / V, C, inv_m);
+  else
+    bn_bwd_apply_kernel<T, 1><<<ew_blocks(n), 256, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n, C, inv_m);
+  L.check();
+}
+
+template <typename T>
+static void scale_tensor(Launch& L, const T* in, T* out, float s, size_t n) {
+  constexpr int V = full_vec<T>();
+  if (n % V == 0) scale_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(in, out, s, n / V);
+  else scale_kernel<T, 1><<<ew_blocks(n), 256, 0, L.st>>>(in, out, s, n);
+  L.check();
+}
+
+template <typename T> static const T* weights_of(const Module& m, int vslot);
+template <> const float* weights_of<float>(const Module& m, int vslot) { return m.wver + (size_t)vslot * align_up(m.n_params, 64); }
+template <> const bf16* weights_of<bf16>(const Module& m, int vslot) { return m.wver16 + (size_t)vslot * align_up(m.n_params, 64); }
+
+static ConvGeom geom(int N, int H, int W, int Ci, int P, int Q, int Co, int R, int stride, int pad) {
+  return ConvGeom{N, H, W, Ci, P, Q, Co, R, R, stride, pad};
+}
+
+template <typename T>
+static void conv_fprop(Launch& L, const ConvGeom& g, const T* x, const T* w, T* y, const T* res) {
+  L.note(launch_conv_simt<T, CONV_FPROP>(L.st, g, x, w, y, nullptr, nullptr, res, (const T*)nullptr, &L.c->launches));
+}
+template <typename T>
+static void conv_dgrad(Launch& L, const ConvGeom& g, const T* dy, const T* w, T* dx, const T* res, const T* mask) {
+  L.note(launch_conv_simt<T, CONV_DGRAD>(L.st, g, dy, w, dx, nullptr, nullptr, res, mask, &L.c->launches));
+}
+template <typename T>
+static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* dy, float* dw) {
+  L.note(launch_conv_simt<T, CONV_WGRAD>(L.st, g, x, dy, (T*)nullptr, m.scratch, dw, (const T*)nullptr, (const T*)nullptr, &L.c->launches));
+}
+
+// ------------------------------------------------------------ module passes ---
+template <typename T> static T* slot_T(const Module& m, int slot) { return reinterpret_cast<T*>(m.fifo) + (size_t)slot * m.slot_elems; }
+static float* slot_F(const Module& m, int slot) { return m.fifo_f + (size_t)slot * std::max<size_t>(m.slot_floats, 64); }
+
+// Input tensor of module m for batch tau: the image ring (module 1) or the upstream module's FIFO slot.
+template <typename T>
+static const T* module_input(fdg_ctx* c, const Module& m, int64_t tau) {
+  if (m.k == 1) return reinterpret_cast<const T*>(m.in_ring) + (size_t)(tau % m.Din) * align_up(m.in_elems, 128);
+  const Module& up = c->mods[m.k - 2];
+  return slot_T<T>(up, (int)(tau % up.D)) + up.units.back().t_y;
+}
+
+template <typename T>
+static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int slot, int vslot) {
+  const int B = c->arch.batch;
+  const float eps = c->arch.bn_eps;
+  const T* wt = weights_of<T>(m, vslot);
+  const float* wf = m.wver + (size_t)vslot * align_up(m.n_params, 64);
+  T* S = slot_T<T>(m, slot);
+  float* F = slot_F(m, slot);
+  const T* x = module_input<T>(c, m, tau);
+  T* tmp = reinterpret_cast<T*>(m.temps[2]);
+  for (const Unit& u : m.units) {
+    const size_t rows_in = (size_t)B * u.H * u.W, rows_out = (size_t)B * u.P * u.Q;
+    switch (u.type) {
+      case U_STEM: {
+        ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
+        if (u.bn) {
+          conv_fprop<T>(L, g, x, wt + u.w1, S + u.t_a, nullptr);
+          bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
+          bn_apply<T>(L, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co);
+        } else {
+          conv_fprop<T>(L, g, x, wt + u.w1, S + u.t_y, nullptr);
+        }
+        break;
+      }
+      case U_BASIC: {
+        ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
+        ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
+        conv_fprop<T>(L, g1, x, wt + u.w1, S + u.t_a, nullptr);                                        // c1
+        bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
+        bn_apply<T>(L, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_b, rows_out, u.co);  // a1
+        conv_fprop<T>(L, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr);                                // c2
+        bn_stats<T>(L, m, S + u.t_c, rows_out, u.co, eps, F + u.st2);
+        if (u.proj) {
+          ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
+          conv_fprop<T>(L, gs, x, wt + u.ws, S + u.t_s, nullptr);                                      // cs
+          bn_stats<T>(L, m, S + u.t_s, rows_out, u.co, eps, F + u.sts);
+          bn_apply<T>(L, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, S + u.t_s, F + u.sts, wf + u.gs, wf + u.bs, true, S + u.t_y, rows_out, u.co);
+        } else {
+          bn_apply<T>(L, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, x, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co);
+        }
+        break;
+      }
+      case U_PREACT: {
+        ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
+        ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
+        bn_stats<T>(L, m, x, rows_in, u.ci, eps, F + u.st1);
+        bn_apply<T>(L, x, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows_in, u.ci);   // o
+        conv_fprop<T>(L, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr);                                // c1
+        bn_stats<T>(L, m, S + u.t_b, rows_out, u.co, eps, F + u.st2);
+        bn_apply<T>(L, S + u.t_b, F + u.st2, wf + u.g2, wf + u.b2, nullptr, nullptr, nullptr, nullptr, true, S + u.t_c, rows_out, u.co); // a2
+        if (u.proj) {
+          ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
+          conv_fprop<T>(L, gs, S + u.t_a, wt + u.ws, tmp, nullptr);
+          conv_fprop<T>(L, g2, S + u.t_c, wt + u.w2, S + u.t_y, tmp);
+        } else {
+          conv_fprop<T>(L, g2, S + u.t_c, wt + u.w2, S + u.t_y, x);
+        }
+        break;
+      }
+      case U_HEAD:
+        break;      // handled by head_forward_backward
+    }
+    if (u.type != U_HEAD) x = S + u.t_y;
+  }
+}
+
+// Module K only: classifier, loss and their backward; leaves the gradient of the last block's
+// output in `gout`.
+template <typename T>
+static void head_forward_backward(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int slot, int vslot, T* gout) {
+  const Unit& u = m.units.back();
+  const int B = c->arch.batch, F = u.ci, classes = u.co, HW = u.H * u.W;
+  const float* wf = m.wver + (size_t)vslot * align_up(m.n_params, 64);
+  T* S = slot_T<T>(m, slot);
+  float* Fs = slot_F(m, slot);
+  const T* x = m.units.size() >= 2 ? S + m.units[m.units.size() - 2].t_y : module_input<T>(c, m, tau);
+  const size_t rows = (size_t)B * HW;
+  const T* feat = x;
+  if (u.bn) {
+    bn_stats<T>(L, m, x, rows, F, c->arch.bn_eps, Fs + u.st1);
+    bn_apply<T>(L, x, Fs + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows, F);
+    feat = S + u.t_a;
+  }
+  const int32_t* labels = c->labels + (size_t)(tau % c->label_ring) * B;
+  T* dfeat = u.bn ? reinterpret_cast<T*>(m.temps[2]) : gout;
+  const size_t smem = (size_t)(2 * F + classes) * 4;
+  head_fwd_bwd_kernel<T><<<B, 128, smem, L.st>>>(feat, wf + u.w1, wf + u.w2, labels, HW, F, classes, B, m.pooled,
+                                                  m.dlogits, m.loss_n, dfeat, c->flags + 1);
+  L.check();
+  head_param_grad_kernel<<<classes, 128, 0, L.st>>>(m.pooled, m.dlogits, m.loss_n, F, classes, B, m.grad + u.w1,
+                                                     m.grad + u.w2, m.loss, c->flags);
+  L.check();
+  if (u.bn)
+    bn_backward<T>(L, m, dfeat, feat, x, Fs + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr, nullptr, nullptr,
+                   nullptr, nullptr, nullptr, gout, nullptr, rows, F);
+}
+
+// Chain rule through the module's blocks (and stem) for the batch saved in `slot`.
+//   gin   gradient with respect to the module output (already shrunk), consumed
+//   gfirst where the gradient of the module input goes (mailbox slot; unused for module 1)
+template <typename T>
+static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int slot, int vslot, T* gin, T* gfirst) {
+  const int B = c->arch.batch;
+  const T* wt = weights_of<T>(m, vslot);
+  const float* wf = m.wver + (size_t)vslot * align_up(m.n_params, 64);
+  T* S = slot_T<T>(m, slot);
+  float* F = slot_F(m, slot);
+  T* G[2] = {reinterpret_cast<T*>(m.temps[0]), reinterpret_cast<T*>(m.temps[1])};
+  T* T1 = reinterpret_cast<T*>(m.temps[2]);
+  T* T2 = reinterpret_cast<T*>(m.temps[3]);
+  T* T3 = reinterpret_cast<T*>(m.temps[4]);
+  T* dy = gin;
+  const int nu = (int)m.units.size();
+  for (int i = nu - 1; i >= 0; --i) {
+    const Unit& u = m.units[i];
+    if (u.type == U_HEAD) continue;
+    const T* x = i > 0 ? S + m.units[i - 1].t_y : module_input<T>(c, m, tau);
+    T* gout = (i == 0) ? gfirst : (dy == G[0] ? G[1] : G[0]);
+    const size_t rows_in = (size_t)B * u.H * u.W, rows_out = (size_t)B * u.P * u.Q;
+    switch (u.type) {
+      case U_STEM: {
+        ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
+        const T* dc = dy;
+        if (u.bn) {
+          bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
+                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co);
+          dc = T1;
+        }
+        conv_wgrad<T>(L, m, g, x, dc, m.grad + u.w1);
+        break;
+      }
+      case U_BASIC: {
+        ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
+        ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
+        if (u.proj)
+          bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_c, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, S + u.t_s,
+                         F + u.sts, wf + u.gs, m.grad + u.gs, m.grad + u.bs, nullptr, T1, T2, rows_out, u.co);
+        else
+          bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_c, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
+                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co);
+        conv_wgrad<T>(L, m, g2, S + u.t_b, T1, m.grad + u.w2);
+        conv_dgrad<T>(L, g2, T1, wt + u.w2, T3, nullptr, nullptr);                                     // da1
+        bn_backward<T>(L, m, T3, S + u.t_b, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
+                       nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co);      // dc1
+        conv_wgrad<T>(L, m, g1, x, T1, m.grad + u.w1);
+        const bool need_dx = !(m.k == 1 && i == 0);
+        if (u.proj) {
+          ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
+          conv_wgrad<T>(L, m, gs, x, T2, m.grad + u.ws);
+          if (need_dx) {
+            conv_dgrad<T>(L, gs, T2, wt + u.ws, T3, nullptr, nullptr);
+            conv_dgrad<T>(L, g1, T1, wt + u.w1, gout, T3, nullptr);
+          }
+        } else if (need_dx) {
+          conv_dgrad<T>(L, g1, T1, wt + u.w1, gout, dy, S + u.t_y);
+        }
+        break;
+      }
+      case U_PREACT: {
+        ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
+        ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
+        conv_wgrad<T>(L, m, g2, S + u.t_c, dy, m.grad + u.w2);
+        conv_dgrad<T>(L, g2, dy, wt + u.w2, T1, nullptr, nullptr);                                     // da2
+        bn_backward<T>(L, m, T1, S + u.t_c, S + u.t_b, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
+                       nullptr, nullptr, nullptr, nullptr, nullptr, T2, nullptr, rows_out, u.co);      // dc1
+        conv_wgrad<T>(L, m, g1, S + u.t_a, T2, m.grad + u.w1);
+        if (u.proj) {
+          ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
+          conv_wgrad<T>(L, m, gs, S + u.t_a, dy, m.grad + u.ws);
+          conv_dgrad<T>(L, gs, dy, wt + u.ws, T3, nullptr, nullptr);
+          conv_dgrad<T>(L, g1, T2, wt + u.w1, T1, T3, nullptr);                                        // do
+        } else {
+          conv_dgrad<T>(L, g1, T2, wt + u.w1, T1, nullptr, nullptr);
+        }
+        bn_backward<T>(L, m, T1, S + u.t_a, x, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr, nullptr,
+                       nullptr, nullptr, nullptr, u.proj ? nullptr : dy, gout, nullptr, rows_in, u.ci);
+        break;
+      }
+      default: break;
+    }
+    dy = gout;
+  }
+}
+
+template <typename T>
+static void update_module(fdg_ctx* c, Module& m, Launch& L, int next_vslot) {
+  const size_t n = m.n_params;
+  float* next32 = m.wver + (size_t)next_vslot * align_up(n, 64);
+  bf16* next16 = c->bf16_mode ? m.wver16 + (size_t)next_vslot * align_up(n, 64) : nullptr;
+  int blocks = (int)std::min<size_t>(std::max<size_t>((n / 4 + 255) / 256, 1), 148 * 8);
+  sgd_kernel<<<blocks, 256, 0, L.st>>>(m.theta, m.mom, m.grad, next32, next16, n, c->lr, c->cfg.momentum, c->cfg.weight_decay);
+  L.check();
+}
+
+// One module-step of module m in iteration t (Algorithm I, body of "Parallel for k").
+template <typename T>
+static cudaError_t module_step(fdg_ctx* c, Module& m, cudaStream_t st, bool serial, float* loss_dev) {
+  const int K = c->K, k = m.k;
+  const int64_t t = c->t;
+  const int64_t tau_f = t - k + 1, tau_b = t - 2 * (int64_t)K + k + 1;
+  const int e_prev = (int)((t - 1) % kEventRing), e_now = (int)(t % kEventRing);
+  Launch L{c, st};
+  fdg_sched_entry row;
+  row.t = t; row.k = k; row.tau_f = row.tau_b = row.ver_f = row.ver_b = -1; row.slot_f = row.slot_b = -1;
+
+  auto wait_act = [&]() {
+    if (serial) return;
+    if (k == 1) L.note(cudaStreamWaitEvent(st, c->ev_in[e_now], 0));
+    else L.note(cudaStreamWaitEvent(st, c->mods[k - 2].ev_act[e_prev], 0));
+  };
+  auto wait_grad = [&]() {
+    if (serial || k == K) return;
+    L.note(cudaStreamWaitEvent(st, c->mods[k].ev_grad[e_prev], 0));
+  };
+  auto do_forward = [&]() {
+    if (tau_f < 1) return;
+    const int slot = (int)(tau_f % m.D), vslot = (int)(m.updates % m.Dw);
+    forward_module<T>(c, m, L, tau_f, slot, vslot);
+    m.slot_version[slot] = m.updates; m.slot_batch[slot] = tau_f;
+    row.tau_f = tau_f; row.ver_f = m.updates; row.slot_f = slot;
+    if (k < K) { m.last_out_batch = tau_f; m.last_out_slot = slot; }
+  };
+  auto do_backward_update = [&]() {
+    if (tau_b < 1) return;
+    const int slot = (int)(tau_b % m.D);
+    const int64_t ver = (c->cfg.weight_reading == FDG_STASHED) ? m.slot_version[slot] : m.updates;
+    const int vslot = (int)(ver % m.Dw);
+    T* gin = reinterpret_cast<T*>(m.temps[0]);
+    if (k < K) {
+      // receive + shrink (Eq. 15): the mailbox of module k+1 holds the gradient it produced at t-1
+      const Module& dn = c->mods[k];
+      const T* recv = reinterpret_cast<const T*>(dn.mail) + (size_t)((t - 1) % kMailRing) * align_up(dn.in_elems, 128);
+      scale_tensor<T>(L, recv, gin, c->cfg.beta, dn.in_elems);
+    } else {
+      head_forward_backward<T>(c, m, L, tau_b, slot, vslot, gin);
+      if (loss_dev) L.note(cudaMemcpyAsync(loss_dev, m.loss, sizeof(float), cudaMemcpyDeviceToDevice, st));
+    }
+    T* gfirst = k >= 2 ? reinterpret_cast<T*>(m.mail) + (size_t)(t % kMailRing) * align_up(m.in_elems, 128) : nullptr;
+    backward_module<T>(c, m, L, tau_b, slot, vslot, gin, gfirst);
+    update_module<T>(c, m, L, (int)((m.updates + 1) % m.Dw));
+    m.updates += 1;
+    row.tau_b = tau_b; row.ver_b = ver; row.slot_b = slot;
+    if (k >= 2) { m.last_grad_batch = tau_b; m.last_grad_slot = (int)(t % kMailRing); }
+  };
+  auto rec = [&](cudaEvent_t e) { if (!serial) L.note(cudaEventRecord(e, st)); };
+
+  if (k == K) {
+    wait_act();
+    do_forward();
+    rec(m.ev_act[e_now]);
+    do_backward_update();
+    rec(m.ev_grad[e_now]);
+  } else if (c->cfg.order == FDG_BACKWARD_FIRST) {
+    wait_grad();
+    do_backward_update();
+    rec(m.ev_grad[e_now]);
+    wait_act();
+    do_forward();
+    rec(m.ev_act[e_now]);
+  } else {
+    wait_act();
+    do_forward();
+    rec(m.ev_act[e_now]);
+    wait_grad();
+    do_backward_update();
+    rec(m.ev_grad[e_now]);
+  }
+  if (c->log.size() >= kLogIterations * (size_t)K) c->log.erase(c->log.begin(), c->log.begin() + K);
+  c->log.push_back(row);
+  return L.err;
+}
+
+static fdg_status fail(const fdg_ctx* c, fdg_status s, const std::string& msg) {
+  if (c) c->err = msg;
+  return s;
+}
+static fdg_status cuda_fail(fdg_ctx* c, cudaError_t e, const char* where) {
+  c->latched = FDG_ERR_CUDA;
+  return fail(c, FDG_ERR_CUDA, std::string(where) + ": " + cudaGetErrorString(e));
+}
+
+static cudaError_t drain(fdg_ctx* c) {
+  cudaError_t e = cudaSuccess;
+  if (c->stepped) e = cudaStreamSynchronize(c->last_stream);
+  for (Module& m : c->mods) { cudaError_t r = cudaStreamSynchronize(m.stream); if (e == cudaSuccess) e = r; }
+  return e;
+}
+
+}  // namespace fdg
+
+// =================================================================== C ABI ====
+extern "C" {
+
+const char* fdg_status_string(fdg_status s) {
+  switch (s) {
+    case FDG_OK: return "ok";
+    case FDG_ERR_INVALID_ARG: return "invalid argument";
+    case FDG_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case FDG_ERR_CUDA: return "CUDA error";
+    case FDG_ERR_STATE: return "call not valid in this state";
+    case FDG_ERR_UNSUPPORTED: return "unsupported configuration";
+    case FDG_ERR_NONFINITE: return "non-finite loss";
+    case FDG_ERR_TIMEOUT: return "timeout";
+  }
+  return "unknown status";
+}
+
+const char* fdg_last_error(const fdg_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+static fdg_status make_plan(const fdg_arch* arch, const fdg_config* cfg, fdg_ctx* c) {
+  std::string why;
+  fdg_status s = validate(arch, cfg, &why);
+  if (s != FDG_OK) { c->err = why; return s; }
+  c->arch = *arch; c->cfg = *cfg; c->K = cfg->K;
+  c->splits.assign(cfg->split_after_block, cfg->split_after_block + (cfg->K - 1));
+  c->cfg.split_after_block = nullptr;
+  c->bf16_mode = cfg->precision == FDG_BF16_TC;
+  c->esize = c->bf16_mode ? 2 : 4;
+  c->lr = cfg->lr;
+  plan_modules(c);
+  return FDG_OK;
+}
+
+fdg_status fdg_workspace_bytes(const fdg_arch* arch, const fdg_config* cfg, size_t* out_bytes) {
+  if (!out_bytes) return FDG_ERR_INVALID_ARG;
+  fdg_ctx tmp;
+  fdg_status s = make_plan(arch, cfg, &tmp);
+  if (s != FDG_OK) return s;
+  *out_bytes = carve(&tmp, nullptr);
+  return FDG_OK;
+}
+
+fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_workspace, size_t bytes,
+                      const fdg_stream* streams, fdg_ctx** out_ctx) {
+  if (!out_ctx) return FDG_ERR_INVALID_ARG;
+  *out_ctx = nullptr;
+  if (!dev_workspace || (reinterpret_cast<uintptr_t>(dev_workspace) & 255)) return FDG_ERR_INVALID_ARG;
+  fdg_ctx* c = new (std::nothrow) fdg_ctx();
+  if (!c) return FDG_ERR_STATE;
+  fdg_status s = make_plan(arch, cfg, c);
+  if (s != FDG_OK) { delete c; return s; }
+  const size_t need = carve(c, nullptr);
+  if (bytes < need) { delete c; return FDG_ERR_WORKSPACE_TOO_SMALL; }
+  cudaError_t e = cudaGetDevice(&c->device);
+  if (e == cudaSuccess) e = cudaMemset(dev_workspace, 0, need);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) { delete c; return FDG_ERR_CUDA; }
+  carve(c, static_cast<char*>(dev_workspace));
+  c->own_streams = streams == nullptr;
+  for (int k = 0; k < c->K && e == cudaSuccess; ++k) {
+    Module& m = c->mods[k];
+    if (streams) m.stream = static_cast<cudaStream_t>(streams[k]);
+    else e = cudaStreamCreateWithFlags(&m.stream, cudaStreamNonBlocking);
+    for (int i = 0; i < kEventRing && e == cudaSuccess; ++i) {
+      e = cudaEventCreateWithFlags(&m.ev_act[i], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.ev_grad[i], cudaEventDisableTiming);
+    }
+  }
+  for (int i = 0; i < kEventRing && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
+  if (e != cudaSuccess) { delete c; return FDG_ERR_CUDA; }
+  *out_ctx = c;
+  return FDG_OK;
+}
+
+fdg_status fdg_destroy(fdg_ctx* c) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  cudaError_t e = drain(c);
+  for (Module& m : c->mods) {
+    for (int i = 0; i < kEventRing; ++i) { cudaEventDestroy(m.ev_act[i]); cudaEventDestroy(m.ev_grad[i]); }
+    if (c->own_streams && m.stream) cudaStreamDestroy(m.stream);
+  }
+  for (int i = 0; i < kEventRing; ++i) cudaEventDestroy(c->ev_in[i]);
+  cudaEventDestroy(c->ev_join);
+  delete c;
+  return e == cudaSuccess ? FDG_OK : FDG_ERR_CUDA;
+}
+
+#define FDG_MODULE_OR_FAIL(c, module)                                        \
+  if (!(c)) return FDG_ERR_INVALID_ARG;                                      \
+  if ((module) < 1 || (module) > (c)->K) return fail((c), FDG_ERR_INVALID_ARG, "module index out of range")
+
+fdg_status fdg_param_count(const fdg_ctx* c, int module, size_t* out_n) {
+  FDG_MODULE_OR_FAIL(c, module);
+  if (!out_n) return FDG_ERR_INVALID_ARG;
+  *out_n = c->mods[module - 1].n_params;
+  return FDG_OK;
+}
+
+fdg_status fdg_param_layout(const fdg_ctx* c, int module, fdg_param_entry* dst, size_t cap, size_t* out_n) {
+  FDG_MODULE_OR_FAIL(c, module);
+  const auto& lay = c->mods[module - 1].layout;
+  if (out_n) *out_n = lay.size();
+  if (dst) for (size_t i = 0; i < std::min(cap, lay.size()); ++i) dst[i] = lay[i];
+  return FDG_OK;
+}
+
+static fdg_status copy_vec(fdg_ctx* c, int module, float* dev_vec, const float* src, float* dst, size_t n, bool refresh) {
+  FDG_MODULE_OR_FAIL(c, module);
+  Module& m = c->mods[module - 1];
+  if (n != m.n_params || (!src && !dst)) return fail(c, FDG_ERR_INVALID_ARG, "element count does not match fdg_param_count");
+  cudaError_t e = drain(c);
+  if (e == cudaSuccess && n) {
+    if (src) e = cudaMemcpy(dev_vec, src, n * 4, cudaMemcpyDefault);
+    else e = cudaMemcpy(dst, dev_vec, n * 4, cudaMemcpyDefault);
+  }
+  if (e == cudaSuccess && refresh && n) {
+    for (int v = 0; v < m.Dw && e == cudaSuccess; ++v) {
+      e = cudaMemcpy(m.wver + (size_t)v * align_up(n, 64), m.theta, n * 4, cudaMemcpyDeviceToDevice);
+      if (e == cudaSuccess && c->bf16_mode) {
+        cast_kernel<bf16><<<(int)std::min<size_t>((n + 255) / 256, 1184), 256, 0, m.stream>>>(m.theta, m.wver16 + (size_t)v * align_up(n, 64), n);
+        ++c->launches;
+        e = cudaGetLastError();
+      }
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(m.stream);
+  }
+  return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "parameter copy");
+}
+
+fdg_status fdg_set_params(fdg_ctx* c, int module, const float* src, size_t n) {
+  if (!src) return FDG_ERR_INVALID_ARG;
+  FDG_MODULE_OR_FAIL(c, module);
+  return copy_vec(c, module, c->mods[module - 1].theta, src, nullptr, n, true);
+}
+fdg_status fdg_set_momentum(fdg_ctx* c, int module, const float* src, size_t n) {
+  if (!src) return FDG_ERR_INVALID_ARG;
+  FDG_MODULE_OR_FAIL(c, module);
+  return copy_vec(c, module, c->mods[module - 1].mom, src, nullptr, n, false);
+}
+fdg_status fdg_get_params(fdg_ctx* c, int module, float* dst, size_t n) {
+  if (!dst) return FDG_ERR_INVALID_ARG;
+  FDG_MODULE_OR_FAIL(c, module);
+  return copy_vec(c, module, c->mods[module - 1].theta, nullptr, dst, n, false);
+}
+fdg_status fdg_get_grads(fdg_ctx* c, int module, float* dst, size_t n) {
+  if (!dst) return FDG_ERR_INVALID_ARG;
+  FDG_MODULE_OR_FAIL(c, module);
+  return copy_vec(c, module, c->mods[module - 1].grad, nullptr, dst, n, false);
+}
+fdg_status fdg_get_momentum(fdg_ctx* c, int module, float* dst, size_t n) {
+  if (!dst) return FDG_ERR_INVALID_ARG;
+  FDG_MODULE_OR_FAIL(c, module);
+  return copy_vec(c, module, c->mods[module - 1].mom, nullptr, dst, n, false);
+}
+
+fdg_status fdg_set_lr(fdg_ctx* c, float lr) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (!(lr >= 0.f)) return fail(c, FDG_ERR_INVALID_ARG, "learning rate must be >= 0");
+  c->lr = lr;
+  return FDG_OK;
+}
+
+fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, const int32_t* labels_dev, float* loss_dev) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (!images_dev || !labels_dev) return fail(c, FDG_ERR_INVALID_ARG, "images and labels must not be null");
+  if (c->latched != FDG_OK) return c->latched;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const bool serial = c->cfg.serial != 0;
+  c->last_stream = cs; c->stepped = true;
+  c->t += 1;
+  const int64_t t = c->t;
+  Module& m1 = c->mods[0];
+  cudaError_t e = cudaSuccess;
+  // a0: ingest batch t into module 1's image ring and the label ring
+  if (!serial) e = cudaStreamWaitEvent(cs, m1.ev_grad[(t - 1) % kEventRing], 0);
+  if (e != cudaSuccess) return cuda_fail(c, e, "ingest wait");
+  {
+    const size_t rows = (size_t)c->arch.batch * c->arch.in_h * c->arch.in_w;
+    int32_t* lab = c->labels + (size_t)(t % c->label_ring) * c->arch.batch;
+    const size_t slot_off = (size_t)(t % m1.Din) * align_up(m1.in_elems, 128);
+    const int blocks = ew_blocks(rows * m1.in_c);
+    if (c->bf16_mode)
+      ingest_kernel<bf16><<<blocks, 256, 0, cs>>>(images_dev, reinterpret_cast<bf16*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch);
+    else
+      ingest_kernel<float><<<blocks, 256, 0, cs>>>(images_dev, reinterpret_cast<float*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch);
+    ++c->launches;
+    e = cudaGetLastError();
+    if (e == cudaSuccess && !serial) e = cudaEventRecord(c->ev_in[t % kEventRing], cs);
+    if (e != cudaSuccess) return cuda_fail(c, e, "ingest");
+  }
+  for (int k = 0; k < c->K; ++k) {
+    Module& m = c->mods[k];
+    cudaStream_t st = serial ? cs : m.stream;
+    e = c->bf16_mode ? module_step<bf16>(c, m, st, serial, loss_dev) : module_step<float>(c, m, st, serial, loss_dev);
+    if (e != cudaSuccess) return cuda_fail(c, e, "module step");
+  }
+  return FDG_OK;
+}
+
+fdg_status fdg_sync(fdg_ctx* c, fdg_stream stream) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaSuccess;
+  if (!c->cfg.serial)
+    for (Module& m : c->mods) {
+      if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, m.stream);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, c->ev_join, 0);
+    }
+  if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
+  int flags[2] = {0, 0};
+  if (e == cudaSuccess) e = cudaMemcpy(flags, c->flags, sizeof(flags), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(c, e, "sync");
+  if (flags[0] || flags[1]) {
+    cudaMemset(c->flags, 0, sizeof(flags));
+    if (flags[1]) return fail(c, FDG_ERR_INVALID_ARG, "a label was outside [0, num_classes)");
+    return fail(c, FDG_ERR_NONFINITE, "a loss computed since the last sync was NaN or Inf");
+  }
+  return c->latched;
+}
+
+static fdg_status export_tensor(fdg_ctx* c, const void* src, size_t rows, int c_store, int c_logical, float* dst, size_t n) {
+  if (n != rows * (size_t)c_logical) return fail(c, FDG_ERR_INVALID_ARG, "element count does not match fdg_boundary_elems");
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  const int blocks = ew_blocks(n);
+  if (c->bf16_mode) export_kernel<bf16><<<blocks, 256>>>(static_cast<const bf16*>(src), c->staging, rows, c_store, c_logical);
+  else export_kernel<float><<<blocks, 256>>>(static_cast<const float*>(src), c->staging, rows, c_store, c_logical);
+  ++c->launches;
+  e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaMemcpy(dst, c->staging, n * 4, cudaMemcpyDefault);
+  return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "export");
+}
+
+fdg_status fdg_boundary_elems(const fdg_ctx* c, int module, size_t* out_elems, size_t* in_elems) {
+  FDG_MODULE_OR_FAIL(c, module);
+  const Module& m = c->mods[module - 1];
+  if (out_elems) *out_elems = m.out_elems;
+  if (in_elems) *in_elems = (size_t)c->arch.batch * m.in_h * m.in_w * m.in_c_logical;
+  return FDG_OK;
+}
+
+fdg_status fdg_get_module_output(fdg_ctx* c, int module, float* dst, size_t n, int64_t* batch_index) {
+  FDG_MODULE_OR_FAIL(c, module);
+  if (!dst || !batch_index) return FDG_ERR_INVALID_ARG;
+  if (module == c->K) return fail(c, FDG_ERR_INVALID_ARG, "the top module has no output activation");
+  Module& m = c->mods[module - 1];
+  *batch_index = m.last_out_batch;
+  if (m.last_out_batch < 0) return FDG_OK;
+  const size_t off = (size_t)m.last_out_slot * m.slot_elems + m.units.back().t_y;
+  const char* src = m.fifo + off * c->esize;
+  const Unit& u = m.units.back();
+  return export_tensor(c, src, (size_t)c->arch.batch * u.P * u.Q, u.co, u.co, dst, n);
+}
+
+fdg_status fdg_get_input_grad(fdg_ctx* c, int module, float* dst, size_t n, int64_t* batch_index) {
+  FDG_MODULE_OR_FAIL(c, module);
+  if (!dst || !batch_index) return FDG_ERR_INVALID_ARG;
+  if (module == 1) return fail(c, FDG_ERR_INVALID_ARG, "the gradient with respect to the images is never formed");
+  Module& m = c->mods[module - 1];
+  *batch_index = m.last_grad_batch;
+  if (m.last_grad_batch < 0) return FDG_OK;
+  const char* src = m.mail + (size_t)m.last_grad_slot * align_up(m.in_elems, 128) * c->esize;
+  return export_tensor(c, src, (size_t)c->arch.batch * m.in_h * m.in_w, m.in_c, m.in_c_logical, dst, n);
+}
+
+fdg_status fdg_get_schedule_log(const fdg_ctx* c, fdg_sched_entry* dst, size_t cap, size_t* out_n) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (out_n) *out_n = c->log.size();
+  if (dst) for (size_t i = 0; i < std::min(cap, c->log.size()); ++i) dst[i] = c->log[i];
+  return FDG_OK;
+}
+
+fdg_status fdg_launch_count(const fdg_ctx* c, uint64_t* out_n) {
+  if (!c || !out_n) return FDG_ERR_INVALID_ARG;
+  *out_n = c->launches;
+  return FDG_OK;
+}
+
+}  // extern "C"

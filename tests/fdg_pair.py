@@ -1,0 +1,76 @@
+"""Runs the CUDA library and the CPU oracle side by side on the same seeded inputs
+and compares them step by step.  Used by the GPU parity tests and the smoke check."""
+import numpy as np
+
+import fdg_synth as S
+from oracle import fdg as ofdg
+from oracle import nets as onets
+
+
+def relmax(a, b):
+    """max|a-b| / max|b| (b = oracle)."""
+    return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-30))
+
+
+def relfro(a, b):
+    return float(np.linalg.norm(a.astype(np.float64) - b) / max(np.linalg.norm(b), 1e-30))
+
+
+def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_decay=5e-4,
+             order="backward_first", weight_reading="stashed", precision="fp32", serial=False, seed=0,
+             jitter=True, oracle_dtype=np.float64, check_every_step=True):
+    """Returns a dict of worst-case errors and the two schedule logs."""
+    import torch
+    from paper_1906_09108_b200 import binding as B
+
+    arch_o = onets.Arch(**arch_kw)
+    cfg_o = ofdg.FDGConfig(K=K, split_after_block=tuple(splits), beta=beta, lr=lr, momentum=momentum,
+                           weight_decay=weight_decay, order=order, weight_reading=weight_reading)
+    orc = ofdg.FDGOracle(arch_o, cfg_o, dtype=oracle_dtype)
+    g = B.FDG(B.make_arch(**arch_kw), K=K, split_after_block=tuple(splits), beta=beta, lr=lr, momentum=momentum,
+              weight_decay=weight_decay,
+              order=B.FDG_BACKWARD_FIRST if order == "backward_first" else B.FDG_FORWARD_FIRST,
+              weight_reading=B.FDG_STASHED if weight_reading == "stashed" else B.FDG_CURRENT,
+              precision=B.FDG_FP32_CUDACORE if precision == "fp32" else B.FDG_BF16_TC, serial=serial)
+    for k in range(1, K + 1):
+        spec_o = [(kind, tuple(shape)) for _, kind, shape in orc.param_spec(k)]
+        spec_g = [(kind, tuple(shape)) for _, kind, shape in g.param_layout(k)]
+        assert spec_o == spec_g, "parameter layouts differ in module %d" % k
+        p = S.init_params(seed, k, orc.param_spec(k), jitter=jitter)
+        orc.set_params(k, p)
+        g.set_params(k, p)
+    a = arch_o
+    res = dict(out=0.0, gin=0.0, loss=0.0, grads=0.0, steps=steps)
+    loss_dev = torch.zeros(1, dtype=torch.float32, device="cuda")
+    for t in range(1, steps + 1):
+        x = S.images(seed, t, a.batch, a.in_h, a.in_w, a.in_c)
+        y = S.labels(seed, t, a.batch, a.num_classes)
+        lo = orc.step(x, y)
+        g.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), loss_dev)
+        if not (check_every_step or t == steps):
+            continue
+        g.sync()
+        if lo is not None:
+            res["loss"] = max(res["loss"], abs(float(loss_dev.item()) - lo) / max(abs(lo), 1e-30))
+        for k in range(1, K + 1):
+            if k < K and orc.module_output[k] is not None:
+                b, out = g.module_output(k)
+                bo, oo = orc.module_output[k]
+                assert b == bo, ("module output batch", t, k, b, bo)
+                res["out"] = max(res["out"], relmax(out, oo.reshape(-1)))
+            if k >= 2 and orc.input_grad[k] is not None:
+                b, gi = g.input_grad(k)
+                bo, go = orc.input_grad[k]
+                assert b == bo, ("input grad batch", t, k, b, bo)
+                res["gin"] = max(res["gin"], relmax(gi, go.reshape(-1)))
+            go = orc.get_grads(k)
+            if go is not None:
+                res["grads"] = max(res["grads"], relfro(g.get_grads(k), go))
+    g.sync()
+    res["params"] = max(relfro(g.get_params(k), orc.get_params(k)) for k in range(1, K + 1))
+    res["momentum"] = max(relfro(g.get_momentum(k), orc.get_momentum(k)) for k in range(1, K + 1))
+    res["log_gpu"] = [(r["t"], r["k"], r["tau_f"], r["tau_b"], r["ver_f"], r["ver_b"]) for r in g.schedule_log()]
+    res["log_oracle"] = [(r["t"], r["k"], r["tau_f"], r["tau_b"], r["ver_f"], r["ver_b"]) for r in orc.log]
+    res["launches"] = g.launch_count()
+    g.close()
+    return res

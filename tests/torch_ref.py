@@ -81,4 +81,4 @@ def loss_and_grad(arch, theta_np, images_np, labels_np):
     loss = network_loss(arch, theta, torch.tensor(images_np, dtype=torch.float64),
                         torch.tensor(labels_np))
     (g,) = torch.autograd.grad(loss, theta)
-    return float(loss), g.numpy()
+    return float(loss.detach()), g.numpy()
