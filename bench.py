@@ -1,0 +1,301 @@
+"""FDG training throughput on B200: `python bench.py --gpus N --steps K --warmup W`.
+
+Workload: ResNet-110 (6n+2, n=18, 16/32/64 channels), K=4 modules split after blocks
+13/27/41, batch 128, 32x32x3 synthetic N(0,1) images, 10 uniform classes, beta 0.2,
+lr 0.01, momentum 0.9, weight decay 5e-4, one CUDA stream per module.  A step is one
+call of fdg_step: one iteration of Algorithm I for all four modules (ingest, shrink,
+backward, update, forward, handoff).  The pipeline is filled before timing.
+
+Prints ONE JSON line (rank 0).  `value` = images/s with the 16 input batches resident in
+HBM; `e2e` = the same through fdg_step_host from pinned host memory with the loss read
+back every step; `roofline` = the dominant kernel class timed alone (serial context, CUDA
+events on its stream) against the measured peak; `cpu_baseline` = the CPU oracle on a
+bounded sample.  `--impl reference` times the oracle alone on the host cores.
+With N > 1 (torchrun) every rank runs an independent replica: the path has no
+inter-GPU step, so there is no collective on the data path.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+ARCH = dict(family="resnet6n2", n_per_stage=18, widths=(16, 32, 64), stem_width=16, in_h=32, in_w=32, in_c=3,
+            num_classes=10, batch=128)
+K_MODULES = 4
+SPLITS = (13, 27, 41)
+BETA, LR, MOM, WD = 0.2, 0.01, 0.9, 5e-4
+WORKLOAD = "ResNet-110 (6n+2, n=18) K=4 batch 128, 32x32x3 synthetic N(0,1), 10 classes"
+METRIC = "FDG train images/sec on 1 B200 (ResNet-110, K=4)"
+POOL = 16
+ORACLE_SAMPLE_BATCH = 16
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------ oracle arm --
+def oracle_images_per_s(steps, warmup, batch=ORACLE_SAMPLE_BATCH):
+    """The CPU oracle as it stands, same network / K / hyper-parameters, on a batch-`batch`
+    sample of the workload; the pipeline is filled (2K iterations) before warm-up."""
+    import torch
+    import fdg_synth as S
+    from oracle import fdg as ofdg
+    from oracle import nets as onets
+    arch = dict(ARCH, batch=batch)
+    o = ofdg.FDGOracle(onets.Arch(**arch), ofdg.FDGConfig(K=K_MODULES, split_after_block=SPLITS, beta=BETA, lr=LR,
+                                                         momentum=MOM, weight_decay=WD))
+    for k in range(1, K_MODULES + 1):
+        o.set_params(k, S.init_params(0, k, o.param_spec(k)))
+    t = 0
+
+    def one():
+        nonlocal t
+        t += 1
+        o.step(S.images(0, t, batch, 32, 32, 3), S.labels(0, t, batch, 10))
+
+    for _ in range(2 * K_MODULES + warmup):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    dt = time.perf_counter() - t0
+    return batch * steps / dt, dt / steps, torch.get_num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = args.steps if args.steps is not None else 4
+    warmup = args.warmup if args.warmup is not None else 1
+    ips, sec, cores = oracle_images_per_s(steps, warmup)
+    sample = ("same network, K and hyper-parameters at batch %d of 128; pipeline filled (2K iterations) before the "
+              "warm-up; numpy float64" % ORACLE_SAMPLE_BATCH)
+    line = dict(impl="reference", metric=METRIC, value=ips, unit="images/s", n_gpus=args.gpus, steps=steps,
+                warmup=warmup, ms_per_step=sec * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", config=dict(workload=WORKLOAD, K=K_MODULES, global_batch=ARCH["batch"]),
+                cpu_baseline=dict(value=ips, unit="images/s", cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=ips, unit="images/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------- GPU arm --
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.file,
+                                         stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def make_fdg(B, precision, serial):
+    import fdg_synth as S
+    g = B.FDG(B.make_arch(**ARCH), K=K_MODULES, split_after_block=SPLITS, beta=BETA, lr=LR, momentum=MOM,
+              weight_decay=WD, precision=precision, serial=serial)
+    for k in range(1, K_MODULES + 1):
+        g.set_params(k, S.init_params(0, k, g.param_layout(k)))
+    return g
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    import fdg_synth as S
+    from paper_1906_09108_b200 import binding as B
+
+    steps = args.steps if args.steps is not None else 50
+    warmup = args.warmup if args.warmup is not None else 10
+    warmup = max(warmup, 3)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    precision = B.FDG_BF16_TC if args.precision == "bf16" else B.FDG_FP32_CUDACORE
+    b = ARCH["batch"]
+
+    pool_x = [torch.from_numpy(S.images(rank, t, b, 32, 32, 3)).cuda() for t in range(1, POOL + 1)]
+    pool_y = [torch.from_numpy(S.labels(rank, t, b, 10)).cuda() for t in range(1, POOL + 1)]
+    host_x = [torch.from_numpy(S.images(rank, t, b, 32, 32, 3)).pin_memory() for t in range(1, POOL + 1)]
+    host_y = [torch.from_numpy(S.labels(rank, t, b, 10)).pin_memory() for t in range(1, POOL + 1)]
+    loss_host = torch.zeros(1, dtype=torch.float32).pin_memory()
+    loss_dev = torch.zeros(1, dtype=torch.float32, device="cuda")
+
+    g = make_fdg(B, precision, serial=False)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(n, step_fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for i in range(n):
+            step_fn(i)
+        g.sync()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            tm = torch.tensor([ms], device="cuda")
+            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+            ms = float(tm.item())
+        return ms
+
+    dev_step = lambda i: g.step(pool_x[i % POOL], pool_y[i % POOL], loss_dev)
+    for i in range(2 * K_MODULES + warmup):          # pipeline fill + warm-up, untimed
+        dev_step(i)
+    g.sync()
+    sampler = ClockSampler(local) if rank == 0 else None
+    n0 = g.launch_count()
+    ms = timed(steps, dev_step)
+    launches = g.launch_count() - n0
+    clocks = sampler.stop() if sampler else None
+    value = world * b * steps / (ms * 1e-3)
+
+    # end to end: host buffers through the C ABI, loss read back every step
+    def host_step(i):
+        g.step_host(host_x[i % POOL], host_y[i % POOL], loss_host)
+    for i in range(3):
+        host_step(i)
+    g.sync()
+    ms_e2e = timed(steps, host_step)
+    e2e_value = world * b * steps / (ms_e2e * 1e-3)
+    h2d = host_x[0].numel() * 4 + host_y[0].numel() * 4
+    final_loss = float(loss_host.item())
+    g.close()
+
+    line = None
+    if rank == 0:
+        # dominant kernel class, timed alone on a serial context of the same workload
+        peaks = measured_peaks()
+        gs = make_fdg(B, precision, serial=True)
+        for i in range(2 * K_MODULES + 3):
+            gs.step(pool_x[i % POOL], pool_y[i % POOL])
+        gs.sync()
+        gs.profile_enable(True)
+        prof_steps = min(steps, 10)
+        for i in range(prof_steps):
+            gs.step(pool_x[i % POOL], pool_y[i % POOL])
+        stats = [s for s in gs.profile_read() if s["launches"]]
+        gs.close()
+        total = sum(s["total_ms"] for s in stats)
+        top = max(stats, key=lambda s: s["total_ms"])
+        sec = top["total_ms"] * 1e-3
+        hbm_frac = top["bytes"] / sec / 1e9 / peaks["hbm_gbs"]
+        if args.precision == "bf16":
+            tensor_peak = peaks["bf16_tflops"]
+            tensor_frac = top["flops"] / sec / 1e12 / tensor_peak
+            if tensor_frac >= hbm_frac:
+                roof = dict(bound="tensor", achieved=top["flops"] / sec / 1e12, peak=tensor_peak, unit="TFLOP/s")
+            else:
+                roof = dict(bound="hbm", achieved=top["bytes"] / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+        elif top["name"].startswith("conv"):
+            # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x max SM clock
+            alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+            roof = dict(bound="alu", achieved=top["flops"] / sec / 1e12, peak=alu_peak, unit="TFLOP/s")
+        else:
+            roof = dict(bound="hbm", achieved=top["bytes"] / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+        roof.update(frac=roof["achieved"] / roof["peak"], traffic=None, kernel=top["name"],
+                    peak_source=peaks["source"], launches=top["launches"],
+                    avg_us=top["total_ms"] * 1e3 / top["launches"],
+                    share_of_gpu_time=top["total_ms"] / total,
+                    how="CUDA events around every launch on its stream, serial context, %d steps" % prof_steps,
+                    per_class={s["name"]: dict(ms_per_step=s["total_ms"] / prof_steps, share=s["total_ms"] / total,
+                                               gbs=s["bytes"] / (s["total_ms"] * 1e-3) / 1e9,
+                                               tflops=s["flops"] / (s["total_ms"] * 1e-3) / 1e12) for s in stats})
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            ips, sec_o, cores = oracle_images_per_s(2, 0)
+            cpu = dict(value=ips, unit="images/s", cores=cores, kind="oracle",
+                       sample="same network, K and hyper-parameters at batch %d of 128, 2 iterations timed after "
+                              "the pipeline fill (2K iterations); numpy float64" % ORACLE_SAMPLE_BATCH)
+        line = dict(metric=METRIC, value=value, unit="images/s", n_gpus=world, steps=steps, warmup=warmup,
+                    ms_per_step=ms / steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="bf16" if args.precision == "bf16" else "f32", data="synthetic",
+                    config=dict(workload=WORKLOAD, K=K_MODULES, splits=list(SPLITS), global_batch=world * b,
+                                beta=BETA, lr=LR, precision=args.precision, streams=K_MODULES,
+                                parallelism="replicas only" if world > 1 else "single GPU",
+                                l2="activation FIFO touched per step (>1 GiB) exceeds the 126 MB L2; "
+                                   "16 input batches cycled"),
+                    clocks=clocks,
+                    e2e=dict(value=e2e_value, unit="images/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=4,
+                             ms_per_step=ms_e2e / steps, final_loss=final_loss),
+                    gpu_launches=int(launches), roofline=roof, cpu_baseline=cpu)
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="fdg", choices=["fdg", "reference"])
+    ap.add_argument("--precision", default="fp32", choices=["fp32", "bf16"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

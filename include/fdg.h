@@ -172,6 +172,15 @@ fdg_status fdg_set_lr(fdg_ctx* ctx, float lr);
 fdg_status fdg_step(fdg_ctx* ctx, fdg_stream stream, const float* images_dev, const int32_t* labels_dev,
                     float* loss_dev);
 
+/* The same iteration fed from host memory: copies `images_host` (fp32, same layout) and
+ * `labels_host` to a staging area of the workspace with cudaMemcpyAsync on `stream`, runs
+ * fdg_step on them, and enqueues a device-to-host copy of the loss of batch t-K+1 into
+ * `loss_host` (nullable; untouched while t < K).  Pinned host buffers keep the call
+ * asynchronous; pageable ones make the copies block.  The host buffers may be reused once
+ * `stream` has passed the copies; read *loss_host after fdg_sync.  Errors as fdg_step. */
+fdg_status fdg_step_host(fdg_ctx* ctx, fdg_stream stream, const float* images_host, const int32_t* labels_host,
+                         float* loss_host);
+
 /* Makes `stream` wait for every module stream, then blocks the host until `stream` is idle.
  * Returns FDG_ERR_NONFINITE if any loss computed since the last call was NaN/Inf,
  * FDG_ERR_CUDA on an asynchronous CUDA error. */
@@ -192,6 +201,24 @@ fdg_status fdg_boundary_elems(const fdg_ctx* ctx, int module, size_t* out_elems,
 /* Copies at most `cap` rows of the schedule log (oldest first) and writes the number
  * of rows recorded so far to *out_n.  The log keeps every row of the last 4096 iterations. */
 fdg_status fdg_get_schedule_log(const fdg_ctx* ctx, fdg_sched_entry* dst, size_t cap, size_t* out_n);
+
+/* Optional per-launch profiler.  While enabled, every kernel launch is bracketed by two
+ * CUDA events on its own stream (up to 65536 launches between reads; later ones are not
+ * timed).  fdg_profile_read blocks until the device is idle, writes one row per kernel class
+ * (at most `cap`; the number of classes goes to *out_n) and clears the record.  `bytes` and
+ * `flops` are algorithmic: each operand tensor counted once per launch, 2 flops per
+ * multiply-add.  With one stream per module the kernels of different modules overlap, so a
+ * launch's duration includes time shared with others; enable on a serial context to time
+ * kernels alone.  Both calls block the host. */
+typedef struct {
+  char name[32];
+  uint64_t launches;
+  double total_ms;
+  double bytes;
+  double flops;
+} fdg_kernel_stat;
+fdg_status fdg_profile_enable(fdg_ctx* ctx, int on);
+fdg_status fdg_profile_read(fdg_ctx* ctx, fdg_kernel_stat* dst, size_t cap, size_t* out_n);
 
 /* Number of kernel launches the library has enqueued since fdg_create. */
 fdg_status fdg_launch_count(const fdg_ctx* ctx, uint64_t* out_n);

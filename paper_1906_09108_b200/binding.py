@@ -23,9 +23,10 @@ PARAM_KINDS = {0: "conv", 1: "bn_gamma", 2: "bn_beta", 3: "fc_w", 4: "fc_b"}
 
 EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count", "fdg_param_layout",
            "fdg_set_params", "fdg_set_momentum", "fdg_get_params", "fdg_get_grads", "fdg_get_momentum",
-           "fdg_set_lr", "fdg_step", "fdg_sync", "fdg_get_module_output", "fdg_get_input_grad",
+           "fdg_set_lr", "fdg_step", "fdg_step_host", "fdg_sync", "fdg_profile_enable", "fdg_profile_read", "fdg_get_module_output", "fdg_get_input_grad",
            "fdg_boundary_elems", "fdg_get_schedule_log", "fdg_launch_count", "fdg_status_string",
-           "fdg_last_error"]
+           "fdg_last_error", "fdg_conv_forward", "fdg_conv_dgrad", "fdg_conv_flip_weights",
+           "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_path"]
 
 
 class fdg_arch(C.Structure):
@@ -50,6 +51,16 @@ class fdg_sched_entry(C.Structure):
                 ("ver_f", C.c_int64), ("ver_b", C.c_int64), ("slot_f", C.c_int32), ("slot_b", C.c_int32)]
 
 
+class fdg_conv_shape(C.Structure):
+    _fields_ = [("N", C.c_int), ("H", C.c_int), ("W", C.c_int), ("Ci", C.c_int), ("Co", C.c_int), ("R", C.c_int),
+                ("stride", C.c_int), ("pad", C.c_int)]
+
+
+class fdg_kernel_stat(C.Structure):
+    _fields_ = [("name", C.c_char * 32), ("launches", C.c_uint64), ("total_ms", C.c_double), ("bytes", C.c_double),
+                ("flops", C.c_double)]
+
+
 def load_library(path=LIB_PATH):
     if not os.path.exists(path):
         raise ImportError("libfdg.so is not built (%s); run `python -m paper_1906_09108_b200.build`" % path)
@@ -69,12 +80,21 @@ def load_library(path=LIB_PATH):
         "fdg_get_momentum": [vp, C.c_int, vp, sz],
         "fdg_set_lr": [vp, C.c_float],
         "fdg_step": [vp, vp, vp, vp, vp],
+        "fdg_step_host": [vp, vp, vp, vp, vp],
         "fdg_sync": [vp, vp],
+        "fdg_profile_enable": [vp, C.c_int],
+        "fdg_profile_read": [vp, P(fdg_kernel_stat), sz, P(sz)],
         "fdg_get_module_output": [vp, C.c_int, vp, sz, P(i64)],
         "fdg_get_input_grad": [vp, C.c_int, vp, sz, P(i64)],
         "fdg_boundary_elems": [vp, C.c_int, P(sz), P(sz)],
         "fdg_get_schedule_log": [vp, P(fdg_sched_entry), sz, P(sz)],
         "fdg_launch_count": [vp, P(C.c_uint64)],
+        "fdg_conv_forward": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, vp, vp],
+        "fdg_conv_dgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, vp, vp, vp, vp],
+        "fdg_conv_flip_weights": [P(fdg_conv_shape), vp, vp, vp],
+        "fdg_conv_wgrad_scratch_bytes": [C.c_int, P(fdg_conv_shape), P(sz)],
+        "fdg_conv_wgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, sz, vp, vp],
+        "fdg_conv_path": [C.c_int, P(fdg_conv_shape), C.c_int, P(C.c_int)],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -195,6 +215,22 @@ class FDG:
         self._check(self.lib.fdg_step(self.ctx, st, images_dev.data_ptr(), labels_dev.data_ptr(),
                                       loss_dev.data_ptr() if loss_dev is not None else None), self.ctx)
 
+    def step_host(self, images_host, labels_host, loss_host=None, stream=None):
+        """images_host / labels_host / loss_host: CPU tensors (pinned for asynchronous copies)."""
+        st = self.torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self._check(self.lib.fdg_step_host(self.ctx, st, images_host.data_ptr(), labels_host.data_ptr(),
+                                           loss_host.data_ptr() if loss_host is not None else None), self.ctx)
+
+    def profile_enable(self, on=True):
+        self._check(self.lib.fdg_profile_enable(self.ctx, int(on)), self.ctx)
+
+    def profile_read(self):
+        n = C.c_size_t()
+        arr = (fdg_kernel_stat * 32)()
+        self._check(self.lib.fdg_profile_read(self.ctx, arr, 32, C.byref(n)), self.ctx)
+        return [dict(name=e.name.decode(), launches=e.launches, total_ms=e.total_ms, bytes=e.bytes, flops=e.flops)
+                for e in arr[:n.value]]
+
     def sync(self, stream=None):
         st = self.torch.cuda.current_stream().cuda_stream if stream is None else stream
         self._check(self.lib.fdg_sync(self.ctx, st), self.ctx)
@@ -231,3 +267,65 @@ class FDG:
         n = C.c_uint64()
         self._check(self.lib.fdg_launch_count(self.ctx, C.byref(n)), self.ctx)
         return n.value
+
+
+# ---- operator level (include/fdg_ops.h): thin wrappers over torch CUDA tensors -----------
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+class ConvOps:
+    """fdg_conv_* on torch CUDA tensors of the precision's storage type (float32 / bfloat16)."""
+
+    def __init__(self, precision):
+        import torch
+        self.torch = torch
+        self.lib = load_library()
+        self.precision = precision
+        self.dtype = torch.bfloat16 if precision == FDG_BF16_TC else torch.float32
+        self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def _stream(self):
+        return self.torch.cuda.current_stream().cuda_stream
+
+    def _chk(self, rc):
+        if rc != FDG_OK:
+            raise FDGError(rc, self.lib.fdg_status_string(rc).decode())
+
+    def out_hw(self, s):
+        return (s.H + 2 * s.pad - s.R) // s.stride + 1, (s.W + 2 * s.pad - s.R) // s.stride + 1
+
+    def path(self, s, op):
+        v = C.c_int()
+        self._chk(self.lib.fdg_conv_path(self.precision, C.byref(s), op, C.byref(v)))
+        return bool(v.value)
+
+    def forward(self, s, x, w, res=None):
+        p, q = self.out_hw(s)
+        y = self.torch.empty((s.N, p, q, s.Co), dtype=self.dtype, device="cuda")
+        self._chk(self.lib.fdg_conv_forward(self.precision, C.byref(s), _ptr(x), _ptr(w), _ptr(y), _ptr(res),
+                                            _ptr(self.status), self._stream()))
+        return y
+
+    def flip_weights(self, s, w):
+        out = self.torch.empty(s.Ci * 9 * s.Co, dtype=self.torch.bfloat16, device="cuda")
+        self._chk(self.lib.fdg_conv_flip_weights(C.byref(s), _ptr(w), _ptr(out), self._stream()))
+        return out
+
+    def dgrad(self, s, dy, w, w_flipped=None, res=None, res_mask=None):
+        dx = self.torch.empty((s.N, s.H, s.W, s.Ci), dtype=self.dtype, device="cuda")
+        self._chk(self.lib.fdg_conv_dgrad(self.precision, C.byref(s), _ptr(dy), _ptr(w), _ptr(w_flipped), _ptr(dx),
+                                          _ptr(res), _ptr(res_mask), _ptr(self.status), self._stream()))
+        return dx
+
+    def wgrad(self, s, x, dy):
+        n = C.c_size_t()
+        self._chk(self.lib.fdg_conv_wgrad_scratch_bytes(self.precision, C.byref(s), C.byref(n)))
+        scratch = self.torch.empty(max(n.value, 16), dtype=self.torch.uint8, device="cuda")
+        dw = self.torch.empty((s.Co, s.R, s.R, s.Ci), dtype=self.torch.float32, device="cuda")
+        self._chk(self.lib.fdg_conv_wgrad(self.precision, C.byref(s), _ptr(x), _ptr(dy), _ptr(dw), _ptr(scratch),
+                                          n.value, _ptr(self.status), self._stream()))
+        return dw
+
+    def timed_out(self):
+        return bool(self.status.item())

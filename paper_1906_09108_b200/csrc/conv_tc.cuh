@@ -1,0 +1,422 @@
+// 3x3 / stride 1 / pad 1 convolution forward and data gradient as an implicit GEMM on the
+// sm_100a tensor cores: bf16 operands staged in shared memory by TMA, tcgen05.mma with fp32
+// accumulators in tensor memory, epilogue through tcgen05.ld.
+//
+//   D[m][n] = sum_{tap, c} A_tap[m][c] * B_tap[n][c]
+//     m   = 128 consecutive output pixels: whole image rows (or whole images) of an NHWC tensor
+//     A   = the input shifted by the tap offset; the TMA box starts at (w-1+s, h-1+r) and the
+//           hardware zero-fills what falls outside the image, which is the padding
+//     B   = weights [N][9*C]: forward [c_out][r][s][c_in]; data gradient: the flipped and
+//           transposed copy [c_in][2-r][2-s][c_out] (dgrad of a stride-1 3x3 conv is a 3x3 conv)
+//   Both operands are K-major with the channel chunk (16/32/64 channels = 32/64/128 bytes) as
+//   the swizzle span, so the TMA swizzle mode and the MMA descriptor layout agree.
+//
+// One persistent CTA per SM walks tiles (m-tile, n-tile); roles by warp:
+//   warp 0      TMA producer: per (tap, channel chunk) one A box and one B box into a ring stage
+//   warp 1      MMA issuer: C_chunk/16 tcgen05.mma per stage, tcgen05.commit frees the stage;
+//               after the last stage of a tile a commit hands the accumulator to the epilogue
+//   warps 2..5  epilogue: TMEM -> registers -> (+ residual) -> bf16 -> global, 32 rows per warp
+// Two accumulators alternate so the epilogue of tile i overlaps the MMAs of tile i+1.
+// Every wait is bounded: on time-out the CTA raises an error word and leaves without hanging.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fdg {
+namespace tc {
+
+constexpr int kTileM = 128;
+constexpr int kThreads = 192;            // 6 warps
+constexpr uint32_t kSpinLimit = 1u << 24;
+
+struct ConvTcParams {
+  int W, H, N;              // image width, height, batch
+  int rows_per_tile;        // image rows per tile when a tile stays inside one image, else H
+  int imgs_per_tile;        // images per tile (1 unless 128 pixels span whole images)
+  int Ci, Co;               // GEMM-K channels per tap, GEMM-N total
+  int kc;                   // channel chunk per stage: 16, 32 or 64
+  int n_tile;               // GEMM-N per tile (multiple of 16, <= 256)
+  int m_tiles, n_tiles;
+  int stages;
+  uint32_t a_bytes, b_bytes, stage_bytes;   // b_bytes is padded to 1 KiB; b_tx_bytes is what TMA moves
+  uint32_t b_tx_bytes;
+  uint32_t tmem_cols;       // allocated columns (power of two >= 2*n_tile)
+};
+
+// ---------------------------------------------------------------- PTX wrappers --
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the limit is hit or another role has raised *abort_flag.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023) == 1023 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, K-major operand whose rows are one swizzle span wide:
+// rows of `row_bytes` (32/64/128), 8-row groups `8*row_bytes` apart.
+__device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t row_bytes) {
+  const uint64_t layout = row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6);   // SWIZZLE_128B / 64B / 32B
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);                 // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                                // leading byte offset (unused for one span)
+  d |= (uint64_t)(((8 * row_bytes) >> 4) & 0x3FFF) << 32;   // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                                // descriptor version of this architecture
+  d |= layout << 61;
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+// ------------------------------------------------------------------- kernel ----
+// out[m][n] (bf16, row stride Co) = conv + (res ? res[m][n] * [mask ? mask[m][n] > 0 : 1] : 0)
+__global__ void __launch_bounds__(kThreads, 1)
+conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  ConvTcParams p, __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
+                  const __nv_bfloat16* __restrict__ res_mask, int* __restrict__ error_word) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * p.stage_bytes);
+  uint64_t* full = bars;                       // [stages]  TMA -> MMA
+  uint64_t* empty = bars + p.stages;           // [stages]  MMA -> TMA
+  uint64_t* acc_full = empty + p.stages;       // [2]       MMA -> epilogue
+  uint64_t* acc_empty = acc_full + 2;          // [2]       epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int chunks = p.Ci / p.kc;
+  const int k_iters = 9 * chunks;
+  const int total_tiles = p.m_tiles * p.n_tiles;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+        const int mt = tile / p.n_tiles, nt = tile - mt * p.n_tiles;
+        int n0, h0;
+        if (p.imgs_per_tile == 1) {
+          const int tiles_per_img = p.H / p.rows_per_tile;
+          n0 = mt / tiles_per_img; h0 = (mt - n0 * tiles_per_img) * p.rows_per_tile;
+        } else {
+          n0 = mt * p.imgs_per_tile; h0 = 0;
+        }
+        for (int ki = 0; ki < k_iters; ++ki, ++it) {
+          const int s = it % p.stages;
+          const uint32_t ph = (it / p.stages) & 1;
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) break;
+          const int tap = ki / chunks, cc = ki - tap * chunks;
+          const int r = tap / 3, sx = tap - r * 3;
+          uint8_t* a_dst = smem + (size_t)s * p.stage_bytes;
+          uint8_t* b_dst = a_dst + p.a_bytes;
+          mbar_expect_tx(&full[s], p.a_bytes + p.b_tx_bytes);
+          tma_load_4d(a_dst, &map_a, &full[s], cc * p.kc, sx - 1, h0 + r - 1, n0);
+          tma_load_2d(b_dst, &map_b, &full[s], tap * p.Ci + cc * p.kc, nt * p.n_tile);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(p.n_tile);
+      const uint32_t row_bytes = p.kc * 2;
+      uint32_t it = 0, tcount = 0;
+      for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
+        const int acc = tcount & 1;
+        const uint32_t acc_ph = (tcount >> 1) & 1;
+        if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * p.n_tile;
+        bool ok = true;
+        for (int ki = 0; ki < k_iters; ++ki, ++it) {
+          const int s = it % p.stages;
+          const uint32_t ph = (it / p.stages) & 1;
+          if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
+          const uint32_t b_addr = a_addr + p.a_bytes;
+          for (int j = 0; j < p.kc / 16; ++j)
+            tc_mma_bf16(d_tmem, smem_desc_kmajor(a_addr + j * 32, row_bytes), smem_desc_kmajor(b_addr + j * 32, row_bytes),
+                        idesc, (ki | j) != 0);
+          tc_commit(&empty[s]);
+        }
+        if (!ok) break;
+        tc_commit(&acc_full[acc]);
+      }
+    }
+  } else {
+    const int ew = warp - 2;                       // TMEM lanes 32*(warp%4) belong to this warp
+    const int lane_grp = warp & 3;
+    (void)ew;
+    uint32_t tcount = 0;
+    for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
+      const int mt = tile / p.n_tiles, nt = tile - mt * p.n_tiles;
+      const int acc = tcount & 1;
+      const uint32_t acc_ph = (tcount >> 1) & 1;
+      if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) break;
+      tc_fence_after();
+      const size_t row = (size_t)mt * kTileM + lane_grp * 32 + lane;
+      const size_t base = row * p.Co + (size_t)nt * p.n_tile;
+      const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)acc * p.n_tile;
+      for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(taddr + c0, v);
+        tmem_ld_wait();
+        float f[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) f[i] = __uint_as_float(v[i]);
+        if (res) {
+          uint4 r0 = *reinterpret_cast<const uint4*>(res + base + c0);
+          uint4 r1 = *reinterpret_cast<const uint4*>(res + base + c0 + 8);
+          const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
+          const __nv_bfloat16* rb1 = reinterpret_cast<const __nv_bfloat16*>(&r1);
+          float g[16];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { g[i] = __bfloat162float(rb0[i]); g[8 + i] = __bfloat162float(rb1[i]); }
+          if (res_mask) {
+            uint4 m0 = *reinterpret_cast<const uint4*>(res_mask + base + c0);
+            uint4 m1 = *reinterpret_cast<const uint4*>(res_mask + base + c0 + 8);
+            const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&m0);
+            const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&m1);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              if (!(__bfloat162float(mb0[i]) > 0.f)) g[i] = 0.f;
+              if (!(__bfloat162float(mb1[i]) > 0.f)) g[8 + i] = 0.f;
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 16; ++i) f[i] += g[i];
+        }
+        uint4 o0, o1;
+        __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
+        __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          ob0[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+          ob1[i] = __floats2bfloat162_rn(f[8 + 2 * i], f[8 + 2 * i + 1]);
+        }
+        *reinterpret_cast<uint4*>(out + base + c0) = o0;
+        *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+    }
+  }
+
+  // Teardown.  After an abort, TMA copies may still be in flight towards this CTA's shared
+  // memory: give every stage that was armed a bounded chance to complete before leaving.
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) {
+      if (error_word) atomicExch(error_word, 1);
+      for (int s = 0; s < p.stages; ++s)
+        for (uint32_t i = 0; i < (1u << 16); ++i)
+          if (mbar_try_wait(&full[s], 0) || mbar_try_wait(&full[s], 1)) break;
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
+// ----------------------------------------------------------------- host side ---
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+inline CUtensorMapSwizzle swizzle_for(int row_bytes) {
+  return row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+
+// Can this convolution run on the tensor-core kernel?  (3x3, stride 1, pad 1, channel counts
+// that are multiples of 16, image rows that tile 128 pixels exactly.)
+inline bool conv_tc_supported(int N, int H, int W, int Ci, int Co) {
+  if (Ci % 16 || Co % 16 || Ci < 16 || Co < 16) return false;
+  if (kTileM % W) return false;
+  const int rows = kTileM / W;
+  if (rows <= H) { if (H % rows) return false; }
+  else { if (rows % H || N % (rows / H)) return false; }
+  if (W > 256 || H > 256) return false;
+  return true;
+}
+
+inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co) {
+  ConvTcParams p{};
+  p.W = W; p.H = H; p.N = N; p.Ci = Ci; p.Co = Co;
+  const int rows = kTileM / W;
+  if (rows <= H) { p.rows_per_tile = rows; p.imgs_per_tile = 1; }
+  else { p.rows_per_tile = H; p.imgs_per_tile = rows / H; }
+  p.kc = Ci % 64 == 0 ? 64 : (Ci % 32 == 0 ? 32 : 16);
+  int nt = Co;
+  if (nt > 256) { nt = 256; while (Co % nt || nt % 16) nt -= 16; }
+  p.n_tile = nt;
+  p.m_tiles = (int)((size_t)N * H * W / kTileM);
+  p.n_tiles = Co / nt;
+  p.a_bytes = (uint32_t)kTileM * p.kc * 2;
+  p.b_tx_bytes = (uint32_t)nt * p.kc * 2;
+  p.b_bytes = (p.b_tx_bytes + 1023u) & ~1023u;
+  p.stage_bytes = p.a_bytes + p.b_bytes;
+  int stages = (int)(160 * 1024 / p.stage_bytes);
+  p.stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
+  uint32_t cols = 32;
+  while (cols < 2u * nt) cols <<= 1;
+  p.tmem_cols = cols;
+  return p;
+}
+
+inline size_t conv_tc_smem_bytes(const ConvTcParams& p) { return (size_t)p.stages * p.stage_bytes + 1024 + 256; }
+
+// act: bf16 [N][H][W][Ci]; wgt: bf16 [Co][9*Ci] (forward layout, or the flipped/transposed copy for dgrad).
+inline cudaError_t conv_tc_make_maps(const ConvTcParams& p, const void* act, const void* wgt, CUtensorMap* map_a,
+                                     CUtensorMap* map_b) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  const CUtensorMapSwizzle sw = swizzle_for(p.kc * 2);
+  {
+    cuuint64_t dims[4] = {(cuuint64_t)p.Ci, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.N};
+    cuuint64_t strides[3] = {(cuuint64_t)p.Ci * 2, (cuuint64_t)p.W * p.Ci * 2, (cuuint64_t)p.H * p.W * p.Ci * 2};
+    cuuint32_t box[4] = {(cuuint32_t)p.kc, (cuuint32_t)p.W, (cuuint32_t)p.rows_per_tile, (cuuint32_t)p.imgs_per_tile};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (enc(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(act), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  {
+    cuuint64_t dims[2] = {(cuuint64_t)9 * p.Ci, (cuuint64_t)p.Co};
+    cuuint64_t strides[1] = {(cuuint64_t)9 * p.Ci * 2};
+    cuuint32_t box[2] = {(cuuint32_t)p.kc, (cuuint32_t)p.n_tile};
+    cuuint32_t estr[2] = {1, 1};
+    if (enc(map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(wgt), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  return cudaSuccess;
+}
+
+inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const CUtensorMap& map_a,
+                                  const CUtensorMap& map_b, __nv_bfloat16* out, const __nv_bfloat16* res,
+                                  const __nv_bfloat16* res_mask, int* error_word, int sm_count) {
+  static bool attr_set = false;
+  const size_t smem = conv_tc_smem_bytes(p);
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int tiles = p.m_tiles * p.n_tiles;
+  const int grid = tiles < sm_count ? tiles : sm_count;
+  conv3x3_tc_kernel<<<grid, kThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, error_word);
+  return cudaGetLastError();
+}
+
+// Flipped / transposed weight copy for the data gradient of a stride-1 3x3 convolution:
+// dst[ci][2-r][2-s][co] = src[co][r][s][ci].  One block row per entry of `table`
+// (src offset, dst offset, Co, Ci), all offsets in elements from the two base pointers.
+struct FlipEntry { unsigned long long src, dst; int Co, Ci; };
+__global__ void wflip_kernel(const __nv_bfloat16* __restrict__ src_base, __nv_bfloat16* __restrict__ dst_base,
+                             const FlipEntry* __restrict__ table) {
+  const FlipEntry e = table[blockIdx.y];
+  const int n = e.Co * 9 * e.Ci;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int co = i % e.Co, t = (i / e.Co) % 9, ci = i / (9 * e.Co);       // i indexes dst[ci][t][co]
+    dst_base[e.dst + i] = src_base[e.src + ((size_t)co * 9 + (8 - t)) * e.Ci + ci];
+  }
+}
+
+}  // namespace tc
+}  // namespace fdg

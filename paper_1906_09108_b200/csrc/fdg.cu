@@ -24,7 +24,8 @@
 #include <vector>
 
 #include "../../include/fdg.h"
-#include "conv_simt.cuh"
+#include "../../include/fdg_ops.h"
+#include "conv_dispatch.cuh"
 #include "elementwise.cuh"
 
 namespace fdg {
@@ -35,6 +36,14 @@ constexpr int kMailRing = 3;
 constexpr size_t kLogIterations = 4096;
 
 enum UnitType { U_STEM, U_BASIC, U_PREACT, U_HEAD };
+
+// Kernel classes for the optional per-launch profiler (fdg_profile_enable).
+enum KClass { KC_CONV_FPROP, KC_CONV_DGRAD, KC_CONV_WGRAD, KC_BN_STATS, KC_BN_APPLY, KC_BN_BWD_REDUCE,
+              KC_BN_BWD_APPLY, KC_HEAD, KC_SGD, KC_SHRINK, KC_INGEST, KC_COUNT };
+static const char* const kClassNames[KC_COUNT] = {"conv_fprop", "conv_dgrad", "conv_wgrad", "bn_stats", "bn_apply",
+                                                  "bn_bwd_reduce", "bn_bwd_apply", "head", "sgd", "shrink", "ingest"};
+constexpr size_t kProfMaxPairs = 1 << 16;
+struct ProfRec { int cls; double bytes, flops; };
 
 struct Unit {
   UnitType type;
@@ -49,6 +58,8 @@ struct Unit {
   size_t t_a, t_b, t_c, t_y, t_s;
   // offsets (floats) of saved statistics inside the slot's fp32 region
   size_t st1, st2, sts;
+  // offsets of the flipped copies of w1 / w2 inside a wflip16 slot, or -1 when that conv's dgrad is not on tensor cores
+  long long f1 = -1, f2 = -1;
 };
 
 struct Module {
@@ -67,6 +78,10 @@ struct Module {
   // device pointers
   float *theta = nullptr, *mom = nullptr, *grad = nullptr, *wver = nullptr;
   bf16* wver16 = nullptr;
+  bf16* wflip16 = nullptr;                 // Dw copies of the flipped/transposed 3x3 weights (dgrad operands)
+  size_t flip_elems = 0;
+  std::vector<tc::FlipEntry> flip_table;   // host copy; src = offset in a wver16 slot, dst = offset in a wflip16 slot
+  tc::FlipEntry* flip_table_dev = nullptr;
   char* fifo = nullptr;                    // D slots of slot_elems*sizeof(T)
   float* fifo_f = nullptr;                 // D slots of slot_floats
   char* in_ring = nullptr;                 // module 1: Din image slots
@@ -103,6 +118,8 @@ struct fdg_ctx {
   int label_ring = 0;
   int* flags = nullptr;               // [0] non-finite loss, [1] label out of range
   float* staging = nullptr;           // fp32 staging for getters
+  float* host_images = nullptr;       // device staging of fdg_step_host
+  int32_t* host_labels = nullptr;
   size_t staging_elems = 0;
   int64_t t = 0;
   float lr = 0.f;
@@ -111,8 +128,14 @@ struct fdg_ctx {
   mutable std::string err;
   fdg_status latched = FDG_OK;
   int device = 0;
+  fdg::TensorMapCache tmaps;
+  int* tc_error = nullptr;            // device word raised by a tensor-core kernel whose wait timed out
   cudaStream_t last_stream = nullptr;   // stream of the most recent fdg_step
   bool stepped = false;
+  // profiler
+  bool profiling = false;
+  std::vector<cudaEvent_t> prof_events;     // 2 per recorded launch
+  std::vector<fdg::ProfRec> prof_recs;
 };
 
 namespace fdg {
@@ -284,6 +307,24 @@ static void plan_modules(fdg_ctx* c) {
           break;
       }
     }
+    if (c->bf16_mode) {
+      size_t fe = 0;
+      auto flip = [&](size_t src, int co, int ci) {
+        tc::FlipEntry e; e.src = src; e.dst = fe; e.Co = co; e.Ci = ci;
+        m.flip_table.push_back(e);
+        long long off = (long long)fe;
+        fe += align_up((size_t)co * 9 * ci, 64);
+        return off;
+      };
+      for (Unit& u : m.units) {
+        if (u.type != U_BASIC && u.type != U_PREACT) continue;
+        ConvGeom g1{a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 3, u.stride, 1};
+        ConvGeom g2{a.batch, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 3, 1, 1};
+        if (tc_eligible(g1)) u.f1 = flip(u.w1, u.co, u.ci);
+        if (tc_eligible(g2)) u.f2 = flip(u.w2, u.co, u.co);
+      }
+      m.flip_elems = fe;
+    }
     m.slot_elems = te; m.slot_floats = tf; m.max_act = maxa; m.scratch_floats = scr;
     const Unit& last = m.units.back();
     if (kp < K) { m.out_elems = B * last.P * last.Q * last.co; m.out_c = last.co; }
@@ -297,6 +338,7 @@ static size_t carve(fdg_ctx* c, char* base) {
   Carver cv(base);
   const size_t es = c->esize;
   c->flags = cv.take<int>(256);
+  c->tc_error = c->flags ? c->flags + 2 : nullptr;
   c->label_ring = 2 * c->K + 2;
   c->labels = cv.take<int32_t>((size_t)c->label_ring * c->arch.batch * sizeof(int32_t));
   size_t stage = 0;
@@ -306,6 +348,8 @@ static size_t carve(fdg_ctx* c, char* base) {
     m.grad = cv.take<float>(m.n_params * 4);
     m.wver = cv.take<float>((size_t)m.Dw * align_up(m.n_params, 64) * 4);
     m.wver16 = c->bf16_mode ? cv.take<bf16>((size_t)m.Dw * align_up(m.n_params, 64) * 2) : nullptr;
+    m.wflip16 = m.flip_elems ? cv.take<bf16>((size_t)m.Dw * m.flip_elems * 2) : nullptr;
+    m.flip_table_dev = m.flip_table.empty() ? nullptr : cv.take<tc::FlipEntry>(m.flip_table.size() * sizeof(tc::FlipEntry));
     m.fifo = cv.take<char>((size_t)m.D * m.slot_elems * es);
     m.fifo_f = cv.take<float>((size_t)m.D * std::max<size_t>(m.slot_floats, 64) * 4);
     m.in_ring = m.Din ? cv.take<char>((size_t)m.Din * align_up(m.in_elems, 128) * es) : nullptr;
@@ -325,6 +369,8 @@ static size_t carve(fdg_ctx* c, char* base) {
     }
     stage = std::max(stage, std::max(m.in_elems, m.out_elems));
   }
+  c->host_images = cv.take<float>((size_t)c->arch.batch * c->arch.in_h * c->arch.in_w * c->arch.in_c * 4);
+  c->host_labels = cv.take<int32_t>((size_t)c->arch.batch * 4);
   c->staging_elems = stage;
   c->staging = cv.take<float>(stage * 4);
   return align_up(cv.off, 256);
@@ -335,8 +381,28 @@ struct Launch {
   fdg_ctx* c;
   cudaStream_t st;
   cudaError_t err = cudaSuccess;
-  void check() { if (err == cudaSuccess) err = cudaGetLastError(); ++c->launches; }
-  void note(cudaError_t e) { if (err == cudaSuccess) err = e; }
+  int open_pair = -1;
+  // begin/check bracket one kernel (or one kernel plus its fixed-order reduction): `bytes` and
+  // `flops` are the algorithmic traffic and arithmetic of the launch, for roofline reports.
+  void begin(int cls, double bytes, double flops) {
+    open_pair = -1;
+    if (!c->profiling || c->prof_recs.size() >= kProfMaxPairs) return;
+    const size_t i = c->prof_recs.size();
+    while (c->prof_events.size() < 2 * (i + 1)) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return;
+      c->prof_events.push_back(e);
+    }
+    c->prof_recs.push_back(ProfRec{cls, bytes, flops});
+    open_pair = (int)i;
+    cudaEventRecord(c->prof_events[2 * i], st);
+  }
+  void end_events() {
+    if (open_pair >= 0) cudaEventRecord(c->prof_events[2 * open_pair + 1], st);
+    open_pair = -1;
+  }
+  void check() { if (err == cudaSuccess) err = cudaGetLastError(); ++c->launches; end_events(); }
+  void note(cudaError_t e) { if (err == cudaSuccess) err = e; end_events(); }
 };
 
 static int ew_blocks(size_t nvec) {
@@ -349,6 +415,7 @@ template <typename T> constexpr int full_vec() { return 16 / sizeof(T); }
 template <typename T>
 static void bn_stats(Launch& L, Module& m, const T* x, size_t rows, int C, float eps, float* stats) {
   constexpr int V = full_vec<T>();
+  L.begin(KC_BN_STATS, (double)rows * C * sizeof(T), 3.0 * rows * C);
   if (C % V == 0) {
     RedGeom g = red_geom((int)rows, C, V);
     bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)g.rp * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
@@ -365,6 +432,7 @@ static void bn_apply(Launch& L, const T* x, const float* stats, const float* gam
                      size_t rows, int C) {
   constexpr int V = full_vec<T>();
   const size_t n = rows * C;
+  L.begin(KC_BN_APPLY, (double)n * sizeof(T) * (res ? 3 : 2), 6.0 * n);
   if (C % V == 0)
     bn_apply_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C);
   else
@@ -387,12 +455,14 @@ static void bn_backward(Launch& L, Module& m, const T* dy, const T* mask, const 
   const size_t smem = (size_t)g.rp * ns * C * 4;
 #define FDG_RED(VV, NS) bn_bwd_reduce_kernel<T, VV, NS><<<g.blocks, kRedThreads, smem, L.st>>>( \
       dy, mask, x, stats, x2, stats2, g, m.bnsums, dgamma, dbeta, dgamma2, dbeta2, m.scratch, m.counter)
+  L.begin(KC_BN_BWD_REDUCE, (double)rows * C * sizeof(T) * (2 + (mask ? 1 : 0) + (two ? 1 : 0)), 8.0 * rows * C);
   if (vec) { if (two) FDG_RED(V, 3); else FDG_RED(V, 2); }
   else     { if (two) FDG_RED(1, 3); else FDG_RED(1, 2); }
 #undef FDG_RED
   L.check();
   const size_t n = rows * C;
   const float inv_m = 1.f / (float)rows;
+  L.begin(KC_BN_BWD_APPLY, (double)n * sizeof(T) * (3 + (mask ? 1 : 0) + (two ? 2 : 0) + (res ? 1 : 0)), 10.0 * n);
   if (vec)
     bn_bwd_apply_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n / V, C, inv_m);
   else
@@ -403,6 +473,7 @@ static void bn_backward(Launch& L, Module& m, const T* dy, const T* mask, const 
 template <typename T>
 static void scale_tensor(Launch& L, const T* in, T* out, float s, size_t n) {
   constexpr int V = full_vec<T>();
+  L.begin(KC_SHRINK, 2.0 * n * sizeof(T), (double)n);
   if (n % V == 0) scale_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(in, out, s, n / V);
   else scale_kernel<T, 1><<<ew_blocks(n), 256, 0, L.st>>>(in, out, s, n);
   L.check();
@@ -416,17 +487,47 @@ static ConvGeom geom(int N, int H, int W, int Ci, int P, int Q, int Co, int R, i
   return ConvGeom{N, H, W, Ci, P, Q, Co, R, R, stride, pad};
 }
 
+static double conv_flops(const ConvGeom& g) { return 2.0 * g.N * g.P * g.Q * g.Co * (double)g.R * g.S * g.Ci; }
+static double in_elems(const ConvGeom& g) { return (double)g.N * g.H * g.W * g.Ci; }
+static double out_elems(const ConvGeom& g) { return (double)g.N * g.P * g.Q * g.Co; }
+static double w_elems(const ConvGeom& g) { return (double)g.Co * g.R * g.S * g.Ci; }
+
 template <typename T>
 static void conv_fprop(Launch& L, const ConvGeom& g, const T* x, const T* w, T* y, const T* res) {
+  L.begin(KC_CONV_FPROP, (in_elems(g) + w_elems(g) + out_elems(g) * (res ? 2 : 1)) * sizeof(T), conv_flops(g));
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (tc_eligible(g)) {
+      ++L.c->launches;
+      L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error));
+      return;
+    }
+  }
   L.note(launch_conv_simt<T, CONV_FPROP>(L.st, g, x, w, y, nullptr, nullptr, res, (const T*)nullptr, &L.c->launches));
 }
+// `wflip` is the flipped/transposed weight copy (bf16 mode, tensor-core eligible shapes) or null.
 template <typename T>
-static void conv_dgrad(Launch& L, const ConvGeom& g, const T* dy, const T* w, T* dx, const T* res, const T* mask) {
+static void conv_dgrad(Launch& L, const ConvGeom& g, const T* dy, const T* w, const T* wflip, T* dx, const T* res,
+                       const T* mask) {
+  L.begin(KC_CONV_DGRAD, (out_elems(g) + w_elems(g) + in_elems(g) * (1 + (res ? 1 : 0) + (mask ? 1 : 0))) * sizeof(T), conv_flops(g));
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (wflip && tc_eligible(g)) {
+      ++L.c->launches;
+      L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error));
+      return;
+    }
+  }
   L.note(launch_conv_simt<T, CONV_DGRAD>(L.st, g, dy, w, dx, nullptr, nullptr, res, mask, &L.c->launches));
 }
 template <typename T>
 static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* dy, float* dw) {
+  L.begin(KC_CONV_WGRAD, (in_elems(g) + out_elems(g)) * sizeof(T) + w_elems(g) * 4, conv_flops(g));
   L.note(launch_conv_simt<T, CONV_WGRAD>(L.st, g, x, dy, (T*)nullptr, m.scratch, dw, (const T*)nullptr, (const T*)nullptr, &L.c->launches));
+}
+
+template <typename T> static const T* flipped_of(const Module& m, int vslot, long long off);
+template <> const float* flipped_of<float>(const Module&, int, long long) { return nullptr; }
+template <> const bf16* flipped_of<bf16>(const Module& m, int vslot, long long off) {
+  return off < 0 ? nullptr : m.wflip16 + (size_t)vslot * m.flip_elems + off;
 }
 
 // ------------------------------------------------------------ module passes ---
@@ -527,9 +628,11 @@ static void head_forward_backward(fdg_ctx* c, Module& m, Launch& L, int64_t tau,
   const int32_t* labels = c->labels + (size_t)(tau % c->label_ring) * B;
   T* dfeat = u.bn ? reinterpret_cast<T*>(m.temps[2]) : gout;
   const size_t smem = (size_t)(2 * F + classes) * 4;
+  L.begin(KC_HEAD, 2.0 * rows * F * sizeof(T), 4.0 * B * F * classes);
   head_fwd_bwd_kernel<T><<<B, 128, smem, L.st>>>(feat, wf + u.w1, wf + u.w2, labels, HW, F, classes, B, m.pooled,
                                                   m.dlogits, m.loss_n, dfeat, c->flags + 1);
   L.check();
+  L.begin(KC_HEAD, 4.0 * B * (F + classes) + 4.0 * classes * F, 2.0 * B * F * classes);
   head_param_grad_kernel<<<classes, 128, 0, L.st>>>(m.pooled, m.dlogits, m.loss_n, F, classes, B, m.grad + u.w1,
                                                      m.grad + u.w2, m.loss, c->flags);
   L.check();
@@ -582,7 +685,7 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_c, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
                          nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co);
         conv_wgrad<T>(L, m, g2, S + u.t_b, T1, m.grad + u.w2);
-        conv_dgrad<T>(L, g2, T1, wt + u.w2, T3, nullptr, nullptr);                                     // da1
+        conv_dgrad<T>(L, g2, T1, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T3, nullptr, nullptr);      // da1
         bn_backward<T>(L, m, T3, S + u.t_b, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
                        nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co);      // dc1
         conv_wgrad<T>(L, m, g1, x, T1, m.grad + u.w1);
@@ -591,11 +694,11 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_wgrad<T>(L, m, gs, x, T2, m.grad + u.ws);
           if (need_dx) {
-            conv_dgrad<T>(L, gs, T2, wt + u.ws, T3, nullptr, nullptr);
-            conv_dgrad<T>(L, g1, T1, wt + u.w1, gout, T3, nullptr);
+            conv_dgrad<T>(L, gs, T2, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
+            conv_dgrad<T>(L, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr);
           }
         } else if (need_dx) {
-          conv_dgrad<T>(L, g1, T1, wt + u.w1, gout, dy, S + u.t_y);
+          conv_dgrad<T>(L, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y);
         }
         break;
       }
@@ -603,17 +706,17 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
         conv_wgrad<T>(L, m, g2, S + u.t_c, dy, m.grad + u.w2);
-        conv_dgrad<T>(L, g2, dy, wt + u.w2, T1, nullptr, nullptr);                                     // da2
+        conv_dgrad<T>(L, g2, dy, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T1, nullptr, nullptr);      // da2
         bn_backward<T>(L, m, T1, S + u.t_c, S + u.t_b, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
                        nullptr, nullptr, nullptr, nullptr, nullptr, T2, nullptr, rows_out, u.co);      // dc1
         conv_wgrad<T>(L, m, g1, S + u.t_a, T2, m.grad + u.w1);
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_wgrad<T>(L, m, gs, S + u.t_a, dy, m.grad + u.ws);
-          conv_dgrad<T>(L, gs, dy, wt + u.ws, T3, nullptr, nullptr);
-          conv_dgrad<T>(L, g1, T2, wt + u.w1, T1, T3, nullptr);                                        // do
+          conv_dgrad<T>(L, gs, dy, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
+          conv_dgrad<T>(L, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, T3, nullptr);         // do
         } else {
-          conv_dgrad<T>(L, g1, T2, wt + u.w1, T1, nullptr, nullptr);
+          conv_dgrad<T>(L, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, nullptr, nullptr);
         }
         bn_backward<T>(L, m, T1, S + u.t_a, x, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr, nullptr,
                        nullptr, nullptr, nullptr, u.proj ? nullptr : dy, gout, nullptr, rows_in, u.ci);
@@ -631,8 +734,14 @@ static void update_module(fdg_ctx* c, Module& m, Launch& L, int next_vslot) {
   float* next32 = m.wver + (size_t)next_vslot * align_up(n, 64);
   bf16* next16 = c->bf16_mode ? m.wver16 + (size_t)next_vslot * align_up(n, 64) : nullptr;
   int blocks = (int)std::min<size_t>(std::max<size_t>((n / 4 + 255) / 256, 1), 148 * 8);
+  L.begin(KC_SGD, (double)n * (24 + (next16 ? 2 : 0)), 6.0 * n);
   sgd_kernel<<<blocks, 256, 0, L.st>>>(m.theta, m.mom, m.grad, next32, next16, n, c->lr, c->cfg.momentum, c->cfg.weight_decay);
   L.check();
+  if (m.flip_table_dev) {
+    L.begin(KC_SGD, 4.0 * m.flip_elems, 0.0);
+    tc::wflip_kernel<<<dim3(8, (unsigned)m.flip_table.size()), 256, 0, L.st>>>(next16, m.wflip16 + (size_t)next_vslot * m.flip_elems, m.flip_table_dev);
+    L.check();
+  }
 }
 
 // One module-step of module m in iteration t (Algorithm I, body of "Parallel for k").
@@ -789,6 +898,9 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) { delete c; return FDG_ERR_CUDA; }
   carve(c, static_cast<char*>(dev_workspace));
+  for (Module& m : c->mods)
+    if (m.flip_table_dev && e == cudaSuccess)
+      e = cudaMemcpy(m.flip_table_dev, m.flip_table.data(), m.flip_table.size() * sizeof(tc::FlipEntry), cudaMemcpyHostToDevice);
   c->own_streams = streams == nullptr;
   for (int k = 0; k < c->K && e == cudaSuccess; ++k) {
     Module& m = c->mods[k];
@@ -815,6 +927,7 @@ fdg_status fdg_destroy(fdg_ctx* c) {
   }
   for (int i = 0; i < kEventRing; ++i) cudaEventDestroy(c->ev_in[i]);
   cudaEventDestroy(c->ev_join);
+  for (cudaEvent_t ev : c->prof_events) cudaEventDestroy(ev);
   delete c;
   return e == cudaSuccess ? FDG_OK : FDG_ERR_CUDA;
 }
@@ -854,6 +967,12 @@ static fdg_status copy_vec(fdg_ctx* c, int module, float* dev_vec, const float* 
         cast_kernel<bf16><<<(int)std::min<size_t>((n + 255) / 256, 1184), 256, 0, m.stream>>>(m.theta, m.wver16 + (size_t)v * align_up(n, 64), n);
         ++c->launches;
         e = cudaGetLastError();
+        if (e == cudaSuccess && m.flip_table_dev) {
+          tc::wflip_kernel<<<dim3(8, (unsigned)m.flip_table.size()), 256, 0, m.stream>>>(
+              m.wver16 + (size_t)v * align_up(n, 64), m.wflip16 + (size_t)v * m.flip_elems, m.flip_table_dev);
+          ++c->launches;
+          e = cudaGetLastError();
+        }
       }
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(m.stream);
@@ -913,12 +1032,14 @@ fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, cons
     int32_t* lab = c->labels + (size_t)(t % c->label_ring) * c->arch.batch;
     const size_t slot_off = (size_t)(t % m1.Din) * align_up(m1.in_elems, 128);
     const int blocks = ew_blocks(rows * m1.in_c);
+    Launch L{c, cs};
+    L.begin(KC_INGEST, (double)rows * (c->arch.in_c * 4 + m1.in_c * c->esize), 0.0);
     if (c->bf16_mode)
       ingest_kernel<bf16><<<blocks, 256, 0, cs>>>(images_dev, reinterpret_cast<bf16*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch);
     else
       ingest_kernel<float><<<blocks, 256, 0, cs>>>(images_dev, reinterpret_cast<float*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch);
-    ++c->launches;
-    e = cudaGetLastError();
+    L.check();
+    e = L.err;
     if (e == cudaSuccess && !serial) e = cudaEventRecord(c->ev_in[t % kEventRing], cs);
     if (e != cudaSuccess) return cuda_fail(c, e, "ingest");
   }
@@ -927,6 +1048,26 @@ fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, cons
     cudaStream_t st = serial ? cs : m.stream;
     e = c->bf16_mode ? module_step<bf16>(c, m, st, serial, loss_dev) : module_step<float>(c, m, st, serial, loss_dev);
     if (e != cudaSuccess) return cuda_fail(c, e, "module step");
+  }
+  return FDG_OK;
+}
+
+fdg_status fdg_step_host(fdg_ctx* c, fdg_stream stream, const float* images_host, const int32_t* labels_host,
+                         float* loss_host) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (!images_host || !labels_host) return fail(c, FDG_ERR_INVALID_ARG, "images and labels must not be null");
+  if (c->latched != FDG_OK) return c->latched;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const size_t img_bytes = (size_t)c->arch.batch * c->arch.in_h * c->arch.in_w * c->arch.in_c * 4;
+  cudaError_t e = cudaMemcpyAsync(c->host_images, images_host, img_bytes, cudaMemcpyHostToDevice, cs);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->host_labels, labels_host, (size_t)c->arch.batch * 4, cudaMemcpyHostToDevice, cs);
+  if (e != cudaSuccess) return cuda_fail(c, e, "host to device copy");
+  fdg_status s = fdg_step(c, stream, c->host_images, c->host_labels, nullptr);
+  if (s != FDG_OK) return s;
+  if (loss_host && c->t >= c->K) {
+    Module& mk = c->mods[c->K - 1];
+    e = cudaMemcpyAsync(loss_host, mk.loss, sizeof(float), cudaMemcpyDeviceToHost, c->cfg.serial ? cs : mk.stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "loss copy");
   }
   return FDG_OK;
 }
@@ -941,11 +1082,12 @@ fdg_status fdg_sync(fdg_ctx* c, fdg_stream stream) {
       if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, c->ev_join, 0);
     }
   if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
-  int flags[2] = {0, 0};
+  int flags[3] = {0, 0, 0};
   if (e == cudaSuccess) e = cudaMemcpy(flags, c->flags, sizeof(flags), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(c, e, "sync");
-  if (flags[0] || flags[1]) {
+  if (flags[0] || flags[1] || flags[2]) {
     cudaMemset(c->flags, 0, sizeof(flags));
+    if (flags[2]) { c->latched = FDG_ERR_TIMEOUT; return fail(c, FDG_ERR_TIMEOUT, "a tensor-core kernel gave up waiting on a barrier"); }
     if (flags[1]) return fail(c, FDG_ERR_INVALID_ARG, "a label was outside [0, num_classes)");
     return fail(c, FDG_ERR_NONFINITE, "a loss computed since the last sync was NaN or Inf");
   }
@@ -1004,6 +1146,36 @@ fdg_status fdg_get_schedule_log(const fdg_ctx* c, fdg_sched_entry* dst, size_t c
   return FDG_OK;
 }
 
+fdg_status fdg_profile_enable(fdg_ctx* c, int on) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  c->profiling = on != 0;
+  c->prof_recs.clear();
+  return FDG_OK;
+}
+
+fdg_status fdg_profile_read(fdg_ctx* c, fdg_kernel_stat* dst, size_t cap, size_t* out_n) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  fdg_kernel_stat agg[KC_COUNT];
+  for (int i = 0; i < KC_COUNT; ++i) {
+    std::memset(&agg[i], 0, sizeof(agg[i]));
+    std::snprintf(agg[i].name, sizeof(agg[i].name), "%s", kClassNames[i]);
+  }
+  for (size_t i = 0; i < c->prof_recs.size(); ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof_events[2 * i], c->prof_events[2 * i + 1]) != cudaSuccess) continue;
+    fdg_kernel_stat& a = agg[c->prof_recs[i].cls];
+    a.launches += 1; a.total_ms += ms; a.bytes += c->prof_recs[i].bytes; a.flops += c->prof_recs[i].flops;
+  }
+  c->prof_recs.clear();
+  if (out_n) *out_n = KC_COUNT;
+  if (dst) for (size_t i = 0; i < std::min<size_t>(cap, KC_COUNT); ++i) dst[i] = agg[i];
+  return FDG_OK;
+}
+
 fdg_status fdg_launch_count(const fdg_ctx* c, uint64_t* out_n) {
   if (!c || !out_n) return FDG_ERR_INVALID_ARG;
   *out_n = c->launches;
@@ -1011,3 +1183,5 @@ fdg_status fdg_launch_count(const fdg_ctx* c, uint64_t* out_n) {
 }
 
 }  // extern "C"
+
+#include "ops_api.inc"

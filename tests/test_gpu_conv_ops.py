@@ -1,0 +1,84 @@
+"""Operator-level parity: fdg_conv_forward / dgrad / wgrad through the C ABI against the
+oracle's convolution (oracle/layers.py), element by element.  bf16 cases feed both sides
+the same bf16-rounded inputs; the oracle then works in float64, so the only differences
+are fp32 accumulation order and the final rounding of the output to bf16 (2^-9 relative)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import layers as L
+
+pytestmark = pytest.mark.gpu
+
+
+def _mk(shape, seed, dtype):
+    g = np.random.default_rng(seed)
+    a = g.standard_normal(shape).astype(np.float32)
+    t = torch.from_numpy(a).cuda().to(dtype)
+    return t, t.float().cpu().numpy().astype(np.float64)
+
+
+def _rel(a, b):
+    return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-30))
+
+
+# (N, H, W, Ci, Co, R, stride, pad)
+SHAPES_ANY = [(3, 12, 20, 5, 7, 3, 1, 1), (2, 16, 16, 8, 16, 3, 2, 1), (2, 16, 16, 16, 32, 1, 2, 0),
+              (5, 8, 8, 3, 8, 3, 1, 1)]
+SHAPES_TC = [(4, 32, 32, 16, 16, 3, 1, 1),      # 32 tiles of 4 image rows, 32-byte swizzle
+             (6, 16, 16, 32, 32, 3, 1, 1),      # 8 rows per tile, 64-byte swizzle
+             (10, 8, 8, 64, 64, 3, 1, 1),       # two images per tile, 128-byte swizzle
+             (2, 32, 32, 16, 48, 3, 1, 1),      # c_in != c_out
+             (2, 16, 16, 128, 160, 3, 1, 1),    # two channel chunks, wide N
+             (300, 8, 8, 64, 64, 3, 1, 1)]      # more tiles than SMs: several tiles per CTA
+
+
+def _run(prec_name, shape, expect_tc):
+    from paper_1906_09108_b200 import binding as B
+    prec = B.FDG_BF16_TC if prec_name == "bf16" else B.FDG_FP32_CUDACORE
+    ops = B.ConvOps(prec)
+    n, h, w, ci, co, r, st, pad = shape
+    s = B.fdg_conv_shape(n, h, w, ci, co, r, st, pad)
+    p, q = ops.out_hw(s)
+    x, xo = _mk((n, h, w, ci), 1, ops.dtype)
+    wt, wo = _mk((co, r, r, ci), 2, ops.dtype)
+    dy, dyo = _mk((n, p, q, co), 3, ops.dtype)
+    res, reso = _mk((n, h, w, ci), 4, ops.dtype)
+    mask, masko = _mk((n, h, w, ci), 5, ops.dtype)
+    resy, resyo = _mk((n, p, q, co), 6, ops.dtype)
+    tol = 1e-2 if prec_name == "bf16" else 2e-5
+    assert ops.path(s, 0) == expect_tc
+
+    y = ops.forward(s, x, wt).float().cpu().numpy()
+    assert _rel(y, L.conv2d_forward(xo, wo, st, pad)) < tol
+    y = ops.forward(s, x, wt, res=resy).float().cpu().numpy()
+    assert _rel(y, L.conv2d_forward(xo, wo, st, pad) + resyo) < tol
+
+    dxo, dwo = L.conv2d_backward(dyo, xo, wo, st, pad)
+    wf = ops.flip_weights(s, wt) if (prec_name == "bf16" and r == 3) else None
+    dx = ops.dgrad(s, dy, wt, wf).float().cpu().numpy()
+    assert _rel(dx, dxo) < tol
+    dx = ops.dgrad(s, dy, wt, wf, res=res, res_mask=mask).float().cpu().numpy()
+    assert _rel(dx, dxo + reso * (masko > 0)) < tol
+    if wf is not None:          # the CUDA-core path of the same call must agree as well
+        dx = ops.dgrad(s, dy, wt, None).float().cpu().numpy()
+        assert _rel(dx, dxo) < tol
+
+    dw = ops.wgrad(s, x, dy).cpu().numpy()
+    assert _rel(dw, dwo) < (1e-3 if prec_name == "bf16" else 2e-5)
+    assert not ops.timed_out()
+
+
+@pytest.mark.parametrize("shape", SHAPES_ANY + SHAPES_TC[:3])
+def test_conv_ops_fp32(shape):
+    _run("fp32", shape, False)
+
+
+@pytest.mark.parametrize("shape", SHAPES_ANY)
+def test_conv_ops_bf16_cuda_core_shapes(shape):
+    _run("bf16", shape, False)
+
+
+@pytest.mark.parametrize("shape", SHAPES_TC)
+def test_conv_ops_bf16_tensor_core_shapes(shape):
+    _run("bf16", shape, True)
