@@ -198,6 +198,20 @@ fdg_status fdg_get_input_grad(fdg_ctx* ctx, int module, float* dst, size_t n, in
 /* Element counts of those two tensors: the output of module k (0 for k = K) and its input. */
 fdg_status fdg_boundary_elems(const fdg_ctx* ctx, int module, size_t* out_elems, size_t* in_elems);
 
+/* Inspection of the activation FIFO: copies one tensor the forward of module `module`
+ * saved for its most recent batch, as fp32 NHWC, to host or device memory.  `unit` is the
+ * position of the stem/block inside the module (0-based); `which` selects the tensor:
+ *   FDG_RESNET_6N2 block: 0 = conv1 output, 1 = ReLU(BN1(.)), 2 = conv2 output, 3 = block output,
+ *                         4 = projection-shortcut convolution output (projection blocks only);
+ *   FDG_RESNET_6N2 stem:  0 = convolution output, 3 = stem output;
+ *   FDG_WRN block:        0 = ReLU(BN1(input)), 1 = conv1 output, 2 = ReLU(BN2(.)), 3 = block output;
+ *   FDG_WRN stem:         3 = stem output.
+ * `n` must equal the tensor's element count, which is written to *out_elems when `dst` is NULL.
+ * *batch_index receives the batch the slot holds, or -1 (nothing copied) before the first
+ * forward.  Blocks the host.  Errors: FDG_ERR_INVALID_ARG (bad module/unit/which/n). */
+fdg_status fdg_get_saved_tensor(fdg_ctx* ctx, int module, int unit, int which, float* dst, size_t n,
+                                size_t* out_elems, int64_t* batch_index);
+
 /* Copies at most `cap` rows of the schedule log (oldest first) and writes the number
  * of rows recorded so far to *out_n.  The log keeps every row of the last 4096 iterations. */
 fdg_status fdg_get_schedule_log(const fdg_ctx* ctx, fdg_sched_entry* dst, size_t cap, size_t* out_n);

@@ -22,6 +22,31 @@ import numpy as np
 
 
 # ----------------------------------------------------------------------------
+# storage precision
+# ----------------------------------------------------------------------------
+def round_bf16(a):
+    """Rounds every element to the nearest bfloat16 (8 exponent bits, 7 stored mantissa
+    bits; ties to even) and returns it in the dtype it came in.
+
+    The paper fixes no precision.  Where a tensor is held in bfloat16 between two
+    steps of the path, the decisions taken on it (the sign test of a ReLU gate)
+    depend on that rounding, so the oracle can reproduce it: bfloat16 is the upper
+    half of an IEEE float32 word, and rounding adds half a unit of the dropped
+    half (plus the tie-break bit) before truncating.  Pin: agreement with
+    torch.Tensor.to(torch.bfloat16) on random and boundary values.
+    """
+    a = np.asarray(a)
+    bits = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    keep = (bits >> np.uint32(16)) & np.uint32(1)
+    bits = (bits + np.uint32(0x7FFF) + keep) & np.uint32(0xFFFF0000)
+    return bits.view(np.float32).astype(a.dtype).reshape(a.shape)
+
+
+def identity(a):
+    return a
+
+
+# ----------------------------------------------------------------------------
 # convolution (cross-correlation, zero padding, no bias)
 # ----------------------------------------------------------------------------
 def conv_out_size(n, r, stride, pad):

@@ -21,6 +21,16 @@ networks it cites (Tables 3-6):
        sc = x, or conv1x1_s(o) when the shape changes;
        stem = conv3x3(image); head = ReLU(BN(.)) -> GAP -> FC -> softmax-CE.
 
+Storage precision.  Every unit carries two maps, `q` (applied to each activation or
+gradient tensor the path keeps between two of its steps) and `qw` (applied to
+convolution weights before they are used).  Both are the identity by default, which
+is the mathematics above and nothing else.  `set_storage(units, "bf16")` makes them
+round to bfloat16, reproducing a path that holds those tensors in bfloat16 while it
+accumulates, normalises and reduces in higher precision: the ReLU gates are then
+decided on the same rounded values on both sides.  Sums that are formed and consumed
+inside one step (a ReLU derivative times its incoming gradient, a residual sum before
+its ReLU) are not rounded.
+
 Parameter order inside a unit (and therefore inside a module's flat vector) is
 the order of `param_spec()`; convolution weights are [C_out, R, S, C_in].
 """
@@ -53,6 +63,7 @@ class Stem:
         self.ci, self.co, self.eps = arch.in_c, arch.stem_width, arch.bn_eps
         self.with_bn = arch.family == "resnet6n2"
         self.name = "stem"
+        self.q = self.qw = L.identity
 
     def param_spec(self):
         spec = [("conv.w", "conv", (self.co, 3, 3, self.ci))]
@@ -61,11 +72,12 @@ class Stem:
         return spec
 
     def forward(self, x, p):
-        c = L.conv2d_forward(x, p["conv.w"], 1, 1)
+        q = self.q
+        c = q(L.conv2d_forward(x, self.qw(p["conv.w"]), 1, 1))
         if not self.with_bn:
             return c, dict(x=x)
         b, sv = L.batchnorm_forward(c, p["bn.g"], p["bn.b"], self.eps)
-        y = L.relu_forward(b)
+        y = q(L.relu_forward(b))
         return y, dict(x=x, sv=sv, y=y)
 
     def backward(self, dy, ctx, p):
@@ -73,10 +85,11 @@ class Stem:
         if self.with_bn:
             db = L.relu_backward(dy, ctx["y"])
             dc, g["bn.g"], g["bn.b"] = L.batchnorm_backward(db, ctx["sv"], p["bn.g"])
+            dc = self.q(dc)
         else:
             dc = dy
-        dx, g["conv.w"] = L.conv2d_backward(dc, ctx["x"], p["conv.w"], 1, 1)
-        return dx, g
+        dx, g["conv.w"] = L.conv2d_backward(dc, ctx["x"], self.qw(p["conv.w"]), 1, 1)
+        return self.q(dx), g
 
 
 class BasicBlock:
@@ -86,6 +99,7 @@ class BasicBlock:
         self.ci, self.co, self.stride, self.eps = ci, co, stride, arch.bn_eps
         self.proj = (ci != co) or (stride != 1)
         self.name = "block%d" % index
+        self.q = self.qw = L.identity
 
     def param_spec(self):
         spec = [("conv1.w", "conv", (self.co, 3, 3, self.ci)),
@@ -98,36 +112,41 @@ class BasicBlock:
         return spec
 
     def forward(self, x, p):
-        c1 = L.conv2d_forward(x, p["conv1.w"], self.stride, 1)
+        q, qw = self.q, self.qw
+        c1 = q(L.conv2d_forward(x, qw(p["conv1.w"]), self.stride, 1))
         b1, sv1 = L.batchnorm_forward(c1, p["bn1.g"], p["bn1.b"], self.eps)
-        a1 = L.relu_forward(b1)
-        c2 = L.conv2d_forward(a1, p["conv2.w"], 1, 1)
+        a1 = q(L.relu_forward(b1))
+        c2 = q(L.conv2d_forward(a1, qw(p["conv2.w"]), 1, 1))
         b2, sv2 = L.batchnorm_forward(c2, p["bn2.g"], p["bn2.b"], self.eps)
         ctx = dict(x=x, sv1=sv1, a1=a1, sv2=sv2)
         if self.proj:
-            cs = L.conv2d_forward(x, p["sc.w"], self.stride, 0)
+            cs = q(L.conv2d_forward(x, qw(p["sc.w"]), self.stride, 0))
             sc, ctx["svs"] = L.batchnorm_forward(cs, p["scbn.g"], p["scbn.b"], self.eps)
         else:
             sc = x
-        y = L.relu_forward(b2 + sc)
+        y = q(L.relu_forward(b2 + sc))
         ctx["y"] = y
         return y, ctx
 
     def backward(self, dy, ctx, p):
         g = {}
+        q, qw = self.q, self.qw
         dsum = L.relu_backward(dy, ctx["y"])          # gradient of b2 + sc
         dc2, g["bn2.g"], g["bn2.b"] = L.batchnorm_backward(dsum, ctx["sv2"], p["bn2.g"])
-        da1, g["conv2.w"] = L.conv2d_backward(dc2, ctx["a1"], p["conv2.w"], 1, 1)
-        db1 = L.relu_backward(da1, ctx["a1"])
+        dc2 = q(dc2)
+        da1, g["conv2.w"] = L.conv2d_backward(dc2, ctx["a1"], qw(p["conv2.w"]), 1, 1)
+        db1 = L.relu_backward(q(da1), ctx["a1"])
         dc1, g["bn1.g"], g["bn1.b"] = L.batchnorm_backward(db1, ctx["sv1"], p["bn1.g"])
-        dx, g["conv1.w"] = L.conv2d_backward(dc1, ctx["x"], p["conv1.w"], self.stride, 1)
+        dc1 = q(dc1)
+        dx, g["conv1.w"] = L.conv2d_backward(dc1, ctx["x"], qw(p["conv1.w"]), self.stride, 1)
         if self.proj:
             dcs, g["scbn.g"], g["scbn.b"] = L.batchnorm_backward(dsum, ctx["svs"], p["scbn.g"])
-            dxs, g["sc.w"] = L.conv2d_backward(dcs, ctx["x"], p["sc.w"], self.stride, 0)
-            dx = dx + dxs
+            dcs = q(dcs)
+            dxs, g["sc.w"] = L.conv2d_backward(dcs, ctx["x"], qw(p["sc.w"]), self.stride, 0)
+            dx = dx + q(dxs)
         else:
             dx = dx + dsum
-        return dx, g
+        return q(dx), g
 
 
 class PreActBlock:
@@ -137,6 +156,7 @@ class PreActBlock:
         self.ci, self.co, self.stride, self.eps = ci, co, stride, arch.bn_eps
         self.proj = (ci != co) or (stride != 1)
         self.name = "block%d" % index
+        self.q = self.qw = L.identity
 
     def param_spec(self):
         spec = [("bn1.g", "bn_gamma", (self.ci,)), ("bn1.b", "bn_beta", (self.ci,)),
@@ -148,33 +168,36 @@ class PreActBlock:
         return spec
 
     def forward(self, x, p):
+        q, qw = self.q, self.qw
         b1, sv1 = L.batchnorm_forward(x, p["bn1.g"], p["bn1.b"], self.eps)
-        o = L.relu_forward(b1)
-        c1 = L.conv2d_forward(o, p["conv1.w"], self.stride, 1)
+        o = q(L.relu_forward(b1))
+        c1 = q(L.conv2d_forward(o, qw(p["conv1.w"]), self.stride, 1))
         b2, sv2 = L.batchnorm_forward(c1, p["bn2.g"], p["bn2.b"], self.eps)
-        a2 = L.relu_forward(b2)
-        c2 = L.conv2d_forward(a2, p["conv2.w"], 1, 1)
+        a2 = q(L.relu_forward(b2))
+        c2 = L.conv2d_forward(a2, qw(p["conv2.w"]), 1, 1)
         if self.proj:
-            sc = L.conv2d_forward(o, p["sc.w"], self.stride, 0)
+            sc = q(L.conv2d_forward(o, qw(p["sc.w"]), self.stride, 0))
         else:
             sc = x
-        y = c2 + sc
+        y = q(c2 + sc)
         return y, dict(sv1=sv1, o=o, sv2=sv2, a2=a2)
 
     def backward(self, dy, ctx, p):
         g = {}
-        da2, g["conv2.w"] = L.conv2d_backward(dy, ctx["a2"], p["conv2.w"], 1, 1)
-        db2 = L.relu_backward(da2, ctx["a2"])
+        q, qw = self.q, self.qw
+        da2, g["conv2.w"] = L.conv2d_backward(dy, ctx["a2"], qw(p["conv2.w"]), 1, 1)
+        db2 = L.relu_backward(q(da2), ctx["a2"])
         dc1, g["bn2.g"], g["bn2.b"] = L.batchnorm_backward(db2, ctx["sv2"], p["bn2.g"])
-        do, g["conv1.w"] = L.conv2d_backward(dc1, ctx["o"], p["conv1.w"], self.stride, 1)
+        dc1 = q(dc1)
+        do, g["conv1.w"] = L.conv2d_backward(dc1, ctx["o"], qw(p["conv1.w"]), self.stride, 1)
         if self.proj:
-            dos, g["sc.w"] = L.conv2d_backward(dy, ctx["o"], p["sc.w"], self.stride, 0)
-            do = do + dos
-        db1 = L.relu_backward(do, ctx["o"])
+            dos, g["sc.w"] = L.conv2d_backward(dy, ctx["o"], qw(p["sc.w"]), self.stride, 0)
+            do = do + q(dos)
+        db1 = L.relu_backward(q(do), ctx["o"])
         dx, g["bn1.g"], g["bn1.b"] = L.batchnorm_backward(db1, ctx["sv1"], p["bn1.g"])
         if not self.proj:
             dx = dx + dy
-        return dx, g
+        return q(dx), g
 
 
 class Head:
@@ -185,6 +208,7 @@ class Head:
         self.feat, self.classes, self.eps = feat, arch.num_classes, arch.bn_eps
         self.with_bn = arch.family == "wrn"
         self.name = "head"
+        self.q = self.qw = L.identity
 
     def param_spec(self):
         spec = []
@@ -197,7 +221,7 @@ class Head:
         ctx = dict(shape=x.shape)
         if self.with_bn:
             b, ctx["sv"] = L.batchnorm_forward(x, p["bn.g"], p["bn.b"], self.eps)
-            x = L.relu_forward(b)
+            x = self.q(L.relu_forward(b))
             ctx["a"] = x
         pooled = L.gap_forward(x)
         logits = L.fc_forward(pooled, p["fc.w"], p["fc.b"])
@@ -209,10 +233,11 @@ class Head:
         g = {}
         dlogits = L.softmax_xent_backward(ctx["probs"], ctx["labels"])
         dpooled, g["fc.w"], g["fc.b"] = L.fc_backward(dlogits, ctx["pooled"], p["fc.w"])
-        dx = L.gap_backward(dpooled, ctx["shape"])
+        dx = self.q(L.gap_backward(dpooled, ctx["shape"]))
         if self.with_bn:
             db = L.relu_backward(dx, ctx["a"])
             dx, g["bn.g"], g["bn.b"] = L.batchnorm_backward(db, ctx["sv"], p["bn.g"])
+            dx = self.q(dx)
         return dx, g
 
 
@@ -232,6 +257,15 @@ def build_units(arch):
             ci = arch.widths[stage]
     units.append(Head(arch, ci))
     return units
+
+
+def set_storage(units, storage):
+    """storage None: exact arithmetic in the working dtype.  "bf16": activations,
+    gradients and convolution weights are rounded to bfloat16 wherever they are kept."""
+    assert storage in (None, "bf16"), storage
+    f = L.round_bf16 if storage == "bf16" else L.identity
+    for u in units:
+        u.q = u.qw = f
 
 
 def split_units(units, split_after_block):

@@ -24,7 +24,7 @@ PARAM_KINDS = {0: "conv", 1: "bn_gamma", 2: "bn_beta", 3: "fc_w", 4: "fc_b"}
 EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count", "fdg_param_layout",
            "fdg_set_params", "fdg_set_momentum", "fdg_get_params", "fdg_get_grads", "fdg_get_momentum",
            "fdg_set_lr", "fdg_step", "fdg_step_host", "fdg_sync", "fdg_profile_enable", "fdg_profile_read", "fdg_get_module_output", "fdg_get_input_grad",
-           "fdg_boundary_elems", "fdg_get_schedule_log", "fdg_launch_count", "fdg_status_string",
+           "fdg_boundary_elems", "fdg_get_saved_tensor", "fdg_get_schedule_log", "fdg_launch_count", "fdg_status_string",
            "fdg_last_error", "fdg_conv_forward", "fdg_conv_dgrad", "fdg_conv_flip_weights",
            "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_path"]
 
@@ -87,6 +87,7 @@ def load_library(path=LIB_PATH):
         "fdg_get_module_output": [vp, C.c_int, vp, sz, P(i64)],
         "fdg_get_input_grad": [vp, C.c_int, vp, sz, P(i64)],
         "fdg_boundary_elems": [vp, C.c_int, P(sz), P(sz)],
+        "fdg_get_saved_tensor": [vp, C.c_int, C.c_int, C.c_int, vp, sz, P(sz), P(i64)],
         "fdg_get_schedule_log": [vp, P(fdg_sched_entry), sz, P(sz)],
         "fdg_launch_count": [vp, P(C.c_uint64)],
         "fdg_conv_forward": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, vp, vp],
@@ -253,6 +254,15 @@ class FDG:
         out = np.empty(n, dtype=np.float32)
         b = C.c_int64()
         self._check(self.lib.fdg_get_input_grad(self.ctx, k, out.ctypes.data, n, C.byref(b)), self.ctx)
+        return b.value, out
+
+    def saved_tensor(self, k, unit, which):
+        """(batch, flat fp32 array) of one tensor in module k's newest activation-FIFO slot."""
+        n, b = C.c_size_t(), C.c_int64()
+        self._check(self.lib.fdg_get_saved_tensor(self.ctx, k, unit, which, None, 0, C.byref(n), None), self.ctx)
+        out = np.empty(n.value, dtype=np.float32)
+        self._check(self.lib.fdg_get_saved_tensor(self.ctx, k, unit, which, out.ctypes.data, n.value, None,
+                                                  C.byref(b)), self.ctx)
         return b.value, out
 
     def schedule_log(self):

@@ -367,7 +367,7 @@ static size_t carve(fdg_ctx* c, char* base) {
       m.loss_n = cv.take<float>((size_t)c->arch.batch * 4);
       m.loss = cv.take<float>(256);
     }
-    stage = std::max(stage, std::max(m.in_elems, m.out_elems));
+    stage = std::max(stage, m.max_act);
   }
   c->host_images = cv.take<float>((size_t)c->arch.batch * c->arch.in_h * c->arch.in_w * c->arch.in_c * 4);
   c->host_labels = cv.take<int32_t>((size_t)c->arch.batch * 4);
@@ -1137,6 +1137,46 @@ fdg_status fdg_get_input_grad(fdg_ctx* c, int module, float* dst, size_t n, int6
   if (m.last_grad_batch < 0) return FDG_OK;
   const char* src = m.mail + (size_t)m.last_grad_slot * align_up(m.in_elems, 128) * c->esize;
   return export_tensor(c, src, (size_t)c->arch.batch * m.in_h * m.in_w, m.in_c, m.in_c_logical, dst, n);
+}
+
+fdg_status fdg_get_saved_tensor(fdg_ctx* c, int module, int unit, int which, float* dst, size_t n, size_t* out_elems,
+                                int64_t* batch_index) {
+  FDG_MODULE_OR_FAIL(c, module);
+  Module& m = c->mods[module - 1];
+  if (unit < 0 || unit >= (int)m.units.size() || m.units[unit].type == U_HEAD)
+    return fail(c, FDG_ERR_INVALID_ARG, "unit index out of range");
+  const Unit& u = m.units[unit];
+  const size_t B = c->arch.batch;
+  const size_t in_e = B * u.H * u.W * u.ci, out_e = B * u.P * u.Q * u.co;
+  size_t off = 0, elems = out_e;
+  int ch = u.co;
+  bool ok = false;
+  if (u.type == U_STEM) {
+    if (which == 0 && u.bn) { off = u.t_a; ok = true; }
+    if (which == 3) { off = u.t_y; ok = true; }
+  } else if (u.type == U_BASIC) {
+    if (which == 0) { off = u.t_a; ok = true; }
+    if (which == 1) { off = u.t_b; ok = true; }
+    if (which == 2) { off = u.t_c; ok = true; }
+    if (which == 3) { off = u.t_y; ok = true; }
+    if (which == 4 && u.proj) { off = u.t_s; ok = true; }
+  } else {
+    if (which == 0) { off = u.t_a; elems = in_e; ch = u.ci; ok = true; }
+    if (which == 1) { off = u.t_b; ok = true; }
+    if (which == 2) { off = u.t_c; ok = true; }
+    if (which == 3) { off = u.t_y; ok = true; }
+  }
+  if (!ok) return fail(c, FDG_ERR_INVALID_ARG, "this unit saves no such tensor");
+  if (out_elems) *out_elems = elems;
+  if (!dst) return FDG_OK;
+  if (!batch_index) return FDG_ERR_INVALID_ARG;
+  // most recent forward = the slot with the largest batch index
+  int slot = -1;
+  for (int i = 0; i < m.D; ++i) if (m.slot_batch[i] >= 0 && (slot < 0 || m.slot_batch[i] > m.slot_batch[slot])) slot = i;
+  *batch_index = slot < 0 ? -1 : m.slot_batch[slot];
+  if (slot < 0) return FDG_OK;
+  const char* src = m.fifo + ((size_t)slot * m.slot_elems + off) * c->esize;
+  return export_tensor(c, src, elems / ch, ch, ch, dst, n);
 }
 
 fdg_status fdg_get_schedule_log(const fdg_ctx* c, fdg_sched_entry* dst, size_t cap, size_t* out_n) {

@@ -26,7 +26,10 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
     arch_o = onets.Arch(**arch_kw)
     cfg_o = ofdg.FDGConfig(K=K, split_after_block=tuple(splits), beta=beta, lr=lr, momentum=momentum,
                            weight_decay=weight_decay, order=order, weight_reading=weight_reading)
-    orc = ofdg.FDGOracle(arch_o, cfg_o, dtype=oracle_dtype)
+    # In bf16 mode the library keeps activations, gradients and convolution weights in
+    # bfloat16; the oracle then rounds the same tensors, so that both sides decide every
+    # ReLU gate on the same values (everything else stays float64 in the oracle).
+    orc = ofdg.FDGOracle(arch_o, cfg_o, dtype=oracle_dtype, storage="bf16" if precision == "bf16" else None)
     g = B.FDG(B.make_arch(**arch_kw), K=K, split_after_block=tuple(splits), beta=beta, lr=lr, momentum=momentum,
               weight_decay=weight_decay,
               order=B.FDG_BACKWARD_FIRST if order == "backward_first" else B.FDG_FORWARD_FIRST,

@@ -114,3 +114,20 @@ def test_head_fd_and_torch():
     assert relerr(dx, fd_grad(f, x)) < 1e-7
     assert relerr(dw, fd_grad(f, w)) < 1e-7
     assert relerr(db, fd_grad(f, b)) < 1e-7
+
+
+def test_round_bf16_matches_torch():
+    """The oracle's bfloat16 rounding against torch's own conversion: random values over
+    many exponents, exact ties (round to even), values that round up into the next
+    binade, zeros and subnormals' neighbours."""
+    import torch
+    g = np.random.default_rng(7)
+    a = (g.standard_normal(200000) * np.exp(g.uniform(-30, 30, 200000))).astype(np.float32)
+    ties = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8), 1.0 + 2.0 ** -7 + 2.0 ** -8,
+                     2.0 - 2.0 ** -9, 0.0, -0.0, 1e-38, 3.0e38], dtype=np.float32)
+    a = np.concatenate([a, ties])
+    want = torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
+    got = L.round_bf16(a)
+    assert got.dtype == np.float32 and np.array_equal(got, want)
+    got64 = L.round_bf16(a.astype(np.float64))
+    assert got64.dtype == np.float64 and np.array_equal(got64.astype(np.float32), want)
