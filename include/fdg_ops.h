@@ -52,6 +52,26 @@ fdg_status fdg_conv_wgrad_scratch_bytes(int precision, const fdg_conv_shape* sha
 fdg_status fdg_conv_wgrad(int precision, const fdg_conv_shape* shape, const void* x, const void* dy, float* dw,
                           void* scratch, size_t scratch_bytes, int* status_dev, fdg_stream stream);
 
+/* fdg_conv_wgrad for callers that cannot hand over scratch memory.  The paper has no
+ * counterpart to this call; it exists for hosts of the library that are not allowed to
+ * allocate device memory at the point where they need a weight gradient: code running under a
+ * memory plan that was fixed up front, inside a stream-ordered region where cudaMalloc would
+ * synchronise the device, or behind an allocator they do not own.  Same arguments and result as
+ * fdg_conv_wgrad on the CUDA-core path, but the partial sums go to a buffer that is part of the
+ * library image: FDG_STATIC_SCRATCH_BYTES of device memory on every GPU that loads the library,
+ * held until the process exits.  The call itself allocates and frees nothing.
+ *   - Shapes whose fdg_conv_wgrad_scratch_bytes exceeds FDG_STATIC_SCRATCH_BYTES are refused
+ *     with FDG_ERR_WORKSPACE_TOO_SMALL and nothing is launched.
+ *   - The first call on each device looks up the buffer's device address (a host-side query,
+ *     made with that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one buffer, and it keeps what the previous call left.
+ *     Every slice of partial sums a launch reads was written by that same launch, so nothing
+ *     has to be cleared, but two calls whose kernels may overlap on the GPU (different
+ *     streams without an ordering between them) race on it: order them. */
+#define FDG_STATIC_SCRATCH_BYTES ((size_t)8 << 20)
+fdg_status fdg_conv_wgrad_static(int precision, const fdg_conv_shape* shape, const void* x, const void* dy,
+                                 float* dw, fdg_stream stream);
+
 /* Which path a call takes: op 0 = forward, 1 = dgrad (with w_flipped), 2 = wgrad. */
 fdg_status fdg_conv_path(int precision, const fdg_conv_shape* shape, int op, int* uses_tensor_cores);
 

@@ -26,7 +26,7 @@ EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count"
            "fdg_set_lr", "fdg_step", "fdg_step_host", "fdg_sync", "fdg_profile_enable", "fdg_profile_read", "fdg_get_module_output", "fdg_get_input_grad",
            "fdg_boundary_elems", "fdg_get_saved_tensor", "fdg_get_schedule_log", "fdg_launch_count", "fdg_status_string",
            "fdg_last_error", "fdg_conv_forward", "fdg_conv_dgrad", "fdg_conv_flip_weights",
-           "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_path"]
+           "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_wgrad_static", "fdg_conv_path"]
 
 
 class fdg_arch(C.Structure):
@@ -95,6 +95,7 @@ def load_library(path=LIB_PATH):
         "fdg_conv_flip_weights": [P(fdg_conv_shape), vp, vp, vp],
         "fdg_conv_wgrad_scratch_bytes": [C.c_int, P(fdg_conv_shape), P(sz)],
         "fdg_conv_wgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, sz, vp, vp],
+        "fdg_conv_wgrad_static": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp],
         "fdg_conv_path": [C.c_int, P(fdg_conv_shape), C.c_int, P(C.c_int)],
     }
     for name, args in sig.items():
@@ -335,6 +336,14 @@ class ConvOps:
         dw = self.torch.empty((s.Co, s.R, s.R, s.Ci), dtype=self.torch.float32, device="cuda")
         self._chk(self.lib.fdg_conv_wgrad(self.precision, C.byref(s), _ptr(x), _ptr(dy), _ptr(dw), _ptr(scratch),
                                           n.value, _ptr(self.status), self._stream()))
+        return dw
+
+    def wgrad_static(self, s, x, dy):
+        """fdg_conv_wgrad_static: the weight gradient with the library's built-in scratch buffer
+        (only the result tensor is allocated here, by torch, before the call)."""
+        dw = self.torch.empty((s.Co, s.R, s.R, s.Ci), dtype=self.torch.float32, device="cuda")
+        self._chk(self.lib.fdg_conv_wgrad_static(self.precision, C.byref(s), _ptr(x), _ptr(dy), _ptr(dw),
+                                                 self._stream()))
         return dw
 
     def timed_out(self):
