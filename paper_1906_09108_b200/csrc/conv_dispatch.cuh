@@ -1,12 +1,14 @@
 // Chooses the kernel for one convolution: the tcgen05 tensor-core kernels for bf16 3x3
 // stride-1 convolutions whose shape they cover, the CUDA-core implicit GEMM otherwise.
 #pragma once
+#include <algorithm>
 #include <cstring>
 #include <map>
 #include <vector>
 
 #include "conv_simt.cuh"
 #include "conv_tc.cuh"
+#include "conv_halo.cuh"
 
 namespace fdg {
 
@@ -52,6 +54,101 @@ inline cudaError_t run_conv_tc(cudaStream_t st, TensorMapCache* cache, int N, in
     ib = cache->maps.insert({kb, mb}).first;
   }
   return tc::conv_tc_launch(st, p, ia->second, ib->second, out, res, res_mask, err_dev, cache->sm_count);
+}
+
+
+// ---- halo-tile kernels (16/32/64-channel layers) ------------------------------------------
+inline int cached_sm_count(TensorMapCache* cache) {
+  if (cache->sm_count == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&cache->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return cache->sm_count;
+}
+
+inline bool halo_shape(const ConvGeom& g) {
+  return g.R == 3 && g.S == 3 && g.stride == 1 && g.pad == 1 && g.P == g.H && g.Q == g.W;
+}
+// forward: K channels = Ci, N channels = Co; data gradient: the other way round
+inline bool halo_fprop_eligible(const ConvGeom& g) { return halo_shape(g) && halo::fwd_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+inline bool halo_dgrad_eligible(const ConvGeom& g) { return halo_shape(g) && halo::fwd_supported(g.N, g.H, g.W, g.Co, g.Ci); }
+inline bool halo_wgrad_eligible(const ConvGeom& g) { return halo_shape(g) && halo::wgrad_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+
+inline cudaError_t cached_tile_map(TensorMapCache* cache, const void* act, int N, int H, int W, int C, int G,
+                                   const CUtensorMap** out) {
+  TensorMapCache::Key k;
+  std::memset(&k, 0, sizeof(k));
+  k.ptr = act; k.d[0] = 3; k.d[1] = N; k.d[2] = H; k.d[3] = W; k.d[4] = C; k.d[5] = G;
+  auto it = cache->maps.find(k);
+  if (it == cache->maps.end()) {
+    CUtensorMap m;
+    cudaError_t e = halo::make_tile_map(act, N, H, W, C, G, &m);
+    if (e != cudaSuccess) return e;
+    it = cache->maps.insert({k, m}).first;
+  }
+  *out = &it->second;
+  return cudaSuccess;
+}
+inline cudaError_t cached_weight_map(TensorMapCache* cache, const void* wgt, int Ck, int Cn, const CUtensorMap** out) {
+  TensorMapCache::Key k;
+  std::memset(&k, 0, sizeof(k));
+  k.ptr = wgt; k.d[0] = 4; k.d[1] = Ck; k.d[2] = Cn;
+  auto it = cache->maps.find(k);
+  if (it == cache->maps.end()) {
+    CUtensorMap m;
+    cudaError_t e = halo::make_weight_map(wgt, Ck, Cn, &m);
+    if (e != cudaSuccess) return e;
+    it = cache->maps.insert({k, m}).first;
+  }
+  *out = &it->second;
+  return cudaSuccess;
+}
+
+// out = conv3x3(act, wgt) [+ res * [mask > 0]]; act [N][H][W][Ck], wgt [Cn][9*Ck], out [N][H][W][Cn].
+inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ck, int Cn,
+                                 const bf16_t* act, const bf16_t* wgt, bf16_t* out, const bf16_t* res,
+                                 const bf16_t* res_mask, int* err_dev) {
+  const int sms = cached_sm_count(cache);
+  halo::FwdParams p = halo::fwd_params(N, H, W, Ck, Cn, sms);
+  const CUtensorMap *mx, *mw;
+  cudaError_t e = cached_tile_map(cache, act, N, H, W, Ck, p.G, &mx);
+  if (e == cudaSuccess) e = cached_weight_map(cache, wgt, Ck, Cn, &mw);
+  if (e == cudaSuccess) e = halo::set_smem_attrs();
+  if (e != cudaSuccess) return e;
+  const int grid = p.tiles < sms ? p.tiles : sms;
+  halo::conv_halo_kernel<<<grid, tc::kThreads, halo::fwd_smem_bytes(p), st>>>(*mx, *mw, p, out, res, res_mask, err_dev);
+  return cudaGetLastError();
+}
+
+// dw[Co][3][3][Ci] (fp32) from x [N][H][W][Ci] and dy [N][H][W][Co]; `scratch` holds the per-CTA partials
+// (halo::wgrad_scratch_elems floats).  Two launches: the tensor-core kernel and the fixed-order sum.
+inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ci, int Co,
+                                  const bf16_t* x, const bf16_t* dy, float* dw, float* scratch, int* err_dev) {
+  halo::WgradParams p = halo::wgrad_params(N, H, W, Ci, Co);
+  const CUtensorMap *mx, *my;
+  cudaError_t e = cached_tile_map(cache, x, N, H, W, Ci, p.G, &mx);
+  if (e == cudaSuccess) e = cached_tile_map(cache, dy, N, H, W, Co, p.G, &my);
+  if (e == cudaSuccess) e = halo::set_smem_attrs();
+  if (e != cudaSuccess) return e;
+  const int ctas = halo::wgrad_ctas(p);
+  halo::wgrad_halo_kernel<<<ctas, tc::kThreads, halo::wgrad_smem_bytes(p), st>>>(*mx, *my, p, scratch, err_dev);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const size_t n = (size_t)Co * 9 * Ci;
+  halo::wgrad_halo_reduce_kernel<<<(int)((n + 31) / 32), 256, 0, st>>>(scratch, dw, n, ctas);
+  return cudaGetLastError();
+}
+
+
+// Does the data gradient of this convolution read the flipped/transposed weight copy?
+inline bool dgrad_uses_flipped(const ConvGeom& g) { return halo_dgrad_eligible(g) || tc_eligible(g); }
+
+// fp32 scratch elements a weight-gradient call may need (bf16 storage: whichever kernel is chosen).
+inline size_t conv_wgrad_scratch_elems(bool bf16_storage, const ConvGeom& g) {
+  size_t n = wgrad_scratch_elems(g);
+  if (bf16_storage && halo_wgrad_eligible(g)) n = std::max(n, halo::wgrad_scratch_elems(g.N, g.H, g.W, g.Ci, g.Co));
+  return n;
 }
 
 }  // namespace fdg

@@ -1,0 +1,553 @@
+// 3x3 / stride 1 / pad 1 convolutions of narrow layers (16, 32 or 64 channels per pixel) on the
+// sm_100a tensor cores, organised around a HALO TILE: one TMA load brings G whole images, each
+// with its one-pixel zero border (the hardware's out-of-bounds fill is the padding), into shared
+// memory as consecutive "padded pixels" of one swizzle span each (32/64/128 bytes).  Every filter
+// tap is then the same tile seen from a start address shifted by (r*Wp + s) pixels, so an
+// activation is read from L2/HBM once per pass instead of once per tap.
+//
+//   padded pixel index  q = (g*Hp + h')*Wp + w'      Hp = H+2, Wp = W+2
+//   output pixel (g,h,w) has accumulator row  m = (g*Hp + h)*Wp + w  and reads q = m + r*Wp + s
+//   rows m with w >= W or h >= H are computed but never stored.
+//
+// Forward / data gradient (conv_halo_kernel):
+//   D[m][n] = sum_tap sum_c X[m + r*Wp + s][c] * Wt[tap][n][c]       (both operands K-major)
+//   M = 128 padded pixels per accumulator, N = output channels, K = 16 channels per instruction.
+//   The data gradient is the same kernel on dy with the flipped/transposed weight copy.
+// Weight gradient (wgrad_halo_kernel):
+//   dW[n][r][s][c] = sum_q dY[q][n] * X[q + r*Wp + s][c]
+//   pixels are the reduction dimension, so both operands are read MN-major from the same kind of
+//   tile; the A operand stacks the filter taps of one filter row along M (its M-blocks start one
+//   pixel apart), B is dY with its border columns and rows zero.  Each CTA keeps its partial sums
+//   in tensor memory over all its tiles, writes them once, and a fixed-order pass adds the CTAs'
+//   partials, so the result does not depend on scheduling.
+//
+// Roles by warp: 0 = TMA producer, 1 = MMA issuer (one elected lane), 2..5 = epilogue (32
+// tensor-memory lanes each).  Every wait is bounded; on time-out the CTA raises an error word.
+#pragma once
+#include "conv_tc.cuh"
+
+namespace fdg {
+namespace halo {
+
+using namespace fdg::tc;
+
+struct FwdParams {
+  int W, H, N, Wp, Hp;
+  int Ck, Cn;                 // channels of the activation operand (16/32/64) and of the output
+  int G;                      // images per tile
+  int tiles;                  // ceil(N / G)
+  int m_tiles;                // 128-row accumulators per tile
+  int img_rows;               // Hp * Wp
+  uint32_t pitch;             // Ck * 2 bytes = swizzle span
+  uint32_t tile_tx_bytes;     // bytes one TMA tile load writes
+  uint32_t stage_bytes;       // shared memory reserved per stage (multiple of 1024)
+  int stages;
+  uint32_t w_tap_bytes;       // shared memory reserved per filter tap of the weights (multiple of 1024)
+  uint32_t w_tx_bytes;        // bytes one weight-tap load writes
+  int nacc;                   // accumulator slots in tensor memory
+  uint32_t tmem_cols;
+};
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Shared-memory descriptor of an MN-major operand made of swizzle-span-wide rows (one per k):
+// `lbo` = byte distance between consecutive MN blocks, 8-row k groups `8*row_bytes` apart.
+__device__ __forceinline__ uint64_t smem_desc_mnmajor(uint32_t addr, uint32_t row_bytes, uint32_t lbo) {
+  const uint64_t layout = row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6);
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)(((8 * row_bytes) >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= layout << 61;
+  return d;
+}
+// bf16 x bf16 -> fp32, M = 128; `mn_major` sets both operands MN-major.
+__device__ __forceinline__ uint32_t instr_desc(int n, bool mn_major) {
+  uint32_t d = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+  if (mn_major) d |= (1u << 15) | (1u << 16);
+  return d;
+}
+
+// ------------------------------------------------------- forward / data gradient --
+// out[pixel][n] (bf16, row stride Cn) = conv + (res ? res * [mask ? mask > 0 : 1] : 0)
+__global__ void __launch_bounds__(kThreads, 1)
+conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, FwdParams p,
+                 __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
+                 const __nv_bfloat16* __restrict__ res_mask, int* __restrict__ error_word) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* w_smem = smem + (size_t)p.stages * p.stage_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(w_smem + 9 * (size_t)p.w_tap_bytes);
+  uint64_t* full = bars;                       // [stages]  TMA -> MMA
+  uint64_t* empty = full + p.stages;           // [stages]  MMA -> TMA
+  uint64_t* w_full = empty + p.stages;         // [1]       weights resident
+  uint64_t* acc_full = w_full + 1;             // [nacc]    MMA -> epilogue
+  uint64_t* acc_empty = acc_full + p.nacc;     // [nacc]    epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + p.nacc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(w_full, 1);
+    for (int a = 0; a < p.nacc; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int ksteps = p.Ck / 16;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(w_full, 9 * p.w_tx_bytes);
+      for (int tap = 0; tap < 9; ++tap) tma_load_2d(w_smem + (size_t)tap * p.w_tap_bytes, &map_w, w_full, tap * p.Ck, 0);
+      uint32_t it = 0;
+      for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(&full[s], p.tile_tx_bytes);
+        tma_load_4d(smem + (size_t)s * p.stage_bytes, &map_x, &full[s], 0, -1, -1, tile * p.G);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(p.Cn, false);
+      bool ok = mbar_wait(w_full, 0, abort_flag);
+      tc_fence_after();
+      // The issuing thread is the bottleneck when the instructions are this small, so the
+      // descriptors are not rebuilt per instruction: a descriptor's low word holds the start
+      // address in 16-byte units, and moving the operand is one 64-bit add.
+      const uint64_t w_desc0 = smem_desc_kmajor(smem_u32(w_smem), p.pitch);
+      const uint64_t w_tap_step = p.w_tap_bytes >> 4;
+      uint64_t tap_off[9];                                   // operand shift of each filter tap, 16-byte units
+#pragma unroll
+      for (int tap = 0; tap < 9; ++tap) tap_off[tap] = (uint64_t)(((tap / 3) * p.Wp + (tap % 3)) * p.pitch) >> 4;
+      const uint64_t mtile_step = (uint64_t)(kTileM * p.pitch) >> 4;
+      // One tcgen05.mma of K = 16 occupies the tensor pipe for max(60, N/2) cycles whatever M is
+      // and whether or not it depends on the previous one (measured), so a 128-row tile costs
+      // 9 * Ck/16 * 60 cycles here and the only overhead worth removing is the issue loop's own.
+      uint32_t it = 0, acount = 0;
+      for (int tile = blockIdx.x; ok && tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!mbar_wait(&full[s], ph, abort_flag)) break;
+        tc_fence_after();
+        uint64_t x_desc = smem_desc_kmajor(smem_u32(smem + (size_t)s * p.stage_bytes), p.pitch);
+        for (int i = 0; i < p.m_tiles; ++i, ++acount, x_desc += mtile_step) {
+          const int slot = acount % p.nacc;
+          const uint32_t aph = (acount / p.nacc) & 1;
+          if (!mbar_wait(&acc_empty[slot], aph ^ 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)slot * p.Cn;
+          if (ksteps == 1) {
+#pragma unroll
+            for (int tap = 0; tap < 9; ++tap)
+              tc_mma_bf16(d_tmem, x_desc + tap_off[tap], w_desc0 + tap * w_tap_step, idesc, tap != 0);
+          } else {
+#pragma unroll
+            for (int tap = 0; tap < 9; ++tap) {
+              const uint64_t a0 = x_desc + tap_off[tap], b0 = w_desc0 + tap * w_tap_step;
+              for (int j = 0; j < ksteps; ++j) tc_mma_bf16(d_tmem, a0 + 2 * j, b0 + 2 * j, idesc, (tap | j) != 0);
+            }
+          }
+          tc_commit(&acc_full[slot]);
+        }
+        if (!ok) break;
+        tc_commit(&empty[s]);
+      }
+    }
+  } else {
+    const int lane_grp = warp & 3;
+    uint32_t acount = 0;
+    for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x) {
+      const int n0 = tile * p.G;
+      bool ok = true;
+      for (int i = 0; i < p.m_tiles; ++i, ++acount) {
+        const int slot = acount % p.nacc;
+        const uint32_t aph = (acount / p.nacc) & 1;
+        if (!mbar_wait(&acc_full[slot], aph, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const int m = kTileM * i + lane_grp * 32 + lane;
+        const int g = m / p.img_rows, rem = m - g * p.img_rows;
+        const int h = rem / p.Wp, w = rem - h * p.Wp;
+        const bool valid = h < p.H && w < p.W && g < p.G && n0 + g < p.N;
+        const size_t base = ((((size_t)(n0 + g) * p.H + h) * p.W) + w) * p.Cn;
+        const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)slot * p.Cn;
+        for (int c0 = 0; c0 < p.Cn; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(taddr + c0, v);
+          tmem_ld_wait();
+          if (!valid) continue;
+          float f[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]);
+          if (res) {
+            uint4 r0 = *reinterpret_cast<const uint4*>(res + base + c0);
+            uint4 r1 = *reinterpret_cast<const uint4*>(res + base + c0 + 8);
+            const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
+            const __nv_bfloat16* rb1 = reinterpret_cast<const __nv_bfloat16*>(&r1);
+            float gq[16];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { gq[e] = __bfloat162float(rb0[e]); gq[8 + e] = __bfloat162float(rb1[e]); }
+            if (res_mask) {
+              uint4 m0 = *reinterpret_cast<const uint4*>(res_mask + base + c0);
+              uint4 m1 = *reinterpret_cast<const uint4*>(res_mask + base + c0 + 8);
+              const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&m0);
+              const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&m1);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                if (!(__bfloat162float(mb0[e]) > 0.f)) gq[e] = 0.f;
+                if (!(__bfloat162float(mb1[e]) > 0.f)) gq[8 + e] = 0.f;
+              }
+            }
+#pragma unroll
+            for (int e = 0; e < 16; ++e) f[e] += gq[e];
+          }
+          uint4 o0, o1;
+          __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
+          __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            ob0[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+            ob1[e] = __floats2bfloat162_rn(f[8 + 2 * e], f[8 + 2 * e + 1]);
+          }
+          *reinterpret_cast<uint4*>(out + base + c0) = o0;
+          *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[slot]);
+      }
+      if (!ok) break;
+    }
+  }
+
+  // Teardown.  After an abort, TMA copies may still be in flight towards this CTA's shared
+  // memory: give every barrier that was armed a bounded chance to complete before leaving.
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) {
+      if (error_word) atomicExch(error_word, 1);
+      for (int s = 0; s <= p.stages; ++s) {
+        uint64_t* b = s < p.stages ? &full[s] : w_full;
+        for (uint32_t i = 0; i < (1u << 16); ++i)
+          if (mbar_try_wait(b, 0) || mbar_try_wait(b, 1)) break;
+      }
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
+// ------------------------------------------------------------- weight gradient --
+// With q' = q + r*Wp the sum becomes dW[n][r][s][c] = sum_q' dY[q' - r*Wp][n] * X[q' + s][c], so ONE
+// instruction per 16-pixel step covers all nine taps: the A operand stacks the taps s of a filter
+// row along M (M-blocks one pixel apart in the x tile), the B operand stacks the filter rows along
+// N (N-blocks Wp pixels apart in the dy tile, which is loaded with two extra zero rows on top so
+// that block b = 2 - r starts at row q' + b*Wp).  N = 3*Co <= 192 costs the same 60..96 cycles as
+// N = Co would.
+struct WgradParams {
+  int W, H, N, Wp, Hp;
+  int Ci, Co;                 // channels of x (16/32/64) and of dy (16/32/64)
+  int G, tiles;               // images per tile, ceil(N / G)
+  int ksteps;                 // 16-pixel reduction steps per tile
+  uint32_t pitch_x, pitch_y;
+  uint32_t x_tx_bytes, y_tx_bytes;
+  uint32_t x_bytes, y_bytes;  // shared memory reserved per stage for the two tiles (multiples of 1024)
+  int stages;
+  int sgroups;                // M-block groups: 1, or 2 when Ci = 64 (128 rows hold only two taps)
+  int taps_per_group;         // min(3, 128 / Ci)
+  uint32_t tmem_cols;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, WgradParams p,
+                  float* __restrict__ partial, int* __restrict__ error_word) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t stage_bytes = p.x_bytes + p.y_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes);
+  uint64_t* full = bars;
+  uint64_t* empty = full + p.stages;
+  uint64_t* done = empty + p.stages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(done, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // The reduction runs over whole 16-pixel steps and the stacked blocks read some pixels past
+  // the tile: that slack is never written by TMA, so it is cleared once (a stray NaN there
+  // would survive the multiplication by a zero of the other operand).
+  for (int s = 0; s < p.stages; ++s) {
+    uint8_t* xs = smem + (size_t)s * stage_bytes;
+    uint8_t* ys = xs + p.x_bytes;
+    for (uint32_t o = p.x_tx_bytes + threadIdx.x * 16; o < p.x_bytes; o += kThreads * 16) *reinterpret_cast<uint4*>(xs + o) = make_uint4(0, 0, 0, 0);
+    for (uint32_t o = p.y_tx_bytes + threadIdx.x * 16; o < p.y_bytes; o += kThreads * 16) *reinterpret_cast<uint4*>(ys + o) = make_uint4(0, 0, 0, 0);
+  }
+  fence_proxy_async();
+  if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int ncols = 3 * p.Co;                                 // N of the instruction
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) break;
+        uint8_t* xs = smem + (size_t)s * stage_bytes;
+        mbar_expect_tx(&full[s], p.x_tx_bytes + p.y_tx_bytes);
+        tma_load_4d(xs, &map_x, &full[s], 0, -1, -1, tile * p.G);
+        tma_load_4d(xs + p.x_bytes, &map_y, &full[s], 0, 0, -2, tile * p.G);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(ncols, true);
+      const uint64_t a_kstep = (uint64_t)(16 * p.pitch_x) >> 4, b_kstep = (uint64_t)(16 * p.pitch_y) >> 4;
+      const uint64_t a_group = (uint64_t)(p.taps_per_group * p.pitch_x) >> 4;
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t x_addr = smem_u32(smem + (size_t)s * stage_bytes);
+        uint64_t a_desc = smem_desc_mnmajor(x_addr, p.pitch_x, p.pitch_x);
+        uint64_t b_desc = smem_desc_mnmajor(x_addr + p.x_bytes, p.pitch_y, (uint32_t)p.Wp * p.pitch_y);
+        if (p.sgroups == 1) {
+          for (int j = 0; j < p.ksteps; ++j, a_desc += a_kstep, b_desc += b_kstep)
+            tc_mma_bf16(tmem_base, a_desc, b_desc, idesc, (it | (uint32_t)j) != 0);
+        } else {
+          for (int j = 0; j < p.ksteps; ++j, a_desc += a_kstep, b_desc += b_kstep) {
+            tc_mma_bf16(tmem_base, a_desc, b_desc, idesc, (it | (uint32_t)j) != 0);
+            tc_mma_bf16(tmem_base + (uint32_t)ncols, a_desc + a_group, b_desc, idesc, (it | (uint32_t)j) != 0);
+          }
+        }
+        tc_commit(&empty[s]);
+      }
+      if (ok) tc_commit(done);
+    }
+  } else {
+    const int lane_grp = warp & 3;
+    if (mbar_wait(done, 0, abort_flag)) {
+      tc_fence_after();
+      const int row = lane_grp * 32 + lane;
+      const int sblk = row / p.Ci, ci = row - sblk * p.Ci;
+      float* dst = partial + (size_t)blockIdx.x * ((size_t)p.Co * 9 * p.Ci);
+      for (int sg = 0; sg < p.sgroups; ++sg) {
+        const int sx = sg * p.taps_per_group + sblk;
+        const bool valid = sblk < p.taps_per_group && sx < 3;
+        const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(sg * ncols);
+        for (int c0 = 0; c0 < ncols; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(taddr + c0, v);
+          tmem_ld_wait();
+          if (!valid) continue;
+          const int b = c0 / p.Co, r = 2 - b, co0 = c0 - b * p.Co;      // Co is a multiple of 16: a chunk stays in one block
+#pragma unroll
+          for (int e = 0; e < 16; ++e)
+            dst[(((size_t)(co0 + e) * 3 + r) * 3 + sx) * p.Ci + ci] = __uint_as_float(v[e]);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) {
+      if (error_word) atomicExch(error_word, 1);
+      for (int s = 0; s < p.stages; ++s)
+        for (uint32_t i = 0; i < (1u << 16); ++i)
+          if (mbar_try_wait(&full[s], 0) || mbar_try_wait(&full[s], 1)) break;
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
+// dw[i] = sum over the pixel-split CTAs of partial[cta][i], in CTA order.  A block owns 32
+// consecutive outputs; its 8 warps take interleaved CTAs and are added in warp order.
+__global__ void __launch_bounds__(256) wgrad_halo_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dw, size_t n, int ctas) {
+  __shared__ float part[8][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const size_t i = (size_t)blockIdx.x * 32 + lane;
+  float a = 0.f;
+  if (i < n)
+    for (int z = warp; z < ctas; z += 8) a += partial[(size_t)z * n + i];
+  part[warp][lane] = a;
+  __syncthreads();
+  if (warp == 0 && i < n) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) t += part[w][lane];
+    dw[i] = t;
+  }
+}
+
+// ----------------------------------------------------------------- host side ---
+inline uint32_t round_up_u32(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
+constexpr size_t kSmemBudget = 200 * 1024;
+
+inline bool chan_ok(int c) { return c == 16 || c == 32 || c == 64; }
+
+inline FwdParams fwd_params(int N, int H, int W, int Ck, int Cn, int sm_count) {
+  FwdParams p{};
+  p.W = W; p.H = H; p.N = N; p.Wp = W + 2; p.Hp = H + 2; p.Ck = Ck; p.Cn = Cn;
+  p.img_rows = p.Hp * p.Wp;
+  p.pitch = (uint32_t)Ck * 2;
+  p.w_tx_bytes = (uint32_t)Cn * p.pitch;
+  p.w_tap_bytes = round_up_u32(p.w_tx_bytes, 1024);
+  // images per tile: as many as keep every SM busy, within the shared-memory budget
+  int G = N / (sm_count > 0 ? sm_count : 148);
+  if (G < 1) G = 1;
+  for (;; --G) {
+    p.G = G;
+    p.m_tiles = (((G - 1) * p.Hp + (H - 1)) * p.Wp + W + kTileM - 1) / kTileM;
+    uint32_t rows = (uint32_t)(kTileM * p.m_tiles + 2 * p.Wp + 2);
+    if (rows < (uint32_t)(G * p.img_rows)) rows = (uint32_t)(G * p.img_rows);
+    p.stage_bytes = round_up_u32(rows * p.pitch, 1024);
+    if (G == 1 || 2 * (size_t)p.stage_bytes + 9 * (size_t)p.w_tap_bytes + 2048 <= kSmemBudget) break;
+  }
+  p.tiles = (N + p.G - 1) / p.G;
+  p.tile_tx_bytes = (uint32_t)(p.G * p.img_rows) * p.pitch;
+  size_t left = kSmemBudget - 9 * (size_t)p.w_tap_bytes - 2048;
+  int stages = (int)(left / p.stage_bytes);
+  const int per_cta = (p.tiles + (sm_count > 0 ? sm_count : 148) - 1) / (sm_count > 0 ? sm_count : 148);
+  if (stages > 3) stages = 3;
+  if (stages > per_cta) stages = per_cta;                     // shared memory left free lets other kernels' CTAs co-reside
+  p.stages = stages;
+  p.nacc = p.m_tiles < 4 ? p.m_tiles : 4;
+  if (p.nacc < 2) p.nacc = 2;
+  uint32_t cols = 32;
+  while (cols < (uint32_t)(p.nacc * Cn)) cols <<= 1;
+  p.tmem_cols = cols;
+  return p;
+}
+
+inline size_t fwd_smem_bytes(const FwdParams& p) {
+  return (size_t)p.stages * p.stage_bytes + 9 * (size_t)p.w_tap_bytes + (size_t)(2 * p.stages + 1 + 2 * p.nacc) * 8 + 16 + 1024;
+}
+
+inline bool fwd_supported(int N, int H, int W, int Ck, int Cn) {
+  if (!chan_ok(Ck) || Cn % 16 || Cn < 16 || Cn > 128) return false;
+  if (W + 2 > 256 || H + 2 > 256 || N < 1) return false;
+  FwdParams p = fwd_params(N, H, W, Ck, Cn, 148);
+  return p.stages >= 1 && fwd_smem_bytes(p) <= kSmemBudget + 4096 && p.tile_tx_bytes < (1u << 20);
+}
+
+inline WgradParams wgrad_params(int N, int H, int W, int Ci, int Co) {
+  WgradParams p{};
+  p.W = W; p.H = H; p.N = N; p.Wp = W + 2; p.Hp = H + 2; p.Ci = Ci; p.Co = Co;
+  p.pitch_x = (uint32_t)Ci * 2; p.pitch_y = (uint32_t)Co * 2;
+  const int img_rows = p.Hp * p.Wp;
+  // images per tile: what two pipeline stages of both tiles fit in shared memory
+  const int max_rows = (int)(96 * 1024 / (p.pitch_x + p.pitch_y));
+  p.G = max_rows / img_rows > 0 ? max_rows / img_rows : 1;
+  if (p.G > N) p.G = N;
+  p.tiles = (N + p.G - 1) / p.G;
+  const int Q = p.G * img_rows;
+  p.ksteps = (Q + 15) / 16;
+  const int blocks = kTileM / Ci;
+  p.taps_per_group = blocks < 3 ? blocks : 3;
+  p.sgroups = (3 + p.taps_per_group - 1) / p.taps_per_group;
+  p.x_tx_bytes = (uint32_t)Q * p.pitch_x; p.y_tx_bytes = (uint32_t)Q * p.pitch_y;
+  p.x_bytes = round_up_u32((uint32_t)(16 * p.ksteps + 2 * blocks + 16) * p.pitch_x, 1024);
+  p.y_bytes = round_up_u32((uint32_t)(16 * p.ksteps + 2 * p.Wp + 16) * p.pitch_y, 1024);
+  const size_t stage = (size_t)p.x_bytes + p.y_bytes;
+  int stages = (int)((kSmemBudget - 2048) / stage);
+  p.stages = stages > 2 ? 2 : stages;
+  uint32_t need = (uint32_t)(p.sgroups * 3 * Co), cols = 32;
+  while (cols < need) cols <<= 1;
+  p.tmem_cols = cols;
+  return p;
+}
+
+// Pixel split: few enough CTAs that their partial sums (Co*9*Ci floats each) stay small next to
+// the operands, enough of them to spread the reduction over the SMs.
+inline int wgrad_ctas(const WgradParams& p) {
+  const size_t wsize = (size_t)p.Co * 9 * p.Ci;
+  int want = (int)((size_t)p.N * p.H * p.W * (p.Ci + p.Co) * 2 / (wsize * 2));     // partial bytes <= ~ 2 x operand bytes
+  if (want > 128) want = 128;
+  if (want < 32) want = 32;
+  return p.tiles < want ? p.tiles : want;
+}
+inline size_t wgrad_smem_bytes(const WgradParams& p) {
+  return (size_t)p.stages * ((size_t)p.x_bytes + p.y_bytes) + (size_t)(2 * p.stages + 1) * 8 + 16 + 1024;
+}
+inline bool wgrad_supported(int N, int H, int W, int Ci, int Co) {
+  if (!chan_ok(Ci) || !chan_ok(Co)) return false;
+  if (W + 2 > 256 || H + 2 > 256 || N < 1) return false;
+  WgradParams p = wgrad_params(N, H, W, Ci, Co);
+  return p.stages >= 1 && p.x_tx_bytes < (1u << 19) && p.y_tx_bytes < (1u << 19) && p.tmem_cols <= 512;
+}
+// fp32 elements of scratch the weight gradient needs for its per-CTA partial sums.
+inline size_t wgrad_scratch_elems(int N, int H, int W, int Ci, int Co) {
+  WgradParams p = wgrad_params(N, H, W, Ci, Co);
+  return (size_t)wgrad_ctas(p) * Co * 9 * Ci;
+}
+
+// Halo-tile tensor map of a bf16 NHWC tensor: box = G whole images with border.
+inline cudaError_t make_tile_map(const void* act, int N, int H, int W, int C, int G, CUtensorMap* map) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+  cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+  cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)(W + 2), (cuuint32_t)(H + 2), (cuuint32_t)G};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  if (enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(act), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(C * 2), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  return cudaSuccess;
+}
+// Weight map: bf16 [Cn][9*Ck], box = one filter tap of all Cn rows.
+inline cudaError_t make_weight_map(const void* wgt, int Ck, int Cn, CUtensorMap* map) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  cuuint64_t dims[2] = {(cuuint64_t)9 * Ck, (cuuint64_t)Cn};
+  cuuint64_t strides[1] = {(cuuint64_t)9 * Ck * 2};
+  cuuint32_t box[2] = {(cuuint32_t)Ck, (cuuint32_t)Cn};
+  cuuint32_t estr[2] = {1, 1};
+  if (enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(wgt), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(Ck * 2), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  return cudaSuccess;
+}
+
+inline cudaError_t set_smem_attrs() {
+  static bool done = false;
+  if (done) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(conv_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 8192);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(wgrad_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget + 8192);
+  if (e == cudaSuccess) done = true;
+  return e;
+}
+
+}  // namespace halo
+}  // namespace fdg

@@ -275,7 +275,7 @@ static void plan_modules(fdg_ctx* c) {
     auto red_scratch = [&](size_t rows, int ch) { scr = std::max(scr, (size_t)kRedMaxBlocks * kRedMaxSums * ch); (void)rows; };
     auto wg_scratch = [&](int n, int h, int w, int cin, int p, int q, int cout, int r, int stride, int pad) {
       ConvGeom g{n, h, w, cin, p, q, cout, r, r, stride, pad};
-      scr = std::max(scr, wgrad_scratch_elems(g));
+      scr = std::max(scr, conv_wgrad_scratch_elems(c->bf16_mode, g));
     };
     for (Unit& u : m.units) {
       const size_t in_e = B * u.H * u.W * u.ci, out_e = B * u.P * u.Q * u.co;
@@ -321,8 +321,8 @@ static void plan_modules(fdg_ctx* c) {
         if (u.type != U_BASIC && u.type != U_PREACT) continue;
         ConvGeom g1{a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 3, u.stride, 1};
         ConvGeom g2{a.batch, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 3, 1, 1};
-        if (tc_eligible(g1)) u.f1 = flip(u.w1, u.co, u.ci);
-        if (tc_eligible(g2)) u.f2 = flip(u.w2, u.co, u.co);
+        if (dgrad_uses_flipped(g1)) u.f1 = flip(u.w1, u.co, u.ci);
+        if (dgrad_uses_flipped(g2)) u.f2 = flip(u.w2, u.co, u.co);
       }
       m.flip_elems = fe;
     }
@@ -497,6 +497,11 @@ template <typename T>
 static void conv_fprop(Launch& L, const ConvGeom& g, const T* x, const T* w, T* y, const T* res) {
   L.begin(KC_CONV_FPROP, (in_elems(g) + w_elems(g) + out_elems(g) * (res ? 2 : 1)) * sizeof(T), conv_flops(g));
   if constexpr (std::is_same<T, bf16>::value) {
+    if (halo_fprop_eligible(g)) {
+      ++L.c->launches;
+      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error));
+      return;
+    }
     if (tc_eligible(g)) {
       ++L.c->launches;
       L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error));
@@ -511,6 +516,11 @@ static void conv_dgrad(Launch& L, const ConvGeom& g, const T* dy, const T* w, co
                        const T* mask) {
   L.begin(KC_CONV_DGRAD, (out_elems(g) + w_elems(g) + in_elems(g) * (1 + (res ? 1 : 0) + (mask ? 1 : 0))) * sizeof(T), conv_flops(g));
   if constexpr (std::is_same<T, bf16>::value) {
+    if (wflip && halo_dgrad_eligible(g)) {
+      ++L.c->launches;
+      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error));
+      return;
+    }
     if (wflip && tc_eligible(g)) {
       ++L.c->launches;
       L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error));
@@ -522,6 +532,13 @@ static void conv_dgrad(Launch& L, const ConvGeom& g, const T* dy, const T* w, co
 template <typename T>
 static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* dy, float* dw) {
   L.begin(KC_CONV_WGRAD, (in_elems(g) + out_elems(g)) * sizeof(T) + w_elems(g) * 4, conv_flops(g));
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (halo_wgrad_eligible(g)) {
+      L.c->launches += 2;
+      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy, dw, m.scratch, L.c->tc_error));
+      return;
+    }
+  }
   L.note(launch_conv_simt<T, CONV_WGRAD>(L.st, g, x, dy, (T*)nullptr, m.scratch, dw, (const T*)nullptr, (const T*)nullptr, &L.c->launches));
 }
 

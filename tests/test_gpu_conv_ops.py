@@ -30,7 +30,16 @@ SHAPES_TC = [(4, 32, 32, 16, 16, 3, 1, 1),      # 32 tiles of 4 image rows, 32-b
              (10, 8, 8, 64, 64, 3, 1, 1),       # two images per tile, 128-byte swizzle
              (2, 32, 32, 16, 48, 3, 1, 1),      # c_in != c_out
              (2, 16, 16, 128, 160, 3, 1, 1),    # two channel chunks, wide N
-             (300, 8, 8, 64, 64, 3, 1, 1)]      # more tiles than SMs: several tiles per CTA
+             (300, 8, 8, 64, 64, 3, 1, 1),      # more tiles than SMs: several tiles per CTA
+             (5, 12, 20, 16, 32, 3, 1, 1),      # non-square image, c_in != c_out, odd batch
+             (3, 6, 10, 64, 16, 3, 1, 1),
+             (37, 16, 16, 32, 64, 3, 1, 1),     # ragged last tile in the weight gradient's pixel split
+             (301, 8, 8, 64, 64, 3, 1, 1),      # ragged last tile with several images per tile
+             (130, 32, 32, 16, 16, 3, 1, 1)]    # stage-1 shape of the 6n+2 networks, more images than weight-gradient CTAs
+
+# shapes whose three operators all take the halo-tile tensor-core kernels
+ALL_TC = {(4, 32, 32, 16, 16), (6, 16, 16, 32, 32), (10, 8, 8, 64, 64), (300, 8, 8, 64, 64), (5, 12, 20, 16, 32),
+          (3, 6, 10, 64, 16), (37, 16, 16, 32, 64), (301, 8, 8, 64, 64), (130, 32, 32, 16, 16)}
 
 
 def _run(prec_name, shape, expect_tc):
@@ -48,6 +57,8 @@ def _run(prec_name, shape, expect_tc):
     resy, resyo = _mk((n, p, q, co), 6, ops.dtype)
     tol = 1e-2 if prec_name == "bf16" else 2e-5
     assert ops.path(s, 0) == expect_tc
+    if prec_name == "bf16" and shape[:5] in ALL_TC:
+        assert ops.path(s, 1) and ops.path(s, 2)
 
     y = ops.forward(s, x, wt).float().cpu().numpy()
     assert _rel(y, L.conv2d_forward(xo, wo, st, pad)) < tol
