@@ -137,10 +137,10 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
-def make_fdg(B, precision, serial):
+def make_fdg(B, precision, serial, graphs=False):
     import fdg_synth as S
     g = B.FDG(B.make_arch(**ARCH), K=K_MODULES, split_after_block=SPLITS, beta=BETA, lr=LR, momentum=MOM,
-              weight_decay=WD, precision=precision, serial=serial)
+              weight_decay=WD, precision=precision, serial=serial, graphs=graphs)
     for k in range(1, K_MODULES + 1):
         g.set_params(k, S.init_params(0, k, g.param_layout(k)))
     return g
@@ -171,7 +171,7 @@ def run_gpu(args):
     loss_host = torch.zeros(1, dtype=torch.float32).pin_memory()
     loss_dev = torch.zeros(1, dtype=torch.float32, device="cuda")
 
-    g = make_fdg(B, precision, serial=False)
+    g = make_fdg(B, precision, serial=False, graphs=not args.no_graphs)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -197,7 +197,7 @@ def run_gpu(args):
         return ms
 
     dev_step = lambda i: g.step(pool_x[i % POOL], pool_y[i % POOL], loss_dev)
-    for i in range(2 * K_MODULES + warmup):          # pipeline fill + warm-up, untimed
+    for i in range(2 * K_MODULES + 2 + (0 if args.no_graphs else 8) + warmup):   # pipeline fill (+ graph recording) + warm-up, untimed
         dev_step(i)
     g.sync()
     sampler = ClockSampler(local) if rank == 0 else None
@@ -269,6 +269,7 @@ def run_gpu(args):
                     dtype="bf16" if args.precision == "bf16" else "f32", data="synthetic",
                     config=dict(workload=WORKLOAD, K=K_MODULES, splits=list(SPLITS), global_batch=world * b,
                                 beta=BETA, lr=LR, precision=args.precision, streams=K_MODULES,
+                                cuda_graphs=not args.no_graphs,
                                 parallelism="replicas only" if world > 1 else "single GPU",
                                 l2="activation FIFO touched per step (>1 GiB) exceeds the 126 MB L2; "
                                    "16 input batches cycled"),
@@ -288,8 +289,9 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="fdg", choices=["fdg", "reference"])
-    ap.add_argument("--precision", default="fp32", choices=["fp32", "bf16"])
+    ap.add_argument("--precision", default="bf16", choices=["fp32", "bf16"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graphs", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

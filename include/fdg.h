@@ -96,6 +96,12 @@ typedef struct {
                                      FDG_BF16_TC: bf16 activations/weights for the convolutions, fp32 accumulation,
                                      fp32 master weights, statistics and loss */
   int serial;                     /* 1 = run all modules on the caller's stream in order (debug) */
+  int graphs;                     /* 1 = once the pipeline is full, record each iteration into a CUDA graph (one per
+                                     phase of the rings, a power of two >= 2K of them) and replay it from then on.
+                                     Iterations then follow one another on the caller's stream while the K modules of
+                                     one iteration still run side by side; the ring buffers are rounded up to powers
+                                     of two, so the workspace grows.  Results are identical to graphs = 0.  Ignored
+                                     when serial = 1; fdg_profile_enable is refused (FDG_ERR_STATE). */
 } fdg_config;
 
 typedef struct {            /* one tensor of a module's flat parameter vector */

@@ -38,7 +38,7 @@ class fdg_arch(C.Structure):
 class fdg_config(C.Structure):
     _fields_ = [("K", C.c_int), ("split_after_block", C.POINTER(C.c_int)), ("beta", C.c_float), ("lr", C.c_float),
                 ("momentum", C.c_float), ("weight_decay", C.c_float), ("order", C.c_int),
-                ("weight_reading", C.c_int), ("precision", C.c_int), ("serial", C.c_int)]
+                ("weight_reading", C.c_int), ("precision", C.c_int), ("serial", C.c_int), ("graphs", C.c_int)]
 
 
 class fdg_param_entry(C.Structure):
@@ -128,7 +128,7 @@ class FDG:
 
     def __init__(self, arch, K=2, split_after_block=(1,), beta=1.0, lr=0.1, momentum=0.9, weight_decay=5e-4,
                  order=FDG_BACKWARD_FIRST, weight_reading=FDG_STASHED, precision=FDG_FP32_CUDACORE, serial=False,
-                 device="cuda:0"):
+                 graphs=False, device="cuda:0"):
         import torch
         self.torch = torch
         self.lib = load_library()
@@ -136,7 +136,7 @@ class FDG:
         self.K = K
         self._splits = (C.c_int * max(len(split_after_block), 1))(*split_after_block)
         self.cfg = fdg_config(K, C.cast(self._splits, C.POINTER(C.c_int)), beta, lr, momentum, weight_decay, order,
-                              weight_reading, precision, int(serial))
+                              weight_reading, precision, int(serial), int(graphs))
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         n = C.c_size_t()

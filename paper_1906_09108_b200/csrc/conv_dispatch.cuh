@@ -106,9 +106,12 @@ inline cudaError_t cached_weight_map(TensorMapCache* cache, const void* wgt, int
 }
 
 // out = conv3x3(act, wgt) [+ res * [mask > 0]]; act [N][H][W][Ck], wgt [Cn][9*Ck], out [N][H][W][Cn].
+// `red` (nullable, Cn <= 64 only) asks for a per-channel reduction in the epilogue; its `partial`
+// must hold 2*Cn floats per CTA and its `counter` must be zero.
+inline bool halo_reduce_ok(int Cn) { return Cn <= 64; }
 inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ck, int Cn,
                                  const bf16_t* act, const bf16_t* wgt, bf16_t* out, const bf16_t* res,
-                                 const bf16_t* res_mask, int* err_dev) {
+                                 const bf16_t* res_mask, int* err_dev, const halo::EpiReduce* red = nullptr) {
   const int sms = cached_sm_count(cache);
   halo::FwdParams p = halo::fwd_params(N, H, W, Ck, Cn, sms);
   const CUtensorMap *mx, *mw;
@@ -117,7 +120,9 @@ inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, 
   if (e == cudaSuccess) e = halo::set_smem_attrs();
   if (e != cudaSuccess) return e;
   const int grid = p.tiles < sms ? p.tiles : sms;
-  halo::conv_halo_kernel<<<grid, tc::kThreads, halo::fwd_smem_bytes(p), st>>>(*mx, *mw, p, out, res, res_mask, err_dev);
+  halo::EpiReduce r{};
+  if (red) { if (!halo_reduce_ok(Cn)) return cudaErrorInvalidValue; r = *red; }
+  halo::conv_halo_kernel<<<grid, tc::kThreads, halo::fwd_smem_bytes(p), st>>>(*mx, *mw, p, out, res, res_mask, r, err_dev);
   return cudaGetLastError();
 }
 

@@ -69,12 +69,48 @@ __device__ __forceinline__ uint32_t instr_desc(int n, bool mn_major) {
   return d;
 }
 
+// Optional per-channel reduction over the tensor the kernel stores, taken in its epilogue (on
+// the values as stored, i.e. after rounding to bf16):
+//   mode 1  batch-norm statistics of the output:  sum v, sum v^2  ->  stats = (mean, 1/sqrt(var + eps))
+//   mode 2  the two sums of the batch-norm backward the output feeds as its upstream gradient:
+//           dz = v * [mask > 0],  sum dz,  sum dz * xhat  with xhat = (xprev - mean) * invstd
+//           -> sums, and the parameter gradients dbeta = sum dz, dgamma = sum dz * xhat
+// Every CTA writes its sums to partial[cta][2*Cn]; the CTA that finishes last adds them in CTA
+// order (fp64), so the result does not depend on scheduling.  Cn <= 64 only.
+struct EpiReduce {
+  int mode;
+  const __nv_bfloat16* mask;
+  const __nv_bfloat16* xprev;
+  const float* pstats;        // mode 2: mean[Cn], invstd[Cn] of xprev's batch norm
+  float* partial;             // [gridDim.x][2*Cn]
+  unsigned int* counter;      // zero before the launch; left at zero
+  float* out;                 // mode 1: stats[2*Cn]; mode 2: sums[2*Cn]
+  float* dgamma;              // mode 2 (Cn each)
+  float* dbeta;
+  float eps, inv_count;       // mode 1: 1 / (pixels per channel)
+};
+constexpr int kRedSmemBytes = 4 * 8 * 32 * 4 + 2 * 128 * 4 + 192 * 8;   // running sums, statistics, finalisation
+
+// 32 lanes each hold 32 items; afterwards lane l holds in q[0] the sum over all lanes of item l.
+__device__ __forceinline__ void transpose_reduce32(float (&q)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < off; ++i) {
+      const float send = upper ? q[i] : q[i + off];
+      const float keep = upper ? q[i + off] : q[i];
+      q[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+}
+
 // ------------------------------------------------------- forward / data gradient --
 // out[pixel][n] (bf16, row stride Cn) = conv + (res ? res * [mask ? mask > 0 : 1] : 0)
 __global__ void __launch_bounds__(kThreads, 1)
 conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, FwdParams p,
                  __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
-                 const __nv_bfloat16* __restrict__ res_mask, int* __restrict__ error_word) {
+                 const __nv_bfloat16* __restrict__ res_mask, EpiReduce red, int* __restrict__ error_word) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* w_smem = smem + (size_t)p.stages * p.stage_bytes;
@@ -86,8 +122,16 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   uint64_t* acc_empty = acc_full + p.nacc;     // [nacc]    epilogue -> MMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + p.nacc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* red_run = reinterpret_cast<float*>(tmem_slot + 4);          // [4 warps][8 chunks][32 items]
+  float* red_stat = red_run + 4 * 8 * 32;                            // mode 2: mean[Cn], invstd[Cn]
+  double* red_fin = reinterpret_cast<double*>(red_stat + 2 * 128);   // [192]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (red.mode) {
+    for (int i = threadIdx.x; i < 4 * 8 * 32; i += kThreads) red_run[i] = 0.f;
+    if (red.mode == 2)
+      for (int i = threadIdx.x; i < 2 * p.Cn; i += kThreads) red_stat[i] = red.pstats[i];
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(w_full, 1);
@@ -183,42 +227,75 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
           uint32_t v[16];
           tmem_ld16(taddr + c0, v);
           tmem_ld_wait();
-          if (!valid) continue;
           float f[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]);
-          if (res) {
-            uint4 r0 = *reinterpret_cast<const uint4*>(res + base + c0);
-            uint4 r1 = *reinterpret_cast<const uint4*>(res + base + c0 + 8);
-            const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
-            const __nv_bfloat16* rb1 = reinterpret_cast<const __nv_bfloat16*>(&r1);
-            float gq[16];
+          if (valid) {
+            if (res) {
+              uint4 r0 = *reinterpret_cast<const uint4*>(res + base + c0);
+              uint4 r1 = *reinterpret_cast<const uint4*>(res + base + c0 + 8);
+              const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
+              const __nv_bfloat16* rb1 = reinterpret_cast<const __nv_bfloat16*>(&r1);
+              float gq[16];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) { gq[e] = __bfloat162float(rb0[e]); gq[8 + e] = __bfloat162float(rb1[e]); }
-            if (res_mask) {
-              uint4 m0 = *reinterpret_cast<const uint4*>(res_mask + base + c0);
-              uint4 m1 = *reinterpret_cast<const uint4*>(res_mask + base + c0 + 8);
+              for (int e = 0; e < 8; ++e) { gq[e] = __bfloat162float(rb0[e]); gq[8 + e] = __bfloat162float(rb1[e]); }
+              if (res_mask) {
+                uint4 m0 = *reinterpret_cast<const uint4*>(res_mask + base + c0);
+                uint4 m1 = *reinterpret_cast<const uint4*>(res_mask + base + c0 + 8);
+                const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&m0);
+                const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&m1);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  if (!(__bfloat162float(mb0[e]) > 0.f)) gq[e] = 0.f;
+                  if (!(__bfloat162float(mb1[e]) > 0.f)) gq[8 + e] = 0.f;
+                }
+              }
+#pragma unroll
+              for (int e = 0; e < 16; ++e) f[e] += gq[e];
+            }
+            uint4 o0, o1;
+            __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
+            __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              ob0[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+              ob1[e] = __floats2bfloat162_rn(f[8 + 2 * e], f[8 + 2 * e + 1]);
+            }
+            *reinterpret_cast<uint4*>(out + base + c0) = o0;
+            *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+          }
+          if (red.mode) {
+            float q[32];
+            if (red.mode == 1) {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                const float sv = valid ? __bfloat162float(__float2bfloat16_rn(f[e])) : 0.f;
+                q[e] = sv; q[16 + e] = sv * sv;
+              }
+            } else {
+              uint4 m0 = make_uint4(0, 0, 0, 0), m1 = m0, x0 = m0, x1 = m0;
+              if (valid) {
+                m0 = *reinterpret_cast<const uint4*>(red.mask + base + c0);
+                m1 = *reinterpret_cast<const uint4*>(red.mask + base + c0 + 8);
+                x0 = *reinterpret_cast<const uint4*>(red.xprev + base + c0);
+                x1 = *reinterpret_cast<const uint4*>(red.xprev + base + c0 + 8);
+              }
               const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&m0);
               const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&m1);
+              const __nv_bfloat16* xb0 = reinterpret_cast<const __nv_bfloat16*>(&x0);
+              const __nv_bfloat16* xb1 = reinterpret_cast<const __nv_bfloat16*>(&x1);
 #pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                if (!(__bfloat162float(mb0[e]) > 0.f)) gq[e] = 0.f;
-                if (!(__bfloat162float(mb1[e]) > 0.f)) gq[8 + e] = 0.f;
+              for (int e = 0; e < 16; ++e) {
+                const float mk = __bfloat162float(e < 8 ? mb0[e] : mb1[e - 8]);
+                const float xp = __bfloat162float(e < 8 ? xb0[e] : xb1[e - 8]);
+                const float dz = (valid && mk > 0.f) ? __bfloat162float(__float2bfloat16_rn(f[e])) : 0.f;
+                q[e] = dz;
+                q[16 + e] = dz * ((xp - red_stat[c0 + e]) * red_stat[p.Cn + c0 + e]);
               }
             }
-#pragma unroll
-            for (int e = 0; e < 16; ++e) f[e] += gq[e];
+            transpose_reduce32(q, lane);
+            red_run[((warp - 2) * 8 + (c0 >> 4)) * 32 + lane] += q[0];
           }
-          uint4 o0, o1;
-          __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
-          __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            ob0[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
-            ob1[e] = __floats2bfloat162_rn(f[8 + 2 * e], f[8 + 2 * e + 1]);
-          }
-          *reinterpret_cast<uint4*>(out + base + c0) = o0;
-          *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
         }
         tc_fence_before();
         __syncwarp();
@@ -246,6 +323,56 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+  if (red.mode && !*abort_flag) {
+    // this CTA's sums: item (chunk, lane) of the four epilogue warps -> partial[cta][stat][channel]
+    const int pairs = 2 * p.Cn;
+    for (int t = threadIdx.x; t < pairs; t += kThreads) {
+      const int stat = t / p.Cn, c = t - stat * p.Cn;
+      const int idx = (c >> 4) * 32 + (c & 15) + 16 * stat;
+      red.partial[(size_t)blockIdx.x * pairs + t] = red_run[idx] + red_run[8 * 32 + idx] + red_run[2 * 8 * 32 + idx] + red_run[3 * 8 * 32 + idx];
+    }
+    __threadfence();
+    __syncthreads();
+    __shared__ bool is_last;
+    if (threadIdx.x == 0) is_last = atomicInc(red.counter, gridDim.x - 1) == gridDim.x - 1;
+    __syncthreads();
+    if (is_last) {
+      __threadfence();
+      // Cn <= 64, so pairs <= 128 <= kThreads: nseg threads share one (stat, channel) pair, each
+      // taking every nseg-th CTA with 8 loads in flight; their sums are then added in segment order.
+      const int nseg = kThreads / pairs;
+      const int t = threadIdx.x % pairs, seg = threadIdx.x / pairs;
+      double a = 0.0;
+      if (seg < nseg)
+        for (unsigned b0 = seg; b0 < gridDim.x; b0 += 8 * nseg) {
+          float v[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const unsigned b = b0 + u * nseg;
+            v[u] = b < gridDim.x ? __ldcg(&red.partial[(size_t)b * pairs + t]) : 0.f;
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) a += (double)v[u];
+        }
+      red_fin[threadIdx.x] = a;
+      __syncthreads();
+      if ((int)threadIdx.x < p.Cn) {
+        const int c = threadIdx.x;
+        double s0 = 0.0, s1 = 0.0;
+        for (int q = 0; q < nseg; ++q) { s0 += red_fin[q * pairs + c]; s1 += red_fin[q * pairs + p.Cn + c]; }
+        if (red.mode == 1) {
+          const double mean = s0 * (double)red.inv_count;
+          double var = s1 * (double)red.inv_count - mean * mean;
+          if (var < 0.0) var = 0.0;
+          red.out[c] = (float)mean;
+          red.out[p.Cn + c] = (float)(1.0 / sqrt(var + (double)red.eps));
+        } else {
+          red.out[c] = (float)s0; red.out[p.Cn + c] = (float)s1;
+          red.dbeta[c] = (float)s0; red.dgamma[c] = (float)s1;
+        }
+      }
+    }
   }
 }
 
@@ -450,7 +577,8 @@ inline FwdParams fwd_params(int N, int H, int W, int Ck, int Cn, int sm_count) {
 }
 
 inline size_t fwd_smem_bytes(const FwdParams& p) {
-  return (size_t)p.stages * p.stage_bytes + 9 * (size_t)p.w_tap_bytes + (size_t)(2 * p.stages + 1 + 2 * p.nacc) * 8 + 16 + 1024;
+  return (size_t)p.stages * p.stage_bytes + 9 * (size_t)p.w_tap_bytes + (size_t)(2 * p.stages + 1 + 2 * p.nacc) * 8 + 16 +
+         kRedSmemBytes + 1024;
 }
 
 inline bool fwd_supported(int N, int H, int W, int Ck, int Cn) {

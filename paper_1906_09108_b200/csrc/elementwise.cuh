@@ -80,9 +80,16 @@ inline RedGeom red_geom(int rows, int C, int vec) {
 
 // Block-level part: NS sums per channel -> partial[block][NS][C]; the last block to
 // finish adds the partials in block order (fp64) and calls `fin(c, sums[NS])`.
+// The dynamic shared memory of the reduction kernels, reused as doubles for the final totals
+// (NS*C doubles <= rp*NS*C floats whenever rp >= 2; the launchers reserve at least that).
+__device__ __forceinline__ double* red_smem_d() {
+  extern __shared__ double red_smem_as_double[];
+  return red_smem_as_double;
+}
+
 template <int NS, int VEC, typename Acc, typename Fin>
 __device__ __forceinline__ void channel_reduce(const RedGeom g, float* __restrict__ partial,
-                                               unsigned int* __restrict__ counter, Acc acc, Fin fin) {
+                                               unsigned int* __restrict__ counter, Acc acc, Fin fin_fn) {
   extern __shared__ float red_smem[];                        // [rp][NS][C]
   __shared__ bool is_last;
   const int tid = threadIdx.x;
@@ -115,15 +122,40 @@ __device__ __forceinline__ void channel_reduce(const RedGeom g, float* __restric
   __syncthreads();
   if (!is_last) return;
   __threadfence();
+  // NS*C (sum, channel) pairs; kRedThreads / pairs threads share a pair, each taking every
+  // nseg-th block with 8 loads in flight; the segment sums are then added in segment order.
+  __shared__ double fin[kRedThreads];
+  const int pairs = NS * C;
+  for (int p0 = 0; p0 < pairs; p0 += kRedThreads) {
+    const int np = min(pairs - p0, kRedThreads);
+    const int nseg = kRedThreads / np;
+    const int t = tid % np, seg = tid / np;
+    double a = 0.0;
+    if (seg < nseg)
+      for (unsigned b0 = seg; b0 < gridDim.x; b0 += 8 * nseg) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const unsigned b = b0 + u * nseg;
+          v[u] = b < gridDim.x ? __ldcg(&partial[(size_t)b * pairs + p0 + t]) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) a += (double)v[u];
+      }
+    fin[tid] = a;
+    __syncthreads();
+    if (tid < np) {
+      double tot = 0.0;
+      for (int q = 0; q < nseg; ++q) tot += fin[q * np + tid];
+      red_smem_d()[p0 + tid] = tot;
+    }
+    __syncthreads();
+  }
   for (int c = tid; c < C; c += blockDim.x) {
     double tot[NS];
 #pragma unroll
-    for (int s = 0; s < NS; ++s) {
-      double a = 0.0;
-      for (unsigned b = 0; b < gridDim.x; ++b) a += (double)__ldcg(&partial[(size_t)b * NS * C + s * C + c]);
-      tot[s] = a;
-    }
-    fin(c, tot);
+    for (int s = 0; s < NS; ++s) tot[s] = red_smem_d()[s * C + c];
+    fin_fn(c, tot);
   }
 }
 
@@ -404,9 +436,12 @@ __global__ void head_param_grad_kernel(const float* __restrict__ pooled, const f
 // g' = g + wd*theta ; v = mu*v + g' ; theta -= lr*v   (v starts at 0, so the first
 // update gives v = g').  Also writes the copies of theta the kernels compute with into
 // the next weight-version slot: fp32 always, bf16 when next16 is given.  g is left untouched.
+// The learning rate is `lr`, or *lr_dev when that pointer is given (a recorded launch can then
+// follow a schedule without being re-recorded).
 __global__ void sgd_kernel(float* __restrict__ theta, float* __restrict__ v, const float* __restrict__ g,
                            float* __restrict__ next32, __nv_bfloat16* __restrict__ next16, size_t n, float lr,
-                           float mu, float wd) {
+                           const float* __restrict__ lr_dev, float mu, float wd) {
+  if (lr_dev) lr = *lr_dev;
   const size_t n4 = n / 4;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
     float4 th = reinterpret_cast<float4*>(theta)[i];
@@ -436,6 +471,8 @@ __global__ void sgd_kernel(float* __restrict__ theta, float* __restrict__ v, con
       if (next16) next16[i] = __float2bfloat16_rn(th);
     }
 }
+
+__global__ void set_scalar_kernel(float* dst, float value) { *dst = value; }
 
 // fp32 -> T copy (refreshing the compute copies after fdg_set_params).
 template <typename T>

@@ -33,8 +33,8 @@ namespace fdg {
 
 typedef __nv_bfloat16 bf16;
 constexpr int kEventRing = 4;
-constexpr int kMailRing = 3;
 constexpr size_t kLogIterations = 4096;
+constexpr int kRedPartialCtas = 256;                 // upper bound of the CTAs of one convolution launch
 
 enum UnitType { U_STEM, U_BASIC, U_PREACT, U_HEAD };
 
@@ -90,6 +90,8 @@ struct Module {
   char* temps[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   float *scratch = nullptr, *bnsums = nullptr;
   unsigned int* counter = nullptr;
+  float* red_partial = nullptr;            // per-CTA partial sums of the reductions fused into convolution epilogues
+  unsigned int* red_counter = nullptr;
   float *pooled = nullptr, *dlogits = nullptr, *loss_n = nullptr, *loss = nullptr;   // head
   // host state
   int64_t updates = 0;
@@ -130,6 +132,21 @@ struct fdg_ctx {
   fdg_status latched = FDG_OK;
   int device = 0;
   fdg::TensorMapCache tmaps;
+  // ring sizes that do not depend on the module
+  int mail_ring = 3;
+  // CUDA-graph replay (cfg.graphs): one executable graph per phase of the rings
+  bool use_graphs = false;
+  int period = 1;                     // all ring sizes divide it
+  bool graph_mode_entered = false;
+  std::vector<cudaGraphExec_t> graph_exec;
+  std::vector<uint64_t> graph_sig, graph_launches;
+  uint64_t step_sig = 0;              // signature of the slots the current iteration touches
+  cudaStream_t cap_stream = nullptr;  // origin stream of the recordings (the caller's stream may be the legacy
+                                      // default stream, which cannot be captured); graphs are launched on the caller's
+  cudaEvent_t ev_fork = nullptr;
+  std::vector<cudaEvent_t> ev_cjoin;
+  float* lr_dev = nullptr;
+  float lr_on_device = -1.f;
   int* tc_error = nullptr;            // device word raised by a tensor-core kernel whose wait timed out
   cudaStream_t last_stream = nullptr;   // stream of the most recent fdg_step
   bool stepped = false;
@@ -157,6 +174,7 @@ struct Carver {
 };
 
 static int conv_out(int n, int r, int stride, int pad) { return (n + 2 * pad - r) / stride + 1; }
+static int pow2_at_least(int x) { int p = 1; while (p < x) p <<= 1; return p; }
 
 static fdg_status validate(const fdg_arch* a, const fdg_config* c, std::string* why) {
   if (!a || !c) { *why = "null arch or config"; return FDG_ERR_INVALID_ARG; }
@@ -268,6 +286,11 @@ static void plan_modules(fdg_ctx* c) {
     m.D = (kp == K) ? 1 : 2 * (K - kp) + (c->cfg.order == FDG_FORWARD_FIRST ? 1 : 0);
     m.Dw = (kp == K) ? 1 : 2 * (K - kp) + 1;
     m.Din = (kp == 1) ? m.D + 2 : 0;
+    if (c->use_graphs) {      // powers of two, so that every ring's phase is a function of t mod period
+      m.D = pow2_at_least(m.D); m.Dw = pow2_at_least(m.Dw);
+      if (m.Din) m.Din = pow2_at_least(m.Din);
+      c->period = std::max(c->period, std::max(m.D, std::max(m.Dw, m.Din)));
+    }
     m.in_elems = B * m.in_h * m.in_w * m.in_c;
     size_t te = 0, tf = 0, maxa = m.in_elems, scr = 0;
     auto tens = [&](size_t e) { size_t o = te; te += align_up(e, 128); maxa = std::max(maxa, e); return o; };
@@ -340,7 +363,10 @@ static size_t carve(fdg_ctx* c, char* base) {
   const size_t es = c->esize;
   c->flags = cv.take<int>(256);
   c->tc_error = c->flags ? c->flags + 2 : nullptr;
-  c->label_ring = 2 * c->K + 2;
+  c->label_ring = c->use_graphs ? pow2_at_least(c->K + 2) : 2 * c->K + 2;
+  c->mail_ring = c->use_graphs ? 4 : 3;
+  if (c->use_graphs) c->period = std::max(c->period, std::max(c->label_ring, c->mail_ring));
+  c->lr_dev = cv.take<float>(256);
   c->labels = cv.take<int32_t>((size_t)c->label_ring * c->arch.batch * sizeof(int32_t));
   size_t stage = 0;
   for (Module& m : c->mods) {
@@ -354,13 +380,15 @@ static size_t carve(fdg_ctx* c, char* base) {
     m.fifo = cv.take<char>((size_t)m.D * m.slot_elems * es);
     m.fifo_f = cv.take<float>((size_t)m.D * std::max<size_t>(m.slot_floats, 64) * 4);
     m.in_ring = m.Din ? cv.take<char>((size_t)m.Din * align_up(m.in_elems, 128) * es) : nullptr;
-    m.mail = m.k >= 2 ? cv.take<char>((size_t)kMailRing * align_up(m.in_elems, 128) * es) : nullptr;
+    m.mail = m.k >= 2 ? cv.take<char>((size_t)c->mail_ring * align_up(m.in_elems, 128) * es) : nullptr;
     for (int i = 0; i < 5; ++i) m.temps[i] = cv.take<char>(align_up(m.max_act, 128) * es);
     m.scratch = cv.take<float>(std::max<size_t>(m.scratch_floats, 64) * 4);
     int maxc = 1;
     for (const Unit& u : m.units) maxc = std::max(maxc, std::max(u.ci, u.co));
     m.bnsums = cv.take<float>((size_t)kRedMaxSums * maxc * 4);
     m.counter = cv.take<unsigned int>(256);
+    m.red_partial = cv.take<float>((size_t)kRedPartialCtas * 2 * 64 * 4);
+    m.red_counter = cv.take<unsigned int>(256);
     if (m.k == c->K) {
       const Unit& h = m.units.back();
       m.pooled = cv.take<float>((size_t)c->arch.batch * h.ci * 4);
@@ -419,10 +447,10 @@ static void bn_stats(Launch& L, Module& m, const T* x, size_t rows, int C, float
   L.begin(KC_BN_STATS, (double)rows * C * sizeof(T), 3.0 * rows * C);
   if (C % V == 0) {
     RedGeom g = red_geom((int)rows, C, V);
-    bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)g.rp * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
+    bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)std::max(g.rp, 2) * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
   } else {
     RedGeom g = red_geom((int)rows, C, 1);
-    bn_stats_kernel<T, 1><<<g.blocks, kRedThreads, (size_t)g.rp * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
+    bn_stats_kernel<T, 1><<<g.blocks, kRedThreads, (size_t)std::max(g.rp, 2) * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
   }
   L.check();
 }
@@ -447,20 +475,22 @@ template <typename T>
 static void bn_backward(Launch& L, Module& m, const T* dy, const T* mask, const T* x, const float* stats,
                         const float* gamma, float* dgamma, float* dbeta, const T* x2, const float* stats2,
                         const float* gamma2, float* dgamma2, float* dbeta2, const T* res, T* dx, T* dx2,
-                        size_t rows, int C) {
+                        size_t rows, int C, bool sums_ready = false) {
   constexpr int V = full_vec<T>();
   const bool two = x2 != nullptr;
   const int ns = two ? 3 : 2;
   const bool vec = C % V == 0;
-  RedGeom g = red_geom((int)rows, C, vec ? V : 1);
-  const size_t smem = (size_t)g.rp * ns * C * 4;
+  if (!sums_ready) {      // otherwise the kernel that produced dy already left the sums in m.bnsums
+    RedGeom g = red_geom((int)rows, C, vec ? V : 1);
+    const size_t smem = (size_t)std::max(g.rp, 2) * ns * C * 4;
 #define FDG_RED(VV, NS) bn_bwd_reduce_kernel<T, VV, NS><<<g.blocks, kRedThreads, smem, L.st>>>( \
       dy, mask, x, stats, x2, stats2, g, m.bnsums, dgamma, dbeta, dgamma2, dbeta2, m.scratch, m.counter)
-  L.begin(KC_BN_BWD_REDUCE, (double)rows * C * sizeof(T) * (2 + (mask ? 1 : 0) + (two ? 1 : 0)), 8.0 * rows * C);
-  if (vec) { if (two) FDG_RED(V, 3); else FDG_RED(V, 2); }
-  else     { if (two) FDG_RED(1, 3); else FDG_RED(1, 2); }
+    L.begin(KC_BN_BWD_REDUCE, (double)rows * C * sizeof(T) * (2 + (mask ? 1 : 0) + (two ? 1 : 0)), 8.0 * rows * C);
+    if (vec) { if (two) FDG_RED(V, 3); else FDG_RED(V, 2); }
+    else     { if (two) FDG_RED(1, 3); else FDG_RED(1, 2); }
 #undef FDG_RED
-  L.check();
+    L.check();
+  }
   const size_t n = rows * C;
   const float inv_m = 1.f / (float)rows;
   L.begin(KC_BN_BWD_APPLY, (double)n * sizeof(T) * (3 + (mask ? 1 : 0) + (two ? 2 : 0) + (res ? 1 : 0)), 10.0 * n);
@@ -493,41 +523,63 @@ static double in_elems(const ConvGeom& g) { return (double)g.N * g.H * g.W * g.C
 static double out_elems(const ConvGeom& g) { return (double)g.N * g.P * g.Q * g.Co; }
 static double w_elems(const ConvGeom& g) { return (double)g.Co * g.R * g.S * g.Ci; }
 
+// `stats` (nullable): where the batch-norm statistics (mean, 1/sigma) of y should go.  Returns true
+// when the convolution kernel produced them in its epilogue; otherwise the caller runs bn_stats.
 template <typename T>
-static void conv_fprop(Launch& L, const ConvGeom& g, const T* x, const T* w, T* y, const T* res) {
+static bool conv_fprop(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* w, T* y, const T* res,
+                       float* stats = nullptr) {
   L.begin(KC_CONV_FPROP, (in_elems(g) + w_elems(g) + out_elems(g) * (res ? 2 : 1)) * sizeof(T), conv_flops(g));
   if constexpr (std::is_same<T, bf16>::value) {
     if (halo_fprop_eligible(g)) {
       ++L.c->launches;
-      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error));
-      return;
+      const bool fuse = stats && halo_reduce_ok(g.Co);
+      halo::EpiReduce r{};
+      if (fuse) {
+        r.mode = 1; r.partial = m.red_partial; r.counter = m.red_counter; r.out = stats;
+        r.eps = L.c->arch.bn_eps; r.inv_count = 1.f / ((float)g.N * g.P * g.Q);
+      }
+      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, fuse ? &r : nullptr));
+      return fuse;
     }
     if (tc_eligible(g)) {
       ++L.c->launches;
       L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error));
-      return;
+      return false;
     }
   }
   L.note(launch_conv_simt<T, CONV_FPROP>(L.st, g, x, w, y, nullptr, nullptr, res, (const T*)nullptr, &L.c->launches));
+  return false;
 }
 // `wflip` is the flipped/transposed weight copy (bf16 mode, tensor-core eligible shapes) or null.
+// The batch-norm backward that will consume dx as its upstream gradient: dz = dx * [mask > 0],
+// xhat from (x, stats).  When the data-gradient kernel can, it forms that backward's two sums
+// (and the parameter gradients) in its epilogue and conv_dgrad returns true.
+template <typename T> struct NextBnBwd { const T* mask; const T* x; const float* stats; float* dgamma; float* dbeta; };
+
 template <typename T>
-static void conv_dgrad(Launch& L, const ConvGeom& g, const T* dy, const T* w, const T* wflip, T* dx, const T* res,
-                       const T* mask) {
-  L.begin(KC_CONV_DGRAD, (out_elems(g) + w_elems(g) + in_elems(g) * (1 + (res ? 1 : 0) + (mask ? 1 : 0))) * sizeof(T), conv_flops(g));
+static bool conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, const T* w, const T* wflip, T* dx,
+                       const T* res, const T* mask, const NextBnBwd<T>* next = nullptr) {
+  L.begin(KC_CONV_DGRAD, (out_elems(g) + w_elems(g) + in_elems(g) * (1 + (res ? 1 : 0) + (mask ? 1 : 0) + (next ? 2 : 0))) * sizeof(T), conv_flops(g));
   if constexpr (std::is_same<T, bf16>::value) {
     if (wflip && halo_dgrad_eligible(g)) {
       ++L.c->launches;
-      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error));
-      return;
+      const bool fuse = next && halo_reduce_ok(g.Ci);
+      halo::EpiReduce r{};
+      if (fuse) {
+        r.mode = 2; r.mask = next->mask; r.xprev = next->x; r.pstats = next->stats; r.partial = m.red_partial;
+        r.counter = m.red_counter; r.out = m.bnsums; r.dgamma = next->dgamma; r.dbeta = next->dbeta;
+      }
+      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error, fuse ? &r : nullptr));
+      return fuse;
     }
     if (wflip && tc_eligible(g)) {
       ++L.c->launches;
       L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error));
-      return;
+      return false;
     }
   }
   L.note(launch_conv_simt<T, CONV_DGRAD>(L.st, g, dy, w, dx, nullptr, nullptr, res, mask, &L.c->launches));
+  return false;
 }
 template <typename T>
 static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* dy, float* dw) {
@@ -576,26 +628,26 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
       case U_STEM: {
         ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
         if (u.bn) {
-          conv_fprop<T>(L, g, x, wt + u.w1, S + u.t_a, nullptr);
-          bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
+          if (!conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_a, nullptr, F + u.st1))
+            bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
           bn_apply<T>(L, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co);
         } else {
-          conv_fprop<T>(L, g, x, wt + u.w1, S + u.t_y, nullptr);
+          conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_y, nullptr);
         }
         break;
       }
       case U_BASIC: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
-        conv_fprop<T>(L, g1, x, wt + u.w1, S + u.t_a, nullptr);                                        // c1
-        bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
+        if (!conv_fprop<T>(L, m, g1, x, wt + u.w1, S + u.t_a, nullptr, F + u.st1))                      // c1
+          bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
         bn_apply<T>(L, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_b, rows_out, u.co);  // a1
-        conv_fprop<T>(L, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr);                                // c2
-        bn_stats<T>(L, m, S + u.t_c, rows_out, u.co, eps, F + u.st2);
+        if (!conv_fprop<T>(L, m, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr, F + u.st2))              // c2
+          bn_stats<T>(L, m, S + u.t_c, rows_out, u.co, eps, F + u.st2);
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
-          conv_fprop<T>(L, gs, x, wt + u.ws, S + u.t_s, nullptr);                                      // cs
-          bn_stats<T>(L, m, S + u.t_s, rows_out, u.co, eps, F + u.sts);
+          if (!conv_fprop<T>(L, m, gs, x, wt + u.ws, S + u.t_s, nullptr, F + u.sts))                    // cs
+            bn_stats<T>(L, m, S + u.t_s, rows_out, u.co, eps, F + u.sts);
           bn_apply<T>(L, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, S + u.t_s, F + u.sts, wf + u.gs, wf + u.bs, true, S + u.t_y, rows_out, u.co);
         } else {
           bn_apply<T>(L, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, x, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co);
@@ -607,15 +659,15 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
         bn_stats<T>(L, m, x, rows_in, u.ci, eps, F + u.st1);
         bn_apply<T>(L, x, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows_in, u.ci);   // o
-        conv_fprop<T>(L, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr);                                // c1
-        bn_stats<T>(L, m, S + u.t_b, rows_out, u.co, eps, F + u.st2);
+        if (!conv_fprop<T>(L, m, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr, F + u.st2))              // c1
+          bn_stats<T>(L, m, S + u.t_b, rows_out, u.co, eps, F + u.st2);
         bn_apply<T>(L, S + u.t_b, F + u.st2, wf + u.g2, wf + u.b2, nullptr, nullptr, nullptr, nullptr, true, S + u.t_c, rows_out, u.co); // a2
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
-          conv_fprop<T>(L, gs, S + u.t_a, wt + u.ws, tmp, nullptr);
-          conv_fprop<T>(L, g2, S + u.t_c, wt + u.w2, S + u.t_y, tmp);
+          conv_fprop<T>(L, m, gs, S + u.t_a, wt + u.ws, tmp, nullptr);
+          conv_fprop<T>(L, m, g2, S + u.t_c, wt + u.w2, S + u.t_y, tmp);
         } else {
-          conv_fprop<T>(L, g2, S + u.t_c, wt + u.w2, S + u.t_y, x);
+          conv_fprop<T>(L, m, g2, S + u.t_c, wt + u.w2, S + u.t_y, x);
         }
         break;
       }
@@ -674,6 +726,7 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
   T* T2 = reinterpret_cast<T*>(m.temps[3]);
   T* T3 = reinterpret_cast<T*>(m.temps[4]);
   T* dy = gin;
+  bool dy_sums_ready = false;      // the kernel that produced dy also left the first batch-norm backward's sums
   const int nu = (int)m.units.size();
   for (int i = nu - 1; i >= 0; --i) {
     const Unit& u = m.units[i];
@@ -681,13 +734,23 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
     const T* x = i > 0 ? S + m.units[i - 1].t_y : module_input<T>(c, m, tau);
     T* gout = (i == 0) ? gfirst : (dy == G[0] ? G[1] : G[0]);
     const size_t rows_in = (size_t)B * u.H * u.W, rows_out = (size_t)B * u.P * u.Q;
+    // The batch-norm backward that unit i-1 will start with, if its sums can be formed by the
+    // data-gradient kernel that writes this unit's input gradient.
+    NextBnBwd<T> nb{};
+    const NextBnBwd<T>* next = nullptr;
+    if (i > 0) {
+      const Unit& pu = m.units[i - 1];
+      if (pu.type == U_BASIC && !pu.proj) { nb = {S + pu.t_y, S + pu.t_c, F + pu.st2, m.grad + pu.g2, m.grad + pu.b2}; next = &nb; }
+      if (pu.type == U_STEM && pu.bn) { nb = {S + pu.t_y, S + pu.t_a, F + pu.st1, m.grad + pu.g1, m.grad + pu.b1}; next = &nb; }
+    }
+    bool out_sums_ready = false;
     switch (u.type) {
       case U_STEM: {
         ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
         const T* dc = dy;
         if (u.bn) {
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
-                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co);
+                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sums_ready);
           dc = T1;
         }
         conv_wgrad<T>(L, m, g, x, dc, m.grad + u.w1);
@@ -701,22 +764,23 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
                          F + u.sts, wf + u.gs, m.grad + u.gs, m.grad + u.bs, nullptr, T1, T2, rows_out, u.co);
         else
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_c, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
-                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co);
+                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sums_ready);
         conv_wgrad<T>(L, m, g2, S + u.t_b, T1, m.grad + u.w2);
-        conv_dgrad<T>(L, g2, T1, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T3, nullptr, nullptr);      // da1
+        const NextBnBwd<T> bn1{S + u.t_b, S + u.t_a, F + u.st1, m.grad + u.g1, m.grad + u.b1};
+        const bool bn1_ready = conv_dgrad<T>(L, m, g2, T1, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T3, nullptr, nullptr, &bn1);   // da1
         bn_backward<T>(L, m, T3, S + u.t_b, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
-                       nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co);      // dc1
+                       nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, bn1_ready);      // dc1
         conv_wgrad<T>(L, m, g1, x, T1, m.grad + u.w1);
         const bool need_dx = !(m.k == 1 && i == 0);
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_wgrad<T>(L, m, gs, x, T2, m.grad + u.ws);
           if (need_dx) {
-            conv_dgrad<T>(L, gs, T2, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
-            conv_dgrad<T>(L, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr);
+            conv_dgrad<T>(L, m, gs, T2, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
+            out_sums_ready = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next);
           }
         } else if (need_dx) {
-          conv_dgrad<T>(L, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y);
+          out_sums_ready = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y, next);
         }
         break;
       }
@@ -724,17 +788,17 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
         conv_wgrad<T>(L, m, g2, S + u.t_c, dy, m.grad + u.w2);
-        conv_dgrad<T>(L, g2, dy, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T1, nullptr, nullptr);      // da2
+        conv_dgrad<T>(L, m, g2, dy, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T1, nullptr, nullptr);   // da2
         bn_backward<T>(L, m, T1, S + u.t_c, S + u.t_b, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
                        nullptr, nullptr, nullptr, nullptr, nullptr, T2, nullptr, rows_out, u.co);      // dc1
         conv_wgrad<T>(L, m, g1, S + u.t_a, T2, m.grad + u.w1);
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_wgrad<T>(L, m, gs, S + u.t_a, dy, m.grad + u.ws);
-          conv_dgrad<T>(L, gs, dy, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
-          conv_dgrad<T>(L, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, T3, nullptr);         // do
+          conv_dgrad<T>(L, m, gs, dy, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
+          conv_dgrad<T>(L, m, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, T3, nullptr);      // do
         } else {
-          conv_dgrad<T>(L, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, nullptr, nullptr);
+          conv_dgrad<T>(L, m, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, nullptr, nullptr);
         }
         bn_backward<T>(L, m, T1, S + u.t_a, x, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr, nullptr,
                        nullptr, nullptr, nullptr, u.proj ? nullptr : dy, gout, nullptr, rows_in, u.ci);
@@ -743,6 +807,7 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
       default: break;
     }
     dy = gout;
+    dy_sums_ready = out_sums_ready;
   }
 }
 
@@ -753,7 +818,8 @@ static void update_module(fdg_ctx* c, Module& m, Launch& L, int next_vslot) {
   bf16* next16 = c->bf16_mode ? m.wver16 + (size_t)next_vslot * align_up(n, 64) : nullptr;
   int blocks = (int)std::min<size_t>(std::max<size_t>((n / 4 + 255) / 256, 1), 148 * 8);
   L.begin(KC_SGD, (double)n * (24 + (next16 ? 2 : 0)), 6.0 * n);
-  sgd_kernel<<<blocks, 256, 0, L.st>>>(m.theta, m.mom, m.grad, next32, next16, n, c->lr, c->cfg.momentum, c->cfg.weight_decay);
+  sgd_kernel<<<blocks, 256, 0, L.st>>>(m.theta, m.mom, m.grad, next32, next16, n, c->lr,
+                                       c->graph_mode_entered ? c->lr_dev : nullptr, c->cfg.momentum, c->cfg.weight_decay);
   L.check();
   if (m.flip_table_dev) {
     L.begin(KC_SGD, 4.0 * m.flip_elems, 0.0);
@@ -762,32 +828,44 @@ static void update_module(fdg_ctx* c, Module& m, Launch& L, int next_vslot) {
   }
 }
 
+// How a module-step is issued.
+//   STREAMS  on the module's own stream, ordered against its neighbours by the events of iteration t-1
+//   SERIAL   on the caller's stream, modules one after the other
+//   CAPTURE  on the module's own stream while an iteration is being recorded into a graph: the
+//            iteration's graph follows the previous iteration's on the caller's stream, so nothing has
+//            to be waited for; the loss is copied by the caller afterwards
+//   DRY      nothing is enqueued; only the host-side bookkeeping advances (a recorded graph is replayed)
+enum StepMode { RUN_STREAMS, RUN_SERIAL, RUN_CAPTURE, RUN_DRY };
+
 // One module-step of module m in iteration t (Algorithm I, body of "Parallel for k").
 template <typename T>
-static cudaError_t module_step(fdg_ctx* c, Module& m, cudaStream_t st, bool serial, float* loss_dev) {
+static cudaError_t module_step(fdg_ctx* c, Module& m, cudaStream_t st, StepMode mode, float* loss_dev) {
   const int K = c->K, k = m.k;
   const int64_t t = c->t;
   const int64_t tau_f = t - k + 1, tau_b = t - 2 * (int64_t)K + k + 1;
   const int e_prev = (int)((t - 1) % kEventRing), e_now = (int)(t % kEventRing);
+  const bool events = mode == RUN_STREAMS, enqueue = mode != RUN_DRY;
   Launch L{c, st};
   fdg_sched_entry row;
   row.t = t; row.k = k; row.tau_f = row.tau_b = row.ver_f = row.ver_b = -1; row.slot_f = row.slot_b = -1;
+  auto sig = [&](int64_t v) { c->step_sig = c->step_sig * 1000003ull + (uint64_t)(v + 7); };
 
   auto wait_act = [&]() {
-    if (serial) return;
+    if (!events) return;
     if (k == 1) L.note(cudaStreamWaitEvent(st, c->ev_in[e_now], 0));
     else L.note(cudaStreamWaitEvent(st, c->mods[k - 2].ev_act[e_prev], 0));
   };
   auto wait_grad = [&]() {
-    if (serial || k == K) return;
+    if (!events || k == K) return;
     L.note(cudaStreamWaitEvent(st, c->mods[k].ev_grad[e_prev], 0));
   };
   auto do_forward = [&]() {
     if (tau_f < 1) return;
     const int slot = (int)(tau_f % m.D), vslot = (int)(m.updates % m.Dw);
-    forward_module<T>(c, m, L, tau_f, slot, vslot);
+    if (enqueue) forward_module<T>(c, m, L, tau_f, slot, vslot);
     m.slot_version[slot] = m.updates; m.slot_batch[slot] = tau_f;
     row.tau_f = tau_f; row.ver_f = m.updates; row.slot_f = slot;
+    sig(slot); sig(vslot); sig(k == 1 ? tau_f % m.Din : 0);
     if (k < K) { m.last_out_batch = tau_f; m.last_out_slot = slot; }
   };
   auto do_backward_update = [&]() {
@@ -795,24 +873,28 @@ static cudaError_t module_step(fdg_ctx* c, Module& m, cudaStream_t st, bool seri
     const int slot = (int)(tau_b % m.D);
     const int64_t ver = (c->cfg.weight_reading == FDG_STASHED) ? m.slot_version[slot] : m.updates;
     const int vslot = (int)(ver % m.Dw);
-    T* gin = reinterpret_cast<T*>(m.temps[0]);
-    if (k < K) {
-      // receive + shrink (Eq. 15): the mailbox of module k+1 holds the gradient it produced at t-1
-      const Module& dn = c->mods[k];
-      const T* recv = reinterpret_cast<const T*>(dn.mail) + (size_t)((t - 1) % kMailRing) * align_up(dn.in_elems, 128);
-      scale_tensor<T>(L, recv, gin, c->cfg.beta, dn.in_elems);
-    } else {
-      head_forward_backward<T>(c, m, L, tau_b, slot, vslot, gin);
-      if (loss_dev) L.note(cudaMemcpyAsync(loss_dev, m.loss, sizeof(float), cudaMemcpyDeviceToDevice, st));
+    const int next_vslot = (int)((m.updates + 1) % m.Dw);
+    sig(slot); sig(vslot); sig(next_vslot); sig(t % c->mail_ring); sig(k == K ? tau_b % c->label_ring : 0);
+    if (enqueue) {
+      T* gin = reinterpret_cast<T*>(m.temps[0]);
+      if (k < K) {
+        // receive + shrink (Eq. 15): the mailbox of module k+1 holds the gradient it produced at t-1
+        const Module& dn = c->mods[k];
+        const T* recv = reinterpret_cast<const T*>(dn.mail) + (size_t)((t - 1) % c->mail_ring) * align_up(dn.in_elems, 128);
+        scale_tensor<T>(L, recv, gin, c->cfg.beta, dn.in_elems);
+      } else {
+        head_forward_backward<T>(c, m, L, tau_b, slot, vslot, gin);
+        if (loss_dev && mode != RUN_CAPTURE) L.note(cudaMemcpyAsync(loss_dev, m.loss, sizeof(float), cudaMemcpyDeviceToDevice, st));
+      }
+      T* gfirst = k >= 2 ? reinterpret_cast<T*>(m.mail) + (size_t)(t % c->mail_ring) * align_up(m.in_elems, 128) : nullptr;
+      backward_module<T>(c, m, L, tau_b, slot, vslot, gin, gfirst);
+      update_module<T>(c, m, L, next_vslot);
     }
-    T* gfirst = k >= 2 ? reinterpret_cast<T*>(m.mail) + (size_t)(t % kMailRing) * align_up(m.in_elems, 128) : nullptr;
-    backward_module<T>(c, m, L, tau_b, slot, vslot, gin, gfirst);
-    update_module<T>(c, m, L, (int)((m.updates + 1) % m.Dw));
     m.updates += 1;
     row.tau_b = tau_b; row.ver_b = ver; row.slot_b = slot;
-    if (k >= 2) { m.last_grad_batch = tau_b; m.last_grad_slot = (int)(t % kMailRing); }
+    if (k >= 2) { m.last_grad_batch = tau_b; m.last_grad_slot = (int)(t % c->mail_ring); }
   };
-  auto rec = [&](cudaEvent_t e) { if (!serial) L.note(cudaEventRecord(e, st)); };
+  auto rec = [&](cudaEvent_t e) { if (events) L.note(cudaEventRecord(e, st)); };
 
   if (k == K) {
     wait_act();
@@ -887,6 +969,8 @@ static fdg_status make_plan(const fdg_arch* arch, const fdg_config* cfg, fdg_ctx
   c->bf16_mode = cfg->precision == FDG_BF16_TC;
   c->esize = c->bf16_mode ? 2 : 4;
   c->lr = cfg->lr;
+  c->use_graphs = cfg->graphs != 0 && cfg->serial == 0;
+  c->period = 1;
   plan_modules(c);
   return FDG_OK;
 }
@@ -931,6 +1015,13 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   }
   for (int i = 0; i < kEventRing && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess && c->use_graphs) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
+  c->ev_cjoin.assign(c->K, nullptr);
+  for (int k = 0; k < c->K && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&c->ev_cjoin[k], cudaEventDisableTiming);
+  c->graph_exec.assign(c->period, nullptr);
+  c->graph_sig.assign(c->period, 0);
+  c->graph_launches.assign(c->period, 0);
   if (e != cudaSuccess) { delete c; return FDG_ERR_CUDA; }
   *out_ctx = c;
   return FDG_OK;
@@ -945,6 +1036,10 @@ fdg_status fdg_destroy(fdg_ctx* c) {
   }
   for (int i = 0; i < kEventRing; ++i) cudaEventDestroy(c->ev_in[i]);
   cudaEventDestroy(c->ev_join);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+  for (cudaEvent_t ev : c->ev_cjoin) if (ev) cudaEventDestroy(ev);
+  for (cudaGraphExec_t g : c->graph_exec) if (g) cudaGraphExecDestroy(g);
   for (cudaEvent_t ev : c->prof_events) cudaEventDestroy(ev);
   delete c;
   return e == cudaSuccess ? FDG_OK : FDG_ERR_CUDA;
@@ -1031,6 +1126,97 @@ fdg_status fdg_set_lr(fdg_ctx* c, float lr) {
   return FDG_OK;
 }
 
+// Host-side state of the modules that a dry run advances (restored if a recorded graph turns out stale).
+struct HostState {
+  std::vector<int64_t> updates, last_out_batch, last_grad_batch;
+  std::vector<int> last_out_slot, last_grad_slot;
+  std::vector<std::vector<int64_t>> slot_version, slot_batch;
+  size_t log_size;
+};
+static HostState save_host_state(const fdg_ctx* c) {
+  HostState h;
+  for (const Module& m : c->mods) {
+    h.updates.push_back(m.updates); h.last_out_batch.push_back(m.last_out_batch); h.last_grad_batch.push_back(m.last_grad_batch);
+    h.last_out_slot.push_back(m.last_out_slot); h.last_grad_slot.push_back(m.last_grad_slot);
+    h.slot_version.push_back(m.slot_version); h.slot_batch.push_back(m.slot_batch);
+  }
+  h.log_size = c->log.size();
+  return h;
+}
+static void restore_host_state(fdg_ctx* c, const HostState& h) {
+  for (size_t i = 0; i < c->mods.size(); ++i) {
+    Module& m = c->mods[i];
+    m.updates = h.updates[i]; m.last_out_batch = h.last_out_batch[i]; m.last_grad_batch = h.last_grad_batch[i];
+    m.last_out_slot = h.last_out_slot[i]; m.last_grad_slot = h.last_grad_slot[i];
+    m.slot_version = h.slot_version[i]; m.slot_batch = h.slot_batch[i];
+  }
+  if (c->log.size() > h.log_size) c->log.resize(h.log_size);
+}
+
+static cudaError_t run_modules(fdg_ctx* c, cudaStream_t cs, StepMode mode, float* loss_dev) {
+  c->step_sig = 0;
+  for (int k = 0; k < c->K; ++k) {
+    Module& m = c->mods[k];
+    cudaStream_t st = mode == RUN_SERIAL ? cs : m.stream;
+    cudaError_t e = cudaSuccess;
+    if (mode == RUN_CAPTURE) e = cudaStreamWaitEvent(st, c->ev_fork, 0);          // the module's stream joins the recording
+    if (e == cudaSuccess)
+      e = c->bf16_mode ? module_step<bf16>(c, m, st, mode, loss_dev) : module_step<float>(c, m, st, mode, loss_dev);
+    if (e == cudaSuccess && mode == RUN_CAPTURE) {
+      e = cudaEventRecord(c->ev_cjoin[k], st);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, c->ev_cjoin[k], 0);
+    }
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+// One iteration through a CUDA graph: replay the graph recorded for this phase of the rings, or
+// record it now.  The ingest and the learning rate stay outside the graph (they depend on the call).
+static cudaError_t graph_step(fdg_ctx* c, cudaStream_t cs, float* loss_dev) {
+  const int phase = (int)(c->t % c->period);
+  cudaError_t e = cudaSuccess;
+  if (c->lr_on_device != c->lr) {
+    set_scalar_kernel<<<1, 1, 0, cs>>>(c->lr_dev, c->lr);
+    ++c->launches;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    c->lr_on_device = c->lr;
+  }
+  if (c->graph_exec[phase]) {
+    const HostState saved = save_host_state(c);
+    e = run_modules(c, cs, RUN_DRY, nullptr);
+    if (e != cudaSuccess) return e;
+    if (c->step_sig == c->graph_sig[phase]) {
+      c->launches += c->graph_launches[phase];
+      e = cudaGraphLaunch(c->graph_exec[phase], cs);
+    } else {                               // the slots moved: record again
+      restore_host_state(c, saved);
+      cudaGraphExecDestroy(c->graph_exec[phase]);
+      c->graph_exec[phase] = nullptr;
+    }
+  }
+  if (!c->graph_exec[phase]) {
+    const uint64_t l0 = c->launches;
+    e = cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) return e;
+    e = cudaEventRecord(c->ev_fork, c->cap_stream);
+    if (e == cudaSuccess) e = run_modules(c, c->cap_stream, RUN_CAPTURE, nullptr);
+    cudaGraph_t graph = nullptr;
+    cudaError_t e2 = cudaStreamEndCapture(c->cap_stream, &graph);
+    if (e == cudaSuccess) e = e2;
+    if (e == cudaSuccess) e = cudaGraphInstantiate(&c->graph_exec[phase], graph, 0);
+    if (graph) cudaGraphDestroy(graph);
+    if (e != cudaSuccess) { c->graph_exec[phase] = nullptr; return e; }
+    c->graph_sig[phase] = c->step_sig;
+    c->graph_launches[phase] = c->launches - l0;
+    e = cudaGraphLaunch(c->graph_exec[phase], cs);
+  }
+  if (e == cudaSuccess && loss_dev && c->t >= c->K)
+    e = cudaMemcpyAsync(loss_dev, c->mods[c->K - 1].loss, sizeof(float), cudaMemcpyDeviceToDevice, cs);
+  return e;
+}
+
 fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, const int32_t* labels_dev, float* loss_dev) {
   if (!c) return FDG_ERR_INVALID_ARG;
   if (!images_dev || !labels_dev) return fail(c, FDG_ERR_INVALID_ARG, "images and labels must not be null");
@@ -1042,8 +1228,19 @@ fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, cons
   const int64_t t = c->t;
   Module& m1 = c->mods[0];
   cudaError_t e = cudaSuccess;
+  // Graphs take over once every module has run each of its passes at least once (all kernels
+  // have been launched the ordinary way, their attributes are set, the pipeline is full).
+  if (c->use_graphs && !c->graph_mode_entered && t > 2 * (int64_t)c->K + 1) {
+    for (Module& m : c->mods) {              // from here on every iteration is ordered on the caller's stream
+      if (e == cudaSuccess) e = cudaEventRecord(c->ev_join, m.stream);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, c->ev_join, 0);
+    }
+    if (e != cudaSuccess) return cuda_fail(c, e, "entering graph mode");
+    c->graph_mode_entered = true;
+  }
+  const bool graph = c->graph_mode_entered;
   // a0: ingest batch t into module 1's image ring and the label ring
-  if (!serial) e = cudaStreamWaitEvent(cs, m1.ev_grad[(t - 1) % kEventRing], 0);
+  if (!serial && !graph) e = cudaStreamWaitEvent(cs, m1.ev_grad[(t - 1) % kEventRing], 0);
   if (e != cudaSuccess) return cuda_fail(c, e, "ingest wait");
   {
     const size_t rows = (size_t)c->arch.batch * c->arch.in_h * c->arch.in_w;
@@ -1058,15 +1255,12 @@ fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, cons
       ingest_kernel<float><<<blocks, 256, 0, cs>>>(images_dev, reinterpret_cast<float*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch);
     L.check();
     e = L.err;
-    if (e == cudaSuccess && !serial) e = cudaEventRecord(c->ev_in[t % kEventRing], cs);
+    if (e == cudaSuccess && !serial && !graph) e = cudaEventRecord(c->ev_in[t % kEventRing], cs);
     if (e != cudaSuccess) return cuda_fail(c, e, "ingest");
   }
-  for (int k = 0; k < c->K; ++k) {
-    Module& m = c->mods[k];
-    cudaStream_t st = serial ? cs : m.stream;
-    e = c->bf16_mode ? module_step<bf16>(c, m, st, serial, loss_dev) : module_step<float>(c, m, st, serial, loss_dev);
-    if (e != cudaSuccess) return cuda_fail(c, e, "module step");
-  }
+  if (graph) e = graph_step(c, cs, loss_dev);
+  else e = run_modules(c, cs, serial ? RUN_SERIAL : RUN_STREAMS, loss_dev);
+  if (e != cudaSuccess) return cuda_fail(c, e, "module step");
   return FDG_OK;
 }
 
@@ -1084,7 +1278,8 @@ fdg_status fdg_step_host(fdg_ctx* c, fdg_stream stream, const float* images_host
   if (s != FDG_OK) return s;
   if (loss_host && c->t >= c->K) {
     Module& mk = c->mods[c->K - 1];
-    e = cudaMemcpyAsync(loss_host, mk.loss, sizeof(float), cudaMemcpyDeviceToHost, c->cfg.serial ? cs : mk.stream);
+    e = cudaMemcpyAsync(loss_host, mk.loss, sizeof(float), cudaMemcpyDeviceToHost,
+                        (c->cfg.serial || c->graph_mode_entered) ? cs : mk.stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "loss copy");
   }
   return FDG_OK;
@@ -1206,6 +1401,7 @@ fdg_status fdg_get_schedule_log(const fdg_ctx* c, fdg_sched_entry* dst, size_t c
 
 fdg_status fdg_profile_enable(fdg_ctx* c, int on) {
   if (!c) return FDG_ERR_INVALID_ARG;
+  if (c->use_graphs && on) return fail(c, FDG_ERR_STATE, "the per-launch profiler cannot time launches replayed from a graph");
   cudaError_t e = drain(c);
   if (e != cudaSuccess) return cuda_fail(c, e, "drain");
   c->profiling = on != 0;

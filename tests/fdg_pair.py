@@ -18,7 +18,7 @@ def relfro(a, b):
 
 def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_decay=5e-4,
              order="backward_first", weight_reading="stashed", precision="fp32", serial=False, seed=0,
-             jitter=True, oracle_dtype=np.float64, check_every_step=True):
+             jitter=True, oracle_dtype=np.float64, check_every_step=True, graphs=False):
     """Returns a dict of worst-case errors and the two schedule logs."""
     import torch
     from paper_1906_09108_b200 import binding as B
@@ -34,7 +34,7 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
               weight_decay=weight_decay,
               order=B.FDG_BACKWARD_FIRST if order == "backward_first" else B.FDG_FORWARD_FIRST,
               weight_reading=B.FDG_STASHED if weight_reading == "stashed" else B.FDG_CURRENT,
-              precision=B.FDG_FP32_CUDACORE if precision == "fp32" else B.FDG_BF16_TC, serial=serial)
+              precision=B.FDG_FP32_CUDACORE if precision == "fp32" else B.FDG_BF16_TC, serial=serial, graphs=graphs)
     for k in range(1, K + 1):
         spec_o = [(kind, tuple(shape)) for _, kind, shape in orc.param_spec(k)]
         spec_g = [(kind, tuple(shape)) for _, kind, shape in g.param_layout(k)]

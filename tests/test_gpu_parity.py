@@ -76,6 +76,53 @@ def test_serial_mode_is_bitwise_identical_to_streams():
         assert np.array_equal(a, b)
 
 
+@pytest.mark.parametrize("precision", ["fp32", "bf16"])
+def test_graph_replay_is_bitwise_identical_to_streams(precision):
+    """graphs=1 records each iteration into a CUDA graph per ring phase and replays it.  The kernels
+    and their order inside a module are the same, so the parameters must agree bit for bit with the
+    event-driven run; 40 iterations cover the pipeline fill, the recording of all 8 phases (K=4) and
+    several replays of each, with a learning-rate change in between (the rate lives on the device)."""
+    import torch
+    import fdg_synth as S
+    from paper_1906_09108_b200 import binding as B
+    arch = dict(TC_NET, n_per_stage=2, batch=8) if precision == "bf16" else dict(CFG1, n_per_stage=2, batch=8)
+    prec = B.FDG_BF16_TC if precision == "bf16" else B.FDG_FP32_CUDACORE
+    outs, losses = [], []
+    for graphs in (False, True):
+        g = B.FDG(B.make_arch(**arch), K=4, split_after_block=(1, 3, 5), beta=0.5, lr=0.05, precision=prec, graphs=graphs)
+        for k in range(1, 5):
+            g.set_params(k, S.init_params(2, k, g.param_layout(k), jitter=True))
+        loss = torch.zeros(1, device="cuda")
+        ls = []
+        for t in range(1, 41):
+            if t == 25:
+                g.set_lr(0.02)
+            x = torch.from_numpy(S.images(2, t, 8, arch["in_h"], arch["in_w"], 3)).cuda()
+            y = torch.from_numpy(S.labels(2, t, 8, 10)).cuda()
+            g.step(x, y, loss)
+            if t % 7 == 0:
+                g.sync()
+                ls.append(float(loss.item()))
+        g.sync()
+        outs.append([g.get_params(k) for k in range(1, 5)] + [g.get_momentum(k) for k in range(1, 5)])
+        losses.append(ls)
+        assert len(g.schedule_log()) == 40 * 4
+        g.close()
+    assert losses[0] == losses[1]
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("K,splits,order,steps", [(1, (), "backward_first", 11), (2, (2,), "forward_first", 14),
+                                                  (3, (1, 3), "backward_first", 20)])
+def test_graph_replay_fp32_against_oracle(K, splits, order, steps):
+    """Enough iterations to fill the pipeline, record every ring phase (4, 4 and 8 of them) and replay
+    some; a small learning rate keeps fp32 and the fp64 oracle from drifting apart over that many
+    updates on a network this small."""
+    arch = dict(CFG1, n_per_stage=2, batch=6)
+    check_fp32(run_pair(arch, K, splits, steps, beta=0.5, lr=0.005, order=order, graphs=True))
+
+
 def test_resnet110_k4_fp32_reduced_batch():
     """The headline network (ResNet-110, K=4, equal-block split) at batch 8, 10 steps, so
     that every module has been updated at least three times.

@@ -33,10 +33,11 @@ def test_status_strings(lib):
 
 def _cfg(K, splits, **kw):
     arr = (C.c_int * max(len(splits), 1))(*splits)
-    d = dict(beta=0.5, lr=0.1, momentum=0.9, weight_decay=5e-4, order=0, weight_reading=0, precision=0, serial=0)
+    d = dict(beta=0.5, lr=0.1, momentum=0.9, weight_decay=5e-4, order=0, weight_reading=0, precision=0, serial=0,
+             graphs=0)
     d.update(kw)
     cfg = B.fdg_config(K, C.cast(arr, C.POINTER(C.c_int)), d["beta"], d["lr"], d["momentum"], d["weight_decay"],
-                       d["order"], d["weight_reading"], d["precision"], d["serial"])
+                       d["order"], d["weight_reading"], d["precision"], d["serial"], d["graphs"])
     cfg._keep = arr
     return cfg
 
