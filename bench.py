@@ -207,6 +207,17 @@ def run_gpu(args):
     clocks = sampler.stop() if sampler else None
     value = world * b * steps / (ms * 1e-3)
 
+    if args.device_arm_only:
+        g.close()
+        if rank == 0:
+            print(json.dumps(dict(metric=METRIC, value=value, unit="images/s", n_gpus=world, steps=steps, warmup=warmup,
+                                  ms_per_step=ms / steps, gpu_launches=int(launches), clocks=clocks,
+                                  note="device arm only; not a bench line")))
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
     # end to end: host buffers through the C ABI, loss read back every step
     def host_step(i):
         g.step_host(host_x[i % POOL], host_y[i % POOL], loss_host)
@@ -292,6 +303,9 @@ def main():
     ap.add_argument("--precision", default="bf16", choices=["fp32", "bf16"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graphs", action="store_true")
+    ap.add_argument("--device-arm-only", action="store_true",
+                    help="time the device-resident arm only (no end-to-end arm, no per-kernel roofline, no CPU "
+                         "baseline): the short run the ncu launch list is taken from")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

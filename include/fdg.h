@@ -100,8 +100,9 @@ typedef struct {
                                      phase of the rings, a power of two >= 2K of them) and replay it from then on.
                                      Iterations then follow one another on the caller's stream while the K modules of
                                      one iteration still run side by side; the ring buffers are rounded up to powers
-                                     of two, so the workspace grows.  Results are identical to graphs = 0.  Ignored
-                                     when serial = 1; fdg_profile_enable is refused (FDG_ERR_STATE). */
+                                     of two, so the workspace grows.  Results are identical to graphs = 0.  With
+                                     serial = 1 the recorded graph is a single chain.  fdg_profile_enable is refused
+                                     (FDG_ERR_STATE). */
 } fdg_config;
 
 typedef struct {            /* one tensor of a module's flat parameter vector */
@@ -238,6 +239,13 @@ typedef struct {
   double flops;
 } fdg_kernel_stat;
 fdg_status fdg_profile_enable(fdg_ctx* ctx, int on);
+/* Per-module busy time while the profiler was on: busy_ms[k-1] = device time between the start and the end
+ * of module k's passes (forward; backward + update), summed over the iterations since the last read, the
+ * waits for its neighbours excluded.  With one stream per module the passes of different modules share
+ * the GPU, so this is the analogue of the per-GPU utilisation column of the paper's speed table; on a
+ * serial context it is each module's share of the iteration.  Writes min(cap, K) values, K to *out_n.
+ * Blocks the host. */
+fdg_status fdg_profile_read_modules(fdg_ctx* ctx, double* busy_ms, size_t cap, size_t* out_n);
 fdg_status fdg_profile_read(fdg_ctx* ctx, fdg_kernel_stat* dst, size_t cap, size_t* out_n);
 
 /* Number of kernel launches the library has enqueued since fdg_create. */

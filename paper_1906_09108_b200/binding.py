@@ -23,7 +23,7 @@ PARAM_KINDS = {0: "conv", 1: "bn_gamma", 2: "bn_beta", 3: "fc_w", 4: "fc_b"}
 
 EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count", "fdg_param_layout",
            "fdg_set_params", "fdg_set_momentum", "fdg_get_params", "fdg_get_grads", "fdg_get_momentum",
-           "fdg_set_lr", "fdg_step", "fdg_step_host", "fdg_sync", "fdg_profile_enable", "fdg_profile_read", "fdg_get_module_output", "fdg_get_input_grad",
+           "fdg_set_lr", "fdg_step", "fdg_step_host", "fdg_sync", "fdg_profile_enable", "fdg_profile_read", "fdg_profile_read_modules", "fdg_get_module_output", "fdg_get_input_grad",
            "fdg_boundary_elems", "fdg_get_saved_tensor", "fdg_get_schedule_log", "fdg_launch_count", "fdg_status_string",
            "fdg_last_error", "fdg_conv_forward", "fdg_conv_dgrad", "fdg_conv_flip_weights",
            "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_wgrad_static", "fdg_conv_path"]
@@ -84,6 +84,7 @@ def load_library(path=LIB_PATH):
         "fdg_sync": [vp, vp],
         "fdg_profile_enable": [vp, C.c_int],
         "fdg_profile_read": [vp, P(fdg_kernel_stat), sz, P(sz)],
+        "fdg_profile_read_modules": [vp, P(C.c_double), sz, P(sz)],
         "fdg_get_module_output": [vp, C.c_int, vp, sz, P(i64)],
         "fdg_get_input_grad": [vp, C.c_int, vp, sz, P(i64)],
         "fdg_boundary_elems": [vp, C.c_int, P(sz), P(sz)],
@@ -232,6 +233,13 @@ class FDG:
         self._check(self.lib.fdg_profile_read(self.ctx, arr, 32, C.byref(n)), self.ctx)
         return [dict(name=e.name.decode(), launches=e.launches, total_ms=e.total_ms, bytes=e.bytes, flops=e.flops)
                 for e in arr[:n.value]]
+
+    def profile_read_modules(self):
+        """Busy milliseconds of each module's passes since the last read (profiler on)."""
+        arr = (C.c_double * self.K)()
+        n = C.c_size_t()
+        self._check(self.lib.fdg_profile_read_modules(self.ctx, arr, self.K, C.byref(n)), self.ctx)
+        return list(arr)
 
     def sync(self, stream=None):
         st = self.torch.cuda.current_stream().cuda_stream if stream is None else stream

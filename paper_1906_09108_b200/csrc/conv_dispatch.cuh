@@ -23,6 +23,8 @@ struct TensorMapCache {
   };
   std::map<Key, CUtensorMap> maps;
   int sm_count = 0;
+  int share = 1;        // kernels expected to run side by side (one per module stream): a launch takes
+                        // about sm_count / share CTAs and walks its tiles with them
 };
 
 inline bool tc_eligible(const ConvGeom& g) {
@@ -107,12 +109,14 @@ inline cudaError_t cached_weight_map(TensorMapCache* cache, const void* wgt, int
 
 // out = conv3x3(act, wgt) [+ res * [mask > 0]]; act [N][H][W][Ck], wgt [Cn][9*Ck], out [N][H][W][Cn].
 // `red` (nullable, Cn <= 64 only) asks for a per-channel reduction in the epilogue; its `partial`
-// must hold 2*Cn floats per CTA and its `counter` must be zero.
+// must hold 2*Cn floats per CTA; *ctas_out receives the number of CTAs, i.e. of partial rows.
 inline bool halo_reduce_ok(int Cn) { return Cn <= 64; }
 inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ck, int Cn,
                                  const bf16_t* act, const bf16_t* wgt, bf16_t* out, const bf16_t* res,
-                                 const bf16_t* res_mask, int* err_dev, const halo::EpiReduce* red = nullptr) {
-  const int sms = cached_sm_count(cache);
+                                 const bf16_t* res_mask, int* err_dev, const halo::EpiReduce* red = nullptr,
+                                 int* ctas_out = nullptr) {
+  int sms = cached_sm_count(cache) / (cache->share > 0 ? cache->share : 1);
+  if (sms < 16) sms = 16;
   halo::FwdParams p = halo::fwd_params(N, H, W, Ck, Cn, sms);
   const CUtensorMap *mx, *mw;
   cudaError_t e = cached_tile_map(cache, act, N, H, W, Ck, p.G, &mx);
@@ -122,7 +126,8 @@ inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, 
   const int grid = p.tiles < sms ? p.tiles : sms;
   halo::EpiReduce r{};
   if (red) { if (!halo_reduce_ok(Cn)) return cudaErrorInvalidValue; r = *red; }
-  halo::conv_halo_kernel<<<grid, tc::kThreads, halo::fwd_smem_bytes(p), st>>>(*mx, *mw, p, out, res, res_mask, r, err_dev);
+  if (ctas_out) *ctas_out = grid;
+  halo::conv_halo_kernel<<<grid, halo::kFwdThreads, halo::fwd_smem_bytes(p), st>>>(*mx, *mw, p, out, res, res_mask, r, err_dev);
   return cudaGetLastError();
 }
 

@@ -71,25 +71,26 @@ __device__ __forceinline__ uint32_t instr_desc(int n, bool mn_major) {
 
 // Optional per-channel reduction over the tensor the kernel stores, taken in its epilogue (on
 // the values as stored, i.e. after rounding to bf16):
-//   mode 1  batch-norm statistics of the output:  sum v, sum v^2  ->  stats = (mean, 1/sqrt(var + eps))
+//   mode 1  batch-norm statistics of the output:  sum v, sum v^2
 //   mode 2  the two sums of the batch-norm backward the output feeds as its upstream gradient:
 //           dz = v * [mask > 0],  sum dz,  sum dz * xhat  with xhat = (xprev - mean) * invstd
-//           -> sums, and the parameter gradients dbeta = sum dz, dgamma = sum dz * xhat
-// Every CTA writes its sums to partial[cta][2*Cn]; the CTA that finishes last adds them in CTA
-// order (fp64), so the result does not depend on scheduling.  Cn <= 64 only.
+// Every CTA writes its sums to partial[cta][2*Cn]; the kernel that consumes the totals adds the
+// CTAs' rows in CTA order (elementwise.cuh, finalize_partials), so the result does not depend on
+// scheduling and no grid-wide synchronisation is needed here.  Cn <= 64 only.
 struct EpiReduce {
   int mode;
   const __nv_bfloat16* mask;
   const __nv_bfloat16* xprev;
   const float* pstats;        // mode 2: mean[Cn], invstd[Cn] of xprev's batch norm
   float* partial;             // [gridDim.x][2*Cn]
-  unsigned int* counter;      // zero before the launch; left at zero
-  float* out;                 // mode 1: stats[2*Cn]; mode 2: sums[2*Cn]
-  float* dgamma;              // mode 2 (Cn each)
-  float* dbeta;
-  float eps, inv_count;       // mode 1: 1 / (pixels per channel)
 };
-constexpr int kRedSmemBytes = 4 * 8 * 32 * 4 + 2 * 128 * 4 + 192 * 8;   // running sums, statistics, finalisation
+// Threads of conv_halo_kernel: TMA warp, MMA warp, kEpiGroups groups of four epilogue warps.  A
+// group takes every kEpiGroups-th 128-row tile: one tile's epilogue is a chain of dependent
+// steps (wait, tensor-memory load, global loads, shuffles), so several must be in flight.
+constexpr int kEpiGroups = 4;
+constexpr int kEpiWarps = 4 * kEpiGroups;
+constexpr int kFwdThreads = 64 + 32 * kEpiWarps;
+constexpr int kRedSmemBytes = kEpiWarps * 8 * 32 * 4 + 2 * 128 * 4;   // running sums, statistics
 
 // 32 lanes each hold 32 items; afterwards lane l holds in q[0] the sum over all lanes of item l.
 __device__ __forceinline__ void transpose_reduce32(float (&q)[32], int lane) {
@@ -105,9 +106,22 @@ __device__ __forceinline__ void transpose_reduce32(float (&q)[32], int lane) {
   }
 }
 
+// The 9 * KS instructions of one 128-row tile, fully unrolled (the issuing thread is the
+// bottleneck: every instruction it spends per tcgen05.mma beyond the add and the issue shows).
+template <int KS>
+__device__ __forceinline__ void issue_tile(uint32_t d_tmem, uint64_t x_desc, const uint64_t (&tap_off)[9], uint64_t w_desc0,
+                                           uint64_t w_tap_step, uint32_t idesc) {
+#pragma unroll
+  for (int tap = 0; tap < 9; ++tap) {
+    const uint64_t a0 = x_desc + tap_off[tap], b0 = w_desc0 + tap * w_tap_step;
+#pragma unroll
+    for (int j = 0; j < KS; ++j) tc_mma_bf16(d_tmem, a0 + 2 * j, b0 + 2 * j, idesc, (tap | j) != 0);
+  }
+}
+
 // ------------------------------------------------------- forward / data gradient --
 // out[pixel][n] (bf16, row stride Cn) = conv + (res ? res * [mask ? mask > 0 : 1] : 0)
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, FwdParams p,
                  __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
                  const __nv_bfloat16* __restrict__ res_mask, EpiReduce red, int* __restrict__ error_word) {
@@ -122,20 +136,20 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   uint64_t* acc_empty = acc_full + p.nacc;     // [nacc]    epilogue -> MMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + p.nacc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* red_run = reinterpret_cast<float*>(tmem_slot + 4);          // [4 warps][8 chunks][32 items]
-  float* red_stat = red_run + 4 * 8 * 32;                            // mode 2: mean[Cn], invstd[Cn]
-  double* red_fin = reinterpret_cast<double*>(red_stat + 2 * 128);   // [192]
+  float* red_run = reinterpret_cast<float*>(tmem_slot + 4);          // [epilogue warps][8 chunks][32 items]
+  float* red_stat = red_run + kEpiWarps * 8 * 32;                    // mode 2: mean[Cn], invstd[Cn]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (red.mode) {
-    for (int i = threadIdx.x; i < 4 * 8 * 32; i += kThreads) red_run[i] = 0.f;
+    for (int i = threadIdx.x; i < kEpiWarps * 8 * 32; i += kFwdThreads) red_run[i] = 0.f;
     if (red.mode == 2)
-      for (int i = threadIdx.x; i < 2 * p.Cn; i += kThreads) red_stat[i] = red.pstats[i];
+      for (int i = threadIdx.x; i < 2 * p.Cn; i += kFwdThreads) red_stat[i] = red.pstats[i];
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(w_full, 1);
-    for (int a = 0; a < p.nacc; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
+    const int groups_per_tile = p.Cn / 16 < kEpiGroups ? p.Cn / 16 : kEpiGroups;
+    for (int a = 0; a < p.nacc; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4 * groups_per_tile); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -177,6 +191,8 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       // and whether or not it depends on the previous one (measured), so a 128-row tile costs
       // 9 * Ck/16 * 60 cycles here and the only overhead worth removing is the issue loop's own.
       uint32_t it = 0, acount = 0;
+      int slot = 0;                                           // acount % nacc and the slot's phase, kept incrementally
+      uint32_t aph = 0;
       for (int tile = blockIdx.x; ok && tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
@@ -184,35 +200,35 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         tc_fence_after();
         uint64_t x_desc = smem_desc_kmajor(smem_u32(smem + (size_t)s * p.stage_bytes), p.pitch);
         for (int i = 0; i < p.m_tiles; ++i, ++acount, x_desc += mtile_step) {
-          const int slot = acount % p.nacc;
-          const uint32_t aph = (acount / p.nacc) & 1;
-          if (!mbar_wait(&acc_empty[slot], aph ^ 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)slot * p.Cn;
-          if (ksteps == 1) {
-#pragma unroll
-            for (int tap = 0; tap < 9; ++tap)
-              tc_mma_bf16(d_tmem, x_desc + tap_off[tap], w_desc0 + tap * w_tap_step, idesc, tap != 0);
-          } else {
-#pragma unroll
-            for (int tap = 0; tap < 9; ++tap) {
-              const uint64_t a0 = x_desc + tap_off[tap], b0 = w_desc0 + tap * w_tap_step;
-              for (int j = 0; j < ksteps; ++j) tc_mma_bf16(d_tmem, a0 + 2 * j, b0 + 2 * j, idesc, (tap | j) != 0);
-            }
+          if (acount >= (uint32_t)p.nacc) {                   // a slot's first use needs no hand-back from the epilogue
+            if (!mbar_wait(&acc_empty[slot], aph ^ 1, abort_flag)) { ok = false; break; }
+            tc_fence_after();
           }
+          const uint32_t d_tmem = tmem_base + (uint32_t)slot * p.Cn;
+          if (ksteps == 1) issue_tile<1>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
+          else if (ksteps == 2) issue_tile<2>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
+          else issue_tile<4>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
           tc_commit(&acc_full[slot]);
+          if (++slot == p.nacc) { slot = 0; aph ^= 1; }
         }
         if (!ok) break;
         tc_commit(&empty[s]);
       }
     }
   } else {
-    const int lane_grp = warp & 3;
+    const int lane_grp = warp & 3;                 // tensor-memory lanes 32*(warp % 4) .. +31
+    const int group = (warp - 2) >> 2;
     uint32_t acount = 0;
     for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x) {
       const int n0 = tile * p.G;
       bool ok = true;
       for (int i = 0; i < p.m_tiles; ++i, ++acount) {
+        // Work item = (tile, 16-column chunk), dealt to the groups in turn.  nacc is a multiple of
+        // kEpiGroups, so the same groups meet a slot every time and see all its phases.
+        const int nch = p.Cn >> 4;
+        const int first = (int)((acount * (uint32_t)nch) % kEpiGroups);
+        int my_first = group - first; if (my_first < 0) my_first += kEpiGroups;      // first chunk of this tile dealt to this group
+        if (my_first >= nch) continue;
         const int slot = acount % p.nacc;
         const uint32_t aph = (acount / p.nacc) & 1;
         if (!mbar_wait(&acc_full[slot], aph, abort_flag)) { ok = false; break; }
@@ -223,7 +239,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const bool valid = h < p.H && w < p.W && g < p.G && n0 + g < p.N;
         const size_t base = ((((size_t)(n0 + g) * p.H + h) * p.W) + w) * p.Cn;
         const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)slot * p.Cn;
-        for (int c0 = 0; c0 < p.Cn; c0 += 16) {
+        for (int c0 = my_first * 16; c0 < p.Cn; c0 += 16 * kEpiGroups) {
           uint32_t v[16];
           tmem_ld16(taddr + c0, v);
           tmem_ld_wait();
@@ -325,53 +341,15 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     tmem_dealloc(tmem_base, p.tmem_cols);
   }
   if (red.mode && !*abort_flag) {
-    // this CTA's sums: item (chunk, lane) of the four epilogue warps -> partial[cta][stat][channel]
+    // this CTA's sums: item (chunk, lane) of all epilogue warps, added in warp order -> partial[cta][stat][channel]
     const int pairs = 2 * p.Cn;
-    for (int t = threadIdx.x; t < pairs; t += kThreads) {
+    for (int t = threadIdx.x; t < pairs; t += kFwdThreads) {
       const int stat = t / p.Cn, c = t - stat * p.Cn;
       const int idx = (c >> 4) * 32 + (c & 15) + 16 * stat;
-      red.partial[(size_t)blockIdx.x * pairs + t] = red_run[idx] + red_run[8 * 32 + idx] + red_run[2 * 8 * 32 + idx] + red_run[3 * 8 * 32 + idx];
-    }
-    __threadfence();
-    __syncthreads();
-    __shared__ bool is_last;
-    if (threadIdx.x == 0) is_last = atomicInc(red.counter, gridDim.x - 1) == gridDim.x - 1;
-    __syncthreads();
-    if (is_last) {
-      __threadfence();
-      // Cn <= 64, so pairs <= 128 <= kThreads: nseg threads share one (stat, channel) pair, each
-      // taking every nseg-th CTA with 8 loads in flight; their sums are then added in segment order.
-      const int nseg = kThreads / pairs;
-      const int t = threadIdx.x % pairs, seg = threadIdx.x / pairs;
-      double a = 0.0;
-      if (seg < nseg)
-        for (unsigned b0 = seg; b0 < gridDim.x; b0 += 8 * nseg) {
-          float v[8];
+      float a = 0.f;
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const unsigned b = b0 + u * nseg;
-            v[u] = b < gridDim.x ? __ldcg(&red.partial[(size_t)b * pairs + t]) : 0.f;
-          }
-#pragma unroll
-          for (int u = 0; u < 8; ++u) a += (double)v[u];
-        }
-      red_fin[threadIdx.x] = a;
-      __syncthreads();
-      if ((int)threadIdx.x < p.Cn) {
-        const int c = threadIdx.x;
-        double s0 = 0.0, s1 = 0.0;
-        for (int q = 0; q < nseg; ++q) { s0 += red_fin[q * pairs + c]; s1 += red_fin[q * pairs + p.Cn + c]; }
-        if (red.mode == 1) {
-          const double mean = s0 * (double)red.inv_count;
-          double var = s1 * (double)red.inv_count - mean * mean;
-          if (var < 0.0) var = 0.0;
-          red.out[c] = (float)mean;
-          red.out[p.Cn + c] = (float)(1.0 / sqrt(var + (double)red.eps));
-        } else {
-          red.out[c] = (float)s0; red.out[p.Cn + c] = (float)s1;
-          red.dbeta[c] = (float)s0; red.dgamma[c] = (float)s1;
-        }
-      }
+      for (int w = 0; w < kEpiWarps; ++w) a += red_run[w * 8 * 32 + idx];
+      red.partial[(size_t)blockIdx.x * pairs + t] = a;
     }
   }
 }
@@ -550,7 +528,7 @@ inline FwdParams fwd_params(int N, int H, int W, int Ck, int Cn, int sm_count) {
   p.w_tx_bytes = (uint32_t)Cn * p.pitch;
   p.w_tap_bytes = round_up_u32(p.w_tx_bytes, 1024);
   // images per tile: as many as keep every SM busy, within the shared-memory budget
-  int G = N / (sm_count > 0 ? sm_count : 148);
+  int G = N / 148;                                            // more than one image per tile only for large batches
   if (G < 1) G = 1;
   for (;; --G) {
     p.G = G;
@@ -568,8 +546,10 @@ inline FwdParams fwd_params(int N, int H, int W, int Ck, int Cn, int sm_count) {
   if (stages > 3) stages = 3;
   if (stages > per_cta) stages = per_cta;                     // shared memory left free lets other kernels' CTAs co-reside
   p.stages = stages;
-  p.nacc = p.m_tiles < 4 ? p.m_tiles : 4;
-  if (p.nacc < 2) p.nacc = 2;
+  // accumulator slots: a multiple of the epilogue groups (a slot then always belongs to one group); a slot
+  // per 128-row tile where 256 columns allow it, so that the issuer seldom waits for the epilogue
+  p.nacc = (p.m_tiles + kEpiGroups - 1) / kEpiGroups * kEpiGroups;
+  while (p.nacc > kEpiGroups && p.nacc * Cn > 256) p.nacc -= kEpiGroups;
   uint32_t cols = 32;
   while (cols < (uint32_t)(p.nacc * Cn)) cols <<= 1;
   p.tmem_cols = cols;

@@ -184,13 +184,71 @@ bn_stats_kernel(const T* __restrict__ x, RedGeom g, float eps, float* __restrict
       });
 }
 
+// Per-CTA partial sums left by a convolution epilogue, partial[nparts][2*C], to be added up by
+// the kernel that consumes the totals (every block does it for itself: the partials are a few KB
+// and sit in L2).  Fixed order: kEwThreads / (2C) threads share a (sum, channel) pair, each taking
+// every nseg-th partial with 8 loads in flight; segment sums are added in segment order.
+//   kind 1  totals are (sum x, sum x^2): out2c = (mean, 1/sqrt(var + eps))
+//   kind 2  totals are the batch-norm backward's (sum dz, sum dz*xhat): out2c = the totals
+struct PartialSums {
+  const float* partial;     // null: nothing to add up (the totals are read from global memory instead)
+  int nparts;
+  int kind;
+  float inv_count, eps;     // kind 1
+  float* save0;             // block 0 stores out2c[0..C) here (kind 1: with save1 contiguous = stats[2C]; kind 2: dbeta)
+  float* save1;             // and out2c[C..2C) here (kind 2: dgamma)
+};
+constexpr int kEwThreads = 256;
+
+// Fills out2c[2*C] (shared memory) from the partials; requires blockDim.x == kEwThreads and 2*C <= kEwThreads.
+__device__ __forceinline__ void finalize_partials(const PartialSums ps, int C, float* out2c) {
+  __shared__ double fin[kEwThreads];
+  const int tid = threadIdx.x, pairs = 2 * C;
+  const int nseg = kEwThreads / pairs;
+  const int t = tid % pairs, seg = tid / pairs;
+  double a = 0.0;
+  if (seg < nseg)
+    for (int b0 = seg; b0 < ps.nparts; b0 += 8 * nseg) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int b = b0 + u * nseg;
+        v[u] = b < ps.nparts ? __ldcg(&ps.partial[(size_t)b * pairs + t]) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) a += (double)v[u];
+    }
+  fin[tid] = a;
+  __syncthreads();
+  if (tid < C) {
+    double s0 = 0.0, s1 = 0.0;
+    for (int q = 0; q < nseg; ++q) { s0 += fin[q * pairs + tid]; s1 += fin[q * pairs + C + tid]; }
+    float o0, o1;
+    if (ps.kind == 1) {
+      const double mean = s0 * (double)ps.inv_count;
+      double var = s1 * (double)ps.inv_count - mean * mean;
+      if (var < 0.0) var = 0.0;
+      o0 = (float)mean; o1 = (float)(1.0 / sqrt(var + (double)ps.eps));
+    } else {
+      o0 = (float)s0; o1 = (float)s1;
+    }
+    out2c[tid] = o0; out2c[C + tid] = o1;
+    if (blockIdx.x == 0) { ps.save0[tid] = o0; ps.save1[tid] = o1; }
+  }
+  __syncthreads();
+}
+
 // y = [relu]( gamma*(x-mean)*invstd + beta + residual ), residual = none | r | BN_r(r).
+// The statistics come from `stats`, or are first formed from `ps.partial` (and saved to stats).
 template <typename T, int VEC>
 __global__ void bn_apply_kernel(const T* __restrict__ x, const float* __restrict__ stats,
                                 const float* __restrict__ gamma, const float* __restrict__ beta,
                                 const T* __restrict__ res, const float* __restrict__ res_stats,
                                 const float* __restrict__ res_gamma, const float* __restrict__ res_beta,
-                                int relu, T* __restrict__ y, size_t nvec, int C) {
+                                int relu, T* __restrict__ y, size_t nvec, int C, PartialSums ps) {
+  __shared__ float s_stats[2 * 128];
+  const float* st = stats;
+  if (ps.partial) { finalize_partials(ps, C, s_stats); st = s_stats; }
   const int cv = C / VEC;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
     const int c0 = (int)(i % cv) * VEC;
@@ -200,7 +258,7 @@ __global__ void bn_apply_kernel(const T* __restrict__ x, const float* __restrict
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
       const int c = c0 + j;
-      float t = gamma[c] * ((v[j] - stats[c]) * stats[C + c]) + beta[c];
+      float t = gamma[c] * ((v[j] - st[c]) * st[C + c]) + beta[c];
       if (res) {
         float rr = r[j];
         if (res_stats) rr = res_gamma[c] * ((rr - res_stats[c]) * res_stats[C + c]) + res_beta[c];
@@ -263,7 +321,9 @@ __global__ void bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restric
                                     const float* __restrict__ sums, const T* __restrict__ x2,
                                     const float* __restrict__ stats2, const float* __restrict__ gamma2,
                                     const T* __restrict__ res, T* __restrict__ dx, T* __restrict__ dx2,
-                                    T* __restrict__ dz_out, size_t nvec, int C, float inv_m) {
+                                    T* __restrict__ dz_out, size_t nvec, int C, float inv_m, PartialSums ps) {
+  __shared__ float s_sums[2 * 128];
+  if (ps.partial) { finalize_partials(ps, C, s_sums); sums = s_sums; }
   const int cv = C / VEC;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
     const int c0 = (int)(i % cv) * VEC;

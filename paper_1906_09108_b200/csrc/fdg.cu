@@ -154,6 +154,8 @@ struct fdg_ctx {
   bool profiling = false;
   std::vector<cudaEvent_t> prof_events;     // 2 per recorded launch
   std::vector<fdg::ProfRec> prof_recs;
+  std::vector<cudaEvent_t> mod_events;      // 2 per recorded module pass (forward, or backward + update)
+  std::vector<int> mod_event_owner;         // module (0-based) of each pair
 };
 
 namespace fdg {
@@ -455,17 +457,27 @@ static void bn_stats(Launch& L, Module& m, const T* x, size_t rows, int C, float
   L.check();
 }
 
+// `nparts` > 0: the statistics are not in `stats` yet; the convolution that produced x left nparts
+// rows of partial sums in m.red_partial, which the kernel adds up first (and saves to `stats`).
 template <typename T>
-static void bn_apply(Launch& L, const T* x, const float* stats, const float* gamma, const float* beta, const T* res,
+static void bn_apply(Launch& L, Module& m, const T* x, float* stats, const float* gamma, const float* beta, const T* res,
                      const float* res_stats, const float* res_gamma, const float* res_beta, bool relu, T* y,
-                     size_t rows, int C) {
+                     size_t rows, int C, int nparts = 0) {
   constexpr int V = full_vec<T>();
   const size_t n = rows * C;
+  PartialSums ps{};
+  if (nparts > 0) {
+    ps.partial = m.red_partial; ps.nparts = nparts; ps.kind = 1; ps.inv_count = 1.f / (float)rows; ps.eps = L.c->arch.bn_eps;
+    ps.save0 = stats; ps.save1 = stats + C;
+  }
   L.begin(KC_BN_APPLY, (double)n * sizeof(T) * (res ? 3 : 2), 6.0 * n);
-  if (C % V == 0)
-    bn_apply_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C);
-  else
-    bn_apply_kernel<T, 1><<<ew_blocks(n), 256, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C);
+  if (C % V == 0) {
+    int blocks = ew_blocks(n / V);
+    if (nparts > 0) blocks = std::min(blocks, 2 * 148);      // every block re-adds the partials: keep them few
+    bn_apply_kernel<T, V><<<blocks, kEwThreads, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
+  } else {
+    bn_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
+  }
   L.check();
 }
 
@@ -475,12 +487,17 @@ template <typename T>
 static void bn_backward(Launch& L, Module& m, const T* dy, const T* mask, const T* x, const float* stats,
                         const float* gamma, float* dgamma, float* dbeta, const T* x2, const float* stats2,
                         const float* gamma2, float* dgamma2, float* dbeta2, const T* res, T* dx, T* dx2,
-                        size_t rows, int C, bool sums_ready = false) {
+                        size_t rows, int C, int nparts = 0) {
   constexpr int V = full_vec<T>();
   const bool two = x2 != nullptr;
   const int ns = two ? 3 : 2;
   const bool vec = C % V == 0;
-  if (!sums_ready) {      // otherwise the kernel that produced dy already left the sums in m.bnsums
+  const bool sums_ready = nparts > 0;
+  PartialSums ps{};
+  if (sums_ready) {       // the kernel that produced dy left nparts rows of partial sums in m.red_partial
+    ps.partial = m.red_partial; ps.nparts = nparts; ps.kind = 2; ps.save0 = dbeta; ps.save1 = dgamma;
+  }
+  if (!sums_ready) {
     RedGeom g = red_geom((int)rows, C, vec ? V : 1);
     const size_t smem = (size_t)std::max(g.rp, 2) * ns * C * 4;
 #define FDG_RED(VV, NS) bn_bwd_reduce_kernel<T, VV, NS><<<g.blocks, kRedThreads, smem, L.st>>>( \
@@ -494,10 +511,13 @@ static void bn_backward(Launch& L, Module& m, const T* dy, const T* mask, const 
   const size_t n = rows * C;
   const float inv_m = 1.f / (float)rows;
   L.begin(KC_BN_BWD_APPLY, (double)n * sizeof(T) * (3 + (mask ? 1 : 0) + (two ? 2 : 0) + (res ? 1 : 0)), 10.0 * n);
-  if (vec)
-    bn_bwd_apply_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n / V, C, inv_m);
-  else
-    bn_bwd_apply_kernel<T, 1><<<ew_blocks(n), 256, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n, C, inv_m);
+  if (vec) {
+    int blocks = ew_blocks(n / V);
+    if (sums_ready) blocks = std::min(blocks, 2 * 148);
+    bn_bwd_apply_kernel<T, V><<<blocks, kEwThreads, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n / V, C, inv_m, ps);
+  } else {
+    bn_bwd_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n, C, inv_m, ps);
+  }
   L.check();
 }
 
@@ -523,41 +543,40 @@ static double in_elems(const ConvGeom& g) { return (double)g.N * g.H * g.W * g.C
 static double out_elems(const ConvGeom& g) { return (double)g.N * g.P * g.Q * g.Co; }
 static double w_elems(const ConvGeom& g) { return (double)g.Co * g.R * g.S * g.Ci; }
 
-// `stats` (nullable): where the batch-norm statistics (mean, 1/sigma) of y should go.  Returns true
-// when the convolution kernel produced them in its epilogue; otherwise the caller runs bn_stats.
+// `want_stats`: the caller will batch-normalise y.  Returns the number of rows of per-channel partial
+// sums (sum y, sum y^2) the convolution kernel left in m.red_partial from its epilogue, or 0 when it
+// left none and the caller has to run bn_stats.
 template <typename T>
-static bool conv_fprop(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* w, T* y, const T* res,
-                       float* stats = nullptr) {
+static int conv_fprop(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* w, T* y, const T* res,
+                      bool want_stats = false) {
   L.begin(KC_CONV_FPROP, (in_elems(g) + w_elems(g) + out_elems(g) * (res ? 2 : 1)) * sizeof(T), conv_flops(g));
   if constexpr (std::is_same<T, bf16>::value) {
     if (halo_fprop_eligible(g)) {
       ++L.c->launches;
-      const bool fuse = stats && halo_reduce_ok(g.Co);
+      const bool fuse = want_stats && halo_reduce_ok(g.Co);
       halo::EpiReduce r{};
-      if (fuse) {
-        r.mode = 1; r.partial = m.red_partial; r.counter = m.red_counter; r.out = stats;
-        r.eps = L.c->arch.bn_eps; r.inv_count = 1.f / ((float)g.N * g.P * g.Q);
-      }
-      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, fuse ? &r : nullptr));
-      return fuse;
+      int ctas = 0;
+      if (fuse) { r.mode = 1; r.partial = m.red_partial; }
+      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, fuse ? &r : nullptr, &ctas));
+      return fuse ? ctas : 0;
     }
     if (tc_eligible(g)) {
       ++L.c->launches;
       L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error));
-      return false;
+      return 0;
     }
   }
   L.note(launch_conv_simt<T, CONV_FPROP>(L.st, g, x, w, y, nullptr, nullptr, res, (const T*)nullptr, &L.c->launches));
-  return false;
+  return 0;
 }
 // `wflip` is the flipped/transposed weight copy (bf16 mode, tensor-core eligible shapes) or null.
 // The batch-norm backward that will consume dx as its upstream gradient: dz = dx * [mask > 0],
 // xhat from (x, stats).  When the data-gradient kernel can, it forms that backward's two sums
-// (and the parameter gradients) in its epilogue and conv_dgrad returns true.
-template <typename T> struct NextBnBwd { const T* mask; const T* x; const float* stats; float* dgamma; float* dbeta; };
+// per CTA in its epilogue and conv_dgrad returns the number of partial rows left in m.red_partial.
+template <typename T> struct NextBnBwd { const T* mask; const T* x; const float* stats; };
 
 template <typename T>
-static bool conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, const T* w, const T* wflip, T* dx,
+static int conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, const T* w, const T* wflip, T* dx,
                        const T* res, const T* mask, const NextBnBwd<T>* next = nullptr) {
   L.begin(KC_CONV_DGRAD, (out_elems(g) + w_elems(g) + in_elems(g) * (1 + (res ? 1 : 0) + (mask ? 1 : 0) + (next ? 2 : 0))) * sizeof(T), conv_flops(g));
   if constexpr (std::is_same<T, bf16>::value) {
@@ -565,21 +584,19 @@ static bool conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, con
       ++L.c->launches;
       const bool fuse = next && halo_reduce_ok(g.Ci);
       halo::EpiReduce r{};
-      if (fuse) {
-        r.mode = 2; r.mask = next->mask; r.xprev = next->x; r.pstats = next->stats; r.partial = m.red_partial;
-        r.counter = m.red_counter; r.out = m.bnsums; r.dgamma = next->dgamma; r.dbeta = next->dbeta;
-      }
-      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error, fuse ? &r : nullptr));
-      return fuse;
+      int ctas = 0;
+      if (fuse) { r.mode = 2; r.mask = next->mask; r.xprev = next->x; r.pstats = next->stats; r.partial = m.red_partial; }
+      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error, fuse ? &r : nullptr, &ctas));
+      return fuse ? ctas : 0;
     }
     if (wflip && tc_eligible(g)) {
       ++L.c->launches;
       L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error));
-      return false;
+      return 0;
     }
   }
   L.note(launch_conv_simt<T, CONV_DGRAD>(L.st, g, dy, w, dx, nullptr, nullptr, res, mask, &L.c->launches));
-  return false;
+  return 0;
 }
 template <typename T>
 static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* dy, float* dw) {
@@ -628,9 +645,9 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
       case U_STEM: {
         ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
         if (u.bn) {
-          if (!conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_a, nullptr, F + u.st1))
-            bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
-          bn_apply<T>(L, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co);
+          const int np = conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_a, nullptr, true);
+          if (!np) bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
+          bn_apply<T>(L, m, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np);
         } else {
           conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_y, nullptr);
         }
@@ -639,29 +656,30 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
       case U_BASIC: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
-        if (!conv_fprop<T>(L, m, g1, x, wt + u.w1, S + u.t_a, nullptr, F + u.st1))                      // c1
-          bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
-        bn_apply<T>(L, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_b, rows_out, u.co);  // a1
-        if (!conv_fprop<T>(L, m, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr, F + u.st2))              // c2
-          bn_stats<T>(L, m, S + u.t_c, rows_out, u.co, eps, F + u.st2);
-        if (u.proj) {
+        const int np1 = conv_fprop<T>(L, m, g1, x, wt + u.w1, S + u.t_a, nullptr, true);               // c1
+        if (!np1) bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
+        bn_apply<T>(L, m, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_b, rows_out, u.co, np1);  // a1
+        if (u.proj) {          // shortcut first: its statistics must not disturb the partial sums conv2 leaves for BN2
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
-          if (!conv_fprop<T>(L, m, gs, x, wt + u.ws, S + u.t_s, nullptr, F + u.sts))                    // cs
-            bn_stats<T>(L, m, S + u.t_s, rows_out, u.co, eps, F + u.sts);
-          bn_apply<T>(L, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, S + u.t_s, F + u.sts, wf + u.gs, wf + u.bs, true, S + u.t_y, rows_out, u.co);
-        } else {
-          bn_apply<T>(L, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, x, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co);
+          conv_fprop<T>(L, m, gs, x, wt + u.ws, S + u.t_s, nullptr);                                   // cs
+          bn_stats<T>(L, m, S + u.t_s, rows_out, u.co, eps, F + u.sts);
         }
+        const int np2 = conv_fprop<T>(L, m, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr, true);       // c2
+        if (!np2) bn_stats<T>(L, m, S + u.t_c, rows_out, u.co, eps, F + u.st2);
+        if (u.proj)
+          bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, S + u.t_s, F + u.sts, wf + u.gs, wf + u.bs, true, S + u.t_y, rows_out, u.co, np2);
+        else
+          bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, x, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np2);
         break;
       }
       case U_PREACT: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
         bn_stats<T>(L, m, x, rows_in, u.ci, eps, F + u.st1);
-        bn_apply<T>(L, x, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows_in, u.ci);   // o
-        if (!conv_fprop<T>(L, m, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr, F + u.st2))              // c1
-          bn_stats<T>(L, m, S + u.t_b, rows_out, u.co, eps, F + u.st2);
-        bn_apply<T>(L, S + u.t_b, F + u.st2, wf + u.g2, wf + u.b2, nullptr, nullptr, nullptr, nullptr, true, S + u.t_c, rows_out, u.co); // a2
+        bn_apply<T>(L, m, x, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows_in, u.ci);   // o
+        const int np = conv_fprop<T>(L, m, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr, true);        // c1
+        if (!np) bn_stats<T>(L, m, S + u.t_b, rows_out, u.co, eps, F + u.st2);
+        bn_apply<T>(L, m, S + u.t_b, F + u.st2, wf + u.g2, wf + u.b2, nullptr, nullptr, nullptr, nullptr, true, S + u.t_c, rows_out, u.co, np); // a2
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_fprop<T>(L, m, gs, S + u.t_a, wt + u.ws, tmp, nullptr);
@@ -692,7 +710,7 @@ static void head_forward_backward(fdg_ctx* c, Module& m, Launch& L, int64_t tau,
   const T* feat = x;
   if (u.bn) {
     bn_stats<T>(L, m, x, rows, F, c->arch.bn_eps, Fs + u.st1);
-    bn_apply<T>(L, x, Fs + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows, F);
+    bn_apply<T>(L, m, x, Fs + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows, F);
     feat = S + u.t_a;
   }
   const int32_t* labels = c->labels + (size_t)(tau % c->label_ring) * B;
@@ -726,7 +744,8 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
   T* T2 = reinterpret_cast<T*>(m.temps[3]);
   T* T3 = reinterpret_cast<T*>(m.temps[4]);
   T* dy = gin;
-  bool dy_sums_ready = false;      // the kernel that produced dy also left the first batch-norm backward's sums
+  int dy_sum_parts = 0;            // > 0: the kernel that produced dy left that many rows of partial sums for the
+                                   // first batch-norm backward it meets
   const int nu = (int)m.units.size();
   for (int i = nu - 1; i >= 0; --i) {
     const Unit& u = m.units[i];
@@ -740,17 +759,17 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
     const NextBnBwd<T>* next = nullptr;
     if (i > 0) {
       const Unit& pu = m.units[i - 1];
-      if (pu.type == U_BASIC && !pu.proj) { nb = {S + pu.t_y, S + pu.t_c, F + pu.st2, m.grad + pu.g2, m.grad + pu.b2}; next = &nb; }
-      if (pu.type == U_STEM && pu.bn) { nb = {S + pu.t_y, S + pu.t_a, F + pu.st1, m.grad + pu.g1, m.grad + pu.b1}; next = &nb; }
+      if (pu.type == U_BASIC && !pu.proj) { nb = {S + pu.t_y, S + pu.t_c, F + pu.st2}; next = &nb; }
+      if (pu.type == U_STEM && pu.bn) { nb = {S + pu.t_y, S + pu.t_a, F + pu.st1}; next = &nb; }
     }
-    bool out_sums_ready = false;
+    int out_sum_parts = 0;
     switch (u.type) {
       case U_STEM: {
         ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
         const T* dc = dy;
         if (u.bn) {
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
-                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sums_ready);
+                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sum_parts);
           dc = T1;
         }
         conv_wgrad<T>(L, m, g, x, dc, m.grad + u.w1);
@@ -764,12 +783,12 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
                          F + u.sts, wf + u.gs, m.grad + u.gs, m.grad + u.bs, nullptr, T1, T2, rows_out, u.co);
         else
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_c, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
-                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sums_ready);
+                         nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sum_parts);
         conv_wgrad<T>(L, m, g2, S + u.t_b, T1, m.grad + u.w2);
-        const NextBnBwd<T> bn1{S + u.t_b, S + u.t_a, F + u.st1, m.grad + u.g1, m.grad + u.b1};
-        const bool bn1_ready = conv_dgrad<T>(L, m, g2, T1, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T3, nullptr, nullptr, &bn1);   // da1
+        const NextBnBwd<T> bn1{S + u.t_b, S + u.t_a, F + u.st1};
+        const int bn1_parts = conv_dgrad<T>(L, m, g2, T1, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T3, nullptr, nullptr, &bn1);   // da1
         bn_backward<T>(L, m, T3, S + u.t_b, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
-                       nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, bn1_ready);      // dc1
+                       nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, bn1_parts);      // dc1
         conv_wgrad<T>(L, m, g1, x, T1, m.grad + u.w1);
         const bool need_dx = !(m.k == 1 && i == 0);
         if (u.proj) {
@@ -777,10 +796,10 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
           conv_wgrad<T>(L, m, gs, x, T2, m.grad + u.ws);
           if (need_dx) {
             conv_dgrad<T>(L, m, gs, T2, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
-            out_sums_ready = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next);
+            out_sum_parts = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next);
           }
         } else if (need_dx) {
-          out_sums_ready = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y, next);
+          out_sum_parts = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y, next);
         }
         break;
       }
@@ -807,7 +826,7 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
       default: break;
     }
     dy = gout;
-    dy_sums_ready = out_sums_ready;
+    dy_sum_parts = out_sum_parts;
   }
 }
 
@@ -895,26 +914,35 @@ static cudaError_t module_step(fdg_ctx* c, Module& m, cudaStream_t st, StepMode 
     if (k >= 2) { m.last_grad_batch = tau_b; m.last_grad_slot = (int)(t % c->mail_ring); }
   };
   auto rec = [&](cudaEvent_t e) { if (events) L.note(cudaEventRecord(e, st)); };
+  // while the profiler is on, each pass of the module is bracketed by two timing events (after its waits)
+  auto pass_mark = [&]() {
+    if (!c->profiling || !enqueue || c->mod_event_owner.size() >= kProfMaxPairs) return;
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    c->mod_events.push_back(e);
+    if (c->mod_events.size() % 2 == 0) c->mod_event_owner.push_back(k - 1);
+    cudaEventRecord(e, st);
+  };
 
   if (k == K) {
     wait_act();
-    do_forward();
+    pass_mark(); do_forward(); pass_mark();
     rec(m.ev_act[e_now]);
-    do_backward_update();
+    pass_mark(); do_backward_update(); pass_mark();
     rec(m.ev_grad[e_now]);
   } else if (c->cfg.order == FDG_BACKWARD_FIRST) {
     wait_grad();
-    do_backward_update();
+    pass_mark(); do_backward_update(); pass_mark();
     rec(m.ev_grad[e_now]);
     wait_act();
-    do_forward();
+    pass_mark(); do_forward(); pass_mark();
     rec(m.ev_act[e_now]);
   } else {
     wait_act();
-    do_forward();
+    pass_mark(); do_forward(); pass_mark();
     rec(m.ev_act[e_now]);
     wait_grad();
-    do_backward_update();
+    pass_mark(); do_backward_update(); pass_mark();
     rec(m.ev_grad[e_now]);
   }
   if (c->log.size() >= kLogIterations * (size_t)K) c->log.erase(c->log.begin(), c->log.begin() + K);
@@ -969,7 +997,7 @@ static fdg_status make_plan(const fdg_arch* arch, const fdg_config* cfg, fdg_ctx
   c->bf16_mode = cfg->precision == FDG_BF16_TC;
   c->esize = c->bf16_mode ? 2 : 4;
   c->lr = cfg->lr;
-  c->use_graphs = cfg->graphs != 0 && cfg->serial == 0;
+  c->use_graphs = cfg->graphs != 0;
   c->period = 1;
   plan_modules(c);
   return FDG_OK;
@@ -1019,6 +1047,7 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   if (e == cudaSuccess && c->use_graphs) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
   c->ev_cjoin.assign(c->K, nullptr);
   for (int k = 0; k < c->K && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&c->ev_cjoin[k], cudaEventDisableTiming);
+  c->tmaps.share = c->cfg.serial ? 1 : c->K;
   c->graph_exec.assign(c->period, nullptr);
   c->graph_sig.assign(c->period, 0);
   c->graph_launches.assign(c->period, 0);
@@ -1041,6 +1070,7 @@ fdg_status fdg_destroy(fdg_ctx* c) {
   for (cudaEvent_t ev : c->ev_cjoin) if (ev) cudaEventDestroy(ev);
   for (cudaGraphExec_t g : c->graph_exec) if (g) cudaGraphExecDestroy(g);
   for (cudaEvent_t ev : c->prof_events) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : c->mod_events) cudaEventDestroy(ev);
   delete c;
   return e == cudaSuccess ? FDG_OK : FDG_ERR_CUDA;
 }
@@ -1157,12 +1187,13 @@ static cudaError_t run_modules(fdg_ctx* c, cudaStream_t cs, StepMode mode, float
   c->step_sig = 0;
   for (int k = 0; k < c->K; ++k) {
     Module& m = c->mods[k];
-    cudaStream_t st = mode == RUN_SERIAL ? cs : m.stream;
+    const bool one_stream = mode == RUN_SERIAL || c->cfg.serial != 0;
+    cudaStream_t st = one_stream ? cs : m.stream;
     cudaError_t e = cudaSuccess;
-    if (mode == RUN_CAPTURE) e = cudaStreamWaitEvent(st, c->ev_fork, 0);          // the module's stream joins the recording
+    if (mode == RUN_CAPTURE && !one_stream) e = cudaStreamWaitEvent(st, c->ev_fork, 0);   // the module's stream joins the recording
     if (e == cudaSuccess)
       e = c->bf16_mode ? module_step<bf16>(c, m, st, mode, loss_dev) : module_step<float>(c, m, st, mode, loss_dev);
-    if (e == cudaSuccess && mode == RUN_CAPTURE) {
+    if (e == cudaSuccess && mode == RUN_CAPTURE && !one_stream) {
       e = cudaEventRecord(c->ev_cjoin[k], st);
       if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, c->ev_cjoin[k], 0);
     }
@@ -1427,6 +1458,22 @@ fdg_status fdg_profile_read(fdg_ctx* c, fdg_kernel_stat* dst, size_t cap, size_t
   c->prof_recs.clear();
   if (out_n) *out_n = KC_COUNT;
   if (dst) for (size_t i = 0; i < std::min<size_t>(cap, KC_COUNT); ++i) dst[i] = agg[i];
+  return FDG_OK;
+}
+
+fdg_status fdg_profile_read_modules(fdg_ctx* c, double* busy_ms, size_t cap, size_t* out_n) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  std::vector<double> tot(c->K, 0.0);
+  for (size_t i = 0; i < c->mod_event_owner.size(); ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->mod_events[2 * i], c->mod_events[2 * i + 1]) == cudaSuccess) tot[c->mod_event_owner[i]] += ms;
+  }
+  for (cudaEvent_t ev : c->mod_events) cudaEventDestroy(ev);
+  c->mod_events.clear(); c->mod_event_owner.clear();
+  if (out_n) *out_n = (size_t)c->K;
+  if (busy_ms) for (size_t k = 0; k < std::min<size_t>(cap, (size_t)c->K); ++k) busy_ms[k] = tot[k];
   return FDG_OK;
 }
 
