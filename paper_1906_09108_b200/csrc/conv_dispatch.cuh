@@ -142,7 +142,7 @@ inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N,
   if (e == cudaSuccess) e = halo::set_smem_attrs();
   if (e != cudaSuccess) return e;
   const int ctas = halo::wgrad_ctas(p);
-  halo::wgrad_halo_kernel<<<ctas, tc::kThreads, halo::wgrad_smem_bytes(p), st>>>(*mx, *my, p, scratch, err_dev);
+  halo::wgrad_halo_kernel<<<ctas, halo::kFwdThreads, halo::wgrad_smem_bytes(p), st>>>(*mx, *my, p, scratch, err_dev);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t n = (size_t)Co * 9 * Ci;

@@ -375,7 +375,7 @@ struct WgradParams {
   uint32_t tmem_cols;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, WgradParams p,
                   float* __restrict__ partial, int* __restrict__ error_word) {
   extern __shared__ uint8_t smem_raw[];
@@ -401,8 +401,8 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   for (int s = 0; s < p.stages; ++s) {
     uint8_t* xs = smem + (size_t)s * stage_bytes;
     uint8_t* ys = xs + p.x_bytes;
-    for (uint32_t o = p.x_tx_bytes + threadIdx.x * 16; o < p.x_bytes; o += kThreads * 16) *reinterpret_cast<uint4*>(xs + o) = make_uint4(0, 0, 0, 0);
-    for (uint32_t o = p.y_tx_bytes + threadIdx.x * 16; o < p.y_bytes; o += kThreads * 16) *reinterpret_cast<uint4*>(ys + o) = make_uint4(0, 0, 0, 0);
+    for (uint32_t o = p.x_tx_bytes + threadIdx.x * 16; o < p.x_bytes; o += kFwdThreads * 16) *reinterpret_cast<uint4*>(xs + o) = make_uint4(0, 0, 0, 0);
+    for (uint32_t o = p.y_tx_bytes + threadIdx.x * 16; o < p.y_bytes; o += kFwdThreads * 16) *reinterpret_cast<uint4*>(ys + o) = make_uint4(0, 0, 0, 0);
   }
   fence_proxy_async();
   if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
@@ -454,26 +454,29 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       if (ok) tc_commit(done);
     }
   } else {
+    // kEpiGroups groups of four warps share the write-out: the (tap group, 16-column chunk)
+    // items are dealt to the groups in turn.
     const int lane_grp = warp & 3;
+    const int group = (warp - 2) >> 2;
     if (mbar_wait(done, 0, abort_flag)) {
       tc_fence_after();
       const int row = lane_grp * 32 + lane;
       const int sblk = row / p.Ci, ci = row - sblk * p.Ci;
       float* dst = partial + (size_t)blockIdx.x * ((size_t)p.Co * 9 * p.Ci);
-      for (int sg = 0; sg < p.sgroups; ++sg) {
+      const int nchunks = ncols >> 4;
+      const size_t co_stride = (size_t)9 * p.Ci;
+      for (int item = group; item < p.sgroups * nchunks; item += kEpiGroups) {
+        const int sg = item / nchunks, c0 = (item - sg * nchunks) << 4;
         const int sx = sg * p.taps_per_group + sblk;
         const bool valid = sblk < p.taps_per_group && sx < 3;
-        const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(sg * ncols);
-        for (int c0 = 0; c0 < ncols; c0 += 16) {
-          uint32_t v[16];
-          tmem_ld16(taddr + c0, v);
-          tmem_ld_wait();
-          if (!valid) continue;
-          const int b = c0 / p.Co, r = 2 - b, co0 = c0 - b * p.Co;      // Co is a multiple of 16: a chunk stays in one block
+        uint32_t v[16];
+        tmem_ld16(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(sg * ncols + c0), v);
+        tmem_ld_wait();
+        if (!valid) continue;
+        const int b = c0 / p.Co, r = 2 - b, co0 = c0 - b * p.Co;        // Co is a multiple of 16: a chunk stays in one block
+        float* d0 = dst + (size_t)co0 * co_stride + (size_t)(r * 3 + sx) * p.Ci + ci;
 #pragma unroll
-          for (int e = 0; e < 16; ++e)
-            dst[(((size_t)(co0 + e) * 3 + r) * 3 + sx) * p.Ci + ci] = __uint_as_float(v[e]);
-        }
+        for (int e = 0; e < 16; ++e) d0[(size_t)e * co_stride] = __uint_as_float(v[e]);
       }
     }
   }
