@@ -77,6 +77,17 @@ inline bool halo_fprop_eligible(const ConvGeom& g) { return halo_shape(g) && hal
 inline bool halo_dgrad_eligible(const ConvGeom& g) { return halo_shape(g) && halo::fwd_supported(g.N, g.H, g.W, g.Co, g.Ci); }
 inline bool halo_wgrad_eligible(const ConvGeom& g) { return halo_shape(g) && halo::wgrad_supported(g.N, g.H, g.W, g.Ci, g.Co); }
 
+// A 3x3 / stride 2 / pad 1 convolution on even image sizes is the stride-1 convolution kept at the
+// even pixels, and its two gradients are the stride-1 ones taken with dy spread onto the even
+// pixels of a zero tensor of the input's size.  Four times the arithmetic, on kernels that are far
+// from arithmetic-bound; the shapes concerned are two layers of a 6n+2 network.
+inline bool halo_s2_shape(const ConvGeom& g) {
+  return g.R == 3 && g.S == 3 && g.stride == 2 && g.pad == 1 && g.H % 2 == 0 && g.W % 2 == 0 && g.P == g.H / 2 && g.Q == g.W / 2;
+}
+inline bool halo_s2_fprop_eligible(const ConvGeom& g) { return halo_s2_shape(g) && halo::fwd_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+inline bool halo_s2_dgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && halo::fwd_supported(g.N, g.H, g.W, g.Co, g.Ci); }
+inline bool halo_s2_wgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && halo::wgrad_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+
 inline cudaError_t cached_tile_map(TensorMapCache* cache, const void* act, int N, int H, int W, int C, int G,
                                    const CUtensorMap** out) {
   TensorMapCache::Key k;
@@ -114,10 +125,11 @@ inline bool halo_reduce_ok(int Cn) { return Cn <= 64; }
 inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ck, int Cn,
                                  const bf16_t* act, const bf16_t* wgt, bf16_t* out, const bf16_t* res,
                                  const bf16_t* res_mask, int* err_dev, const halo::EpiReduce* red = nullptr,
-                                 int* ctas_out = nullptr) {
+                                 int* ctas_out = nullptr, int sub = 1) {
   int sms = cached_sm_count(cache) / (cache->share > 0 ? cache->share : 1);
   if (sms < 16) sms = 16;
   halo::FwdParams p = halo::fwd_params(N, H, W, Ck, Cn, sms);
+  p.sub = sub;
   const CUtensorMap *mx, *mw;
   cudaError_t e = cached_tile_map(cache, act, N, H, W, Ck, p.G, &mx);
   if (e == cudaSuccess) e = cached_weight_map(cache, wgt, Ck, Cn, &mw);
@@ -152,12 +164,13 @@ inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N,
 
 
 // Does the data gradient of this convolution read the flipped/transposed weight copy?
-inline bool dgrad_uses_flipped(const ConvGeom& g) { return halo_dgrad_eligible(g) || tc_eligible(g); }
+inline bool dgrad_uses_flipped(const ConvGeom& g) { return halo_dgrad_eligible(g) || halo_s2_dgrad_eligible(g) || tc_eligible(g); }
 
 // fp32 scratch elements a weight-gradient call may need (bf16 storage: whichever kernel is chosen).
 inline size_t conv_wgrad_scratch_elems(bool bf16_storage, const ConvGeom& g) {
   size_t n = wgrad_scratch_elems(g);
-  if (bf16_storage && halo_wgrad_eligible(g)) n = std::max(n, halo::wgrad_scratch_elems(g.N, g.H, g.W, g.Ci, g.Co));
+  if (bf16_storage && (halo_wgrad_eligible(g) || halo_s2_wgrad_eligible(g)))
+    n = std::max(n, halo::wgrad_scratch_elems(g.N, g.H, g.W, g.Ci, g.Co));
   return n;
 }
 

@@ -46,6 +46,8 @@ struct FwdParams {
   uint32_t w_tx_bytes;        // bytes one weight-tap load writes
   int nacc;                   // accumulator slots in tensor memory
   uint32_t tmem_cols;
+  int sub;                    // 1, or 2: keep only the pixels with even h and w and store them as an
+                              // [N][H/2][W/2][Cn] tensor (a stride-2 convolution is the stride-1 one subsampled)
 };
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -236,8 +238,9 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         const int m = kTileM * i + lane_grp * 32 + lane;
         const int g = m / p.img_rows, rem = m - g * p.img_rows;
         const int h = rem / p.Wp, w = rem - h * p.Wp;
-        const bool valid = h < p.H && w < p.W && g < p.G && n0 + g < p.N;
-        const size_t base = ((((size_t)(n0 + g) * p.H + h) * p.W) + w) * p.Cn;
+        const bool valid = h < p.H && w < p.W && g < p.G && n0 + g < p.N && (p.sub == 1 || ((h | w) & 1) == 0);
+        const size_t base = p.sub == 1 ? ((((size_t)(n0 + g) * p.H + h) * p.W) + w) * p.Cn
+                                       : ((((size_t)(n0 + g) * (p.H >> 1) + (h >> 1)) * (p.W >> 1)) + (w >> 1)) * p.Cn;
         const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)slot * p.Cn;
         for (int c0 = my_first * 16; c0 < p.Cn; c0 += 16 * kEpiGroups) {
           uint32_t v[16];
@@ -521,11 +524,13 @@ __global__ void __launch_bounds__(256) wgrad_halo_reduce_kernel(const float* __r
 inline uint32_t round_up_u32(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 constexpr size_t kSmemBudget = 200 * 1024;
 
+constexpr size_t kFixedSmem = kRedSmemBytes + 4096;      // reduction scratch, barriers, alignment slack
 inline bool chan_ok(int c) { return c == 16 || c == 32 || c == 64; }
 
 inline FwdParams fwd_params(int N, int H, int W, int Ck, int Cn, int sm_count) {
   FwdParams p{};
   p.W = W; p.H = H; p.N = N; p.Wp = W + 2; p.Hp = H + 2; p.Ck = Ck; p.Cn = Cn;
+  p.sub = 1;
   p.img_rows = p.Hp * p.Wp;
   p.pitch = (uint32_t)Ck * 2;
   p.w_tx_bytes = (uint32_t)Cn * p.pitch;
@@ -539,12 +544,12 @@ inline FwdParams fwd_params(int N, int H, int W, int Ck, int Cn, int sm_count) {
     uint32_t rows = (uint32_t)(kTileM * p.m_tiles + 2 * p.Wp + 2);
     if (rows < (uint32_t)(G * p.img_rows)) rows = (uint32_t)(G * p.img_rows);
     p.stage_bytes = round_up_u32(rows * p.pitch, 1024);
-    if (G == 1 || 2 * (size_t)p.stage_bytes + 9 * (size_t)p.w_tap_bytes + 2048 <= kSmemBudget) break;
+    if (G == 1 || 2 * (size_t)p.stage_bytes + 9 * (size_t)p.w_tap_bytes + kFixedSmem <= kSmemBudget) break;
   }
   p.tiles = (N + p.G - 1) / p.G;
   p.tile_tx_bytes = (uint32_t)(p.G * p.img_rows) * p.pitch;
-  size_t left = kSmemBudget - 9 * (size_t)p.w_tap_bytes - 2048;
-  int stages = (int)(left / p.stage_bytes);
+  const size_t fixed = 9 * (size_t)p.w_tap_bytes + kFixedSmem;
+  int stages = fixed < kSmemBudget ? (int)((kSmemBudget - fixed) / p.stage_bytes) : 0;
   const int per_cta = (p.tiles + (sm_count > 0 ? sm_count : 148) - 1) / (sm_count > 0 ? sm_count : 148);
   if (stages > 3) stages = 3;
   if (stages > per_cta) stages = per_cta;                     // shared memory left free lets other kernels' CTAs co-reside

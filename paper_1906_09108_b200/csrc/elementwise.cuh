@@ -378,6 +378,22 @@ __global__ void add_kernel(const T* __restrict__ a, const T* __restrict__ b, T* 
   }
 }
 
+// up[n][2p][2q][:] = dy[n][p][q][:], zero at the other pixels; dy [N][P][Q][C], up [N][2P][2Q][C], 16-byte vectors.
+template <typename T, int VEC>
+__global__ void upsample2_kernel(const T* __restrict__ dy, T* __restrict__ up, size_t nvec_up, int P, int Q, int C) {
+  const int cv = C / VEC;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec_up; i += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i % cv);
+    size_t pix = i / cv;
+    const int w = (int)(pix % (2 * Q)); pix /= 2 * Q;
+    const int h = (int)(pix % (2 * P));
+    const size_t n = pix / (2 * P);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (((h | w) & 1) == 0) v = reinterpret_cast<const uint4*>(dy)[((n * P + (h >> 1)) * Q + (w >> 1)) * cv + c];
+    reinterpret_cast<uint4*>(up)[i] = v;
+  }
+}
+
 // fp32 [rows][c_in] -> T [rows][c_out], channels c_in..c_out-1 zero (image ingest); labels copied alongside.
 template <typename T>
 __global__ void ingest_kernel(const float* __restrict__ img, T* __restrict__ out, size_t rows, int c_in, int c_out,

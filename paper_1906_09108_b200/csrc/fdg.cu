@@ -90,6 +90,8 @@ struct Module {
   char* temps[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   float *scratch = nullptr, *bnsums = nullptr;
   unsigned int* counter = nullptr;
+  char* up = nullptr;                      // dy of a stride-2 convolution spread onto the input's pixel grid
+  size_t up_elems = 0;
   float* red_partial = nullptr;            // per-CTA partial sums of the reductions fused into convolution epilogues
   unsigned int* red_counter = nullptr;
   float *pooled = nullptr, *dlogits = nullptr, *loss_n = nullptr, *loss = nullptr;   // head
@@ -333,6 +335,12 @@ static void plan_modules(fdg_ctx* c) {
           break;
       }
     }
+    if (c->bf16_mode)
+      for (const Unit& u : m.units) {
+        if ((u.type != U_BASIC && u.type != U_PREACT) || u.stride != 2) continue;
+        ConvGeom g1{a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 3, u.stride, 1};
+        if (halo_s2_dgrad_eligible(g1) || halo_s2_wgrad_eligible(g1)) m.up_elems = std::max(m.up_elems, B * u.H * u.W * u.co);
+      }
     if (c->bf16_mode) {
       size_t fe = 0;
       auto flip = [&](size_t src, int co, int ci) {
@@ -389,6 +397,7 @@ static size_t carve(fdg_ctx* c, char* base) {
     for (const Unit& u : m.units) maxc = std::max(maxc, std::max(u.ci, u.co));
     m.bnsums = cv.take<float>((size_t)kRedMaxSums * maxc * 4);
     m.counter = cv.take<unsigned int>(256);
+    m.up = m.up_elems ? cv.take<char>(align_up(m.up_elems, 128) * es) : nullptr;
     m.red_partial = cv.take<float>((size_t)kRedPartialCtas * 2 * 64 * 4);
     m.red_counter = cv.take<unsigned int>(256);
     if (m.k == c->K) {
@@ -560,6 +569,15 @@ static int conv_fprop(Launch& L, Module& m, const ConvGeom& g, const T* x, const
       L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, fuse ? &r : nullptr, &ctas));
       return fuse ? ctas : 0;
     }
+    if (halo_s2_fprop_eligible(g)) {      // the stride-1 convolution, stored at the even pixels only
+      ++L.c->launches;
+      const bool fuse = want_stats && halo_reduce_ok(g.Co);
+      halo::EpiReduce r{};
+      int ctas = 0;
+      if (fuse) { r.mode = 1; r.partial = m.red_partial; }
+      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, fuse ? &r : nullptr, &ctas, 2));
+      return fuse ? ctas : 0;
+    }
     if (tc_eligible(g)) {
       ++L.c->launches;
       L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error));
@@ -577,7 +595,7 @@ template <typename T> struct NextBnBwd { const T* mask; const T* x; const float*
 
 template <typename T>
 static int conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, const T* w, const T* wflip, T* dx,
-                       const T* res, const T* mask, const NextBnBwd<T>* next = nullptr) {
+                       const T* res, const T* mask, const NextBnBwd<T>* next = nullptr, const T* dy_up = nullptr) {
   L.begin(KC_CONV_DGRAD, (out_elems(g) + w_elems(g) + in_elems(g) * (1 + (res ? 1 : 0) + (mask ? 1 : 0) + (next ? 2 : 0))) * sizeof(T), conv_flops(g));
   if constexpr (std::is_same<T, bf16>::value) {
     if (wflip && halo_dgrad_eligible(g)) {
@@ -587,6 +605,15 @@ static int conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, cons
       int ctas = 0;
       if (fuse) { r.mode = 2; r.mask = next->mask; r.xprev = next->x; r.pstats = next->stats; r.partial = m.red_partial; }
       L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error, fuse ? &r : nullptr, &ctas));
+      return fuse ? ctas : 0;
+    }
+    if (wflip && dy_up && halo_s2_dgrad_eligible(g)) {      // stride 2: the stride-1 data gradient of the spread-out dy
+      ++L.c->launches;
+      const bool fuse = next && halo_reduce_ok(g.Ci);
+      halo::EpiReduce r{};
+      int ctas = 0;
+      if (fuse) { r.mode = 2; r.mask = next->mask; r.xprev = next->x; r.pstats = next->stats; r.partial = m.red_partial; }
+      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy_up, wflip, dx, res, mask, L.c->tc_error, fuse ? &r : nullptr, &ctas));
       return fuse ? ctas : 0;
     }
     if (wflip && tc_eligible(g)) {
@@ -599,9 +626,14 @@ static int conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, cons
   return 0;
 }
 template <typename T>
-static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* dy, float* dw) {
+static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* dy, float* dw, const T* dy_up = nullptr) {
   L.begin(KC_CONV_WGRAD, (in_elems(g) + out_elems(g)) * sizeof(T) + w_elems(g) * 4, conv_flops(g));
   if constexpr (std::is_same<T, bf16>::value) {
+    if (dy_up && halo_s2_wgrad_eligible(g)) {                // stride 2: the stride-1 weight gradient with the spread-out dy
+      L.c->launches += 2;
+      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy_up, dw, m.scratch, L.c->tc_error));
+      return;
+    }
     if (halo_wgrad_eligible(g)) {
       L.c->launches += 2;
       L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy, dw, m.scratch, L.c->tc_error));
@@ -615,6 +647,22 @@ template <typename T> static const T* flipped_of(const Module& m, int vslot, lon
 template <> const float* flipped_of<float>(const Module&, int, long long) { return nullptr; }
 template <> const bf16* flipped_of<bf16>(const Module& m, int vslot, long long off) {
   return off < 0 ? nullptr : m.wflip16 + (size_t)vslot * m.flip_elems + off;
+}
+
+// dy [N][P][Q][Co] of a stride-2 convolution, spread onto the even pixels of a zero [N][H][W][Co] tensor
+// (module scratch); null when the stride-2 gradients of this shape stay on the CUDA cores.
+template <typename T>
+static const T* upsample_dy(Launch& L, Module& m, const ConvGeom& g, const T* dy) {
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (!m.up || !(halo_s2_dgrad_eligible(g) || halo_s2_wgrad_eligible(g)) || g.Co % 8) return nullptr;
+    T* up = reinterpret_cast<T*>(m.up);
+    const size_t nvec = (size_t)g.N * g.H * g.W * g.Co / 8;
+    L.begin(KC_CONV_DGRAD, (double)nvec * 16 * 1.25, 0.0);
+    upsample2_kernel<T, 8><<<ew_blocks(nvec), 256, 0, L.st>>>(dy, up, nvec, g.P, g.Q, g.Co);
+    L.check();
+    return up;
+  }
+  return nullptr;
 }
 
 // ------------------------------------------------------------ module passes ---
@@ -789,14 +837,15 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
         const int bn1_parts = conv_dgrad<T>(L, m, g2, T1, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T3, nullptr, nullptr, &bn1);   // da1
         bn_backward<T>(L, m, T3, S + u.t_b, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
                        nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, bn1_parts);      // dc1
-        conv_wgrad<T>(L, m, g1, x, T1, m.grad + u.w1);
+        const T* up = u.stride == 2 ? upsample_dy<T>(L, m, g1, T1) : nullptr;
+        conv_wgrad<T>(L, m, g1, x, T1, m.grad + u.w1, up);
         const bool need_dx = !(m.k == 1 && i == 0);
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_wgrad<T>(L, m, gs, x, T2, m.grad + u.ws);
           if (need_dx) {
             conv_dgrad<T>(L, m, gs, T2, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
-            out_sum_parts = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next);
+            out_sum_parts = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next, up);
           }
         } else if (need_dx) {
           out_sum_parts = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y, next);

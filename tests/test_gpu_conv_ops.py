@@ -35,7 +35,9 @@ SHAPES_TC = [(4, 32, 32, 16, 16, 3, 1, 1),      # 32 tiles of 4 image rows, 32-b
              (3, 6, 10, 64, 16, 3, 1, 1),
              (37, 16, 16, 32, 64, 3, 1, 1),     # ragged last tile in the weight gradient's pixel split
              (301, 8, 8, 64, 64, 3, 1, 1),      # ragged last tile with several images per tile
-             (130, 32, 32, 16, 16, 3, 1, 1)]    # stage-1 shape of the 6n+2 networks, more images than weight-gradient CTAs
+             (130, 32, 32, 16, 16, 3, 1, 1),    # stage-1 shape of the 6n+2 networks, more images than weight-gradient CTAs
+             (6, 32, 32, 16, 32, 3, 2, 1),      # stride 2: forward = the stride-1 kernel stored at the even pixels
+             (9, 16, 16, 32, 64, 3, 2, 1)]
 
 # shapes whose three operators all take the halo-tile tensor-core kernels
 ALL_TC = {(4, 32, 32, 16, 16), (6, 16, 16, 32, 32), (10, 8, 8, 64, 64), (300, 8, 8, 64, 64), (5, 12, 20, 16, 32),
