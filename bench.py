@@ -142,7 +142,7 @@ KERNEL_SHAPES = {     # the three 3x3 stride-1 layer shapes of the workload: (N,
     "stage1": (128, 32, 32, 16), "stage2": (128, 16, 16, 32), "stage3": (128, 8, 8, 64)}
 
 
-def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5):
+def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5, use_graph=True):
     """Average duration of one convolution kernel launch, timed alone: `launches` calls of the operator-level
     entry point, each on its own input/output pair out of a pool larger than the L2 cache (so every launch
     reads HBM), recorded once into a CUDA graph and replayed; CUDA events around the replay on its stream.
@@ -181,16 +181,22 @@ def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5):
         for i in range(pool):                      # ordinary launches first: tensor maps and attributes get set up
             call(i)
         st.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=st):
-            for i in range(launches):
-                call(i)
-        graph.replay()
+        if use_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=st):
+                for i in range(launches):
+                    call(i)
+            replay = graph.replay
+        else:                                      # plain launches: what a profiler run uses
+            def replay():
+                for i in range(launches):
+                    call(i)
+        replay()
         st.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(st)
         for _ in range(reps):
-            graph.replay()
+            replay()
         e1.record(st)
         st.synchronize()
     assert not ops.timed_out()
@@ -204,9 +210,11 @@ def run_kernel_bench(args):
     peaks = measured_peaks()
     out = {}
     which_list = [args.kernel_bench] if args.kernel_bench != "all" else ["fprop", "dgrad", "wgrad"]
+    stages = [args.kernel_stage] if args.kernel_stage else list(KERNEL_SHAPES)
     for which in which_list:
-        for stage in KERNEL_SHAPES:
-            us, nbytes, flops = kernel_bench(B, which, stage, launches=args.kernel_launches)
+        for stage in stages:
+            us, nbytes, flops = kernel_bench(B, which, stage, launches=args.kernel_launches,
+                                             reps=1 if args.kernel_launches <= 8 else 5, use_graph=args.kernel_launches > 8)
             out["%s_%s" % (which, stage)] = dict(us=us, gbs=nbytes / us / 1e3, tflops=flops / us / 1e6,
                                                  hbm_frac=nbytes / us / 1e3 / peaks["hbm_gbs"])
     print(json.dumps(dict(kernel_bench=out, peak_source=peaks["source"], hbm_gbs=peaks["hbm_gbs"])))
@@ -227,8 +235,8 @@ def run_gpu(args):
     import fdg_synth as S
     from paper_1906_09108_b200 import binding as B
 
-    steps = args.steps if args.steps is not None else 50
-    warmup = args.warmup if args.warmup is not None else 10
+    steps = args.steps if args.steps is not None else 300
+    warmup = args.warmup if args.warmup is not None else 20
     warmup = max(warmup, 3)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -390,7 +398,9 @@ def main():
     ap.add_argument("--no-graphs", action="store_true")
     ap.add_argument("--kernel-bench", default=None, choices=["fprop", "dgrad", "wgrad", "all"],
                     help="time the convolution kernels alone through the operator-level C ABI and exit")
-    ap.add_argument("--kernel-launches", type=int, default=64)
+    ap.add_argument("--kernel-launches", type=int, default=64,
+                    help="launches per replay; 8 or fewer are issued as plain launches (profiler runs)")
+    ap.add_argument("--kernel-stage", default=None, choices=list(KERNEL_SHAPES))
     ap.add_argument("--device-arm-only", action="store_true",
                     help="time the device-resident arm only (no end-to-end arm, no per-kernel roofline, no CPU "
                          "baseline): the short run the ncu launch list is taken from")
