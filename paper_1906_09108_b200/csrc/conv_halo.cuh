@@ -91,7 +91,11 @@ struct EpiReduce {
 // steps (wait, tensor-memory load, global loads, shuffles), so several must be in flight.
 constexpr int kEpiGroups = 4;
 constexpr int kEpiWarps = 4 * kEpiGroups;
-constexpr int kFwdThreads = 64 + 32 * kEpiWarps;
+// One thread can issue a tcgen05.mma every ~75 cycles, the tensor pipe takes one of these small
+// instructions every ~40: two issuing warps (alternate 128-row tiles) keep it busier (measured).
+constexpr int kMmaWarps = 2;
+constexpr int kFirstEpiWarp = 1 + kMmaWarps;
+constexpr int kFwdThreads = 32 * (kFirstEpiWarp + kEpiWarps);
 constexpr int kRedSmemBytes = kEpiWarps * 8 * 32 * 4 + 2 * 128 * 4;   // running sums, statistics
 
 // 32 lanes each hold 32 items; afterwards lane l holds in q[0] the sum over all lanes of item l.
@@ -148,7 +152,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       for (int i = threadIdx.x; i < 2 * p.Cn; i += kFwdThreads) red_stat[i] = red.pstats[i];
   }
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kMmaWarps); }
     mbar_init(w_full, 1);
     const int groups_per_tile = p.Cn / 16 < kEpiGroups ? p.Cn / 16 : kEpiGroups;
     for (int a = 0; a < p.nacc; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4 * groups_per_tile); }
@@ -175,8 +179,9 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         tma_load_4d(smem + (size_t)s * p.stage_bytes, &map_x, &full[s], 0, -1, -1, tile * p.G);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp < kFirstEpiWarp) {
     if (lane == 0) {
+      const uint32_t issuer = warp - 1;                       // takes the 128-row tiles with acount % kMmaWarps == issuer
       const uint32_t idesc = instr_desc(p.Cn, false);
       bool ok = mbar_wait(w_full, 0, abort_flag);
       tc_fence_after();
@@ -202,15 +207,17 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         tc_fence_after();
         uint64_t x_desc = smem_desc_kmajor(smem_u32(smem + (size_t)s * p.stage_bytes), p.pitch);
         for (int i = 0; i < p.m_tiles; ++i, ++acount, x_desc += mtile_step) {
-          if (acount >= (uint32_t)p.nacc) {                   // a slot's first use needs no hand-back from the epilogue
-            if (!mbar_wait(&acc_empty[slot], aph ^ 1, abort_flag)) { ok = false; break; }
-            tc_fence_after();
+          if (acount % kMmaWarps == issuer) {
+            if (acount >= (uint32_t)p.nacc) {                 // a slot's first use needs no hand-back from the epilogue
+              if (!mbar_wait(&acc_empty[slot], aph ^ 1, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+            }
+            const uint32_t d_tmem = tmem_base + (uint32_t)slot * p.Cn;
+            if (ksteps == 1) issue_tile<1>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
+            else if (ksteps == 2) issue_tile<2>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
+            else issue_tile<4>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
+            tc_commit(&acc_full[slot]);
           }
-          const uint32_t d_tmem = tmem_base + (uint32_t)slot * p.Cn;
-          if (ksteps == 1) issue_tile<1>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
-          else if (ksteps == 2) issue_tile<2>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
-          else issue_tile<4>(d_tmem, x_desc, tap_off, w_desc0, w_tap_step, idesc);
-          tc_commit(&acc_full[slot]);
           if (++slot == p.nacc) { slot = 0; aph ^= 1; }
         }
         if (!ok) break;
@@ -219,7 +226,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     }
   } else {
     const int lane_grp = warp & 3;                 // tensor-memory lanes 32*(warp % 4) .. +31
-    const int group = (warp - 2) >> 2;
+    const int group = (warp - kFirstEpiWarp) >> 2;
     uint32_t acount = 0;
     for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x) {
       const int n0 = tile * p.G;
@@ -313,7 +320,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
               }
             }
             transpose_reduce32(q, lane);
-            red_run[((warp - 2) * 8 + (c0 >> 4)) * 32 + lane] += q[0];
+            red_run[((warp - kFirstEpiWarp) * 8 + (c0 >> 4)) * 32 + lane] += q[0];
           }
         }
         tc_fence_before();
@@ -460,8 +467,8 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // kEpiGroups groups of four warps share the write-out: the (tap group, 16-column chunk)
     // items are dealt to the groups in turn.
     const int lane_grp = warp & 3;
-    const int group = (warp - 2) >> 2;
-    if (mbar_wait(done, 0, abort_flag)) {
+    const int group = ((warp - 2) >> 2) % kEpiGroups;        // (this kernel has one issuing warp; warp 18 idles with group 0's lanes taken)
+    if (warp < 2 + kEpiWarps && mbar_wait(done, 0, abort_flag)) {
       tc_fence_after();
       const int row = lane_grp * 32 + lane;
       const int sblk = row / p.Ci, ci = row - sblk * p.Ci;
