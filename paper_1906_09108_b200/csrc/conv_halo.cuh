@@ -400,8 +400,8 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(done, 1);
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kMmaWarps); }
+    mbar_init(done, kMmaWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -435,11 +435,15 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         tma_load_4d(xs + p.x_bytes, &map_y, &full[s], 0, 0, -2, tile * p.G);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp < kFirstEpiWarp) {
     if (lane == 0) {
+      // Two issuing warps.  One tap group (Ci <= 32): the reduction steps alternate between them, each
+      // into its own copy of the accumulator (the epilogue adds the two).  Two tap groups: one each.
+      const uint32_t issuer = warp - 1;
       const uint32_t idesc = instr_desc(ncols, true);
       const uint64_t a_kstep = (uint64_t)(16 * p.pitch_x) >> 4, b_kstep = (uint64_t)(16 * p.pitch_y) >> 4;
       const uint64_t a_group = (uint64_t)(p.taps_per_group * p.pitch_x) >> 4;
+      const uint32_t d_tmem = tmem_base + issuer * (uint32_t)ncols;
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
@@ -451,13 +455,13 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         uint64_t a_desc = smem_desc_mnmajor(x_addr, p.pitch_x, p.pitch_x);
         uint64_t b_desc = smem_desc_mnmajor(x_addr + p.x_bytes, p.pitch_y, (uint32_t)p.Wp * p.pitch_y);
         if (p.sgroups == 1) {
-          for (int j = 0; j < p.ksteps; ++j, a_desc += a_kstep, b_desc += b_kstep)
-            tc_mma_bf16(tmem_base, a_desc, b_desc, idesc, (it | (uint32_t)j) != 0);
+          a_desc += issuer * a_kstep; b_desc += issuer * b_kstep;
+          for (int j = (int)issuer; j < p.ksteps; j += kMmaWarps, a_desc += kMmaWarps * a_kstep, b_desc += kMmaWarps * b_kstep)
+            tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, it != 0 || j >= kMmaWarps);
         } else {
-          for (int j = 0; j < p.ksteps; ++j, a_desc += a_kstep, b_desc += b_kstep) {
-            tc_mma_bf16(tmem_base, a_desc, b_desc, idesc, (it | (uint32_t)j) != 0);
-            tc_mma_bf16(tmem_base + (uint32_t)ncols, a_desc + a_group, b_desc, idesc, (it | (uint32_t)j) != 0);
-          }
+          a_desc += issuer * a_group;
+          for (int j = 0; j < p.ksteps; ++j, a_desc += a_kstep, b_desc += b_kstep)
+            tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, (it | (uint32_t)j) != 0);
         }
         tc_commit(&empty[s]);
       }
@@ -467,8 +471,8 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // kEpiGroups groups of four warps share the write-out: the (tap group, 16-column chunk)
     // items are dealt to the groups in turn.
     const int lane_grp = warp & 3;
-    const int group = ((warp - 2) >> 2) % kEpiGroups;        // (this kernel has one issuing warp; warp 18 idles with group 0's lanes taken)
-    if (warp < 2 + kEpiWarps && mbar_wait(done, 0, abort_flag)) {
+    const int group = (warp - kFirstEpiWarp) >> 2;
+    if (mbar_wait(done, 0, abort_flag)) {
       tc_fence_after();
       const int row = lane_grp * 32 + lane;
       const int sblk = row / p.Ci, ci = row - sblk * p.Ci;
@@ -482,6 +486,13 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         uint32_t v[16];
         tmem_ld16(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(sg * ncols + c0), v);
         tmem_ld_wait();
+        if (p.sgroups == 1) {                     // the second issuer's copy of the accumulator
+          uint32_t u[16];
+          tmem_ld16(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(ncols + c0), u);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(u[e]));
+        }
         if (!valid) continue;
         const int b = c0 / p.Co, r = 2 - b, co0 = c0 - b * p.Co;        // Co is a multiple of 16: a chunk stays in one block
         float* d0 = dst + (size_t)co0 * co_stride + (size_t)(r * 3 + sx) * p.Ci + ci;
@@ -604,7 +615,7 @@ inline WgradParams wgrad_params(int N, int H, int W, int Ci, int Co) {
   const size_t stage = (size_t)p.x_bytes + p.y_bytes;
   int stages = (int)((kSmemBudget - 2048) / stage);
   p.stages = stages > 2 ? 2 : stages;
-  uint32_t need = (uint32_t)(p.sgroups * 3 * Co), cols = 32;
+  uint32_t need = (uint32_t)(2 * 3 * Co), cols = 32;            // two accumulators: two tap groups, or two copies of one
   while (cols < need) cols <<= 1;
   p.tmem_cols = cols;
   return p;
