@@ -87,8 +87,10 @@ struct Module {
   float* fifo_f = nullptr;                 // D slots of slot_floats
   char* in_ring = nullptr;                 // module 1: Din image slots
   char* mail = nullptr;                    // kMailRing slots of in_elems (k >= 2)
-  char* temps[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  char* temps[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   float *scratch = nullptr, *bnsums = nullptr;
+  float* wscratch = nullptr;               // partial sums of the weight-gradient kernels (they run on the side stream)
+  size_t wscratch_floats = 0;
   unsigned int* counter = nullptr;
   char* up = nullptr;                      // dy of a stride-2 convolution spread onto the input's pixel grid
   size_t up_elems = 0;
@@ -101,6 +103,8 @@ struct Module {
   int64_t last_out_batch = -1, last_grad_batch = -1;
   int last_out_slot = -1, last_grad_slot = -1;
   cudaStream_t stream = nullptr;
+  cudaStream_t stream2 = nullptr;          // side stream: weight gradients run beside the data-gradient chain
+  cudaEvent_t ev_fork2 = nullptr, ev_join2 = nullptr, ev_buf[4] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t ev_act[kEventRing], ev_grad[kEventRing];
 };
 
@@ -296,13 +300,13 @@ static void plan_modules(fdg_ctx* c) {
       c->period = std::max(c->period, std::max(m.D, std::max(m.Dw, m.Din)));
     }
     m.in_elems = B * m.in_h * m.in_w * m.in_c;
-    size_t te = 0, tf = 0, maxa = m.in_elems, scr = 0;
+    size_t te = 0, tf = 0, maxa = m.in_elems, scr = 0, wscr = 0;
     auto tens = [&](size_t e) { size_t o = te; te += align_up(e, 128); maxa = std::max(maxa, e); return o; };
     auto stat = [&](int ch) { size_t o = tf; tf += align_up((size_t)2 * ch, 64); return o; };
     auto red_scratch = [&](size_t rows, int ch) { scr = std::max(scr, (size_t)kRedMaxBlocks * kRedMaxSums * ch); (void)rows; };
     auto wg_scratch = [&](int n, int h, int w, int cin, int p, int q, int cout, int r, int stride, int pad) {
       ConvGeom g{n, h, w, cin, p, q, cout, r, r, stride, pad};
-      scr = std::max(scr, conv_wgrad_scratch_elems(c->bf16_mode, g));
+      wscr = std::max(wscr, conv_wgrad_scratch_elems(c->bf16_mode, g));
     };
     for (Unit& u : m.units) {
       const size_t in_e = B * u.H * u.W * u.ci, out_e = B * u.P * u.Q * u.co;
@@ -359,7 +363,7 @@ static void plan_modules(fdg_ctx* c) {
       }
       m.flip_elems = fe;
     }
-    m.slot_elems = te; m.slot_floats = tf; m.max_act = maxa; m.scratch_floats = scr;
+    m.slot_elems = te; m.slot_floats = tf; m.max_act = maxa; m.scratch_floats = scr; m.wscratch_floats = wscr;
     const Unit& last = m.units.back();
     if (kp < K) { m.out_elems = B * last.P * last.Q * last.co; m.out_c = last.co; }
     m.slot_version.assign(m.D, -1);
@@ -391,8 +395,9 @@ static size_t carve(fdg_ctx* c, char* base) {
     m.fifo_f = cv.take<float>((size_t)m.D * std::max<size_t>(m.slot_floats, 64) * 4);
     m.in_ring = m.Din ? cv.take<char>((size_t)m.Din * align_up(m.in_elems, 128) * es) : nullptr;
     m.mail = m.k >= 2 ? cv.take<char>((size_t)c->mail_ring * align_up(m.in_elems, 128) * es) : nullptr;
-    for (int i = 0; i < 5; ++i) m.temps[i] = cv.take<char>(align_up(m.max_act, 128) * es);
+    for (int i = 0; i < 6; ++i) m.temps[i] = cv.take<char>(align_up(m.max_act, 128) * es);
     m.scratch = cv.take<float>(std::max<size_t>(m.scratch_floats, 64) * 4);
+    m.wscratch = cv.take<float>(std::max<size_t>(m.wscratch_floats, 64) * 4);
     int maxc = 1;
     for (const Unit& u : m.units) maxc = std::max(maxc, std::max(u.ci, u.co));
     m.bnsums = cv.take<float>((size_t)kRedMaxSums * maxc * 4);
@@ -631,16 +636,16 @@ static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, cons
   if constexpr (std::is_same<T, bf16>::value) {
     if (dy_up && halo_s2_wgrad_eligible(g)) {                // stride 2: the stride-1 weight gradient with the spread-out dy
       L.c->launches += 2;
-      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy_up, dw, m.scratch, L.c->tc_error));
+      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy_up, dw, m.wscratch, L.c->tc_error));
       return;
     }
     if (halo_wgrad_eligible(g)) {
       L.c->launches += 2;
-      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy, dw, m.scratch, L.c->tc_error));
+      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy, dw, m.wscratch, L.c->tc_error));
       return;
     }
   }
-  L.note(launch_conv_simt<T, CONV_WGRAD>(L.st, g, x, dy, (T*)nullptr, m.scratch, dw, (const T*)nullptr, (const T*)nullptr, &L.c->launches));
+  L.note(launch_conv_simt<T, CONV_WGRAD>(L.st, g, x, dy, (T*)nullptr, m.wscratch, dw, (const T*)nullptr, (const T*)nullptr, &L.c->launches));
 }
 
 template <typename T> static const T* flipped_of(const Module& m, int vslot, long long off);
@@ -780,8 +785,13 @@ static void head_forward_backward(fdg_ctx* c, Module& m, Launch& L, int64_t tau,
 // Chain rule through the module's blocks (and stem) for the batch saved in `slot`.
 //   gin   gradient with respect to the module output (already shrunk), consumed
 //   gfirst where the gradient of the module input goes (mailbox slot; unused for module 1)
+// `LS` issues on the module's side stream (the same stream as L when `forked` is false): the weight
+// gradients run there, beside the chain batch-norm backward -> data gradient -> next layer.  Buffers
+// a weight gradient reads (0: T1, 1: T4, 2: T2, 3: the spread-out dy) are not rewritten on the main
+// stream before the event recorded behind their last reader.
 template <typename T>
-static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int slot, int vslot, T* gin, T* gfirst) {
+static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool forked, int64_t tau, int slot, int vslot,
+                            T* gin, T* gfirst) {
   const int B = c->arch.batch;
   const T* wt = weights_of<T>(m, vslot);
   const float* wf = m.wver + (size_t)vslot * align_up(m.n_params, 64);
@@ -791,6 +801,15 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
   T* T1 = reinterpret_cast<T*>(m.temps[2]);
   T* T2 = reinterpret_cast<T*>(m.temps[3]);
   T* T3 = reinterpret_cast<T*>(m.temps[4]);
+  T* T4 = reinterpret_cast<T*>(m.temps[5]);
+  bool buf_read[4] = {false, false, false, false};
+  auto fork = [&]() {
+    if (!forked) return;
+    L.note(cudaEventRecord(m.ev_fork2, L.st));
+    LS.note(cudaStreamWaitEvent(LS.st, m.ev_fork2, 0));
+  };
+  auto side_done = [&](int b) { if (forked) { LS.note(cudaEventRecord(m.ev_buf[b], LS.st)); buf_read[b] = true; } };
+  auto wait_buf = [&](int b) { if (forked && buf_read[b]) L.note(cudaStreamWaitEvent(L.st, m.ev_buf[b], 0)); };
   T* dy = gin;
   int dy_sum_parts = 0;            // > 0: the kernel that produced dy left that many rows of partial sums for the
                                    // first batch-norm backward it meets
@@ -816,39 +835,53 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
         ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
         const T* dc = dy;
         if (u.bn) {
+          wait_buf(0);
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
                          nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sum_parts);
           dc = T1;
         }
-        conv_wgrad<T>(L, m, g, x, dc, m.grad + u.w1);
+        fork();
+        conv_wgrad<T>(LS, m, g, x, dc, m.grad + u.w1);
+        side_done(0);
         break;
       }
       case U_BASIC: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
-        if (u.proj)
+        wait_buf(0);
+        if (u.proj) {
+          wait_buf(2);
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_c, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, S + u.t_s,
                          F + u.sts, wf + u.gs, m.grad + u.gs, m.grad + u.bs, nullptr, T1, T2, rows_out, u.co);
-        else
+        } else {
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_c, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
                          nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sum_parts);
-        conv_wgrad<T>(L, m, g2, S + u.t_b, T1, m.grad + u.w2);
+        }
+        fork();
+        conv_wgrad<T>(LS, m, g2, S + u.t_b, T1, m.grad + u.w2);                                          // side
+        side_done(0);
         const NextBnBwd<T> bn1{S + u.t_b, S + u.t_a, F + u.st1};
         const int bn1_parts = conv_dgrad<T>(L, m, g2, T1, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T3, nullptr, nullptr, &bn1);   // da1
+        wait_buf(1);
         bn_backward<T>(L, m, T3, S + u.t_b, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
-                       nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, bn1_parts);      // dc1
-        const T* up = u.stride == 2 ? upsample_dy<T>(L, m, g1, T1) : nullptr;
-        conv_wgrad<T>(L, m, g1, x, T1, m.grad + u.w1, up);
+                       nullptr, nullptr, nullptr, nullptr, nullptr, T4, nullptr, rows_out, u.co, bn1_parts);      // dc1
+        const T* up = nullptr;
+        if (u.stride == 2) { wait_buf(3); up = upsample_dy<T>(L, m, g1, T4); }
+        fork();
+        conv_wgrad<T>(LS, m, g1, x, T4, m.grad + u.w1, up);                                              // side
+        side_done(1);
+        if (up) side_done(3);
         const bool need_dx = !(m.k == 1 && i == 0);
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
-          conv_wgrad<T>(L, m, gs, x, T2, m.grad + u.ws);
+          conv_wgrad<T>(LS, m, gs, x, T2, m.grad + u.ws);                                                // side
+          side_done(2);
           if (need_dx) {
             conv_dgrad<T>(L, m, gs, T2, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
-            out_sum_parts = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next, up);
+            out_sum_parts = conv_dgrad<T>(L, m, g1, T4, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next, up);
           }
         } else if (need_dx) {
-          out_sum_parts = conv_dgrad<T>(L, m, g1, T1, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y, next);
+          out_sum_parts = conv_dgrad<T>(L, m, g1, T4, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y, next);
         }
         break;
       }
@@ -876,6 +909,10 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int s
     }
     dy = gout;
     dy_sum_parts = out_sum_parts;
+  }
+  if (forked) {      // every parameter gradient is in place before the update that follows
+    LS.note(cudaEventRecord(m.ev_join2, LS.st));
+    L.note(cudaStreamWaitEvent(L.st, m.ev_join2, 0));
   }
 }
 
@@ -955,7 +992,10 @@ static cudaError_t module_step(fdg_ctx* c, Module& m, cudaStream_t st, StepMode 
         if (loss_dev && mode != RUN_CAPTURE) L.note(cudaMemcpyAsync(loss_dev, m.loss, sizeof(float), cudaMemcpyDeviceToDevice, st));
       }
       T* gfirst = k >= 2 ? reinterpret_cast<T*>(m.mail) + (size_t)(t % c->mail_ring) * align_up(m.in_elems, 128) : nullptr;
-      backward_module<T>(c, m, L, tau_b, slot, vslot, gin, gfirst);
+      const bool forked = (mode == RUN_STREAMS || mode == RUN_CAPTURE) && c->cfg.serial == 0;
+      Launch LS{c, forked ? m.stream2 : st};
+      backward_module<T>(c, m, L, LS, forked, tau_b, slot, vslot, gin, gfirst);
+      if (L.err == cudaSuccess) L.err = LS.err;
       update_module<T>(c, m, L, next_vslot);
     }
     m.updates += 1;
@@ -1011,7 +1051,11 @@ static fdg_status cuda_fail(fdg_ctx* c, cudaError_t e, const char* where) {
 static cudaError_t drain(fdg_ctx* c) {
   cudaError_t e = cudaSuccess;
   if (c->stepped) e = cudaStreamSynchronize(c->last_stream);
-  for (Module& m : c->mods) { cudaError_t r = cudaStreamSynchronize(m.stream); if (e == cudaSuccess) e = r; }
+  for (Module& m : c->mods) {
+    cudaError_t r = cudaStreamSynchronize(m.stream);
+    if (e == cudaSuccess) e = r;
+    if (m.stream2) { r = cudaStreamSynchronize(m.stream2); if (e == cudaSuccess) e = r; }
+  }
   return e;
 }
 
@@ -1085,6 +1129,10 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
     Module& m = c->mods[k];
     if (streams) m.stream = static_cast<cudaStream_t>(streams[k]);
     else e = cudaStreamCreateWithFlags(&m.stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&m.stream2, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.ev_fork2, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.ev_join2, cudaEventDisableTiming);
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&m.ev_buf[i], cudaEventDisableTiming);
     for (int i = 0; i < kEventRing && e == cudaSuccess; ++i) {
       e = cudaEventCreateWithFlags(&m.ev_act[i], cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m.ev_grad[i], cudaEventDisableTiming);
@@ -1111,6 +1159,10 @@ fdg_status fdg_destroy(fdg_ctx* c) {
   for (Module& m : c->mods) {
     for (int i = 0; i < kEventRing; ++i) { cudaEventDestroy(m.ev_act[i]); cudaEventDestroy(m.ev_grad[i]); }
     if (c->own_streams && m.stream) cudaStreamDestroy(m.stream);
+    if (m.stream2) cudaStreamDestroy(m.stream2);
+    if (m.ev_fork2) cudaEventDestroy(m.ev_fork2);
+    if (m.ev_join2) cudaEventDestroy(m.ev_join2);
+    for (int i = 0; i < 4; ++i) if (m.ev_buf[i]) cudaEventDestroy(m.ev_buf[i]);
   }
   for (int i = 0; i < kEventRing; ++i) cudaEventDestroy(c->ev_in[i]);
   cudaEventDestroy(c->ev_join);
