@@ -803,8 +803,10 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
   T* T3 = reinterpret_cast<T*>(m.temps[4]);
   T* T4 = reinterpret_cast<T*>(m.temps[5]);
   bool buf_read[4] = {false, false, false, false};
+  bool side_used = false;
   auto fork = [&]() {
     if (!forked) return;
+    side_used = true;
     L.note(cudaEventRecord(m.ev_fork2, L.st));
     LS.note(cudaStreamWaitEvent(LS.st, m.ev_fork2, 0));
   };
@@ -910,7 +912,7 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
     dy = gout;
     dy_sum_parts = out_sum_parts;
   }
-  if (forked) {      // every parameter gradient is in place before the update that follows
+  if (forked && side_used) {      // every parameter gradient is in place before the update that follows
     LS.note(cudaEventRecord(m.ev_join2, LS.st));
     L.note(cudaStreamWaitEvent(L.st, m.ev_join2, 0));
   }
