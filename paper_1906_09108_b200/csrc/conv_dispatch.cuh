@@ -89,14 +89,15 @@ inline bool halo_s2_dgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) 
 inline bool halo_s2_wgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && halo::wgrad_supported(g.N, g.H, g.W, g.Ci, g.Co); }
 
 inline cudaError_t cached_tile_map(TensorMapCache* cache, const void* act, int N, int H, int W, int C, int G,
-                                   const CUtensorMap** out) {
+                                   const CUtensorMap** out, int boxC = 0) {
+  if (boxC == 0) boxC = C;
   TensorMapCache::Key k;
   std::memset(&k, 0, sizeof(k));
-  k.ptr = act; k.d[0] = 3; k.d[1] = N; k.d[2] = H; k.d[3] = W; k.d[4] = C; k.d[5] = G;
+  k.ptr = act; k.d[0] = 3; k.d[1] = N; k.d[2] = H; k.d[3] = W; k.d[4] = C; k.d[5] = G; k.d[6] = boxC;
   auto it = cache->maps.find(k);
   if (it == cache->maps.end()) {
     CUtensorMap m;
-    cudaError_t e = halo::make_tile_map(act, N, H, W, C, G, &m);
+    cudaError_t e = halo::make_tile_map(act, N, H, W, C, G, &m, boxC);
     if (e != cudaSuccess) return e;
     it = cache->maps.insert({k, m}).first;
   }
@@ -149,12 +150,12 @@ inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N,
                                   const bf16_t* x, const bf16_t* dy, float* dw, float* scratch, int* err_dev) {
   halo::WgradParams p = halo::wgrad_params(N, H, W, Ci, Co);
   const CUtensorMap *mx, *my;
-  cudaError_t e = cached_tile_map(cache, x, N, H, W, Ci, p.G, &mx);
-  if (e == cudaSuccess) e = cached_tile_map(cache, dy, N, H, W, Co, p.G, &my);
+  cudaError_t e = cached_tile_map(cache, x, N, H, W, Ci, p.G, &mx, p.kcx);
+  if (e == cudaSuccess) e = cached_tile_map(cache, dy, N, H, W, Co, p.G, &my, p.kcy);
   if (e == cudaSuccess) e = halo::set_smem_attrs();
   if (e != cudaSuccess) return e;
   const int ctas = halo::wgrad_ctas(p);
-  halo::wgrad_halo_kernel<<<ctas, halo::kFwdThreads, halo::wgrad_smem_bytes(p), st>>>(*mx, *my, p, scratch, err_dev);
+  halo::wgrad_halo_kernel<<<dim3(ctas, halo::wgrad_pairs(p)), halo::kFwdThreads, halo::wgrad_smem_bytes(p), st>>>(*mx, *my, p, scratch, err_dev);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t n = (size_t)Co * 9 * Ci;

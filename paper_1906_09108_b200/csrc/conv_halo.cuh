@@ -373,15 +373,17 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 // N = Co would.
 struct WgradParams {
   int W, H, N, Wp, Hp;
-  int Ci, Co;                 // channels of x (16/32/64) and of dy (16/32/64)
+  int Ci, Co;                 // channels of x and of dy
+  int kcx, kcy;               // channel chunk of the x and of the dy tile (16/32/64): a CTA computes the block
+  int nyb;                    //   dW[co chunk b][.][.][ci chunk a], blockIdx.y = a * nyb + b
   int G, tiles;               // images per tile, ceil(N / G)
   int ksteps;                 // 16-pixel reduction steps per tile
   uint32_t pitch_x, pitch_y;
   uint32_t x_tx_bytes, y_tx_bytes;
   uint32_t x_bytes, y_bytes;  // shared memory reserved per stage for the two tiles (multiples of 1024)
   int stages;
-  int sgroups;                // M-block groups: 1, or 2 when Ci = 64 (128 rows hold only two taps)
-  int taps_per_group;         // min(3, 128 / Ci)
+  int sgroups;                // M-block groups: 1, or 2 when kcx = 64 (128 rows hold only two taps)
+  int taps_per_group;         // min(3, 128 / kcx)
   uint32_t tmem_cols;
 };
 
@@ -420,7 +422,8 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int ncols = 3 * p.Co;                                 // N of the instruction
+  const int ncols = 3 * p.kcy;                                // N of the instruction
+  const int chunk_a = blockIdx.y / p.nyb, chunk_b = blockIdx.y - chunk_a * p.nyb;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -431,8 +434,8 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) break;
         uint8_t* xs = smem + (size_t)s * stage_bytes;
         mbar_expect_tx(&full[s], p.x_tx_bytes + p.y_tx_bytes);
-        tma_load_4d(xs, &map_x, &full[s], 0, -1, -1, tile * p.G);
-        tma_load_4d(xs + p.x_bytes, &map_y, &full[s], 0, 0, -2, tile * p.G);
+        tma_load_4d(xs, &map_x, &full[s], chunk_a * p.kcx, -1, -1, tile * p.G);
+        tma_load_4d(xs + p.x_bytes, &map_y, &full[s], chunk_b * p.kcy, 0, -2, tile * p.G);
       }
     }
   } else if (warp < kFirstEpiWarp) {
@@ -475,7 +478,7 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     if (mbar_wait(done, 0, abort_flag)) {
       tc_fence_after();
       const int row = lane_grp * 32 + lane;
-      const int sblk = row / p.Ci, ci = row - sblk * p.Ci;
+      const int sblk = row / p.kcx, ci = chunk_a * p.kcx + (row - sblk * p.kcx);
       float* dst = partial + (size_t)blockIdx.x * ((size_t)p.Co * 9 * p.Ci);
       const int nchunks = ncols >> 4;
       const size_t co_stride = (size_t)9 * p.Ci;
@@ -494,7 +497,7 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(u[e]));
         }
         if (!valid) continue;
-        const int b = c0 / p.Co, r = 2 - b, co0 = c0 - b * p.Co;        // Co is a multiple of 16: a chunk stays in one block
+        const int b = c0 / p.kcy, r = 2 - b, co0 = chunk_b * p.kcy + (c0 - b * p.kcy);   // kcy is a multiple of 16: a chunk stays in one block
         float* d0 = dst + (size_t)co0 * co_stride + (size_t)(r * 3 + sx) * p.Ci + ci;
 #pragma unroll
         for (int e = 0; e < 16; ++e) d0[(size_t)e * co_stride] = __uint_as_float(v[e]);
@@ -594,10 +597,16 @@ inline bool fwd_supported(int N, int H, int W, int Ck, int Cn) {
   return p.stages >= 1 && fwd_smem_bytes(p) <= kSmemBudget + 4096 && p.tile_tx_bytes < (1u << 20);
 }
 
+// Channel chunk of a tile: the whole pixel when it is one swizzle span, else 64- or 32-channel slices.
+inline int wgrad_chunk(int C) { return chan_ok(C) ? C : (C % 64 == 0 ? 64 : (C % 32 == 0 ? 32 : 0)); }
+
 inline WgradParams wgrad_params(int N, int H, int W, int Ci, int Co) {
   WgradParams p{};
   p.W = W; p.H = H; p.N = N; p.Wp = W + 2; p.Hp = H + 2; p.Ci = Ci; p.Co = Co;
-  p.pitch_x = (uint32_t)Ci * 2; p.pitch_y = (uint32_t)Co * 2;
+  p.kcx = wgrad_chunk(Ci); p.kcy = wgrad_chunk(Co);
+  if (p.kcx == 0 || p.kcy == 0) { p.stages = 0; return p; }
+  p.nyb = Co / p.kcy;
+  p.pitch_x = (uint32_t)p.kcx * 2; p.pitch_y = (uint32_t)p.kcy * 2;
   const int img_rows = p.Hp * p.Wp;
   // images per tile: what two pipeline stages of both tiles fit in shared memory
   const int max_rows = (int)(96 * 1024 / (p.pitch_x + p.pitch_y));
@@ -606,7 +615,7 @@ inline WgradParams wgrad_params(int N, int H, int W, int Ci, int Co) {
   p.tiles = (N + p.G - 1) / p.G;
   const int Q = p.G * img_rows;
   p.ksteps = (Q + 15) / 16;
-  const int blocks = kTileM / Ci;
+  const int blocks = kTileM / p.kcx;
   p.taps_per_group = blocks < 3 ? blocks : 3;
   p.sgroups = (3 + p.taps_per_group - 1) / p.taps_per_group;
   p.x_tx_bytes = (uint32_t)Q * p.pitch_x; p.y_tx_bytes = (uint32_t)Q * p.pitch_y;
@@ -615,15 +624,22 @@ inline WgradParams wgrad_params(int N, int H, int W, int Ci, int Co) {
   const size_t stage = (size_t)p.x_bytes + p.y_bytes;
   int stages = (int)((kSmemBudget - 2048) / stage);
   p.stages = stages > 2 ? 2 : stages;
-  uint32_t need = (uint32_t)(2 * 3 * Co), cols = 32;            // two accumulators: two tap groups, or two copies of one
+  uint32_t need = (uint32_t)(2 * 3 * p.kcy), cols = 32;         // two accumulators: two tap groups, or two copies of one
   while (cols < need) cols <<= 1;
   p.tmem_cols = cols;
   return p;
 }
+inline int wgrad_pairs(const WgradParams& p) { return (p.Ci / p.kcx) * (p.Co / p.kcy); }
 
 // Pixel split: few enough CTAs that their partial sums (Co*9*Ci floats each) stay small next to
 // the operands, enough of them to spread the reduction over the SMs.
 inline int wgrad_ctas(const WgradParams& p) {
+  const int pairs = wgrad_pairs(p);
+  if (pairs > 1) {                                              // chunked (wide) layers: about 1.5 CTAs per SM in all
+    int want = (222 + pairs / 2) / pairs;
+    if (want < 1) want = 1;
+    return p.tiles < want ? p.tiles : want;
+  }
   const size_t wsize = (size_t)p.Co * 9 * p.Ci;
   int want = (int)((size_t)p.N * p.H * p.W * (p.Ci + p.Co) * 2 / (wsize * 2));     // partial bytes <= ~ 2 x operand bytes
   if (want > 128) want = 128;
@@ -634,10 +650,11 @@ inline size_t wgrad_smem_bytes(const WgradParams& p) {
   return (size_t)p.stages * ((size_t)p.x_bytes + p.y_bytes) + (size_t)(2 * p.stages + 1) * 8 + 16 + 1024;
 }
 inline bool wgrad_supported(int N, int H, int W, int Ci, int Co) {
-  if (!chan_ok(Ci) || !chan_ok(Co)) return false;
+  if (wgrad_chunk(Ci) == 0 || wgrad_chunk(Co) == 0) return false;
   if (W + 2 > 256 || H + 2 > 256 || N < 1) return false;
   WgradParams p = wgrad_params(N, H, W, Ci, Co);
-  return p.stages >= 1 && p.x_tx_bytes < (1u << 19) && p.y_tx_bytes < (1u << 19) && p.tmem_cols <= 512;
+  return p.stages >= 1 && p.x_tx_bytes < (1u << 19) && p.y_tx_bytes < (1u << 19) && p.tmem_cols <= 512 &&
+         wgrad_pairs(p) <= 65535;
 }
 // fp32 elements of scratch the weight gradient needs for its per-CTA partial sums.
 inline size_t wgrad_scratch_elems(int N, int H, int W, int Ci, int Co) {
@@ -646,15 +663,16 @@ inline size_t wgrad_scratch_elems(int N, int H, int W, int Ci, int Co) {
 }
 
 // Halo-tile tensor map of a bf16 NHWC tensor: box = G whole images with border.
-inline cudaError_t make_tile_map(const void* act, int N, int H, int W, int C, int G, CUtensorMap* map) {
+inline cudaError_t make_tile_map(const void* act, int N, int H, int W, int C, int G, CUtensorMap* map, int boxC = 0) {
+  if (boxC == 0) boxC = C;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
   cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
   cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-  cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)(W + 2), (cuuint32_t)(H + 2), (cuuint32_t)G};
+  cuuint32_t box[4] = {(cuuint32_t)boxC, (cuuint32_t)(W + 2), (cuuint32_t)(H + 2), (cuuint32_t)G};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   if (enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(act), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(C * 2), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(boxC * 2), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
   return cudaSuccess;
