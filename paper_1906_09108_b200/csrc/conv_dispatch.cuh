@@ -36,13 +36,14 @@ inline bool tc_eligible(const ConvGeom& g) {
 // counts (forward: Ci/Co; data gradient: Co/Ci with the flipped weight copy).
 inline cudaError_t run_conv_tc(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ck, int Cn,
                                const bf16_t* act, const bf16_t* wgt, bf16_t* out, const bf16_t* res,
-                               const bf16_t* res_mask, int* err_dev) {
+                               const bf16_t* res_mask, int* err_dev, int sub = 1) {
   if (cache->sm_count == 0) {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&cache->sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
   tc::ConvTcParams p = tc::conv_tc_params(N, H, W, Ck, Cn);
+  p.sub = sub;
   TensorMapCache::Key ka, kb;
   std::memset(&ka, 0, sizeof(ka)); std::memset(&kb, 0, sizeof(kb));
   ka.ptr = act; ka.d[0] = 1; ka.d[1] = N; ka.d[2] = H; ka.d[3] = W; ka.d[4] = Ck; ka.d[5] = p.kc;
@@ -86,6 +87,9 @@ inline bool halo_s2_shape(const ConvGeom& g) {
 }
 inline bool halo_s2_fprop_eligible(const ConvGeom& g) { return halo_s2_shape(g) && halo::fwd_supported(g.N, g.H, g.W, g.Ci, g.Co); }
 inline bool halo_s2_dgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && halo::fwd_supported(g.N, g.H, g.W, g.Co, g.Ci); }
+// the same for layers too wide for the halo kernel: the per-tap kernel at full resolution
+inline bool tc_s2_fprop_eligible(const ConvGeom& g) { return halo_s2_shape(g) && tc::conv_tc_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+inline bool tc_s2_dgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && tc::conv_tc_supported(g.N, g.H, g.W, g.Co, g.Ci); }
 inline bool halo_s2_wgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && halo::wgrad_supported(g.N, g.H, g.W, g.Ci, g.Co); }
 
 inline cudaError_t cached_tile_map(TensorMapCache* cache, const void* act, int N, int H, int W, int C, int G,
@@ -165,7 +169,9 @@ inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N,
 
 
 // Does the data gradient of this convolution read the flipped/transposed weight copy?
-inline bool dgrad_uses_flipped(const ConvGeom& g) { return halo_dgrad_eligible(g) || halo_s2_dgrad_eligible(g) || tc_eligible(g); }
+inline bool dgrad_uses_flipped(const ConvGeom& g) {
+  return halo_dgrad_eligible(g) || halo_s2_dgrad_eligible(g) || tc_eligible(g) || tc_s2_dgrad_eligible(g);
+}
 
 // fp32 scratch elements a weight-gradient call may need (bf16 storage: whichever kernel is chosen).
 inline size_t conv_wgrad_scratch_elems(bool bf16_storage, const ConvGeom& g) {

@@ -43,6 +43,7 @@ struct ConvTcParams {
   uint32_t a_bytes, b_bytes, stage_bytes;   // b_bytes is padded to 1 KiB; b_tx_bytes is what TMA moves
   uint32_t b_tx_bytes;
   uint32_t tmem_cols;       // allocated columns (power of two >= 2*n_tile)
+  int sub;                  // 1, or 2: store only the pixels with even h and w, as an [N][H/2][W/2][Co] tensor
 };
 
 // ---------------------------------------------------------------- PTX wrappers --
@@ -231,12 +232,20 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) break;
       tc_fence_after();
       const size_t row = (size_t)mt * kTileM + lane_grp * 32 + lane;
-      const size_t base = row * p.Co + (size_t)nt * p.n_tile;
+      size_t base = row * p.Co + (size_t)nt * p.n_tile;
+      bool keep = true;
+      if (p.sub == 2) {
+        const size_t hw = (size_t)p.H * p.W, n = row / hw, rem = row - n * hw;
+        const int h = (int)(rem / p.W), w = (int)(rem - (size_t)h * p.W);
+        keep = ((h | w) & 1) == 0;
+        base = (((n * (p.H >> 1) + (h >> 1)) * (p.W >> 1)) + (w >> 1)) * p.Co + (size_t)nt * p.n_tile;
+      }
       const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)acc * p.n_tile;
       for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
         uint32_t v[16];
         tmem_ld16(taddr + c0, v);
         tmem_ld_wait();
+        if (!keep) continue;
         float f[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) f[i] = __uint_as_float(v[i]);
@@ -335,7 +344,7 @@ inline bool conv_tc_supported(int N, int H, int W, int Ci, int Co) {
 
 inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co) {
   ConvTcParams p{};
-  p.W = W; p.H = H; p.N = N; p.Ci = Ci; p.Co = Co;
+  p.W = W; p.H = H; p.N = N; p.Ci = Ci; p.Co = Co; p.sub = 1;
   const int rows = kTileM / W;
   if (rows <= H) { p.rows_per_tile = rows; p.imgs_per_tile = 1; }
   else { p.rows_per_tile = H; p.imgs_per_tile = rows / H; }

@@ -343,7 +343,8 @@ static void plan_modules(fdg_ctx* c) {
       for (const Unit& u : m.units) {
         if ((u.type != U_BASIC && u.type != U_PREACT) || u.stride != 2) continue;
         ConvGeom g1{a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 3, u.stride, 1};
-        if (halo_s2_dgrad_eligible(g1) || halo_s2_wgrad_eligible(g1)) m.up_elems = std::max(m.up_elems, B * u.H * u.W * u.co);
+        if (halo_s2_dgrad_eligible(g1) || halo_s2_wgrad_eligible(g1) || tc_s2_dgrad_eligible(g1))
+          m.up_elems = std::max(m.up_elems, B * u.H * u.W * u.co);
       }
     if (c->bf16_mode) {
       size_t fe = 0;
@@ -583,9 +584,9 @@ static int conv_fprop(Launch& L, Module& m, const ConvGeom& g, const T* x, const
       L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, fuse ? &r : nullptr, &ctas, 2));
       return fuse ? ctas : 0;
     }
-    if (tc_eligible(g)) {
+    if (tc_eligible(g) || tc_s2_fprop_eligible(g)) {
       ++L.c->launches;
-      L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error));
+      L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, g.stride));
       return 0;
     }
   }
@@ -626,6 +627,11 @@ static int conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, cons
       L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error));
       return 0;
     }
+    if (wflip && dy_up && tc_s2_dgrad_eligible(g)) {
+      ++L.c->launches;
+      L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy_up, wflip, dx, res, mask, L.c->tc_error));
+      return 0;
+    }
   }
   L.note(launch_conv_simt<T, CONV_DGRAD>(L.st, g, dy, w, dx, nullptr, nullptr, res, mask, &L.c->launches));
   return 0;
@@ -659,7 +665,7 @@ template <> const bf16* flipped_of<bf16>(const Module& m, int vslot, long long o
 template <typename T>
 static const T* upsample_dy(Launch& L, Module& m, const ConvGeom& g, const T* dy) {
   if constexpr (std::is_same<T, bf16>::value) {
-    if (!m.up || !(halo_s2_dgrad_eligible(g) || halo_s2_wgrad_eligible(g)) || g.Co % 8) return nullptr;
+    if (!m.up || !(halo_s2_dgrad_eligible(g) || halo_s2_wgrad_eligible(g) || tc_s2_dgrad_eligible(g)) || g.Co % 8) return nullptr;
     T* up = reinterpret_cast<T*>(m.up);
     const size_t nvec = (size_t)g.N * g.H * g.W * g.Co / 8;
     L.begin(KC_CONV_DGRAD, (double)nvec * 16 * 1.25, 0.0);
@@ -894,12 +900,13 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
         conv_dgrad<T>(L, m, g2, dy, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T1, nullptr, nullptr);   // da2
         bn_backward<T>(L, m, T1, S + u.t_c, S + u.t_b, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
                        nullptr, nullptr, nullptr, nullptr, nullptr, T2, nullptr, rows_out, u.co);      // dc1
-        conv_wgrad<T>(L, m, g1, S + u.t_a, T2, m.grad + u.w1);
+        const T* up = u.stride == 2 ? upsample_dy<T>(L, m, g1, T2) : nullptr;
+        conv_wgrad<T>(L, m, g1, S + u.t_a, T2, m.grad + u.w1, up);
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_wgrad<T>(L, m, gs, S + u.t_a, dy, m.grad + u.ws);
           conv_dgrad<T>(L, m, gs, dy, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
-          conv_dgrad<T>(L, m, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, T3, nullptr);      // do
+          conv_dgrad<T>(L, m, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, T3, nullptr, nullptr, up);   // do
         } else {
           conv_dgrad<T>(L, m, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, nullptr, nullptr);
         }

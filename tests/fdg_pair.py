@@ -44,6 +44,9 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
         g.set_params(k, p)
     a = arch_o
     res = dict(out=0.0, gin=0.0, loss=0.0, grads=0.0, steps=steps)
+    res["grads_by_step"] = []          # (t, k, error): where a failure started, for the assertion message
+    res["worst_tensors"] = []          # the three worst parameter tensors at the worst (t, k)
+    layouts = {k: g.param_layout(k) for k in range(1, K + 1)}
     loss_dev = torch.zeros(1, dtype=torch.float32, device="cuda")
     for t in range(1, steps + 1):
         x = S.images(seed, t, a.batch, a.in_h, a.in_w, a.in_c)
@@ -68,7 +71,16 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
                 res["gin"] = max(res["gin"], relmax(gi, go.reshape(-1)))
             go = orc.get_grads(k)
             if go is not None:
-                res["grads"] = max(res["grads"], relfro(g.get_grads(k), go))
+                gg = g.get_grads(k)
+                err = relfro(gg, go)
+                res["grads_by_step"].append((t, k, round(err, 4)))
+                if err > res["grads"]:
+                    res["grads"] = err
+                    per = []
+                    for name, _, shape in layouts[k]:
+                        off, n = int(name.split("@")[1]), int(np.prod(shape))
+                        per.append((round(relfro(gg[off:off + n], go[off:off + n]), 4), t, k, name, tuple(shape)))
+                    res["worst_tensors"] = sorted(per, reverse=True)[:3]
     g.sync()
     res["params"] = max(relfro(g.get_params(k), orc.get_params(k)) for k in range(1, K + 1))
     res["momentum"] = max(relfro(g.get_momentum(k), orc.get_momentum(k)) for k in range(1, K + 1))
