@@ -140,7 +140,9 @@ inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, 
   if (e == cudaSuccess) e = cached_weight_map(cache, wgt, Ck, Cn, &mw);
   if (e == cudaSuccess) e = halo::set_smem_attrs();
   if (e != cudaSuccess) return e;
-  const int grid = p.tiles < sms ? p.tiles : sms;
+  // the fewest CTAs that keep the number of tiles of the busiest one at ceil(tiles / sms)
+  const int per_cta = (p.tiles + sms - 1) / sms;
+  const int grid = (p.tiles + per_cta - 1) / per_cta;
   halo::EpiReduce r{};
   if (red) { if (!halo_reduce_ok(Cn)) return cudaErrorInvalidValue; r = *red; }
   if (ctas_out) *ctas_out = grid;

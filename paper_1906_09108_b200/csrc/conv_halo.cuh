@@ -86,10 +86,12 @@ struct EpiReduce {
   const float* pstats;        // mode 2: mean[Cn], invstd[Cn] of xprev's batch norm
   float* partial;             // [gridDim.x][2*Cn]
 };
-// Threads of conv_halo_kernel: TMA warp, MMA warp, kEpiGroups groups of four epilogue warps.  A
-// group takes every kEpiGroups-th 128-row tile: one tile's epilogue is a chain of dependent
-// steps (wait, tensor-memory load, global loads, shuffles), so several must be in flight.
-constexpr int kEpiGroups = 4;
+// Threads of conv_halo_kernel: TMA warp, two MMA warps, kEpiGroups groups of four epilogue warps.
+// The groups take the (128-row tile, 16-column chunk) items in turn: an item's epilogue is a chain
+// of dependent steps (wait, tensor-memory load, shuffles), so several must be in flight.  Three
+// groups divide the 9 tiles of a 32x32 image evenly and leave each thread the registers to hold
+// the next item's global operands while it works on the current one.
+constexpr int kEpiGroups = 3;
 constexpr int kEpiWarps = 4 * kEpiGroups;
 // One thread can issue a tcgen05.mma every ~75 cycles, the tensor pipe takes one of these small
 // instructions every ~40: two issuing warps (alternate 128-row tiles) keep it busier (measured).
@@ -225,109 +227,166 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       }
     }
   } else {
+    // Work item = (128-row tile, 16-column chunk), dealt to the groups in turn; the number of slots is
+    // chosen (fwd_params) so that the same groups meet a slot every time and see all its phases.  The
+    // global operands of an item (residual, its gate, the two tensors of a fused batch-norm-backward
+    // sum) do not depend on the accumulator: they are requested one item ahead into the other of two
+    // register sets, so that their latency runs beside the previous item's work.  Everything an item
+    // needs (slot, phase, the pixel of this thread's row) is carried from item to item by additions:
+    // a division per item costs more here than the item's arithmetic.
     const int lane_grp = warp & 3;                 // tensor-memory lanes 32*(warp % 4) .. +31
     const int group = (warp - kFirstEpiWarp) >> 2;
-    uint32_t acount = 0;
-    for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x) {
-      const int n0 = tile * p.G;
-      bool ok = true;
-      for (int i = 0; i < p.m_tiles; ++i, ++acount) {
-        // Work item = (tile, 16-column chunk), dealt to the groups in turn.  nacc is a multiple of
-        // kEpiGroups, so the same groups meet a slot every time and see all its phases.
-        const int nch = p.Cn >> 4;
-        const int first = (int)((acount * (uint32_t)nch) % kEpiGroups);
-        int my_first = group - first; if (my_first < 0) my_first += kEpiGroups;      // first chunk of this tile dealt to this group
-        if (my_first >= nch) continue;
-        const int slot = acount % p.nacc;
-        const uint32_t aph = (acount / p.nacc) & 1;
-        if (!mbar_wait(&acc_full[slot], aph, abort_flag)) { ok = false; break; }
+    const int nch = p.Cn >> 4;
+    // Items are numbered J = (128-row tiles so far) * nch + chunk over the whole CTA; group g takes
+    // J = g, g + kEpiGroups, ...  One step of J is `step_a` 128-row tiles and `step_c` chunks.
+    const int step_a = kEpiGroups / nch, step_c = kEpiGroups - step_a * nch;
+    struct Cursor {
+      int tile, i;              // image tile, 128-row tile inside it
+      int slot; uint32_t aph;   // accumulator slot of (tile, i) and the phase of its barriers
+      int g, h, w;              // this thread's row of (tile, i) as (image in tile, padded row, padded column)
+      int chunk; bool first_chunk;
+    };
+    struct Operands { bool valid; size_t base; uint4 r0, r1, g0, g1, k0, k1, x0, x1; };
+    const int row0 = lane_grp * 32 + lane;
+    const int g_first = row0 / p.img_rows, h_first = (row0 - g_first * p.img_rows) / p.Wp;
+    const int w_first = row0 - g_first * p.img_rows - h_first * p.Wp;
+    const int dh = kTileM / p.Wp, dw = kTileM - dh * p.Wp;            // 128 rows further on
+    auto move_rows = [&](Cursor& c, int mtiles) {                     // this thread's row, `mtiles` 128-row tiles further on
+      c.w += mtiles * dw; c.h += mtiles * dh;
+      while (c.w >= p.Wp) { c.w -= p.Wp; ++c.h; }
+      while (c.h >= p.Hp && c.g < p.G) { c.h -= p.Hp; ++c.g; }
+    };
+    auto move_mtiles = [&](Cursor& c, int da) {                       // da <= kEpiGroups <= nacc
+      c.slot += da;
+      if (c.slot >= p.nacc) { c.slot -= p.nacc; c.aph ^= 1; }
+      c.i += da;
+      if (c.i < p.m_tiles) { move_rows(c, da); return; }
+      while (c.i >= p.m_tiles) { c.i -= p.m_tiles; c.tile += gridDim.x; }
+      c.g = g_first; c.h = h_first; c.w = w_first;
+      move_rows(c, c.i);
+    };
+    auto advance = [&](Cursor& c) -> bool {
+      c.chunk += step_c;
+      int da = step_a;
+      if (c.chunk >= nch) { c.chunk -= nch; ++da; }
+      c.first_chunk = da != 0;
+      if (da) move_mtiles(c, da);
+      return c.tile < p.tiles;
+    };
+    auto fetch = [&](const Cursor& c, Operands& o) {
+      const int n = c.tile * p.G + c.g;
+      o.valid = c.h < p.H && c.w < p.W && c.g < p.G && n < p.N && (p.sub == 1 || ((c.h | c.w) & 1) == 0);
+      const int pix = p.sub == 1 ? (n * p.H + c.h) * p.W + c.w : (n * (p.H >> 1) + (c.h >> 1)) * (p.W >> 1) + (c.w >> 1);
+      o.base = (size_t)pix * p.Cn + c.chunk * 16;
+      if (red.mode == 2) o.k0 = o.k1 = o.x0 = o.x1 = make_uint4(0, 0, 0, 0);   // read below whether or not the row is valid
+      if (!o.valid) return;
+      if (res) {
+        o.r0 = *reinterpret_cast<const uint4*>(res + o.base);
+        o.r1 = *reinterpret_cast<const uint4*>(res + o.base + 8);
+        if (res_mask) {
+          o.g0 = *reinterpret_cast<const uint4*>(res_mask + o.base);
+          o.g1 = *reinterpret_cast<const uint4*>(res_mask + o.base + 8);
+        }
+      }
+      if (red.mode == 2) {
+        o.k0 = *reinterpret_cast<const uint4*>(red.mask + o.base);
+        o.k1 = *reinterpret_cast<const uint4*>(red.mask + o.base + 8);
+        o.x0 = *reinterpret_cast<const uint4*>(red.xprev + o.base);
+        o.x1 = *reinterpret_cast<const uint4*>(red.xprev + o.base + 8);
+      }
+    };
+    // the group's first item: J = group
+    Cursor cur{(int)blockIdx.x, 0, 0, 0u, g_first, h_first, w_first, 0, true};
+    {
+      const int a0 = group / nch;
+      cur.chunk = group - a0 * nch;
+      if (a0) move_mtiles(cur, a0);
+    }
+    // One item: request the next item's operands into `fill`, then finish the current one with `use`.
+    // Returns false when there is no next item (or a wait gave up).
+    auto item = [&](Operands& use, Operands& fill) -> bool {
+      Cursor nxt = cur;
+      const bool have_next = advance(nxt);
+      if (have_next) fetch(nxt, fill);
+      const int slot = cur.slot;
+      if (cur.first_chunk) {
+        if (!mbar_wait(&acc_full[slot], cur.aph, abort_flag)) return false;
         tc_fence_after();
-        const int m = kTileM * i + lane_grp * 32 + lane;
-        const int g = m / p.img_rows, rem = m - g * p.img_rows;
-        const int h = rem / p.Wp, w = rem - h * p.Wp;
-        const bool valid = h < p.H && w < p.W && g < p.G && n0 + g < p.N && (p.sub == 1 || ((h | w) & 1) == 0);
-        const size_t base = p.sub == 1 ? ((((size_t)(n0 + g) * p.H + h) * p.W) + w) * p.Cn
-                                       : ((((size_t)(n0 + g) * (p.H >> 1) + (h >> 1)) * (p.W >> 1)) + (w >> 1)) * p.Cn;
-        const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)slot * p.Cn;
-        for (int c0 = my_first * 16; c0 < p.Cn; c0 += 16 * kEpiGroups) {
-          uint32_t v[16];
-          tmem_ld16(taddr + c0, v);
-          tmem_ld_wait();
-          float f[16];
+      }
+      const int c0 = cur.chunk * 16;
+      uint32_t v[16];
+      tmem_ld16(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)slot * p.Cn + c0, v);
+      tmem_ld_wait();
+      float f[16];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]);
-          if (valid) {
-            if (res) {
-              uint4 r0 = *reinterpret_cast<const uint4*>(res + base + c0);
-              uint4 r1 = *reinterpret_cast<const uint4*>(res + base + c0 + 8);
-              const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
-              const __nv_bfloat16* rb1 = reinterpret_cast<const __nv_bfloat16*>(&r1);
-              float gq[16];
+      for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]);
+      if (use.valid) {
+        if (res) {
+          const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&use.r0);
+          const __nv_bfloat16* rb1 = reinterpret_cast<const __nv_bfloat16*>(&use.r1);
+          float gq[16];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) { gq[e] = __bfloat162float(rb0[e]); gq[8 + e] = __bfloat162float(rb1[e]); }
-              if (res_mask) {
-                uint4 m0 = *reinterpret_cast<const uint4*>(res_mask + base + c0);
-                uint4 m1 = *reinterpret_cast<const uint4*>(res_mask + base + c0 + 8);
-                const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&m0);
-                const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&m1);
+          for (int e = 0; e < 8; ++e) { gq[e] = __bfloat162float(rb0[e]); gq[8 + e] = __bfloat162float(rb1[e]); }
+          if (res_mask) {
+            const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&use.g0);
+            const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&use.g1);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  if (!(__bfloat162float(mb0[e]) > 0.f)) gq[e] = 0.f;
-                  if (!(__bfloat162float(mb1[e]) > 0.f)) gq[8 + e] = 0.f;
-                }
-              }
-#pragma unroll
-              for (int e = 0; e < 16; ++e) f[e] += gq[e];
+            for (int e = 0; e < 8; ++e) {
+              if (!(__bfloat162float(mb0[e]) > 0.f)) gq[e] = 0.f;
+              if (!(__bfloat162float(mb1[e]) > 0.f)) gq[8 + e] = 0.f;
             }
-            uint4 o0, o1;
-            __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
-            __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              ob0[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
-              ob1[e] = __floats2bfloat162_rn(f[8 + 2 * e], f[8 + 2 * e + 1]);
-            }
-            *reinterpret_cast<uint4*>(out + base + c0) = o0;
-            *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
           }
-          if (red.mode) {
-            float q[32];
-            if (red.mode == 1) {
 #pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                const float sv = valid ? __bfloat162float(__float2bfloat16_rn(f[e])) : 0.f;
-                q[e] = sv; q[16 + e] = sv * sv;
-              }
-            } else {
-              uint4 m0 = make_uint4(0, 0, 0, 0), m1 = m0, x0 = m0, x1 = m0;
-              if (valid) {
-                m0 = *reinterpret_cast<const uint4*>(red.mask + base + c0);
-                m1 = *reinterpret_cast<const uint4*>(red.mask + base + c0 + 8);
-                x0 = *reinterpret_cast<const uint4*>(red.xprev + base + c0);
-                x1 = *reinterpret_cast<const uint4*>(red.xprev + base + c0 + 8);
-              }
-              const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&m0);
-              const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&m1);
-              const __nv_bfloat16* xb0 = reinterpret_cast<const __nv_bfloat16*>(&x0);
-              const __nv_bfloat16* xb1 = reinterpret_cast<const __nv_bfloat16*>(&x1);
+          for (int e = 0; e < 16; ++e) f[e] += gq[e];
+        }
+        uint4 o0, o1;
+        __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
+        __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
 #pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                const float mk = __bfloat162float(e < 8 ? mb0[e] : mb1[e - 8]);
-                const float xp = __bfloat162float(e < 8 ? xb0[e] : xb1[e - 8]);
-                const float dz = (valid && mk > 0.f) ? __bfloat162float(__float2bfloat16_rn(f[e])) : 0.f;
-                q[e] = dz;
-                q[16 + e] = dz * ((xp - red_stat[c0 + e]) * red_stat[p.Cn + c0 + e]);
-              }
-            }
-            transpose_reduce32(q, lane);
-            red_run[((warp - kFirstEpiWarp) * 8 + (c0 >> 4)) * 32 + lane] += q[0];
+        for (int e = 0; e < 4; ++e) {
+          ob0[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+          ob1[e] = __floats2bfloat162_rn(f[8 + 2 * e], f[8 + 2 * e + 1]);
+        }
+        *reinterpret_cast<uint4*>(out + use.base) = o0;
+        *reinterpret_cast<uint4*>(out + use.base + 8) = o1;
+      }
+      if (red.mode) {
+        float q[32];
+        if (red.mode == 1) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float sv = use.valid ? __bfloat162float(__float2bfloat16_rn(f[e])) : 0.f;
+            q[e] = sv; q[16 + e] = sv * sv;
+          }
+        } else {
+          const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&use.k0);
+          const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&use.k1);
+          const __nv_bfloat16* xb0 = reinterpret_cast<const __nv_bfloat16*>(&use.x0);
+          const __nv_bfloat16* xb1 = reinterpret_cast<const __nv_bfloat16*>(&use.x1);
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float mk = __bfloat162float(e < 8 ? mb0[e] : mb1[e - 8]);
+            const float xp = __bfloat162float(e < 8 ? xb0[e] : xb1[e - 8]);
+            const float dz = (use.valid && mk > 0.f) ? __bfloat162float(__float2bfloat16_rn(f[e])) : 0.f;
+            q[e] = dz;
+            q[16 + e] = dz * ((xp - red_stat[c0 + e]) * red_stat[p.Cn + c0 + e]);
           }
         }
+        transpose_reduce32(q, lane);
+        red_run[((warp - kFirstEpiWarp) * 8 + (c0 >> 4)) * 32 + lane] += q[0];
+      }
+      if (!have_next || nxt.first_chunk) {           // this group's last chunk of the 128-row tile: hand the slot back
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[slot]);
       }
-      if (!ok) break;
+      cur = nxt;
+      return have_next;
+    };
+    Operands op_a, op_b;
+    if (!*abort_flag && cur.tile < p.tiles) {
+      fetch(cur, op_a);
+      while (item(op_a, op_b) && item(op_b, op_a)) {}
     }
   }
 
@@ -575,10 +634,23 @@ inline FwdParams fwd_params(int N, int H, int W, int Ck, int Cn, int sm_count) {
   if (stages > 3) stages = 3;
   if (stages > per_cta) stages = per_cta;                     // shared memory left free lets other kernels' CTAs co-reside
   p.stages = stages;
-  // accumulator slots: a multiple of the epilogue groups (a slot then always belongs to one group); a slot
-  // per 128-row tile where 256 columns allow it, so that the issuer seldom waits for the epilogue
-  p.nacc = (p.m_tiles + kEpiGroups - 1) / kEpiGroups * kEpiGroups;
-  while (p.nacc > kEpiGroups && p.nacc * Cn > 256) p.nacc -= kEpiGroups;
+  // Accumulator slots.  Two conditions keep every waiter in step with the phases of a slot's barriers:
+  // an even count, so that a slot always belongs to the same issuing warp (the warps take alternate
+  // 128-row tiles); and, where a tile has fewer chunks than there are epilogue groups, a count whose
+  // chunk total is a multiple of the groups, so that the same groups meet a slot every time.  Within
+  // that, a slot per 128-row tile where 256 columns allow it, so the issuers seldom wait for the epilogue.
+  {
+    const int nch = Cn / 16;
+    int step = kMmaWarps;
+    if (nch < kEpiGroups) {
+      int g = kEpiGroups, a = nch;                           // kEpiGroups / gcd(kEpiGroups, nch)
+      while (a) { const int t = g % a; g = a; a = t; }
+      const int need = kEpiGroups / g;
+      step = need % kMmaWarps == 0 ? need : need * kMmaWarps;
+    }
+    p.nacc = (p.m_tiles + step - 1) / step * step;
+    while (p.nacc > step && p.nacc * Cn > 256) p.nacc -= step;
+  }
   uint32_t cols = 32;
   while (cols < (uint32_t)(p.nacc * Cn)) cols <<= 1;
   p.tmem_cols = cols;
@@ -594,7 +666,7 @@ inline bool fwd_supported(int N, int H, int W, int Ck, int Cn) {
   if (!chan_ok(Ck) || Cn % 16 || Cn < 16 || Cn > 128) return false;
   if (W + 2 > 256 || H + 2 > 256 || N < 1) return false;
   FwdParams p = fwd_params(N, H, W, Ck, Cn, 148);
-  return p.stages >= 1 && fwd_smem_bytes(p) <= kSmemBudget + 4096 && p.tile_tx_bytes < (1u << 20);
+  return p.stages >= 1 && fwd_smem_bytes(p) <= kSmemBudget + 4096 && p.tile_tx_bytes < (1u << 20) && p.tmem_cols <= 512;
 }
 
 // Channel chunk of a tile: the whole pixel when it is one swizzle span, else 64- or 32-channel slices.

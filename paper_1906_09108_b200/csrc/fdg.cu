@@ -1153,7 +1153,10 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   if (e == cudaSuccess && c->use_graphs) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
   c->ev_cjoin.assign(c->K, nullptr);
   for (int k = 0; k < c->K && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&c->ev_cjoin[k], cudaEventDisableTiming);
-  c->tmaps.share = c->cfg.serial ? 1 : c->K;
+  // Convolution launches are sized for the module streams running side by side.  With 128 image tiles
+  // per layer, 148 / K SMs each gives 2 tiles per CTA at K = 2 and 4 at K = 4; three per CTA (43 CTAs)
+  // measured faster at K = 4 than both two and four, so one stream's share is left unclaimed there.
+  c->tmaps.share = c->cfg.serial ? 1 : (c->K > 2 ? c->K - 1 : c->K);
   c->graph_exec.assign(c->period, nullptr);
   c->graph_sig.assign(c->period, 0);
   c->graph_launches.assign(c->period, 0);

@@ -179,9 +179,10 @@ def test_bf16_forward_with_frozen_weights():
 def test_bf16_ten_steps(arch, K, splits):
     res = run_pair(arch, K, splits, 10, beta=0.5, lr=0.05, precision="bf16")
     assert res["log_gpu"] == res["log_oracle"]
-    assert res["params"] <= 2e-2, res                           # stated bar
-    assert res["loss"] <= 1e-2 and res["out"] <= 5e-2, res      # forward after diverging updates
-    assert res["grads"] <= 0.5 and res["gin"] <= 1.0, res       # gate flips: see the note above
+    msg = str({k: v for k, v in res.items() if not k.startswith("log_")})
+    assert res["params"] <= 2e-2, msg                           # stated bar
+    assert res["loss"] <= 1e-2 and res["out"] <= 5e-2, msg      # forward after diverging updates
+    assert res["grads"] <= 0.5 and res["gin"] <= 1.0, msg       # gate flips: see the note above
 
 
 def test_resnet110_k4_bf16_reduced_batch():
