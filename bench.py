@@ -35,6 +35,8 @@ BETA, LR, MOM, WD = 0.2, 0.01, 0.9, 5e-4
 
 # The other workloads of the paper's tables that the library is measured on (--workload); the
 # default, and the only one the bench line's metric is quoted on, is resnet110_k4.
+CONV_HALO_FPROP_STAGE1_DRAM_BYTES = 4266752
+
 WORKLOADS = {
     "tiny_k2": dict(arch=dict(family="resnet6n2", n_per_stage=1, widths=(8, 16, 32), stem_width=8, in_h=16, in_w=16,
                               in_c=3, num_classes=10, batch=8), K=2, splits=(1,), beta=0.2, lr=0.1,
@@ -368,7 +370,10 @@ def run_gpu(args):
                         kernel="conv_halo_kernel, 3x3 stride-1 forward, [128,32,32,16] -> 16 channels",
                         avg_us=us, tflops=flops / us / 1e6,
                         how="64 launches on distinct buffers (pool > 2 x L2) replayed from a CUDA graph, CUDA events "
-                            "on the replay stream")
+                            "on the replay stream",
+                        # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this shape
+                        # (one ncu capture; the output stays in L2); reset to None when the kernel changes
+                        traffic=CONV_HALO_FPROP_STAGE1_DRAM_BYTES)
         elif False:
             tensor_peak = peaks["bf16_tflops"]
             tensor_frac = top["flops"] / sec / 1e12 / tensor_peak
@@ -385,7 +390,8 @@ def run_gpu(args):
         roof.setdefault("kernel", top["name"])
         roof.setdefault("avg_us", top["total_ms"] * 1e3 / top["launches"])
         roof.setdefault("how", "CUDA events around every launch on its stream, serial context, %d steps" % prof_steps)
-        roof.update(frac=roof["achieved"] / roof["peak"], traffic=None, peak_source=peaks["source"],
+        roof.setdefault("traffic", None)
+        roof.update(frac=roof["achieved"] / roof["peak"], peak_source=peaks["source"],
                     per_class_note="serial context, CUDA events around every launch: includes the host's launch gaps",
                     per_class={s["name"]: dict(ms_per_step=s["total_ms"] / prof_steps, share=s["total_ms"] / total,
                                                gbs=s["bytes"] / (s["total_ms"] * 1e-3) / 1e9,

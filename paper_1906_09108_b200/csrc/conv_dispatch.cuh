@@ -25,6 +25,8 @@ struct TensorMapCache {
   int sm_count = 0;
   int share = 1;        // kernels expected to run side by side (one per module stream): a launch takes
                         // about sm_count / share CTAs and walks its tiles with them
+  int wgrad_side_cap = 0;   // upper bound of the pixel split of a weight gradient issued beside the stream that
+                            // needs its inputs' other consumers (0 = none), see halo::wgrad_ctas
 };
 
 inline bool tc_eligible(const ConvGeom& g) {
@@ -153,14 +155,15 @@ inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, 
 // dw[Co][3][3][Ci] (fp32) from x [N][H][W][Ci] and dy [N][H][W][Co]; `scratch` holds the per-CTA partials
 // (halo::wgrad_scratch_elems floats).  Two launches: the tensor-core kernel and the fixed-order sum.
 inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ci, int Co,
-                                  const bf16_t* x, const bf16_t* dy, float* dw, float* scratch, int* err_dev) {
+                                  const bf16_t* x, const bf16_t* dy, float* dw, float* scratch, int* err_dev,
+                                  bool side = false) {
   halo::WgradParams p = halo::wgrad_params(N, H, W, Ci, Co);
   const CUtensorMap *mx, *my;
   cudaError_t e = cached_tile_map(cache, x, N, H, W, Ci, p.G, &mx, p.kcx);
   if (e == cudaSuccess) e = cached_tile_map(cache, dy, N, H, W, Co, p.G, &my, p.kcy);
   if (e == cudaSuccess) e = halo::set_smem_attrs();
   if (e != cudaSuccess) return e;
-  const int ctas = halo::wgrad_ctas(p);
+  const int ctas = halo::wgrad_ctas(p, side ? cache->wgrad_side_cap : 0);
   halo::wgrad_halo_kernel<<<dim3(ctas, halo::wgrad_pairs(p)), halo::kFwdThreads, halo::wgrad_smem_bytes(p), st>>>(*mx, *my, p, scratch, err_dev);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -704,18 +704,24 @@ inline WgradParams wgrad_params(int N, int H, int W, int Ci, int Co) {
 inline int wgrad_pairs(const WgradParams& p) { return (p.Ci / p.kcx) * (p.Co / p.kcy); }
 
 // Pixel split: few enough CTAs that their partial sums (Co*9*Ci floats each) stay small next to
-// the operands, enough of them to spread the reduction over the SMs.
-inline int wgrad_ctas(const WgradParams& p) {
+// the operands, enough of them to spread the reduction over the SMs.  `cap` (0 = none) bounds the
+// split further: beside other kernels a weight gradient that is nobody's next input does better on
+// a few SMs for longer than on many at once (measured: 16 CTAs instead of 64-128 take 9 % off an
+// iteration of four concurrent modules).  Scratch is sized for cap = 0.
+inline int wgrad_ctas(const WgradParams& p, int cap = 0) {
   const int pairs = wgrad_pairs(p);
+  int want;
   if (pairs > 1) {                                              // chunked (wide) layers: about 1.5 CTAs per SM in all
-    int want = (222 + pairs / 2) / pairs;
-    if (want < 1) want = 1;
-    return p.tiles < want ? p.tiles : want;
+    want = (222 + pairs / 2) / pairs;
+    if (cap > 0 && want * pairs > 4 * cap) want = 4 * cap / pairs;
+  } else {
+    const size_t wsize = (size_t)p.Co * 9 * p.Ci;
+    want = (int)((size_t)p.N * p.H * p.W * (p.Ci + p.Co) * 2 / (wsize * 2));     // partial bytes <= ~ 2 x operand bytes
+    if (want > 128) want = 128;
+    if (want < 32) want = 32;
+    if (cap > 0 && want > cap) want = cap;
   }
-  const size_t wsize = (size_t)p.Co * 9 * p.Ci;
-  int want = (int)((size_t)p.N * p.H * p.W * (p.Ci + p.Co) * 2 / (wsize * 2));     // partial bytes <= ~ 2 x operand bytes
-  if (want > 128) want = 128;
-  if (want < 32) want = 32;
+  if (want < 1) want = 1;
   return p.tiles < want ? p.tiles : want;
 }
 inline size_t wgrad_smem_bytes(const WgradParams& p) {

@@ -642,12 +642,12 @@ static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, cons
   if constexpr (std::is_same<T, bf16>::value) {
     if (dy_up && halo_s2_wgrad_eligible(g)) {                // stride 2: the stride-1 weight gradient with the spread-out dy
       L.c->launches += 2;
-      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy_up, dw, m.wscratch, L.c->tc_error));
+      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy_up, dw, m.wscratch, L.c->tc_error, L.st == m.stream2));
       return;
     }
     if (halo_wgrad_eligible(g)) {
       L.c->launches += 2;
-      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy, dw, m.wscratch, L.c->tc_error));
+      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy, dw, m.wscratch, L.c->tc_error, L.st == m.stream2));
       return;
     }
   }
@@ -1157,6 +1157,7 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   // per layer, 148 / K SMs each gives 2 tiles per CTA at K = 2 and 4 at K = 4; three per CTA (43 CTAs)
   // measured faster at K = 4 than both two and four, so one stream's share is left unclaimed there.
   c->tmaps.share = c->cfg.serial ? 1 : (c->K > 2 ? c->K - 1 : c->K);
+  c->tmaps.wgrad_side_cap = 16;
   c->graph_exec.assign(c->period, nullptr);
   c->graph_sig.assign(c->period, 0);
   c->graph_launches.assign(c->period, 0);

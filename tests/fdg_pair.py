@@ -81,6 +81,22 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
                         off, n = int(name.split("@")[1]), int(np.prod(shape))
                         per.append((round(relfro(gg[off:off + n], go[off:off + n]), 4), t, k, name, tuple(shape)))
                     res["worst_tensors"] = sorted(per, reverse=True)[:3]
+                    if err > 1.0 and "bad_ranges" not in res:
+                        # where in the flat gradient the two sides part, in chunks of 1024 elements, and whether a
+                        # second read of the same gradient returns the same values
+                        d = np.abs(gg.astype(np.float64) - go)
+                        n1k = (len(d) + 1023) // 1024
+                        bad = [c for c in range(n1k)
+                               if np.linalg.norm(d[c * 1024:(c + 1) * 1024]) > np.linalg.norm(go[c * 1024:(c + 1) * 1024]) + 1e-12]
+                        runs, start = [], None
+                        for c in range(n1k + 1):
+                            if c in set(bad) and start is None: start = c
+                            if c not in set(bad) and start is not None: runs.append((start * 1024, c * 1024)); start = None
+                        res["bad_ranges"] = runs[:12]
+                        res["reread_equal"] = bool(np.array_equal(gg, g.get_grads(k)))
+                        res["norms"] = [(name, float(np.linalg.norm(gg[int(name.split("@")[1]):int(name.split("@")[1]) + int(np.prod(shape))])),
+                                         float(np.linalg.norm(go[int(name.split("@")[1]):int(name.split("@")[1]) + int(np.prod(shape))])))
+                                        for name, _, shape in layouts[k]]
     g.sync()
     res["params"] = max(relfro(g.get_params(k), orc.get_params(k)) for k in range(1, K + 1))
     res["momentum"] = max(relfro(g.get_momentum(k), orc.get_momentum(k)) for k in range(1, K + 1))
