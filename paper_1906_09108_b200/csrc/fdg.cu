@@ -143,6 +143,7 @@ struct fdg_ctx {
   // CUDA-graph replay (cfg.graphs): one executable graph per phase of the rings
   bool use_graphs = false;
   int period = 1;                     // all ring sizes divide it
+  int ew_block_cap = 2 * 148;         // grid bound of the batch-norm apply kernels that re-add partial sums
   bool graph_mode_entered = false;
   std::vector<cudaGraphExec_t> graph_exec;
   std::vector<uint64_t> graph_sig, graph_launches;
@@ -488,7 +489,7 @@ static void bn_apply(Launch& L, Module& m, const T* x, float* stats, const float
   L.begin(KC_BN_APPLY, (double)n * sizeof(T) * (res ? 3 : 2), 6.0 * n);
   if (C % V == 0) {
     int blocks = ew_blocks(n / V);
-    if (nparts > 0) blocks = std::min(blocks, 2 * 148);      // every block re-adds the partials: keep them few
+    if (nparts > 0) blocks = std::min(blocks, L.c->ew_block_cap);   // every block re-adds the partials: keep them few
     bn_apply_kernel<T, V><<<blocks, kEwThreads, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
   } else {
     bn_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
@@ -528,7 +529,7 @@ static void bn_backward(Launch& L, Module& m, const T* dy, const T* mask, const 
   L.begin(KC_BN_BWD_APPLY, (double)n * sizeof(T) * (3 + (mask ? 1 : 0) + (two ? 2 : 0) + (res ? 1 : 0)), 10.0 * n);
   if (vec) {
     int blocks = ew_blocks(n / V);
-    if (sums_ready) blocks = std::min(blocks, 2 * 148);
+    if (sums_ready) blocks = std::min(blocks, L.c->ew_block_cap);
     bn_bwd_apply_kernel<T, V><<<blocks, kEwThreads, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n / V, C, inv_m, ps);
   } else {
     bn_bwd_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n, C, inv_m, ps);
@@ -1158,6 +1159,9 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   // measured faster at K = 4 than both two and four, so one stream's share is left unclaimed there.
   c->tmaps.share = c->cfg.serial ? 1 : (c->K > 2 ? c->K - 1 : c->K);
   c->tmaps.wgrad_side_cap = 16;
+  // Blocks of a batch-norm apply kernel that first re-adds a convolution's partial sums: 4 per SM shared
+  // between the module streams (measured optimum: 148 blocks at K = 4, 296 at K = 2).
+  c->ew_block_cap = c->cfg.serial ? 4 * 148 : std::max(74, 4 * 148 / c->K);
   c->graph_exec.assign(c->period, nullptr);
   c->graph_sig.assign(c->period, 0);
   c->graph_launches.assign(c->period, 0);
