@@ -362,7 +362,7 @@ def run_gpu(args):
         sec = top["total_ms"] * 1e-3
         hbm_frac = top["bytes"] / sec / 1e9 / peaks["hbm_gbs"]
         if args.precision == "bf16":
-            # Dominant kernel (share of device time in the ncu launch list under profiles/): the halo-tile
+            # Dominant kernel (largest share of device time in an ncu launch list of this workload): the halo-tile
             # convolution.  Timed alone on its most frequent shape; a 16-channel 3x3 layer has 72 flop per byte,
             # far below the machine balance, so HBM is the roofline that bounds it.
             us, nbytes, flops = kernel_bench(B, "fprop", "stage1")
@@ -382,7 +382,7 @@ def run_gpu(args):
             else:
                 roof = dict(bound="hbm", achieved=top["bytes"] / sec / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
         elif top["name"].startswith("conv"):
-            # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x max SM clock (see DESIGN.md)
+            # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x max SM clock
             alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
             roof = dict(bound="alu", achieved=top["flops"] / sec / 1e12, peak=alu_peak, unit="TFLOP/s")
         else:
