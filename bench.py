@@ -168,8 +168,9 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------ kernel-level arm --
-KERNEL_SHAPES = {     # the three 3x3 stride-1 layer shapes of the workload: (N, H, W, C)
-    "stage1": (128, 32, 32, 16), "stage2": (128, 16, 16, 32), "stage3": (128, 8, 8, 64)}
+KERNEL_SHAPES = {     # the 3x3 stride-1 layer shapes of the 6n+2 workloads and of WRN-28-10: (N, H, W, C)
+    "stage1": (128, 32, 32, 16), "stage2": (128, 16, 16, 32), "stage3": (128, 8, 8, 64),
+    "wrn_stage1": (128, 32, 32, 160), "wrn_stage2": (128, 16, 16, 320), "wrn_stage3": (128, 8, 8, 640)}
 
 
 def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5, use_graph=True):
@@ -246,7 +247,8 @@ def run_kernel_bench(args):
             us, nbytes, flops = kernel_bench(B, which, stage, launches=args.kernel_launches,
                                              reps=1 if args.kernel_launches <= 8 else 5, use_graph=args.kernel_launches > 8)
             out["%s_%s" % (which, stage)] = dict(us=us, gbs=nbytes / us / 1e3, tflops=flops / us / 1e6,
-                                                 hbm_frac=nbytes / us / 1e3 / peaks["hbm_gbs"])
+                                                 hbm_frac=nbytes / us / 1e3 / peaks["hbm_gbs"],
+                                                 tensor_frac=flops / us / 1e6 / peaks["bf16_tflops"])
     print(json.dumps(dict(kernel_bench=out, peak_source=peaks["source"], hbm_gbs=peaks["hbm_gbs"])))
 
 
