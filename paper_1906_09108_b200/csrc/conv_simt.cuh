@@ -15,6 +15,7 @@
 //          A = x[n, p*st+r-pad, q*st+s-pad, c_in]     B = dy[pixel][c_out]
 //          C -> partial[z][c_out][r][s][c_in], summed over z in a fixed order afterwards
 #pragma once
+#include <algorithm>
 #include <type_traits>
 
 #include "elementwise.cuh"
@@ -265,13 +266,76 @@ inline cudaError_t launch_conv_simt(cudaStream_t st, const ConvGeom& g, const T*
   return e;
 }
 
+// ---- weight gradient of a 3x3 / stride 1 / pad 1 convolution with very few input channels ----
+// (the stem: 3 image channels).  The GEMM view has M = 9*Ci <= 36 rows against 128-row tiles, so
+// the tiled kernel above spends its time gathering.  Here a block takes one image, stages strips of
+// x (with its one-pixel border, zero outside the image) and dy in shared memory as floats, and
+// thread (m, co) with m = (r*3+s)*Ci + ci accumulates dW[co][r][s][ci] over the strip's pixels.
+// Partial sums: partial[image][co*9*Ci + m], added over the images afterwards in image order.
+constexpr int kSmallWgradRows = 8;        // output rows per strip
+inline bool small_wgrad_eligible(const ConvGeom& g) {
+  return g.R == 3 && g.S == 3 && g.stride == 1 && g.pad == 1 && g.P == g.H && g.Q == g.W && g.Ci <= 4 &&
+         9 * g.Ci * g.Co <= 1024 && g.W <= 64 &&
+         ((size_t)(kSmallWgradRows + 2) * (g.W + 2) * g.Ci + (size_t)kSmallWgradRows * g.W * g.Co) * 4 <= 48 * 1024;
+}
+template <typename T>
+__global__ void small_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial,
+                                   int H, int W, int Ci, int Co) {
+  extern __shared__ float sw_smem[];
+  const int Wp = W + 2;
+  float* xs = sw_smem;                                          // [kSmallWgradRows + 2][Wp][Ci]
+  float* ds = sw_smem + (kSmallWgradRows + 2) * Wp * Ci;          // [kSmallWgradRows][W][Co]
+  const int n = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+  const int outs = 9 * Ci * Co;
+  const int co = tid % Co, m = tid / Co, tap = m / Ci, ci = m - tap * Ci, r = tap / 3, sx = tap - 3 * r;
+  const T* xn = x + (size_t)n * H * W * Ci;
+  const T* dn = dy + (size_t)n * H * W * Co;
+  double acc = 0.0;                       // a row's products in fp32, the rows in fp64: this gradient is compared at 1e-4
+  for (int h0 = 0; h0 < H; h0 += kSmallWgradRows) {
+    const int rows = min(kSmallWgradRows, H - h0);
+    __syncthreads();
+    for (int i = tid; i < (rows + 2) * Wp * Ci; i += nt) {
+      const int c = i % Ci, w = (i / Ci) % Wp - 1, h = h0 + i / (Ci * Wp) - 1;
+      xs[i] = (h >= 0 && h < H && w >= 0 && w < W) ? to_f(xn[((size_t)h * W + w) * Ci + c]) : 0.f;
+    }
+    for (int i = tid; i < rows * W * Co; i += nt) ds[i] = to_f(dn[(size_t)h0 * W * Co + i]);
+    __syncthreads();
+    if (tid < outs)
+      for (int p = 0; p < rows; ++p) {
+        const float* xr = xs + ((p + r) * Wp + sx) * Ci + ci;
+        const float* dr = ds + (size_t)p * W * Co + co;
+        float row = 0.f;
+        for (int q = 0; q < W; ++q) row += xr[q * Ci] * dr[q * Co];
+        acc += (double)row;
+      }
+  }
+  if (tid < outs) partial[(size_t)n * outs + (size_t)co * 9 * Ci + m] = (float)acc;
+}
+// dw[Co][3][3][Ci] from x [N][H][W][Ci] and dy [N][H][W][Co]; `scratch` holds N * 9*Ci*Co floats.
+template <typename T>
+inline cudaError_t launch_small_wgrad(cudaStream_t st, const ConvGeom& g, const T* x, const T* dy, float* scratch,
+                                      float* dw, uint64_t* launches) {
+  const int outs = 9 * g.Ci * g.Co;
+  const int threads = (outs + 31) / 32 * 32;
+  const size_t smem = ((size_t)(kSmallWgradRows + 2) * (g.W + 2) * g.Ci + (size_t)kSmallWgradRows * g.W * g.Co) * 4;
+  small_wgrad_kernel<T><<<g.N, threads, smem, st>>>(x, dy, scratch, g.H, g.W, g.Ci, g.Co);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  int blocks = (outs + 255) / 256;
+  wgrad_reduce_kernel<<<blocks, 256, 0, st>>>(scratch, dw, (size_t)outs, g.N);
+  *launches += 2;
+  return cudaGetLastError();
+}
+
 // Upper bound of the fp32 scratch elements a weight-gradient launch may need.
 inline size_t wgrad_scratch_elems(const ConvGeom& g) {
   long Ndim = g.Co;
   int bm = Ndim <= 32 ? 128 : 64, bn = Ndim <= 16 ? 16 : (Ndim <= 32 ? 32 : 64);
   int splits, chunk;
   wgrad_split(g, bm, bn, &splits, &chunk);
-  return (size_t)splits * g.R * g.S * g.Ci * g.Co;
+  size_t n = (size_t)splits * g.R * g.S * g.Ci * g.Co;
+  if (small_wgrad_eligible(g)) n = std::max(n, (size_t)g.N * 9 * g.Ci * g.Co);
+  return n;
 }
 
 }  // namespace fdg

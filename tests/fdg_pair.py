@@ -73,7 +73,7 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
             if go is not None:
                 gg = g.get_grads(k)
                 err = relfro(gg, go)
-                res["grads_by_step"].append((t, k, round(err, 4)))
+                res["grads_by_step"].append((t, k, float("%.3g" % err)))
                 if err > res["grads"]:
                     res["grads"] = err
                     per = []
