@@ -327,6 +327,68 @@ inline cudaError_t launch_small_wgrad(cudaStream_t st, const ConvGeom& g, const 
   return cudaGetLastError();
 }
 
+// ---- weight gradient of a 1x1 convolution (projection shortcut), stride 1 or 2, few channels ----
+// dW[co][ci] = sum over output pixels of dy[n,p,q,co] * x[n,p*stride,q*stride,ci]: a Ci x Co matrix
+// (512 or 2048 entries on the 6n+2 networks) from tens of thousands of pixels.  Same scheme as above:
+// one image per block, strips staged in shared memory, thread (ci, co) with consecutive co in a warp.
+inline bool proj_wgrad_eligible(const ConvGeom& g) {
+  return g.R == 1 && g.S == 1 && g.pad == 0 && (g.stride == 1 || g.stride == 2) && g.Ci * g.Co <= 2048 && g.Co % 32 == 0 &&
+         (size_t)kSmallWgradRows * g.Q * (g.Ci + g.Co) * 4 <= 48 * 1024;
+}
+template <typename T>
+__global__ void proj_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial,
+                                  int H, int W, int P, int Q, int Ci, int Co, int stride) {
+  extern __shared__ float pw_smem[];
+  float* xs = pw_smem;                                      // [kSmallWgradRows][Q][Ci]
+  float* ds = pw_smem + kSmallWgradRows * Q * Ci;             // [kSmallWgradRows][Q][Co]
+  const int n = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+  const int outs = Ci * Co;
+  const T* xn = x + (size_t)n * H * W * Ci;
+  const T* dn = dy + (size_t)n * P * Q * Co;
+  double acc[2] = {0.0, 0.0};                               // thread tid owns outputs tid and tid + nt (if any)
+  for (int p0 = 0; p0 < P; p0 += kSmallWgradRows) {
+    const int rows = min(kSmallWgradRows, P - p0);
+    __syncthreads();
+    for (int i = tid; i < rows * Q * Ci; i += nt) {
+      const int c = i % Ci, q = (i / Ci) % Q, p = p0 + i / (Ci * Q);
+      xs[i] = to_f(xn[((size_t)(p * stride) * W + q * stride) * Ci + c]);
+    }
+    for (int i = tid; i < rows * Q * Co; i += nt) ds[i] = to_f(dn[(size_t)p0 * Q * Co + i]);
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int o = tid + k * nt;
+      if (o >= outs) break;
+      const int co = o % Co, ci = o / Co;
+      for (int p = 0; p < rows; ++p) {
+        const float* xr = xs + (size_t)p * Q * Ci + ci;
+        const float* dr = ds + (size_t)p * Q * Co + co;
+        float row = 0.f;
+        for (int q = 0; q < Q; ++q) row += xr[q * Ci] * dr[q * Co];
+        acc[k] += (double)row;
+      }
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const int o = tid + k * nt;
+    if (o < outs) partial[(size_t)n * outs + (size_t)(o % Co) * Ci + o / Co] = (float)acc[k];
+  }
+}
+template <typename T>
+inline cudaError_t launch_proj_wgrad(cudaStream_t st, const ConvGeom& g, const T* x, const T* dy, float* scratch,
+                                     float* dw, uint64_t* launches) {
+  const int outs = g.Ci * g.Co;
+  const int threads = outs >= 1024 ? 1024 : (outs + 31) / 32 * 32;
+  const size_t smem = (size_t)kSmallWgradRows * g.Q * (g.Ci + g.Co) * 4;
+  proj_wgrad_kernel<T><<<g.N, threads, smem, st>>>(x, dy, scratch, g.H, g.W, g.P, g.Q, g.Ci, g.Co, g.stride);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  wgrad_reduce_kernel<<<(outs + 255) / 256, 256, 0, st>>>(scratch, dw, (size_t)outs, g.N);
+  *launches += 2;
+  return cudaGetLastError();
+}
+
 // Upper bound of the fp32 scratch elements a weight-gradient launch may need.
 inline size_t wgrad_scratch_elems(const ConvGeom& g) {
   long Ndim = g.Co;
@@ -335,6 +397,7 @@ inline size_t wgrad_scratch_elems(const ConvGeom& g) {
   wgrad_split(g, bm, bn, &splits, &chunk);
   size_t n = (size_t)splits * g.R * g.S * g.Ci * g.Co;
   if (small_wgrad_eligible(g)) n = std::max(n, (size_t)g.N * 9 * g.Ci * g.Co);
+  if (proj_wgrad_eligible(g)) n = std::max(n, (size_t)g.N * g.Ci * g.Co);
   return n;
 }
 

@@ -657,6 +657,10 @@ static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, cons
     L.note(launch_small_wgrad<T>(L.st, g, x, dy, m.wscratch, dw, &L.c->launches));
     return;
   }
+  if (std::is_same<T, bf16>::value && proj_wgrad_eligible(g)) {
+    L.note(launch_proj_wgrad<T>(L.st, g, x, dy, m.wscratch, dw, &L.c->launches));
+    return;
+  }
   L.note(launch_conv_simt<T, CONV_WGRAD>(L.st, g, x, dy, (T*)nullptr, m.wscratch, dw, (const T*)nullptr, (const T*)nullptr, &L.c->launches));
 }
 
