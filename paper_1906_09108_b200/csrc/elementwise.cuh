@@ -122,12 +122,19 @@ __device__ __forceinline__ void channel_reduce(const RedGeom g, float* __restric
     for (int rr = 0; rr < g.rp; ++rr) a += red_smem[rr * NS * C + j];
     partial[(size_t)blockIdx.x * NS * C + j] = a;
   }
-  __threadfence();
+  // Release: the block's partial sums were written by all of its threads, the ticket is taken by one.
+  // The fence that makes them visible before the ticket has to be executed by the ticket's thread
+  // AFTER the barrier that orders it behind the other threads' writes: a fence each writer executes
+  // before the barrier orders only that writer's own later accesses, and the ticket could then reach
+  // L2 ahead of another warp's partial sums (seen on some GPUs as a last block adding stale rows).
   __syncthreads();
-  if (tid == 0) is_last = (atomicInc(counter, gridDim.x - 1) == gridDim.x - 1);
+  if (tid == 0) {
+    __threadfence();
+    is_last = (atomicInc(counter, gridDim.x - 1) == gridDim.x - 1);
+  }
   __syncthreads();
   if (!is_last) return;
-  __threadfence();
+  __threadfence();                                           // acquire: before the other blocks' partial sums are read
   // NS*C (sum, channel) pairs; kRedThreads / pairs threads share a pair, each taking every
   // nseg-th block with 8 loads in flight; the segment sums are then added in segment order.
   __shared__ double fin[kRedThreads];

@@ -1174,6 +1174,9 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   c->graph_exec.assign(c->period, nullptr);
   c->graph_sig.assign(c->period, 0);
   c->graph_launches.assign(c->period, 0);
+  // The clearing of the workspace and the table uploads above ran on the default stream, which the module
+  // streams (non-blocking) do not wait for: nothing may be enqueued on them before those have finished.
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) { delete c; return FDG_ERR_CUDA; }
   *out_ctx = c;
   return FDG_OK;
@@ -1229,10 +1232,14 @@ static fdg_status copy_vec(fdg_ctx* c, int module, float* dev_vec, const float* 
   if (e == cudaSuccess && n) {
     if (src) e = cudaMemcpy(dev_vec, src, n * 4, cudaMemcpyDefault);
     else e = cudaMemcpy(dst, dev_vec, n * 4, cudaMemcpyDefault);
+    // A copy from pageable host memory returns when the data is staged, not when it has reached the device,
+    // and the module streams (non-blocking) do not wait for the default stream the copy runs on: everything
+    // below, and every later kernel that reads this vector, has to start after the copy has landed.
+    if (e == cudaSuccess && src) e = cudaDeviceSynchronize();
   }
   if (e == cudaSuccess && refresh && n) {
     for (int v = 0; v < m.Dw && e == cudaSuccess; ++v) {
-      e = cudaMemcpy(m.wver + (size_t)v * align_up(n, 64), m.theta, n * 4, cudaMemcpyDeviceToDevice);
+      e = cudaMemcpyAsync(m.wver + (size_t)v * align_up(n, 64), m.theta, n * 4, cudaMemcpyDeviceToDevice, m.stream);
       if (e == cudaSuccess && c->bf16_mode) {
         cast_kernel<bf16><<<(int)std::min<size_t>((n + 255) / 256, 1184), 256, 0, m.stream>>>(m.theta, m.wver16 + (size_t)v * align_up(n, 64), n);
         ++c->launches;
