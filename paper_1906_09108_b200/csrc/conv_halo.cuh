@@ -154,12 +154,20 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       for (int i = threadIdx.x; i < 2 * p.Cn; i += kFwdThreads) red_stat[i] = red.pstats[i];
   }
   if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kMmaWarps); }
     mbar_init(w_full, 1);
     const int groups_per_tile = p.Cn / 16 < kEpiGroups ? p.Cn / 16 : kEpiGroups;
     for (int a = 0; a < p.nacc; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4 * groups_per_tile); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // This thread is also the producer: the weights and the first tile are requested now, so that their
+    // latency runs beside the tensor-memory allocation and the barrier below instead of after them.
+    mbar_expect_tx(w_full, 9 * p.w_tx_bytes);
+    for (int tap = 0; tap < 9; ++tap) tma_load_2d(w_smem + (size_t)tap * p.w_tap_bytes, &map_w, w_full, tap * p.Ck, 0);
+    mbar_expect_tx(&full[0], p.tile_tx_bytes);
+    tma_load_4d(smem, &map_x, &full[0], 0, -1, -1, (int)blockIdx.x * p.G);
   }
   if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
   tc_fence_before();
@@ -170,10 +178,8 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_expect_tx(w_full, 9 * p.w_tx_bytes);
-      for (int tap = 0; tap < 9; ++tap) tma_load_2d(w_smem + (size_t)tap * p.w_tap_bytes, &map_w, w_full, tap * p.Ck, 0);
-      uint32_t it = 0;
-      for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
+      uint32_t it = 1;                                       // weights and tile 0 were requested during set-up
+      for (int tile = blockIdx.x + gridDim.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
         if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) break;
@@ -460,11 +466,18 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk_a = blockIdx.y / p.nyb, chunk_b = blockIdx.y - chunk_a * p.nyb;
   if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_y)) : "memory");
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kMmaWarps); }
     mbar_init(done, kMmaWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // the producer's first pair of tiles, requested during set-up (they do not touch the slack cleared below)
+    mbar_expect_tx(&full[0], p.x_tx_bytes + p.y_tx_bytes);
+    tma_load_4d(smem, &map_x, &full[0], chunk_a * p.kcx, -1, -1, (int)blockIdx.x * p.G);
+    tma_load_4d(smem + p.x_bytes, &map_y, &full[0], chunk_b * p.kcy, 0, -2, (int)blockIdx.x * p.G);
   }
   // The reduction runs over whole 16-pixel steps and the stacked blocks read some pixels past
   // the tile: that slack is never written by TMA, so it is cleared once (a stray NaN there
@@ -482,12 +495,11 @@ wgrad_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int ncols = 3 * p.kcy;                                // N of the instruction
-  const int chunk_a = blockIdx.y / p.nyb, chunk_b = blockIdx.y - chunk_a * p.nyb;
 
   if (warp == 0) {
     if (lane == 0) {
-      uint32_t it = 0;
-      for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
+      uint32_t it = 1;                                        // the first pair was requested during set-up
+      for (int tile = blockIdx.x + gridDim.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
         if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) break;
