@@ -389,10 +389,61 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       cur = nxt;
       return have_next;
     };
-    Operands op_a, op_b;
-    if (!*abort_flag && cur.tile < p.tiles) {
-      fetch(cur, op_a);
-      while (item(op_a, op_b) && item(op_b, op_a)) {}
+    // 16-channel layers with batch-norm statistics and no residual (the forward convolutions of the first
+    // stage, nine items per image): every item of a thread belongs to the same 16 channels, so the sums are
+    // kept per thread and the lanes are combined once at the end; no global operands, no second register set.
+    auto item_stats16 = [&](float (&run)[32]) -> bool {
+      Cursor nxt = cur;
+      const bool have_next = advance(nxt);
+      const int n = cur.tile * p.G + cur.g;
+      const bool valid = cur.h < p.H && cur.w < p.W && cur.g < p.G && n < p.N && (p.sub == 1 || ((cur.h | cur.w) & 1) == 0);
+      const int pix = p.sub == 1 ? (n * p.H + cur.h) * p.W + cur.w : (n * (p.H >> 1) + (cur.h >> 1)) * (p.W >> 1) + (cur.w >> 1);
+      const int slot = cur.slot;
+      if (!mbar_wait(&acc_full[slot], cur.aph, abort_flag)) return false;
+      tc_fence_after();
+      uint32_t v[16];
+      tmem_ld16(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)slot * p.Cn, v);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[slot]);            // the values are in registers: the slot is free
+      if (valid) {
+        uint4 o0, o1;
+        __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
+        __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          ob0[e] = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+          ob1[e] = __floats2bfloat162_rn(__uint_as_float(v[8 + 2 * e]), __uint_as_float(v[8 + 2 * e + 1]));
+        }
+        __nv_bfloat16* out_row = out + (size_t)pix * p.Cn;
+        *reinterpret_cast<uint4*>(out_row) = o0;
+        *reinterpret_cast<uint4*>(out_row + 8) = o1;
+        const __nv_bfloat16* sb0 = reinterpret_cast<const __nv_bfloat16*>(&o0);
+        const __nv_bfloat16* sb1 = reinterpret_cast<const __nv_bfloat16*>(&o1);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {                         // the statistics of the values as stored
+          const float a = __bfloat162float(sb0[e]), b = __bfloat162float(sb1[e]);
+          run[e] += a; run[16 + e] += a * a;
+          run[8 + e] += b; run[24 + e] += b * b;
+        }
+      }
+      cur = nxt;
+      return have_next;
+    };
+    if (red.mode == 1 && nch == 1 && !res) {
+      float run[32];
+#pragma unroll
+      for (int e = 0; e < 32; ++e) run[e] = 0.f;
+      if (!*abort_flag && cur.tile < p.tiles) while (item_stats16(run)) {}
+      transpose_reduce32(run, lane);
+      red_run[((warp - kFirstEpiWarp) * 8) * 32 + lane] += run[0];
+    } else {
+      Operands op_a, op_b;
+      if (!*abort_flag && cur.tile < p.tiles) {
+        fetch(cur, op_a);
+        while (item(op_a, op_b) && item(op_b, op_a)) {}
+      }
     }
   }
 
