@@ -431,7 +431,76 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       cur = nxt;
       return have_next;
     };
-    if (red.mode == 1 && nch == 1 && !res) {
+    // The same for the data gradient that also forms the sums of the batch-norm backward it feeds
+    // (no residual): the gate and the normalised tensor of an item are requested one item ahead.
+    struct Operands2 { bool valid; int pix; uint4 k0, k1, x0, x1; };
+    auto fetch2 = [&](const Cursor& c, Operands2& o) {
+      const int n = c.tile * p.G + c.g;
+      o.valid = c.h < p.H && c.w < p.W && c.g < p.G && n < p.N && (p.sub == 1 || ((c.h | c.w) & 1) == 0);
+      o.pix = p.sub == 1 ? (n * p.H + c.h) * p.W + c.w : (n * (p.H >> 1) + (c.h >> 1)) * (p.W >> 1) + (c.w >> 1);
+      o.k0 = o.k1 = o.x0 = o.x1 = make_uint4(0, 0, 0, 0);
+      if (!o.valid) return;
+      const size_t base = (size_t)o.pix * p.Cn;
+      o.k0 = *reinterpret_cast<const uint4*>(red.mask + base);
+      o.k1 = *reinterpret_cast<const uint4*>(red.mask + base + 8);
+      o.x0 = *reinterpret_cast<const uint4*>(red.xprev + base);
+      o.x1 = *reinterpret_cast<const uint4*>(red.xprev + base + 8);
+    };
+    auto item_bwd16 = [&](float (&run)[32], Operands2& use, Operands2& fill) -> bool {
+      Cursor nxt = cur;
+      const bool have_next = advance(nxt);
+      if (have_next) fetch2(nxt, fill);
+      const int slot = cur.slot;
+      if (!mbar_wait(&acc_full[slot], cur.aph, abort_flag)) return false;
+      tc_fence_after();
+      uint32_t v[16];
+      tmem_ld16(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)slot * p.Cn, v);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[slot]);
+      if (use.valid) {
+        uint4 o0, o1;
+        __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
+        __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          ob0[e] = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+          ob1[e] = __floats2bfloat162_rn(__uint_as_float(v[8 + 2 * e]), __uint_as_float(v[8 + 2 * e + 1]));
+        }
+        __nv_bfloat16* out_row = out + (size_t)use.pix * p.Cn;
+        *reinterpret_cast<uint4*>(out_row) = o0;
+        *reinterpret_cast<uint4*>(out_row + 8) = o1;
+        const __nv_bfloat16* sb0 = reinterpret_cast<const __nv_bfloat16*>(&o0);
+        const __nv_bfloat16* sb1 = reinterpret_cast<const __nv_bfloat16*>(&o1);
+        const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&use.k0);
+        const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&use.k1);
+        const __nv_bfloat16* xb0 = reinterpret_cast<const __nv_bfloat16*>(&use.x0);
+        const __nv_bfloat16* xb1 = reinterpret_cast<const __nv_bfloat16*>(&use.x1);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float mk = __bfloat162float(e < 8 ? mb0[e] : mb1[e - 8]);
+          const float xp = __bfloat162float(e < 8 ? xb0[e] : xb1[e - 8]);
+          const float dz = mk > 0.f ? __bfloat162float(e < 8 ? sb0[e] : sb1[e - 8]) : 0.f;
+          run[e] += dz;
+          run[16 + e] += dz * ((xp - red_stat[e]) * red_stat[p.Cn + e]);
+        }
+      }
+      cur = nxt;
+      return have_next;
+    };
+    if (red.mode == 2 && nch == 1 && !res) {
+      float run[32];
+#pragma unroll
+      for (int e = 0; e < 32; ++e) run[e] = 0.f;
+      Operands2 oa, ob;
+      if (!*abort_flag && cur.tile < p.tiles) {
+        fetch2(cur, oa);
+        while (item_bwd16(run, oa, ob) && item_bwd16(run, ob, oa)) {}
+      }
+      transpose_reduce32(run, lane);
+      red_run[((warp - kFirstEpiWarp) * 8) * 32 + lane] += run[0];
+    } else if (red.mode == 1 && nch == 1 && !res) {
       float run[32];
 #pragma unroll
       for (int e = 0; e < 32; ++e) run[e] = 0.f;
