@@ -189,9 +189,19 @@ fdg_status fdg_step_host(fdg_ctx* ctx, fdg_stream stream, const float* images_ho
                          float* loss_host);
 
 /* Makes `stream` wait for every module stream, then blocks the host until `stream` is idle.
- * Returns FDG_ERR_NONFINITE if any loss computed since the last call was NaN/Inf,
- * FDG_ERR_CUDA on an asynchronous CUDA error. */
+ * Returns FDG_ERR_NONFINITE if any loss computed since the last call was NaN/Inf, FDG_ERR_INVALID_ARG if a
+ * label was outside [0, num_classes) (it was treated as class 0), FDG_ERR_TIMEOUT (latched) if a bounded wait
+ * inside a tensor-core kernel ran out, FDG_ERR_CUDA on an asynchronous CUDA error.  The first two are
+ * reported once and cleared. */
 fdg_status fdg_sync(fdg_ctx* ctx, fdg_stream stream);
+
+/* Fault injection from the host, for testing the error paths without making a kernel misbehave: sets one of
+ * the device status words exactly as a kernel would (0: a non-finite loss, 1: a label out of range, 2: a
+ * bounded wait of a tensor-core kernel ran out).  The next fdg_sync reports it: FDG_ERR_NONFINITE,
+ * FDG_ERR_INVALID_ARG, or FDG_ERR_TIMEOUT; the first two clear with that report and the context carries on,
+ * the time-out is latched (a kernel left early, the in-flight state is undefined) and every later fdg_step /
+ * fdg_sync returns it.  Blocks the host. */
+fdg_status fdg_debug_raise_flag(fdg_ctx* ctx, int which);
 
 /* The most recent output activation of module k (1..K-1), and the most recent gradient
  * with respect to the input of module k (2..K; the gradient with respect to the images
@@ -218,6 +228,35 @@ fdg_status fdg_boundary_elems(const fdg_ctx* ctx, int module, size_t* out_elems,
  * forward.  Blocks the host.  Errors: FDG_ERR_INVALID_ARG (bad module/unit/which/n). */
 fdg_status fdg_get_saved_tensor(fdg_ctx* ctx, int module, int unit, int which, float* dst, size_t n,
                                 size_t* out_elems, int64_t* batch_index);
+
+/* The same for the slot that holds batch `batch` (a batch still in flight in this module, e.g. the one the
+ * next backward will read); `batch` < 0 selects the most recent forward.  *batch_index = -1 and nothing is
+ * copied when no slot holds that batch. */
+fdg_status fdg_get_saved_tensor_of(fdg_ctx* ctx, int module, int unit, int which, int64_t batch, float* dst, size_t n,
+                                   size_t* out_elems, int64_t* batch_index);
+
+/* Inspection of the delayed backward (Eq. 10 with the shrunk gradient of Eq. 15): while a capture is on for a
+ * module, every backward pass of that module copies each gradient tensor it forms, in stream order, into
+ * `dev_buffer` (device memory owned by the caller, 16-byte aligned, at least fdg_capture_bytes; it must stay
+ * valid until fdg_capture_end).  The kernels and their launch shapes are unchanged; only device-to-device
+ * copies are added.  Refused with FDG_ERR_STATE on a context created with graphs = 1.  Both calls block the host.
+ * fdg_get_captured returns one tensor of the most recent captured pass as fp32 NHWC (host or device memory);
+ * `unit` as in fdg_get_saved_tensor, `which`:
+ *   FDG_RESNET_6N2 block: 0 = gradient of the block output (already shrunk for the module's last block),
+ *                         1 = gradient of conv2's output (after the backward of ReLU and BN2),
+ *                         2 = gradient of ReLU(BN1(.)) (conv2's data gradient), 3 = gradient of conv1's output,
+ *                         4 = gradient of the block input, 5 = gradient of the projection convolution's output;
+ *   FDG_RESNET_6N2 stem:  0 = gradient of the stem output, 3 = gradient of the convolution output;
+ *   FDG_WRN block:        0 = gradient of the block output, 1 = gradient of ReLU(BN2(.)), 2 = gradient of conv1's
+ *                         output, 3 = gradient of ReLU(BN1(input)), 4 = gradient of the block input,
+ *                         5 = the projection's share of 3;
+ *   FDG_WRN stem:         0 = gradient of the stem output.
+ * *batch_index receives the batch of that pass, or -1 (nothing copied) before the first captured pass. */
+fdg_status fdg_capture_bytes(const fdg_ctx* ctx, int module, size_t* out_bytes);
+fdg_status fdg_capture_begin(fdg_ctx* ctx, int module, void* dev_buffer, size_t bytes);
+fdg_status fdg_capture_end(fdg_ctx* ctx, int module);
+fdg_status fdg_get_captured(fdg_ctx* ctx, int module, int unit, int which, float* dst, size_t n, size_t* out_elems,
+                            int64_t* batch_index);
 
 /* Copies at most `cap` rows of the schedule log (oldest first) and writes the number
  * of rows recorded so far to *out_n.  The log keeps every row of the last 4096 iterations. */

@@ -26,7 +26,10 @@ EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count"
            "fdg_set_lr", "fdg_step", "fdg_step_host", "fdg_sync", "fdg_profile_enable", "fdg_profile_read", "fdg_profile_read_modules", "fdg_get_module_output", "fdg_get_input_grad",
            "fdg_boundary_elems", "fdg_get_saved_tensor", "fdg_get_schedule_log", "fdg_launch_count", "fdg_status_string",
            "fdg_last_error", "fdg_conv_forward", "fdg_conv_dgrad", "fdg_conv_flip_weights",
-           "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_wgrad_static", "fdg_conv_path"]
+           "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_wgrad_static", "fdg_conv_path",
+           "fdg_get_saved_tensor_of", "fdg_capture_bytes", "fdg_capture_begin", "fdg_capture_end", "fdg_get_captured",
+           "fdg_bn_scratch_bytes", "fdg_bn_stats", "fdg_bn_apply", "fdg_bn_backward", "fdg_shrink", "fdg_sgd_update",
+           "fdg_ingest", "fdg_head", "fdg_debug_raise_flag"]
 
 
 class fdg_arch(C.Structure):
@@ -54,6 +57,15 @@ class fdg_sched_entry(C.Structure):
 class fdg_conv_shape(C.Structure):
     _fields_ = [("N", C.c_int), ("H", C.c_int), ("W", C.c_int), ("Ci", C.c_int), ("Co", C.c_int), ("R", C.c_int),
                 ("stride", C.c_int), ("pad", C.c_int)]
+
+
+class fdg_conv_extra(C.Structure):
+    _fields_ = [("share", C.c_int), ("wgrad_cta_cap", C.c_int), ("dy_spread", C.c_void_p), ("reduce", C.c_int),
+                ("next_mask", C.c_void_p), ("next_x", C.c_void_p), ("next_stats", C.c_void_p), ("partial", C.c_void_p),
+                ("partial_floats", C.c_size_t), ("nparts", C.c_int)]
+
+
+FDG_CONV_PARTIAL_ROWS = 256
 
 
 class fdg_kernel_stat(C.Structure):
@@ -91,11 +103,27 @@ def load_library(path=LIB_PATH):
         "fdg_get_saved_tensor": [vp, C.c_int, C.c_int, C.c_int, vp, sz, P(sz), P(i64)],
         "fdg_get_schedule_log": [vp, P(fdg_sched_entry), sz, P(sz)],
         "fdg_launch_count": [vp, P(C.c_uint64)],
-        "fdg_conv_forward": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, vp, vp],
-        "fdg_conv_dgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, vp, vp, vp, vp],
+        "fdg_conv_forward": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, P(fdg_conv_extra), vp, vp],
+        "fdg_conv_dgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, vp, vp, P(fdg_conv_extra), vp, vp],
         "fdg_conv_flip_weights": [P(fdg_conv_shape), vp, vp, vp],
         "fdg_conv_wgrad_scratch_bytes": [C.c_int, P(fdg_conv_shape), P(sz)],
-        "fdg_conv_wgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, sz, vp, vp],
+        "fdg_conv_wgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, sz, P(fdg_conv_extra), vp, vp],
+        "fdg_get_saved_tensor_of": [vp, C.c_int, C.c_int, C.c_int, i64, vp, sz, P(sz), P(i64)],
+        "fdg_debug_raise_flag": [vp, C.c_int],
+        "fdg_capture_bytes": [vp, C.c_int, P(sz)],
+        "fdg_capture_begin": [vp, C.c_int, vp, sz],
+        "fdg_capture_end": [vp, C.c_int],
+        "fdg_get_captured": [vp, C.c_int, C.c_int, C.c_int, vp, sz, P(sz), P(i64)],
+        "fdg_bn_scratch_bytes": [C.c_int, P(sz)],
+        "fdg_bn_stats": [C.c_int, vp, sz, C.c_int, C.c_float, vp, vp, sz, vp],
+        "fdg_bn_apply": [C.c_int, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int, vp, sz, C.c_int, C.c_float, vp, C.c_int,
+                         C.c_int, vp],
+        "fdg_bn_backward": [C.c_int, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, C.c_int, vp,
+                            C.c_int, C.c_int, vp, sz, vp],
+        "fdg_shrink": [C.c_int, vp, vp, C.c_float, sz, vp],
+        "fdg_sgd_update": [vp, vp, vp, vp, vp, sz, C.c_float, C.c_float, C.c_float, vp],
+        "fdg_ingest": [C.c_int, vp, vp, sz, C.c_int, C.c_int, vp, vp, C.c_int, vp],
+        "fdg_head": [C.c_int, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, vp, vp, vp, vp, vp, vp],
         "fdg_conv_wgrad_static": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp],
         "fdg_conv_path": [C.c_int, P(fdg_conv_shape), C.c_int, P(C.c_int)],
     }
@@ -274,6 +302,38 @@ class FDG:
                                                   C.byref(b)), self.ctx)
         return b.value, out
 
+    def saved_tensor_of(self, k, unit, which, batch):
+        """The same for the slot that holds `batch` (one still in flight in module k)."""
+        n, b = C.c_size_t(), C.c_int64()
+        self._check(self.lib.fdg_get_saved_tensor_of(self.ctx, k, unit, which, batch, None, 0, C.byref(n), None), self.ctx)
+        out = np.empty(n.value, dtype=np.float32)
+        self._check(self.lib.fdg_get_saved_tensor_of(self.ctx, k, unit, which, batch, out.ctypes.data, n.value, None,
+                                                     C.byref(b)), self.ctx)
+        return b.value, out
+
+    def capture_begin(self, k):
+        """Keeps a copy of every gradient tensor of module k's backward passes (torch owns the buffer)."""
+        n = C.c_size_t()
+        self._check(self.lib.fdg_capture_bytes(self.ctx, k, C.byref(n)), self.ctx)
+        buf = self.torch.empty(n.value + 256, dtype=self.torch.uint8, device=self.device)
+        base = (buf.data_ptr() + 255) // 256 * 256
+        self._check(self.lib.fdg_capture_begin(self.ctx, k, base, n.value), self.ctx)
+        self._capture = getattr(self, "_capture", {})
+        self._capture[k] = buf
+
+    def capture_end(self, k):
+        self._check(self.lib.fdg_capture_end(self.ctx, k), self.ctx)
+        self._capture.pop(k, None)
+
+    def captured(self, k, unit, which):
+        """(batch, flat fp32 array) of one gradient tensor of module k's most recent captured backward."""
+        n, b = C.c_size_t(), C.c_int64()
+        self._check(self.lib.fdg_get_captured(self.ctx, k, unit, which, None, 0, C.byref(n), None), self.ctx)
+        out = np.empty(n.value, dtype=np.float32)
+        self._check(self.lib.fdg_get_captured(self.ctx, k, unit, which, out.ctypes.data, n.value, None, C.byref(b)),
+                    self.ctx)
+        return b.value, out
+
     def schedule_log(self):
         n = C.c_size_t()
         self._check(self.lib.fdg_get_schedule_log(self.ctx, None, 0, C.byref(n)), self.ctx)
@@ -319,31 +379,55 @@ class ConvOps:
         self._chk(self.lib.fdg_conv_path(self.precision, C.byref(s), op, C.byref(v)))
         return bool(v.value)
 
-    def forward(self, s, x, w, res=None):
+    def _extra(self, s, share=0, wgrad_cta_cap=0, spread=False, reduce=0, next_mask=None, next_x=None, next_stats=None,
+               C_red=0):
+        """fdg_conv_extra plus the torch tensors it points to (kept alive by the caller)."""
+        ex = fdg_conv_extra()
+        ex.share, ex.wgrad_cta_cap, ex.reduce = share, wgrad_cta_cap, reduce
+        keep = []
+        if spread:
+            up = self.torch.empty((s.N, s.H, s.W, s.Co), dtype=self.dtype, device="cuda")
+            ex.dy_spread = up.data_ptr()
+            keep.append(up)
+        if reduce:
+            part = self.torch.full((FDG_CONV_PARTIAL_ROWS, 2 * C_red), float("nan"), dtype=self.torch.float32, device="cuda")
+            ex.partial, ex.partial_floats = part.data_ptr(), part.numel()
+            ex.next_mask, ex.next_x, ex.next_stats = _ptr(next_mask), _ptr(next_x), _ptr(next_stats)
+            keep.append(part)
+        return ex, keep
+
+    def forward(self, s, x, w, res=None, share=0, reduce=False):
+        """y, or (y, partial rows [nparts, 2*Co]) with reduce=True."""
         p, q = self.out_hw(s)
         y = self.torch.empty((s.N, p, q, s.Co), dtype=self.dtype, device="cuda")
+        ex, keep = self._extra(s, share=share, reduce=1 if reduce else 0, C_red=s.Co)
         self._chk(self.lib.fdg_conv_forward(self.precision, C.byref(s), _ptr(x), _ptr(w), _ptr(y), _ptr(res),
-                                            _ptr(self.status), self._stream()))
-        return y
+                                            C.byref(ex), _ptr(self.status), self._stream()))
+        return (y, keep[-1][:ex.nparts]) if reduce else y
 
     def flip_weights(self, s, w):
         out = self.torch.empty(s.Ci * 9 * s.Co, dtype=self.torch.bfloat16, device="cuda")
         self._chk(self.lib.fdg_conv_flip_weights(C.byref(s), _ptr(w), _ptr(out), self._stream()))
         return out
 
-    def dgrad(self, s, dy, w, w_flipped=None, res=None, res_mask=None):
+    def dgrad(self, s, dy, w, w_flipped=None, res=None, res_mask=None, share=0, spread=False, next_bn=None):
+        """dx, or (dx, partial rows [nparts, 2*Ci]) with next_bn = (mask, x, stats) of the batch norm dx feeds."""
         dx = self.torch.empty((s.N, s.H, s.W, s.Ci), dtype=self.dtype, device="cuda")
+        nm, nx, ns = next_bn if next_bn else (None, None, None)
+        ex, keep = self._extra(s, share=share, spread=spread, reduce=2 if next_bn else 0, next_mask=nm, next_x=nx,
+                               next_stats=ns, C_red=s.Ci)
         self._chk(self.lib.fdg_conv_dgrad(self.precision, C.byref(s), _ptr(dy), _ptr(w), _ptr(w_flipped), _ptr(dx),
-                                          _ptr(res), _ptr(res_mask), _ptr(self.status), self._stream()))
-        return dx
+                                          _ptr(res), _ptr(res_mask), C.byref(ex), _ptr(self.status), self._stream()))
+        return (dx, keep[-1][:ex.nparts]) if next_bn else dx
 
-    def wgrad(self, s, x, dy):
+    def wgrad(self, s, x, dy, cta_cap=0, spread=False):
         n = C.c_size_t()
         self._chk(self.lib.fdg_conv_wgrad_scratch_bytes(self.precision, C.byref(s), C.byref(n)))
         scratch = self.torch.empty(max(n.value, 16), dtype=self.torch.uint8, device="cuda")
         dw = self.torch.empty((s.Co, s.R, s.R, s.Ci), dtype=self.torch.float32, device="cuda")
+        ex, keep = self._extra(s, wgrad_cta_cap=cta_cap, spread=spread)
         self._chk(self.lib.fdg_conv_wgrad(self.precision, C.byref(s), _ptr(x), _ptr(dy), _ptr(dw), _ptr(scratch),
-                                          n.value, _ptr(self.status), self._stream()))
+                                          n.value, C.byref(ex), _ptr(self.status), self._stream()))
         return dw
 
     def wgrad_static(self, s, x, dy):
@@ -356,3 +440,100 @@ class ConvOps:
 
     def timed_out(self):
         return bool(self.status.item())
+
+
+class EwOps:
+    """The memory-bound operator-level calls (fdg_bn_*, fdg_shrink, fdg_sgd_update, fdg_ingest, fdg_head) on
+    torch CUDA tensors; activations [rows, C] (any leading shape) in the precision's storage type."""
+
+    def __init__(self, precision):
+        import torch
+        self.torch = torch
+        self.lib = load_library()
+        self.precision = precision
+        self.dtype = torch.bfloat16 if precision == FDG_BF16_TC else torch.float32
+
+    def _stream(self):
+        return self.torch.cuda.current_stream().cuda_stream
+
+    def _chk(self, rc):
+        if rc != FDG_OK:
+            raise FDGError(rc, self.lib.fdg_status_string(rc).decode())
+
+    def _scratch(self, ch):
+        n = C.c_size_t()
+        self._chk(self.lib.fdg_bn_scratch_bytes(ch, C.byref(n)))
+        return self.torch.empty(n.value, dtype=self.torch.uint8, device="cuda"), n.value
+
+    def _f32(self, *shape):
+        return self.torch.empty(shape, dtype=self.torch.float32, device="cuda")
+
+    def bn_stats(self, x, eps=1e-5):
+        ch = x.shape[-1]
+        rows = x.numel() // ch
+        stats = self._f32(2 * ch)
+        sc, nb = self._scratch(ch)
+        self._chk(self.lib.fdg_bn_stats(self.precision, _ptr(x), rows, ch, eps, _ptr(stats), _ptr(sc), nb, self._stream()))
+        return stats
+
+    def bn_apply(self, x, stats, gamma, beta, res=None, res_bn=None, relu=True, eps=1e-5, partial=None, block_cap=0):
+        """res_bn = (stats, gamma, beta) of the residual's own batch norm.  With `partial` (rows from a fused
+        convolution) `stats` is an output."""
+        ch = x.shape[-1]
+        rows = x.numel() // ch
+        y = self.torch.empty_like(x)
+        rs, rg, rb = res_bn if res_bn else (None, None, None)
+        self._chk(self.lib.fdg_bn_apply(self.precision, _ptr(x), _ptr(stats), _ptr(gamma), _ptr(beta), _ptr(res), _ptr(rs),
+                                        _ptr(rg), _ptr(rb), int(relu), _ptr(y), rows, ch, eps, _ptr(partial),
+                                        0 if partial is None else partial.shape[0], block_cap, self._stream()))
+        return y
+
+    def bn_backward(self, dy, mask, x, stats, gamma, second=None, res=None, partial=None, block_cap=0):
+        """Returns (dx, dgamma, dbeta) or, with second = (x2, stats2, gamma2), (dx, dgamma, dbeta, dx2, dgamma2, dbeta2)."""
+        ch = x.shape[-1]
+        rows = x.numel() // ch
+        dx = self.torch.empty_like(x)
+        dg, db = self._f32(ch), self._f32(ch)
+        x2, s2, g2 = second if second else (None, None, None)
+        dx2 = self.torch.empty_like(x) if second else None
+        dg2, db2 = (self._f32(ch), self._f32(ch)) if second else (None, None)
+        sc, nb = self._scratch(ch)
+        self._chk(self.lib.fdg_bn_backward(self.precision, _ptr(dy), _ptr(mask), _ptr(x), _ptr(stats), _ptr(gamma), _ptr(x2),
+                                           _ptr(s2), _ptr(g2), _ptr(res), _ptr(dx), _ptr(dx2), _ptr(dg), _ptr(db), _ptr(dg2),
+                                           _ptr(db2), rows, ch, _ptr(partial), 0 if partial is None else partial.shape[0],
+                                           block_cap, _ptr(sc), nb, self._stream()))
+        return (dx, dg, db, dx2, dg2, db2) if second else (dx, dg, db)
+
+    def shrink(self, x, beta):
+        out = self.torch.empty_like(x)
+        self._chk(self.lib.fdg_shrink(self.precision, _ptr(x), _ptr(out), beta, x.numel(), self._stream()))
+        return out
+
+    def sgd_update(self, theta, mom, grad, lr, momentum, weight_decay, bf16_copy=True):
+        """In place on theta and mom; returns (next fp32 copy, next bf16 copy or None)."""
+        n32 = self.torch.empty_like(theta)
+        n16 = self.torch.empty(theta.numel(), dtype=self.torch.bfloat16, device="cuda") if bf16_copy else None
+        self._chk(self.lib.fdg_sgd_update(_ptr(theta), _ptr(mom), _ptr(grad), _ptr(n32), _ptr(n16), theta.numel(), lr,
+                                          momentum, weight_decay, self._stream()))
+        return n32, n16
+
+    def ingest(self, images, c_out, labels):
+        rows = images.numel() // images.shape[-1]
+        out = self.torch.empty(tuple(images.shape[:-1]) + (c_out,), dtype=self.dtype, device="cuda")
+        lab = self.torch.empty_like(labels)
+        self._chk(self.lib.fdg_ingest(self.precision, _ptr(images), _ptr(out), rows, images.shape[-1], c_out, _ptr(labels),
+                                      _ptr(lab), labels.numel(), self._stream()))
+        return out, lab
+
+    def head(self, x, w, b, labels):
+        """x [B, HW.., F].  Returns dict(pooled, dlogits, loss_n, dx, dw, db, loss, flags)."""
+        bsz, feat = x.shape[0], x.shape[-1]
+        hw = x.numel() // (bsz * feat)
+        classes = w.shape[0]
+        o = dict(pooled=self._f32(bsz, feat), dlogits=self._f32(bsz, classes), loss_n=self._f32(bsz),
+                 dx=self.torch.empty_like(x), dw=self._f32(classes, feat), db=self._f32(classes), loss=self._f32(1),
+                 flags=self.torch.zeros(4, dtype=self.torch.int32, device="cuda"))
+        self._chk(self.lib.fdg_head(self.precision, _ptr(x), _ptr(w), _ptr(b), _ptr(labels), bsz, hw, feat, classes,
+                                    _ptr(o["pooled"]), _ptr(o["dlogits"]), _ptr(o["loss_n"]), _ptr(o["dx"]), _ptr(o["dw"]),
+                                    _ptr(o["db"]), _ptr(o["loss"]), _ptr(o["flags"]), self._stream()))
+        return o

@@ -9,6 +9,7 @@
 #include "conv_simt.cuh"
 #include "conv_tc.cuh"
 #include "conv_halo.cuh"
+#include "elementwise.cuh"
 
 namespace fdg {
 
@@ -177,6 +178,10 @@ inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N,
 inline bool dgrad_uses_flipped(const ConvGeom& g) {
   return halo_dgrad_eligible(g) || halo_s2_dgrad_eligible(g) || tc_eligible(g) || tc_s2_dgrad_eligible(g);
 }
+// Do the stride-2 gradients of this convolution run on the tensor cores, given a spread-out copy of dy?
+inline bool s2_uses_spread_dy(const ConvGeom& g) {
+  return (halo_s2_dgrad_eligible(g) || halo_s2_wgrad_eligible(g) || tc_s2_dgrad_eligible(g)) && g.Co % 8 == 0;
+}
 
 // fp32 scratch elements a weight-gradient call may need (bf16 storage: whichever kernel is chosen).
 inline size_t conv_wgrad_scratch_elems(bool bf16_storage, const ConvGeom& g) {
@@ -184,6 +189,85 @@ inline size_t conv_wgrad_scratch_elems(bool bf16_storage, const ConvGeom& g) {
   if (bf16_storage && (halo_wgrad_eligible(g) || halo_s2_wgrad_eligible(g)))
     n = std::max(n, halo::wgrad_scratch_elems(g.N, g.H, g.W, g.Ci, g.Co));
   return n;
+}
+
+// ---- one convolution operator in bf16 storage: which kernel, in which launch shape ------------------
+// Used by the module runtime and by the operator-level entry points alike.  `launches` counts kernels.
+
+// dy [N][P][Q][Co] of a stride-2 convolution spread onto the even pixels of a zero [N][H][W][Co] tensor `up`.
+inline cudaError_t bf16_spread_dy(cudaStream_t st, const ConvGeom& g, const bf16_t* dy, bf16_t* up, uint64_t* launches) {
+  const size_t nvec = (size_t)g.N * g.H * g.W * g.Co / 8;
+  upsample2_kernel<bf16_t, 8><<<ew_blocks(nvec), 256, 0, st>>>(dy, up, nvec, g.P, g.Q, g.Co);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+// y = conv(x, w) [+ res].  `red` (mode 1) asks for the per-CTA sums of y and y^2; *nparts receives the number
+// of rows left in red->partial, 0 when the chosen kernel forms none.
+inline cudaError_t bf16_conv_fprop(cudaStream_t st, TensorMapCache* cache, const ConvGeom& g, const bf16_t* x,
+                                   const bf16_t* w, bf16_t* y, const bf16_t* res, const halo::EpiReduce* red, int* nparts,
+                                   int* err_dev, uint64_t* launches) {
+  if (nparts) *nparts = 0;
+  const bool s1 = halo_fprop_eligible(g), s2 = !s1 && halo_s2_fprop_eligible(g);
+  if (s1 || s2) {
+    ++*launches;
+    const bool fuse = red && red->mode == 1 && halo_reduce_ok(g.Co);
+    int ctas = 0;
+    cudaError_t e = run_conv_halo(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, err_dev, fuse ? red : nullptr, &ctas, s2 ? 2 : 1);
+    if (fuse && nparts) *nparts = ctas;
+    return e;
+  }
+  if (tc_eligible(g) || tc_s2_fprop_eligible(g)) {
+    ++*launches;
+    return run_conv_tc(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, err_dev, g.stride);
+  }
+  return launch_conv_simt<bf16_t, CONV_FPROP>(st, g, x, w, y, nullptr, nullptr, res, (const bf16_t*)nullptr, launches);
+}
+
+// dx = conv^T(dy, w) [+ res * [mask > 0]].  `wflip` is the flipped/transposed weight copy (null: CUDA cores);
+// `dy_up` the spread-out dy of a stride-2 layer (null: its gradient stays on the CUDA cores).  `red` (mode 2)
+// asks for the sums of the batch-norm backward that dx feeds.
+inline cudaError_t bf16_conv_dgrad(cudaStream_t st, TensorMapCache* cache, const ConvGeom& g, const bf16_t* dy,
+                                   const bf16_t* w, const bf16_t* wflip, const bf16_t* dy_up, bf16_t* dx, const bf16_t* res,
+                                   const bf16_t* mask, const halo::EpiReduce* red, int* nparts, int* err_dev,
+                                   uint64_t* launches) {
+  if (nparts) *nparts = 0;
+  const bool h1 = wflip && halo_dgrad_eligible(g), h2 = !h1 && wflip && dy_up && halo_s2_dgrad_eligible(g);
+  if (h1 || h2) {
+    ++*launches;
+    const bool fuse = red && red->mode == 2 && halo_reduce_ok(g.Ci);
+    int ctas = 0;
+    cudaError_t e = run_conv_halo(st, cache, g.N, g.H, g.W, g.Co, g.Ci, h1 ? dy : dy_up, wflip, dx, res, mask, err_dev, fuse ? red : nullptr, &ctas);
+    if (fuse && nparts) *nparts = ctas;
+    return e;
+  }
+  if (wflip && tc_eligible(g)) {
+    ++*launches;
+    return run_conv_tc(st, cache, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, err_dev);
+  }
+  if (wflip && dy_up && tc_s2_dgrad_eligible(g)) {
+    ++*launches;
+    return run_conv_tc(st, cache, g.N, g.H, g.W, g.Co, g.Ci, dy_up, wflip, dx, res, mask, err_dev);
+  }
+  return launch_conv_simt<bf16_t, CONV_DGRAD>(st, g, dy, w, dx, nullptr, nullptr, res, mask, launches);
+}
+
+// dw (fp32) from x and dy; `scratch` of conv_wgrad_scratch_elems floats; `side`: bound the pixel split by
+// cache->wgrad_side_cap (a weight gradient issued beside the chain that needs the SMs more).
+inline cudaError_t bf16_conv_wgrad(cudaStream_t st, TensorMapCache* cache, const ConvGeom& g, const bf16_t* x,
+                                   const bf16_t* dy, const bf16_t* dy_up, float* dw, float* scratch, int* err_dev,
+                                   bool side, uint64_t* launches) {
+  if (dy_up && halo_s2_wgrad_eligible(g)) {
+    *launches += 2;
+    return run_wgrad_halo(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, dy_up, dw, scratch, err_dev, side);
+  }
+  if (halo_wgrad_eligible(g)) {
+    *launches += 2;
+    return run_wgrad_halo(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, dy, dw, scratch, err_dev, side);
+  }
+  if (small_wgrad_eligible(g)) return launch_small_wgrad<bf16_t>(st, g, x, dy, scratch, dw, launches);
+  if (proj_wgrad_eligible(g)) return launch_proj_wgrad<bf16_t>(st, g, x, dy, scratch, dw, launches);
+  return launch_conv_simt<bf16_t, CONV_WGRAD>(st, g, x, dy, (bf16_t*)nullptr, scratch, dw, (const bf16_t*)nullptr, (const bf16_t*)nullptr, launches);
 }
 
 }  // namespace fdg

@@ -21,8 +21,9 @@
 //   in tensor memory over all its tiles, writes them once, and a fixed-order pass adds the CTAs'
 //   partials, so the result does not depend on scheduling.
 //
-// Roles by warp: 0 = TMA producer, 1 = MMA issuer (one elected lane), 2..5 = epilogue (32
-// tensor-memory lanes each).  Every wait is bounded; on time-out the CTA raises an error word.
+// Roles by warp: 0 = TMA producer, 1..2 = MMA issuers (one elected lane each, alternate 128-row
+// tiles), 3..14 = epilogue (three groups of four warps, 32 tensor-memory lanes per warp).  Every
+// wait is bounded; on time-out the CTA raises an error word.
 #pragma once
 #include "conv_tc.cuh"
 

@@ -570,4 +570,127 @@ __global__ void cast_kernel(const float* __restrict__ in, T* __restrict__ out, s
     out[i] = from_f<T>(in[i]);
 }
 
+// ---------------------------------------------------------- host launchers ---
+// Shared by the module runtime and the operator-level entry points, so that both issue the same
+// kernels in the same launch shapes.
+inline int ew_blocks(size_t nvec) {
+  size_t b = (nvec + 255) / 256;
+  return (int)(b < 1 ? 1 : (b > 148 * 8 ? 148 * 8 : b));
+}
+template <typename T> constexpr int full_vec() { return 16 / sizeof(T); }
+
+// Floats of scratch a channel reduction over C channels may write (per-block partial sums).
+inline size_t red_scratch_floats(int C) { return (size_t)kRedMaxBlocks * kRedMaxSums * C; }
+
+// stats[0..C) = mean, stats[C..2C) = 1/sqrt(var + eps) of x [rows][C]; `counter` is a zeroed ticket word
+// (the kernel leaves it zero again).
+template <typename T>
+inline cudaError_t launch_bn_stats(cudaStream_t st, const T* x, size_t rows, int C, float eps, float* stats,
+                                   float* scratch, unsigned int* counter) {
+  constexpr int V = full_vec<T>();
+  if (C % V == 0) {
+    RedGeom g = red_geom((int)rows, C, V);
+    bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * C * 4, st>>>(x, g, eps, stats, scratch, counter);
+  } else {
+    RedGeom g = red_geom((int)rows, C, 1);
+    bn_stats_kernel<T, 1><<<g.blocks, kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * C * 4, st>>>(x, g, eps, stats, scratch, counter);
+  }
+  return cudaGetLastError();
+}
+
+// y = [relu](BN(x) + residual).  `partial` != null: the statistics are not in `stats` yet; a convolution left
+// `nparts` rows of per-CTA sums (sum x, sum x^2) there, which every block adds up first (block 0 saves the
+// result to `stats`); `block_cap` then bounds the grid, since every block repeats that addition.
+template <typename T>
+inline cudaError_t launch_bn_apply(cudaStream_t st, const T* x, float* stats, const float* gamma, const float* beta,
+                                   const T* res, const float* res_stats, const float* res_gamma, const float* res_beta,
+                                   bool relu, T* y, size_t rows, int C, float eps, const float* partial, int nparts,
+                                   int block_cap) {
+  constexpr int V = full_vec<T>();
+  const size_t n = rows * C;
+  PartialSums ps{};
+  if (partial && nparts > 0) {
+    if (2 * C > kEwThreads) return cudaErrorInvalidValue;
+    ps.partial = partial; ps.nparts = nparts; ps.kind = 1; ps.inv_count = 1.f / (float)rows; ps.eps = eps;
+    ps.save0 = stats; ps.save1 = stats + C;
+  }
+  if (C % V == 0) {
+    int blocks = ew_blocks(n / V);
+    if (ps.partial && block_cap > 0 && blocks > block_cap) blocks = block_cap;
+    bn_apply_kernel<T, V><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
+  } else {
+    bn_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
+  }
+  return cudaGetLastError();
+}
+
+// First half of the batch-norm backward: the per-channel sums of dz = dy*[mask>0] (and dz*xhat, dz*xhat2),
+// which are also the parameter gradients; totals to `sums` [3*C].
+template <typename T>
+inline cudaError_t launch_bn_bwd_reduce(cudaStream_t st, const T* dy, const T* mask, const T* x, const float* stats,
+                                        const T* x2, const float* stats2, size_t rows, int C, float* sums,
+                                        float* dgamma, float* dbeta, float* dgamma2, float* dbeta2, float* scratch,
+                                        unsigned int* counter) {
+  constexpr int V = full_vec<T>();
+  const bool two = x2 != nullptr, vec = C % V == 0;
+  const int ns = two ? 3 : 2;
+  RedGeom g = red_geom((int)rows, C, vec ? V : 1);
+  const size_t smem = (size_t)(g.rp > 2 ? g.rp : 2) * ns * C * 4;
+#define FDG_RED(VV, NS) bn_bwd_reduce_kernel<T, VV, NS><<<g.blocks, kRedThreads, smem, st>>>( \
+      dy, mask, x, stats, x2, stats2, g, sums, dgamma, dbeta, dgamma2, dbeta2, scratch, counter)
+  if (vec) { if (two) FDG_RED(V, 3); else FDG_RED(V, 2); }
+  else     { if (two) FDG_RED(1, 3); else FDG_RED(1, 2); }
+#undef FDG_RED
+  return cudaGetLastError();
+}
+
+// Second half: dx = gamma*invstd*(dz - s0/M - xhat*s1/M) [+ res] (and dx2 for the second normalised tensor).
+// The sums come from `sums`, or, when `partial` != null, from `nparts` rows of per-CTA sums (sum dz, sum dz*xhat)
+// left by the data-gradient kernel that produced dy (block 0 then also writes dbeta / dgamma).
+template <typename T>
+inline cudaError_t launch_bn_bwd_apply(cudaStream_t st, const T* dy, const T* mask, const T* x, const float* stats,
+                                       const float* gamma, const float* sums, const T* x2, const float* stats2,
+                                       const float* gamma2, const T* res, T* dx, T* dx2, size_t rows, int C,
+                                       const float* partial, int nparts, float* dgamma, float* dbeta, int block_cap) {
+  constexpr int V = full_vec<T>();
+  const size_t n = rows * C;
+  const float inv_m = 1.f / (float)rows;
+  PartialSums ps{};
+  if (partial && nparts > 0) {
+    if (2 * C > kEwThreads) return cudaErrorInvalidValue;
+    ps.partial = partial; ps.nparts = nparts; ps.kind = 2; ps.save0 = dbeta; ps.save1 = dgamma;
+  }
+  if (C % V == 0) {
+    int blocks = ew_blocks(n / V);
+    if (ps.partial && block_cap > 0 && blocks > block_cap) blocks = block_cap;
+    bn_bwd_apply_kernel<T, V><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n / V, C, inv_m, ps);
+  } else {
+    bn_bwd_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n, C, inv_m, ps);
+  }
+  return cudaGetLastError();
+}
+
+template <typename T>
+inline cudaError_t launch_scale(cudaStream_t st, const T* in, T* out, float s, size_t n) {
+  constexpr int V = full_vec<T>();
+  if (n % V == 0) scale_kernel<T, V><<<ew_blocks(n / V), 256, 0, st>>>(in, out, s, n / V);
+  else scale_kernel<T, 1><<<ew_blocks(n), 256, 0, st>>>(in, out, s, n);
+  return cudaGetLastError();
+}
+
+inline cudaError_t launch_sgd(cudaStream_t st, float* theta, float* v, const float* g, float* next32,
+                              __nv_bfloat16* next16, size_t n, float lr, const float* lr_dev, float mu, float wd) {
+  size_t b = (n / 4 + 255) / 256;
+  const int blocks = (int)(b < 1 ? 1 : (b > 148 * 8 ? 148 * 8 : b));
+  sgd_kernel<<<blocks, 256, 0, st>>>(theta, v, g, next32, next16, n, lr, lr_dev, mu, wd);
+  return cudaGetLastError();
+}
+
+template <typename T>
+inline cudaError_t launch_ingest(cudaStream_t st, const float* img, T* out, size_t rows, int c_in, int c_out,
+                                 const int32_t* labels_in, int32_t* labels_out, int batch) {
+  ingest_kernel<T><<<ew_blocks(rows * c_out), 256, 0, st>>>(img, out, rows, c_in, c_out, labels_in, labels_out, batch);
+  return cudaGetLastError();
+}
+
 }  // namespace fdg

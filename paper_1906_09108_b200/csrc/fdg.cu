@@ -46,6 +46,9 @@ static const char* const kClassNames[KC_COUNT] = {"conv_fprop", "conv_dgrad", "c
 constexpr size_t kProfMaxPairs = 1 << 16;
 struct ProfRec { int cls; double bytes, flops; };
 
+// One gradient tensor of a module's backward pass that fdg_capture_begin can keep a copy of.
+struct CaptureEntry { int unit, which, ch; size_t off, elems; };
+
 struct Unit {
   UnitType type;
   int index;                 // 0 stem, b block, -1 head
@@ -106,6 +109,11 @@ struct Module {
   cudaStream_t stream2 = nullptr;          // side stream: weight gradients run beside the data-gradient chain
   cudaEvent_t ev_fork2 = nullptr, ev_join2 = nullptr, ev_buf[4] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t ev_act[kEventRing], ev_grad[kEventRing];
+  // gradient capture (fdg_capture_begin): where each gradient tensor of a backward pass is copied to
+  std::vector<CaptureEntry> cap_table;
+  size_t cap_elems = 0;
+  char* cap_buf = nullptr;
+  int64_t cap_batch = -1;
 };
 
 }  // namespace fdg
@@ -125,7 +133,7 @@ struct fdg_ctx {
   cudaEvent_t ev_join;
   int32_t* labels = nullptr;          // ring of label_ring batches
   int label_ring = 0;
-  int* flags = nullptr;               // [0] non-finite loss, [1] label out of range
+  int* flags = nullptr;               // [0] non-finite loss, [1] label out of range, [2] a tensor-core kernel's wait ran out
   float* staging = nullptr;           // fp32 staging for getters
   float* host_images = nullptr;       // device staging of fdg_step_host
   int32_t* host_labels = nullptr;
@@ -344,7 +352,7 @@ static void plan_modules(fdg_ctx* c) {
       for (const Unit& u : m.units) {
         if ((u.type != U_BASIC && u.type != U_PREACT) || u.stride != 2) continue;
         ConvGeom g1{a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 3, u.stride, 1};
-        if (halo_s2_dgrad_eligible(g1) || halo_s2_wgrad_eligible(g1) || tc_s2_dgrad_eligible(g1))
+        if (s2_uses_spread_dy(g1))
           m.up_elems = std::max(m.up_elems, B * u.H * u.W * u.co);
       }
     if (c->bf16_mode) {
@@ -366,6 +374,24 @@ static void plan_modules(fdg_ctx* c) {
       m.flip_elems = fe;
     }
     m.slot_elems = te; m.slot_floats = tf; m.max_act = maxa; m.scratch_floats = scr; m.wscratch_floats = wscr;
+    {   // the gradient tensors a capture keeps (fdg_capture_begin), one region each
+      size_t ce = 0;
+      auto cap = [&](int ui, int which, size_t e, int ch) { m.cap_table.push_back(CaptureEntry{ui, which, ch, ce, e}); ce += align_up(e, 128); };
+      for (int ui = 0; ui < (int)m.units.size(); ++ui) {
+        const Unit& u = m.units[ui];
+        const size_t in_e = B * u.H * u.W * u.ci, out_e = B * u.P * u.Q * u.co;
+        if (u.type == U_STEM) { cap(ui, 0, out_e, u.co); if (u.bn) cap(ui, 3, out_e, u.co); }
+        if (u.type == U_BASIC) {
+          cap(ui, 0, out_e, u.co); cap(ui, 1, out_e, u.co); cap(ui, 2, out_e, u.co); cap(ui, 3, out_e, u.co); cap(ui, 4, in_e, u.ci);
+          if (u.proj) cap(ui, 5, out_e, u.co);
+        }
+        if (u.type == U_PREACT) {
+          cap(ui, 0, out_e, u.co); cap(ui, 1, out_e, u.co); cap(ui, 2, out_e, u.co); cap(ui, 3, in_e, u.ci); cap(ui, 4, in_e, u.ci);
+          if (u.proj) cap(ui, 5, in_e, u.ci);
+        }
+      }
+      m.cap_elems = ce;
+    }
     const Unit& last = m.units.back();
     if (kp < K) { m.out_elems = B * last.P * last.Q * last.co; m.out_c = last.co; }
     m.slot_version.assign(m.D, -1);
@@ -452,25 +478,11 @@ struct Launch {
   void note(cudaError_t e) { if (err == cudaSuccess) err = e; end_events(); }
 };
 
-static int ew_blocks(size_t nvec) {
-  size_t b = (nvec + 255) / 256;
-  return (int)std::min<size_t>(std::max<size_t>(b, 1), 148 * 8);
-}
-
-template <typename T> constexpr int full_vec() { return 16 / sizeof(T); }
-
 template <typename T>
 static void bn_stats(Launch& L, Module& m, const T* x, size_t rows, int C, float eps, float* stats) {
-  constexpr int V = full_vec<T>();
   L.begin(KC_BN_STATS, (double)rows * C * sizeof(T), 3.0 * rows * C);
-  if (C % V == 0) {
-    RedGeom g = red_geom((int)rows, C, V);
-    bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)std::max(g.rp, 2) * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
-  } else {
-    RedGeom g = red_geom((int)rows, C, 1);
-    bn_stats_kernel<T, 1><<<g.blocks, kRedThreads, (size_t)std::max(g.rp, 2) * 2 * C * 4, L.st>>>(x, g, eps, stats, m.scratch, m.counter);
-  }
-  L.check();
+  L.note(launch_bn_stats<T>(L.st, x, rows, C, eps, stats, m.scratch, m.counter));
+  ++L.c->launches;
 }
 
 // `nparts` > 0: the statistics are not in `stats` yet; the convolution that produced x left nparts
@@ -479,22 +491,11 @@ template <typename T>
 static void bn_apply(Launch& L, Module& m, const T* x, float* stats, const float* gamma, const float* beta, const T* res,
                      const float* res_stats, const float* res_gamma, const float* res_beta, bool relu, T* y,
                      size_t rows, int C, int nparts = 0) {
-  constexpr int V = full_vec<T>();
   const size_t n = rows * C;
-  PartialSums ps{};
-  if (nparts > 0) {
-    ps.partial = m.red_partial; ps.nparts = nparts; ps.kind = 1; ps.inv_count = 1.f / (float)rows; ps.eps = L.c->arch.bn_eps;
-    ps.save0 = stats; ps.save1 = stats + C;
-  }
   L.begin(KC_BN_APPLY, (double)n * sizeof(T) * (res ? 3 : 2), 6.0 * n);
-  if (C % V == 0) {
-    int blocks = ew_blocks(n / V);
-    if (nparts > 0) blocks = std::min(blocks, L.c->ew_block_cap);   // every block re-adds the partials: keep them few
-    bn_apply_kernel<T, V><<<blocks, kEwThreads, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
-  } else {
-    bn_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, L.st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
-  }
-  L.check();
+  L.note(launch_bn_apply<T>(L.st, x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, rows, C,
+                            L.c->arch.bn_eps, nparts > 0 ? m.red_partial : nullptr, nparts, L.c->ew_block_cap));
+  ++L.c->launches;
 }
 
 // Backward of y = BN(x) (and optionally y2 = BN2(x2) sharing the same upstream gradient):
@@ -504,46 +505,26 @@ static void bn_backward(Launch& L, Module& m, const T* dy, const T* mask, const 
                         const float* gamma, float* dgamma, float* dbeta, const T* x2, const float* stats2,
                         const float* gamma2, float* dgamma2, float* dbeta2, const T* res, T* dx, T* dx2,
                         size_t rows, int C, int nparts = 0) {
-  constexpr int V = full_vec<T>();
   const bool two = x2 != nullptr;
-  const int ns = two ? 3 : 2;
-  const bool vec = C % V == 0;
-  const bool sums_ready = nparts > 0;
-  PartialSums ps{};
-  if (sums_ready) {       // the kernel that produced dy left nparts rows of partial sums in m.red_partial
-    ps.partial = m.red_partial; ps.nparts = nparts; ps.kind = 2; ps.save0 = dbeta; ps.save1 = dgamma;
-  }
+  const bool sums_ready = nparts > 0;    // the kernel that produced dy left nparts rows of partial sums in m.red_partial
   if (!sums_ready) {
-    RedGeom g = red_geom((int)rows, C, vec ? V : 1);
-    const size_t smem = (size_t)std::max(g.rp, 2) * ns * C * 4;
-#define FDG_RED(VV, NS) bn_bwd_reduce_kernel<T, VV, NS><<<g.blocks, kRedThreads, smem, L.st>>>( \
-      dy, mask, x, stats, x2, stats2, g, m.bnsums, dgamma, dbeta, dgamma2, dbeta2, m.scratch, m.counter)
     L.begin(KC_BN_BWD_REDUCE, (double)rows * C * sizeof(T) * (2 + (mask ? 1 : 0) + (two ? 1 : 0)), 8.0 * rows * C);
-    if (vec) { if (two) FDG_RED(V, 3); else FDG_RED(V, 2); }
-    else     { if (two) FDG_RED(1, 3); else FDG_RED(1, 2); }
-#undef FDG_RED
-    L.check();
+    L.note(launch_bn_bwd_reduce<T>(L.st, dy, mask, x, stats, x2, stats2, rows, C, m.bnsums, dgamma, dbeta, dgamma2, dbeta2,
+                                   m.scratch, m.counter));
+    ++L.c->launches;
   }
   const size_t n = rows * C;
-  const float inv_m = 1.f / (float)rows;
   L.begin(KC_BN_BWD_APPLY, (double)n * sizeof(T) * (3 + (mask ? 1 : 0) + (two ? 2 : 0) + (res ? 1 : 0)), 10.0 * n);
-  if (vec) {
-    int blocks = ew_blocks(n / V);
-    if (sums_ready) blocks = std::min(blocks, L.c->ew_block_cap);
-    bn_bwd_apply_kernel<T, V><<<blocks, kEwThreads, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n / V, C, inv_m, ps);
-  } else {
-    bn_bwd_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, L.st>>>(dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n, C, inv_m, ps);
-  }
-  L.check();
+  L.note(launch_bn_bwd_apply<T>(L.st, dy, mask, x, stats, gamma, m.bnsums, x2, stats2, gamma2, res, dx, dx2, rows, C,
+                                sums_ready ? m.red_partial : nullptr, nparts, dgamma, dbeta, L.c->ew_block_cap));
+  ++L.c->launches;
 }
 
 template <typename T>
 static void scale_tensor(Launch& L, const T* in, T* out, float s, size_t n) {
-  constexpr int V = full_vec<T>();
   L.begin(KC_SHRINK, 2.0 * n * sizeof(T), (double)n);
-  if (n % V == 0) scale_kernel<T, V><<<ew_blocks(n / V), 256, 0, L.st>>>(in, out, s, n / V);
-  else scale_kernel<T, 1><<<ew_blocks(n), 256, 0, L.st>>>(in, out, s, n);
-  L.check();
+  L.note(launch_scale<T>(L.st, in, out, s, n));
+  ++L.c->launches;
 }
 
 template <typename T> static const T* weights_of(const Module& m, int vslot);
@@ -566,33 +547,15 @@ template <typename T>
 static int conv_fprop(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* w, T* y, const T* res,
                       bool want_stats = false) {
   L.begin(KC_CONV_FPROP, (in_elems(g) + w_elems(g) + out_elems(g) * (res ? 2 : 1)) * sizeof(T), conv_flops(g));
+  int nparts = 0;
   if constexpr (std::is_same<T, bf16>::value) {
-    if (halo_fprop_eligible(g)) {
-      ++L.c->launches;
-      const bool fuse = want_stats && halo_reduce_ok(g.Co);
-      halo::EpiReduce r{};
-      int ctas = 0;
-      if (fuse) { r.mode = 1; r.partial = m.red_partial; }
-      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, fuse ? &r : nullptr, &ctas));
-      return fuse ? ctas : 0;
-    }
-    if (halo_s2_fprop_eligible(g)) {      // the stride-1 convolution, stored at the even pixels only
-      ++L.c->launches;
-      const bool fuse = want_stats && halo_reduce_ok(g.Co);
-      halo::EpiReduce r{};
-      int ctas = 0;
-      if (fuse) { r.mode = 1; r.partial = m.red_partial; }
-      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, fuse ? &r : nullptr, &ctas, 2));
-      return fuse ? ctas : 0;
-    }
-    if (tc_eligible(g) || tc_s2_fprop_eligible(g)) {
-      ++L.c->launches;
-      L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, L.c->tc_error, g.stride));
-      return 0;
-    }
+    halo::EpiReduce r{};
+    r.mode = 1; r.partial = m.red_partial;
+    L.note(bf16_conv_fprop(L.st, &L.c->tmaps, g, x, w, y, res, want_stats ? &r : nullptr, &nparts, L.c->tc_error, &L.c->launches));
+  } else {
+    L.note(launch_conv_simt<T, CONV_FPROP>(L.st, g, x, w, y, nullptr, nullptr, res, (const T*)nullptr, &L.c->launches));
   }
-  L.note(launch_conv_simt<T, CONV_FPROP>(L.st, g, x, w, y, nullptr, nullptr, res, (const T*)nullptr, &L.c->launches));
-  return 0;
+  return nparts;
 }
 // `wflip` is the flipped/transposed weight copy (bf16 mode, tensor-core eligible shapes) or null.
 // The batch-norm backward that will consume dx as its upstream gradient: dz = dx * [mask > 0],
@@ -604,64 +567,25 @@ template <typename T>
 static int conv_dgrad(Launch& L, Module& m, const ConvGeom& g, const T* dy, const T* w, const T* wflip, T* dx,
                        const T* res, const T* mask, const NextBnBwd<T>* next = nullptr, const T* dy_up = nullptr) {
   L.begin(KC_CONV_DGRAD, (out_elems(g) + w_elems(g) + in_elems(g) * (1 + (res ? 1 : 0) + (mask ? 1 : 0) + (next ? 2 : 0))) * sizeof(T), conv_flops(g));
+  int nparts = 0;
   if constexpr (std::is_same<T, bf16>::value) {
-    if (wflip && halo_dgrad_eligible(g)) {
-      ++L.c->launches;
-      const bool fuse = next && halo_reduce_ok(g.Ci);
-      halo::EpiReduce r{};
-      int ctas = 0;
-      if (fuse) { r.mode = 2; r.mask = next->mask; r.xprev = next->x; r.pstats = next->stats; r.partial = m.red_partial; }
-      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error, fuse ? &r : nullptr, &ctas));
-      return fuse ? ctas : 0;
-    }
-    if (wflip && dy_up && halo_s2_dgrad_eligible(g)) {      // stride 2: the stride-1 data gradient of the spread-out dy
-      ++L.c->launches;
-      const bool fuse = next && halo_reduce_ok(g.Ci);
-      halo::EpiReduce r{};
-      int ctas = 0;
-      if (fuse) { r.mode = 2; r.mask = next->mask; r.xprev = next->x; r.pstats = next->stats; r.partial = m.red_partial; }
-      L.note(run_conv_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy_up, wflip, dx, res, mask, L.c->tc_error, fuse ? &r : nullptr, &ctas));
-      return fuse ? ctas : 0;
-    }
-    if (wflip && tc_eligible(g)) {
-      ++L.c->launches;
-      L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy, wflip, dx, res, mask, L.c->tc_error));
-      return 0;
-    }
-    if (wflip && dy_up && tc_s2_dgrad_eligible(g)) {
-      ++L.c->launches;
-      L.note(run_conv_tc(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Co, g.Ci, dy_up, wflip, dx, res, mask, L.c->tc_error));
-      return 0;
-    }
+    halo::EpiReduce r{};
+    if (next) { r.mode = 2; r.mask = next->mask; r.xprev = next->x; r.pstats = next->stats; r.partial = m.red_partial; }
+    L.note(bf16_conv_dgrad(L.st, &L.c->tmaps, g, dy, w, wflip, dy_up, dx, res, mask, next ? &r : nullptr, &nparts, L.c->tc_error, &L.c->launches));
+  } else {
+    L.note(launch_conv_simt<T, CONV_DGRAD>(L.st, g, dy, w, dx, nullptr, nullptr, res, mask, &L.c->launches));
   }
-  L.note(launch_conv_simt<T, CONV_DGRAD>(L.st, g, dy, w, dx, nullptr, nullptr, res, mask, &L.c->launches));
-  return 0;
+  return nparts;
 }
 template <typename T>
 static void conv_wgrad(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* dy, float* dw, const T* dy_up = nullptr) {
   L.begin(KC_CONV_WGRAD, (in_elems(g) + out_elems(g)) * sizeof(T) + w_elems(g) * 4, conv_flops(g));
-  if constexpr (std::is_same<T, bf16>::value) {
-    if (dy_up && halo_s2_wgrad_eligible(g)) {                // stride 2: the stride-1 weight gradient with the spread-out dy
-      L.c->launches += 2;
-      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy_up, dw, m.wscratch, L.c->tc_error, L.st == m.stream2));
-      return;
-    }
-    if (halo_wgrad_eligible(g)) {
-      L.c->launches += 2;
-      L.note(run_wgrad_halo(L.st, &L.c->tmaps, g.N, g.H, g.W, g.Ci, g.Co, x, dy, dw, m.wscratch, L.c->tc_error, L.st == m.stream2));
-      return;
-    }
-  }
-  // bf16 storage only: the fp32 mode keeps one summation scheme for all its weight gradients
-  if (std::is_same<T, bf16>::value && small_wgrad_eligible(g)) {
-    L.note(launch_small_wgrad<T>(L.st, g, x, dy, m.wscratch, dw, &L.c->launches));
-    return;
-  }
-  if (std::is_same<T, bf16>::value && proj_wgrad_eligible(g)) {
-    L.note(launch_proj_wgrad<T>(L.st, g, x, dy, m.wscratch, dw, &L.c->launches));
-    return;
-  }
-  L.note(launch_conv_simt<T, CONV_WGRAD>(L.st, g, x, dy, (T*)nullptr, m.wscratch, dw, (const T*)nullptr, (const T*)nullptr, &L.c->launches));
+  // the tensor-core and small-shape kernels serve bf16 storage only: the fp32 mode keeps one summation
+  // scheme for all its weight gradients
+  if constexpr (std::is_same<T, bf16>::value)
+    L.note(bf16_conv_wgrad(L.st, &L.c->tmaps, g, x, dy, dy_up, dw, m.wscratch, L.c->tc_error, L.st == m.stream2, &L.c->launches));
+  else
+    L.note(launch_conv_simt<T, CONV_WGRAD>(L.st, g, x, dy, (T*)nullptr, m.wscratch, dw, (const T*)nullptr, (const T*)nullptr, &L.c->launches));
 }
 
 template <typename T> static const T* flipped_of(const Module& m, int vslot, long long off);
@@ -675,12 +599,10 @@ template <> const bf16* flipped_of<bf16>(const Module& m, int vslot, long long o
 template <typename T>
 static const T* upsample_dy(Launch& L, Module& m, const ConvGeom& g, const T* dy) {
   if constexpr (std::is_same<T, bf16>::value) {
-    if (!m.up || !(halo_s2_dgrad_eligible(g) || halo_s2_wgrad_eligible(g) || tc_s2_dgrad_eligible(g)) || g.Co % 8) return nullptr;
+    if (!m.up || !s2_uses_spread_dy(g)) return nullptr;
     T* up = reinterpret_cast<T*>(m.up);
-    const size_t nvec = (size_t)g.N * g.H * g.W * g.Co / 8;
-    L.begin(KC_CONV_DGRAD, (double)nvec * 16 * 1.25, 0.0);
-    upsample2_kernel<T, 8><<<ew_blocks(nvec), 256, 0, L.st>>>(dy, up, nvec, g.P, g.Q, g.Co);
-    L.check();
+    L.begin(KC_CONV_DGRAD, (double)g.N * g.H * g.W * g.Co * 2 * 1.25, 0.0);
+    L.note(bf16_spread_dy(L.st, g, dy, up, &L.c->launches));
     return up;
   }
   return nullptr;
@@ -828,6 +750,16 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
   };
   auto side_done = [&](int b) { if (forked) { LS.note(cudaEventRecord(m.ev_buf[b], LS.st)); buf_read[b] = true; } };
   auto wait_buf = [&](int b) { if (forked && buf_read[b]) L.note(cudaStreamWaitEvent(L.st, m.ev_buf[b], 0)); };
+  // While a capture is on (fdg_capture_begin), every gradient tensor of the pass is copied aside in stream order.
+  auto keep = [&](int ui, int which, const T* src) {
+    if (!m.cap_buf || !src) return;
+    for (const CaptureEntry& ce : m.cap_table)
+      if (ce.unit == ui && ce.which == which) {
+        L.note(cudaMemcpyAsync(m.cap_buf + ce.off * sizeof(T), src, ce.elems * sizeof(T), cudaMemcpyDeviceToDevice, L.st));
+        return;
+      }
+  };
+  if (m.cap_buf) m.cap_batch = tau;
   T* dy = gin;
   int dy_sum_parts = 0;            // > 0: the kernel that produced dy left that many rows of partial sums for the
                                    // first batch-norm backward it meets
@@ -852,11 +784,13 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
       case U_STEM: {
         ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
         const T* dc = dy;
+        keep(i, 0, dy);
         if (u.bn) {
           wait_buf(0);
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
                          nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sum_parts);
           dc = T1;
+          keep(i, 3, T1);
         }
         fork();
         conv_wgrad<T>(LS, m, g, x, dc, m.grad + u.w1);
@@ -866,6 +800,7 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
       case U_BASIC: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
+        keep(i, 0, dy);
         wait_buf(0);
         if (u.proj) {
           wait_buf(2);
@@ -875,14 +810,18 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
           bn_backward<T>(L, m, dy, S + u.t_y, S + u.t_c, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
                          nullptr, nullptr, nullptr, nullptr, nullptr, T1, nullptr, rows_out, u.co, dy_sum_parts);
         }
+        keep(i, 1, T1);
+        if (u.proj) keep(i, 5, T2);
         fork();
         conv_wgrad<T>(LS, m, g2, S + u.t_b, T1, m.grad + u.w2);                                          // side
         side_done(0);
         const NextBnBwd<T> bn1{S + u.t_b, S + u.t_a, F + u.st1};
         const int bn1_parts = conv_dgrad<T>(L, m, g2, T1, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T3, nullptr, nullptr, &bn1);   // da1
+        keep(i, 2, T3);
         wait_buf(1);
         bn_backward<T>(L, m, T3, S + u.t_b, S + u.t_a, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr,
                        nullptr, nullptr, nullptr, nullptr, nullptr, T4, nullptr, rows_out, u.co, bn1_parts);      // dc1
+        keep(i, 3, T4);
         const T* up = nullptr;
         if (u.stride == 2) { wait_buf(3); up = upsample_dy<T>(L, m, g1, T4); }
         fork();
@@ -901,27 +840,34 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
         } else if (need_dx) {
           out_sum_parts = conv_dgrad<T>(L, m, g1, T4, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y, next);
         }
+        if (need_dx) keep(i, 4, gout);
         break;
       }
       case U_PREACT: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
+        keep(i, 0, dy);
         conv_wgrad<T>(L, m, g2, S + u.t_c, dy, m.grad + u.w2);
         conv_dgrad<T>(L, m, g2, dy, wt + u.w2, flipped_of<T>(m, vslot, u.f2), T1, nullptr, nullptr);   // da2
+        keep(i, 1, T1);
         bn_backward<T>(L, m, T1, S + u.t_c, S + u.t_b, F + u.st2, wf + u.g2, m.grad + u.g2, m.grad + u.b2, nullptr,
                        nullptr, nullptr, nullptr, nullptr, nullptr, T2, nullptr, rows_out, u.co);      // dc1
+        keep(i, 2, T2);
         const T* up = u.stride == 2 ? upsample_dy<T>(L, m, g1, T2) : nullptr;
         conv_wgrad<T>(L, m, g1, S + u.t_a, T2, m.grad + u.w1, up);
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_wgrad<T>(L, m, gs, S + u.t_a, dy, m.grad + u.ws);
           conv_dgrad<T>(L, m, gs, dy, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
+          keep(i, 5, T3);
           conv_dgrad<T>(L, m, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, T3, nullptr, nullptr, up);   // do
         } else {
           conv_dgrad<T>(L, m, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, nullptr, nullptr);
         }
+        keep(i, 3, T1);
         bn_backward<T>(L, m, T1, S + u.t_a, x, F + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr, nullptr,
                        nullptr, nullptr, nullptr, u.proj ? nullptr : dy, gout, nullptr, rows_in, u.ci);
+        keep(i, 4, gout);
         break;
       }
       default: break;
@@ -940,11 +886,10 @@ static void update_module(fdg_ctx* c, Module& m, Launch& L, int next_vslot) {
   const size_t n = m.n_params;
   float* next32 = m.wver + (size_t)next_vslot * align_up(n, 64);
   bf16* next16 = c->bf16_mode ? m.wver16 + (size_t)next_vslot * align_up(n, 64) : nullptr;
-  int blocks = (int)std::min<size_t>(std::max<size_t>((n / 4 + 255) / 256, 1), 148 * 8);
   L.begin(KC_SGD, (double)n * (24 + (next16 ? 2 : 0)), 6.0 * n);
-  sgd_kernel<<<blocks, 256, 0, L.st>>>(m.theta, m.mom, m.grad, next32, next16, n, c->lr,
-                                       c->graph_mode_entered ? c->lr_dev : nullptr, c->cfg.momentum, c->cfg.weight_decay);
-  L.check();
+  L.note(launch_sgd(L.st, m.theta, m.mom, m.grad, next32, next16, n, c->lr, c->graph_mode_entered ? c->lr_dev : nullptr,
+                    c->cfg.momentum, c->cfg.weight_decay));
+  ++c->launches;
   if (m.flip_table_dev) {
     L.begin(KC_SGD, 4.0 * m.flip_elems, 0.0);
     tc::wflip_kernel<<<dim3(8, (unsigned)m.flip_table.size()), 256, 0, L.st>>>(next16, m.wflip16 + (size_t)next_vslot * m.flip_elems, m.flip_table_dev);
@@ -1411,14 +1356,13 @@ fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, cons
     const size_t rows = (size_t)c->arch.batch * c->arch.in_h * c->arch.in_w;
     int32_t* lab = c->labels + (size_t)(t % c->label_ring) * c->arch.batch;
     const size_t slot_off = (size_t)(t % m1.Din) * align_up(m1.in_elems, 128);
-    const int blocks = ew_blocks(rows * m1.in_c);
     Launch L{c, cs};
     L.begin(KC_INGEST, (double)rows * (c->arch.in_c * 4 + m1.in_c * c->esize), 0.0);
     if (c->bf16_mode)
-      ingest_kernel<bf16><<<blocks, 256, 0, cs>>>(images_dev, reinterpret_cast<bf16*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch);
+      L.note(launch_ingest<bf16>(cs, images_dev, reinterpret_cast<bf16*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch));
     else
-      ingest_kernel<float><<<blocks, 256, 0, cs>>>(images_dev, reinterpret_cast<float*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch);
-    L.check();
+      L.note(launch_ingest<float>(cs, images_dev, reinterpret_cast<float*>(m1.in_ring) + slot_off, rows, c->arch.in_c, m1.in_c, labels_dev, lab, c->arch.batch));
+    ++c->launches;
     e = L.err;
     if (e == cudaSuccess && !serial && !graph) e = cudaEventRecord(c->ev_in[t % kEventRing], cs);
     if (e != cudaSuccess) return cuda_fail(c, e, "ingest");
@@ -1472,6 +1416,16 @@ fdg_status fdg_sync(fdg_ctx* c, fdg_stream stream) {
   return c->latched;
 }
 
+fdg_status fdg_debug_raise_flag(fdg_ctx* c, int which) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (which < 0 || which > 2) return fail(c, FDG_ERR_INVALID_ARG, "no such status word");
+  cudaError_t e = drain(c);
+  const int one = 1;
+  if (e == cudaSuccess) e = cudaMemcpy(c->flags + which, &one, sizeof(int), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "raising a status word");
+}
+
 static fdg_status export_tensor(fdg_ctx* c, const void* src, size_t rows, int c_store, int c_logical, float* dst, size_t n) {
   if (n != rows * (size_t)c_logical) return fail(c, FDG_ERR_INVALID_ARG, "element count does not match fdg_boundary_elems");
   cudaError_t e = drain(c);
@@ -1517,8 +1471,8 @@ fdg_status fdg_get_input_grad(fdg_ctx* c, int module, float* dst, size_t n, int6
   return export_tensor(c, src, (size_t)c->arch.batch * m.in_h * m.in_w, m.in_c, m.in_c_logical, dst, n);
 }
 
-fdg_status fdg_get_saved_tensor(fdg_ctx* c, int module, int unit, int which, float* dst, size_t n, size_t* out_elems,
-                                int64_t* batch_index) {
+fdg_status fdg_get_saved_tensor_of(fdg_ctx* c, int module, int unit, int which, int64_t batch, float* dst, size_t n,
+                                   size_t* out_elems, int64_t* batch_index) {
   FDG_MODULE_OR_FAIL(c, module);
   Module& m = c->mods[module - 1];
   if (unit < 0 || unit >= (int)m.units.size() || m.units[unit].type == U_HEAD)
@@ -1548,13 +1502,65 @@ fdg_status fdg_get_saved_tensor(fdg_ctx* c, int module, int unit, int which, flo
   if (out_elems) *out_elems = elems;
   if (!dst) return FDG_OK;
   if (!batch_index) return FDG_ERR_INVALID_ARG;
-  // most recent forward = the slot with the largest batch index
+  // batch < 0: the most recent forward = the slot with the largest batch index
   int slot = -1;
-  for (int i = 0; i < m.D; ++i) if (m.slot_batch[i] >= 0 && (slot < 0 || m.slot_batch[i] > m.slot_batch[slot])) slot = i;
+  for (int i = 0; i < m.D; ++i) {
+    if (m.slot_batch[i] < 0) continue;
+    if (batch >= 0 ? m.slot_batch[i] == batch : (slot < 0 || m.slot_batch[i] > m.slot_batch[slot])) slot = i;
+  }
   *batch_index = slot < 0 ? -1 : m.slot_batch[slot];
   if (slot < 0) return FDG_OK;
   const char* src = m.fifo + ((size_t)slot * m.slot_elems + off) * c->esize;
   return export_tensor(c, src, elems / ch, ch, ch, dst, n);
+}
+
+fdg_status fdg_get_saved_tensor(fdg_ctx* c, int module, int unit, int which, float* dst, size_t n, size_t* out_elems,
+                                int64_t* batch_index) {
+  return fdg_get_saved_tensor_of(c, module, unit, which, -1, dst, n, out_elems, batch_index);
+}
+
+fdg_status fdg_capture_bytes(const fdg_ctx* c, int module, size_t* out_bytes) {
+  FDG_MODULE_OR_FAIL(c, module);
+  if (!out_bytes) return FDG_ERR_INVALID_ARG;
+  *out_bytes = c->mods[module - 1].cap_elems * c->esize;
+  return FDG_OK;
+}
+
+fdg_status fdg_capture_begin(fdg_ctx* c, int module, void* dev_buffer, size_t bytes) {
+  FDG_MODULE_OR_FAIL(c, module);
+  if (!dev_buffer || (reinterpret_cast<uintptr_t>(dev_buffer) & 15)) return fail(c, FDG_ERR_INVALID_ARG, "capture buffer is null or not 16-byte aligned");
+  if (c->use_graphs) return fail(c, FDG_ERR_STATE, "a capture cannot be switched on and off inside recorded graphs");
+  Module& m = c->mods[module - 1];
+  if (bytes < m.cap_elems * c->esize) return fail(c, FDG_ERR_WORKSPACE_TOO_SMALL, "capture buffer smaller than fdg_capture_bytes");
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  m.cap_buf = static_cast<char*>(dev_buffer);
+  m.cap_batch = -1;
+  return FDG_OK;
+}
+
+fdg_status fdg_capture_end(fdg_ctx* c, int module) {
+  FDG_MODULE_OR_FAIL(c, module);
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  c->mods[module - 1].cap_buf = nullptr;
+  return FDG_OK;
+}
+
+fdg_status fdg_get_captured(fdg_ctx* c, int module, int unit, int which, float* dst, size_t n, size_t* out_elems,
+                            int64_t* batch_index) {
+  FDG_MODULE_OR_FAIL(c, module);
+  Module& m = c->mods[module - 1];
+  const CaptureEntry* ce = nullptr;
+  for (const CaptureEntry& x : m.cap_table) if (x.unit == unit && x.which == which) ce = &x;
+  if (!ce) return fail(c, FDG_ERR_INVALID_ARG, "this unit's backward produces no such gradient tensor");
+  if (out_elems) *out_elems = ce->elems;
+  if (!dst) return FDG_OK;
+  if (!batch_index) return FDG_ERR_INVALID_ARG;
+  if (!m.cap_buf) return fail(c, FDG_ERR_STATE, "no capture is on for this module");
+  *batch_index = m.cap_batch;
+  if (m.cap_batch < 0) return FDG_OK;
+  return export_tensor(c, m.cap_buf + ce->off * c->esize, ce->elems / ce->ch, ce->ch, ce->ch, dst, n);
 }
 
 fdg_status fdg_get_schedule_log(const fdg_ctx* c, fdg_sched_entry* dst, size_t cap, size_t* out_n) {

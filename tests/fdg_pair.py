@@ -18,8 +18,14 @@ def relfro(a, b):
 
 def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_decay=5e-4,
              order="backward_first", weight_reading="stashed", precision="fp32", serial=False, seed=0,
-             jitter=True, oracle_dtype=np.float64, check_every_step=True, graphs=False):
-    """Returns a dict of worst-case errors and the two schedule logs."""
+             jitter=True, oracle_dtype=np.float64, check_every_step=True, graphs=False, plain=None):
+    """Returns a dict of worst-case errors and the two schedule logs.
+
+    In bf16 mode every error is measured twice: against the oracle with bfloat16 storage (keys "out", "gin",
+    "loss", "grads", "params": the same tensors rounded on both sides, so every ReLU gate is decided on the
+    same values) and against the plain float64 oracle, which rounds nothing (the same keys with "_plain"):
+    the second figure includes what keeping activations, gradients and weights in bfloat16 costs.
+    `plain=False` skips the second oracle (deep networks, where it doubles a long CPU run)."""
     import torch
     from paper_1906_09108_b200 import binding as B
 
@@ -30,6 +36,9 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
     # bfloat16; the oracle then rounds the same tensors, so that both sides decide every
     # ReLU gate on the same values (everything else stays float64 in the oracle).
     orc = ofdg.FDGOracle(arch_o, cfg_o, dtype=oracle_dtype, storage="bf16" if precision == "bf16" else None)
+    if plain is None:
+        plain = precision == "bf16"
+    orc_plain = ofdg.FDGOracle(arch_o, cfg_o, dtype=oracle_dtype, storage=None) if plain else None
     g = B.FDG(B.make_arch(**arch_kw), K=K, split_after_block=tuple(splits), beta=beta, lr=lr, momentum=momentum,
               weight_decay=weight_decay,
               order=B.FDG_BACKWARD_FIRST if order == "backward_first" else B.FDG_FORWARD_FIRST,
@@ -41,9 +50,13 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
         assert spec_o == spec_g, "parameter layouts differ in module %d" % k
         p = S.init_params(seed, k, orc.param_spec(k), jitter=jitter)
         orc.set_params(k, p)
+        if orc_plain is not None:
+            orc_plain.set_params(k, p)
         g.set_params(k, p)
     a = arch_o
     res = dict(out=0.0, gin=0.0, loss=0.0, grads=0.0, steps=steps)
+    if orc_plain is not None:
+        res.update(out_plain=0.0, gin_plain=0.0, loss_plain=0.0, grads_plain=0.0)
     res["grads_by_step"] = []          # (t, k, error): where a failure started, for the assertion message
     res["worst_tensors"] = []          # the three worst parameter tensors at the worst (t, k)
     layouts = {k: g.param_layout(k) for k in range(1, K + 1)}
@@ -52,26 +65,35 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
         x = S.images(seed, t, a.batch, a.in_h, a.in_w, a.in_c)
         y = S.labels(seed, t, a.batch, a.num_classes)
         lo = orc.step(x, y)
+        lo_plain = orc_plain.step(x, y) if orc_plain is not None else None
         g.step(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), loss_dev)
         if not (check_every_step or t == steps):
             continue
         g.sync()
         if lo is not None:
             res["loss"] = max(res["loss"], abs(float(loss_dev.item()) - lo) / max(abs(lo), 1e-30))
+            if lo_plain is not None:
+                res["loss_plain"] = max(res["loss_plain"], abs(float(loss_dev.item()) - lo_plain) / max(abs(lo_plain), 1e-30))
         for k in range(1, K + 1):
             if k < K and orc.module_output[k] is not None:
                 b, out = g.module_output(k)
                 bo, oo = orc.module_output[k]
                 assert b == bo, ("module output batch", t, k, b, bo)
                 res["out"] = max(res["out"], relmax(out, oo.reshape(-1)))
+                if orc_plain is not None:
+                    res["out_plain"] = max(res["out_plain"], relmax(out, orc_plain.module_output[k][1].reshape(-1)))
             if k >= 2 and orc.input_grad[k] is not None:
                 b, gi = g.input_grad(k)
                 bo, go = orc.input_grad[k]
                 assert b == bo, ("input grad batch", t, k, b, bo)
                 res["gin"] = max(res["gin"], relmax(gi, go.reshape(-1)))
+                if orc_plain is not None:
+                    res["gin_plain"] = max(res["gin_plain"], relmax(gi, orc_plain.input_grad[k][1].reshape(-1)))
             go = orc.get_grads(k)
             if go is not None:
                 gg = g.get_grads(k)
+                if orc_plain is not None:
+                    res["grads_plain"] = max(res["grads_plain"], relfro(gg, orc_plain.get_grads(k)))
                 err = relfro(gg, go)
                 res["grads_by_step"].append((t, k, float("%.3g" % err)))
                 if err > res["grads"]:
@@ -81,25 +103,11 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
                         off, n = int(name.split("@")[1]), int(np.prod(shape))
                         per.append((round(relfro(gg[off:off + n], go[off:off + n]), 4), t, k, name, tuple(shape)))
                     res["worst_tensors"] = sorted(per, reverse=True)[:3]
-                    if err > 1.0 and "bad_ranges" not in res:
-                        # where in the flat gradient the two sides part, in chunks of 1024 elements, and whether a
-                        # second read of the same gradient returns the same values
-                        d = np.abs(gg.astype(np.float64) - go)
-                        n1k = (len(d) + 1023) // 1024
-                        bad = [c for c in range(n1k)
-                               if np.linalg.norm(d[c * 1024:(c + 1) * 1024]) > np.linalg.norm(go[c * 1024:(c + 1) * 1024]) + 1e-12]
-                        runs, start = [], None
-                        for c in range(n1k + 1):
-                            if c in set(bad) and start is None: start = c
-                            if c not in set(bad) and start is not None: runs.append((start * 1024, c * 1024)); start = None
-                        res["bad_ranges"] = runs[:12]
-                        res["reread_equal"] = bool(np.array_equal(gg, g.get_grads(k)))
-                        res["norms"] = [(name, float(np.linalg.norm(gg[int(name.split("@")[1]):int(name.split("@")[1]) + int(np.prod(shape))])),
-                                         float(np.linalg.norm(go[int(name.split("@")[1]):int(name.split("@")[1]) + int(np.prod(shape))])))
-                                        for name, _, shape in layouts[k]]
     g.sync()
     res["params"] = max(relfro(g.get_params(k), orc.get_params(k)) for k in range(1, K + 1))
     res["momentum"] = max(relfro(g.get_momentum(k), orc.get_momentum(k)) for k in range(1, K + 1))
+    if orc_plain is not None:
+        res["params_plain"] = max(relfro(g.get_params(k), orc_plain.get_params(k)) for k in range(1, K + 1))
     res["log_gpu"] = [(r["t"], r["k"], r["tau_f"], r["tau_b"], r["ver_f"], r["ver_b"]) for r in g.schedule_log()]
     res["log_oracle"] = [(r["t"], r["k"], r["tau_f"], r["tau_b"], r["ver_f"], r["ver_b"]) for r in orc.log]
     res["launches"] = g.launch_count()

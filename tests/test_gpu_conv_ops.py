@@ -37,7 +37,11 @@ SHAPES_TC = [(4, 32, 32, 16, 16, 3, 1, 1),      # 32 tiles of 4 image rows, 32-b
              (301, 8, 8, 64, 64, 3, 1, 1),      # ragged last tile with several images per tile
              (130, 32, 32, 16, 16, 3, 1, 1),    # stage-1 shape of the 6n+2 networks, more images than weight-gradient CTAs
              (6, 32, 32, 16, 32, 3, 2, 1),      # stride 2: forward = the stride-1 kernel stored at the even pixels
-             (9, 16, 16, 32, 64, 3, 2, 1)]
+             (9, 16, 16, 32, 64, 3, 2, 1),
+             (2, 16, 16, 320, 320, 3, 1, 1),    # WRN stage 2: five 64-channel chunks, two 160-column N tiles
+             (4, 8, 8, 640, 640, 3, 1, 1),      # WRN stage 3: four N tiles, the weight gradient in 10 x 10 channel chunks
+             (2, 32, 32, 160, 320, 3, 2, 1),    # the stride-2 layers of WRN-28-10 (per-tap kernel at full resolution)
+             (2, 16, 16, 320, 640, 3, 2, 1)]
 
 # shapes whose three operators all take the halo-tile tensor-core kernels
 ALL_TC = {(4, 32, 32, 16, 16), (6, 16, 16, 32, 32), (10, 8, 8, 64, 64), (300, 8, 8, 64, 64), (5, 12, 20, 16, 32),
@@ -79,6 +83,22 @@ def _run(prec_name, shape, expect_tc):
 
     dw = ops.wgrad(s, x, dy).cpu().numpy()
     assert _rel(dw, dwo) < (1e-3 if prec_name == "bf16" else 2e-5)
+    if expect_tc:
+        # the launch shapes of a module-step: a third of the SMs per kernel (four modules side by side),
+        # the weight gradient's pixel split capped at 16 CTAs (side stream), and, for stride 2, both
+        # gradients on the tensor cores through the spread-out dy
+        sp = st == 2
+        if sp:
+            assert ops.path(s, 1)
+        y = ops.forward(s, x, wt, res=resy, share=3).float().cpu().numpy()
+        assert _rel(y, L.conv2d_forward(xo, wo, st, pad) + resyo) < tol
+        dx = ops.dgrad(s, dy, wt, wf, res=res, res_mask=mask, share=3, spread=sp).float().cpu().numpy()
+        assert _rel(dx, dxo + reso * (masko > 0)) < tol
+        dx = ops.dgrad(s, dy, wt, wf, spread=sp).float().cpu().numpy()
+        assert _rel(dx, dxo) < tol
+        for cap in (0, 16):
+            dw = ops.wgrad(s, x, dy, cta_cap=cap, spread=sp).cpu().numpy()
+            assert _rel(dw, dwo) < 1e-3, cap
     assert not ops.timed_out()
 
 

@@ -1,0 +1,94 @@
+"""Error paths of the library, exercised without making any kernel misbehave: bad inputs the kernels detect
+and survive (a non-finite loss, a label out of range), and status words raised from the host the way a
+kernel would raise them (fdg_debug_raise_flag), checked through what fdg_sync and fdg_step report."""
+import numpy as np
+import pytest
+import torch
+
+import fdg_synth as S
+
+pytestmark = pytest.mark.gpu
+
+ARCH = dict(family="resnet6n2", n_per_stage=1, widths=(8, 16, 32), stem_width=8, in_h=16, in_w=16, in_c=3,
+            num_classes=10, batch=8)
+
+
+def _make(B, K, splits, **kw):
+    g = B.FDG(B.make_arch(**ARCH), K=K, split_after_block=splits, beta=0.5, lr=0.05, **kw)
+    for k in range(1, K + 1):
+        g.set_params(k, S.init_params(0, k, g.param_layout(k)))
+    return g
+
+
+def _batch(t):
+    return (torch.from_numpy(S.images(0, t, 8, 16, 16, 3)).cuda(), torch.from_numpy(S.labels(0, t, 8, 10)).cuda())
+
+
+def _status(g, fn, *args):
+    from paper_1906_09108_b200 import binding as B
+    try:
+        fn(*args)
+        return B.FDG_OK
+    except B.FDGError as e:
+        return e.status
+
+
+@pytest.mark.parametrize("precision", ["fp32", "bf16"])
+def test_nonfinite_loss_is_reported_once_and_the_context_carries_on(precision):
+    from paper_1906_09108_b200 import binding as B
+    g = _make(B, 1, (), precision=B.FDG_BF16_TC if precision == "bf16" else B.FDG_FP32_CUDACORE)
+    loss = torch.zeros(1, device="cuda")
+    x, y = _batch(1)
+    g.step(x, y, loss)
+    g.sync()
+    assert np.isfinite(loss.item())
+    bad = x.clone()
+    bad[0, 0, 0, 0] = float("nan")
+    g.step(bad, y, loss)
+    assert _status(g, g.sync) == 6                                  # FDG_ERR_NONFINITE
+    assert "NaN" in g.lib.fdg_last_error(g.ctx).decode()
+    assert _status(g, g.sync) == B.FDG_OK                           # reported once, then cleared
+    # the update that followed spread the NaN into the weights: a cold restart (parameters, momentum) recovers
+    for k in (1,):
+        g.set_params(k, S.init_params(0, k, g.param_layout(k)))
+        g.set_momentum(k, np.zeros(g.param_count(k), dtype=np.float32))
+    g.step(x, y, loss)
+    assert _status(g, g.sync) == B.FDG_OK and np.isfinite(loss.item())
+    g.close()
+
+
+def test_label_out_of_range_is_reported_and_treated_as_class_zero():
+    from paper_1906_09108_b200 import binding as B
+    g = _make(B, 2, (1,))
+    x, y = _batch(1)
+    bad = y.clone()
+    bad[3] = ARCH["num_classes"]
+    g.step(x, bad)                                                   # module 2 meets these labels at t = 2
+    assert _status(g, g.sync) == B.FDG_OK
+    g.step(*_batch(2))
+    assert _status(g, g.sync) == 1                                   # FDG_ERR_INVALID_ARG
+    assert "label" in g.lib.fdg_last_error(g.ctx).decode()
+    g.step(*_batch(3))
+    assert _status(g, g.sync) == B.FDG_OK
+    g.close()
+
+
+def test_raised_status_words_reach_the_caller():
+    """The three device status words, raised from the host as a kernel would raise them.  The time-out of a
+    tensor-core kernel's bounded wait is latched: the kernel left early, so the context refuses to go on."""
+    from paper_1906_09108_b200 import binding as B
+    g = _make(B, 2, (1,))
+    g.step(*_batch(1))
+    g.sync()
+    for which, status in ((0, 6), (1, 1)):
+        assert g.lib.fdg_debug_raise_flag(g.ctx, which) == B.FDG_OK
+        assert _status(g, g.sync) == status
+        assert _status(g, g.sync) == B.FDG_OK
+        g.step(*_batch(2 + which))
+    assert g.lib.fdg_debug_raise_flag(g.ctx, 3) == 1
+    assert g.lib.fdg_debug_raise_flag(g.ctx, 2) == B.FDG_OK
+    assert _status(g, g.sync) == 7                                   # FDG_ERR_TIMEOUT
+    assert "waiting" in g.lib.fdg_last_error(g.ctx).decode()
+    assert _status(g, g.sync) == 7                                   # latched
+    assert _status(g, g.step, *_batch(9)) == 7
+    g.close()

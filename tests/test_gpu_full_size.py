@@ -107,6 +107,26 @@ def test_forward_of_every_block_at_full_size():
     print("worst relative errors over %d blocks:" % checked, worst)
 
 
+def test_backward_of_every_block_at_full_size():
+    """The backward twin of the test above (Eq. 10 with the shrunk gradient of Eq. 15): ResNet-110, K = 4, batch 128,
+    one stream per module plus the side stream of the weight gradients, i.e. the kernels and launch shapes the
+    benchmark's graphs replay (a convolution on a third of the SMs, the weight gradients' pixel split capped at
+    16 CTAs).  A capture keeps every gradient tensor of each module's backward pass at iteration 2K - 1, the first
+    one in which all four modules back-propagate.  Every layer of every block is then recomputed by the oracle
+    from the library's own inputs to that layer -- the incoming gradient it captured and the activations it saved
+    for that batch, so every ReLU gate is the same on both sides -- and compared element by element at 1e-2: the
+    batch-norm backwards (whose sums come from the data-gradient epilogues for identity blocks and from the
+    reduction kernel for projection blocks), the 3x3 data gradients with their fused residual, the stride-2 and
+    1x1 projection gradients, all weight gradients, the stem and the classifier."""
+    from paper_1906_09108_b200 import binding as B
+    from tests.layerwise import check_backward_layerwise
+    g, params = _make(B, lr=0.0, weight_decay=0.0)
+    checked, worst = check_backward_layerwise(g, params, ARCH, 4)
+    g.close()
+    assert checked == 54
+    print("worst relative errors over %d blocks:" % checked, {k_: float("%.2g" % v) for k_, v in worst.items()})
+
+
 def test_bench_launch_shapes_against_oracle():
     """Forward, backward and update at the benchmark's layer shapes, batch and launch shapes, end to end
     against the oracle: a 6n+2 network with n = 2 (14 layers) cut into K = 4 modules, batch 128, graphs on.

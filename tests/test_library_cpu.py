@@ -77,3 +77,17 @@ def test_workspace_bytes_and_argument_checks(lib):
     assert lib.fdg_last_error(None) == b"null context"
     ctx = C.c_void_p()
     assert lib.fdg_create(C.byref(arch), C.byref(cfg), None, 0, None, C.byref(ctx)) == 1 and not ctx.value
+    # a workspace that is there but one byte short is refused before anything touches it (the pointer is never
+    # dereferenced on this path, so any aligned address will do)
+    assert lib.fdg_workspace_bytes(C.byref(arch), C.byref(cfg), C.byref(n)) == 0
+    assert lib.fdg_create(C.byref(arch), C.byref(cfg), C.c_void_p(1 << 20), n.value - 1, None, C.byref(ctx)) == 2
+    assert not ctx.value
+    assert lib.fdg_create(C.byref(arch), C.byref(cfg), C.c_void_p((1 << 20) + 8), n.value, None, C.byref(ctx)) == 1   # misaligned
+    assert lib.fdg_debug_raise_flag(None, 0) == 1
+    # operator level: argument checks that answer without a GPU
+    s = B.fdg_conv_shape(2, 8, 8, 512, 512, 3, 1, 1)
+    assert lib.fdg_conv_wgrad_static(0, C.byref(s), C.c_void_p(256), C.c_void_p(256), C.c_void_p(256), None) == 2
+    assert lib.fdg_conv_wgrad_static(0, C.byref(s), None, C.c_void_p(256), C.c_void_p(256), None) == 1
+    assert lib.fdg_bn_scratch_bytes(64, C.byref(n)) == 0 and n.value >= 74 * 3 * 64 * 4
+    assert lib.fdg_bn_scratch_bytes(0, C.byref(n)) == 1
+    assert lib.fdg_bn_stats(0, C.c_void_p(256), 16, 64, 1e-5, C.c_void_p(256), C.c_void_p(256), 16, None) == 2

@@ -2,6 +2,8 @@
 (its partial sums go to a buffer built into the library).  Checked through the C ABI against
 fdg_conv_wgrad, which takes caller-provided scratch, on two calls in a row with different
 inputs, so that anything the first call left in the shared buffer would show in the second.
+fdg_conv_wgrad is itself held to the oracle on shapes of this kind (tests/test_gpu_conv_ops.py);
+the second call here is compared with the oracle's convolution backward directly as well.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run
 every other test."""
@@ -38,6 +40,10 @@ def test_static_scratch_matches_caller_scratch_twice(prec_name):
             got = ops.wgrad_static(s, x, dy).cpu().numpy()
             err = np.abs(got - want).max() / max(np.abs(want).max(), 1e-30)
             assert err <= tol, (shape, call, err)
+        from oracle import layers as L
+        dwo = L.conv2d_backward(dy.float().cpu().numpy().astype(np.float64), x.float().cpu().numpy().astype(np.float64),
+                                np.zeros((co, r, r, ci)), st, pad)[1]
+        assert np.abs(got - dwo).max() / np.abs(dwo).max() <= tol, shape
 
 
 def test_static_scratch_rejects_oversized_shapes():
