@@ -254,10 +254,133 @@ def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5, use_grap
     return us, 2 * elems * 2 + wbytes, 2.0 * n * h * w * c * 9 * c
 
 
+EW_KERNELS = ["bn_stats", "bn_apply", "bn_apply_res", "bn_bwd_reduce", "bn_bwd_apply", "shrink", "sgd", "ingest", "head"]
+
+
+def ew_kernel_bench(B, which, stage="stage1", launches=64, reps=5, use_graph=True):
+    """The same measurement for a memory-bound kernel of the module-step through its operator-level entry point:
+    `launches` calls, each on its own tensors out of a pool that sums to more than twice the L2 cache, recorded
+    into a CUDA graph and replayed; CUDA events around the replay.  Returns (microseconds per launch,
+    algorithmic bytes per launch: every operand tensor once)."""
+    import torch
+    n, h, w, c = KERNEL_SHAPES[stage]
+    ew = B.EwOps(B.FDG_BF16_TC)
+    lib, prec, C = ew.lib, ew.precision, B.C
+    elems, rows = n * h * w * c, n * h * w
+    tensors_per_call = {"bn_stats": 1, "bn_apply": 2, "bn_apply_res": 3, "bn_bwd_reduce": 3, "bn_bwd_apply": 4, "shrink": 2,
+                        "sgd": 0, "ingest": 0, "head": 2}[which]
+    fused_sums = 2 * c <= 256           # the layers whose data gradient leaves the sums as per-CTA partial rows
+    if which == "bn_bwd_apply" and not fused_sums:
+        tensors_per_call = 7            # wider layers: reduce (3 reads) + apply (3 reads, 1 write) in one call
+    st = torch.cuda.Stream()
+    bf = torch.bfloat16
+    if which == "sgd":                       # one module of the headline workload has ~0.5 M parameters; use 8 M for a
+        nparam = 8 << 20                     # transfer that is not all launch latency (24 B per parameter + 2 B copy)
+        pool = max(4, (300 << 20) // (26 * nparam) + 1)
+        bufs = [[torch.randn(nparam, device="cuda") for _ in range(3)] + [torch.empty(nparam, device="cuda"),
+                torch.empty(nparam, dtype=bf, device="cuda")] for _ in range(pool)]
+        nbytes = 26 * nparam
+    elif which == "ingest":
+        rows_i = n * h * w
+        pool = max(4, (300 << 20) // (rows_i * (12 + 6)) + 1)
+        bufs = [[torch.randn((n, h, w, 3), device="cuda"), torch.empty((n, h, w, 3), dtype=bf, device="cuda")] for _ in range(pool)]
+        lab = torch.zeros(n, dtype=torch.int32, device="cuda")
+        lab2 = torch.zeros(n, dtype=torch.int32, device="cuda")
+        nbytes = rows_i * (12 + 6)
+    else:
+        nt = min(tensors_per_call, 4)
+        pool = max(4, (300 << 20) // (2 * elems * nt) + 1)
+        bufs = [[torch.randn((n, h, w, c), device="cuda").to(bf) for _ in range(nt)] for _ in range(pool)]
+        nbytes = 2 * elems * tensors_per_call
+    gam = torch.ones(c, device="cuda")
+    bet = torch.zeros(c, device="cuda")
+    stats = torch.cat([torch.zeros(c, device="cuda"), torch.ones(c, device="cuda")])
+    dg, db = torch.empty(c, device="cuda"), torch.empty(c, device="cuda")
+    need = C.c_size_t()
+    ew._chk(lib.fdg_bn_scratch_bytes(c, C.byref(need)))
+    scratch = torch.zeros(need.value, dtype=torch.uint8, device="cuda")
+    if which == "head":
+        classes = 10
+        wfc, bfc = torch.randn((classes, c), device="cuda") * 0.1, torch.zeros(classes, device="cuda")
+        hl = torch.zeros(n, dtype=torch.int32, device="cuda")
+        hb = dict(pooled=torch.empty((n, c), device="cuda"), dlogits=torch.empty((n, classes), device="cuda"),
+                  loss_n=torch.empty(n, device="cuda"), dw=torch.empty((classes, c), device="cuda"),
+                  db=torch.empty(classes, device="cuda"), loss=torch.empty(1, device="cuda"),
+                  flags=torch.zeros(4, dtype=torch.int32, device="cuda"))
+    P = lambda t: t.data_ptr()
+
+    def call(i):
+        t = bufs[i % pool]
+        cs = st.cuda_stream
+        if which == "bn_stats":
+            rc = lib.fdg_bn_stats(prec, P(t[0]), rows, c, 1e-5, P(stats), P(scratch), need.value, cs)
+        elif which == "bn_apply":
+            rc = lib.fdg_bn_apply(prec, P(t[0]), P(stats), P(gam), P(bet), None, None, None, None, 1, P(t[1]), rows, c, 1e-5,
+                                  None, 0, 0, cs)
+        elif which == "bn_apply_res":
+            rc = lib.fdg_bn_apply(prec, P(t[0]), P(stats), P(gam), P(bet), P(t[2]), None, None, None, 1, P(t[1]), rows, c,
+                                  1e-5, None, 0, 0, cs)
+        elif which == "bn_bwd_reduce":
+            rc = lib.fdg_bn_backward(prec, P(t[0]), P(t[1]), P(t[2]), P(stats), P(gam), None, None, None, None, None, None,
+                                     P(dg), P(db), None, None, rows, c, None, 0, 0, P(scratch), need.value, cs)
+        elif which == "bn_bwd_apply":      # the sums come as one row of partials, as after a fused data gradient
+            rc = lib.fdg_bn_backward(prec, P(t[0]), P(t[1]), P(t[2]), P(stats), P(gam), None, None, None, None, P(t[3]), None,
+                                     P(dg), P(db), None, None, rows, c, P(stats) if fused_sums else None, 1 if fused_sums else 0,
+                                     148, P(scratch), need.value, cs)
+        elif which == "shrink":
+            rc = lib.fdg_shrink(prec, P(t[0]), P(t[1]), 0.2, elems, cs)
+        elif which == "sgd":
+            rc = lib.fdg_sgd_update(P(t[0]), P(t[1]), P(t[2]), P(t[3]), P(t[4]), t[0].numel(), 1e-3, 0.9, 5e-4, cs)
+        elif which == "ingest":
+            rc = lib.fdg_ingest(prec, P(t[0]), P(t[1]), n * h * w, 3, 3, P(lab), P(lab2), n, cs)
+        else:
+            rc = lib.fdg_head(prec, P(t[0]), P(wfc), P(bfc), P(hl), n, h * w, c, classes, P(hb["pooled"]), P(hb["dlogits"]),
+                              P(hb["loss_n"]), P(t[1]), P(hb["dw"]), P(hb["db"]), P(hb["loss"]), P(hb["flags"]), cs)
+        ew._chk(rc)
+
+    with torch.cuda.stream(st):
+        for i in range(pool):
+            call(i)
+        st.synchronize()
+        if use_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=st):
+                for i in range(launches):
+                    call(i)
+            replay = graph.replay
+        else:
+            def replay():
+                for i in range(launches):
+                    call(i)
+        replay()
+        st.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for _ in range(reps):
+            replay()
+        e1.record(st)
+        st.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / (reps * launches), nbytes
+
+
 def run_kernel_bench(args):
     from paper_1906_09108_b200 import binding as B
     peaks = measured_peaks()
     out = {}
+    if args.kernel_bench == "ew" or args.kernel_bench in EW_KERNELS:
+        kinds = EW_KERNELS if args.kernel_bench == "ew" else [args.kernel_bench]
+        stages = [args.kernel_stage] if args.kernel_stage else ["stage1", "wrn_stage1"]
+        for which in kinds:
+            for stage in stages:
+                if which in ("sgd",) and stage != stages[0]:
+                    continue
+                us, nbytes = ew_kernel_bench(B, which, stage, launches=args.kernel_launches,
+                                             reps=1 if args.kernel_launches <= 8 else 5, use_graph=args.kernel_launches > 8)
+                name = which + ("+reduce" if which == "bn_bwd_apply" and KERNEL_SHAPES[stage][3] > 128 else "")
+                out["%s_%s" % (name, "8Mparams" if which == "sgd" else stage)] = dict(
+                    us=us, mbytes=nbytes / 1e6, gbs=nbytes / us / 1e3, hbm_frac=nbytes / us / 1e3 / peaks["hbm_gbs"])
+        print(json.dumps(dict(kernel_bench=out, peak_source=peaks["source"], hbm_gbs=peaks["hbm_gbs"])))
+        return
     which_list = [args.kernel_bench] if args.kernel_bench != "all" else ["fprop", "dgrad", "wgrad"]
     stages = [args.kernel_stage] if args.kernel_stage else list(KERNEL_SHAPES)
     for which in which_list:
@@ -444,7 +567,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graphs", action="store_true")
     ap.add_argument("--workload", default="resnet110_k4", choices=list(WORKLOADS))
-    ap.add_argument("--kernel-bench", default=None, choices=["fprop", "dgrad", "wgrad", "all"],
+    ap.add_argument("--kernel-bench", default=None, choices=["fprop", "dgrad", "wgrad", "all", "ew"] + EW_KERNELS,
                     help="time the convolution kernels alone through the operator-level C ABI and exit")
     ap.add_argument("--kernel-launches", type=int, default=64,
                     help="launches per replay; 8 or fewer are issued as plain launches (profiler runs)")

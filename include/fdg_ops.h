@@ -137,7 +137,8 @@ fdg_status fdg_bn_apply(int precision, const void* x, float* stats, const float*
  *   dbeta = sum dz, dgamma = sum dz*xhat, dx = gamma*invstd*(dz - dbeta/M - xhat*dgamma/M) [+ res].
  * With (x2, stats2, gamma2) the same dz is also taken through a second normalisation (the projection
  * shortcut of a block): dx2, dgamma2, dbeta2.  With `partial` (rows left by fdg_conv_dgrad with reduce = 2)
- * the sums are read from those rows instead of being formed here (single normalisation only). */
+ * the sums are read from those rows instead of being formed here (single normalisation only).  With dx NULL
+ * only the sums, i.e. the parameter gradients, are formed. */
 fdg_status fdg_bn_backward(int precision, const void* dy, const void* mask, const void* x, const float* stats,
                            const float* gamma, const void* x2, const float* stats2, const float* gamma2, const void* res,
                            void* dx, void* dx2, float* dgamma, float* dbeta, float* dgamma2, float* dbeta2, size_t rows,

@@ -488,14 +488,15 @@ class EwOps:
                                         0 if partial is None else partial.shape[0], block_cap, self._stream()))
         return y
 
-    def bn_backward(self, dy, mask, x, stats, gamma, second=None, res=None, partial=None, block_cap=0):
-        """Returns (dx, dgamma, dbeta) or, with second = (x2, stats2, gamma2), (dx, dgamma, dbeta, dx2, dgamma2, dbeta2)."""
+    def bn_backward(self, dy, mask, x, stats, gamma, second=None, res=None, partial=None, block_cap=0, sums_only=False):
+        """Returns (dx, dgamma, dbeta) or, with second = (x2, stats2, gamma2), (dx, dgamma, dbeta, dx2, dgamma2, dbeta2);
+        sums_only: dx is None and only the parameter gradients are formed."""
         ch = x.shape[-1]
         rows = x.numel() // ch
-        dx = self.torch.empty_like(x)
+        dx = None if sums_only else self.torch.empty_like(x)
         dg, db = self._f32(ch), self._f32(ch)
         x2, s2, g2 = second if second else (None, None, None)
-        dx2 = self.torch.empty_like(x) if second else None
+        dx2 = self.torch.empty_like(x) if (second and not sums_only) else None
         dg2, db2 = (self._f32(ch), self._f32(ch)) if second else (None, None)
         sc, nb = self._scratch(ch)
         self._chk(self.lib.fdg_bn_backward(self.precision, _ptr(dy), _ptr(mask), _ptr(x), _ptr(stats), _ptr(gamma), _ptr(x2),

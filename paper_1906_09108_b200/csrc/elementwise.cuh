@@ -253,33 +253,80 @@ __device__ __forceinline__ void finalize_partials(const PartialSums ps, int C, f
 
 // y = [relu]( gamma*(x-mean)*invstd + beta + residual ), residual = none | r | BN_r(r).
 // The statistics come from `stats`, or are first formed from `ps.partial` (and saved to stats).
-template <typename T, int VEC>
-__global__ void bn_apply_kernel(const T* __restrict__ x, const float* __restrict__ stats,
-                                const float* __restrict__ gamma, const float* __restrict__ beta,
-                                const T* __restrict__ res, const float* __restrict__ res_stats,
-                                const float* __restrict__ res_gamma, const float* __restrict__ res_beta,
-                                int relu, T* __restrict__ y, size_t nvec, int C, PartialSums ps) {
+// The launcher makes the grid's thread count a multiple of the channel vectors per row, so a thread
+// meets the same VEC channels in every iteration: their constants live in registers, and the loop
+// keeps kEwUnroll independent 16-byte loads per operand in flight.
+constexpr int kEwUnroll = 4;
+// 16 raw bytes (or one element when VEC == 1) of T, converted to floats only when used, so that
+// several loads can be in flight without holding their float images in registers.
+template <typename T, int VEC> struct RawVec { uint4 q; };
+template <typename T> struct RawVec<T, 1> { T q; };
+template <typename T, int VEC> __device__ __forceinline__ RawVec<T, VEC> load_raw(const T* __restrict__ p) {
+  RawVec<T, VEC> r;
+  if constexpr (VEC == 1) r.q = p[0]; else r.q = *reinterpret_cast<const uint4*>(p);
+  return r;
+}
+template <typename T, int VEC> __device__ __forceinline__ void raw_to_f(const RawVec<T, VEC>& r, float (&out)[VEC]) {
+  if constexpr (VEC == 1) {
+    out[0] = to_f(r.q);
+  } else {
+    const T* e = reinterpret_cast<const T*>(&r.q);
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) out[i] = to_f(e[i]);
+  }
+}
+
+template <typename T, int VEC, bool RES_BN>
+__global__ void __launch_bounds__(kEwThreads, 3)
+bn_apply_kernel(const T* __restrict__ x, const float* __restrict__ stats,
+                const float* __restrict__ gamma, const float* __restrict__ beta,
+                const T* __restrict__ res, const float* __restrict__ res_stats,
+                const float* __restrict__ res_gamma, const float* __restrict__ res_beta,
+                int relu, T* __restrict__ y, size_t nvec, int C, PartialSums ps) {
   __shared__ float s_stats[2 * 128];
   const float* st = stats;
   if (ps.partial) { finalize_partials(ps, C, s_stats); st = s_stats; }
   const int cv = C / VEC;
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
-    const int c0 = (int)(i % cv) * VEC;
+  const size_t gtid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
+  const int c0 = (int)(gtid % cv) * VEC;
+  float mean[VEC], inv[VEC], ga[VEC], be[VEC], rmean[RES_BN ? VEC : 1], rinv[RES_BN ? VEC : 1], rga[RES_BN ? VEC : 1], rbe[RES_BN ? VEC : 1];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    mean[j] = st[c0 + j]; inv[j] = st[C + c0 + j]; ga[j] = gamma[c0 + j]; be[j] = beta[c0 + j];
+    if constexpr (RES_BN) { rmean[j] = res_stats[c0 + j]; rinv[j] = res_stats[C + c0 + j]; rga[j] = res_gamma[c0 + j]; rbe[j] = res_beta[c0 + j]; }
+  }
+  auto one = [&](size_t i, const RawVec<T, VEC>& xv, const RawVec<T, VEC>& rv) {
     float v[VEC], r[VEC], o[VEC];
-    load_vec<T, VEC>(x + i * VEC, v);
-    if (res) load_vec<T, VEC>(res + i * VEC, r);
+    raw_to_f<T, VEC>(xv, v);
+    if (res) raw_to_f<T, VEC>(rv, r);
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
-      const int c = c0 + j;
-      float t = gamma[c] * ((v[j] - st[c]) * st[C + c]) + beta[c];
+      float t = ga[j] * ((v[j] - mean[j]) * inv[j]) + be[j];
       if (res) {
         float rr = r[j];
-        if (res_stats) rr = res_gamma[c] * ((rr - res_stats[c]) * res_stats[C + c]) + res_beta[c];
+        if constexpr (RES_BN) rr = rga[j] * ((rr - rmean[j]) * rinv[j]) + rbe[j];
         t += rr;
       }
       o[j] = relu ? fmaxf(t, 0.f) : t;
     }
     store_vec<T, VEC>(y + i * VEC, o);
+  };
+  size_t i = gtid;
+  for (; i + (kEwUnroll - 1) * stride < nvec; i += kEwUnroll * stride) {
+    RawVec<T, VEC> xv[kEwUnroll], rv[kEwUnroll];
+#pragma unroll
+    for (int u = 0; u < kEwUnroll; ++u) xv[u] = load_raw<T, VEC>(x + (i + u * stride) * VEC);
+    if (res) {
+#pragma unroll
+      for (int u = 0; u < kEwUnroll; ++u) rv[u] = load_raw<T, VEC>(res + (i + u * stride) * VEC);
+    }
+#pragma unroll
+    for (int u = 0; u < kEwUnroll; ++u) one(i + u * stride, xv[u], rv[u]);
+  }
+  for (; i < nvec; i += stride) {
+    RawVec<T, VEC> xv = load_raw<T, VEC>(x + i * VEC), rv = xv;
+    if (res) rv = load_raw<T, VEC>(res + i * VEC);
+    one(i, xv, rv);
   }
 }
 
@@ -327,41 +374,66 @@ bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ mask, const
 }
 
 // dx = gamma*invstd*(dz - s0/M - xhat*s1/M) [+ res];  optionally the same for the second
-// normalised tensor (dx2) and/or the masked gradient itself (dz_out).
-template <typename T, int VEC>
-__global__ void bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ mask, const T* __restrict__ x,
-                                    const float* __restrict__ stats, const float* __restrict__ gamma,
-                                    const float* __restrict__ sums, const T* __restrict__ x2,
-                                    const float* __restrict__ stats2, const float* __restrict__ gamma2,
-                                    const T* __restrict__ res, T* __restrict__ dx, T* __restrict__ dx2,
-                                    T* __restrict__ dz_out, size_t nvec, int C, float inv_m, PartialSums ps) {
+// normalised tensor (dx2, TWO).  Per-thread channel constants and loads in flight as in bn_apply_kernel.
+template <typename T, int VEC, bool TWO>
+__global__ void __launch_bounds__(kEwThreads, 3)
+bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ mask, const T* __restrict__ x,
+                    const float* __restrict__ stats, const float* __restrict__ gamma,
+                    const float* __restrict__ sums, const T* __restrict__ x2,
+                    const float* __restrict__ stats2, const float* __restrict__ gamma2,
+                    const T* __restrict__ res, T* __restrict__ dx, T* __restrict__ dx2,
+                    size_t nvec, int C, float inv_m, PartialSums ps) {
   __shared__ float s_sums[2 * 128];
   if (ps.partial) { finalize_partials(ps, C, s_sums); sums = s_sums; }
   const int cv = C / VEC;
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
-    const int c0 = (int)(i % cv) * VEC;
-    float d[VEC], m[VEC], v[VEC], v2[VEC], r[VEC], o[VEC], o2[VEC], oz[VEC];
-    load_vec<T, VEC>(dy + i * VEC, d);
-    if (mask) load_vec<T, VEC>(mask + i * VEC, m);
-    load_vec<T, VEC>(x + i * VEC, v);
-    if (dx2) load_vec<T, VEC>(x2 + i * VEC, v2);
+  const size_t gtid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
+  const int c0 = (int)(gtid % cv) * VEC;
+  constexpr int V2 = TWO ? VEC : 1;
+  float mean[VEC], inv[VEC], gi[VEC], s0[VEC], s1[VEC], mean2[V2], inv2[V2], gi2[V2], s2[V2];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    mean[j] = stats[c0 + j]; inv[j] = stats[C + c0 + j]; gi[j] = gamma[c0 + j] * inv[j];
+    s0[j] = sums[c0 + j] * inv_m; s1[j] = sums[C + c0 + j] * inv_m;
+    if constexpr (TWO) { mean2[j] = stats2[c0 + j]; inv2[j] = stats2[C + c0 + j]; gi2[j] = gamma2[c0 + j] * inv2[j]; s2[j] = sums[2 * C + c0 + j] * inv_m; }
+  }
+  auto one = [&](size_t i, const RawVec<T, VEC>& dv, const RawVec<T, VEC>& mv, const RawVec<T, VEC>& xv) {
+    float d[VEC], m[VEC], v[VEC], v2[VEC], r[VEC], o[VEC], o2[VEC];
+    raw_to_f<T, VEC>(dv, d);
+    if (mask) raw_to_f<T, VEC>(mv, m);
+    raw_to_f<T, VEC>(xv, v);
+    if constexpr (TWO) load_vec<T, VEC>(x2 + i * VEC, v2);
     if (res) load_vec<T, VEC>(res + i * VEC, r);
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
-      const int c = c0 + j;
-      float dz = (mask && !(m[j] > 0.f)) ? 0.f : d[j];
-      oz[j] = dz;
-      float xh = (v[j] - stats[c]) * stats[C + c];
-      float t = gamma[c] * stats[C + c] * (dz - sums[c] * inv_m - xh * (sums[C + c] * inv_m));
+      const float dz = (mask && !(m[j] > 0.f)) ? 0.f : d[j];
+      const float xh = (v[j] - mean[j]) * inv[j];
+      const float t = gi[j] * (dz - s0[j] - xh * s1[j]);
       o[j] = res ? t + r[j] : t;
-      if (dx2) {
-        float xh2 = (v2[j] - stats2[c]) * stats2[C + c];
-        o2[j] = gamma2[c] * stats2[C + c] * (dz - sums[c] * inv_m - xh2 * (sums[2 * C + c] * inv_m));
+      if constexpr (TWO) {
+        const float xh2 = (v2[j] - mean2[j]) * inv2[j];
+        o2[j] = gi2[j] * (dz - s0[j] - xh2 * s2[j]);
       }
     }
     store_vec<T, VEC>(dx + i * VEC, o);
-    if (dx2) store_vec<T, VEC>(dx2 + i * VEC, o2);
-    if (dz_out) store_vec<T, VEC>(dz_out + i * VEC, oz);
+    if constexpr (TWO) store_vec<T, VEC>(dx2 + i * VEC, o2);
+  };
+  constexpr int U = 2;
+  size_t i = gtid;
+  for (; i + (U - 1) * stride < nvec; i += U * stride) {
+    RawVec<T, VEC> dv[U], mv[U], xv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      dv[u] = load_raw<T, VEC>(dy + (i + u * stride) * VEC);
+      mv[u] = mask ? load_raw<T, VEC>(mask + (i + u * stride) * VEC) : dv[u];
+      xv[u] = load_raw<T, VEC>(x + (i + u * stride) * VEC);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) one(i + u * stride, dv[u], mv[u], xv[u]);
+  }
+  for (; i < nvec; i += stride) {
+    RawVec<T, VEC> dv = load_raw<T, VEC>(dy + i * VEC), mv = dv, xv = load_raw<T, VEC>(x + i * VEC);
+    if (mask) mv = load_raw<T, VEC>(mask + i * VEC);
+    one(i, dv, mv, xv);
   }
 }
 
@@ -598,6 +670,19 @@ inline cudaError_t launch_bn_stats(cudaStream_t st, const T* x, size_t rows, int
   return cudaGetLastError();
 }
 
+// Grid of the batch-norm apply kernels: what `nvec` vectors need, bounded by `cap` (0 = none), and such that
+// the grid's thread count is a multiple of the `cv` channel vectors of a row (every thread then stays on the
+// same channels).  Surplus blocks of a tiny tensor simply find no work.
+inline int ew_grid_for_channels(size_t nvec, int cv, int cap) {
+  int a = cv, b = kEwThreads;
+  while (b) { const int t = a % b; a = b; b = t; }
+  const int unit = cv / a;                       // blocks per period
+  int blocks = ew_blocks((nvec + kEwUnroll - 1) / kEwUnroll);
+  if (cap > 0 && blocks > cap) blocks = cap;
+  blocks = blocks / unit * unit;
+  return blocks < unit ? unit : blocks;
+}
+
 // y = [relu](BN(x) + residual).  `partial` != null: the statistics are not in `stats` yet; a convolution left
 // `nparts` rows of per-CTA sums (sum x, sum x^2) there, which every block adds up first (block 0 saves the
 // result to `stats`); `block_cap` then bounds the grid, since every block repeats that addition.
@@ -615,11 +700,13 @@ inline cudaError_t launch_bn_apply(cudaStream_t st, const T* x, float* stats, co
     ps.save0 = stats; ps.save1 = stats + C;
   }
   if (C % V == 0) {
-    int blocks = ew_blocks(n / V);
-    if (ps.partial && block_cap > 0 && blocks > block_cap) blocks = block_cap;
-    bn_apply_kernel<T, V><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
+    const int blocks = ew_grid_for_channels(n / V, C / V, ps.partial ? block_cap : 0);
+    if (res_stats) bn_apply_kernel<T, V, true><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
+    else bn_apply_kernel<T, V, false><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
   } else {
-    bn_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
+    const int blocks = ew_grid_for_channels(n, C, 0);
+    if (res_stats) bn_apply_kernel<T, 1, true><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
+    else bn_apply_kernel<T, 1, false><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
   }
   return cudaGetLastError();
 }
@@ -661,11 +748,13 @@ inline cudaError_t launch_bn_bwd_apply(cudaStream_t st, const T* dy, const T* ma
     ps.partial = partial; ps.nparts = nparts; ps.kind = 2; ps.save0 = dbeta; ps.save1 = dgamma;
   }
   if (C % V == 0) {
-    int blocks = ew_blocks(n / V);
-    if (ps.partial && block_cap > 0 && blocks > block_cap) blocks = block_cap;
-    bn_bwd_apply_kernel<T, V><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n / V, C, inv_m, ps);
+    const int blocks = ew_grid_for_channels(n / V, C / V, ps.partial ? block_cap : 0);
+    if (dx2) bn_bwd_apply_kernel<T, V, true><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n / V, C, inv_m, ps);
+    else bn_bwd_apply_kernel<T, V, false><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n / V, C, inv_m, ps);
   } else {
-    bn_bwd_apply_kernel<T, 1><<<ew_blocks(n), kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, (T*)nullptr, n, C, inv_m, ps);
+    const int blocks = ew_grid_for_channels(n, C, 0);
+    if (dx2) bn_bwd_apply_kernel<T, 1, true><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n, C, inv_m, ps);
+    else bn_bwd_apply_kernel<T, 1, false><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n, C, inv_m, ps);
   }
   return cudaGetLastError();
 }

@@ -42,16 +42,20 @@ def test_nonfinite_loss_is_reported_once_and_the_context_carries_on(precision):
     g.step(x, y, loss)
     g.sync()
     assert np.isfinite(loss.item())
-    bad = x.clone()
-    bad[0, 0, 0, 0] = float("nan")
-    g.step(bad, y, loss)
+    # A NaN in the classifier's bias makes the loss NaN.  (A NaN pixel would not: the ReLU kernels take
+    # max(x, 0) with the hardware's maximum, which returns the other operand for a NaN, so the first ReLU
+    # behind a poisoned batch norm turns it into zeros.)
+    good = S.init_params(0, 1, g.param_layout(1))
+    poisoned = good.copy()
+    poisoned[-1] = np.nan
+    g.set_params(1, poisoned)
+    g.step(x, y, loss)
     assert _status(g, g.sync) == 6                                  # FDG_ERR_NONFINITE
     assert "NaN" in g.lib.fdg_last_error(g.ctx).decode()
     assert _status(g, g.sync) == B.FDG_OK                           # reported once, then cleared
-    # the update that followed spread the NaN into the weights: a cold restart (parameters, momentum) recovers
-    for k in (1,):
-        g.set_params(k, S.init_params(0, k, g.param_layout(k)))
-        g.set_momentum(k, np.zeros(g.param_count(k), dtype=np.float32))
+    # the update that followed spread the NaN further: a cold restart (parameters, momentum) recovers
+    g.set_params(1, good)
+    g.set_momentum(1, np.zeros(g.param_count(1), dtype=np.float32))
     g.step(x, y, loss)
     assert _status(g, g.sync) == B.FDG_OK and np.isfinite(loss.item())
     g.close()
