@@ -125,6 +125,28 @@ def batchnorm_backward(dy, saved, gamma):
     return dx, dgamma, dbeta
 
 
+def batchnorm_running_update(running, x, momentum=0.1):
+    """Running statistics kept beside a training-mode batch norm for later inference.
+
+    The paper reports test errors (Tables 3-6), so its networks normalise test batches with
+    statistics gathered during training; it does not say how.  Reading taken: the exponential
+    running average of the framework its experiments ran on, momentum 0.1, started at mean 0 /
+    variance 1, fed with the batch mean and the UNBIASED batch variance (divisor M - 1):
+        running <- (1 - momentum) * running + momentum * batch statistic.
+    `running` = [mean, var], updated in place.
+    """
+    m = x.shape[0] * x.shape[1] * x.shape[2]
+    mean = x.mean(axis=(0, 1, 2))
+    var = ((x - mean) ** 2).sum(axis=(0, 1, 2)) / (m - 1)
+    running[0][:] = (1.0 - momentum) * running[0] + momentum * mean
+    running[1][:] = (1.0 - momentum) * running[1] + momentum * var
+
+
+def batchnorm_eval(x, gamma, beta, running, eps):
+    """Inference-mode batch norm: y = gamma * (x - running mean) / sqrt(running var + eps) + beta."""
+    return gamma * ((x - running[0]) / np.sqrt(running[1] + x.dtype.type(eps))) + beta
+
+
 # ----------------------------------------------------------------------------
 # ReLU
 # ----------------------------------------------------------------------------

@@ -71,14 +71,27 @@ class Stem:
             spec += [("bn.g", "bn_gamma", (self.co,)), ("bn.b", "bn_beta", (self.co,))]
         return spec
 
-    def forward(self, x, p):
+    def bn_spec(self):
+        """[(name, channels)] of the unit's batch norms, in the order their running statistics are kept."""
+        return [("bn", self.co)] if self.with_bn else []
+
+    def forward(self, x, p, running=None):
         q = self.q
         c = q(L.conv2d_forward(x, self.qw(p["conv.w"]), 1, 1))
         if not self.with_bn:
             return c, dict(x=x)
+        if running is not None:
+            L.batchnorm_running_update(running["bn"], c)
         b, sv = L.batchnorm_forward(c, p["bn.g"], p["bn.b"], self.eps)
         y = q(L.relu_forward(b))
         return y, dict(x=x, sv=sv, y=y)
+
+    def forward_eval(self, x, p, running):
+        q = self.q
+        c = q(L.conv2d_forward(x, self.qw(p["conv.w"]), 1, 1))
+        if not self.with_bn:
+            return c
+        return q(L.relu_forward(L.batchnorm_eval(c, p["bn.g"], p["bn.b"], running["bn"], self.eps)))
 
     def backward(self, dy, ctx, p):
         g = {}
@@ -111,7 +124,10 @@ class BasicBlock:
                      ("scbn.g", "bn_gamma", (self.co,)), ("scbn.b", "bn_beta", (self.co,))]
         return spec
 
-    def forward(self, x, p):
+    def bn_spec(self):
+        return [("bn1", self.co), ("bn2", self.co)] + ([("scbn", self.co)] if self.proj else [])
+
+    def forward(self, x, p, running=None):
         q, qw = self.q, self.qw
         c1 = q(L.conv2d_forward(x, qw(p["conv1.w"]), self.stride, 1))
         b1, sv1 = L.batchnorm_forward(c1, p["bn1.g"], p["bn1.b"], self.eps)
@@ -119,14 +135,32 @@ class BasicBlock:
         c2 = q(L.conv2d_forward(a1, qw(p["conv2.w"]), 1, 1))
         b2, sv2 = L.batchnorm_forward(c2, p["bn2.g"], p["bn2.b"], self.eps)
         ctx = dict(x=x, sv1=sv1, a1=a1, sv2=sv2)
+        if running is not None:
+            L.batchnorm_running_update(running["bn1"], c1)
+            L.batchnorm_running_update(running["bn2"], c2)
         if self.proj:
             cs = q(L.conv2d_forward(x, qw(p["sc.w"]), self.stride, 0))
             sc, ctx["svs"] = L.batchnorm_forward(cs, p["scbn.g"], p["scbn.b"], self.eps)
+            if running is not None:
+                L.batchnorm_running_update(running["scbn"], cs)
         else:
             sc = x
         y = q(L.relu_forward(b2 + sc))
         ctx["y"] = y
         return y, ctx
+
+    def forward_eval(self, x, p, running):
+        q, qw = self.q, self.qw
+        c1 = q(L.conv2d_forward(x, qw(p["conv1.w"]), self.stride, 1))
+        a1 = q(L.relu_forward(L.batchnorm_eval(c1, p["bn1.g"], p["bn1.b"], running["bn1"], self.eps)))
+        c2 = q(L.conv2d_forward(a1, qw(p["conv2.w"]), 1, 1))
+        b2 = L.batchnorm_eval(c2, p["bn2.g"], p["bn2.b"], running["bn2"], self.eps)
+        if self.proj:
+            cs = q(L.conv2d_forward(x, qw(p["sc.w"]), self.stride, 0))
+            sc = L.batchnorm_eval(cs, p["scbn.g"], p["scbn.b"], running["scbn"], self.eps)
+        else:
+            sc = x
+        return q(L.relu_forward(b2 + sc))
 
     def backward(self, dy, ctx, p):
         g = {}
@@ -167,11 +201,27 @@ class PreActBlock:
             spec += [("sc.w", "conv", (self.co, 1, 1, self.ci))]
         return spec
 
-    def forward(self, x, p):
+    def bn_spec(self):
+        return [("bn1", self.ci), ("bn2", self.co)]
+
+    def forward_eval(self, x, p, running):
         q, qw = self.q, self.qw
+        o = q(L.relu_forward(L.batchnorm_eval(x, p["bn1.g"], p["bn1.b"], running["bn1"], self.eps)))
+        c1 = q(L.conv2d_forward(o, qw(p["conv1.w"]), self.stride, 1))
+        a2 = q(L.relu_forward(L.batchnorm_eval(c1, p["bn2.g"], p["bn2.b"], running["bn2"], self.eps)))
+        c2 = L.conv2d_forward(a2, qw(p["conv2.w"]), 1, 1)
+        sc = q(L.conv2d_forward(o, qw(p["sc.w"]), self.stride, 0)) if self.proj else x
+        return q(c2 + sc)
+
+    def forward(self, x, p, running=None):
+        q, qw = self.q, self.qw
+        if running is not None:
+            L.batchnorm_running_update(running["bn1"], x)
         b1, sv1 = L.batchnorm_forward(x, p["bn1.g"], p["bn1.b"], self.eps)
         o = q(L.relu_forward(b1))
         c1 = q(L.conv2d_forward(o, qw(p["conv1.w"]), self.stride, 1))
+        if running is not None:
+            L.batchnorm_running_update(running["bn2"], c1)
         b2, sv2 = L.batchnorm_forward(c1, p["bn2.g"], p["bn2.b"], self.eps)
         a2 = q(L.relu_forward(b2))
         c2 = L.conv2d_forward(a2, qw(p["conv2.w"]), 1, 1)
@@ -217,9 +267,19 @@ class Head:
         spec += [("fc.w", "fc_w", (self.classes, self.feat)), ("fc.b", "fc_b", (self.classes,))]
         return spec
 
-    def forward_loss(self, x, labels, p):
+    def bn_spec(self):
+        return [("bn", self.feat)] if self.with_bn else []
+
+    def logits_eval(self, x, p, running):
+        if self.with_bn:
+            x = self.q(L.relu_forward(L.batchnorm_eval(x, p["bn.g"], p["bn.b"], running["bn"], self.eps)))
+        return L.fc_forward(L.gap_forward(x), p["fc.w"], p["fc.b"])
+
+    def forward_loss(self, x, labels, p, running=None):
         ctx = dict(shape=x.shape)
         if self.with_bn:
+            if running is not None:
+                L.batchnorm_running_update(running["bn"], x)
             b, ctx["sv"] = L.batchnorm_forward(x, p["bn.g"], p["bn.b"], self.eps)
             x = self.q(L.relu_forward(b))
             ctx["a"] = x
@@ -286,6 +346,12 @@ def module_param_spec(module_units):
         for name, kind, shape in u.param_spec():
             spec.append((u.name + "." + name, kind, shape))
     return spec
+
+
+def module_bn_spec(module_units):
+    """[(qualified name, channels)] of a module's batch norms; a module's flat vector of running statistics is,
+    for each of them in this order, the running mean then the running variance."""
+    return [(u.name + "." + name, ch) for u in module_units for name, ch in u.bn_spec()]
 
 
 def spec_size(spec):

@@ -25,13 +25,33 @@ class _Reader:
         return self.take(co, r, r, ci).permute(0, 3, 1, 2)      # -> [co, ci, r, r]
 
 
-def _bn(x, g, b, eps):
-    return F.batch_norm(x, None, None, g, b, training=True, momentum=0.0, eps=eps)
+class _Norms:
+    """Batch norms in network order.  buffers None: training mode without running statistics.  Otherwise a
+    list that is filled with [running_mean, running_var] tensors on first use (zeros / ones, as
+    torch.nn.BatchNorm2d starts them) and updated by torch itself in training mode (momentum 0.1), or read
+    in inference mode."""
+
+    def __init__(self, buffers, training):
+        self.buffers, self.training, self.i = buffers, training, 0
+
+    def __call__(self, x, g, b, eps):
+        if self.buffers is None:
+            return F.batch_norm(x, None, None, g, b, training=True, momentum=0.0, eps=eps)
+        if self.i == len(self.buffers):
+            self.buffers.append([torch.zeros(x.shape[1], dtype=x.dtype), torch.ones(x.shape[1], dtype=x.dtype)])
+        rm, rv = self.buffers[self.i]
+        self.i += 1
+        return F.batch_norm(x, rm, rv, g, b, training=self.training, momentum=0.1, eps=eps)
 
 
-def network_loss(arch, theta, images_nhwc, labels):
+def network_loss(arch, theta, images_nhwc, labels, buffers=None):
     """Mean softmax cross-entropy of the network `arch` with parameters `theta`
     (1-D torch tensor) on one batch.  images_nhwc: [B,H,W,C] tensor."""
+    return F.cross_entropy(network_logits(arch, theta, images_nhwc, buffers, True), labels.long())
+
+
+def network_logits(arch, theta, images_nhwc, buffers=None, training=True):
+    _bn = _Norms(buffers, training)
     rd = _Reader(theta)
     eps = arch.bn_eps
     x = images_nhwc.permute(0, 3, 1, 2)
@@ -73,7 +93,7 @@ def network_loss(arch, theta, images_nhwc, labels):
     x = x.mean(dim=(2, 3))
     logits = F.linear(x, rd.take(arch.num_classes, ci), rd.take(arch.num_classes))
     assert rd.off == theta.numel(), (rd.off, theta.numel())
-    return F.cross_entropy(logits, labels.long())
+    return logits
 
 
 def loss_and_grad(arch, theta_np, images_np, labels_np):
