@@ -168,6 +168,60 @@ fdg_status fdg_get_momentum(fdg_ctx* ctx, int module, float* dst, size_t n);
  * (Algorithm I takes gamma_t per iteration). */
 fdg_status fdg_set_lr(fdg_ctx* ctx, float lr);
 
+/* The learning-rate schedule of the experiments section: start at base_lr, multiply by `gamma` at each
+ * milestone epoch (150, 225, 275 with gamma 0.1 in the paper), and optionally run the first `warmup_epochs`
+ * epochs at `warmup_lr` (3 epochs at 0.01 for the deep networks and K = 3, 4).  Epoch e (from 0) holds
+ * iterations e*iters_per_epoch + 1 .. (e+1)*iters_per_epoch.  fdg_lr_at is the pure function;
+ * fdg_set_lr_schedule (NULL: off) makes every following fdg_step set gamma_t = fdg_lr_at(schedule, t) itself. */
+typedef struct {
+  int64_t iters_per_epoch;
+  float base_lr;
+  int n_milestones;            /* at most 8 */
+  int milestones[8];           /* ascending epochs */
+  float gamma;
+  int warmup_epochs;
+  float warmup_lr;
+} fdg_lr_schedule;
+fdg_status fdg_lr_at(const fdg_lr_schedule* schedule, int64_t iteration, float* out_lr);
+fdg_status fdg_set_lr_schedule(fdg_ctx* ctx, const fdg_lr_schedule* schedule);
+
+/* Running batch-norm statistics, kept for inference (the paper reports test errors, Tables 3-6, without saying
+ * how test batches are normalised; reading taken: exponential running average with momentum 0.1 of the batch
+ * mean and the unbiased batch variance, started at mean 0 / variance 1, updated by every training forward).
+ * Flat vector of a module: for each batch norm in network order (block: BN1, BN2, shortcut BN), its running
+ * mean [C] then its running variance [C].  Host or device memory; both calls block the host. */
+fdg_status fdg_bn_running_count(const fdg_ctx* ctx, int module, size_t* out_n);
+fdg_status fdg_get_bn_running(fdg_ctx* ctx, int module, float* dst, size_t n);
+fdg_status fdg_set_bn_running(fdg_ctx* ctx, int module, const float* src, size_t n);
+
+/* Inference: forwards one batch (fp32 [batch][in_h][in_w][in_c], device) through all K modules with their
+ * current weights and the running statistics, outside the training pipeline (nothing in flight is touched).
+ * `logits_dev` (nullable) receives fp32 [batch][num_classes]; `correct_dev` (nullable, needs `labels_dev`) is
+ * INCREMENTED by the number of samples whose largest logit is at their label (top-1; ties go to the lowest
+ * class), so a test set can be summed over batches.  Waits for the training work in flight first (blocks the
+ * host), then enqueues on `stream`. */
+fdg_status fdg_eval(fdg_ctx* ctx, fdg_stream stream, const float* images_dev, const int32_t* labels_dev,
+                    float* logits_dev, int* correct_dev);
+
+/* End of training.  After T iterations module k still holds 2(K-k) batches whose gradient has not arrived
+ * (Section 3.1: the backward of batch b reaches module k at iteration b + 2K - k - 1); the paper does not say
+ * what becomes of them.  fdg_drain runs the 2K - 2 further iterations of Algorithm I in which no new batch
+ * enters, so that every batch is back-propagated and applied by every module; `losses_dev` (nullable, device,
+ * 2K - 2 floats) receives the loss of the batch the top module handles in each of them (entries of
+ * iterations where it has none are left untouched).  Afterwards nothing is in flight and the iteration
+ * counter restarts at 0 with the trained weights, momentum and running statistics.  Blocks the host. */
+fdg_status fdg_drain(fdg_ctx* ctx, fdg_stream stream, float* losses_dev);
+
+/* Checkpoint of a run in flight: everything a continued run depends on (weights and their versions, momentum,
+ * activation FIFOs, mailboxes, label ring, running statistics, counters), so that fdg_load_state followed by
+ * the same inputs continues bit for bit.  `dst` / `src`: fdg_state_bytes bytes of host or device memory.
+ * A state can be loaded only into a context created with the same architecture and configuration
+ * (FDG_ERR_INVALID_ARG otherwise).  The learning rate is part of the state; a schedule is not (set it again).
+ * Both block the host. */
+fdg_status fdg_state_bytes(const fdg_ctx* ctx, size_t* out_bytes);
+fdg_status fdg_save_state(fdg_ctx* ctx, void* dst, size_t bytes);
+fdg_status fdg_load_state(fdg_ctx* ctx, const void* src, size_t bytes);
+
 /* One iteration of Algorithm I.  `images_dev` is batch t, fp32 [batch][in_h][in_w][in_c];
  * `labels_dev` int32 [batch] in [0, num_classes).  Both are read only by work enqueued
  * behind `stream` inside this call, so the caller may overwrite them as soon as `stream`

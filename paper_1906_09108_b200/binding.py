@@ -29,7 +29,9 @@ EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count"
            "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_wgrad_static", "fdg_conv_path",
            "fdg_get_saved_tensor_of", "fdg_capture_bytes", "fdg_capture_begin", "fdg_capture_end", "fdg_get_captured",
            "fdg_bn_scratch_bytes", "fdg_bn_stats", "fdg_bn_apply", "fdg_bn_backward", "fdg_shrink", "fdg_sgd_update",
-           "fdg_ingest", "fdg_head", "fdg_debug_raise_flag"]
+           "fdg_ingest", "fdg_head", "fdg_debug_raise_flag", "fdg_lr_at", "fdg_set_lr_schedule", "fdg_bn_running_count",
+           "fdg_get_bn_running", "fdg_set_bn_running", "fdg_eval", "fdg_drain", "fdg_state_bytes", "fdg_save_state",
+           "fdg_load_state"]
 
 
 class fdg_arch(C.Structure):
@@ -59,6 +61,16 @@ class fdg_conv_shape(C.Structure):
                 ("stride", C.c_int), ("pad", C.c_int)]
 
 
+class fdg_lr_schedule(C.Structure):
+    _fields_ = [("iters_per_epoch", C.c_int64), ("base_lr", C.c_float), ("n_milestones", C.c_int),
+                ("milestones", C.c_int * 8), ("gamma", C.c_float), ("warmup_epochs", C.c_int), ("warmup_lr", C.c_float)]
+
+
+def make_schedule(iters_per_epoch, base_lr=0.1, milestones=(150, 225, 275), gamma=0.1, warmup_epochs=0, warmup_lr=0.01):
+    ms = list(milestones) + [0] * (8 - len(milestones))
+    return fdg_lr_schedule(iters_per_epoch, base_lr, len(milestones), (C.c_int * 8)(*ms), gamma, warmup_epochs, warmup_lr)
+
+
 class fdg_conv_extra(C.Structure):
     _fields_ = [("share", C.c_int), ("wgrad_cta_cap", C.c_int), ("dy_spread", C.c_void_p), ("reduce", C.c_int),
                 ("next_mask", C.c_void_p), ("next_x", C.c_void_p), ("next_stats", C.c_void_p), ("partial", C.c_void_p),
@@ -71,6 +83,10 @@ FDG_CONV_PARTIAL_ROWS = 256
 class fdg_kernel_stat(C.Structure):
     _fields_ = [("name", C.c_char * 32), ("launches", C.c_uint64), ("total_ms", C.c_double), ("bytes", C.c_double),
                 ("flops", C.c_double)]
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
 
 
 def load_library(path=LIB_PATH):
@@ -110,6 +126,16 @@ def load_library(path=LIB_PATH):
         "fdg_conv_wgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, sz, P(fdg_conv_extra), vp, vp],
         "fdg_get_saved_tensor_of": [vp, C.c_int, C.c_int, C.c_int, i64, vp, sz, P(sz), P(i64)],
         "fdg_debug_raise_flag": [vp, C.c_int],
+        "fdg_lr_at": [P(fdg_lr_schedule), i64, P(C.c_float)],
+        "fdg_set_lr_schedule": [vp, P(fdg_lr_schedule)],
+        "fdg_bn_running_count": [vp, C.c_int, P(sz)],
+        "fdg_get_bn_running": [vp, C.c_int, vp, sz],
+        "fdg_set_bn_running": [vp, C.c_int, vp, sz],
+        "fdg_eval": [vp, vp, vp, vp, vp, vp],
+        "fdg_drain": [vp, vp, vp],
+        "fdg_state_bytes": [vp, P(sz)],
+        "fdg_save_state": [vp, vp, sz],
+        "fdg_load_state": [vp, vp, sz],
         "fdg_capture_bytes": [vp, C.c_int, P(sz)],
         "fdg_capture_begin": [vp, C.c_int, vp, sz],
         "fdg_capture_end": [vp, C.c_int],
@@ -239,6 +265,45 @@ class FDG:
     def set_lr(self, lr):
         self._check(self.lib.fdg_set_lr(self.ctx, lr), self.ctx)
 
+    def set_lr_schedule(self, schedule):
+        """schedule: fdg_lr_schedule (see make_schedule) or None to switch it off."""
+        self._schedule = schedule
+        self._check(self.lib.fdg_set_lr_schedule(self.ctx, C.byref(schedule) if schedule is not None else None), self.ctx)
+
+    def get_running(self, k):
+        n = C.c_size_t()
+        self._check(self.lib.fdg_bn_running_count(self.ctx, k, C.byref(n)), self.ctx)
+        out = np.empty(n.value, dtype=np.float32)
+        if n.value:
+            self._check(self.lib.fdg_get_bn_running(self.ctx, k, out.ctypes.data, out.size), self.ctx)
+        return out
+
+    def set_running(self, k, flat):
+        flat = np.ascontiguousarray(flat, dtype=np.float32)
+        if flat.size:
+            self._check(self.lib.fdg_set_bn_running(self.ctx, k, flat.ctypes.data, flat.size), self.ctx)
+
+    def eval(self, images_dev, labels_dev=None, logits_dev=None, correct_dev=None, stream=None):
+        """Inference forward of one batch; correct_dev (int32 CUDA tensor of one element) is incremented."""
+        st = self.torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self._check(self.lib.fdg_eval(self.ctx, st, images_dev.data_ptr(), _ptr(labels_dev), _ptr(logits_dev),
+                                      _ptr(correct_dev)), self.ctx)
+
+    def drain(self, losses_dev=None, stream=None):
+        st = self.torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self._check(self.lib.fdg_drain(self.ctx, st, _ptr(losses_dev)), self.ctx)
+
+    def save_state(self):
+        """The run's state as a pinned-size CPU uint8 tensor (fdg_save_state to host memory)."""
+        n = C.c_size_t()
+        self._check(self.lib.fdg_state_bytes(self.ctx, C.byref(n)), self.ctx)
+        blob = self.torch.empty(n.value, dtype=self.torch.uint8)
+        self._check(self.lib.fdg_save_state(self.ctx, blob.data_ptr(), n.value), self.ctx)
+        return blob
+
+    def load_state(self, blob):
+        self._check(self.lib.fdg_load_state(self.ctx, blob.data_ptr(), blob.numel()), self.ctx)
+
     # ---- stepping -------------------------------------------------------------
     def step(self, images_dev, labels_dev, loss_dev=None, stream=None):
         """images_dev: float32 CUDA tensor [B,H,W,C]; labels_dev: int32 CUDA tensor [B]."""
@@ -349,9 +414,6 @@ class FDG:
 
 
 # ---- operator level (include/fdg_ops.h): thin wrappers over torch CUDA tensors -----------
-def _ptr(t):
-    return None if t is None else t.data_ptr()
-
 
 class ConvOps:
     """fdg_conv_* on torch CUDA tensors of the precision's storage type (float32 / bfloat16)."""

@@ -397,15 +397,23 @@ inline cudaError_t conv_tc_make_maps(const ConvTcParams& p, const void* act, con
   return cudaSuccess;
 }
 
+// The kernel's dynamic shared memory exceeds the default limit: raised once (also callable up front, so
+// that the first launch may happen inside a stream capture).
+inline cudaError_t conv_tc_set_attrs() {
+  static bool attr_set = false;
+  if (attr_set) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e == cudaSuccess) attr_set = true;
+  return e;
+}
+
 inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const CUtensorMap& map_a,
                                   const CUtensorMap& map_b, __nv_bfloat16* out, const __nv_bfloat16* res,
                                   const __nv_bfloat16* res_mask, int* error_word, int sm_count) {
-  static bool attr_set = false;
   const size_t smem = conv_tc_smem_bytes(p);
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  {
+    cudaError_t e = conv_tc_set_attrs();
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   const int tiles = p.m_tiles * p.n_tiles;
   const int grid = tiles < sm_count ? tiles : sm_count;

@@ -56,6 +56,19 @@ __device__ __forceinline__ void store_vec(T* __restrict__ p, const float (&in)[V
   }
 }
 
+// Running statistics of a batch norm, kept for inference beside the batch statistics of training:
+// running[0..C) mean, running[C..2C) variance; each forward folds in the batch mean and the unbiased batch
+// variance with weight `momentum` (null pointer: not kept).
+struct RunningStats {
+  float* running;
+  float momentum;
+  float unbias;      // M / (M - 1) for M values per channel
+};
+__device__ __forceinline__ void update_running(const RunningStats& r, int C, int c, float mean, float biased_var) {
+  r.running[c] = (1.f - r.momentum) * r.running[c] + r.momentum * mean;
+  r.running[C + c] = (1.f - r.momentum) * r.running[C + c] + r.momentum * (biased_var * r.unbias);
+}
+
 constexpr int kRedThreads = 256;      // threads per block of the channel-reduction kernels
 // Blocks of a channel reduction.  The last block to finish adds all blocks' partial sums, a serial
 // tail that grows with the block count; with the row loop keeping four loads in flight per thread,
@@ -177,7 +190,7 @@ __device__ __forceinline__ void channel_reduce(const RedGeom g, float* __restric
 template <typename T, int VEC>
 __global__ void __launch_bounds__(kRedThreads)
 bn_stats_kernel(const T* __restrict__ x, RedGeom g, float eps, float* __restrict__ stats,
-                float* __restrict__ partial, unsigned int* __restrict__ counter) {
+                float* __restrict__ partial, unsigned int* __restrict__ counter, RunningStats run) {
   const int C = g.C;
   const double inv_m = 1.0 / (double)g.rows;
   channel_reduce<2, VEC>(
@@ -194,6 +207,7 @@ bn_stats_kernel(const T* __restrict__ x, RedGeom g, float eps, float* __restrict
         if (var < 0.0) var = 0.0;
         stats[c] = (float)mean;
         stats[C + c] = (float)(1.0 / sqrt(var + (double)eps));
+        if (run.running) update_running(run, C, c, (float)mean, (float)var);
       });
 }
 
@@ -210,6 +224,7 @@ struct PartialSums {
   float inv_count, eps;     // kind 1
   float* save0;             // block 0 stores out2c[0..C) here (kind 1: with save1 contiguous = stats[2C]; kind 2: dbeta)
   float* save1;             // and out2c[C..2C) here (kind 2: dgamma)
+  RunningStats run;         // kind 1: block 0 also folds the batch statistics into the running ones
 };
 constexpr int kEwThreads = 256;
 
@@ -242,6 +257,7 @@ __device__ __forceinline__ void finalize_partials(const PartialSums ps, int C, f
       double var = s1 * (double)ps.inv_count - mean * mean;
       if (var < 0.0) var = 0.0;
       o0 = (float)mean; o1 = (float)(1.0 / sqrt(var + (double)ps.eps));
+      if (blockIdx.x == 0 && ps.run.running) update_running(ps.run, C, tid, (float)mean, (float)var);
     } else {
       o0 = (float)s0; o1 = (float)s1;
     }
@@ -642,6 +658,52 @@ __global__ void cast_kernel(const float* __restrict__ in, T* __restrict__ out, s
     out[i] = from_f<T>(in[i]);
 }
 
+// ------------------------------------------------------------- inference ----
+// Inference-mode statistics of all batch norms of a module in one launch: for table entry e,
+// out[soff .. soff+C) = running mean, out[soff+C .. soff+2C) = 1/sqrt(running variance + eps).
+struct EvalStatEntry { size_t roff, soff; int C; };
+__global__ void bn_eval_stats_kernel(const float* __restrict__ running, float* __restrict__ out,
+                                     const EvalStatEntry* __restrict__ table, float eps) {
+  const EvalStatEntry e = table[blockIdx.x];
+  for (int c = threadIdx.x; c < e.C; c += blockDim.x) {
+    out[e.soff + c] = running[e.roff + c];
+    out[e.soff + e.C + c] = 1.f / sqrtf(running[e.roff + e.C + c] + eps);
+  }
+}
+
+// Classifier in inference mode, one block per sample: global average pool -> FC -> logits (optional copy
+// out) -> arg-max (lowest index among equal logits) compared with the label; *correct counts the matches.
+template <typename T>
+__global__ void head_eval_kernel(const T* __restrict__ x, const float* __restrict__ w, const float* __restrict__ b,
+                                 const int32_t* __restrict__ labels, int HW, int F, int classes,
+                                 float* __restrict__ logits_out, int* __restrict__ correct) {
+  extern __shared__ float hs[];            // pooled[F] | logits[classes]
+  float* s_pool = hs;
+  float* s_logit = hs + F;
+  const int n = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+  const T* xn = x + (size_t)n * HW * F;
+  for (int f = tid; f < F; f += nt) {
+    float a = 0.f;
+    for (int p = 0; p < HW; ++p) a += to_f(xn[(size_t)p * F + f]);
+    s_pool[f] = a / (float)HW;
+  }
+  __syncthreads();
+  const int warp = tid >> 5, lane = tid & 31, nwarps = nt >> 5;
+  for (int c = warp; c < classes; c += nwarps) {
+    float a = 0.f;
+    for (int f = lane; f < F; f += 32) a += w[(size_t)c * F + f] * s_pool[f];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) { s_logit[c] = a + b[c]; if (logits_out) logits_out[(size_t)n * classes + c] = a + b[c]; }
+  }
+  __syncthreads();
+  if (tid == 0 && labels && correct) {
+    int best = 0;
+    for (int c = 1; c < classes; ++c) if (s_logit[c] > s_logit[best]) best = c;
+    if (best == labels[n]) atomicAdd(correct, 1);
+  }
+}
+
 // ---------------------------------------------------------- host launchers ---
 // Shared by the module runtime and the operator-level entry points, so that both issue the same
 // kernels in the same launch shapes.
@@ -658,14 +720,15 @@ inline size_t red_scratch_floats(int C) { return (size_t)kRedMaxBlocks * kRedMax
 // (the kernel leaves it zero again).
 template <typename T>
 inline cudaError_t launch_bn_stats(cudaStream_t st, const T* x, size_t rows, int C, float eps, float* stats,
-                                   float* scratch, unsigned int* counter) {
+                                   float* scratch, unsigned int* counter, float* running = nullptr, float momentum = 0.f) {
   constexpr int V = full_vec<T>();
+  const RunningStats run{running, momentum, rows > 1 ? (float)((double)rows / (double)(rows - 1)) : 1.f};
   if (C % V == 0) {
     RedGeom g = red_geom((int)rows, C, V);
-    bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * C * 4, st>>>(x, g, eps, stats, scratch, counter);
+    bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * C * 4, st>>>(x, g, eps, stats, scratch, counter, run);
   } else {
     RedGeom g = red_geom((int)rows, C, 1);
-    bn_stats_kernel<T, 1><<<g.blocks, kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * C * 4, st>>>(x, g, eps, stats, scratch, counter);
+    bn_stats_kernel<T, 1><<<g.blocks, kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * C * 4, st>>>(x, g, eps, stats, scratch, counter, run);
   }
   return cudaGetLastError();
 }
@@ -690,7 +753,7 @@ template <typename T>
 inline cudaError_t launch_bn_apply(cudaStream_t st, const T* x, float* stats, const float* gamma, const float* beta,
                                    const T* res, const float* res_stats, const float* res_gamma, const float* res_beta,
                                    bool relu, T* y, size_t rows, int C, float eps, const float* partial, int nparts,
-                                   int block_cap) {
+                                   int block_cap, float* running = nullptr, float momentum = 0.f) {
   constexpr int V = full_vec<T>();
   const size_t n = rows * C;
   PartialSums ps{};
@@ -698,6 +761,7 @@ inline cudaError_t launch_bn_apply(cudaStream_t st, const T* x, float* stats, co
     if (2 * C > kEwThreads) return cudaErrorInvalidValue;
     ps.partial = partial; ps.nparts = nparts; ps.kind = 1; ps.inv_count = 1.f / (float)rows; ps.eps = eps;
     ps.save0 = stats; ps.save1 = stats + C;
+    ps.run = RunningStats{running, momentum, rows > 1 ? (float)((double)rows / (double)(rows - 1)) : 1.f};
   }
   if (C % V == 0) {
     const int blocks = ew_grid_for_channels(n / V, C / V, ps.partial ? block_cap : 0);

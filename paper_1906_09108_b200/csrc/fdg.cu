@@ -35,6 +35,7 @@ typedef __nv_bfloat16 bf16;
 constexpr int kEventRing = 4;
 constexpr size_t kLogIterations = 4096;
 constexpr int kRedPartialCtas = 256;                 // upper bound of the CTAs of one convolution launch
+constexpr float kBnMomentum = 0.1f;                  // weight of the newest batch in the running statistics
 
 enum UnitType { U_STEM, U_BASIC, U_PREACT, U_HEAD };
 
@@ -64,6 +65,8 @@ struct Unit {
   size_t st1, st2, sts;
   // offsets of the flipped copies of w1 / w2 inside a wflip16 slot, or -1 when that conv's dgrad is not on tensor cores
   long long f1 = -1, f2 = -1;
+  // offsets of the running statistics (mean[C], var[C]) of BN1 / BN2 / the shortcut BN in the module's vector, or -1
+  long long r1 = -1, r2 = -1, rs = -1;
 };
 
 struct Module {
@@ -109,6 +112,11 @@ struct Module {
   cudaStream_t stream2 = nullptr;          // side stream: weight gradients run beside the data-gradient chain
   cudaEvent_t ev_fork2 = nullptr, ev_join2 = nullptr, ev_buf[4] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t ev_act[kEventRing], ev_grad[kEventRing];
+  // running batch-norm statistics (inference): flat vector, and the table the inference pass reads them through
+  float* running = nullptr;
+  size_t n_running = 0;
+  std::vector<EvalStatEntry> eval_table;
+  EvalStatEntry* eval_table_dev = nullptr;
   // gradient capture (fdg_capture_begin): where each gradient tensor of a backward pass is copied to
   std::vector<CaptureEntry> cap_table;
   size_t cap_elems = 0;
@@ -139,6 +147,11 @@ struct fdg_ctx {
   int32_t* host_labels = nullptr;
   size_t staging_elems = 0;
   int64_t t = 0;
+  int64_t last_batch = INT64_MAX;     // no batch beyond this one exists (set while draining)
+  bool has_schedule = false;
+  fdg_lr_schedule schedule;
+  char* ws_base = nullptr;            // the caller's workspace, as carved
+  size_t ws_bytes = 0;
   float lr = 0.f;
   uint64_t launches = 0;
   std::vector<fdg_sched_entry> log;
@@ -236,6 +249,12 @@ static void add_param(Module& m, int kind, int unit, int d0, int d1, int d2, int
   m.layout.push_back(e);
 }
 
+static long long add_running(Module& m, int C) {
+  const long long off = (long long)m.n_running;
+  m.n_running += (size_t)2 * C;
+  return off;
+}
+
 // Builds the unit lists, parameter tables and slot layouts of all modules (no pointers yet).
 static void plan_modules(fdg_ctx* c) {
   const fdg_arch& a = c->arch;
@@ -255,7 +274,7 @@ static void plan_modules(fdg_ctx* c) {
     Unit u{}; u.type = U_STEM; u.index = 0; u.ci = in_c_store; u.co = a.stem_width; u.stride = 1; u.bn = !wrn;
     u.H = H; u.W = W; u.P = H; u.Q = W;
     add_param(m, FDG_PARAM_CONV, 0, u.co, 3, 3, a.in_c, &u.w1);
-    if (u.bn) { add_param(m, FDG_PARAM_BN_GAMMA, 0, u.co, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, 0, u.co, 1, 1, 1, &u.b1); }
+    if (u.bn) { add_param(m, FDG_PARAM_BN_GAMMA, 0, u.co, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, 0, u.co, 1, 1, 1, &u.b1); u.r1 = add_running(m, u.co); }
     m.units.push_back(u);
     m.in_h = H; m.in_w = W; m.in_c = in_c_store; m.in_c_logical = a.in_c;
   }
@@ -277,12 +296,15 @@ static void plan_modules(fdg_ctx* c) {
         add_param(m, FDG_PARAM_CONV, b, u.co, 1, 1, u.ci, &u.ws);
         add_param(m, FDG_PARAM_BN_GAMMA, b, u.co, 1, 1, 1, &u.gs); add_param(m, FDG_PARAM_BN_BETA, b, u.co, 1, 1, 1, &u.bs);
       }
+      u.r1 = add_running(m, u.co); u.r2 = add_running(m, u.co);
+      if (u.proj) u.rs = add_running(m, u.co);
     } else {
       add_param(m, FDG_PARAM_BN_GAMMA, b, u.ci, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, b, u.ci, 1, 1, 1, &u.b1);
       add_param(m, FDG_PARAM_CONV, b, u.co, 3, 3, u.ci, &u.w1);
       add_param(m, FDG_PARAM_BN_GAMMA, b, u.co, 1, 1, 1, &u.g2); add_param(m, FDG_PARAM_BN_BETA, b, u.co, 1, 1, 1, &u.b2);
       add_param(m, FDG_PARAM_CONV, b, u.co, 3, 3, u.co, &u.w2);
       if (u.proj) add_param(m, FDG_PARAM_CONV, b, u.co, 1, 1, u.ci, &u.ws);
+      u.r1 = add_running(m, u.ci); u.r2 = add_running(m, u.co);
     }
     m.units.push_back(u);
     H = u.P; W = u.Q; ci = u.co;
@@ -290,7 +312,7 @@ static void plan_modules(fdg_ctx* c) {
   {   // head
     Module& m = c->mods[K - 1];
     Unit u{}; u.type = U_HEAD; u.index = -1; u.ci = ci; u.co = a.num_classes; u.bn = wrn; u.H = H; u.W = W; u.P = 1; u.Q = 1; u.stride = 1;
-    if (u.bn) { add_param(m, FDG_PARAM_BN_GAMMA, -1, ci, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, -1, ci, 1, 1, 1, &u.b1); }
+    if (u.bn) { add_param(m, FDG_PARAM_BN_GAMMA, -1, ci, 1, 1, 1, &u.g1); add_param(m, FDG_PARAM_BN_BETA, -1, ci, 1, 1, 1, &u.b1); u.r1 = add_running(m, ci); }
     add_param(m, FDG_PARAM_FC_W, -1, a.num_classes, ci, 1, 1, &u.w1);
     add_param(m, FDG_PARAM_FC_B, -1, a.num_classes, 1, 1, 1, &u.w2);
     m.units.push_back(u);
@@ -374,6 +396,12 @@ static void plan_modules(fdg_ctx* c) {
       m.flip_elems = fe;
     }
     m.slot_elems = te; m.slot_floats = tf; m.max_act = maxa; m.scratch_floats = scr; m.wscratch_floats = wscr;
+    for (const Unit& u : m.units) {     // where the inference pass finds each batch norm's statistics
+      const int c1 = (u.type == U_PREACT || u.type == U_HEAD) ? u.ci : u.co;
+      if (u.r1 >= 0) m.eval_table.push_back(EvalStatEntry{(size_t)u.r1, u.st1, c1});
+      if (u.r2 >= 0) m.eval_table.push_back(EvalStatEntry{(size_t)u.r2, u.st2, u.co});
+      if (u.rs >= 0) m.eval_table.push_back(EvalStatEntry{(size_t)u.rs, u.sts, u.co});
+    }
     {   // the gradient tensors a capture keeps (fdg_capture_begin), one region each
       size_t ce = 0;
       auto cap = [&](int ui, int which, size_t e, int ch) { m.cap_table.push_back(CaptureEntry{ui, which, ch, ce, e}); ce += align_up(e, 128); };
@@ -419,9 +447,12 @@ static size_t carve(fdg_ctx* c, char* base) {
     m.wver16 = c->bf16_mode ? cv.take<bf16>((size_t)m.Dw * align_up(m.n_params, 64) * 2) : nullptr;
     m.wflip16 = m.flip_elems ? cv.take<bf16>((size_t)m.Dw * m.flip_elems * 2) : nullptr;
     m.flip_table_dev = m.flip_table.empty() ? nullptr : cv.take<tc::FlipEntry>(m.flip_table.size() * sizeof(tc::FlipEntry));
-    m.fifo = cv.take<char>((size_t)m.D * m.slot_elems * es);
-    m.fifo_f = cv.take<float>((size_t)m.D * std::max<size_t>(m.slot_floats, 64) * 4);
-    m.in_ring = m.Din ? cv.take<char>((size_t)m.Din * align_up(m.in_elems, 128) * es) : nullptr;
+    // one slot beyond the FIFO's (and the image ring's) own: the inference pass works there
+    m.fifo = cv.take<char>((size_t)(m.D + 1) * m.slot_elems * es);
+    m.fifo_f = cv.take<float>((size_t)(m.D + 1) * std::max<size_t>(m.slot_floats, 64) * 4);
+    m.in_ring = m.Din ? cv.take<char>((size_t)(m.Din + 1) * align_up(m.in_elems, 128) * es) : nullptr;
+    m.running = cv.take<float>(std::max<size_t>(m.n_running, 64) * 4);
+    m.eval_table_dev = m.eval_table.empty() ? nullptr : cv.take<EvalStatEntry>(m.eval_table.size() * sizeof(EvalStatEntry));
     m.mail = m.k >= 2 ? cv.take<char>((size_t)c->mail_ring * align_up(m.in_elems, 128) * es) : nullptr;
     for (int i = 0; i < 6; ++i) m.temps[i] = cv.take<char>(align_up(m.max_act, 128) * es);
     m.scratch = cv.take<float>(std::max<size_t>(m.scratch_floats, 64) * 4);
@@ -478,10 +509,12 @@ struct Launch {
   void note(cudaError_t e) { if (err == cudaSuccess) err = e; end_events(); }
 };
 
+// `run`: offset of this batch norm's running statistics in the module's vector (the kernel that forms the
+// batch statistics also folds them into the running ones).
 template <typename T>
-static void bn_stats(Launch& L, Module& m, const T* x, size_t rows, int C, float eps, float* stats) {
+static void bn_stats(Launch& L, Module& m, const T* x, size_t rows, int C, float eps, float* stats, long long run) {
   L.begin(KC_BN_STATS, (double)rows * C * sizeof(T), 3.0 * rows * C);
-  L.note(launch_bn_stats<T>(L.st, x, rows, C, eps, stats, m.scratch, m.counter));
+  L.note(launch_bn_stats<T>(L.st, x, rows, C, eps, stats, m.scratch, m.counter, run >= 0 ? m.running + run : nullptr, kBnMomentum));
   ++L.c->launches;
 }
 
@@ -490,11 +523,12 @@ static void bn_stats(Launch& L, Module& m, const T* x, size_t rows, int C, float
 template <typename T>
 static void bn_apply(Launch& L, Module& m, const T* x, float* stats, const float* gamma, const float* beta, const T* res,
                      const float* res_stats, const float* res_gamma, const float* res_beta, bool relu, T* y,
-                     size_t rows, int C, int nparts = 0) {
+                     size_t rows, int C, int nparts = 0, long long run = -1) {
   const size_t n = rows * C;
   L.begin(KC_BN_APPLY, (double)n * sizeof(T) * (res ? 3 : 2), 6.0 * n);
   L.note(launch_bn_apply<T>(L.st, x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, rows, C,
-                            L.c->arch.bn_eps, nparts > 0 ? m.red_partial : nullptr, nparts, L.c->ew_block_cap));
+                            L.c->arch.bn_eps, nparts > 0 ? m.red_partial : nullptr, nparts, L.c->ew_block_cap,
+                            (nparts > 0 && run >= 0) ? m.running + run : nullptr, kBnMomentum));
   ++L.c->launches;
 }
 
@@ -613,32 +647,41 @@ template <typename T> static T* slot_T(const Module& m, int slot) { return reint
 static float* slot_F(const Module& m, int slot) { return m.fifo_f + (size_t)slot * std::max<size_t>(m.slot_floats, 64); }
 
 // Input tensor of module m for batch tau: the image ring (module 1) or the upstream module's FIFO slot.
+// `eval`: the inference pass reads the extra slot behind each ring instead of batch tau's.
 template <typename T>
-static const T* module_input(fdg_ctx* c, const Module& m, int64_t tau) {
-  if (m.k == 1) return reinterpret_cast<const T*>(m.in_ring) + (size_t)(tau % m.Din) * align_up(m.in_elems, 128);
+static const T* module_input(fdg_ctx* c, const Module& m, int64_t tau, bool eval = false) {
+  if (m.k == 1) return reinterpret_cast<const T*>(m.in_ring) + (size_t)(eval ? m.Din : tau % m.Din) * align_up(m.in_elems, 128);
   const Module& up = c->mods[m.k - 2];
-  return slot_T<T>(up, (int)(tau % up.D)) + up.units.back().t_y;
+  return slot_T<T>(up, eval ? up.D : (int)(tau % up.D)) + up.units.back().t_y;
 }
 
+// Forward of the module's units into FIFO slot `slot` with weight version `vslot`.  Training (`eval` false):
+// batch statistics, formed in the convolution epilogues where the kernel can, saved for the backward and
+// folded into the running statistics.  Inference (`eval` true): the statistics of every batch norm were put
+// into the slot beforehand from the running ones (bn_eval_stats_kernel), nothing is reduced.
 template <typename T>
-static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int slot, int vslot) {
+static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int slot, int vslot, bool eval = false) {
   const int B = c->arch.batch;
   const float eps = c->arch.bn_eps;
   const T* wt = weights_of<T>(m, vslot);
   const float* wf = m.wver + (size_t)vslot * align_up(m.n_params, 64);
   T* S = slot_T<T>(m, slot);
   float* F = slot_F(m, slot);
-  const T* x = module_input<T>(c, m, tau);
+  const T* x = module_input<T>(c, m, tau, eval);
   T* tmp = reinterpret_cast<T*>(m.temps[2]);
+  // statistics of a convolution output y that left `np` rows of partial sums (0: reduce y now)
+  auto stats_of = [&](int np, const T* y, size_t rows, int C, float* stats, long long run) {
+    if (!eval && !np) bn_stats<T>(L, m, y, rows, C, eps, stats, run);
+  };
   for (const Unit& u : m.units) {
     const size_t rows_in = (size_t)B * u.H * u.W, rows_out = (size_t)B * u.P * u.Q;
     switch (u.type) {
       case U_STEM: {
         ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
         if (u.bn) {
-          const int np = conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_a, nullptr, true);
-          if (!np) bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
-          bn_apply<T>(L, m, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np);
+          const int np = conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_a, nullptr, !eval);
+          stats_of(np, S + u.t_a, rows_out, u.co, F + u.st1, u.r1);
+          bn_apply<T>(L, m, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np, u.r1);
         } else {
           conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_y, nullptr);
         }
@@ -647,30 +690,30 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
       case U_BASIC: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
-        const int np1 = conv_fprop<T>(L, m, g1, x, wt + u.w1, S + u.t_a, nullptr, true);               // c1
-        if (!np1) bn_stats<T>(L, m, S + u.t_a, rows_out, u.co, eps, F + u.st1);
-        bn_apply<T>(L, m, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_b, rows_out, u.co, np1);  // a1
+        const int np1 = conv_fprop<T>(L, m, g1, x, wt + u.w1, S + u.t_a, nullptr, !eval);               // c1
+        stats_of(np1, S + u.t_a, rows_out, u.co, F + u.st1, u.r1);
+        bn_apply<T>(L, m, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_b, rows_out, u.co, np1, u.r1);  // a1
         if (u.proj) {          // shortcut first: its statistics must not disturb the partial sums conv2 leaves for BN2
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_fprop<T>(L, m, gs, x, wt + u.ws, S + u.t_s, nullptr);                                   // cs
-          bn_stats<T>(L, m, S + u.t_s, rows_out, u.co, eps, F + u.sts);
+          stats_of(0, S + u.t_s, rows_out, u.co, F + u.sts, u.rs);
         }
-        const int np2 = conv_fprop<T>(L, m, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr, true);       // c2
-        if (!np2) bn_stats<T>(L, m, S + u.t_c, rows_out, u.co, eps, F + u.st2);
+        const int np2 = conv_fprop<T>(L, m, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr, !eval);       // c2
+        stats_of(np2, S + u.t_c, rows_out, u.co, F + u.st2, u.r2);
         if (u.proj)
-          bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, S + u.t_s, F + u.sts, wf + u.gs, wf + u.bs, true, S + u.t_y, rows_out, u.co, np2);
+          bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, S + u.t_s, F + u.sts, wf + u.gs, wf + u.bs, true, S + u.t_y, rows_out, u.co, np2, u.r2);
         else
-          bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, x, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np2);
+          bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, x, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np2, u.r2);
         break;
       }
       case U_PREACT: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
-        bn_stats<T>(L, m, x, rows_in, u.ci, eps, F + u.st1);
+        stats_of(0, x, rows_in, u.ci, F + u.st1, u.r1);
         bn_apply<T>(L, m, x, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows_in, u.ci);   // o
-        const int np = conv_fprop<T>(L, m, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr, true);        // c1
-        if (!np) bn_stats<T>(L, m, S + u.t_b, rows_out, u.co, eps, F + u.st2);
-        bn_apply<T>(L, m, S + u.t_b, F + u.st2, wf + u.g2, wf + u.b2, nullptr, nullptr, nullptr, nullptr, true, S + u.t_c, rows_out, u.co, np); // a2
+        const int np = conv_fprop<T>(L, m, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr, !eval);        // c1
+        stats_of(np, S + u.t_b, rows_out, u.co, F + u.st2, u.r2);
+        bn_apply<T>(L, m, S + u.t_b, F + u.st2, wf + u.g2, wf + u.b2, nullptr, nullptr, nullptr, nullptr, true, S + u.t_c, rows_out, u.co, np, u.r2); // a2
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_fprop<T>(L, m, gs, S + u.t_a, wt + u.ws, tmp, nullptr);
@@ -681,10 +724,31 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
         break;
       }
       case U_HEAD:
-        break;      // handled by head_forward_backward
+        break;      // handled by head_forward_backward / head_eval
     }
     if (u.type != U_HEAD) x = S + u.t_y;
   }
+}
+
+// Module K, inference: [BN + ReLU,] global average pool, FC, arg-max against the labels.
+template <typename T>
+static void head_eval(fdg_ctx* c, Module& m, Launch& L, int slot, int vslot, const int32_t* labels_dev, float* logits_dev,
+                      int* correct_dev) {
+  const Unit& u = m.units.back();
+  const int B = c->arch.batch, F = u.ci, classes = u.co, HW = u.H * u.W;
+  const float* wf = m.wver + (size_t)vslot * align_up(m.n_params, 64);
+  T* S = slot_T<T>(m, slot);
+  float* Fs = slot_F(m, slot);
+  const T* x = m.units.size() >= 2 ? S + m.units[m.units.size() - 2].t_y : module_input<T>(c, m, 0, true);
+  const T* feat = x;
+  if (u.bn) {
+    bn_apply<T>(L, m, x, Fs + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, (size_t)B * HW, F);
+    feat = S + u.t_a;
+  }
+  L.begin(KC_HEAD, (double)B * HW * F * sizeof(T), 2.0 * B * F * classes);
+  head_eval_kernel<T><<<B, 128, (size_t)(F + classes) * 4, L.st>>>(feat, wf + u.w1, wf + u.w2, labels_dev, HW, F, classes,
+                                                                  logits_dev, correct_dev);
+  L.check();
 }
 
 // Module K only: classifier, loss and their backward; leaves the gradient of the last block's
@@ -700,7 +764,7 @@ static void head_forward_backward(fdg_ctx* c, Module& m, Launch& L, int64_t tau,
   const size_t rows = (size_t)B * HW;
   const T* feat = x;
   if (u.bn) {
-    bn_stats<T>(L, m, x, rows, F, c->arch.bn_eps, Fs + u.st1);
+    bn_stats<T>(L, m, x, rows, F, c->arch.bn_eps, Fs + u.st1, u.r1);
     bn_apply<T>(L, m, x, Fs + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows, F);
     feat = S + u.t_a;
   }
@@ -929,7 +993,7 @@ static cudaError_t module_step(fdg_ctx* c, Module& m, cudaStream_t st, StepMode 
     L.note(cudaStreamWaitEvent(st, c->mods[k].ev_grad[e_prev], 0));
   };
   auto do_forward = [&]() {
-    if (tau_f < 1) return;
+    if (tau_f < 1 || tau_f > c->last_batch) return;
     const int slot = (int)(tau_f % m.D), vslot = (int)(m.updates % m.Dw);
     if (enqueue) forward_module<T>(c, m, L, tau_f, slot, vslot);
     m.slot_version[slot] = m.updates; m.slot_batch[slot] = tau_f;
@@ -938,7 +1002,7 @@ static cudaError_t module_step(fdg_ctx* c, Module& m, cudaStream_t st, StepMode 
     if (k < K) { m.last_out_batch = tau_f; m.last_out_slot = slot; }
   };
   auto do_backward_update = [&]() {
-    if (tau_b < 1) return;
+    if (tau_b < 1 || tau_b > c->last_batch) return;
     const int slot = (int)(tau_b % m.D);
     const int64_t ver = (c->cfg.weight_reading == FDG_STASHED) ? m.slot_version[slot] : m.updates;
     const int vslot = (int)(ver % m.Dw);
@@ -1085,9 +1149,23 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) { delete c; return FDG_ERR_CUDA; }
   carve(c, static_cast<char*>(dev_workspace));
-  for (Module& m : c->mods)
+  c->ws_base = static_cast<char*>(dev_workspace);
+  c->ws_bytes = need;
+  for (Module& m : c->mods) {
     if (m.flip_table_dev && e == cudaSuccess)
       e = cudaMemcpy(m.flip_table_dev, m.flip_table.data(), m.flip_table.size() * sizeof(tc::FlipEntry), cudaMemcpyHostToDevice);
+    if (m.eval_table_dev && e == cudaSuccess)
+      e = cudaMemcpy(m.eval_table_dev, m.eval_table.data(), m.eval_table.size() * sizeof(EvalStatEntry), cudaMemcpyHostToDevice);
+    if (m.n_running && e == cudaSuccess) {      // running mean 0 (the cleared workspace), running variance 1
+      std::vector<float> init(m.n_running, 0.f);
+      for (const EvalStatEntry& en : m.eval_table)
+        for (int ch = 0; ch < en.C; ++ch) init[en.roff + en.C + ch] = 1.f;
+      e = cudaMemcpy(m.running, init.data(), m.n_running * 4, cudaMemcpyHostToDevice);
+    }
+  }
+  // shared-memory limits of the tensor-core kernels, raised here so that a kernel's first launch may be a recorded one
+  if (e == cudaSuccess && c->bf16_mode) e = halo::set_smem_attrs();
+  if (e == cudaSuccess && c->bf16_mode) e = tc::conv_tc_set_attrs();
   c->own_streams = streams == nullptr;
   for (int k = 0; k < c->K && e == cudaSuccess; ++k) {
     Module& m = c->mods[k];
@@ -1336,6 +1414,7 @@ fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, cons
   c->last_stream = cs; c->stepped = true;
   c->t += 1;
   const int64_t t = c->t;
+  if (c->has_schedule) fdg_lr_at(&c->schedule, t, &c->lr);
   Module& m1 = c->mods[0];
   cudaError_t e = cudaSuccess;
   // Graphs take over once every module has run each of its passes at least once (all kernels
@@ -1437,6 +1516,188 @@ static fdg_status export_tensor(fdg_ctx* c, const void* src, size_t rows, int c_
   e = cudaGetLastError();
   if (e == cudaSuccess) e = cudaMemcpy(dst, c->staging, n * 4, cudaMemcpyDefault);
   return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "export");
+}
+
+fdg_status fdg_lr_at(const fdg_lr_schedule* s, int64_t iteration, float* out_lr) {
+  if (!s || !out_lr || iteration < 1 || s->iters_per_epoch < 1 || s->n_milestones < 0 || s->n_milestones > 8 ||
+      !(s->base_lr >= 0.f) || !(s->gamma >= 0.f) || s->warmup_epochs < 0 || !(s->warmup_lr >= 0.f)) return FDG_ERR_INVALID_ARG;
+  const int64_t epoch = (iteration - 1) / s->iters_per_epoch;
+  if (epoch < s->warmup_epochs) { *out_lr = s->warmup_lr; return FDG_OK; }
+  double lr = s->base_lr;
+  for (int i = 0; i < s->n_milestones; ++i) if (epoch >= s->milestones[i]) lr *= s->gamma;
+  *out_lr = (float)lr;
+  return FDG_OK;
+}
+
+fdg_status fdg_set_lr_schedule(fdg_ctx* c, const fdg_lr_schedule* s) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (!s) { c->has_schedule = false; return FDG_OK; }
+  float probe;
+  if (fdg_lr_at(s, 1, &probe) != FDG_OK) return fail(c, FDG_ERR_INVALID_ARG, "bad learning-rate schedule");
+  c->schedule = *s;
+  c->has_schedule = true;
+  return FDG_OK;
+}
+
+fdg_status fdg_bn_running_count(const fdg_ctx* c, int module, size_t* out_n) {
+  FDG_MODULE_OR_FAIL(c, module);
+  if (!out_n) return FDG_ERR_INVALID_ARG;
+  *out_n = c->mods[module - 1].n_running;
+  return FDG_OK;
+}
+static fdg_status copy_running(fdg_ctx* c, int module, const float* src, float* dst, size_t n) {
+  FDG_MODULE_OR_FAIL(c, module);
+  Module& m = c->mods[module - 1];
+  if (n != m.n_running || (!src && !dst)) return fail(c, FDG_ERR_INVALID_ARG, "element count does not match fdg_bn_running_count");
+  cudaError_t e = drain(c);
+  if (e == cudaSuccess && n) e = src ? cudaMemcpy(m.running, src, n * 4, cudaMemcpyDefault) : cudaMemcpy(dst, m.running, n * 4, cudaMemcpyDefault);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "running statistics copy");
+}
+fdg_status fdg_get_bn_running(fdg_ctx* c, int module, float* dst, size_t n) { return dst ? copy_running(c, module, nullptr, dst, n) : FDG_ERR_INVALID_ARG; }
+fdg_status fdg_set_bn_running(fdg_ctx* c, int module, const float* src, size_t n) { return src ? copy_running(c, module, src, nullptr, n) : FDG_ERR_INVALID_ARG; }
+
+}  // extern "C"
+
+template <typename T>
+static cudaError_t eval_all(fdg_ctx* c, cudaStream_t cs, const float* images_dev, const int32_t* labels_dev, float* logits_dev,
+                            int* correct_dev) {
+  Module& m1 = c->mods[0];
+  const size_t rows = (size_t)c->arch.batch * c->arch.in_h * c->arch.in_w;
+  Launch L{c, cs};
+  L.begin(KC_INGEST, (double)rows * (c->arch.in_c * 4 + m1.in_c * c->esize), 0.0);
+  L.note(launch_ingest<T>(cs, images_dev, reinterpret_cast<T*>(m1.in_ring) + (size_t)m1.Din * align_up(m1.in_elems, 128), rows,
+                          c->arch.in_c, m1.in_c, nullptr, nullptr, 0));
+  ++c->launches;
+  for (Module& m : c->mods) {
+    const int vslot = (int)(m.updates % m.Dw);
+    if (m.eval_table_dev) {
+      bn_eval_stats_kernel<<<(unsigned)m.eval_table.size(), 128, 0, cs>>>(m.running, slot_F(m, m.D), m.eval_table_dev, c->arch.bn_eps);
+      L.check();
+    }
+    forward_module<T>(c, m, L, 0, m.D, vslot, true);
+    if (m.k == c->K) head_eval<T>(c, m, L, m.D, vslot, labels_dev, logits_dev, correct_dev);
+  }
+  return L.err;
+}
+
+extern "C" {
+
+fdg_status fdg_eval(fdg_ctx* c, fdg_stream stream, const float* images_dev, const int32_t* labels_dev, float* logits_dev,
+                    int* correct_dev) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (!images_dev || (correct_dev && !labels_dev)) return fail(c, FDG_ERR_INVALID_ARG, "images (and labels, to count) must not be null");
+  if (c->latched != FDG_OK) return c->latched;
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const int share = c->tmaps.share;
+  c->tmaps.share = 1;                    // the pass runs alone: a launch may take every SM
+  e = c->bf16_mode ? eval_all<bf16>(c, cs, images_dev, labels_dev, logits_dev, correct_dev)
+                   : eval_all<float>(c, cs, images_dev, labels_dev, logits_dev, correct_dev);
+  c->tmaps.share = share;
+  c->last_stream = cs; c->stepped = true;
+  return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "inference pass");
+}
+
+fdg_status fdg_drain(fdg_ctx* c, fdg_stream stream, float* losses_dev) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (c->latched != FDG_OK) return c->latched;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  if (c->t > 0) {
+    // From here on the iterations are issued the ordinary way (a recorded graph holds passes that must now be
+    // skipped); the host has waited for everything, so stream order is all that is needed.
+    c->graph_mode_entered = false;
+    c->last_batch = c->t;
+    c->last_stream = cs; c->stepped = true;
+    for (int i = 0; i < 2 * c->K - 2 && e == cudaSuccess; ++i) {
+      c->t += 1;
+      if (c->has_schedule) fdg_lr_at(&c->schedule, c->t, &c->lr);
+      e = run_modules(c, cs, c->cfg.serial ? RUN_SERIAL : RUN_STREAMS, losses_dev ? losses_dev + i : nullptr);
+    }
+    c->last_batch = INT64_MAX;
+    if (e != cudaSuccess) return cuda_fail(c, e, "draining iterations");
+    e = drain(c);
+    if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  }
+  c->t = 0;
+  for (Module& m : c->mods) {
+    std::fill(m.slot_version.begin(), m.slot_version.end(), -1);
+    std::fill(m.slot_batch.begin(), m.slot_batch.end(), -1);
+    m.last_out_batch = m.last_grad_batch = -1;
+    m.last_out_slot = m.last_grad_slot = -1;
+  }
+  return FDG_OK;
+}
+
+// Host-side part of a saved state: a fixed header, then per module its counters and slot tables.
+struct StateHeader {
+  uint64_t magic, ws_bytes;
+  int64_t t;
+  float lr;
+  int32_t K, period, graph_mode_entered;
+};
+constexpr uint64_t kStateMagic = 0x4644475354415445ull;      // "FDGSTATE"
+static size_t state_host_bytes(const fdg_ctx* c) {
+  size_t n = sizeof(StateHeader);
+  for (const Module& m : c->mods) n += (5 + 2 * (size_t)m.D) * sizeof(int64_t);
+  return align_up(n, 256);
+}
+
+fdg_status fdg_state_bytes(const fdg_ctx* c, size_t* out_bytes) {
+  if (!c || !out_bytes) return FDG_ERR_INVALID_ARG;
+  *out_bytes = state_host_bytes(c) + c->ws_bytes;
+  return FDG_OK;
+}
+
+fdg_status fdg_save_state(fdg_ctx* c, void* dst, size_t bytes) {
+  if (!c || !dst) return FDG_ERR_INVALID_ARG;
+  const size_t hb = state_host_bytes(c);
+  if (bytes < hb + c->ws_bytes) return fail(c, FDG_ERR_WORKSPACE_TOO_SMALL, "buffer smaller than fdg_state_bytes");
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  std::vector<char> host(hb, 0);
+  StateHeader h{kStateMagic, c->ws_bytes, c->t, c->lr, c->K, c->period, c->graph_mode_entered ? 1 : 0};
+  std::memcpy(host.data(), &h, sizeof(h));
+  int64_t* p = reinterpret_cast<int64_t*>(host.data() + sizeof(StateHeader));
+  for (const Module& m : c->mods) {
+    *p++ = m.updates; *p++ = m.last_out_batch; *p++ = m.last_grad_batch; *p++ = m.last_out_slot; *p++ = m.last_grad_slot;
+    for (int i = 0; i < m.D; ++i) { *p++ = m.slot_version[i]; *p++ = m.slot_batch[i]; }
+  }
+  e = cudaMemcpy(dst, host.data(), hb, cudaMemcpyDefault);
+  if (e == cudaSuccess) e = cudaMemcpy(static_cast<char*>(dst) + hb, c->ws_base, c->ws_bytes, cudaMemcpyDefault);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "saving the state");
+}
+
+fdg_status fdg_load_state(fdg_ctx* c, const void* src, size_t bytes) {
+  if (!c || !src) return FDG_ERR_INVALID_ARG;
+  const size_t hb = state_host_bytes(c);
+  if (bytes < hb + c->ws_bytes) return fail(c, FDG_ERR_INVALID_ARG, "buffer smaller than this context's state");
+  cudaError_t e = drain(c);
+  if (e != cudaSuccess) return cuda_fail(c, e, "drain");
+  std::vector<char> host(hb);
+  e = cudaMemcpy(host.data(), src, hb, cudaMemcpyDefault);
+  if (e != cudaSuccess) return cuda_fail(c, e, "reading the state");
+  StateHeader h;
+  std::memcpy(&h, host.data(), sizeof(h));
+  if (h.magic != kStateMagic || h.ws_bytes != c->ws_bytes || h.K != c->K || h.period != c->period)
+    return fail(c, FDG_ERR_INVALID_ARG, "the state belongs to another architecture or configuration");
+  e = cudaMemcpy(c->ws_base, static_cast<const char*>(src) + hb, c->ws_bytes, cudaMemcpyDefault);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) { c->latched = FDG_ERR_CUDA; return cuda_fail(c, e, "loading the state"); }
+  c->t = h.t; c->lr = h.lr; c->lr_on_device = -1.f;
+  c->graph_mode_entered = c->use_graphs && h.graph_mode_entered != 0;
+  const int64_t* p = reinterpret_cast<const int64_t*>(host.data() + sizeof(StateHeader));
+  for (Module& m : c->mods) {
+    m.updates = *p++; m.last_out_batch = *p++; m.last_grad_batch = *p++; m.last_out_slot = (int)*p++; m.last_grad_slot = (int)*p++;
+    for (int i = 0; i < m.D; ++i) { m.slot_version[i] = *p++; m.slot_batch[i] = *p++; }
+    m.cap_batch = -1;
+  }
+  c->latched = FDG_OK;
+  return FDG_OK;
 }
 
 fdg_status fdg_boundary_elems(const fdg_ctx* c, int module, size_t* out_elems, size_t* in_elems) {
