@@ -12,9 +12,13 @@ layers.
 
 The paper defines no architecture; these are the standard definitions of the
 networks it cites (Tables 3-6):
-  * "resnet6n2": post-activation basic blocks, 3 stages of n blocks,
+  * "resnet6n2": post-activation basic blocks, stages of n blocks (three stages of n for the
+       6n+2 networks; four stages of two at widths 64..512 for the CIFAR ResNet-18),
        block(x) = ReLU( BN(conv3x3(ReLU(BN(conv3x3_s(x))))) + sc(x) ),
-       sc = identity, or BN(conv1x1_s(x)) when the shape changes;
+       sc = identity, or, when the shape changes, BN(conv1x1_s(x)) ("projection") or the
+       parameter-free x taken at every second pixel with zero channels added on both sides
+       ("zero_pad", the other standard choice for the 6n+2 networks; the printed parameter
+       counts cannot tell the two apart);
        stem = ReLU(BN(conv3x3(image))); head = GAP -> FC -> softmax-CE.
   * "wrn": pre-activation basic blocks,
        o = ReLU(BN(x)); block(x) = conv3x3(ReLU(BN(conv3x3_s(o)))) + sc,
@@ -53,6 +57,11 @@ class Arch:
     num_classes: int = 10
     batch: int = 128
     bn_eps: float = 1e-5
+    blocks: Tuple[int, ...] = None     # residual blocks per stage; None: n_per_stage in each of len(widths) stages
+    shortcut: str = "projection"       # "projection" | "zero_pad" (resnet6n2 only)
+
+    def stage_blocks(self):
+        return tuple(self.blocks) if self.blocks is not None else (self.n_per_stage,) * len(self.widths)
 
 
 # ----------------------------------------------------------------------------
@@ -110,9 +119,26 @@ class BasicBlock:
 
     def __init__(self, arch, ci, co, stride, index):
         self.ci, self.co, self.stride, self.eps = ci, co, stride, arch.bn_eps
-        self.proj = (ci != co) or (stride != 1)
+        changes = (ci != co) or (stride != 1)
+        self.proj = changes and arch.shortcut == "projection"
+        self.zero_pad = changes and arch.shortcut == "zero_pad"
+        assert not self.zero_pad or (co >= ci and (co - ci) % 2 == 0)
         self.name = "block%d" % index
         self.q = self.qw = L.identity
+
+    def _pad_shortcut(self, x):
+        """x at every stride-th pixel, (co - ci)/2 zero channels in front and behind."""
+        lo = (self.co - self.ci) // 2
+        xs = x[:, ::self.stride, ::self.stride, :]
+        out = np.zeros(xs.shape[:3] + (self.co,), dtype=x.dtype)
+        out[..., lo:lo + self.ci] = xs
+        return out
+
+    def _pad_shortcut_backward(self, dsc, x_shape):
+        lo = (self.co - self.ci) // 2
+        dx = np.zeros(x_shape, dtype=dsc.dtype)
+        dx[:, ::self.stride, ::self.stride, :] = dsc[..., lo:lo + self.ci]
+        return dx
 
     def param_spec(self):
         spec = [("conv1.w", "conv", (self.co, 3, 3, self.ci)),
@@ -143,6 +169,8 @@ class BasicBlock:
             sc, ctx["svs"] = L.batchnorm_forward(cs, p["scbn.g"], p["scbn.b"], self.eps)
             if running is not None:
                 L.batchnorm_running_update(running["scbn"], cs)
+        elif self.zero_pad:
+            sc = self._pad_shortcut(x)
         else:
             sc = x
         y = q(L.relu_forward(b2 + sc))
@@ -158,6 +186,8 @@ class BasicBlock:
         if self.proj:
             cs = q(L.conv2d_forward(x, qw(p["sc.w"]), self.stride, 0))
             sc = L.batchnorm_eval(cs, p["scbn.g"], p["scbn.b"], running["scbn"], self.eps)
+        elif self.zero_pad:
+            sc = self._pad_shortcut(x)
         else:
             sc = x
         return q(L.relu_forward(b2 + sc))
@@ -178,6 +208,8 @@ class BasicBlock:
             dcs = q(dcs)
             dxs, g["sc.w"] = L.conv2d_backward(dcs, ctx["x"], qw(p["sc.w"]), self.stride, 0)
             dx = dx + q(dxs)
+        elif self.zero_pad:
+            dx = dx + self._pad_shortcut_backward(dsum, dx.shape)
         else:
             dx = dx + dsum
         return q(dx), g
@@ -307,10 +339,11 @@ class Head:
 def build_units(arch):
     units = [Stem(arch)]
     block_cls = BasicBlock if arch.family == "resnet6n2" else PreActBlock
+    assert arch.shortcut in ("projection", "zero_pad") and (arch.shortcut == "projection" or arch.family == "resnet6n2")
     ci = arch.stem_width
     index = 0
-    for stage in range(3):
-        for j in range(arch.n_per_stage):
+    for stage, n_blocks in enumerate(arch.stage_blocks()):
+        for j in range(n_blocks):
             index += 1
             stride = 2 if (stage > 0 and j == 0) else 1
             units.append(block_cls(arch, ci, arch.widths[stage], stride, index))

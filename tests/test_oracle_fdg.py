@@ -302,3 +302,36 @@ def test_planted_mistakes_are_caught(monkeypatch):
     assert run() > 1e-3
     monkeypatch.setattr(L, "relu_backward", real_relu)
     assert run() < 1e-9
+
+
+@pytest.mark.parametrize("shortcut,blocks,widths", [("zero_pad", None, (4, 8, 12)), ("projection", (1, 2, 1, 1), (4, 8, 8, 12)),
+                                                    ("zero_pad", (2, 1, 1, 1), (4, 4, 8, 16))])
+def test_other_architectures_equal_backprop_sgd(shortcut, blocks, widths):
+    """The zero-padded shortcut and networks of up to four stages (the CIFAR ResNet-18 form), K = 1 against torch
+    autograd + torch.optim.SGD step for step, then K = 2 with frozen weights against the Eq. 16 identity."""
+    arch = nets.Arch(n_per_stage=1, widths=widths, blocks=blocks, shortcut=shortcut, stem_width=4, in_h=16, in_w=16,
+                     num_classes=5, batch=4)
+    o = make(arch, 1, [], lr=0.05, momentum=0.9, weight_decay=5e-4)
+    theta = torch.tensor(all_params(o), requires_grad=True)
+    opt = torch.optim.SGD([theta], lr=0.05, momentum=0.9, weight_decay=5e-4)
+    for t in range(1, 4):
+        x, y = batch(arch, t)
+        loss_o = o.step(x, y)
+        opt.zero_grad()
+        loss_t = torch_ref.network_loss(arch, theta, torch.tensor(x), torch.tensor(y))
+        loss_t.backward()
+        assert relerr(o.get_grads(1), theta.grad.numpy()) < 1e-9
+        opt.step()
+        assert abs(loss_o - float(loss_t.detach())) < 1e-10
+        assert relerr(o.get_params(1), theta.detach().numpy()) < 1e-10
+    n_blocks = sum(arch.stage_blocks())
+    o = make(arch, 2, [n_blocks // 2], beta=0.5, lr=0.0)
+    theta = all_params(o)
+    n1 = o.param_count(1)
+    for t in range(1, 5):
+        x, y = batch(arch, t)
+        o.step(x, y)
+    th = torch.tensor(theta, requires_grad=True)
+    x, y = batch(arch, 2)                                         # module 1 back-propagates batch t - 2 at t = 4
+    (g,) = torch.autograd.grad(torch_ref.network_loss(arch, th, torch.tensor(x), torch.tensor(y)), th)
+    assert relerr(o.get_grads(1), 0.5 * g.numpy()[:n1]) < 1e-9

@@ -60,9 +60,9 @@ def network_logits(arch, theta, images_nhwc, buffers=None, training=True):
     if not wrn:
         x = F.relu(_bn(x, rd.take(arch.stem_width), rd.take(arch.stem_width), eps))
     ci = arch.stem_width
-    for stage in range(3):
+    for stage, n_blocks in enumerate(arch.stage_blocks()):
         co = arch.widths[stage]
-        for j in range(arch.n_per_stage):
+        for j in range(n_blocks):
             stride = 2 if (stage > 0 and j == 0) else 1
             proj = ci != co or stride != 1
             if not wrn:
@@ -70,7 +70,10 @@ def network_logits(arch, theta, images_nhwc, buffers=None, training=True):
                 w2 = rd.conv(co, 3, co); g2 = rd.take(co); b2 = rd.take(co)
                 h = F.relu(_bn(F.conv2d(x, w1, stride=stride, padding=1), g1, b1, eps))
                 h = _bn(F.conv2d(h, w2, padding=1), g2, b2, eps)
-                if proj:
+                if proj and arch.shortcut == "zero_pad":
+                    lo = (co - ci) // 2
+                    sc = F.pad(x[:, :, ::stride, ::stride], (0, 0, 0, 0, lo, co - ci - lo))
+                elif proj:
                     ws = rd.conv(co, 1, ci); gs = rd.take(co); bs = rd.take(co)
                     sc = _bn(F.conv2d(x, ws, stride=stride), gs, bs, eps)
                 else:
