@@ -63,21 +63,27 @@ typedef enum {
 } fdg_status;
 
 enum { FDG_RESNET_6N2 = 0, FDG_WRN = 1 };                 /* fdg_arch.family   */
+enum { FDG_SHORTCUT_PROJECTION = 0, FDG_SHORTCUT_ZERO_PAD = 1 };   /* fdg_arch.shortcut */
 enum { FDG_BACKWARD_FIRST = 0, FDG_FORWARD_FIRST = 1 };   /* fdg_config.order  */
 enum { FDG_STASHED = 0, FDG_CURRENT = 1 };                /* fdg_config.weight_reading */
 enum { FDG_FP32_CUDACORE = 0, FDG_BF16_TC = 1 };          /* fdg_config.precision */
 enum { FDG_PARAM_CONV = 0, FDG_PARAM_BN_GAMMA = 1, FDG_PARAM_BN_BETA = 2,
        FDG_PARAM_FC_W = 3, FDG_PARAM_FC_B = 4 };          /* fdg_param_entry.kind */
 
-/* The network: a stem convolution, three stages of n_per_stage residual blocks
- * (stride 2 at the first block of stages 2 and 3), a classifier.  The paper
- * defines no architecture of its own; these are the networks of its tables. */
+/* The network: a stem convolution, n_stages stages of residual blocks (stride 2 at the first block of every
+ * stage but the first), a classifier.  The paper defines no architecture of its own; these are the networks of
+ * its tables: the 6n+2 networks (3 stages of n blocks at 16/32/64), the CIFAR ResNet-18 (4 stages of 2 blocks at
+ * 64/128/256/512), WRN-28-10 (3 stages of 4 pre-activation blocks at 160/320/640). */
 typedef struct {
   int family;            /* FDG_RESNET_6N2 (post-activation blocks) | FDG_WRN (pre-activation blocks) */
-  int n_per_stage;       /* blocks per stage (ResNet-110: 18, WRN-28-10: 4) */
-  int widths[3];         /* channels of the three stages */
+  int n_stages;          /* 1..4 */
+  int blocks[4];         /* residual blocks per stage (ResNet-110: 18,18,18; WRN-28-10: 4,4,4) */
+  int widths[4];         /* channels per stage */
   int stem_width;        /* output channels of the stem convolution */
-  int in_h, in_w, in_c;  /* image size */
+  int shortcut;          /* where a block changes the shape: FDG_SHORTCUT_PROJECTION = 1x1 convolution (+ BN in the
+                            post-activation family); FDG_SHORTCUT_ZERO_PAD (FDG_RESNET_6N2 only) = the input at every
+                            second pixel with (C_out - C_in)/2 zero channels in front and behind, no parameters */
+  int in_h, in_w, in_c;  /* image size; in_h and in_w multiples of 2^(n_stages-1), at least 4 */
   int num_classes;
   int batch;
   float bn_eps;
@@ -87,7 +93,7 @@ typedef struct {
  * beta" (Algorithm I), plus the optimiser constants of the experiments section. */
 typedef struct {
   int K;                          /* number of modules, >= 1 */
-  const int* split_after_block;   /* K-1 ascending block indices in [1, 3n-1]: module k ends after that block */
+  const int* split_after_block;   /* K-1 ascending block indices in [1, total blocks - 1]: module k ends after that block */
   float beta;                     /* shrinking factor, 0 < beta <= 1 (Eq. 15) */
   float lr, momentum, weight_decay;
   int order;                      /* FDG_BACKWARD_FIRST = Algorithm I; FDG_FORWARD_FIRST = Appendix A variant */

@@ -16,6 +16,7 @@ FDG_OK = 0
 STATUS_NAMES = {0: "FDG_OK", 1: "FDG_ERR_INVALID_ARG", 2: "FDG_ERR_WORKSPACE_TOO_SMALL", 3: "FDG_ERR_CUDA",
                 4: "FDG_ERR_STATE", 5: "FDG_ERR_UNSUPPORTED", 6: "FDG_ERR_NONFINITE", 7: "FDG_ERR_TIMEOUT"}
 FDG_RESNET_6N2, FDG_WRN = 0, 1
+FDG_SHORTCUT_PROJECTION, FDG_SHORTCUT_ZERO_PAD = 0, 1
 FDG_BACKWARD_FIRST, FDG_FORWARD_FIRST = 0, 1
 FDG_STASHED, FDG_CURRENT = 0, 1
 FDG_FP32_CUDACORE, FDG_BF16_TC = 0, 1
@@ -35,9 +36,9 @@ EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count"
 
 
 class fdg_arch(C.Structure):
-    _fields_ = [("family", C.c_int), ("n_per_stage", C.c_int), ("widths", C.c_int * 3), ("stem_width", C.c_int),
-                ("in_h", C.c_int), ("in_w", C.c_int), ("in_c", C.c_int), ("num_classes", C.c_int),
-                ("batch", C.c_int), ("bn_eps", C.c_float)]
+    _fields_ = [("family", C.c_int), ("n_stages", C.c_int), ("blocks", C.c_int * 4), ("widths", C.c_int * 4),
+                ("stem_width", C.c_int), ("shortcut", C.c_int), ("in_h", C.c_int), ("in_w", C.c_int), ("in_c", C.c_int),
+                ("num_classes", C.c_int), ("batch", C.c_int), ("bn_eps", C.c_float)]
 
 
 class fdg_config(C.Structure):
@@ -171,10 +172,16 @@ class FDGError(RuntimeError):
 
 
 def make_arch(family="resnet6n2", n_per_stage=1, widths=(16, 32, 64), stem_width=16, in_h=32, in_w=32, in_c=3,
-              num_classes=10, batch=128, bn_eps=1e-5):
+              num_classes=10, batch=128, bn_eps=1e-5, blocks=None, shortcut="projection"):
+    """`blocks`: residual blocks per stage; None: n_per_stage in each of len(widths) stages."""
     fam = {"resnet6n2": FDG_RESNET_6N2, "wrn": FDG_WRN}[family]
-    return fdg_arch(fam, n_per_stage, (C.c_int * 3)(*widths), stem_width, in_h, in_w, in_c, num_classes, batch,
-                    bn_eps)
+    sc = {"projection": FDG_SHORTCUT_PROJECTION, "zero_pad": FDG_SHORTCUT_ZERO_PAD}[shortcut]
+    ns = len(widths)
+    bl = list(blocks) if blocks is not None else [n_per_stage] * ns
+    assert len(bl) == ns and 1 <= ns <= 4
+    pad = [0] * (4 - ns)
+    return fdg_arch(fam, ns, (C.c_int * 4)(*(bl + pad)), (C.c_int * 4)(*(list(widths) + pad)), stem_width, sc, in_h, in_w,
+                    in_c, num_classes, batch, bn_eps)
 
 
 class FDG:

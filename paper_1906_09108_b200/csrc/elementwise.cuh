@@ -495,6 +495,45 @@ __global__ void upsample2_kernel(const T* __restrict__ dy, T* __restrict__ up, s
   }
 }
 
+// Zero-padded shortcut of a block that changes the shape: out [N][P][Q][Co] = x [N][H][W][Ci] at every stride-th
+// pixel, in channels lo .. lo+Ci-1 with lo = (Co - Ci)/2, zero elsewhere; and its backward, which puts the
+// gated upstream gradient's middle channels back at those pixels of a zero [N][H][W][Ci] tensor.
+template <typename T>
+__global__ void pad_shortcut_kernel(const T* __restrict__ x, T* __restrict__ out, size_t rows_out, int P, int Q, int H, int W,
+                                    int Ci, int Co, int stride) {
+  const int lo = (Co - Ci) / 2;
+  const size_t n = rows_out * (size_t)Co;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i % Co);
+    size_t pix = i / Co;
+    const int q = (int)(pix % Q); pix /= Q;
+    const int p = (int)(pix % P);
+    const size_t img = pix / P;
+    T v = from_f<T>(0.f);
+    if (c >= lo && c < lo + Ci) v = x[((img * H + (size_t)p * stride) * W + (size_t)q * stride) * Ci + (c - lo)];
+    out[i] = v;
+  }
+}
+template <typename T>
+__global__ void pad_shortcut_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ y, T* __restrict__ dx, size_t rows_in,
+                                        int P, int Q, int H, int W, int Ci, int Co, int stride) {
+  const int lo = (Co - Ci) / 2;
+  const size_t n = rows_in * (size_t)Ci;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i % Ci);
+    size_t pix = i / Ci;
+    const int w = (int)(pix % W); pix /= W;
+    const int h = (int)(pix % H);
+    const size_t img = pix / H;
+    T v = from_f<T>(0.f);
+    if (h % stride == 0 && w % stride == 0) {
+      const size_t o = ((img * P + h / stride) * Q + w / stride) * Co + lo + c;
+      if (to_f(y[o]) > 0.f) v = dy[o];
+    }
+    dx[i] = v;
+  }
+}
+
 // fp32 [rows][c_in] -> T [rows][c_out], channels c_in..c_out-1 zero (image ingest); labels copied alongside.
 template <typename T>
 __global__ void ingest_kernel(const float* __restrict__ img, T* __restrict__ out, size_t rows, int c_in, int c_out,

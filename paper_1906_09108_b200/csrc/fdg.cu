@@ -55,6 +55,7 @@ struct Unit {
   int index;                 // 0 stem, b block, -1 head
   int ci, co, stride;
   bool proj;
+  bool zpad;                 // shape change bridged by the parameter-free zero-padded shortcut
   bool bn;                   // stem: has BN+ReLU (6n+2); head: has BN+ReLU (WRN)
   int H, W, P, Q;            // input / output spatial size
   // offsets into the module's flat parameter vector
@@ -209,17 +210,28 @@ static int pow2_at_least(int x) { int p = 1; while (p < x) p <<= 1; return p; }
 static fdg_status validate(const fdg_arch* a, const fdg_config* c, std::string* why) {
   if (!a || !c) { *why = "null arch or config"; return FDG_ERR_INVALID_ARG; }
   if (a->family != FDG_RESNET_6N2 && a->family != FDG_WRN) { *why = "unknown family"; return FDG_ERR_INVALID_ARG; }
-  if (a->n_per_stage < 1 || a->stem_width < 1 || a->in_h < 4 || a->in_w < 4 || a->in_c < 1 || a->num_classes < 2 ||
+  if (a->n_stages < 1 || a->n_stages > 4 || a->stem_width < 1 || a->in_h < 4 || a->in_w < 4 || a->in_c < 1 || a->num_classes < 2 ||
       a->batch < 1 || !(a->bn_eps > 0.f)) { *why = "bad architecture sizes"; return FDG_ERR_INVALID_ARG; }
-  for (int i = 0; i < 3; ++i) if (a->widths[i] < 1) { *why = "bad stage width"; return FDG_ERR_INVALID_ARG; }
-  if (a->in_h % 4 || a->in_w % 4) { *why = "image size must be a multiple of 4"; return FDG_ERR_INVALID_ARG; }
+  for (int i = 0; i < a->n_stages; ++i) if (a->widths[i] < 1 || a->blocks[i] < 1) { *why = "bad stage width or block count"; return FDG_ERR_INVALID_ARG; }
+  const int down = 1 << (a->n_stages - 1);
+  if (a->in_h % down || a->in_w % down) { *why = "image size must be a multiple of 2^(stages-1)"; return FDG_ERR_INVALID_ARG; }
+  if (a->shortcut != FDG_SHORTCUT_PROJECTION && a->shortcut != FDG_SHORTCUT_ZERO_PAD) { *why = "unknown shortcut"; return FDG_ERR_INVALID_ARG; }
+  if (a->shortcut == FDG_SHORTCUT_ZERO_PAD) {
+    if (a->family != FDG_RESNET_6N2) { *why = "the zero-padded shortcut belongs to the post-activation family"; return FDG_ERR_INVALID_ARG; }
+    int prev = a->stem_width;
+    for (int i = 0; i < a->n_stages; ++i) {
+      if (a->widths[i] < prev || (a->widths[i] - prev) % 2) { *why = "zero-padded shortcut needs widths that grow by an even amount"; return FDG_ERR_INVALID_ARG; }
+      prev = a->widths[i];
+    }
+  }
   if (c->K < 1 || c->K > 64) { *why = "K out of range"; return FDG_ERR_INVALID_ARG; }
   if (c->K > 1 && !c->split_after_block) { *why = "split_after_block is null"; return FDG_ERR_INVALID_ARG; }
-  const int nblocks = 3 * a->n_per_stage;
+  int nblocks = 0;
+  for (int i = 0; i < a->n_stages; ++i) nblocks += a->blocks[i];
   int prev = 0;
   for (int i = 0; i + 1 < c->K; ++i) {
     int s = c->split_after_block[i];
-    if (s <= prev || s >= nblocks) { *why = "split points must ascend inside [1, 3n-1]"; return FDG_ERR_INVALID_ARG; }
+    if (s <= prev || s >= nblocks) { *why = "split points must ascend inside [1, blocks-1]"; return FDG_ERR_INVALID_ARG; }
     prev = s;
   }
   if (!(c->beta > 0.f && c->beta <= 1.f)) { *why = "beta must be in (0, 1]"; return FDG_ERR_INVALID_ARG; }
@@ -230,12 +242,13 @@ static fdg_status validate(const fdg_arch* a, const fdg_config* c, std::string* 
       (c->precision != FDG_FP32_CUDACORE && c->precision != FDG_BF16_TC)) { *why = "bad enum value"; return FDG_ERR_INVALID_ARG; }
   // channel counts the vectorised kernels can address
   const int vec = c->precision == FDG_BF16_TC ? 8 : 4;
-  int chans[4] = {a->stem_width, a->widths[0], a->widths[1], a->widths[2]};
+  int chans[5] = {a->stem_width, a->widths[0], a->widths[0], a->widths[0], a->widths[0]};
+  for (int i = 0; i < a->n_stages; ++i) chans[1 + i] = a->widths[i];
   for (int ch : chans) {
     if ((ch % vec != 0 && ch > kRedThreads) || ch / vec > kRedThreads) { *why = "channel count not addressable by the reduction kernels"; return FDG_ERR_UNSUPPORTED; }
     if (c->precision == FDG_BF16_TC && ch % 8 != 0) { *why = "bf16 mode needs channel counts that are multiples of 8"; return FDG_ERR_UNSUPPORTED; }
   }
-  if ((size_t)a->batch * a->in_h * a->in_w * (size_t)std::max({chans[0], chans[1], chans[2], chans[3]}) > (size_t)1 << 31) {
+  if ((size_t)a->batch * a->in_h * a->in_w * (size_t)std::max({chans[0], chans[1], chans[2], chans[3], chans[4]}) > (size_t)1 << 31) {
     *why = "activation tensor exceeds 2^31 elements"; return FDG_ERR_UNSUPPORTED; }
   return FDG_OK;
 }
@@ -260,7 +273,8 @@ static void plan_modules(fdg_ctx* c) {
   const fdg_arch& a = c->arch;
   const int K = c->K;
   const bool wrn = a.family == FDG_WRN;
-  const int nblocks = 3 * a.n_per_stage;
+  int nblocks = 0;
+  for (int i = 0; i < a.n_stages; ++i) nblocks += a.blocks[i];
   c->mods.assign(K, Module());
   std::vector<int> last_block(K);
   for (int k = 0; k < K; ++k) last_block[k] = (k + 1 < K) ? c->splits[k] : nblocks;
@@ -281,10 +295,13 @@ static void plan_modules(fdg_ctx* c) {
   for (int b = 1; b <= nblocks; ++b) {
     while (b > last_block[k]) ++k;
     Module& m = c->mods[k];
-    const int stage = (b - 1) / a.n_per_stage, j = (b - 1) % a.n_per_stage;
+    int stage = 0, j = b - 1;
+    while (j >= a.blocks[stage]) { j -= a.blocks[stage]; ++stage; }
     Unit u{}; u.type = wrn ? U_PREACT : U_BASIC; u.index = b; u.ci = ci; u.co = a.widths[stage];
     u.stride = (stage > 0 && j == 0) ? 2 : 1;
-    u.proj = (u.ci != u.co) || u.stride != 1;
+    const bool changes = (u.ci != u.co) || u.stride != 1;
+    u.proj = changes && a.shortcut == FDG_SHORTCUT_PROJECTION;
+    u.zpad = changes && a.shortcut == FDG_SHORTCUT_ZERO_PAD;
     u.H = H; u.W = W; u.P = conv_out(H, 3, u.stride, 1); u.Q = conv_out(W, 3, u.stride, 1);
     if (m.units.empty()) { m.in_h = H; m.in_w = W; m.in_c = ci; m.in_c_logical = ci; }
     if (!wrn) {
@@ -700,10 +717,16 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
         }
         const int np2 = conv_fprop<T>(L, m, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr, !eval);       // c2
         stats_of(np2, S + u.t_c, rows_out, u.co, F + u.st2, u.r2);
-        if (u.proj)
+        if (u.proj) {
           bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, S + u.t_s, F + u.sts, wf + u.gs, wf + u.bs, true, S + u.t_y, rows_out, u.co, np2, u.r2);
-        else
+        } else if (u.zpad) {   // the shortcut is x at every stride-th pixel between zero channels: built in a temporary
+          L.begin(KC_BN_APPLY, (double)rows_out * (u.ci + u.co) * sizeof(T), 0.0);
+          pad_shortcut_kernel<T><<<ew_blocks(rows_out * u.co), 256, 0, L.st>>>(x, tmp, rows_out, u.P, u.Q, u.H, u.W, u.ci, u.co, u.stride);
+          L.check();
+          bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, tmp, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np2, u.r2);
+        } else {
           bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, x, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np2, u.r2);
+        }
         break;
       }
       case U_PREACT: {
@@ -901,6 +924,12 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
             conv_dgrad<T>(L, m, gs, T2, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
             out_sum_parts = conv_dgrad<T>(L, m, g1, T4, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next, up);
           }
+        } else if (need_dx && u.zpad) {
+          // the shortcut's share: the gated upstream gradient's middle channels, put back at every stride-th pixel
+          L.begin(KC_BN_BWD_APPLY, (double)(rows_out * u.co * 2 + rows_in * u.ci) * sizeof(T), 0.0);
+          pad_shortcut_bwd_kernel<T><<<ew_blocks(rows_in * u.ci), 256, 0, L.st>>>(dy, S + u.t_y, T3, rows_in, u.P, u.Q, u.H, u.W, u.ci, u.co, u.stride);
+          L.check();
+          out_sum_parts = conv_dgrad<T>(L, m, g1, T4, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next, up);
         } else if (need_dx) {
           out_sum_parts = conv_dgrad<T>(L, m, g1, T4, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, dy, S + u.t_y, next);
         }
