@@ -191,6 +191,16 @@ KERNEL_SHAPES = {     # the 3x3 stride-1 layer shapes of the 6n+2 workloads and 
     "wrn_stage1": (128, 32, 32, 160), "wrn_stage2": (128, 16, 16, 320), "wrn_stage3": (128, 8, 8, 640)}
 
 
+# The convolution launches as the module-step issues them: on a third of the SMs (four modules side by side),
+# several image tiles per CTA, with the reductions fused into their epilogues.
+STEP_VARIANTS = {
+    "fprop_stats": "forward + batch-norm statistics of its output (conv1, conv2 of a block)",
+    "dgrad_bn": "data gradient + the sums of the batch-norm backward it feeds (conv2's data gradient)",
+    "dgrad_res_bn": "data gradient + gated residual + those sums (the block-input gradient of an identity block)",
+    "wgrad_side": "weight gradient with its pixel split capped at 16 CTAs (side stream)",
+}
+
+
 def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5, use_graph=True):
     """Average duration of one convolution kernel launch, timed alone: `launches` calls of the operator-level
     entry point, each on its own input/output pair out of a pool larger than the L2 cache (so every launch
@@ -199,6 +209,7 @@ def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5, use_grap
     import torch
     n, h, w, c = KERNEL_SHAPES[stage]
     ops = B.ConvOps(B.FDG_BF16_TC)
+    variant = which if which in STEP_VARIANTS else None
     s = B.fdg_conv_shape(n, h, w, c, c, 3, 1, 1)
     elems = n * h * w * c
     pool = max(8, (300 << 20) // (4 * elems) + 1)                 # in + out pairs summing to > 2 x 126 MB
@@ -212,10 +223,31 @@ def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5, use_grap
     dw = torch.empty((c, 3, 3, c), dtype=torch.float32, device="cuda")
     st = torch.cuda.Stream()
 
+    extra = None
+    extra_tensors = 0
+    if variant:
+        ex, keep = ops._extra(s, share=3, wgrad_cta_cap=16 if variant == "wgrad_side" else 0,
+                              reduce={"fprop_stats": 1, "dgrad_bn": 2, "dgrad_res_bn": 2, "wgrad_side": 0}[variant],
+                              next_mask=xs[0], next_x=xs[0], next_stats=torch.zeros(2 * c, device="cuda") + 1.0, C_red=c)
+        extra = B.C.byref(ex)
+        extra_tensors = {"fprop_stats": 0, "dgrad_bn": 2, "dgrad_res_bn": 4, "wgrad_side": 0}[variant]
+
     def call(i):
         x, y = xs[i % pool], ys[i % pool]
         cs = st.cuda_stream
-        if which == "fprop":
+        if variant in ("dgrad_bn", "dgrad_res_bn"):
+            ex.next_mask, ex.next_x = xs[(i + 1) % pool].data_ptr(), xs[(i + 2) % pool].data_ptr()
+            res = xs[(i + 3) % pool].data_ptr() if variant == "dgrad_res_bn" else None
+            msk = xs[(i + 4) % pool].data_ptr() if variant == "dgrad_res_bn" else None
+            rc = ops.lib.fdg_conv_dgrad(ops.precision, B.C.byref(s), x.data_ptr(), wt.data_ptr(), wf.data_ptr(), y.data_ptr(),
+                                        res, msk, extra, ops.status.data_ptr(), cs)
+        elif variant == "fprop_stats":
+            rc = ops.lib.fdg_conv_forward(ops.precision, B.C.byref(s), x.data_ptr(), wt.data_ptr(), y.data_ptr(), None,
+                                          extra, ops.status.data_ptr(), cs)
+        elif variant == "wgrad_side":
+            rc = ops.lib.fdg_conv_wgrad(ops.precision, B.C.byref(s), x.data_ptr(), xs[(i + 1) % pool].data_ptr(),
+                                        dw.data_ptr(), scratch.data_ptr(), need.value, extra, ops.status.data_ptr(), cs)
+        elif which == "fprop":
             rc = ops.lib.fdg_conv_forward(ops.precision, B.C.byref(s), x.data_ptr(), wt.data_ptr(), y.data_ptr(), None,
                                           None, ops.status.data_ptr(), cs)
         elif which == "dgrad":
@@ -250,8 +282,8 @@ def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5, use_grap
         st.synchronize()
     assert not ops.timed_out()
     us = e0.elapsed_time(e1) * 1e3 / (reps * launches)
-    wbytes = c * 9 * c * (4 if which == "wgrad" else 2)
-    return us, 2 * elems * 2 + wbytes, 2.0 * n * h * w * c * 9 * c
+    wbytes = c * 9 * c * (4 if which in ("wgrad", "wgrad_side") else 2)
+    return us, (2 + extra_tensors) * elems * 2 + wbytes, 2.0 * n * h * w * c * 9 * c
 
 
 EW_KERNELS = ["bn_stats", "bn_apply", "bn_apply_res", "bn_bwd_reduce", "bn_bwd_apply", "shrink", "sgd", "ingest", "head"]
@@ -381,7 +413,9 @@ def run_kernel_bench(args):
                     us=us, mbytes=nbytes / 1e6, gbs=nbytes / us / 1e3, hbm_frac=nbytes / us / 1e3 / peaks["hbm_gbs"])
         print(json.dumps(dict(kernel_bench=out, peak_source=peaks["source"], hbm_gbs=peaks["hbm_gbs"])))
         return
-    which_list = [args.kernel_bench] if args.kernel_bench != "all" else ["fprop", "dgrad", "wgrad"]
+    which_list = {"all": ["fprop", "dgrad", "wgrad"], "step": list(STEP_VARIANTS)}.get(args.kernel_bench, [args.kernel_bench])
+    if args.kernel_bench == "step" and not args.kernel_stage:
+        args.kernel_stage = "stage1"
     stages = [args.kernel_stage] if args.kernel_stage else list(KERNEL_SHAPES)
     for which in which_list:
         for stage in stages:
@@ -567,7 +601,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graphs", action="store_true")
     ap.add_argument("--workload", default="resnet110_k4", choices=list(WORKLOADS))
-    ap.add_argument("--kernel-bench", default=None, choices=["fprop", "dgrad", "wgrad", "all", "ew"] + EW_KERNELS,
+    ap.add_argument("--kernel-bench", default=None, choices=["fprop", "dgrad", "wgrad", "all", "ew", "step"] + EW_KERNELS + list(STEP_VARIANTS),
                     help="time the convolution kernels alone through the operator-level C ABI and exit")
     ap.add_argument("--kernel-launches", type=int, default=64,
                     help="launches per replay; 8 or fewer are issued as plain launches (profiler runs)")
