@@ -26,6 +26,7 @@
 // wait is bounded; on time-out the CTA raises an error word.
 #pragma once
 #include "conv_tc.cuh"
+#include "elementwise.cuh"
 
 namespace fdg {
 namespace halo {
@@ -149,11 +150,10 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   float* red_stat = red_run + kEpiWarps * 8 * 32;                    // mode 2: mean[Cn], invstd[Cn]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (red.mode) {
+  // Start-up that needs nothing from global memory: it may run while the preceding kernel of the stream is
+  // still at work (programmatic dependent launch, see elementwise.cuh).
+  if (red.mode)
     for (int i = threadIdx.x; i < kEpiWarps * 8 * 32; i += kFwdThreads) red_run[i] = 0.f;
-    if (red.mode == 2)
-      for (int i = threadIdx.x; i < 2 * p.Cn; i += kFwdThreads) red_stat[i] = red.pstats[i];
-  }
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
@@ -163,14 +163,19 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     for (int a = 0; a < p.nacc; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4 * groups_per_tile); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
+  grid_dependency_wait();                  // from here on the preceding kernel's results may be read
+  if (red.mode == 2)
+    for (int i = threadIdx.x; i < 2 * p.Cn; i += kFwdThreads) red_stat[i] = red.pstats[i];
+  if (threadIdx.x == 0) {
     // This thread is also the producer: the weights and the first tile are requested now, so that their
-    // latency runs beside the tensor-memory allocation and the barrier below instead of after them.
+    // latency runs beside the barrier below instead of after it.
     mbar_expect_tx(w_full, 9 * p.w_tx_bytes);
     for (int tap = 0; tap < 9; ++tap) tma_load_2d(w_smem + (size_t)tap * p.w_tap_bytes, &map_w, w_full, tap * p.Ck, 0);
     mbar_expect_tx(&full[0], p.tile_tx_bytes);
     tma_load_4d(smem, &map_x, &full[0], 0, -1, -1, (int)blockIdx.x * p.G);
   }
-  if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();

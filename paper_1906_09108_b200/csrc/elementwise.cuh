@@ -13,6 +13,30 @@
 
 namespace fdg {
 
+// ------------------------------------------------ programmatic dependent launch --
+// The kernels that follow one another in a module's chain (convolution, batch-norm apply, batch-norm
+// backward apply) are launched with programmatic stream serialisation: the next kernel of the stream may be
+// scheduled while this one still runs, does the part of its start-up that needs nothing from global
+// memory (barriers, tensor-memory allocation, descriptor prefetch), and then blocks in grid_dependency_wait()
+// until the preceding kernel has completed and its writes are visible.  Nothing may be read from or written
+// to global memory before that wait.  grid_dependency_release() tells the scheduler that, as far as this
+// block is concerned, the next kernel may start being scheduled (it fires once every block has called it or
+// exited).  Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Launch with the attribute that allows the overlap described above.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------- helpers ---
 template <typename T> struct Vec;   // 16-byte vector of T
 template <> struct Vec<float> {
@@ -300,6 +324,8 @@ bn_apply_kernel(const T* __restrict__ x, const float* __restrict__ stats,
                 const float* __restrict__ res_gamma, const float* __restrict__ res_beta,
                 int relu, T* __restrict__ y, size_t nvec, int C, PartialSums ps) {
   __shared__ float s_stats[2 * 128];
+  grid_dependency_wait();
+  grid_dependency_release();
   const float* st = stats;
   if (ps.partial) { finalize_partials(ps, C, s_stats); st = s_stats; }
   const int cv = C / VEC;
@@ -400,6 +426,8 @@ bn_bwd_apply_kernel(const T* __restrict__ dy, const T* __restrict__ mask, const 
                     const T* __restrict__ res, T* __restrict__ dx, T* __restrict__ dx2,
                     size_t nvec, int C, float inv_m, PartialSums ps) {
   __shared__ float s_sums[2 * 128];
+  grid_dependency_wait();
+  grid_dependency_release();
   if (ps.partial) { finalize_partials(ps, C, s_sums); sums = s_sums; }
   const int cv = C / VEC;
   const size_t gtid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
@@ -804,14 +832,12 @@ inline cudaError_t launch_bn_apply(cudaStream_t st, const T* x, float* stats, co
   }
   if (C % V == 0) {
     const int blocks = ew_grid_for_channels(n / V, C / V, ps.partial ? block_cap : 0);
-    if (res_stats) bn_apply_kernel<T, V, true><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
-    else bn_apply_kernel<T, V, false><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n / V, C, ps);
-  } else {
-    const int blocks = ew_grid_for_channels(n, C, 0);
-    if (res_stats) bn_apply_kernel<T, 1, true><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
-    else bn_apply_kernel<T, 1, false><<<blocks, kEwThreads, 0, st>>>(x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, n, C, ps);
+    if (res_stats) return launch_chained(bn_apply_kernel<T, V, true>, blocks, kEwThreads, 0, st, x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, (int)relu, y, n / V, C, ps);
+    return launch_chained(bn_apply_kernel<T, V, false>, blocks, kEwThreads, 0, st, x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, (int)relu, y, n / V, C, ps);
   }
-  return cudaGetLastError();
+  const int blocks = ew_grid_for_channels(n, C, 0);
+  if (res_stats) return launch_chained(bn_apply_kernel<T, 1, true>, blocks, kEwThreads, 0, st, x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, (int)relu, y, n, C, ps);
+  return launch_chained(bn_apply_kernel<T, 1, false>, blocks, kEwThreads, 0, st, x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, (int)relu, y, n, C, ps);
 }
 
 // First half of the batch-norm backward: the per-channel sums of dz = dy*[mask>0] (and dz*xhat, dz*xhat2),
@@ -852,14 +878,12 @@ inline cudaError_t launch_bn_bwd_apply(cudaStream_t st, const T* dy, const T* ma
   }
   if (C % V == 0) {
     const int blocks = ew_grid_for_channels(n / V, C / V, ps.partial ? block_cap : 0);
-    if (dx2) bn_bwd_apply_kernel<T, V, true><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n / V, C, inv_m, ps);
-    else bn_bwd_apply_kernel<T, V, false><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n / V, C, inv_m, ps);
-  } else {
-    const int blocks = ew_grid_for_channels(n, C, 0);
-    if (dx2) bn_bwd_apply_kernel<T, 1, true><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n, C, inv_m, ps);
-    else bn_bwd_apply_kernel<T, 1, false><<<blocks, kEwThreads, 0, st>>>(dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n, C, inv_m, ps);
+    if (dx2) return launch_chained(bn_bwd_apply_kernel<T, V, true>, blocks, kEwThreads, 0, st, dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n / V, C, inv_m, ps);
+    return launch_chained(bn_bwd_apply_kernel<T, V, false>, blocks, kEwThreads, 0, st, dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n / V, C, inv_m, ps);
   }
-  return cudaGetLastError();
+  const int blocks = ew_grid_for_channels(n, C, 0);
+  if (dx2) return launch_chained(bn_bwd_apply_kernel<T, 1, true>, blocks, kEwThreads, 0, st, dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n, C, inv_m, ps);
+  return launch_chained(bn_bwd_apply_kernel<T, 1, false>, blocks, kEwThreads, 0, st, dy, mask, x, stats, gamma, sums, x2, stats2, gamma2, res, dx, dx2, n, C, inv_m, ps);
 }
 
 template <typename T>
