@@ -94,23 +94,29 @@ __device__ __forceinline__ void update_running(const RunningStats& r, int C, int
 }
 
 constexpr int kRedThreads = 256;      // threads per block of the channel-reduction kernels
-// Blocks of a channel reduction.  The last block to finish adds all blocks' partial sums, a serial
-// tail that grows with the block count; with the row loop keeping four loads in flight per thread,
-// half a block per SM measured fastest on the wide layers (74: 16.7 ms per WRN-28-10 iteration,
-// 148: 17.2, 592: 19.5).
-constexpr int kRedMaxBlocks = 74;
+// Blocks of a channel reduction along the rows.  The last block of a channel slab to finish adds that slab's
+// partial sums, a serial tail that grows with the block count and with the slab's width; wide tensors are
+// therefore cut into slabs of kRedSlab channels (grid.y), each with its own tail on its own SM.
+constexpr int kRedMaxBlocks = 148;
 constexpr int kRedMaxSums = 3;
+constexpr int kRedSlab = 32;
+constexpr int kRedMaxSlabs = 64;      // ticket words available
 
 // Per-channel statistics record written by the forward and read by the backward.
 // stats[0..C) = mean, stats[C..2C) = 1/sqrt(var+eps).
 
 // Geometry shared by the channel-reduction kernels: a block owns a contiguous range
 // of rows; thread (r, cv) walks rows r, r+RP, ... of channel vector cv.
+// C: channels of one slab (what a block reduces); ld: channels of a row of the tensor; the slab of block
+// (x, y) starts at channel y * C.
 struct RedGeom {
-  int rows, C, cv, rp, blocks, rows_per_block;
+  int rows, C, cv, rp, blocks, rows_per_block, ld, slabs;
 };
 inline RedGeom red_geom(int rows, int C, int vec) {
   RedGeom g;
+  g.ld = C;
+  g.slabs = 1;
+  if (C > 2 * kRedSlab && C % kRedSlab == 0 && kRedSlab % vec == 0 && C / kRedSlab <= kRedMaxSlabs) { g.slabs = C / kRedSlab; C = kRedSlab; }
   g.rows = rows; g.C = C; g.cv = C / vec;
   g.rp = kRedThreads / g.cv; if (g.rp < 1) g.rp = 1;
   int want = (rows + g.rp * 4 - 1) / (g.rp * 4);           // >= 4 passes per block
@@ -136,6 +142,9 @@ __device__ __forceinline__ void channel_reduce(const RedGeom g, float* __restric
   const int tid = threadIdx.x;
   const int cvi = tid % g.cv, r = tid / g.cv;
   const int C = g.C;
+  const int c_off = blockIdx.y * C;                          // first channel of this block's slab
+  partial += (size_t)blockIdx.y * gridDim.x * NS * C;         // this slab's partial sums
+  counter += blockIdx.y;
   float sums[NS][VEC];
 #pragma unroll
   for (int s = 0; s < NS; ++s)
@@ -145,7 +154,7 @@ __device__ __forceinline__ void channel_reduce(const RedGeom g, float* __restric
   const int row1 = min(row0 + g.rows_per_block, g.rows);
   if (r < g.rp) {
 #pragma unroll 4
-    for (int row = row0 + r; row < row1; row += g.rp) acc(row, cvi * VEC, sums);
+    for (int row = row0 + r; row < row1; row += g.rp) acc(row, c_off + cvi * VEC, sums);
   }
   if (r < g.rp) {
 #pragma unroll
@@ -205,7 +214,7 @@ __device__ __forceinline__ void channel_reduce(const RedGeom g, float* __restric
     double tot[NS];
 #pragma unroll
     for (int s = 0; s < NS; ++s) tot[s] = red_smem_d()[s * C + c];
-    fin_fn(c, tot);
+    fin_fn(c_off + c, tot);
   }
 }
 
@@ -215,7 +224,7 @@ template <typename T, int VEC>
 __global__ void __launch_bounds__(kRedThreads)
 bn_stats_kernel(const T* __restrict__ x, RedGeom g, float eps, float* __restrict__ stats,
                 float* __restrict__ partial, unsigned int* __restrict__ counter, RunningStats run) {
-  const int C = g.C;
+  const int C = g.ld;
   const double inv_m = 1.0 / (double)g.rows;
   channel_reduce<2, VEC>(
       g, partial, counter,
@@ -383,7 +392,7 @@ bn_bwd_reduce_kernel(const T* __restrict__ dy, const T* __restrict__ mask, const
                      RedGeom g, float* __restrict__ sums, float* __restrict__ dgamma, float* __restrict__ dbeta,
                      float* __restrict__ dgamma2, float* __restrict__ dbeta2, float* __restrict__ partial,
                      unsigned int* __restrict__ counter) {
-  const int C = g.C;
+  const int C = g.ld;
   channel_reduce<NS, VEC>(
       g, partial, counter,
       [&](int row, int c0, float (&s)[NS][VEC]) {
@@ -792,10 +801,10 @@ inline cudaError_t launch_bn_stats(cudaStream_t st, const T* x, size_t rows, int
   const RunningStats run{running, momentum, rows > 1 ? (float)((double)rows / (double)(rows - 1)) : 1.f};
   if (C % V == 0) {
     RedGeom g = red_geom((int)rows, C, V);
-    bn_stats_kernel<T, V><<<g.blocks, kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * C * 4, st>>>(x, g, eps, stats, scratch, counter, run);
+    bn_stats_kernel<T, V><<<dim3(g.blocks, g.slabs), kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * g.C * 4, st>>>(x, g, eps, stats, scratch, counter, run);
   } else {
     RedGeom g = red_geom((int)rows, C, 1);
-    bn_stats_kernel<T, 1><<<g.blocks, kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * C * 4, st>>>(x, g, eps, stats, scratch, counter, run);
+    bn_stats_kernel<T, 1><<<dim3(g.blocks, g.slabs), kRedThreads, (size_t)(g.rp > 2 ? g.rp : 2) * 2 * g.C * 4, st>>>(x, g, eps, stats, scratch, counter, run);
   }
   return cudaGetLastError();
 }
@@ -851,8 +860,8 @@ inline cudaError_t launch_bn_bwd_reduce(cudaStream_t st, const T* dy, const T* m
   const bool two = x2 != nullptr, vec = C % V == 0;
   const int ns = two ? 3 : 2;
   RedGeom g = red_geom((int)rows, C, vec ? V : 1);
-  const size_t smem = (size_t)(g.rp > 2 ? g.rp : 2) * ns * C * 4;
-#define FDG_RED(VV, NS) bn_bwd_reduce_kernel<T, VV, NS><<<g.blocks, kRedThreads, smem, st>>>( \
+  const size_t smem = (size_t)(g.rp > 2 ? g.rp : 2) * ns * g.C * 4;
+#define FDG_RED(VV, NS) bn_bwd_reduce_kernel<T, VV, NS><<<dim3(g.blocks, g.slabs), kRedThreads, smem, st>>>( \
       dy, mask, x, stats, x2, stats2, g, sums, dgamma, dbeta, dgamma2, dbeta2, scratch, counter)
   if (vec) { if (two) FDG_RED(V, 3); else FDG_RED(V, 2); }
   else     { if (two) FDG_RED(1, 3); else FDG_RED(1, 2); }

@@ -88,6 +88,7 @@ struct Module {
   bf16* wver16 = nullptr;
   bf16* wflip16 = nullptr;                 // Dw copies of the flipped/transposed 3x3 weights (dgrad operands)
   size_t flip_elems = 0;
+  unsigned flip_blocks = 8;                // blocks per table entry of the flip kernel: one per 8192 weights of the largest
   std::vector<tc::FlipEntry> flip_table;   // host copy; src = offset in a wver16 slot, dst = offset in a wflip16 slot
   tc::FlipEntry* flip_table_dev = nullptr;
   char* fifo = nullptr;                    // D slots of slot_elems*sizeof(T)
@@ -411,6 +412,9 @@ static void plan_modules(fdg_ctx* c) {
         if (dgrad_uses_flipped(g2)) u.f2 = flip(u.w2, u.co, u.co);
       }
       m.flip_elems = fe;
+      size_t largest = 0;
+      for (const tc::FlipEntry& fe_ : m.flip_table) largest = std::max(largest, (size_t)fe_.Co * 9 * fe_.Ci);
+      m.flip_blocks = (unsigned)std::min<size_t>(std::max<size_t>(largest / 8192, 8), 128);
     }
     m.slot_elems = te; m.slot_floats = tf; m.max_act = maxa; m.scratch_floats = scr; m.wscratch_floats = wscr;
     for (const Unit& u : m.units) {     // where the inference pass finds each batch norm's statistics
@@ -985,7 +989,7 @@ static void update_module(fdg_ctx* c, Module& m, Launch& L, int next_vslot) {
   ++c->launches;
   if (m.flip_table_dev) {
     L.begin(KC_SGD, 4.0 * m.flip_elems, 0.0);
-    tc::wflip_kernel<<<dim3(8, (unsigned)m.flip_table.size()), 256, 0, L.st>>>(next16, m.wflip16 + (size_t)next_vslot * m.flip_elems, m.flip_table_dev);
+    tc::wflip_kernel<<<dim3(m.flip_blocks, (unsigned)m.flip_table.size()), 256, 0, L.st>>>(next16, m.wflip16 + (size_t)next_vslot * m.flip_elems, m.flip_table_dev);
     L.check();
   }
 }
@@ -1297,7 +1301,7 @@ static fdg_status copy_vec(fdg_ctx* c, int module, float* dev_vec, const float* 
         ++c->launches;
         e = cudaGetLastError();
         if (e == cudaSuccess && m.flip_table_dev) {
-          tc::wflip_kernel<<<dim3(8, (unsigned)m.flip_table.size()), 256, 0, m.stream>>>(
+          tc::wflip_kernel<<<dim3(m.flip_blocks, (unsigned)m.flip_table.size()), 256, 0, m.stream>>>(
               m.wver16 + (size_t)v * align_up(n, 64), m.wflip16 + (size_t)v * m.flip_elems, m.flip_table_dev);
           ++c->launches;
           e = cudaGetLastError();
