@@ -149,7 +149,7 @@ inline cudaError_t run_conv_halo(cudaStream_t st, TensorMapCache* cache, int N, 
   halo::EpiReduce r{};
   if (red) { if (!halo_reduce_ok(Cn)) return cudaErrorInvalidValue; r = *red; }
   if (ctas_out) *ctas_out = grid;
-  return launch_chained(halo::conv_halo_kernel, grid, halo::kFwdThreads, halo::fwd_smem_bytes(p), st, *mx, *mw, p, out, res, res_mask, r, err_dev);
+  return launch_chained(halo::conv_halo_kernel, grid, halo::kConvThreads, halo::fwd_smem_bytes(p), st, *mx, *mw, p, out, res, res_mask, r, err_dev);
 }
 
 // dw[Co][3][3][Ci] (fp32) from x [N][H][W][Ci] and dy [N][H][W][Co]; `scratch` holds the per-CTA partials

@@ -101,6 +101,13 @@ constexpr int kMmaWarps = 2;
 constexpr int kFirstEpiWarp = 1 + kMmaWarps;
 constexpr int kFwdThreads = 32 * (kFirstEpiWarp + kEpiWarps);
 constexpr int kRedSmemBytes = kEpiWarps * 8 * 32 * 4 + 2 * 128 * 4;   // running sums, statistics
+// conv_halo_kernel: four issuing warps, one per warp scheduler (a warp's scheduler and its tensor-memory lane
+// quarter are both warp % 4, so every scheduler also hosts epilogue warps, and an issuing thread competes with
+// them for issue slots: while the epilogue of earlier tiles runs, one issuer gets an instruction out only every
+// ~150 cycles; four of them keep the pipe fed).  Warp 0's issuing thread is also the TMA producer.
+constexpr int kConvMmaWarps = 4;
+constexpr int kConvFirstEpiWarp = kConvMmaWarps;
+constexpr int kConvThreads = 32 * (kConvFirstEpiWarp + kEpiWarps);
 
 // 32 lanes each hold 32 items; afterwards lane l holds in q[0] the sum over all lanes of item l.
 __device__ __forceinline__ void transpose_reduce32(float (&q)[32], int lane) {
@@ -131,7 +138,7 @@ __device__ __forceinline__ void issue_tile(uint32_t d_tmem, uint64_t x_desc, con
 
 // ------------------------------------------------------- forward / data gradient --
 // out[pixel][n] (bf16, row stride Cn) = conv + (res ? res * [mask ? mask > 0 : 1] : 0)
-__global__ void __launch_bounds__(kFwdThreads, 1)
+__global__ void __launch_bounds__(kConvThreads, 1)
 conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, FwdParams p,
                  __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
                  const __nv_bfloat16* __restrict__ res_mask, EpiReduce red, int* __restrict__ error_word) {
@@ -153,11 +160,11 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   // Start-up that needs nothing from global memory: it may run while the preceding kernel of the stream is
   // still at work (programmatic dependent launch, see elementwise.cuh).
   if (red.mode)
-    for (int i = threadIdx.x; i < kEpiWarps * 8 * 32; i += kFwdThreads) red_run[i] = 0.f;
+    for (int i = threadIdx.x; i < kEpiWarps * 8 * 32; i += kConvThreads) red_run[i] = 0.f;
   if (threadIdx.x == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kMmaWarps); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kConvMmaWarps); }
     mbar_init(w_full, 1);
     const int groups_per_tile = p.Cn / 16 < kEpiGroups ? p.Cn / 16 : kEpiGroups;
     for (int a = 0; a < p.nacc; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4 * groups_per_tile); }
@@ -167,7 +174,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
   grid_dependency_wait();                  // from here on the preceding kernel's results may be read
   if (red.mode == 2)
-    for (int i = threadIdx.x; i < 2 * p.Cn; i += kFwdThreads) red_stat[i] = red.pstats[i];
+    for (int i = threadIdx.x; i < 2 * p.Cn; i += kConvThreads) red_stat[i] = red.pstats[i];
   if (threadIdx.x == 0) {
     // This thread is also the producer: the weights and the first tile are requested now, so that their
     // latency runs beside the barrier below instead of after it.
@@ -182,20 +189,26 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const uint32_t tmem_base = *tmem_slot;
   const int ksteps = p.Ck / 16;
 
-  if (warp == 0) {
+  if (warp < kConvFirstEpiWarp) {
     if (lane == 0) {
-      uint32_t it = 1;                                       // weights and tile 0 were requested during set-up
-      for (int tile = blockIdx.x + gridDim.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(&full[s], p.tile_tx_bytes);
-        tma_load_4d(smem + (size_t)s * p.stage_bytes, &map_x, &full[s], 0, -1, -1, tile * p.G);
-      }
-    }
-  } else if (warp < kFirstEpiWarp) {
-    if (lane == 0) {
-      const uint32_t issuer = warp - 1;                       // takes the 128-row tiles with acount % kMmaWarps == issuer
+      const uint32_t issuer = warp;                           // takes the 128-row tiles with acount % kConvMmaWarps == issuer
+      // Issuer 0 is also the producer: before it starts on a tile it requests the tiles that fit into the free
+      // stages (the weights and tile 0 were requested during set-up).  A stage's first use needs no wait; a
+      // later one waits until every issuer has handed the stage back.
+      uint32_t next_load = 1;
+      auto refill = [&](uint32_t upto) {
+        if (issuer != 0) return true;
+        for (; next_load < upto; ++next_load) {
+          const int tile = (int)blockIdx.x + (int)next_load * (int)gridDim.x;
+          if (tile >= p.tiles) return true;
+          const int s = next_load % p.stages;
+          const uint32_t ph = (next_load / p.stages) & 1;
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) return false;
+          mbar_expect_tx(&full[s], p.tile_tx_bytes);
+          tma_load_4d(smem + (size_t)s * p.stage_bytes, &map_x, &full[s], 0, -1, -1, tile * p.G);
+        }
+        return true;
+      };
       const uint32_t idesc = instr_desc(p.Cn, false);
       bool ok = mbar_wait(w_full, 0, abort_flag);
       tc_fence_after();
@@ -215,13 +228,14 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       int slot = 0;                                           // acount % nacc and the slot's phase, kept incrementally
       uint32_t aph = 0;
       for (int tile = blockIdx.x; ok && tile < p.tiles && !*abort_flag; tile += gridDim.x, ++it) {
+        if (!refill(it + (uint32_t)p.stages)) break;
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
         if (!mbar_wait(&full[s], ph, abort_flag)) break;
         tc_fence_after();
         uint64_t x_desc = smem_desc_kmajor(smem_u32(smem + (size_t)s * p.stage_bytes), p.pitch);
         for (int i = 0; i < p.m_tiles; ++i, ++acount, x_desc += mtile_step) {
-          if (acount % kMmaWarps == issuer) {
+          if (acount % kConvMmaWarps == issuer) {
             if (acount >= (uint32_t)p.nacc) {                 // a slot's first use needs no hand-back from the epilogue
               if (!mbar_wait(&acc_empty[slot], aph ^ 1, abort_flag)) { ok = false; break; }
               tc_fence_after();
@@ -247,7 +261,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // needs (slot, phase, the pixel of this thread's row) is carried from item to item by additions:
     // a division per item costs more here than the item's arithmetic.
     const int lane_grp = warp & 3;                 // tensor-memory lanes 32*(warp % 4) .. +31
-    const int group = (warp - kFirstEpiWarp) >> 2;
+    const int group = (warp - kConvFirstEpiWarp) >> 2;
     const int nch = p.Cn >> 4;
     // Items are numbered J = (128-row tiles so far) * nch + chunk over the whole CTA; group g takes
     // J = g, g + kEpiGroups, ...  One step of J is `step_a` 128-row tiles and `step_c` chunks.
@@ -385,7 +399,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
           }
         }
         transpose_reduce32(q, lane);
-        red_run[((warp - kFirstEpiWarp) * 8 + (c0 >> 4)) * 32 + lane] += q[0];
+        red_run[((warp - kConvFirstEpiWarp) * 8 + (c0 >> 4)) * 32 + lane] += q[0];
       }
       if (!have_next || nxt.first_chunk) {           // this group's last chunk of the 128-row tile: hand the slot back
         tc_fence_before();
@@ -505,14 +519,14 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         while (item_bwd16(run, oa, ob) && item_bwd16(run, ob, oa)) {}
       }
       transpose_reduce32(run, lane);
-      red_run[((warp - kFirstEpiWarp) * 8) * 32 + lane] += run[0];
+      red_run[((warp - kConvFirstEpiWarp) * 8) * 32 + lane] += run[0];
     } else if (red.mode == 1 && nch == 1 && !res) {
       float run[32];
 #pragma unroll
       for (int e = 0; e < 32; ++e) run[e] = 0.f;
       if (!*abort_flag && cur.tile < p.tiles) while (item_stats16(run)) {}
       transpose_reduce32(run, lane);
-      red_run[((warp - kFirstEpiWarp) * 8) * 32 + lane] += run[0];
+      red_run[((warp - kConvFirstEpiWarp) * 8) * 32 + lane] += run[0];
     } else {
       Operands op_a, op_b;
       if (!*abort_flag && cur.tile < p.tiles) {
@@ -544,7 +558,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   if (red.mode && !*abort_flag) {
     // this CTA's sums: item (chunk, lane) of all epilogue warps, added in warp order -> partial[cta][stat][channel]
     const int pairs = 2 * p.Cn;
-    for (int t = threadIdx.x; t < pairs; t += kFwdThreads) {
+    for (int t = threadIdx.x; t < pairs; t += kConvThreads) {
       const int stat = t / p.Cn, c = t - stat * p.Cn;
       const int idx = (c >> 4) * 32 + (c & 15) + 16 * stat;
       float a = 0.f;
@@ -779,12 +793,12 @@ inline FwdParams fwd_params(int N, int H, int W, int Ck, int Cn, int sm_count) {
   // that, a slot per 128-row tile where 256 columns allow it, so the issuers seldom wait for the epilogue.
   {
     const int nch = Cn / 16;
-    int step = kMmaWarps;
+    int step = kConvMmaWarps;
     if (nch < kEpiGroups) {
       int g = kEpiGroups, a = nch;                           // kEpiGroups / gcd(kEpiGroups, nch)
       while (a) { const int t = g % a; g = a; a = t; }
       const int need = kEpiGroups / g;
-      step = need % kMmaWarps == 0 ? need : need * kMmaWarps;
+      step = need % kConvMmaWarps == 0 ? need : need * kConvMmaWarps;
     }
     p.nacc = (p.m_tiles + step - 1) / step * step;
     while (p.nacc > step && p.nacc * Cn > 256) p.nacc -= step;
