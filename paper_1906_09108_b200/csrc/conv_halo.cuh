@@ -53,6 +53,10 @@ struct FwdParams {
 };
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Asks for `bytes` (a multiple of 16, from a 16-byte aligned address) to be brought into L2.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
 
 // Shared-memory descriptor of an MN-major operand made of swizzle-span-wide rows (one per k):
 // `lbo` = byte distance between consecutive MN blocks, 8-row k groups `8*row_bytes` apart.
@@ -196,6 +200,19 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       // stages (the weights and tile 0 were requested during set-up).  A stage's first use needs no wait; a
       // later one waits until every issuer has handed the stage back.
       uint32_t next_load = 1;
+      // The tensors the epilogue reads row by row (residual, its gate, the two operands of a fused batch-norm
+      // backward sum) are asked into L2 a whole tile ahead, so that the epilogue's loads do not wait for DRAM.
+      auto prefetch_operands = [&](int tile) {
+        int n0 = tile * p.G, n1 = n0 + p.G;
+        if (n1 > p.N) n1 = p.N;
+        const size_t img = (size_t)(p.sub == 1 ? p.H * p.W : (p.H >> 1) * (p.W >> 1)) * p.Cn;   // elements per image
+        const size_t off = (size_t)n0 * img;
+        const uint32_t bytes = (uint32_t)((size_t)(n1 - n0) * img * 2);
+        if (res) prefetch_l2_bulk(res + off, bytes);
+        if (res_mask) prefetch_l2_bulk(res_mask + off, bytes);
+        if (red.mode == 2) { prefetch_l2_bulk(red.mask + off, bytes); prefetch_l2_bulk(red.xprev + off, bytes); }
+      };
+      if (issuer == 0) prefetch_operands((int)blockIdx.x);
       auto refill = [&](uint32_t upto) {
         if (issuer != 0) return true;
         for (; next_load < upto; ++next_load) {
@@ -206,6 +223,7 @@ conv_halo_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) return false;
           mbar_expect_tx(&full[s], p.tile_tx_bytes);
           tma_load_4d(smem + (size_t)s * p.stage_bytes, &map_x, &full[s], 0, -1, -1, tile * p.G);
+          prefetch_operands(tile);
         }
         return true;
       };
