@@ -406,6 +406,10 @@ def run_kernel_bench(args):
             for stage in stages:
                 if which in ("sgd",) and stage != stages[0]:
                     continue
+                if which == "head" and not args.kernel_stage:      # the classifier sees the last stage's maps
+                    if stage != stages[0]:
+                        continue
+                    stage = "stage3"
                 us, nbytes = ew_kernel_bench(B, which, stage, launches=args.kernel_launches,
                                              reps=1 if args.kernel_launches <= 8 else 5, use_graph=args.kernel_launches > 8)
                 name = which + ("+reduce" if which == "bn_bwd_apply" and KERNEL_SHAPES[stage][3] > 128 else "")
