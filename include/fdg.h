@@ -89,8 +89,8 @@ typedef struct {
   float bn_eps;
 } fdg_arch;
 
-/* "Required: learning rate, number of split modules K, gradient shrinking factor
- * beta" (Algorithm I), plus the optimiser constants of the experiments section. */
+/* The inputs Algorithm I asks for (a learning rate per iteration, the number of modules K, the shrinking
+ * factor beta), plus the optimiser constants of the experiments section. */
 typedef struct {
   int K;                          /* number of modules, >= 1 */
   const int* split_after_block;   /* K-1 ascending block indices in [1, total blocks - 1]: module k ends after that block */

@@ -12,7 +12,8 @@ One call of `step` is one iteration t of Algorithm I for every module k=1..K:
     the end of iteration t-1, multiplied by beta (modules k<K only; the top
     module's gradient comes from the loss and is not shrunk, paragraph after
     Eq. 15).  The Jacobians are taken at the activations saved by the forward
-    of that same batch ("the activations generated by the same training batch").
+    of that same batch (the paragraph after Eq. 10 requires forward and backward of a
+    batch to meet the same activations).
   * update (Eq. 11) with the SGD-momentum / weight-decay optimiser of the
     experiments section.
   * communication (Section 3.1, "communication"; Fig. 1(a): "right before the

@@ -6,7 +6,7 @@
 //     written by the update kernel, so that the delayed backward of a batch can read
 //     the weights its forward used (superscripts of Eq. 10);
 //   * an activation FIFO: one slot per batch in flight holding everything the backward
-//     of that batch needs (Fig. 1(b): "the previously saved computation graph");
+//     of that batch needs (what Fig. 1(b) keeps as the computation graph saved by the forward);
 //   * a gradient mailbox (ring of 3) that receives the gradient of the module input
 //     and is read by the upstream module in the next iteration (Section 3.1,
 //     "communication");

@@ -151,7 +151,7 @@ def test_lr0_shrunk_gradient_is_beta_power_times_bp(family, K, splits, order):
 
 
 def test_beta_one_is_unshrunk():
-    """beta = 1: "the GS process is not used"; and beta only enters through the
+    """beta = 1 switches gradient shrinking off (Section 3.2); and beta only enters through the
     received gradient, so the top module's first update is beta-independent."""
     arch = tiny_arch(n=1)
     outs = []
