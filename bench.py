@@ -605,6 +605,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graphs", action="store_true")
     ap.add_argument("--workload", default="resnet110_k4", choices=list(WORKLOADS))
+    ap.add_argument("--splits", default=None,
+                    help="comma-separated block indices after which the modules end, instead of the workload's own")
     ap.add_argument("--kernel-bench", default=None, choices=["fprop", "dgrad", "wgrad", "all", "ew", "step"] + EW_KERNELS + list(STEP_VARIANTS),
                     help="time the convolution kernels alone through the operator-level C ABI and exit")
     ap.add_argument("--kernel-launches", type=int, default=64,
@@ -615,6 +617,10 @@ def main():
                          "baseline): the short run the ncu launch list is taken from")
     args = ap.parse_args()
     select_workload(args.workload)
+    if args.splits:
+        global SPLITS
+        SPLITS = tuple(int(v) for v in args.splits.split(","))
+        assert len(SPLITS) == K_MODULES - 1
     if args.kernel_bench:
         run_kernel_bench(args)
     elif args.impl == "reference":
