@@ -43,6 +43,9 @@ struct ConvTcParams {
   uint32_t a_bytes, b_bytes, stage_bytes;   // b_bytes is padded to 1 KiB; b_tx_bytes is what TMA moves
   uint32_t b_tx_bytes;
   uint32_t tmem_cols;       // allocated columns (power of two >= 2*n_tile)
+  int mpair;                // 128-row tiles a CTA works on at once with one weight tile: 1 (two accumulator sets, the
+                            // epilogue of a tile overlaps the next tile's instructions) or 2 (one set of two accumulators:
+                            // every weight tile fetched from L2 serves 256 rows)
   int sub;                  // 1, or 2: store only the pixels with even h and w, as an [N][H/2][W/2][Co] tensor
 };
 
@@ -162,21 +165,25 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int chunks = p.Ci / p.kc;
+  const int chunks = (p.Ci + p.kc - 1) / p.kc;
   const int k_iters = 9 * chunks;
-  const int total_tiles = p.m_tiles * p.n_tiles;
+  const int total_tiles = ((p.m_tiles + p.mpair - 1) / p.mpair) * p.n_tiles;     // tiles of mpair * 128 rows
 
   if (warp == 0) {
     if (lane == 0) {
       uint32_t it = 0;
       for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
-        const int mt = tile / p.n_tiles, nt = tile - mt * p.n_tiles;
-        int n0, h0;
-        if (p.imgs_per_tile == 1) {
-          const int tiles_per_img = p.H / p.rows_per_tile;
-          n0 = mt / tiles_per_img; h0 = (mt - n0 * tiles_per_img) * p.rows_per_tile;
-        } else {
-          n0 = mt * p.imgs_per_tile; h0 = 0;
+        const int mg = tile / p.n_tiles, nt = tile - mg * p.n_tiles;
+        int n0[2], h0[2];
+        const int halves = (mg * p.mpair + 1 < p.m_tiles) ? p.mpair : 1;
+        for (int hf = 0; hf < halves; ++hf) {
+          const int mt = mg * p.mpair + hf;
+          if (p.imgs_per_tile == 1) {
+            const int tiles_per_img = p.H / p.rows_per_tile;
+            n0[hf] = mt / tiles_per_img; h0[hf] = (mt - n0[hf] * tiles_per_img) * p.rows_per_tile;
+          } else {
+            n0[hf] = mt * p.imgs_per_tile; h0[hf] = 0;
+          }
         }
         for (int ki = 0; ki < k_iters; ++ki, ++it) {
           const int s = it % p.stages;
@@ -185,9 +192,10 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           const int tap = ki / chunks, cc = ki - tap * chunks;
           const int r = tap / 3, sx = tap - r * 3;
           uint8_t* a_dst = smem + (size_t)s * p.stage_bytes;
-          uint8_t* b_dst = a_dst + p.a_bytes;
-          mbar_expect_tx(&full[s], p.a_bytes + p.b_tx_bytes);
-          tma_load_4d(a_dst, &map_a, &full[s], cc * p.kc, sx - 1, h0 + r - 1, n0);
+          uint8_t* b_dst = a_dst + (size_t)p.mpair * p.a_bytes;
+          mbar_expect_tx(&full[s], (uint32_t)halves * p.a_bytes + p.b_tx_bytes);
+          for (int hf = 0; hf < halves; ++hf)
+            tma_load_4d(a_dst + (size_t)hf * p.a_bytes, &map_a, &full[s], cc * p.kc, sx - 1, h0[hf] + r - 1, n0[hf]);
           tma_load_2d(b_dst, &map_b, &full[s], tap * p.Ci + cc * p.kc, nt * p.n_tile);
         }
       }
@@ -197,12 +205,15 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t idesc = instr_desc_bf16(p.n_tile);
       const uint32_t row_bytes = p.kc * 2;
       uint32_t it = 0, tcount = 0;
+      const int nsets = p.mpair == 1 ? 2 : 1;                  // accumulator sets in tensor memory
       for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
-        const int acc = tcount & 1;
-        const uint32_t acc_ph = (tcount >> 1) & 1;
+        const int acc = (int)(tcount % nsets);
+        const uint32_t acc_ph = (tcount / nsets) & 1;
         if (!mbar_wait(&acc_empty[acc], acc_ph ^ 1, abort_flag)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * p.n_tile;
+        const int mg = tile / p.n_tiles;
+        const int halves = (mg * p.mpair + 1 < p.m_tiles) ? p.mpair : 1;
         bool ok = true;
         for (int ki = 0; ki < k_iters; ++ki, ++it) {
           const int s = it % p.stages;
@@ -210,10 +221,11 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
-          const uint32_t b_addr = a_addr + p.a_bytes;
-          for (int j = 0; j < p.kc / 16; ++j)
-            tc_mma_bf16(d_tmem, smem_desc_kmajor(a_addr + j * 32, row_bytes), smem_desc_kmajor(b_addr + j * 32, row_bytes),
-                        idesc, (ki | j) != 0);
+          const uint32_t b_addr = a_addr + (uint32_t)p.mpair * p.a_bytes;
+          for (int hf = 0; hf < halves; ++hf)
+            for (int j = 0; j < p.kc / 16; ++j)
+              tc_mma_bf16(d_tmem + (uint32_t)hf * p.n_tile, smem_desc_kmajor(a_addr + hf * p.a_bytes + j * 32, row_bytes),
+                          smem_desc_kmajor(b_addr + j * 32, row_bytes), idesc, (ki | j) != 0);
           tc_commit(&empty[s]);
         }
         if (!ok) break;
@@ -225,12 +237,16 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int lane_grp = warp & 3;
     (void)ew;
     uint32_t tcount = 0;
+    const int nsets = p.mpair == 1 ? 2 : 1;
     for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
-      const int mt = tile / p.n_tiles, nt = tile - mt * p.n_tiles;
-      const int acc = tcount & 1;
-      const uint32_t acc_ph = (tcount >> 1) & 1;
+      const int mg = tile / p.n_tiles, nt = tile - mg * p.n_tiles;
+      const int acc = (int)(tcount % nsets);
+      const uint32_t acc_ph = (tcount / nsets) & 1;
       if (!mbar_wait(&acc_full[acc], acc_ph, abort_flag)) break;
       tc_fence_after();
+      const int halves = (mg * p.mpair + 1 < p.m_tiles) ? p.mpair : 1;
+      for (int hf = 0; hf < halves; ++hf) {
+      const int mt = mg * p.mpair + hf;
       const size_t row = (size_t)mt * kTileM + lane_grp * 32 + lane;
       size_t base = row * p.Co + (size_t)nt * p.n_tile;
       bool keep = true;
@@ -240,7 +256,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         keep = ((h | w) & 1) == 0;
         base = (((n * (p.H >> 1) + (h >> 1)) * (p.W >> 1)) + (w >> 1)) * p.Co + (size_t)nt * p.n_tile;
       }
-      const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)acc * p.n_tile;
+      const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc + hf) * p.n_tile;
       for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
         uint32_t v[16];
         tmem_ld16(taddr + c0, v);
@@ -281,6 +297,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
         *reinterpret_cast<uint4*>(out + base + c0) = o0;
         *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+      }
       }
       tc_fence_before();
       __syncwarp();
@@ -348,7 +365,11 @@ inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co) {
   const int rows = kTileM / W;
   if (rows <= H) { p.rows_per_tile = rows; p.imgs_per_tile = 1; }
   else { p.rows_per_tile = H; p.imgs_per_tile = rows / H; }
-  p.kc = Ci % 64 == 0 ? 64 : (Ci % 32 == 0 ? 32 : 16);
+  // Channel chunk of a pipeline stage = one swizzle span.  Operand tiles arrive from L2 row by row, and a 128-byte
+  // row costs the same as a 64-byte one, so wide layers whose channel count is not a multiple of 64 (160) still
+  // take 64-channel chunks: the last chunk's surplus channels lie outside the activation tensor, are filled with
+  // zeros by the hardware, and so cancel whatever weights they meet.
+  p.kc = (Ci % 64 == 0 || Ci >= 128) ? 64 : (Ci % 32 == 0 ? 32 : 16);
   int nt = Co;
   if (nt > 256) { nt = 256; while (Co % nt || nt % 16) nt -= 16; }
   p.n_tile = nt;
@@ -357,7 +378,10 @@ inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co) {
   p.a_bytes = (uint32_t)kTileM * p.kc * 2;
   p.b_tx_bytes = (uint32_t)nt * p.kc * 2;
   p.b_bytes = (p.b_tx_bytes + 1023u) & ~1023u;
-  p.stage_bytes = p.a_bytes + p.b_bytes;
+  // The kernel is bound by the rate at which operand tiles arrive from L2, so a weight tile is shared by two
+  // 128-row tiles.
+  p.mpair = p.m_tiles >= 2 ? 2 : 1;
+  p.stage_bytes = (uint32_t)p.mpair * p.a_bytes + p.b_bytes;
   int stages = (int)(160 * 1024 / p.stage_bytes);
   p.stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
   uint32_t cols = 32;
@@ -415,7 +439,7 @@ inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const 
     cudaError_t e = conv_tc_set_attrs();
     if (e != cudaSuccess) return e;
   }
-  const int tiles = p.m_tiles * p.n_tiles;
+  const int tiles = ((p.m_tiles + p.mpair - 1) / p.mpair) * p.n_tiles;
   const int grid = tiles < sm_count ? tiles : sm_count;
   conv3x3_tc_kernel<<<grid, kThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, error_word);
   return cudaGetLastError();
