@@ -49,7 +49,7 @@ inline cudaError_t run_conv_tc(cudaStream_t st, TensorMapCache* cache, int N, in
   p.sub = sub;
   TensorMapCache::Key ka, kb;
   std::memset(&ka, 0, sizeof(ka)); std::memset(&kb, 0, sizeof(kb));
-  ka.ptr = act; ka.d[0] = 1; ka.d[1] = N; ka.d[2] = H; ka.d[3] = W; ka.d[4] = Ck; ka.d[5] = p.kc;
+  ka.ptr = act; ka.d[0] = 1; ka.d[1] = N; ka.d[2] = H; ka.d[3] = W; ka.d[4] = Ck; ka.d[5] = p.kc; ka.d[6] = p.patch;
   kb.ptr = wgt; kb.d[0] = 2; kb.d[1] = Ck; kb.d[2] = Cn; kb.d[3] = p.kc; kb.d[4] = p.n_tile;
   auto ia = cache->maps.find(ka), ib = cache->maps.find(kb);
   if (ia == cache->maps.end() || ib == cache->maps.end()) {

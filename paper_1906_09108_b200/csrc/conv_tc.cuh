@@ -47,7 +47,12 @@ struct ConvTcParams {
                             // epilogue of a tile overlaps the next tile's instructions) or 2 (one set of two accumulators:
                             // every weight tile fetched from L2 serves 256 rows)
   int sub;                  // 1, or 2: store only the pixels with even h and w, as an [N][H/2][W/2][Co] tensor
+  int patch;                // 1: conv3x3_patch_kernel (16x16-pixel patches with their halo), 0: conv3x3_tc_kernel
+  uint32_t halo_bytes;      // patch mode: shared memory of one 18x18-pixel halo tile of kc channels (multiple of 1 KiB)
+  int b_stages;             // patch mode: weight tiles in flight
 };
+constexpr int kPatch = 16;                         // patch side in pixels
+constexpr int kPatchHalo = kPatch + 2;             // with the one-pixel border
 
 // ---------------------------------------------------------------- PTX wrappers --
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -128,6 +133,17 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t row
   d |= (uint64_t)1 << 16;                                // leading byte offset (unused for one span)
   d |= (uint64_t)(((8 * row_bytes) >> 4) & 0x3FFF) << 32;   // stride byte offset between 8-row groups
   d |= (uint64_t)1 << 46;                                // descriptor version of this architecture
+  d |= layout << 61;
+  return d;
+}
+// The same with an explicit distance between 8-row groups (rows inside a group stay one span apart).
+__device__ __forceinline__ uint64_t smem_desc_kmajor_sbo(uint32_t addr, uint32_t row_bytes, uint32_t group_bytes) {
+  const uint64_t layout = row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6);
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)((group_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
   d |= layout << 61;
   return d;
 }
@@ -324,6 +340,226 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   }
 }
 
+// ------------------------------------------------------- patch-tile kernel ----
+// Wide layers on images whose sides are multiples of 16.  conv3x3_tc_kernel fetches a 128-pixel activation tile
+// again for each of the nine filter taps, and the rate at which operand rows arrive from L2 is what bounds it.
+// Here a CTA works on a 16x16-pixel patch: for each 64-channel chunk ONE load brings the patch with its one-pixel
+// border (18x18 pixels, out-of-bounds pixels filled with zeros: the padding) into swizzled shared memory, and
+// the nine taps are nine start addresses into it.  The patch is two 128-row tiles: tile g holds pixel columns
+// 8g..8g+7 of the 16 patch rows, so that consecutive 8-row groups of an operand are always one halo row (18
+// pixels) apart and one shared-memory descriptor describes them.  Only the weight tiles (one per tap and chunk,
+// shared by both 128-row tiles) still stream per tap.
+//   A operand of (tap r,s; tile g): start = halo + ((r*18 + s + 8g) pixels), groups 18 pixels apart
+//   accumulator row i of tile g  <->  patch pixel (h = i / 8, w = 8g + i % 8)
+// Shared memory: two halo buffers (chunk c+1 lands while chunk c is multiplied) and a ring of weight tiles.
+__global__ void __launch_bounds__(kThreads, 1)
+conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     ConvTcParams p, __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
+                     const __nv_bfloat16* __restrict__ res_mask, int* __restrict__ error_word) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* b_smem = smem + 2 * (size_t)p.halo_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(b_smem + (size_t)p.b_stages * p.b_bytes);
+  uint64_t* a_full = bars;                     // [2]         TMA -> MMA, halo tiles
+  uint64_t* a_empty = a_full + 2;              // [2]         MMA -> TMA
+  uint64_t* full = a_empty + 2;                // [b_stages]  TMA -> MMA, weight tiles
+  uint64_t* empty = full + p.b_stages;         // [b_stages]  MMA -> TMA
+  uint64_t* acc_full = empty + p.b_stages;     // [1]         MMA -> epilogue
+  uint64_t* acc_empty = acc_full + 1;          // [1]         epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 2; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
+    for (int s = 0; s < p.b_stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 4);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, p.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int chunks = (p.Ci + p.kc - 1) / p.kc;
+  const int pw_cnt = p.W / kPatch, ph_cnt = p.H / kPatch;
+  const int total_tiles = p.N * ph_cnt * pw_cnt * p.n_tiles;
+  const uint32_t halo_tx = (uint32_t)kPatchHalo * kPatchHalo * p.kc * 2;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // One step = (tile, channel chunk): its halo tile, then its nine weight tiles.  The next step's halo tile is
+      // requested from the middle of this step's taps: by then the multiplier has started on this step, so the
+      // buffer the next tile goes to (the previous step's) has been handed back and nothing blocks here.
+      uint32_t q = 0, itb = 0;                  // steps and weight tiles requested so far
+      bool ok = true;
+      auto load_halo = [&](int tile, int cc, uint32_t step) {
+        const int pt = tile / p.n_tiles;
+        const int n = pt / (ph_cnt * pw_cnt), rem = pt - n * ph_cnt * pw_cnt;
+        const int ph = rem / pw_cnt, pw = rem - ph * pw_cnt;
+        const int sa = step & 1;
+        if (!mbar_wait(&a_empty[sa], ((step >> 1) & 1) ^ 1, abort_flag)) return false;
+        mbar_expect_tx(&a_full[sa], halo_tx);
+        tma_load_4d(smem + (size_t)sa * p.halo_bytes, &map_a, &a_full[sa], cc * p.kc, pw * kPatch - 1, ph * kPatch - 1, n);
+        return true;
+      };
+      if ((int)blockIdx.x < total_tiles) ok = load_halo(blockIdx.x, 0, 0);
+      for (int tile = blockIdx.x; ok && tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+        const int nt = tile % p.n_tiles;
+        for (int cc = 0; ok && cc < chunks; ++cc, ++q) {
+          // the step after this one
+          int ntile = tile, ncc = cc + 1;
+          if (ncc == chunks) { ncc = 0; ntile = tile + gridDim.x; }
+          for (int tap = 0; tap < 9; ++tap, ++itb) {
+            if (tap == 4 && ntile < total_tiles) { ok = load_halo(ntile, ncc, q + 1); if (!ok) break; }
+            const int s = itb % p.b_stages;
+            const uint32_t ph = (itb / p.b_stages) & 1;
+            if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(&full[s], p.b_tx_bytes);
+            tma_load_2d(b_smem + (size_t)s * p.b_bytes, &map_b, &full[s], tap * p.Ci + cc * p.kc, nt * p.n_tile);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(p.n_tile);
+      const uint32_t row_bytes = p.kc * 2;
+      const uint32_t group_bytes = kPatchHalo * row_bytes;
+      // The issuing thread is alone in its warp: every instruction it spends between two tcgen05.mma costs its full
+      // latency.  All descriptors are therefore formed once, and moving an operand is a 64-bit add on the
+      // descriptor's address field (16-byte units).
+      uint64_t halo_desc[2], b_desc[6], tap_off[9];
+      for (int i = 0; i < 2; ++i) halo_desc[i] = smem_desc_kmajor_sbo(smem_u32(smem + (size_t)i * p.halo_bytes), row_bytes, group_bytes);
+      for (int i = 0; i < 6; ++i) b_desc[i] = smem_desc_kmajor(smem_u32(b_smem + (size_t)(i < p.b_stages ? i : 0) * p.b_bytes), row_bytes);
+#pragma unroll
+      for (int tap = 0; tap < 9; ++tap) tap_off[tap] = (uint64_t)(((tap / 3) * kPatchHalo + (tap % 3)) * row_bytes) >> 4;
+      const uint64_t g_off = (uint64_t)(8 * row_bytes) >> 4;
+      const uint32_t acc1 = tmem_base + (uint32_t)p.n_tile;
+      uint32_t q = 0, itb = 0, tcount = 0;
+      int s = 0;
+      uint32_t ph = 0;                                         // itb % b_stages and that stage's phase, kept incrementally
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
+        if (!mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag)) break;
+        tc_fence_after();
+        for (int cc = 0; ok && cc < chunks; ++cc, ++q) {
+          const int sa = q & 1;
+          if (!mbar_wait(&a_full[sa], (q >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int tap = 0; tap < 9; ++tap, ++itb) {
+            if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t a0 = halo_desc[sa] + tap_off[tap], b0 = b_desc[s];
+            const uint32_t first = (uint32_t)(cc | tap);
+            tc_mma_bf16(tmem_base, a0, b0, idesc, first);
+            tc_mma_bf16(tmem_base, a0 + 2, b0 + 2, idesc, 1);
+            tc_mma_bf16(tmem_base, a0 + 4, b0 + 4, idesc, 1);
+            tc_mma_bf16(tmem_base, a0 + 6, b0 + 6, idesc, 1);
+            tc_mma_bf16(acc1, a0 + g_off, b0, idesc, first);
+            tc_mma_bf16(acc1, a0 + g_off + 2, b0 + 2, idesc, 1);
+            tc_mma_bf16(acc1, a0 + g_off + 4, b0 + 4, idesc, 1);
+            tc_mma_bf16(acc1, a0 + g_off + 6, b0 + 6, idesc, 1);
+            tc_commit(&empty[s]);
+            if (++s == p.b_stages) { s = 0; ph ^= 1; }
+          }
+          if (ok) tc_commit(&a_empty[sa]);
+        }
+        if (ok) tc_commit(acc_full);
+      }
+    }
+  } else {
+    const int lane_grp = warp & 3;
+    uint32_t tcount = 0;
+    for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
+      const int pt = tile / p.n_tiles, nt = tile - pt * p.n_tiles;
+      const int n = pt / (ph_cnt * pw_cnt), rem = pt - n * ph_cnt * pw_cnt;
+      const int ph = rem / pw_cnt, pw = rem - ph * pw_cnt;
+      if (!mbar_wait(acc_full, tcount & 1, abort_flag)) break;
+      tc_fence_after();
+      const int i = lane_grp * 32 + lane;                       // accumulator row of this thread
+      for (int g = 0; g < 2; ++g) {
+        const int h = ph * kPatch + (i >> 3), w = pw * kPatch + 8 * g + (i & 7);
+        size_t base;
+        bool keep = true;
+        if (p.sub == 1) {
+          base = (((size_t)n * p.H + h) * p.W + w) * p.Co + (size_t)nt * p.n_tile;
+        } else {
+          keep = ((h | w) & 1) == 0;
+          base = (((size_t)n * (p.H >> 1) + (h >> 1)) * (p.W >> 1) + (w >> 1)) * p.Co + (size_t)nt * p.n_tile;
+        }
+        const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)g * p.n_tile;
+        for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(taddr + c0, v);
+          tmem_ld_wait();
+          if (!keep) continue;
+          float f[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]);
+          if (res) {
+            uint4 r0 = *reinterpret_cast<const uint4*>(res + base + c0);
+            uint4 r1 = *reinterpret_cast<const uint4*>(res + base + c0 + 8);
+            const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
+            const __nv_bfloat16* rb1 = reinterpret_cast<const __nv_bfloat16*>(&r1);
+            float gq[16];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { gq[e] = __bfloat162float(rb0[e]); gq[8 + e] = __bfloat162float(rb1[e]); }
+            if (res_mask) {
+              uint4 m0 = *reinterpret_cast<const uint4*>(res_mask + base + c0);
+              uint4 m1 = *reinterpret_cast<const uint4*>(res_mask + base + c0 + 8);
+              const __nv_bfloat16* mb0 = reinterpret_cast<const __nv_bfloat16*>(&m0);
+              const __nv_bfloat16* mb1 = reinterpret_cast<const __nv_bfloat16*>(&m1);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                if (!(__bfloat162float(mb0[e]) > 0.f)) gq[e] = 0.f;
+                if (!(__bfloat162float(mb1[e]) > 0.f)) gq[8 + e] = 0.f;
+              }
+            }
+#pragma unroll
+            for (int e = 0; e < 16; ++e) f[e] += gq[e];
+          }
+          uint4 o0, o1;
+          __nv_bfloat162* ob0 = reinterpret_cast<__nv_bfloat162*>(&o0);
+          __nv_bfloat162* ob1 = reinterpret_cast<__nv_bfloat162*>(&o1);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            ob0[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+            ob1[e] = __floats2bfloat162_rn(f[8 + 2 * e], f[8 + 2 * e + 1]);
+          }
+          *reinterpret_cast<uint4*>(out + base + c0) = o0;
+          *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) {
+      if (error_word) atomicExch(error_word, 1);
+      for (int s = 0; s < 2 + p.b_stages; ++s) {
+        uint64_t* b = s < 2 ? &a_full[s] : &full[s - 2];
+        for (uint32_t i = 0; i < (1u << 16); ++i)
+          if (mbar_try_wait(b, 0) || mbar_try_wait(b, 1)) break;
+      }
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, p.tmem_cols);
+  }
+}
+
 // ----------------------------------------------------------------- host side ---
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -382,6 +618,12 @@ inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co) {
   // 128-row tiles.
   p.mpair = p.m_tiles >= 2 ? 2 : 1;
   p.stage_bytes = (uint32_t)p.mpair * p.a_bytes + p.b_bytes;
+  // 16x16-pixel patches with their halo wherever the image allows it and the chunks are full swizzle spans
+  p.patch = (H % kPatch == 0 && W % kPatch == 0 && p.kc == 64) ? 1 : 0;
+  p.halo_bytes = ((uint32_t)kPatchHalo * kPatchHalo * p.kc * 2 + 1023u) & ~1023u;
+  p.b_stages = (int)((176 * 1024 - 2 * (size_t)p.halo_bytes) / p.b_bytes);
+  if (p.b_stages > 6) p.b_stages = 6;
+  if (p.b_stages < 2) p.patch = 0;
   int stages = (int)(160 * 1024 / p.stage_bytes);
   p.stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
   uint32_t cols = 32;
@@ -390,7 +632,10 @@ inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co) {
   return p;
 }
 
-inline size_t conv_tc_smem_bytes(const ConvTcParams& p) { return (size_t)p.stages * p.stage_bytes + 1024 + 256; }
+inline size_t conv_tc_smem_bytes(const ConvTcParams& p) {
+  if (p.patch) return 2 * (size_t)p.halo_bytes + (size_t)p.b_stages * p.b_bytes + 1024 + 256;
+  return (size_t)p.stages * p.stage_bytes + 1024 + 256;
+}
 
 // act: bf16 [N][H][W][Ci]; wgt: bf16 [Co][9*Ci] (forward layout, or the flipped/transposed copy for dgrad).
 inline cudaError_t conv_tc_make_maps(const ConvTcParams& p, const void* act, const void* wgt, CUtensorMap* map_a,
@@ -402,6 +647,7 @@ inline cudaError_t conv_tc_make_maps(const ConvTcParams& p, const void* act, con
     cuuint64_t dims[4] = {(cuuint64_t)p.Ci, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.N};
     cuuint64_t strides[3] = {(cuuint64_t)p.Ci * 2, (cuuint64_t)p.W * p.Ci * 2, (cuuint64_t)p.H * p.W * p.Ci * 2};
     cuuint32_t box[4] = {(cuuint32_t)p.kc, (cuuint32_t)p.W, (cuuint32_t)p.rows_per_tile, (cuuint32_t)p.imgs_per_tile};
+    if (p.patch) { box[1] = kPatchHalo; box[2] = kPatchHalo; box[3] = 1; }
     cuuint32_t estr[4] = {1, 1, 1, 1};
     if (enc(map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(act), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -427,6 +673,7 @@ inline cudaError_t conv_tc_set_attrs() {
   static bool attr_set = false;
   if (attr_set) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(conv3x3_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_patch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e == cudaSuccess) attr_set = true;
   return e;
 }
@@ -438,6 +685,12 @@ inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const 
   {
     cudaError_t e = conv_tc_set_attrs();
     if (e != cudaSuccess) return e;
+  }
+  if (p.patch) {
+    const int tiles = p.N * (p.H / kPatch) * (p.W / kPatch) * p.n_tiles;
+    const int grid = tiles < sm_count ? tiles : sm_count;
+    conv3x3_patch_kernel<<<grid, kThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, error_word);
+    return cudaGetLastError();
   }
   const int tiles = ((p.m_tiles + p.mpair - 1) / p.mpair) * p.n_tiles;
   const int grid = tiles < sm_count ? tiles : sm_count;
