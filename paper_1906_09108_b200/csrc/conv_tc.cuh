@@ -222,6 +222,18 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t row_bytes = p.kc * 2;
       uint32_t it = 0, tcount = 0;
       const int nsets = p.mpair == 1 ? 2 : 1;                  // accumulator sets in tensor memory
+      // Descriptors are formed once per stage; moving an operand is a 64-bit add on the address field (the issuing
+      // thread is alone in its warp, so every instruction between two tcgen05.mma costs its full latency).
+      uint64_t a_desc[8], b_desc[8];
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t a_addr = smem_u32(smem + (size_t)(i < p.stages ? i : 0) * p.stage_bytes);
+        a_desc[i] = smem_desc_kmajor(a_addr, row_bytes);
+        b_desc[i] = smem_desc_kmajor(a_addr + (uint32_t)p.mpair * p.a_bytes, row_bytes);
+      }
+      const uint64_t half_off = (uint64_t)p.a_bytes >> 4;
+      const int ksub = p.kc / 16;
+      int s = 0;
+      uint32_t ph = 0;                                         // it % stages and that stage's phase, kept incrementally
       for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
         const int acc = (int)(tcount % nsets);
         const uint32_t acc_ph = (tcount / nsets) & 1;
@@ -232,17 +244,14 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int halves = (mg * p.mpair + 1 < p.m_tiles) ? p.mpair : 1;
         bool ok = true;
         for (int ki = 0; ki < k_iters; ++ki, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1;
           if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
-          const uint32_t b_addr = a_addr + (uint32_t)p.mpair * p.a_bytes;
-          for (int hf = 0; hf < halves; ++hf)
-            for (int j = 0; j < p.kc / 16; ++j)
-              tc_mma_bf16(d_tmem + (uint32_t)hf * p.n_tile, smem_desc_kmajor(a_addr + hf * p.a_bytes + j * 32, row_bytes),
-                          smem_desc_kmajor(b_addr + j * 32, row_bytes), idesc, (ki | j) != 0);
+          const uint64_t a0 = a_desc[s], b0 = b_desc[s];
+          for (int j = 0; j < ksub; ++j) tc_mma_bf16(d_tmem, a0 + 2 * j, b0 + 2 * j, idesc, (ki | j) != 0);
+          if (halves == 2)
+            for (int j = 0; j < ksub; ++j) tc_mma_bf16(d_tmem + (uint32_t)p.n_tile, a0 + half_off + 2 * j, b0 + 2 * j, idesc, (ki | j) != 0);
           tc_commit(&empty[s]);
+          if (++s == p.stages) { s = 0; ph ^= 1; }
         }
         if (!ok) break;
         tc_commit(&acc_full[acc]);
