@@ -361,7 +361,8 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 //   A operand of (tap r,s; tile g): start = halo + ((r*18 + s + 8g) pixels), groups 18 pixels apart
 //   accumulator row i of tile g  <->  patch pixel (h = i / 8, w = 8g + i % 8)
 // Shared memory: two halo buffers (chunk c+1 lands while chunk c is multiplied) and a ring of weight tiles.
-__global__ void __launch_bounds__(kThreads, 1)
+constexpr int kPatchThreads = 224;       // TMA warp, issuing warp of tile 0, four epilogue warps, issuing warp of tile 1
+__global__ void __launch_bounds__(kPatchThreads, 1)
 conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      ConvTcParams p, __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
                      const __nv_bfloat16* __restrict__ res_mask, int* __restrict__ error_word) {
@@ -380,9 +381,9 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 2; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 1); }
-    for (int s = 0; s < p.b_stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(acc_full, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 2); }
+    for (int s = 0; s < p.b_stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 2); }
+    mbar_init(acc_full, 2);
     mbar_init(acc_empty, 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -433,8 +434,11 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == 6) {
+    // Two issuing threads, one per 128-row tile of the patch (each into its own accumulator): one thread gets a
+    // tcgen05.mma out only every ~110 cycles, the pipe takes one of N = 160 every 80.
     if (lane == 0) {
+      const int g = warp == 1 ? 0 : 1;
       const uint32_t idesc = instr_desc_bf16(p.n_tile);
       const uint32_t row_bytes = p.kc * 2;
       const uint32_t group_bytes = kPatchHalo * row_bytes;
@@ -446,8 +450,8 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       for (int i = 0; i < 6; ++i) b_desc[i] = smem_desc_kmajor(smem_u32(b_smem + (size_t)(i < p.b_stages ? i : 0) * p.b_bytes), row_bytes);
 #pragma unroll
       for (int tap = 0; tap < 9; ++tap) tap_off[tap] = (uint64_t)(((tap / 3) * kPatchHalo + (tap % 3)) * row_bytes) >> 4;
-      const uint64_t g_off = (uint64_t)(8 * row_bytes) >> 4;
-      const uint32_t acc1 = tmem_base + (uint32_t)p.n_tile;
+      const uint64_t g_off = (uint64_t)(8 * g * row_bytes) >> 4;
+      const uint32_t d_tmem = tmem_base + (uint32_t)(g * p.n_tile);
       uint32_t q = 0, itb = 0, tcount = 0;
       int s = 0;
       uint32_t ph = 0;                                         // itb % b_stages and that stage's phase, kept incrementally
@@ -463,16 +467,11 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           for (int tap = 0; tap < 9; ++tap, ++itb) {
             if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const uint64_t a0 = halo_desc[sa] + tap_off[tap], b0 = b_desc[s];
-            const uint32_t first = (uint32_t)(cc | tap);
-            tc_mma_bf16(tmem_base, a0, b0, idesc, first);
-            tc_mma_bf16(tmem_base, a0 + 2, b0 + 2, idesc, 1);
-            tc_mma_bf16(tmem_base, a0 + 4, b0 + 4, idesc, 1);
-            tc_mma_bf16(tmem_base, a0 + 6, b0 + 6, idesc, 1);
-            tc_mma_bf16(acc1, a0 + g_off, b0, idesc, first);
-            tc_mma_bf16(acc1, a0 + g_off + 2, b0 + 2, idesc, 1);
-            tc_mma_bf16(acc1, a0 + g_off + 4, b0 + 4, idesc, 1);
-            tc_mma_bf16(acc1, a0 + g_off + 6, b0 + 6, idesc, 1);
+            const uint64_t a0 = halo_desc[sa] + tap_off[tap] + g_off, b0 = b_desc[s];
+            tc_mma_bf16(d_tmem, a0, b0, idesc, (uint32_t)(cc | tap));
+            tc_mma_bf16(d_tmem, a0 + 2, b0 + 2, idesc, 1);
+            tc_mma_bf16(d_tmem, a0 + 4, b0 + 4, idesc, 1);
+            tc_mma_bf16(d_tmem, a0 + 6, b0 + 6, idesc, 1);
             tc_commit(&empty[s]);
             if (++s == p.b_stages) { s = 0; ph ^= 1; }
           }
@@ -481,7 +480,7 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (ok) tc_commit(acc_full);
       }
     }
-  } else {
+  } else if (warp >= 2 && warp <= 5) {
     const int lane_grp = warp & 3;
     uint32_t tcount = 0;
     for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
@@ -698,7 +697,7 @@ inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const 
   if (p.patch) {
     const int tiles = p.N * (p.H / kPatch) * (p.W / kPatch) * p.n_tiles;
     const int grid = tiles < sm_count ? tiles : sm_count;
-    conv3x3_patch_kernel<<<grid, kThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, error_word);
+    conv3x3_patch_kernel<<<grid, kPatchThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, error_word);
     return cudaGetLastError();
   }
   const int tiles = ((p.m_tiles + p.mpair - 1) / p.mpair) * p.n_tiles;
