@@ -66,6 +66,9 @@ WORKLOADS = {
     "wrn28_10_k2": dict(arch=dict(family="wrn", n_per_stage=4, widths=(160, 320, 640), stem_width=16, in_h=32, in_w=32,
                                   in_c=3, num_classes=100, batch=128), K=2, splits=(6,), beta=0.6, lr=0.1,
                         name="WRN-28-10 K=2 batch 128, 32x32x3 synthetic N(0,1), 100 classes"),
+    "resnet18_k2": dict(arch=dict(family="resnet6n2", blocks=(2, 2, 2, 2), widths=(64, 128, 256, 512), stem_width=64, in_h=32,
+                                  in_w=32, in_c=3, num_classes=10, batch=128), K=2, splits=(4,), beta=0.5, lr=0.1,
+                        name="CIFAR ResNet-18 (4 stages of 2 basic blocks, 64..512 channels) K=2 batch 128, 32x32x3 synthetic N(0,1)"),
     "resnet1202_k4": dict(arch=dict(family="resnet6n2", n_per_stage=200, widths=(16, 32, 64), stem_width=16, in_h=32,
                                     in_w=32, in_c=3, num_classes=10, batch=64), K=4, splits=(150, 300, 450), beta=0.5,
                           lr=0.01, name="ResNet-1202 (6n+2, n=200) K=4 batch 64, 32x32x3 synthetic N(0,1), 10 classes"),
@@ -555,6 +558,20 @@ def run_gpu(args):
                         # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this shape,
                         # from the committed ncu summary; null once the kernel's source has changed since
                         traffic=profiled_traffic())
+            # The same kernels in the launch shape the module-step issues them in (a third of the SMs, three image
+            # tiles per CTA, reductions fused into the epilogue), the two batch-norm apply kernels at the stage-1
+            # shape, and the wide-layer convolution against the tensor roofline: each timed alone the same way.
+            iso = {}
+            for kind in STEP_VARIANTS:
+                u2, b2, f2 = kernel_bench(B, kind, "stage1")
+                iso[kind + "_stage1"] = dict(us=u2, gbs=b2 / u2 / 1e3, frac_hbm=b2 / u2 / 1e3 / peaks["hbm_gbs"])
+            for kind in ("bn_apply_res", "bn_bwd_apply"):
+                u2, b2 = ew_kernel_bench(B, kind, "stage1")
+                iso[kind + "_stage1"] = dict(us=u2, gbs=b2 / u2 / 1e3, frac_hbm=b2 / u2 / 1e3 / peaks["hbm_gbs"])
+            u2, b2, f2 = kernel_bench(B, "fprop", "wrn_stage2", launches=16)
+            iso["fprop_wrn_stage2"] = dict(us=u2, tflops=f2 / u2 / 1e6, frac_tensor=f2 / u2 / 1e6 / peaks["bf16_tflops"],
+                                           kernel="conv3x3_patch_kernel, [128,16,16,320] -> 320 channels")
+            roof["isolated"] = iso
         elif top["name"].startswith("conv"):
             # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x max SM clock
             alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
