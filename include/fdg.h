@@ -263,6 +263,13 @@ fdg_status fdg_sync(fdg_ctx* ctx, fdg_stream stream);
  * fdg_sync returns it.  Blocks the host. */
 fdg_status fdg_debug_raise_flag(fdg_ctx* ctx, int which);
 
+/* A wait that really runs out, without a kernel that misbehaves: enqueues on `stream` a one-warp kernel that
+ * waits, with the bounded wait of the tensor-core kernels, on a barrier nothing ever arrives at.  After
+ * `poll_limit` polls (1..2^20; a poll is well under a microsecond) the wait gives up, the kernel raises the
+ * time-out status word as a convolution kernel would, and returns: no copy is in flight and no tensor memory
+ * is held.  The next fdg_sync returns FDG_ERR_TIMEOUT (latched); the CUDA context stays usable.  Does not block. */
+fdg_status fdg_debug_wait_probe(fdg_ctx* ctx, fdg_stream stream, unsigned poll_limit);
+
 /* The most recent output activation of module k (1..K-1), and the most recent gradient
  * with respect to the input of module k (2..K; the gradient with respect to the images
  * is never formed, so k = 1 is FDG_ERR_INVALID_ARG), as fp32 NHWC to host or device memory.  `n` must equal the tensor's element

@@ -30,7 +30,7 @@ EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count"
            "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_wgrad_static", "fdg_conv_path",
            "fdg_get_saved_tensor_of", "fdg_capture_bytes", "fdg_capture_begin", "fdg_capture_end", "fdg_get_captured",
            "fdg_bn_scratch_bytes", "fdg_bn_stats", "fdg_bn_apply", "fdg_bn_backward", "fdg_shrink", "fdg_sgd_update",
-           "fdg_ingest", "fdg_head", "fdg_debug_raise_flag", "fdg_lr_at", "fdg_set_lr_schedule", "fdg_bn_running_count",
+           "fdg_ingest", "fdg_head", "fdg_debug_raise_flag", "fdg_debug_wait_probe", "fdg_lr_at", "fdg_set_lr_schedule", "fdg_bn_running_count",
            "fdg_get_bn_running", "fdg_set_bn_running", "fdg_eval", "fdg_drain", "fdg_state_bytes", "fdg_save_state",
            "fdg_load_state"]
 
@@ -127,6 +127,7 @@ def load_library(path=LIB_PATH):
         "fdg_conv_wgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, sz, P(fdg_conv_extra), vp, vp],
         "fdg_get_saved_tensor_of": [vp, C.c_int, C.c_int, C.c_int, i64, vp, sz, P(sz), P(i64)],
         "fdg_debug_raise_flag": [vp, C.c_int],
+        "fdg_debug_wait_probe": [vp, vp, C.c_uint],
         "fdg_lr_at": [P(fdg_lr_schedule), i64, P(C.c_float)],
         "fdg_set_lr_schedule": [vp, P(fdg_lr_schedule)],
         "fdg_bn_running_count": [vp, C.c_int, P(sz)],

@@ -76,13 +76,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false when the limit is hit or another role has raised *abort_flag.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t limit = kSpinLimit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023) == 1023 && *abort_flag) return false;
   }
   *abort_flag = 1;
   return false;
+}
+
+// One warp waits, with the bounded wait above, on a barrier that nothing ever arrives at: after `limit`
+// polls the wait gives up and the kernel reports it the way the convolution kernels do.  Nothing is in
+// flight and no tensor memory is held when it leaves.  Lets the host-side handling of a wait that ran
+// out be exercised without making a real kernel misbehave.
+__global__ void wait_probe_kernel(uint32_t limit, int* error_word) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int flag;
+  volatile int* abort_flag = &flag;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(&bar, 0, abort_flag, limit);
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0 && error_word) atomicExch(error_word, 1);
 }
 
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3) {

@@ -1538,6 +1538,15 @@ fdg_status fdg_debug_raise_flag(fdg_ctx* c, int which) {
   return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "raising a status word");
 }
 
+fdg_status fdg_debug_wait_probe(fdg_ctx* c, fdg_stream stream, unsigned poll_limit) {
+  if (!c) return FDG_ERR_INVALID_ARG;
+  if (poll_limit < 1 || poll_limit > (1u << 20)) return fail(c, FDG_ERR_INVALID_ARG, "poll limit outside 1..2^20");
+  tc::wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(poll_limit, c->flags + 2);
+  ++c->launches;
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "wait probe");
+}
+
 static fdg_status export_tensor(fdg_ctx* c, const void* src, size_t rows, int c_store, int c_logical, float* dst, size_t n) {
   if (n != rows * (size_t)c_logical) return fail(c, FDG_ERR_INVALID_ARG, "element count does not match fdg_boundary_elems");
   cudaError_t e = drain(c);

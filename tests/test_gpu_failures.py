@@ -1,6 +1,7 @@
 """Error paths of the library, exercised without making any kernel misbehave: bad inputs the kernels detect
 and survive (a non-finite loss, a label out of range), and status words raised from the host the way a
-kernel would raise them (fdg_debug_raise_flag), checked through what fdg_sync and fdg_step report."""
+kernel would raise them (fdg_debug_raise_flag), and a bounded wait that is made to run out on a barrier nothing
+sets (fdg_debug_wait_probe); all checked through what fdg_sync and fdg_step report."""
 import numpy as np
 import pytest
 import torch
@@ -96,3 +97,29 @@ def test_raised_status_words_reach_the_caller():
     assert _status(g, g.sync) == 7                                   # latched
     assert _status(g, g.step, *_batch(9)) == 7
     g.close()
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    """A one-warp kernel waits, with the bounded wait of the tensor-core kernels, on a barrier nothing arrives
+    at; after a few thousand polls it gives up, raises the time-out word and returns (nothing is in flight, no
+    tensor memory held).  The context latches FDG_ERR_TIMEOUT; the device and a new context carry on."""
+    import torch
+    from paper_1906_09108_b200 import binding as B
+    g = _make(B, 2, (1,))
+    g.step(*_batch(1))
+    assert _status(g, g.sync) == B.FDG_OK
+    assert g.lib.fdg_debug_wait_probe(g.ctx, None, 0) == 1            # limits outside 1..2^20 are refused
+    assert g.lib.fdg_debug_wait_probe(g.ctx, None, (1 << 20) + 1) == 1
+    assert _status(g, g.sync) == B.FDG_OK
+    assert g.lib.fdg_debug_wait_probe(g.ctx, torch.cuda.current_stream().cuda_stream, 4096) == B.FDG_OK
+    assert _status(g, g.sync) == 7                                   # FDG_ERR_TIMEOUT
+    assert "waiting" in g.lib.fdg_last_error(g.ctx).decode()
+    assert _status(g, g.step, *_batch(2)) == 7                       # latched
+    g.close()
+    torch.cuda.synchronize()                                         # no CUDA error was left behind
+    g2 = _make(B, 2, (1,))
+    loss = torch.zeros(1, device="cuda")
+    g2.step(*_batch(1))
+    g2.step(*_batch(2), loss)
+    assert _status(g2, g2.sync) == B.FDG_OK and np.isfinite(loss.item())
+    g2.close()
