@@ -70,12 +70,13 @@ fdg_status fdg_conv_forward(int precision, const fdg_conv_shape* shape, const vo
 
 /* dx = conv^T(dy, w) [+ res * [res_mask > 0]], dx/res/res_mask [N][H][W][Ci], dy [N][P][Q][Co].
  * `w_flipped` (nullable) is the copy made by fdg_conv_flip_weights; with it, bf16 3x3 shapes run on the
- * tensor cores (stride 2: also needs extra->dy_spread), without it every shape runs on the CUDA cores. */
+ * tensor cores (stride 2: also needs extra->dy_spread) and so do 1x1 shapes without padding (stride 2 without
+ * res: dx is cleared, then written at its even pixels); without it every shape runs on the CUDA cores. */
 fdg_status fdg_conv_dgrad(int precision, const fdg_conv_shape* shape, const void* dy, const void* w,
                           const void* w_flipped, void* dx, const void* res, const void* res_mask,
                           fdg_conv_extra* extra, int* status_dev, fdg_stream stream);
 
-/* w_flipped[ci][2-r][2-s][co] = w[co][r][s][ci] (bf16, R = 3): the operand layout of the
+/* w_flipped[ci][R-1-r][R-1-s][co] = w[co][r][s][ci] (bf16, R = 3 or 1): the operand layout of the
  * tensor-core data-gradient kernel. */
 fdg_status fdg_conv_flip_weights(const fdg_conv_shape* shape, const void* w_bf16, void* w_flipped_bf16,
                                  fdg_stream stream);

@@ -476,7 +476,7 @@ class ConvOps:
         return (y, keep[-1][:ex.nparts]) if reduce else y
 
     def flip_weights(self, s, w):
-        out = self.torch.empty(s.Ci * 9 * s.Co, dtype=self.torch.bfloat16, device="cuda")
+        out = self.torch.empty(s.Ci * s.R * s.R * s.Co, dtype=self.torch.bfloat16, device="cuda")
         self._chk(self.lib.fdg_conv_flip_weights(C.byref(s), _ptr(w), _ptr(out), self._stream()))
         return out
 

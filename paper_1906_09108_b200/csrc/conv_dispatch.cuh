@@ -9,6 +9,7 @@
 #include "conv_simt.cuh"
 #include "conv_tc.cuh"
 #include "conv_halo.cuh"
+#include "wgrad_wide.cuh"
 #include "elementwise.cuh"
 
 namespace fdg {
@@ -39,18 +40,19 @@ inline bool tc_eligible(const ConvGeom& g) {
 // counts (forward: Ci/Co; data gradient: Co/Ci with the flipped weight copy).
 inline cudaError_t run_conv_tc(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ck, int Cn,
                                const bf16_t* act, const bf16_t* wgt, bf16_t* out, const bf16_t* res,
-                               const bf16_t* res_mask, int* err_dev, int sub = 1) {
+                               const bf16_t* res_mask, int* err_dev, int sub = 1, int taps = 9, int act_sub = 1) {
   if (cache->sm_count == 0) {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&cache->sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
-  tc::ConvTcParams p = tc::conv_tc_params(N, H, W, Ck, Cn);
+  tc::ConvTcParams p = tc::conv_tc_params(N, H, W, Ck, Cn, taps);
   p.sub = sub;
+  p.act_sub = act_sub;
   TensorMapCache::Key ka, kb;
   std::memset(&ka, 0, sizeof(ka)); std::memset(&kb, 0, sizeof(kb));
-  ka.ptr = act; ka.d[0] = 1; ka.d[1] = N; ka.d[2] = H; ka.d[3] = W; ka.d[4] = Ck; ka.d[5] = p.kc; ka.d[6] = p.patch;
-  kb.ptr = wgt; kb.d[0] = 2; kb.d[1] = Ck; kb.d[2] = Cn; kb.d[3] = p.kc; kb.d[4] = p.n_tile;
+  ka.ptr = act; ka.d[0] = 1; ka.d[1] = N; ka.d[2] = H; ka.d[3] = W; ka.d[4] = Ck; ka.d[5] = p.kc; ka.d[6] = p.patch; ka.d[7] = act_sub;
+  kb.ptr = wgt; kb.d[0] = 2; kb.d[1] = Ck; kb.d[2] = Cn; kb.d[3] = p.kc; kb.d[4] = p.n_tile; kb.d[5] = taps;
   auto ia = cache->maps.find(ka), ib = cache->maps.find(kb);
   if (ia == cache->maps.end() || ib == cache->maps.end()) {
     CUtensorMap ma, mb;
@@ -94,6 +96,19 @@ inline bool halo_s2_dgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) 
 inline bool tc_s2_fprop_eligible(const ConvGeom& g) { return halo_s2_shape(g) && tc::conv_tc_supported(g.N, g.H, g.W, g.Ci, g.Co); }
 inline bool tc_s2_dgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && tc::conv_tc_supported(g.N, g.H, g.W, g.Co, g.Ci); }
 inline bool halo_s2_wgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && halo::wgrad_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+// 1x1 convolutions without padding (projection shortcuts), stride 1 or 2: one "tap" of the per-tap kernel on the output
+// grid; a stride-2 forward reads the even pixels of x as a strided tensor, a stride-2 data gradient writes dx at the
+// even pixels (dx is cleared first).
+inline bool tc_1x1_shape(const ConvGeom& g) {
+  return g.R == 1 && g.S == 1 && g.pad == 0 && (g.stride == 1 || (g.stride == 2 && g.H % 2 == 0 && g.W % 2 == 0)) &&
+         g.P == g.H / g.stride && g.Q == g.W / g.stride;
+}
+inline bool tc_1x1_fprop_eligible(const ConvGeom& g) { return tc_1x1_shape(g) && tc::conv_tc_supported(g.N, g.P, g.Q, g.Ci, g.Co); }
+inline bool tc_1x1_dgrad_eligible(const ConvGeom& g) { return tc_1x1_shape(g) && tc::conv_tc_supported(g.N, g.P, g.Q, g.Co, g.Ci); }
+// wide layers: the exact-tile weight-gradient kernel (stride 2 with dy spread onto the input grid; 1x1 filters on the output grid)
+inline bool wide_wgrad_eligible(const ConvGeom& g) { return halo_shape(g) && wide::wide_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+inline bool wide_s2_wgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && wide::wide_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+inline bool wide_1x1_wgrad_eligible(const ConvGeom& g) { return tc_1x1_shape(g) && wide::wide_supported(g.N, g.P, g.Q, g.Ci, g.Co, 1); }
 
 inline cudaError_t cached_tile_map(TensorMapCache* cache, const void* act, int N, int H, int W, int C, int G,
                                    const CUtensorMap** out, int boxC = 0) {
@@ -172,14 +187,49 @@ inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N,
   return cudaGetLastError();
 }
 
+// The same contract for wide layers and 1x1 filters (wide::wgrad_wide_kernel; scratch of wide::wide_scratch_elems
+// floats).  R = 1: H, W are the output grid and `x_sub` the stride (2: x is [N][2H][2W][Ci], read at its even pixels).
+inline cudaError_t cached_slab_map(TensorMapCache* cache, const void* act, int N, int H, int W, int C, int box_w, int box_h,
+                                   const CUtensorMap** out, int sub = 1) {
+  TensorMapCache::Key k;
+  std::memset(&k, 0, sizeof(k));
+  k.ptr = act; k.d[0] = 5; k.d[1] = N; k.d[2] = H; k.d[3] = W; k.d[4] = C; k.d[5] = box_w; k.d[6] = box_h; k.d[7] = sub;
+  auto it = cache->maps.find(k);
+  if (it == cache->maps.end()) {
+    CUtensorMap m;
+    cudaError_t e = wide::make_slab_map(act, N, H, W, C, box_w, box_h, &m, sub);
+    if (e != cudaSuccess) return e;
+    it = cache->maps.insert({k, m}).first;
+  }
+  *out = &it->second;
+  return cudaSuccess;
+}
+inline cudaError_t run_wgrad_wide(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ci, int Co,
+                                  const bf16_t* x, const bf16_t* dy, float* dw, float* scratch, int* err_dev, int R = 3,
+                                  int x_sub = 1) {
+  const wide::WideParams p = wide::wide_params(N, H, W, Ci, Co, cached_sm_count(cache), R);
+  const CUtensorMap *mx, *my;
+  cudaError_t e = cached_slab_map(cache, x, N, H, W, Ci, p.xw, p.S, &mx, x_sub);
+  if (e == cudaSuccess) e = cached_slab_map(cache, dy, N, H, W, Co, p.W, p.S, &my);
+  if (e == cudaSuccess) e = wide::wide_set_attrs();
+  if (e != cudaSuccess) return e;
+  wide::wgrad_wide_kernel<<<dim3(p.co_blocks * p.ci_chunks * p.rdim, p.splits), wide::kWideThreads, wide::wide_smem_bytes(p), st>>>(
+      *mx, *my, p, scratch, err_dev);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const size_t n4 = (size_t)Co * R * R * Ci / 4;                 // Ci is a multiple of 16
+  wide::wgrad_wide_sum_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const float4*>(scratch),
+                                                                          reinterpret_cast<float4*>(dw), n4, p.splits);
+  return cudaGetLastError();
+}
 
 // Does the data gradient of this convolution read the flipped/transposed weight copy?
 inline bool dgrad_uses_flipped(const ConvGeom& g) {
-  return halo_dgrad_eligible(g) || halo_s2_dgrad_eligible(g) || tc_eligible(g) || tc_s2_dgrad_eligible(g);
+  return halo_dgrad_eligible(g) || halo_s2_dgrad_eligible(g) || tc_eligible(g) || tc_s2_dgrad_eligible(g) || tc_1x1_dgrad_eligible(g);
 }
 // Do the stride-2 gradients of this convolution run on the tensor cores, given a spread-out copy of dy?
 inline bool s2_uses_spread_dy(const ConvGeom& g) {
-  return (halo_s2_dgrad_eligible(g) || halo_s2_wgrad_eligible(g) || tc_s2_dgrad_eligible(g)) && g.Co % 8 == 0;
+  return (halo_s2_dgrad_eligible(g) || halo_s2_wgrad_eligible(g) || tc_s2_dgrad_eligible(g) || wide_s2_wgrad_eligible(g)) && g.Co % 8 == 0;
 }
 
 // fp32 scratch elements a weight-gradient call may need (bf16 storage: whichever kernel is chosen).
@@ -187,6 +237,10 @@ inline size_t conv_wgrad_scratch_elems(bool bf16_storage, const ConvGeom& g) {
   size_t n = wgrad_scratch_elems(g);
   if (bf16_storage && (halo_wgrad_eligible(g) || halo_s2_wgrad_eligible(g)))
     n = std::max(n, halo::wgrad_scratch_elems(g.N, g.H, g.W, g.Ci, g.Co));
+  if (bf16_storage && (wide_wgrad_eligible(g) || wide_s2_wgrad_eligible(g)))
+    n = std::max(n, wide::wide_scratch_elems(g.N, g.H, g.W, g.Ci, g.Co));
+  if (bf16_storage && wide_1x1_wgrad_eligible(g))
+    n = std::max(n, wide::wide_scratch_elems(g.N, g.P, g.Q, g.Ci, g.Co, 1));
   return n;
 }
 
@@ -220,6 +274,10 @@ inline cudaError_t bf16_conv_fprop(cudaStream_t st, TensorMapCache* cache, const
     ++*launches;
     return run_conv_tc(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, err_dev, g.stride);
   }
+  if (tc_1x1_fprop_eligible(g)) {
+    ++*launches;
+    return run_conv_tc(st, cache, g.N, g.P, g.Q, g.Ci, g.Co, x, w, y, res, nullptr, err_dev, 1, 1, g.stride);
+  }
   return launch_conv_simt<bf16_t, CONV_FPROP>(st, g, x, w, y, nullptr, nullptr, res, (const bf16_t*)nullptr, launches);
 }
 
@@ -248,6 +306,15 @@ inline cudaError_t bf16_conv_dgrad(cudaStream_t st, TensorMapCache* cache, const
     ++*launches;
     return run_conv_tc(st, cache, g.N, g.H, g.W, g.Co, g.Ci, dy_up, wflip, dx, res, mask, err_dev);
   }
+  if (wflip && tc_1x1_dgrad_eligible(g) && (g.stride == 1 || (!res && !mask))) {
+    // stride 2: only the even pixels of dx receive a gradient; the rest of dx is cleared first
+    if (g.stride == 2) {
+      const cudaError_t e = cudaMemsetAsync(dx, 0, (size_t)g.N * g.H * g.W * g.Ci * sizeof(bf16_t), st);
+      if (e != cudaSuccess) return e;
+    }
+    ++*launches;
+    return run_conv_tc(st, cache, g.N, g.P, g.Q, g.Co, g.Ci, dy, wflip, dx, res, mask, err_dev, g.stride == 2 ? 3 : 1, 1, 1);
+  }
   return launch_conv_simt<bf16_t, CONV_DGRAD>(st, g, dy, w, dx, nullptr, nullptr, res, mask, launches);
 }
 
@@ -256,6 +323,14 @@ inline cudaError_t bf16_conv_dgrad(cudaStream_t st, TensorMapCache* cache, const
 inline cudaError_t bf16_conv_wgrad(cudaStream_t st, TensorMapCache* cache, const ConvGeom& g, const bf16_t* x,
                                    const bf16_t* dy, const bf16_t* dy_up, float* dw, float* scratch, int* err_dev,
                                    bool side, uint64_t* launches) {
+  if ((dy_up && wide_s2_wgrad_eligible(g)) || wide_wgrad_eligible(g)) {
+    *launches += 2;
+    return run_wgrad_wide(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, wide_wgrad_eligible(g) ? dy : dy_up, dw, scratch, err_dev);
+  }
+  if (wide_1x1_wgrad_eligible(g)) {
+    *launches += 2;
+    return run_wgrad_wide(st, cache, g.N, g.P, g.Q, g.Ci, g.Co, x, dy, dw, scratch, err_dev, 1, g.stride);
+  }
   if (dy_up && halo_s2_wgrad_eligible(g)) {
     *launches += 2;
     return run_wgrad_halo(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, dy_up, dw, scratch, err_dev, side);

@@ -46,7 +46,11 @@ struct ConvTcParams {
   int mpair;                // 128-row tiles a CTA works on at once with one weight tile: 1 (two accumulator sets, the
                             // epilogue of a tile overlaps the next tile's instructions) or 2 (one set of two accumulators:
                             // every weight tile fetched from L2 serves 256 rows)
-  int sub;                  // 1, or 2: store only the pixels with even h and w, as an [N][H/2][W/2][Co] tensor
+  int sub;                  // 1, or 2: store only the pixels with even h and w, as an [N][H/2][W/2][Co] tensor,
+                            // or 3: store pixel (h, w) at (2h, 2w) of an [N][2H][2W][Co] tensor (the data gradient of a
+                            // stride-2 1x1 convolution; the other pixels of that tensor are not touched)
+  int taps;                 // 9 (3x3, pad 1) or 1 (1x1, pad 0)
+  int act_sub;              // 1, or 2: the activation operand is the even pixels of an [N][2H][2W][Ci] tensor
   int patch;                // 1: conv3x3_patch_kernel (16x16-pixel patches with their halo), 0: conv3x3_tc_kernel
   uint32_t halo_bytes;      // patch mode: shared memory of one 18x18-pixel halo tile of kc channels (multiple of 1 KiB)
   int b_stages;             // patch mode: weight tiles in flight
@@ -202,7 +206,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   const uint32_t tmem_base = *tmem_slot;
 
   const int chunks = (p.Ci + p.kc - 1) / p.kc;
-  const int k_iters = 9 * chunks;
+  const int k_iters = p.taps * chunks;
   const int total_tiles = ((p.m_tiles + p.mpair - 1) / p.mpair) * p.n_tiles;     // tiles of mpair * 128 rows
 
   if (warp == 0) {
@@ -227,11 +231,12 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag)) break;
           const int tap = ki / chunks, cc = ki - tap * chunks;
           const int r = tap / 3, sx = tap - r * 3;
+          const int dw = p.taps == 1 ? 0 : sx - 1, dh = p.taps == 1 ? 0 : r - 1;
           uint8_t* a_dst = smem + (size_t)s * p.stage_bytes;
           uint8_t* b_dst = a_dst + (size_t)p.mpair * p.a_bytes;
           mbar_expect_tx(&full[s], (uint32_t)halves * p.a_bytes + p.b_tx_bytes);
           for (int hf = 0; hf < halves; ++hf)
-            tma_load_4d(a_dst + (size_t)hf * p.a_bytes, &map_a, &full[s], cc * p.kc, sx - 1, h0[hf] + r - 1, n0[hf]);
+            tma_load_4d(a_dst + (size_t)hf * p.a_bytes, &map_a, &full[s], cc * p.kc, dw, h0[hf] + dh, n0[hf]);
           tma_load_2d(b_dst, &map_b, &full[s], tap * p.Ci + cc * p.kc, nt * p.n_tile);
         }
       }
@@ -300,6 +305,10 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int h = (int)(rem / p.W), w = (int)(rem - (size_t)h * p.W);
         keep = ((h | w) & 1) == 0;
         base = (((n * (p.H >> 1) + (h >> 1)) * (p.W >> 1)) + (w >> 1)) * p.Co + (size_t)nt * p.n_tile;
+      } else if (p.sub == 3) {
+        const size_t hw = (size_t)p.H * p.W, n = row / hw, rem = row - n * hw;
+        const int h = (int)(rem / p.W), w = (int)(rem - (size_t)h * p.W);
+        base = (((n * (2 * p.H) + 2 * h) * (2 * p.W)) + 2 * w) * p.Co + (size_t)nt * p.n_tile;
       }
       const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(acc + hf) * p.n_tile;
       for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
@@ -623,9 +632,9 @@ inline bool conv_tc_supported(int N, int H, int W, int Ci, int Co) {
   return true;
 }
 
-inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co) {
+inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co, int taps = 9) {
   ConvTcParams p{};
-  p.W = W; p.H = H; p.N = N; p.Ci = Ci; p.Co = Co; p.sub = 1;
+  p.W = W; p.H = H; p.N = N; p.Ci = Ci; p.Co = Co; p.sub = 1; p.taps = taps; p.act_sub = 1;
   const int rows = kTileM / W;
   if (rows <= H) { p.rows_per_tile = rows; p.imgs_per_tile = 1; }
   else { p.rows_per_tile = H; p.imgs_per_tile = rows / H; }
@@ -647,7 +656,7 @@ inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co) {
   p.mpair = p.m_tiles >= 2 ? 2 : 1;
   p.stage_bytes = (uint32_t)p.mpair * p.a_bytes + p.b_bytes;
   // 16x16-pixel patches with their halo wherever the image allows it and the chunks are full swizzle spans
-  p.patch = (H % kPatch == 0 && W % kPatch == 0 && p.kc == 64) ? 1 : 0;
+  p.patch = (taps == 9 && H % kPatch == 0 && W % kPatch == 0 && p.kc == 64) ? 1 : 0;
   p.halo_bytes = ((uint32_t)kPatchHalo * kPatchHalo * p.kc * 2 + 1023u) & ~1023u;
   p.b_stages = (int)((176 * 1024 - 2 * (size_t)p.halo_bytes) / p.b_bytes);
   if (p.b_stages > 6) p.b_stages = 6;
@@ -672,8 +681,11 @@ inline cudaError_t conv_tc_make_maps(const ConvTcParams& p, const void* act, con
   if (!enc) return cudaErrorNotSupported;
   const CUtensorMapSwizzle sw = swizzle_for(p.kc * 2);
   {
+    // act_sub = 2: the even pixels of an [N][2H][2W][Ci] tensor are themselves a regular [N][H][W][Ci] tensor
+    // with doubled pixel strides and quadrupled row and image strides
+    const cuuint64_t q = (cuuint64_t)p.act_sub;
     cuuint64_t dims[4] = {(cuuint64_t)p.Ci, (cuuint64_t)p.W, (cuuint64_t)p.H, (cuuint64_t)p.N};
-    cuuint64_t strides[3] = {(cuuint64_t)p.Ci * 2, (cuuint64_t)p.W * p.Ci * 2, (cuuint64_t)p.H * p.W * p.Ci * 2};
+    cuuint64_t strides[3] = {q * p.Ci * 2, q * q * p.W * p.Ci * 2, q * q * p.H * p.W * p.Ci * 2};
     cuuint32_t box[4] = {(cuuint32_t)p.kc, (cuuint32_t)p.W, (cuuint32_t)p.rows_per_tile, (cuuint32_t)p.imgs_per_tile};
     if (p.patch) { box[1] = kPatchHalo; box[2] = kPatchHalo; box[3] = 1; }
     cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -683,8 +695,8 @@ inline cudaError_t conv_tc_make_maps(const ConvTcParams& p, const void* act, con
       return cudaErrorInvalidValue;
   }
   {
-    cuuint64_t dims[2] = {(cuuint64_t)9 * p.Ci, (cuuint64_t)p.Co};
-    cuuint64_t strides[1] = {(cuuint64_t)9 * p.Ci * 2};
+    cuuint64_t dims[2] = {(cuuint64_t)p.taps * p.Ci, (cuuint64_t)p.Co};
+    cuuint64_t strides[1] = {(cuuint64_t)p.taps * p.Ci * 2};
     cuuint32_t box[2] = {(cuuint32_t)p.kc, (cuuint32_t)p.n_tile};
     cuuint32_t estr[2] = {1, 1};
     if (enc(map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(wgt), dims, strides, box, estr,
@@ -726,17 +738,18 @@ inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const 
   return cudaGetLastError();
 }
 
-// Flipped / transposed weight copy for the data gradient of a stride-1 3x3 convolution:
-// dst[ci][2-r][2-s][co] = src[co][r][s][ci].  One block row per entry of `table`
-// (src offset, dst offset, Co, Ci), all offsets in elements from the two base pointers.
-struct FlipEntry { unsigned long long src, dst; int Co, Ci; };
+// Flipped / transposed weight copy for the data gradient of a 3x3 convolution (taps = 9):
+// dst[ci][2-r][2-s][co] = src[co][r][s][ci]; taps = 1: the transpose of a 1x1 filter.  One block row per entry of
+// `table` (src offset, dst offset, Co, Ci, taps), all offsets in elements from the two base pointers.
+struct FlipEntry { unsigned long long src, dst; int Co, Ci, taps; };
 __global__ void wflip_kernel(const __nv_bfloat16* __restrict__ src_base, __nv_bfloat16* __restrict__ dst_base,
                              const FlipEntry* __restrict__ table) {
   const FlipEntry e = table[blockIdx.y];
-  const int n = e.Co * 9 * e.Ci;
+  const int T = e.taps;
+  const int n = e.Co * T * e.Ci;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-    const int co = i % e.Co, t = (i / e.Co) % 9, ci = i / (9 * e.Co);       // i indexes dst[ci][t][co]
-    dst_base[e.dst + i] = src_base[e.src + ((size_t)co * 9 + (8 - t)) * e.Ci + ci];
+    const int co = i % e.Co, t = (i / e.Co) % T, ci = i / (T * e.Co);         // i indexes dst[ci][t][co]
+    dst_base[e.dst + i] = src_base[e.src + ((size_t)co * T + (T - 1 - t)) * e.Ci + ci];
   }
 }
 

@@ -64,8 +64,9 @@ struct Unit {
   size_t t_a, t_b, t_c, t_y, t_s;
   // offsets (floats) of saved statistics inside the slot's fp32 region
   size_t st1, st2, sts;
-  // offsets of the flipped copies of w1 / w2 inside a wflip16 slot, or -1 when that conv's dgrad is not on tensor cores
-  long long f1 = -1, f2 = -1;
+  // offsets of the flipped copies of w1 / w2 (and of the transposed 1x1 shortcut filter) inside a wflip16 slot, or -1
+  // when that conv's dgrad is not on tensor cores
+  long long f1 = -1, f2 = -1, fs = -1;
   // offsets of the running statistics (mean[C], var[C]) of BN1 / BN2 / the shortcut BN in the module's vector, or -1
   long long r1 = -1, r2 = -1, rs = -1;
 };
@@ -397,11 +398,11 @@ static void plan_modules(fdg_ctx* c) {
       }
     if (c->bf16_mode) {
       size_t fe = 0;
-      auto flip = [&](size_t src, int co, int ci) {
-        tc::FlipEntry e; e.src = src; e.dst = fe; e.Co = co; e.Ci = ci;
+      auto flip = [&](size_t src, int co, int ci, int taps = 9) {
+        tc::FlipEntry e; e.src = src; e.dst = fe; e.Co = co; e.Ci = ci; e.taps = taps;
         m.flip_table.push_back(e);
         long long off = (long long)fe;
-        fe += align_up((size_t)co * 9 * ci, 64);
+        fe += align_up((size_t)co * taps * ci, 64);
         return off;
       };
       for (Unit& u : m.units) {
@@ -410,10 +411,14 @@ static void plan_modules(fdg_ctx* c) {
         ConvGeom g2{a.batch, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 3, 1, 1};
         if (dgrad_uses_flipped(g1)) u.f1 = flip(u.w1, u.co, u.ci);
         if (dgrad_uses_flipped(g2)) u.f2 = flip(u.w2, u.co, u.co);
+        if (u.proj) {
+          ConvGeom gs{a.batch, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, 1, u.stride, 0};
+          if (dgrad_uses_flipped(gs)) u.fs = flip(u.ws, u.co, u.ci, 1);
+        }
       }
       m.flip_elems = fe;
       size_t largest = 0;
-      for (const tc::FlipEntry& fe_ : m.flip_table) largest = std::max(largest, (size_t)fe_.Co * 9 * fe_.Ci);
+      for (const tc::FlipEntry& fe_ : m.flip_table) largest = std::max(largest, (size_t)fe_.Co * fe_.taps * fe_.Ci);
       m.flip_blocks = (unsigned)std::min<size_t>(std::max<size_t>(largest / 8192, 8), 128);
     }
     m.slot_elems = te; m.slot_floats = tf; m.max_act = maxa; m.scratch_floats = scr; m.wscratch_floats = wscr;
@@ -925,7 +930,7 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
           conv_wgrad<T>(LS, m, gs, x, T2, m.grad + u.ws);                                                // side
           side_done(2);
           if (need_dx) {
-            conv_dgrad<T>(L, m, gs, T2, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
+            conv_dgrad<T>(L, m, gs, T2, wt + u.ws, flipped_of<T>(m, vslot, u.fs), T3, nullptr, nullptr);
             out_sum_parts = conv_dgrad<T>(L, m, g1, T4, wt + u.w1, flipped_of<T>(m, vslot, u.f1), gout, T3, nullptr, next, up);
           }
         } else if (need_dx && u.zpad) {
@@ -955,7 +960,7 @@ static void backward_module(fdg_ctx* c, Module& m, Launch& L, Launch& LS, bool f
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_wgrad<T>(L, m, gs, S + u.t_a, dy, m.grad + u.ws);
-          conv_dgrad<T>(L, m, gs, dy, wt + u.ws, (const T*)nullptr, T3, nullptr, nullptr);
+          conv_dgrad<T>(L, m, gs, dy, wt + u.ws, flipped_of<T>(m, vslot, u.fs), T3, nullptr, nullptr);
           keep(i, 5, T3);
           conv_dgrad<T>(L, m, g1, T2, wt + u.w1, flipped_of<T>(m, vslot, u.f1), T1, T3, nullptr, nullptr, up);   // do
         } else {

@@ -23,7 +23,7 @@ def _rel(a, b):
 
 
 # (N, H, W, Ci, Co, R, stride, pad)
-SHAPES_ANY = [(3, 12, 20, 5, 7, 3, 1, 1), (2, 16, 16, 8, 16, 3, 2, 1), (2, 16, 16, 16, 32, 1, 2, 0),
+SHAPES_ANY = [(3, 12, 20, 5, 7, 3, 1, 1), (2, 16, 16, 8, 16, 3, 2, 1), (2, 16, 16, 16, 24, 1, 2, 0),
               (5, 8, 8, 3, 8, 3, 1, 1)]
 SHAPES_TC = [(4, 32, 32, 16, 16, 3, 1, 1),      # 32 tiles of 4 image rows, 32-byte swizzle
              (6, 16, 16, 32, 32, 3, 1, 1),      # 8 rows per tile, 64-byte swizzle
@@ -41,7 +41,19 @@ SHAPES_TC = [(4, 32, 32, 16, 16, 3, 1, 1),      # 32 tiles of 4 image rows, 32-b
              (2, 16, 16, 320, 320, 3, 1, 1),    # WRN stage 2: five 64-channel chunks, two 160-column N tiles
              (4, 8, 8, 640, 640, 3, 1, 1),      # WRN stage 3: four N tiles, the weight gradient in 10 x 10 channel chunks
              (2, 32, 32, 160, 320, 3, 2, 1),    # the stride-2 layers of WRN-28-10 (per-tap kernel at full resolution)
-             (2, 16, 16, 320, 640, 3, 2, 1)]
+             (2, 16, 16, 320, 640, 3, 2, 1),
+             # the exact-tile weight-gradient kernel of wide layers: several 64-pixel slabs per CTA (the shared-memory
+             # ring wraps), a last block of 32 output channels, two rows of 8 pixels per reduction step
+             (24, 16, 16, 320, 320, 3, 1, 1),
+             (3, 32, 32, 160, 160, 3, 1, 1),
+             (16, 8, 8, 640, 640, 3, 1, 1),
+             (5, 16, 16, 128, 256, 3, 1, 1),
+             # 1x1 projection shortcuts on the per-tap kernel: stride 2 reads the even pixels of x as a strided tensor
+             # and writes dx at the even pixels of a cleared tensor; the weight gradient of wide ones on the exact-tile kernel
+             (4, 32, 32, 160, 320, 1, 2, 0),
+             (8, 16, 16, 320, 640, 1, 2, 0),
+             (2, 32, 32, 16, 160, 1, 1, 0),
+             (6, 16, 16, 32, 64, 1, 2, 0)]
 
 # shapes whose three operators all take the halo-tile tensor-core kernels
 ALL_TC = {(4, 32, 32, 16, 16), (6, 16, 16, 32, 32), (10, 8, 8, 64, 64), (300, 8, 8, 64, 64), (5, 12, 20, 16, 32),
@@ -72,7 +84,7 @@ def _run(prec_name, shape, expect_tc):
     assert _rel(y, L.conv2d_forward(xo, wo, st, pad) + resyo) < tol
 
     dxo, dwo = L.conv2d_backward(dyo, xo, wo, st, pad)
-    wf = ops.flip_weights(s, wt) if (prec_name == "bf16" and r == 3) else None
+    wf = ops.flip_weights(s, wt) if (prec_name == "bf16" and r in (1, 3)) else None
     dx = ops.dgrad(s, dy, wt, wf).float().cpu().numpy()
     assert _rel(dx, dxo) < tol
     dx = ops.dgrad(s, dy, wt, wf, res=res, res_mask=mask).float().cpu().numpy()
