@@ -213,8 +213,9 @@ inline cudaError_t run_wgrad_wide(cudaStream_t st, TensorMapCache* cache, int N,
   if (e == cudaSuccess) e = cached_slab_map(cache, dy, N, H, W, Co, p.W, p.S, &my);
   if (e == cudaSuccess) e = wide::wide_set_attrs();
   if (e != cudaSuccess) return e;
-  wide::wgrad_wide_kernel<<<dim3(p.co_blocks * p.ci_chunks * p.rdim, p.splits), wide::kWideThreads, wide::wide_smem_bytes(p), st>>>(
-      *mx, *my, p, scratch, err_dev);
+  const dim3 grid(p.co_blocks * p.ci_chunks * p.rdim, p.splits);
+  if (R == 3) wide::wgrad_wide_kernel<3><<<grid, wide::kWideThreads, wide::wide_smem_bytes(p), st>>>(*mx, *my, p, scratch, err_dev);
+  else wide::wgrad_wide_kernel<1><<<grid, wide::kWideThreads, wide::wide_smem_bytes(p), st>>>(*mx, *my, p, scratch, err_dev);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t n4 = (size_t)Co * R * R * Ci / 4;                 // Ci is a multiple of 16

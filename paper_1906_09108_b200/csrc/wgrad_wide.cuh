@@ -66,6 +66,7 @@ __device__ __forceinline__ uint64_t desc_mn128(uint32_t addr, uint32_t lbo, uint
   return d;
 }
 
+template <int TAPS>
 __global__ void __launch_bounds__(kWideThreads, 1)
 wgrad_wide_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, WideParams p,
                   float* __restrict__ partial, int* __restrict__ error_word) {
@@ -119,26 +120,42 @@ wgrad_wide_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     }
   } else if (warp == 1) {
     if (lane == 0) {
+      // The issuing thread is alone in its warp, so every instruction between two tcgen05.mma costs its full
+      // latency: the descriptors of a stage are formed once, a reduction step moves them by additions on the
+      // address field (16-byte units), and the loops over steps and taps are unrolled.
       const uint32_t idesc = halo::instr_desc(p.nci, true);
-      const int ksteps = kSlabPixels / 16;
+      constexpr int ksteps = kSlabPixels / 16;
+      const uint32_t y_first = smem_u32(smem);
+      const uint64_t a_first = desc_mn128(y_first, p.y_sub_bytes, 1024u);
+      const uint64_t b_first = desc_mn128(y_first + p.y_bytes, p.x_sub_bytes, p.sbo_x);
+      const uint64_t stage_units = (uint64_t)(stage_bytes >> 4);
+      uint64_t b_off[ksteps];
+      for (int ks = 0; ks < ksteps; ++ks) {
+        const int pix = ks * 16;                                 // first pixel of the step inside the dY slab
+        const int row = pix / p.W, col = pix - row * p.W;        // W = 8: row is even and the step takes rows row, row+1
+        b_off[ks] = (uint64_t)((row * p.xw + col) * 8);          // one pixel = 128 bytes = 8 units
+      }
+      const uint32_t d1 = tmem_base + (uint32_t)p.nci, d2 = tmem_base + 2u * (uint32_t)p.nci;
       uint32_t it = 0;
+      int s = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int slab = blockIdx.y; slab < p.slabs && !*abort_flag; slab += gridDim.y, ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
         if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t y_addr = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint32_t x_addr = y_addr + p.y_bytes;
+        const uint64_t a0 = a_first + (uint64_t)s * stage_units, b0 = b_first + (uint64_t)s * stage_units;
+#pragma unroll
         for (int ks = 0; ks < ksteps; ++ks) {
-          const int pix = ks * 16;                               // first pixel of the step inside the dY slab
-          const int row = pix / p.W, col = pix - row * p.W;      // W = 8: row is even and the step takes rows row, row+1
-          const uint64_t a_desc = desc_mn128(y_addr + (uint32_t)pix * 128u, p.y_sub_bytes, 1024u);
-          uint64_t b_desc = desc_mn128(x_addr + (uint32_t)(row * p.xw + col) * 128u, p.x_sub_bytes, p.sbo_x);
-          for (int sx = 0; sx < p.taps; ++sx, b_desc += 8)       // one pixel = 128 bytes = 8 units of the address field
-            tc_mma_bf16(tmem_base + (uint32_t)(sx * p.nci), a_desc, b_desc, idesc, (it | (uint32_t)ks) != 0);
+          const uint64_t a = a0 + (uint64_t)(ks * 128), b = b0 + b_off[ks];      // 16 pixels = 2048 bytes = 128 units
+          const uint32_t acc = (it | (uint32_t)ks) != 0;
+          tc_mma_bf16(tmem_base, a, b, idesc, acc);
+          if (TAPS == 3) {
+            tc_mma_bf16(d1, a, b + 8, idesc, acc);
+            tc_mma_bf16(d2, a, b + 16, idesc, acc);
+          }
         }
         tc_commit(&empty[s]);
+        if (++s == p.stages) { s = 0; ph ^= 1; }
       }
       if (ok) tc_commit(done);
     }
@@ -281,7 +298,8 @@ inline cudaError_t make_slab_map(const void* act, int N, int H, int W, int C, in
 inline cudaError_t wide_set_attrs() {
   static bool done = false;
   if (done) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(wgrad_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmemBudget + 8192);
+  cudaError_t e = cudaFuncSetAttribute(wgrad_wide_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmemBudget + 8192);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(wgrad_wide_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWideSmemBudget + 8192);
   if (e == cudaSuccess) done = true;
   return e;
 }
