@@ -106,8 +106,13 @@ inline bool tc_1x1_shape(const ConvGeom& g) {
 inline bool tc_1x1_fprop_eligible(const ConvGeom& g) { return tc_1x1_shape(g) && tc::conv_tc_supported(g.N, g.P, g.Q, g.Ci, g.Co); }
 inline bool tc_1x1_dgrad_eligible(const ConvGeom& g) { return tc_1x1_shape(g) && tc::conv_tc_supported(g.N, g.P, g.Q, g.Co, g.Ci); }
 // wide layers: the exact-tile weight-gradient kernel (stride 2 with dy spread onto the input grid; 1x1 filters on the output grid)
-inline bool wide_wgrad_eligible(const ConvGeom& g) { return halo_shape(g) && wide::wide_supported(g.N, g.H, g.W, g.Ci, g.Co); }
-inline bool wide_s2_wgrad_eligible(const ConvGeom& g) { return halo_s2_shape(g) && wide::wide_supported(g.N, g.H, g.W, g.Ci, g.Co); }
+// (layers under 128 channels stay with the halo-tile kernel where it covers them)
+inline bool wide_wgrad_eligible(const ConvGeom& g) {
+  return halo_shape(g) && wide::wide_supported(g.N, g.H, g.W, g.Ci, g.Co) && ((g.Ci >= 128 && g.Co >= 128) || !halo_wgrad_eligible(g));
+}
+inline bool wide_s2_wgrad_eligible(const ConvGeom& g) {
+  return halo_s2_shape(g) && wide::wide_supported(g.N, g.H, g.W, g.Ci, g.Co) && ((g.Ci >= 128 && g.Co >= 128) || !halo_s2_wgrad_eligible(g));
+}
 inline bool wide_1x1_wgrad_eligible(const ConvGeom& g) { return tc_1x1_shape(g) && wide::wide_supported(g.N, g.P, g.Q, g.Ci, g.Co, 1); }
 
 inline cudaError_t cached_tile_map(TensorMapCache* cache, const void* act, int N, int H, int W, int C, int G,
@@ -183,7 +188,11 @@ inline cudaError_t run_wgrad_halo(cudaStream_t st, TensorMapCache* cache, int N,
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t n = (size_t)Co * 9 * Ci;
-  halo::wgrad_halo_reduce_kernel<<<(int)((n + 31) / 32), 256, 0, st>>>(scratch, dw, n, ctas);
+  if (n >= ((size_t)1 << 17) && ctas <= 8)        // large filters, few partials: four outputs per thread, partials in turn
+    wide::wgrad_wide_sum_kernel<<<(unsigned)((n / 4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const float4*>(scratch),
+                                                                               reinterpret_cast<float4*>(dw), n / 4, ctas);
+  else
+    halo::wgrad_halo_reduce_kernel<<<(int)((n + 31) / 32), 256, 0, st>>>(scratch, dw, n, ctas);
   return cudaGetLastError();
 }
 

@@ -645,18 +645,24 @@ inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co, int taps
   p.kc = (Ci % 64 == 0 || Ci >= 128) ? 64 : (Ci % 32 == 0 ? 32 : 16);
   int nt = Co;
   if (nt > 256) { nt = 256; while (Co % nt || nt % 16) nt -= 16; }
-  p.n_tile = nt;
   p.m_tiles = (int)((size_t)N * H * W / kTileM);
+  // 16x16-pixel patches with their halo wherever the image allows it and the chunks are full swizzle spans
+  p.patch = (taps == 9 && H % kPatch == 0 && W % kPatch == 0 && p.kc == 64) ? 1 : 0;
+  // The kernel is bound by the rate at which operand tiles arrive from L2, so a weight tile is shared by two
+  // 128-row tiles -- unless the layer has so few pixels (small images, many channels) that the tiles would leave
+  // most SMs idle: then single 128-row tiles and narrower column tiles, down to 64, until there are about 96.
+  p.mpair = p.m_tiles >= 2 ? 2 : 1;
+  if (!p.patch) {
+    auto tiles = [&]() { return ((p.m_tiles + p.mpair - 1) / p.mpair) * (Co / nt); };
+    if (tiles() < 96) p.mpair = 1;
+    while (tiles() < 96 && nt % 32 == 0 && nt / 2 >= 64 && Co % (nt / 2) == 0) nt /= 2;
+  }
+  p.n_tile = nt;
   p.n_tiles = Co / nt;
   p.a_bytes = (uint32_t)kTileM * p.kc * 2;
   p.b_tx_bytes = (uint32_t)nt * p.kc * 2;
   p.b_bytes = (p.b_tx_bytes + 1023u) & ~1023u;
-  // The kernel is bound by the rate at which operand tiles arrive from L2, so a weight tile is shared by two
-  // 128-row tiles.
-  p.mpair = p.m_tiles >= 2 ? 2 : 1;
   p.stage_bytes = (uint32_t)p.mpair * p.a_bytes + p.b_bytes;
-  // 16x16-pixel patches with their halo wherever the image allows it and the chunks are full swizzle spans
-  p.patch = (taps == 9 && H % kPatch == 0 && W % kPatch == 0 && p.kc == 64) ? 1 : 0;
   p.halo_bytes = ((uint32_t)kPatchHalo * kPatchHalo * p.kc * 2 + 1023u) & ~1023u;
   p.b_stages = (int)((176 * 1024 - 2 * (size_t)p.halo_bytes) / p.b_bytes);
   if (p.b_stages > 6) p.b_stages = 6;

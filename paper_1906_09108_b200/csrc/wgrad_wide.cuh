@@ -262,12 +262,11 @@ inline WideParams wide_params(int N, int H, int W, int Ci, int Co, int sm_count,
 inline size_t wide_smem_bytes(const WideParams& p) {
   return (size_t)p.stages * ((size_t)p.y_bytes + p.x_bytes) + (size_t)(2 * p.stages + 1) * 8 + 16 + 1024;
 }
-// Wide 3x3 layers only: narrower ones are bound by memory traffic, where the halo-tile kernel's single pass wins.
-// 1x1 filters (projection shortcuts) of 64 channels and more take the same kernel: on the CUDA cores they cost
-// more than the 3x3 layers beside them.
+// 64 channels and more on both sides (a 64-channel sub-tile is one swizzle span).  Narrow 3x3 layers that the
+// halo-tile kernel covers are left to it by the dispatcher: they are bound by memory traffic, where its single
+// pass over whole images wins.
 inline bool wide_supported(int N, int H, int W, int Ci, int Co, int R = 3) {
-  const int least = R == 3 ? 128 : 64;
-  if (Ci < least || Co < least || Ci % 16 || Co % 16 || N < 1 || H < 1) return false;
+  if (Ci < 64 || Co < 64 || Ci % 16 || Co % 16 || N < 1 || H < 1) return false;
   WideParams p = wide_params(N, H, W, Ci, Co, 148, R);
   return p.stages >= 2 && p.tmem_cols <= 512 && p.co_blocks * p.ci_chunks * p.rdim <= 65535;
 }

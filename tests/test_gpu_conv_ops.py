@@ -53,7 +53,13 @@ SHAPES_TC = [(4, 32, 32, 16, 16, 3, 1, 1),      # 32 tiles of 4 image rows, 32-b
              (4, 32, 32, 160, 320, 1, 2, 0),
              (8, 16, 16, 320, 640, 1, 2, 0),
              (2, 32, 32, 16, 160, 1, 1, 0),
-             (6, 16, 16, 32, 64, 1, 2, 0)]
+             (6, 16, 16, 32, 64, 1, 2, 0),
+             # CIFAR ResNet-18 shapes: 64 channels on 32x32 images (too large for a halo tile: exact-tile weight gradient
+             # with one 64-channel sub-tile), and few-pixel layers whose forward tiles are narrowed to fill the SMs
+             (8, 32, 32, 64, 64, 3, 1, 1),
+             (8, 32, 32, 64, 128, 3, 2, 1),
+             (16, 4, 4, 512, 512, 3, 1, 1),
+             (32, 8, 8, 256, 256, 3, 1, 1)]
 
 # shapes whose three operators all take the halo-tile tensor-core kernels
 ALL_TC = {(4, 32, 32, 16, 16), (6, 16, 16, 32, 32), (10, 8, 8, 64, 64), (300, 8, 8, 64, 64), (5, 12, 20, 16, 32),
