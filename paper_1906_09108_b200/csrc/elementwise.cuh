@@ -615,6 +615,7 @@ __global__ void head_fwd_bwd_kernel(const T* __restrict__ x, const float* __rest
   const T* xn = x + (size_t)n * HW * F;
   for (int f = tid; f < F; f += nt) {
     float a = 0.f;
+#pragma unroll 8
     for (int p = 0; p < HW; ++p) a += to_f(xn[(size_t)p * F + f]);
     a /= (float)HW;
     s_pool[f] = a;
@@ -633,13 +634,19 @@ __global__ void head_fwd_bwd_kernel(const T* __restrict__ x, const float* __rest
   __shared__ float s_max, s_sum;
   int label = labels[n];
   if (label < 0 || label >= classes) { if (tid == 0) atomicExch(bad_label, 1); label = 0; }
-  if (tid == 0) {
-    float m = s_logit[0];
-    for (int c = 1; c < classes; ++c) m = fmaxf(m, s_logit[c]);
+  if (warp == 0) {                       // the lanes share the classes; the partial sums meet in a fixed butterfly
+    float m = -INFINITY;
+    for (int c = lane; c < classes; c += 32) m = fmaxf(m, s_logit[c]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     float s = 0.f;
-    for (int c = 0; c < classes; ++c) s += expf(s_logit[c] - m);
-    s_max = m; s_sum = s;
-    loss_n[n] = -(s_logit[label] - m - logf(s));
+    for (int c = lane; c < classes; c += 32) s += expf(s_logit[c] - m);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) {
+      s_max = m; s_sum = s;
+      loss_n[n] = -(s_logit[label] - m - logf(s));
+    }
   }
   __syncthreads();
   for (int c = tid; c < classes; c += nt) {
@@ -651,6 +658,7 @@ __global__ void head_fwd_bwd_kernel(const T* __restrict__ x, const float* __rest
   __syncthreads();
   for (int f = tid; f < F; f += nt) {
     float a = 0.f;
+#pragma unroll 4
     for (int c = 0; c < classes; ++c) a += w[(size_t)c * F + f] * s_logit[c];
     s_dpool[f] = a / (float)HW;
   }
@@ -666,19 +674,27 @@ __global__ void head_param_grad_kernel(const float* __restrict__ pooled, const f
                                        float* __restrict__ dW, float* __restrict__ db, float* __restrict__ loss,
                                        int* __restrict__ nonfinite) {
   const int c = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int f = threadIdx.x; f < F; f += blockDim.x) {
     float a = 0.f;
+#pragma unroll 8
     for (int n = 0; n < batch; ++n) a += dlogits[(size_t)n * classes + c] * pooled[(size_t)n * F + f];
     dW[(size_t)c * F + f] = a;
   }
-  if (threadIdx.x == 0) {
+  // the sums over the batch: lanes take every 32nd sample, the partial sums meet in a fixed butterfly
+  if (warp == 0) {
     float a = 0.f;
-    for (int n = 0; n < batch; ++n) a += dlogits[(size_t)n * classes + c];
-    db[c] = a;
-    if (c == 0) {
-      double l = 0.0;
-      for (int n = 0; n < batch; ++n) l += (double)loss_n[n];
-      float lf = (float)(l / (double)batch);
+    for (int n = lane; n < batch; n += 32) a += dlogits[(size_t)n * classes + c];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) db[c] = a;
+  } else if (warp == 1 && c == 0) {
+    double l = 0.0;
+    for (int n = lane; n < batch; n += 32) l += (double)loss_n[n];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    if (lane == 0) {
+      const float lf = (float)(l / (double)batch);
       *loss = lf;
       if (!isfinite(lf)) atomicExch(nonfinite, 1);
     }
