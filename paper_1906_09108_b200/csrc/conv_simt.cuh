@@ -332,22 +332,27 @@ inline cudaError_t launch_small_wgrad(cudaStream_t st, const ConvGeom& g, const 
 // (512 or 2048 entries on the 6n+2 networks) from tens of thousands of pixels.  Same scheme as above:
 // one image per block, strips staged in shared memory, thread (ci, co) with consecutive co in a warp.
 inline bool proj_wgrad_eligible(const ConvGeom& g) {
-  return g.R == 1 && g.S == 1 && g.pad == 0 && (g.stride == 1 || g.stride == 2) && g.Ci * g.Co <= 2048 && g.Co % 32 == 0 &&
-         (size_t)kSmallWgradRows * g.Q * (g.Ci + g.Co) * 4 <= 48 * 1024;
+  return g.R == 1 && g.S == 1 && g.pad == 0 && (g.stride == 1 || g.stride == 2) && g.Ci * g.Co <= 4096 && g.Co % 32 == 0 &&
+         (size_t)g.Q * (g.Ci + g.Co) * 4 <= 48 * 1024;
+}
+// output rows per strip: what fits 48 KiB of shared memory, at most kSmallWgradRows
+inline int proj_wgrad_strip(const ConvGeom& g) {
+  const int fit = (int)((48 * 1024) / ((size_t)g.Q * (g.Ci + g.Co) * 4));
+  return fit < kSmallWgradRows ? fit : kSmallWgradRows;
 }
 template <typename T>
 __global__ void proj_wgrad_kernel(const T* __restrict__ x, const T* __restrict__ dy, float* __restrict__ partial,
-                                  int H, int W, int P, int Q, int Ci, int Co, int stride) {
+                                  int H, int W, int P, int Q, int Ci, int Co, int stride, int strip) {
   extern __shared__ float pw_smem[];
-  float* xs = pw_smem;                                      // [kSmallWgradRows][Q][Ci]
-  float* ds = pw_smem + kSmallWgradRows * Q * Ci;             // [kSmallWgradRows][Q][Co]
+  float* xs = pw_smem;                                      // [strip][Q][Ci]
+  float* ds = pw_smem + strip * Q * Ci;                     // [strip][Q][Co]
   const int n = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
   const int outs = Ci * Co;
   const T* xn = x + (size_t)n * H * W * Ci;
   const T* dn = dy + (size_t)n * P * Q * Co;
-  double acc[2] = {0.0, 0.0};                               // thread tid owns outputs tid and tid + nt (if any)
-  for (int p0 = 0; p0 < P; p0 += kSmallWgradRows) {
-    const int rows = min(kSmallWgradRows, P - p0);
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};                     // thread tid owns outputs tid, tid + nt, ... (if any)
+  for (int p0 = 0; p0 < P; p0 += strip) {
+    const int rows = min(strip, P - p0);
     __syncthreads();
     for (int i = tid; i < rows * Q * Ci; i += nt) {
       const int c = i % Ci, q = (i / Ci) % Q, p = p0 + i / (Ci * Q);
@@ -356,7 +361,7 @@ __global__ void proj_wgrad_kernel(const T* __restrict__ x, const T* __restrict__
     for (int i = tid; i < rows * Q * Co; i += nt) ds[i] = to_f(dn[(size_t)p0 * Q * Co + i]);
     __syncthreads();
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
+    for (int k = 0; k < 4; ++k) {
       const int o = tid + k * nt;
       if (o >= outs) break;
       const int co = o % Co, ci = o / Co;
@@ -370,7 +375,7 @@ __global__ void proj_wgrad_kernel(const T* __restrict__ x, const T* __restrict__
     }
   }
 #pragma unroll
-  for (int k = 0; k < 2; ++k) {
+  for (int k = 0; k < 4; ++k) {
     const int o = tid + k * nt;
     if (o < outs) partial[(size_t)n * outs + (size_t)(o % Co) * Ci + o / Co] = (float)acc[k];
   }
@@ -380,8 +385,9 @@ inline cudaError_t launch_proj_wgrad(cudaStream_t st, const ConvGeom& g, const T
                                      float* dw, uint64_t* launches) {
   const int outs = g.Ci * g.Co;
   const int threads = outs >= 1024 ? 1024 : (outs + 31) / 32 * 32;
-  const size_t smem = (size_t)kSmallWgradRows * g.Q * (g.Ci + g.Co) * 4;
-  proj_wgrad_kernel<T><<<g.N, threads, smem, st>>>(x, dy, scratch, g.H, g.W, g.P, g.Q, g.Ci, g.Co, g.stride);
+  const int strip = proj_wgrad_strip(g);
+  const size_t smem = (size_t)strip * g.Q * (g.Ci + g.Co) * 4;
+  proj_wgrad_kernel<T><<<g.N, threads, smem, st>>>(x, dy, scratch, g.H, g.W, g.P, g.Q, g.Ci, g.Co, g.stride, strip);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   wgrad_reduce_kernel<<<(outs + 255) / 256, 256, 0, st>>>(scratch, dw, (size_t)outs, g.N);
