@@ -748,14 +748,29 @@ inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const 
 // dst[ci][2-r][2-s][co] = src[co][r][s][ci]; taps = 1: the transpose of a 1x1 filter.  One block row per entry of
 // `table` (src offset, dst offset, Co, Ci, taps), all offsets in elements from the two base pointers.
 struct FlipEntry { unsigned long long src, dst; int Co, Ci, taps; };
-__global__ void wflip_kernel(const __nv_bfloat16* __restrict__ src_base, __nv_bfloat16* __restrict__ dst_base,
-                             const FlipEntry* __restrict__ table) {
+__global__ void __launch_bounds__(256) wflip_kernel(const __nv_bfloat16* __restrict__ src_base, __nv_bfloat16* __restrict__ dst_base,
+                                                    const FlipEntry* __restrict__ table) {
+  // 32 x 32 tiles of one tap's [Co][Ci] matrix go through shared memory, so that both the reads (along ci) and
+  // the writes (along co) are contiguous.  256 threads = 32 columns x 8 rows.
+  __shared__ __nv_bfloat16 tile[32][34];
   const FlipEntry e = table[blockIdx.y];
-  const int T = e.taps;
-  const int n = e.Co * T * e.Ci;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-    const int co = i % e.Co, t = (i / e.Co) % T, ci = i / (T * e.Co);         // i indexes dst[ci][t][co]
-    dst_base[e.dst + i] = src_base[e.src + ((size_t)co * T + (T - 1 - t)) * e.Ci + ci];
+  const int T = e.taps;                                                       // 9, or 1: the plain transpose of a 1x1 filter
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int tco = (e.Co + 31) / 32, tci = (e.Ci + 31) / 32;
+  const int total = T * tco * tci;
+  for (int id = blockIdx.x; id < total; id += gridDim.x) {
+    const int t = id / (tco * tci), rem = id - t * tco * tci;
+    const int co0 = (rem / tci) * 32, ci0 = (rem - (rem / tci) * tci) * 32;
+    for (int j = ty; j < 32; j += 8) {
+      const int co = co0 + j, ci = ci0 + tx;
+      if (co < e.Co && ci < e.Ci) tile[j][tx] = src_base[e.src + ((size_t)co * T + t) * e.Ci + ci];
+    }
+    __syncthreads();
+    for (int j = ty; j < 32; j += 8) {
+      const int ci = ci0 + j, co = co0 + tx;
+      if (co < e.Co && ci < e.Ci) dst_base[e.dst + ((size_t)ci * T + (T - 1 - t)) * e.Co + co] = tile[tx][j];
+    }
+    __syncthreads();
   }
 }
 
