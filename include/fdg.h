@@ -263,6 +263,17 @@ fdg_status fdg_sync(fdg_ctx* ctx, fdg_stream stream);
  * fdg_sync returns it.  Blocks the host. */
 fdg_status fdg_debug_raise_flag(fdg_ctx* ctx, int which);
 
+/* Guard regions.  Every buffer the library carves out of the workspace is followed by 256 bytes that no kernel
+ * may write; fdg_create fills them with a pattern.  fdg_debug_check_guards waits for the context's work, compares
+ * every region and returns in *first_bad the index of the first region (in workspace order) that changed, or -1:
+ * a kernel that ran past the end of its buffer is then named by the buffer it overran.  fdg_debug_guard_count and
+ * fdg_debug_guard_offset give the number of regions and the byte offset of region `index` from the workspace
+ * base the caller passed to fdg_create (for a report, or for a test that damages one on purpose from the host).
+ * The regions are part of fdg_workspace_bytes and of a saved state.  No counterpart in the paper: a debugging aid. */
+fdg_status fdg_debug_guard_count(const fdg_ctx* ctx, size_t* out_count);
+fdg_status fdg_debug_guard_offset(const fdg_ctx* ctx, size_t index, size_t* out_byte_offset);
+fdg_status fdg_debug_check_guards(fdg_ctx* ctx, long long* first_bad);
+
 /* A wait that really runs out, without a kernel that misbehaves: enqueues on `stream` a one-warp kernel that
  * waits, with the bounded wait of the tensor-core kernels, on a barrier nothing ever arrives at.  After
  * `poll_limit` polls (1..2^20; a poll is well under a microsecond) the wait gives up, the kernel raises the

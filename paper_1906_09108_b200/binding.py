@@ -30,7 +30,8 @@ EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count"
            "fdg_conv_wgrad_scratch_bytes", "fdg_conv_wgrad", "fdg_conv_wgrad_static", "fdg_conv_path",
            "fdg_get_saved_tensor_of", "fdg_capture_bytes", "fdg_capture_begin", "fdg_capture_end", "fdg_get_captured",
            "fdg_bn_scratch_bytes", "fdg_bn_stats", "fdg_bn_apply", "fdg_bn_backward", "fdg_shrink", "fdg_sgd_update",
-           "fdg_ingest", "fdg_head", "fdg_debug_raise_flag", "fdg_debug_wait_probe", "fdg_lr_at", "fdg_set_lr_schedule", "fdg_bn_running_count",
+           "fdg_ingest", "fdg_head", "fdg_debug_raise_flag", "fdg_debug_wait_probe", "fdg_debug_guard_count", "fdg_debug_guard_offset",
+           "fdg_debug_check_guards", "fdg_lr_at", "fdg_set_lr_schedule", "fdg_bn_running_count",
            "fdg_get_bn_running", "fdg_set_bn_running", "fdg_eval", "fdg_drain", "fdg_state_bytes", "fdg_save_state",
            "fdg_load_state"]
 
@@ -128,6 +129,9 @@ def load_library(path=LIB_PATH):
         "fdg_get_saved_tensor_of": [vp, C.c_int, C.c_int, C.c_int, i64, vp, sz, P(sz), P(i64)],
         "fdg_debug_raise_flag": [vp, C.c_int],
         "fdg_debug_wait_probe": [vp, vp, C.c_uint],
+        "fdg_debug_guard_count": [vp, C.POINTER(C.c_size_t)],
+        "fdg_debug_guard_offset": [vp, C.c_size_t, C.POINTER(C.c_size_t)],
+        "fdg_debug_check_guards": [vp, C.POINTER(C.c_longlong)],
         "fdg_lr_at": [P(fdg_lr_schedule), i64, P(C.c_float)],
         "fdg_set_lr_schedule": [vp, P(fdg_lr_schedule)],
         "fdg_bn_running_count": [vp, C.c_int, P(sz)],
@@ -207,6 +211,7 @@ class FDG:
         self.workspace_bytes = n.value
         self.workspace = torch.empty(n.value + 256, dtype=torch.uint8, device=self.device)
         base = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.workspace_skip = base - self.workspace.data_ptr()     # bytes of `workspace` before the library's base
         ctx = C.c_void_p()
         self._check(self.lib.fdg_create(C.byref(self.arch), C.byref(self.cfg), base, n.value, None, C.byref(ctx)), None)
         self.ctx = ctx
@@ -324,6 +329,21 @@ class FDG:
         st = self.torch.cuda.current_stream().cuda_stream if stream is None else stream
         self._check(self.lib.fdg_step_host(self.ctx, st, images_host.data_ptr(), labels_host.data_ptr(),
                                            loss_host.data_ptr() if loss_host is not None else None), self.ctx)
+
+    def guard_offsets(self):
+        """Byte offsets (from the workspace base given to fdg_create) of the guard regions behind the buffers."""
+        n, off, out = C.c_size_t(), C.c_size_t(), []
+        self._check(self.lib.fdg_debug_guard_count(self.ctx, C.byref(n)), self.ctx)
+        for i in range(n.value):
+            self._check(self.lib.fdg_debug_guard_offset(self.ctx, i, C.byref(off)), self.ctx)
+            out.append(off.value)
+        return out
+
+    def check_guards(self):
+        """-1, or the index of the first guard region that was overwritten."""
+        bad = C.c_longlong()
+        self._check(self.lib.fdg_debug_check_guards(self.ctx, C.byref(bad)), self.ctx)
+        return bad.value
 
     def profile_enable(self, on=True):
         self._check(self.lib.fdg_profile_enable(self.ctx, int(on)), self.ctx)

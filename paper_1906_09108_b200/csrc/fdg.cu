@@ -19,6 +19,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <climits>
 #include <cstring>
 #include <mutex>
 #include <string>
@@ -144,7 +145,10 @@ struct fdg_ctx {
   cudaEvent_t ev_join;
   int32_t* labels = nullptr;          // ring of label_ring batches
   int label_ring = 0;
-  int* flags = nullptr;               // [0] non-finite loss, [1] label out of range, [2] a tensor-core kernel's wait ran out
+  int* flags = nullptr;               // [0] non-finite loss, [1] label out of range, [2] a tensor-core kernel's wait ran out,
+                                      // [3] result word of the guard check
+  std::vector<size_t> guard_offsets;  // byte offsets of the guard regions behind the workspace buffers
+  unsigned long long* guard_table = nullptr;   // the same on the device
   float* staging = nullptr;           // fp32 staging for getters
   float* host_images = nullptr;       // device staging of fdg_step_host
   int32_t* host_labels = nullptr;
@@ -194,17 +198,36 @@ namespace fdg {
 // ------------------------------------------------------------------ planning --
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Every buffer carved out of the workspace is followed by kGuardBytes that no kernel may write: they are
+// filled with a pattern at creation and compared on request (fdg_debug_check_guards), so a kernel that
+// runs past the end of its buffer is found at the buffer it overran instead of in its neighbour's results.
+constexpr size_t kGuardBytes = 256;
+constexpr unsigned int kGuardWord = 0xA5C3F00Du;
 struct Carver {
   char* base;
   size_t off = 0;
+  size_t count = 0;                        // buffers taken so far
+  std::vector<size_t>* guards = nullptr;   // byte offsets of the guard regions, in order (recorded when set)
   explicit Carver(char* b) : base(b) {}
   template <typename P> P* take(size_t bytes) {
     off = align_up(off, 256);
     P* p = base ? reinterpret_cast<P*>(base + off) : nullptr;
-    off += bytes;
+    off = align_up(off + bytes, 256);
+    if (guards) guards->push_back(off);
+    off += kGuardBytes;
+    ++count;
     return p;
   }
 };
+__global__ void guard_fill_kernel(char* __restrict__ base, const unsigned long long* __restrict__ offsets) {
+  reinterpret_cast<unsigned int*>(base + offsets[blockIdx.x])[threadIdx.x] = kGuardWord;
+}
+// *first_bad = the lowest index of a guard region that no longer holds the pattern (left untouched if all do)
+__global__ void guard_check_kernel(const char* __restrict__ base, const unsigned long long* __restrict__ offsets,
+                                   int* __restrict__ first_bad) {
+  if (reinterpret_cast<const unsigned int*>(base + offsets[blockIdx.x])[threadIdx.x] != kGuardWord)
+    atomicMin(first_bad, (int)blockIdx.x);
+}
 
 static int conv_out(int n, int r, int stride, int pad) { return (n + 2 * pad - r) / stride + 1; }
 static int pow2_at_least(int x) { int p = 1; while (p < x) p <<= 1; return p; }
@@ -456,6 +479,8 @@ static void plan_modules(fdg_ctx* c) {
 // Assigns every device pointer; with base == nullptr only measures.
 static size_t carve(fdg_ctx* c, char* base) {
   Carver cv(base);
+  c->guard_offsets.clear();
+  cv.guards = &c->guard_offsets;
   const size_t es = c->esize;
   c->flags = cv.take<int>(256);
   c->tc_error = c->flags ? c->flags + 2 : nullptr;
@@ -503,6 +528,7 @@ static size_t carve(fdg_ctx* c, char* base) {
   c->host_labels = cv.take<int32_t>((size_t)c->arch.batch * 4);
   c->staging_elems = stage;
   c->staging = cv.take<float>(stage * 4);
+  c->guard_table = cv.take<unsigned long long>((cv.count + 1) * sizeof(unsigned long long));   // one entry per buffer, itself included
   return align_up(cv.off, 256);
 }
 
@@ -1189,6 +1215,14 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   carve(c, static_cast<char*>(dev_workspace));
   c->ws_base = static_cast<char*>(dev_workspace);
   c->ws_bytes = need;
+  {
+    std::vector<unsigned long long> table(c->guard_offsets.begin(), c->guard_offsets.end());
+    e = cudaMemcpy(c->guard_table, table.data(), table.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) {
+      guard_fill_kernel<<<(unsigned)table.size(), (unsigned)(kGuardBytes / 4)>>>(c->ws_base, c->guard_table);
+      e = cudaGetLastError();
+    }
+  }
   for (Module& m : c->mods) {
     if (m.flip_table_dev && e == cudaSuccess)
       e = cudaMemcpy(m.flip_table_dev, m.flip_table.data(), m.flip_table.size() * sizeof(tc::FlipEntry), cudaMemcpyHostToDevice);
@@ -1541,6 +1575,35 @@ fdg_status fdg_debug_raise_flag(fdg_ctx* c, int which) {
   if (e == cudaSuccess) e = cudaMemcpy(c->flags + which, &one, sizeof(int), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   return e == cudaSuccess ? FDG_OK : cuda_fail(c, e, "raising a status word");
+}
+
+fdg_status fdg_debug_guard_count(const fdg_ctx* c, size_t* out_count) {
+  if (!c || !out_count) return FDG_ERR_INVALID_ARG;
+  *out_count = c->guard_offsets.size();
+  return FDG_OK;
+}
+
+fdg_status fdg_debug_guard_offset(const fdg_ctx* c, size_t index, size_t* out_byte_offset) {
+  if (!c || !out_byte_offset || index >= c->guard_offsets.size()) return FDG_ERR_INVALID_ARG;
+  *out_byte_offset = c->guard_offsets[index];
+  return FDG_OK;
+}
+
+fdg_status fdg_debug_check_guards(fdg_ctx* c, long long* out_first_bad) {
+  if (!c || !out_first_bad) return FDG_ERR_INVALID_ARG;
+  cudaError_t e = drain(c);
+  const int none = INT_MAX;
+  if (e == cudaSuccess) e = cudaMemcpy(c->flags + 3, &none, sizeof(int), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) {
+    guard_check_kernel<<<(unsigned)c->guard_offsets.size(), (unsigned)(kGuardBytes / 4)>>>(c->ws_base, c->guard_table, c->flags + 3);
+    ++c->launches;
+    e = cudaGetLastError();
+  }
+  int got = none;
+  if (e == cudaSuccess) e = cudaMemcpy(&got, c->flags + 3, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(c, e, "guard check");
+  *out_first_bad = got == none ? -1 : (long long)got;
+  return FDG_OK;
 }
 
 fdg_status fdg_debug_wait_probe(fdg_ctx* c, fdg_stream stream, unsigned poll_limit) {

@@ -111,5 +111,6 @@ def run_pair(arch_kw, K, splits, steps, beta=0.5, lr=0.1, momentum=0.9, weight_d
     res["log_gpu"] = [(r["t"], r["k"], r["tau_f"], r["tau_b"], r["ver_f"], r["ver_b"]) for r in g.schedule_log()]
     res["log_oracle"] = [(r["t"], r["k"], r["tau_f"], r["tau_b"], r["ver_f"], r["ver_b"]) for r in orc.log]
     res["launches"] = g.launch_count()
+    assert g.check_guards() == -1          # no kernel wrote past the end of a workspace buffer
     g.close()
     return res

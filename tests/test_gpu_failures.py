@@ -123,3 +123,30 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
     g2.step(*_batch(2), loss)
     assert _status(g2, g2.sync) == B.FDG_OK and np.isfinite(loss.item())
     g2.close()
+
+
+@pytest.mark.parametrize("precision", ["fp32", "bf16"])
+def test_guard_regions_stay_clean_and_a_damaged_one_is_named(precision):
+    """Every workspace buffer is followed by 256 guard bytes.  After real work (stream issue and graph replay) they
+    all still hold their pattern; one byte changed from the host, standing in for a kernel that ran past its
+    buffer, is reported with the index of that region, and a restored byte clears the report."""
+    from paper_1906_09108_b200 import binding as B
+    g = _make(B, 2, (1,), precision=B.FDG_BF16_TC if precision == "bf16" else B.FDG_FP32_CUDACORE, graphs=True)
+    offs = g.guard_offsets()
+    assert len(offs) > 20 and offs == sorted(offs) and all(o % 256 == 0 for o in offs)
+    assert offs[-1] + 256 <= g.workspace_bytes
+    assert g.check_guards() == -1
+    for t in range(1, 12):
+        g.step(*_batch(t))
+    g.sync()
+    assert g.check_guards() == -1
+    for idx in (len(offs) // 2, 3):
+        at = g.workspace_skip + offs[idx] + 17
+        old = int(g.workspace[at].item())
+        g.workspace[at] = old ^ 0x5A
+        assert g.check_guards() == idx
+        g.workspace[at] = old
+        assert g.check_guards() == -1
+    g.step(*_batch(12))
+    assert _status(g, g.sync) == B.FDG_OK
+    g.close()

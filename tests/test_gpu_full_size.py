@@ -102,6 +102,7 @@ def test_forward_of_every_block_at_full_size():
                 worst[key] = max(worst.get(key, 0.0), err)
                 assert err <= 1e-2, (k, name, key, err)         # one bfloat16 ulp of the largest element is 4e-3
             checked += 1
+    assert g.check_guards() == -1          # no kernel wrote past the end of a workspace buffer
     g.close()
     assert checked == 51                                      # every block whose input is saved in the same module (13 + 13 + 13 + 12)
     print("worst relative errors over %d blocks:" % checked, worst)
@@ -122,6 +123,7 @@ def test_backward_of_every_block_at_full_size():
     from tests.layerwise import check_backward_layerwise
     g, params = _make(B, lr=0.0, weight_decay=0.0)
     checked, worst = check_backward_layerwise(g, params, ARCH, 4)
+    assert g.check_guards() == -1          # no kernel wrote past the end of a workspace buffer
     g.close()
     assert checked == 54
     print("worst relative errors over %d blocks:" % checked, {k_: float("%.2g" % v) for k_, v in worst.items()})

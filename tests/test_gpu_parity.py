@@ -71,6 +71,7 @@ def test_serial_mode_is_bitwise_identical_to_streams():
             g.step(x, y)
         g.sync()
         outs.append([g.get_params(k) for k in range(1, 5)])
+        assert g.check_guards() == -1          # no kernel wrote past the end of a workspace buffer
         g.close()
     for a, b in zip(*outs):
         assert np.array_equal(a, b)
@@ -107,6 +108,7 @@ def test_graph_replay_is_bitwise_identical_to_streams(precision):
         outs.append([g.get_params(k) for k in range(1, 5)] + [g.get_momentum(k) for k in range(1, 5)])
         losses.append(ls)
         assert len(g.schedule_log()) == 40 * 4
+        assert g.check_guards() == -1          # no kernel wrote past the end of a workspace buffer
         g.close()
     assert losses[0] == losses[1]
     for a, b in zip(*outs):
@@ -216,6 +218,7 @@ def test_wrn_runs_are_bitwise_repeatable():
             g.step(torch.from_numpy(S.images(0, t, 8, 32, 32, 3)).cuda(), torch.from_numpy(S.labels(0, t, 8, 20)).cuda())
         g.sync()
         outs.append([g.get_params(k) for k in (1, 2)] + [g.get_grads(k) for k in (1, 2)])
+        assert g.check_guards() == -1          # no kernel wrote past the end of a workspace buffer
         g.close()
     for other in outs[1:]:
         for a, b in zip(outs[0], other):
@@ -311,6 +314,7 @@ def test_resnet18_form_bf16():
     for k in (1, 2):
         g.set_params(k, params[k])
     checked, worst = check_backward_layerwise(g, params, arch, 2)
+    assert g.check_guards() == -1          # no kernel wrote past the end of a workspace buffer
     g.close()
     assert checked == 8, worst
     arch = dict(TC_NET, n_per_stage=2, shortcut="zero_pad")

@@ -84,6 +84,7 @@ def test_workspace_bytes_and_argument_checks(lib):
     assert not ctx.value
     assert lib.fdg_create(C.byref(arch), C.byref(cfg), C.c_void_p((1 << 20) + 8), n.value, None, C.byref(ctx)) == 1   # misaligned
     assert lib.fdg_debug_raise_flag(None, 0) == 1
+    assert lib.fdg_debug_guard_count(None, C.byref(n)) == 1 and lib.fdg_debug_check_guards(None, None) == 1
     # operator level: argument checks that answer without a GPU
     s = B.fdg_conv_shape(2, 8, 8, 512, 512, 3, 1, 1)
     assert lib.fdg_conv_wgrad_static(0, C.byref(s), C.c_void_p(256), C.c_void_p(256), C.c_void_p(256), None) == 2
