@@ -1,5 +1,6 @@
-"""Layer-by-layer check of one backward pass of every module of a 6n+2 network against the oracle's layer
-functions (oracle/layers.py), used by the full-size test and by the smoke check.
+"""Layer-by-layer check of one backward pass of every module of a network (post-activation 6n+2 / ResNet-18 blocks,
+or the pre-activation blocks of the wide residual networks) against the oracle's layer functions
+(oracle/layers.py), used by the full-size test, the architecture tests and the smoke check.
 
 A capture (fdg_capture_begin) keeps every gradient tensor of each module's backward pass at iteration 2K - 1,
 the first one in which all K modules back-propagate (module k then handles batch k).  Every layer of every
@@ -58,7 +59,12 @@ def check_backward_layerwise(g, params, arch, K, seed=0, tol=1e-2):
         for u, (name, ent) in enumerate(units):
             if name == "head":
                 continue
-            for which in ((0, 3) if name == "stem" else (0, 1, 2, 3) + ((4,) if len(ent) > 6 else ())):
+            preact = len(ent[0][1]) == 1                             # a pre-activation block starts with a batch norm
+            if name == "stem":
+                want = (0, 3) if len(ent) > 1 else (3,)              # the wide networks' stem is a bare convolution
+            else:
+                want = (0, 1, 2, 3) + ((4,) if (len(ent) > 6 and not preact) else ())
+            for which in want:
                 bb, a = g.saved_tensor_of(k, u, which, k)
                 assert bb == k, (k, u, which, bb)
                 saved[(k, u, which)] = a
@@ -91,16 +97,42 @@ def check_backward_layerwise(g, params, arch, K, seed=0, tol=1e-2):
         for u, (name, ent) in enumerate(units):
             where = (k, name)
             if name == "head":
-                feat = int(ent[0][1][1])
+                with_bn = len(ent) == 4                              # wide networks: batch norm + ReLU before the pooling
+                efc = ent[2:] if with_bn else ent
+                feat = int(efc[0][1][1])
                 hwl = int(round((saved[(k, u - 1, 3)].size / (b * feat)) ** 0.5))
                 ylast = saved[(k, u - 1, 3)].reshape(b, hwl, hwl, feat).astype(np.float64)
-                wfc, bfc = _take(flat, ent[0]), _take(flat, ent[1])
-                pooled = L.gap_forward(ylast)
-                loss, probs = L.softmax_xent_forward(L.fc_forward(pooled, wfc, bfc), S.labels(seed, k, b, classes).astype(np.int64))
-                dpool, dwo, dbo = L.fc_backward(L.softmax_xent_backward(probs, S.labels(seed, k, b, classes).astype(np.int64)), pooled, wfc)
-                cmp("head.dx", cap(u - 1, 0, ylast.shape), q(L.gap_backward(dpool, ylast.shape)), where)
-                cmp("fc.dw", _take(grads, ent[0]), dwo, where, 1e-4)
-                cmp("fc.db", _take(grads, ent[1]), dbo, where, 1e-4)
+                wfc, bfc = _take(flat, efc[0]), _take(flat, efc[1])
+                labels = S.labels(seed, k, b, classes).astype(np.int64)
+                if with_bn:
+                    gh, bh = _take(flat, ent[0]), _take(flat, ent[1])
+                    bno, svh = L.batchnorm_forward(ylast, gh, bh, EPS)
+                    feat_in = q(L.relu_forward(bno))
+                else:
+                    feat_in = ylast
+                pooled = L.gap_forward(feat_in)
+                loss, probs = L.softmax_xent_forward(L.fc_forward(pooled, wfc, bfc), labels)
+                dpool, dwo, dbo = L.fc_backward(L.softmax_xent_backward(probs, labels), pooled, wfc)
+                dfeat = q(L.gap_backward(dpool, ylast.shape))
+                if with_bn:
+                    dyl, dgh, dbh = L.batchnorm_backward(L.relu_backward(dfeat, feat_in), svh, gh)
+                    cmp("head.dx", cap(u - 1, 0, ylast.shape), q(dyl), where)
+                    cmp("head.bn.dgamma", _take(grads, ent[0]), dgh, where, 1e-3)
+                    cmp("head.bn.dbeta", _take(grads, ent[1]), dbh, where, 1e-3)
+                else:
+                    cmp("head.dx", cap(u - 1, 0, ylast.shape), dfeat, where)
+                cmp("fc.dw", _take(grads, efc[0]), dwo, where, 1e-3 if with_bn else 1e-4)
+                cmp("fc.db", _take(grads, efc[1]), dbo, where, 1e-3 if with_bn else 1e-4)
+                continue
+            if name == "stem" and len(ent) == 1:                     # a bare convolution: only its weight gradient
+                w1 = q(_take(flat, ent[0]))
+                x_in = q(S.images(seed, k, b, hw0, hw0, 3).astype(np.float64))
+                dy = cap(u, 0, (b, hw0, hw0, w1.shape[0]))
+                cmp("stem.dw", _take(grads, ent[0]), L.conv2d_backward(dy, x_in, w1, 1, 1)[1], where)
+                continue
+            if len(ent[0][1]) == 1:
+                _check_preact(k, u, ent, flat, grads, saved, cap, cmp, q, g, b, where, _units, _take)
+                checked += 1
                 continue
             if name == "stem":
                 w1 = q(_take(flat, ent[0])); g1, b1 = _take(flat, ent[1]), _take(flat, ent[2])
@@ -163,3 +195,50 @@ def check_backward_layerwise(g, params, arch, K, seed=0, tol=1e-2):
     for k in range(1, K + 1):
         g.capture_end(k)
     return checked, worst
+
+
+def _check_preact(k, u, ent, flat, grads, saved, cap, cmp, q, g, b, where, _units, _take):
+    """One pre-activation block: o = relu(bn1(x)), c1 = conv1(o), a2 = relu(bn2(c1)), y = conv2(a2) + shortcut, the
+    shortcut being x or a 1x1 convolution of o.  Saved: o, c1, a2, y.  Captured: dy, da2, dc1, do (+ the shortcut's
+    share), dx, and the shortcut's share alone."""
+    g1, b1 = _take(flat, ent[0]), _take(flat, ent[1])
+    w1 = q(_take(flat, ent[2]))
+    g2, b2 = _take(flat, ent[3]), _take(flat, ent[4])
+    w2 = q(_take(flat, ent[5]))
+    proj = len(ent) > 6
+    co, ci = w1.shape[0], w1.shape[3]
+    x_flat = saved[(k, u - 1, 3)] if u > 0 else g.saved_tensor_of(k - 1, len(_units(g.param_layout(k - 1))) - 1, 3, k)[1]
+    hw_in = int(round((x_flat.size / (b * ci)) ** 0.5))
+    x_in = x_flat.reshape(b, hw_in, hw_in, ci).astype(np.float64)
+    hw = int(round((saved[(k, u, 3)].size / (b * co)) ** 0.5))
+    stride = hw_in // hw
+    shp = (b, hw, hw, co)
+    o = saved[(k, u, 0)].reshape(x_in.shape).astype(np.float64)
+    c1, a2 = (saved[(k, u, i)].reshape(shp).astype(np.float64) for i in (1, 2))
+    dy = cap(u, 0, shp)
+    da2_o, dw2_o = L.conv2d_backward(dy, a2, w2, 1, 1)
+    da2 = cap(u, 1, shp)
+    cmp("da2", da2, q(da2_o), where)
+    cmp("conv2.dw", _take(grads, ent[5]), dw2_o, where)
+    dc1_o, dg2_o, db2_o = L.batchnorm_backward(L.relu_backward(da2, a2), L.batchnorm_forward(c1, g2, b2, EPS)[1], g2)
+    dc1 = cap(u, 2, shp)
+    cmp("dc1", dc1, q(dc1_o), where)
+    cmp("bn2.dgamma", _take(grads, ent[3]), dg2_o, where)
+    cmp("bn2.dbeta", _take(grads, ent[4]), db2_o, where)
+    do_o, dw1_o = L.conv2d_backward(dc1, o, w1, stride, 1)
+    cmp("conv1.dw", _take(grads, ent[2]), dw1_o, where)
+    if proj:
+        ws = q(_take(flat, ent[6]))
+        dos_o, dws_o = L.conv2d_backward(dy, o, ws, stride, 0)
+        dos = cap(u, 5, x_in.shape)
+        cmp("dos", dos, q(dos_o), where)
+        cmp("sc.dw", _take(grads, ent[6]), dws_o, where)
+        do_o = do_o + dos
+    do = cap(u, 3, x_in.shape)
+    cmp("do", do, q(do_o), where)
+    dx_o, dg1_o, db1_o = L.batchnorm_backward(L.relu_backward(do, o), L.batchnorm_forward(x_in, g1, b1, EPS)[1], g1)
+    if not proj:
+        dx_o = dx_o + dy
+    cmp("dx", cap(u, 4, x_in.shape), q(dx_o), where)
+    cmp("bn1.dgamma", _take(grads, ent[0]), dg1_o, where)
+    cmp("bn1.dbeta", _take(grads, ent[1]), db1_o, where)

@@ -322,3 +322,25 @@ def test_resnet18_form_bf16():
     assert res["log_gpu"] == res["log_oracle"]
     msg = str({k: v for k, v in res.items() if not k.startswith("log_")})
     assert res["params"] <= 2e-2 and res["loss"] <= 1e-2 and res["out"] <= 5e-2 and res["params_plain"] <= 2e-2, msg
+
+
+def test_wrn_widths_bf16_layer_by_layer():
+    """Pre-activation blocks at the channel widths of WRN-28-10 (160 / 320 / 640, two blocks per stage, batch 4, K = 2):
+    every layer of one backward pass of both modules -- the patch-tile and per-tap tensor-core convolutions, the
+    exact-tile weight gradient, the strided 3x3 layers through the spread-out dy, the 1x1 shortcuts (stride 1 from 16
+    channels, stride 2 through the strided tensor map), the head with its batch norm -- recomputed by the oracle's
+    layer functions from the library's own inputs to that layer, at 1e-2."""
+    import fdg_synth as S
+    from paper_1906_09108_b200 import binding as B
+    from tests.layerwise import check_backward_layerwise
+    arch = dict(family="wrn", n_per_stage=2, widths=(160, 320, 640), stem_width=16, in_h=32, in_w=32, in_c=3,
+                num_classes=10, batch=4)
+    g = B.FDG(B.make_arch(**arch), K=2, split_after_block=(3,), beta=0.5, lr=0.0, weight_decay=0.0, precision=B.FDG_BF16_TC)
+    params = {k: S.init_params(0, k, g.param_layout(k), jitter=True) for k in (1, 2)}
+    for k in (1, 2):
+        g.set_params(k, params[k])
+    checked, worst = check_backward_layerwise(g, params, arch, 2)
+    assert g.check_guards() == -1          # no kernel wrote past the end of a workspace buffer
+    g.close()
+    assert checked == 6, worst
+    print("worst relative errors:", {k: float("%.2g" % v) for k, v in worst.items()})
