@@ -228,9 +228,9 @@ inline cudaError_t run_wgrad_wide(cudaStream_t st, TensorMapCache* cache, int N,
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const size_t n4 = (size_t)Co * R * R * Ci / 4;                 // Ci is a multiple of 16
-  wide::wgrad_wide_sum_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const float4*>(scratch),
-                                                                          reinterpret_cast<float4*>(dw), n4, p.splits);
-  return cudaGetLastError();
+  // the sum's launch overlaps the tail of the kernel above; it waits for that kernel before it reads
+  return launch_chained(wide::wgrad_wide_sum_kernel, dim3((unsigned)((n4 + 255) / 256)), dim3(256), 0, st,
+                        reinterpret_cast<const float4*>(scratch), reinterpret_cast<float4*>(dw), n4, p.splits);
 }
 
 // Does the data gradient of this convolution read the flipped/transposed weight copy?

@@ -160,25 +160,45 @@ wgrad_wide_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       if (ok) tc_commit(done);
     }
   } else {
+    // Write-out.  A lane holds one output row (an output channel) of the accumulators; written straight from
+    // registers, a warp's store would touch 32 rows 11 KB apart with 16 bytes each.  Each 32 x 32 block therefore
+    // goes through shared memory (the pipeline's stages are idle by now) and leaves as 128-byte row segments.
     const int lane_grp = warp & 3;
     if (mbar_wait(done, 0, abort_flag)) {
       tc_fence_after();
-      const int co = co0 + lane_grp * 32 + lane;
-      const bool row_ok = co < p.Co;
+      float* stage = reinterpret_cast<float*>(smem) + (size_t)lane_grp * (32 * 33);   // this warp's [32][33] block
+      const int row_base = co0 + lane_grp * 32;
       const size_t ftaps = (size_t)p.rdim * p.taps;                        // taps of the whole filter: 9 or 1
-      float* dst = partial + (size_t)blockIdx.y * ((size_t)p.Co * ftaps * p.Ci) +
-                   ((size_t)co * ftaps + (size_t)r * p.taps) * p.Ci + ci0;
+      const size_t row_stride = ftaps * p.Ci;
+      float* dst = partial + (size_t)blockIdx.y * ((size_t)p.Co * row_stride) + ((size_t)row_base * ftaps + (size_t)r * p.taps) * p.Ci + ci0;
+      const int sub_row = lane >> 3, col4 = (lane & 7) * 4;                // write-out: 4 rows x 8 lanes x 4 columns
       for (int sx = 0; sx < p.taps; ++sx) {
-        for (int c0 = 0; c0 < p.nci; c0 += 16) {
+        for (int c0 = 0; c0 < p.nci; c0 += 32) {
+          const int ncol = min(32, p.nci - c0);                            // 32, or 16 at the end of a chunk
           uint32_t v[16];
           tmem_ld16(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(sx * p.nci + c0), v);
           tmem_ld_wait();
-          if (!row_ok || ci0 + c0 >= p.Ci) continue;
-          float4* d4 = reinterpret_cast<float4*>(dst + (size_t)sx * p.Ci + c0);
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            d4[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]),
-                                __uint_as_float(v[4 * e + 3]));
+          for (int e = 0; e < 16; ++e) stage[lane * 33 + e] = __uint_as_float(v[e]);
+          if (ncol == 32) {
+            tmem_ld16(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(sx * p.nci + c0 + 16), v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) stage[lane * 33 + 16 + e] = __uint_as_float(v[e]);
+          }
+          __syncwarp();
+          if (col4 < ncol && ci0 + c0 + col4 < p.Ci) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int rr = i * 4 + sub_row;
+              if (row_base + rr < p.Co) {
+                const float* src = stage + rr * 33 + col4;
+                *reinterpret_cast<float4*>(dst + (size_t)rr * row_stride + (size_t)sx * p.Ci + c0 + col4) =
+                    make_float4(src[0], src[1], src[2], src[3]);
+              }
+            }
+          }
+          __syncwarp();
         }
       }
     }
@@ -206,6 +226,7 @@ wgrad_wide_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 // dw[i] = partial[0][i] + partial[1][i] + ... in split order; four consecutive outputs per thread.
 __global__ void __launch_bounds__(256) wgrad_wide_sum_kernel(const float4* __restrict__ partial, float4* __restrict__ dw,
                                                              size_t n4, int splits) {
+  grid_dependency_wait();                 // launched ahead of the end of the kernel that writes `partial`
   const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= n4) return;
   float4 a = partial[i];
