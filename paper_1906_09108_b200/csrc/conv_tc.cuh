@@ -272,9 +272,16 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint64_t a0 = a_desc[s], b0 = b_desc[s];
-          for (int j = 0; j < ksub; ++j) tc_mma_bf16(d_tmem, a0 + 2 * j, b0 + 2 * j, idesc, (ki | j) != 0);
-          if (halves == 2)
-            for (int j = 0; j < ksub; ++j) tc_mma_bf16(d_tmem + (uint32_t)p.n_tile, a0 + half_off + 2 * j, b0 + 2 * j, idesc, (ki | j) != 0);
+          // Two instructions in a row into the same accumulator wait for each other (about 137 cycles apart,
+          // whatever N is); the two 128-row tiles therefore take turns.
+          if (halves == 2) {
+            for (int j = 0; j < ksub; ++j) {
+              tc_mma_bf16(d_tmem, a0 + 2 * j, b0 + 2 * j, idesc, (ki | j) != 0);
+              tc_mma_bf16(d_tmem + (uint32_t)p.n_tile, a0 + half_off + 2 * j, b0 + 2 * j, idesc, (ki | j) != 0);
+            }
+          } else {
+            for (int j = 0; j < ksub; ++j) tc_mma_bf16(d_tmem, a0 + 2 * j, b0 + 2 * j, idesc, (ki | j) != 0);
+          }
           tc_commit(&empty[s]);
           if (++s == p.stages) { s = 0; ph ^= 1; }
         }
