@@ -420,6 +420,28 @@ def run_kernel_bench(args):
                     us=us, mbytes=nbytes / 1e6, gbs=nbytes / us / 1e3, hbm_frac=nbytes / us / 1e3 / peaks["hbm_gbs"])
         print(json.dumps(dict(kernel_bench=out, peak_source=peaks["source"], hbm_gbs=peaks["hbm_gbs"])))
         return
+    if args.kernel_bench == "mma_rate":
+        # cycles per tcgen05.mma (M = 128, K = 16) issued back to back by one thread per SM, for N and for the number
+        # of accumulators the instructions rotate over (fdg_probe_mma_rate): the two rates the wide kernels are built on
+        import torch
+        ops = B.ConvOps(B.FDG_BF16_TC)
+        cyc = torch.zeros(2, dtype=torch.int64, device="cuda")
+        reps = 200
+        table = {}
+        for unrolled in (1, 0):
+            for accs in (1, 3):
+                for n in (16, 64, 128, 160, 256):
+                    if n * accs > 512:
+                        continue
+                    ops._chk(ops.lib.fdg_probe_mma_rate(n, accs, reps, unrolled, cyc.data_ptr(), ops.status.data_ptr(),
+                                                        torch.cuda.current_stream().cuda_stream))
+                    torch.cuda.synchronize()
+                    issued, done = (int(v) for v in cyc.cpu())
+                    table["%s_N%d_acc%d" % ("straight" if unrolled else "looped", n, accs)] = dict(
+                        issue=round(issued / (reps * 4 * accs), 1), complete=round(done / (reps * 4 * accs), 1))
+        assert not ops.timed_out()
+        print(json.dumps(dict(mma_rate_cycles_per_instruction=table)))
+        return
     which_list = {"all": ["fprop", "dgrad", "wgrad"], "step": list(STEP_VARIANTS)}.get(args.kernel_bench, [args.kernel_bench])
     if args.kernel_bench == "step" and not args.kernel_stage:
         args.kernel_stage = "stage1"
@@ -624,7 +646,7 @@ def main():
     ap.add_argument("--workload", default="resnet110_k4", choices=list(WORKLOADS))
     ap.add_argument("--splits", default=None,
                     help="comma-separated block indices after which the modules end, instead of the workload's own")
-    ap.add_argument("--kernel-bench", default=None, choices=["fprop", "dgrad", "wgrad", "all", "ew", "step"] + EW_KERNELS + list(STEP_VARIANTS),
+    ap.add_argument("--kernel-bench", default=None, choices=["fprop", "dgrad", "wgrad", "all", "ew", "step", "mma_rate"] + EW_KERNELS + list(STEP_VARIANTS),
                     help="time the convolution kernels alone through the operator-level C ABI and exit")
     ap.add_argument("--kernel-launches", type=int, default=64,
                     help="launches per replay; 8 or fewer are issued as plain launches (profiler runs)")

@@ -76,6 +76,17 @@ fdg_status fdg_conv_dgrad(int precision, const fdg_conv_shape* shape, const void
                           const void* w_flipped, void* dx, const void* res, const void* res_mask,
                           fdg_conv_extra* extra, int* status_dev, fdg_stream stream);
 
+/* Probe of the tensor pipe, for roofline arguments (no counterpart in the paper): on every SM one thread issues
+ * reps * 4 * accumulators tcgen05.mma instructions (M = 128, N = n, K = 16, bf16, operands in shared memory) back to
+ * back, rotating over `accumulators` (1..3, n * accumulators <= 512) accumulators in tensor memory; `unrolled` = 1
+ * issues them as straight-line code, 0 keeps the rotation as a run-time loop (a counter and a branch between two
+ * instructions: what a kernel's issuing loop costs when it is not unrolled).
+ * cycles_dev[0] = SM cycles until the last one was issued, cycles_dev[1] = until it completed (device pointer to two
+ * 64-bit integers, written by the first CTA).  n: multiple of 16 in 16..256.  Its wait is bounded like every other;
+ * status_dev as above.  Asynchronous on `stream`. */
+fdg_status fdg_probe_mma_rate(int n, int accumulators, int reps, int unrolled, long long* cycles_dev, int* status_dev,
+                              fdg_stream stream);
+
 /* w_flipped[ci][R-1-r][R-1-s][co] = w[co][r][s][ci] (bf16, R = 3 or 1): the operand layout of the
  * tensor-core data-gradient kernel. */
 fdg_status fdg_conv_flip_weights(const fdg_conv_shape* shape, const void* w_bf16, void* w_flipped_bf16,

@@ -272,8 +272,9 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint64_t a0 = a_desc[s], b0 = b_desc[s];
-          // Two instructions in a row into the same accumulator wait for each other (about 137 cycles apart,
-          // whatever N is); the two 128-row tiles therefore take turns.
+          // Straight-line issue: the choice between one and two 128-row tiles is made outside the loop over the
+          // K steps (a branch between two tcgen05.mma costs the lone issuing thread tens of cycles, see
+          // mma_rate_kernel), and the two tiles take turns.
           if (halves == 2) {
             for (int j = 0; j < ksub; ++j) {
               tc_mma_bf16(d_tmem, a0 + 2 * j, b0 + 2 * j, idesc, (ki | j) != 0);
@@ -749,6 +750,70 @@ inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const 
   const int grid = tiles < sm_count ? tiles : sm_count;
   conv3x3_tc_kernel<<<grid, kThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, error_word);
   return cudaGetLastError();
+}
+
+// Probe of the tensor pipe's instruction rate, for the roofline arguments about the kernels above: one thread of one
+// CTA per SM issues `reps` x 4 x `accs` instructions (M = 128, N = n, K = 16, bf16, both operands K-major in
+// 128-byte-swizzled shared memory whose contents do not matter) back to back, rotating over `accs` accumulators, and
+// waits for the last one.  out[0] = cycles until the last one was issued, out[1] = until it completed (CTA 0).
+// `unrolled` = 0 keeps the rotation over the accumulators as a run-time loop: the same instructions with a loop
+// counter and a branch between them, which is what an issuing loop that is not unrolled looks like.
+__global__ void __launch_bounds__(128, 1) mma_rate_kernel(int n, int accs, int reps, int unrolled, long long* __restrict__ out,
+                                                          int* __restrict__ error_word) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t slot;
+  __shared__ int flag;
+  volatile int* abort_flag = &flag;
+  // A: 128 rows x 128 bytes; B: 256 rows x 128 bytes; finite values
+  for (int i = threadIdx.x; i < 48 * 1024 / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem)[i] = 0x3c003c00u;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (threadIdx.x < 32) tmem_alloc(&slot, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = slot;
+  if (threadIdx.x == 0) {
+    const uint32_t a_addr = smem_u32(smem), b_addr = a_addr + 16 * 1024;
+    const uint64_t a = smem_desc_kmajor(a_addr, 128), b = smem_desc_kmajor(b_addr, 128);
+    const uint32_t idesc = instr_desc_bf16(n);
+    const long long t0 = clock64();
+    const uint32_t d1 = tmem + (uint32_t)n, d2 = tmem + 2u * (uint32_t)n;
+    if (unrolled) {
+      for (int r = 0; r < reps; ++r) {
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          tc_mma_bf16(tmem, a + 2 * ks, b + 2 * ks, idesc, 1);
+          if (accs >= 2) tc_mma_bf16(d1, a + 2 * ks, b + 2 * ks, idesc, 1);
+          if (accs >= 3) tc_mma_bf16(d2, a + 2 * ks, b + 2 * ks, idesc, 1);
+        }
+      }
+    } else {
+      for (int r = 0; r < reps; ++r)
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll 1
+          for (int q = 0; q < accs; ++q) tc_mma_bf16(tmem + (uint32_t)(q * n), a + 2 * ks, b + 2 * ks, idesc, 1);
+    }
+    const long long t1 = clock64();
+    tc_commit(&bar);
+    mbar_wait(&bar, 0, abort_flag);
+    const long long t2 = clock64();
+    if (blockIdx.x == 0) { out[0] = t1 - t0; out[1] = t2 - t0; }
+    if (*abort_flag && error_word) atomicExch(error_word, 1);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
 }
 
 // Flipped / transposed weight copy for the data gradient of a 3x3 convolution (taps = 9):
