@@ -41,12 +41,14 @@ typedef struct {
  *                  weight gradients of a 3x3 stride-2 layer run as the stride-1 tensor-core kernels on dy
  *                  spread onto the even pixels of the input grid (the call fills it); without it they
  *                  run on the CUDA cores.
- *   reduce         a per-channel reduction formed in the epilogue of the bf16 halo-tile kernel (3x3
- *                  layers whose stored tensor has 16, 32 or 64 channels), one row of 2*C floats per CTA in
- *                  `partial` (capacity `partial_floats` >= FDG_CONV_PARTIAL_ROWS*2*C); `nparts` receives
- *                  the number of rows, 0 if the shape took another kernel.  The consumer adds the rows in
- *                  row order (fdg_bn_apply / fdg_bn_backward with `partial`).
- *                    1 (fdg_conv_forward): sum y, sum y^2 over the stored y: the batch-norm statistics;
+ *   reduce         a per-channel reduction formed in the epilogue of the bf16 tensor-core kernels, one row of
+ *                  2*C floats per CTA in `partial` (capacity `partial_floats` >= FDG_CONV_PARTIAL_ROWS*2*C);
+ *                  `nparts` receives the number of rows, 0 if the shape took a kernel that forms none.  The
+ *                  consumer adds the rows in row order: fdg_bn_apply / fdg_bn_backward with `partial` (up to
+ *                  128 channels), or fdg_bn_stats_from_partials (any width).
+ *                    1 (fdg_conv_forward): sum y, sum y^2 over the stored y: the batch-norm statistics; the
+ *                      halo-tile kernel (3x3, stored tensor of 16, 32 or 64 channels) and the per-tap and
+ *                      patch-tile kernels of wider layers and of 1x1 shortcuts (up to 640 output channels);
  *                    2 (fdg_conv_dgrad):   sum dz, sum dz*xhat with dz = dx*[next_mask > 0] and
  *                      xhat = (next_x - mean)*invstd from next_stats[2*C]: the two sums of the batch-norm
  *                      backward that dx feeds (Eq. 9 applied to a normalisation layer). */
@@ -75,6 +77,12 @@ fdg_status fdg_conv_forward(int precision, const fdg_conv_shape* shape, const vo
 fdg_status fdg_conv_dgrad(int precision, const fdg_conv_shape* shape, const void* dy, const void* w,
                           const void* w_flipped, void* dx, const void* res, const void* res_mask,
                           fdg_conv_extra* extra, int* status_dev, fdg_stream stream);
+
+/* stats[0..C) = mean, stats[C..2C) = 1/sqrt(var + eps) from `nparts` rows of (sum, sum of squares) partial sums,
+ * partial[nparts][2*C], that a convolution with reduce = 1 left; `rows` = values per channel behind the sums.
+ * The rows are added in a fixed order (fp64).  Asynchronous on `stream`. */
+fdg_status fdg_bn_stats_from_partials(const float* partial, int nparts, size_t rows, int C, float eps, float* stats,
+                                      fdg_stream stream);
 
 /* Probe of the tensor pipe, for roofline arguments (no counterpart in the paper): on every SM one thread issues
  * reps * 4 * accumulators tcgen05.mma instructions (M = 128, N = n, K = 16, bf16, operands in shared memory) back to

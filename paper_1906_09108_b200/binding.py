@@ -31,7 +31,7 @@ EXPORTS = ["fdg_workspace_bytes", "fdg_create", "fdg_destroy", "fdg_param_count"
            "fdg_get_saved_tensor_of", "fdg_capture_bytes", "fdg_capture_begin", "fdg_capture_end", "fdg_get_captured",
            "fdg_bn_scratch_bytes", "fdg_bn_stats", "fdg_bn_apply", "fdg_bn_backward", "fdg_shrink", "fdg_sgd_update",
            "fdg_ingest", "fdg_head", "fdg_debug_raise_flag", "fdg_debug_wait_probe", "fdg_debug_guard_count", "fdg_debug_guard_offset",
-           "fdg_debug_check_guards", "fdg_probe_mma_rate", "fdg_lr_at", "fdg_set_lr_schedule", "fdg_bn_running_count",
+           "fdg_debug_check_guards", "fdg_probe_mma_rate", "fdg_bn_stats_from_partials", "fdg_lr_at", "fdg_set_lr_schedule", "fdg_bn_running_count",
            "fdg_get_bn_running", "fdg_set_bn_running", "fdg_eval", "fdg_drain", "fdg_state_bytes", "fdg_save_state",
            "fdg_load_state"]
 
@@ -125,6 +125,7 @@ def load_library(path=LIB_PATH):
         "fdg_conv_dgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, vp, vp, P(fdg_conv_extra), vp, vp],
         "fdg_conv_flip_weights": [P(fdg_conv_shape), vp, vp, vp],
         "fdg_probe_mma_rate": [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp],
+        "fdg_bn_stats_from_partials": [vp, C.c_int, C.c_size_t, C.c_int, C.c_float, vp, vp],
         "fdg_conv_wgrad_scratch_bytes": [C.c_int, P(fdg_conv_shape), P(sz)],
         "fdg_conv_wgrad": [C.c_int, P(fdg_conv_shape), vp, vp, vp, vp, sz, P(fdg_conv_extra), vp, vp],
         "fdg_get_saved_tensor_of": [vp, C.c_int, C.c_int, C.c_int, i64, vp, sz, P(sz), P(i64)],

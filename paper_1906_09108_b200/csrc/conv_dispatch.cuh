@@ -40,7 +40,8 @@ inline bool tc_eligible(const ConvGeom& g) {
 // counts (forward: Ci/Co; data gradient: Co/Ci with the flipped weight copy).
 inline cudaError_t run_conv_tc(cudaStream_t st, TensorMapCache* cache, int N, int H, int W, int Ck, int Cn,
                                const bf16_t* act, const bf16_t* wgt, bf16_t* out, const bf16_t* res,
-                               const bf16_t* res_mask, int* err_dev, int sub = 1, int taps = 9, int act_sub = 1) {
+                               const bf16_t* res_mask, int* err_dev, int sub = 1, int taps = 9, int act_sub = 1,
+                               float* stat_partial = nullptr, int* ctas_out = nullptr) {
   if (cache->sm_count == 0) {
     int dev = 0;
     cudaGetDevice(&dev);
@@ -61,7 +62,7 @@ inline cudaError_t run_conv_tc(cudaStream_t st, TensorMapCache* cache, int N, in
     ia = cache->maps.insert({ka, ma}).first;
     ib = cache->maps.insert({kb, mb}).first;
   }
-  return tc::conv_tc_launch(st, p, ia->second, ib->second, out, res, res_mask, err_dev, cache->sm_count);
+  return tc::conv_tc_launch(st, p, ia->second, ib->second, out, res, res_mask, err_dev, cache->sm_count, stat_partial, ctas_out);
 }
 
 
@@ -267,9 +268,31 @@ inline cudaError_t bf16_spread_dy(cudaStream_t st, const ConvGeom& g, const bf16
 
 // y = conv(x, w) [+ res].  `red` (mode 1) asks for the per-CTA sums of y and y^2; *nparts receives the number
 // of rows left in red->partial, 0 when the chosen kernel forms none.
+// Where the statistics of y go when a wide layer's kernel forms their partial sums (WideStats): `partial` holds one
+// row of 2 * Co floats per CTA; with `stats` set, the totals are finalised right behind the convolution (mean and
+// 1/sqrt(var + eps) over `rows` values per channel, running statistics included) and *nparts = -1 tells the caller
+// that nothing is left to do; without, *nparts = the rows left in `partial`.
+struct WideStats {
+  float* partial; size_t partial_floats;
+  float* stats; size_t rows; float eps;
+  float* running; float momentum;
+};
+inline bool wide_stats_ok(TensorMapCache* cache, const ConvGeom& g, const WideStats* ws) {
+  return ws && ws->partial && g.Co <= tc::kStatChunks * 16 && (size_t)cached_sm_count(cache) * 2 * g.Co <= ws->partial_floats;
+}
+inline cudaError_t finish_wide_stats(cudaStream_t st, const ConvGeom& g, const WideStats* ws, int ctas, int* nparts,
+                                     uint64_t* launches) {
+  if (!ws->stats) { if (nparts) *nparts = ctas; return cudaSuccess; }
+  const RunningStats run{ws->running, ws->momentum, ws->rows > 1 ? (float)((double)ws->rows / (double)(ws->rows - 1)) : 1.f};
+  ++*launches;
+  if (nparts) *nparts = -1;
+  return launch_chained(stats_finalize_kernel, dim3((unsigned)((g.Co + 31) / 32)), dim3(256), 0, st, (const float*)ws->partial, ctas,
+                        g.Co, 1.0 / (double)ws->rows, ws->eps, ws->stats, run);
+}
+
 inline cudaError_t bf16_conv_fprop(cudaStream_t st, TensorMapCache* cache, const ConvGeom& g, const bf16_t* x,
                                    const bf16_t* w, bf16_t* y, const bf16_t* res, const halo::EpiReduce* red, int* nparts,
-                                   int* err_dev, uint64_t* launches) {
+                                   int* err_dev, uint64_t* launches, const WideStats* ws = nullptr) {
   if (nparts) *nparts = 0;
   const bool s1 = halo_fprop_eligible(g), s2 = !s1 && halo_s2_fprop_eligible(g);
   if (s1 || s2) {
@@ -282,10 +305,20 @@ inline cudaError_t bf16_conv_fprop(cudaStream_t st, TensorMapCache* cache, const
   }
   if (tc_eligible(g) || tc_s2_fprop_eligible(g)) {
     ++*launches;
+    if (wide_stats_ok(cache, g, ws)) {
+      int ctas = 0;
+      const cudaError_t e = run_conv_tc(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, err_dev, g.stride, 9, 1, ws->partial, &ctas);
+      return e != cudaSuccess ? e : finish_wide_stats(st, g, ws, ctas, nparts, launches);
+    }
     return run_conv_tc(st, cache, g.N, g.H, g.W, g.Ci, g.Co, x, w, y, res, nullptr, err_dev, g.stride);
   }
   if (tc_1x1_fprop_eligible(g)) {
     ++*launches;
+    if (wide_stats_ok(cache, g, ws)) {
+      int ctas = 0;
+      const cudaError_t e = run_conv_tc(st, cache, g.N, g.P, g.Q, g.Ci, g.Co, x, w, y, res, nullptr, err_dev, 1, 1, g.stride, ws->partial, &ctas);
+      return e != cudaSuccess ? e : finish_wide_stats(st, g, ws, ctas, nparts, launches);
+    }
     return run_conv_tc(st, cache, g.N, g.P, g.Q, g.Ci, g.Co, x, w, y, res, nullptr, err_dev, 1, 1, g.stride);
   }
   return launch_conv_simt<bf16_t, CONV_FPROP>(st, g, x, w, y, nullptr, nullptr, res, (const bf16_t*)nullptr, launches);

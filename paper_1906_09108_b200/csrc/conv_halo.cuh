@@ -113,20 +113,6 @@ constexpr int kConvMmaWarps = 4;
 constexpr int kConvFirstEpiWarp = kConvMmaWarps;
 constexpr int kConvThreads = 32 * (kConvFirstEpiWarp + kEpiWarps);
 
-// 32 lanes each hold 32 items; afterwards lane l holds in q[0] the sum over all lanes of item l.
-__device__ __forceinline__ void transpose_reduce32(float (&q)[32], int lane) {
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) {
-    const bool upper = (lane & off) != 0;
-#pragma unroll
-    for (int i = 0; i < off; ++i) {
-      const float send = upper ? q[i] : q[i + off];
-      const float keep = upper ? q[i + off] : q[i];
-      q[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-    }
-  }
-}
-
 // The 9 * KS instructions of one 128-row tile, fully unrolled (the issuing thread is the
 // bottleneck: every instruction it spends per tcgen05.mma beyond the add and the issue shows).
 template <int KS>

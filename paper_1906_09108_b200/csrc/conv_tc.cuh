@@ -54,6 +54,8 @@ struct ConvTcParams {
   int patch;                // 1: conv3x3_patch_kernel (16x16-pixel patches with their halo), 0: conv3x3_tc_kernel
   uint32_t halo_bytes;      // patch mode: shared memory of one 18x18-pixel halo tile of kc channels (multiple of 1 KiB)
   int b_stages;             // patch mode: weight tiles in flight
+  int acc_slots;            // patch mode: accumulators of n_tile columns the 128-row tiles rotate over (3 where tensor
+                            // memory holds them: the write-out of a tile then runs beside the next tiles' instructions)
 };
 constexpr int kPatch = 16;                         // patch side in pixels
 constexpr int kPatchHalo = kPatch + 2;             // with the one-pixel border
@@ -176,12 +178,58 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 }
 
+// 32 lanes each hold 32 items; afterwards lane l holds in q[0] the sum over all lanes of item l.
+__device__ __forceinline__ void transpose_reduce32(float (&q)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < off; ++i) {
+      const float send = upper ? q[i] : q[i + off];
+      const float keep = upper ? q[i + off] : q[i];
+      q[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+}
+
+// Batch-norm statistics of the output, formed in the epilogue (optional): every epilogue warp adds, per 16-channel
+// chunk, the sums of the values it stores and of their squares over its 32 rows into its own array in shared
+// memory; at the end the CTA writes one row stat_partial[blockIdx.x][2][Co] (sum, sum of squares), which
+// stats_finalize_kernel adds over the CTAs in CTA order.  Up to kStatChunks * 16 output channels.
+constexpr int kStatChunks = 40;
+constexpr int kStatFloats = 4 * kStatChunks * 32;
+__device__ __forceinline__ void stat_add(float* stat_run, int ew, int chunk, const uint4& o0, const uint4& o1, int lane) {
+  const __nv_bfloat16* sb0 = reinterpret_cast<const __nv_bfloat16*>(&o0);
+  const __nv_bfloat16* sb1 = reinterpret_cast<const __nv_bfloat16*>(&o1);
+  float q[32];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const float a = __bfloat162float(sb0[e]), b = __bfloat162float(sb1[e]);      // the values as stored
+    q[e] = a; q[8 + e] = b; q[16 + e] = a * a; q[24 + e] = b * b;
+  }
+  transpose_reduce32(q, lane);
+  stat_run[(ew * kStatChunks + chunk) * 32 + lane] += q[0];
+}
+// The CTA's row of partial sums (after all epilogue warps are done).
+__device__ __forceinline__ void stat_flush(const float* stat_run, float* __restrict__ stat_partial, int Co) {
+  for (int t = threadIdx.x; t < 2 * Co; t += blockDim.x) {
+    const int stat = t / Co, c = t - stat * Co;
+    const int idx = (c >> 4) * 32 + (c & 15) + 16 * stat;
+    float a = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) a += stat_run[w * kStatChunks * 32 + idx];
+    stat_partial[(size_t)blockIdx.x * 2 * Co + t] = a;
+  }
+}
+
 // ------------------------------------------------------------------- kernel ----
 // out[m][n] (bf16, row stride Co) = conv + (res ? res[m][n] * [mask ? mask[m][n] > 0 : 1] : 0)
 __global__ void __launch_bounds__(kThreads, 1)
 conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   ConvTcParams p, __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
-                  const __nv_bfloat16* __restrict__ res_mask, int* __restrict__ error_word) {
+                  const __nv_bfloat16* __restrict__ res_mask, float* __restrict__ stat_partial, int* __restrict__ error_word) {
+  __shared__ float stat_run[kStatFloats];
+  if (stat_partial) for (int i = threadIdx.x; i < kStatFloats; i += blockDim.x) stat_run[i] = 0.f;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * p.stage_bytes);
@@ -323,11 +371,11 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         uint32_t v[16];
         tmem_ld16(taddr + c0, v);
         tmem_ld_wait();
-        if (!keep) continue;
+        if (!keep && !stat_partial) continue;
         float f[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) f[i] = __uint_as_float(v[i]);
-        if (res) {
+        if (res && keep) {
           uint4 r0 = *reinterpret_cast<const uint4*>(res + base + c0);
           uint4 r1 = *reinterpret_cast<const uint4*>(res + base + c0 + 8);
           const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
@@ -357,8 +405,13 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           ob0[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
           ob1[i] = __floats2bfloat162_rn(f[8 + 2 * i], f[8 + 2 * i + 1]);
         }
-        *reinterpret_cast<uint4*>(out + base + c0) = o0;
-        *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+        if (keep) {
+          *reinterpret_cast<uint4*>(out + base + c0) = o0;
+          *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+        } else {
+          o0 = o1 = make_uint4(0, 0, 0, 0);
+        }
+        if (stat_partial) stat_add(stat_run, ew, (nt * p.n_tile + c0) >> 4, o0, o1, lane);
       }
       }
       tc_fence_before();
@@ -384,6 +437,7 @@ conv3x3_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     tc_fence_after();
     tmem_dealloc(tmem_base, p.tmem_cols);
   }
+  if (stat_partial && !*abort_flag) stat_flush(stat_run, stat_partial, p.Co);
 }
 
 // ------------------------------------------------------- patch-tile kernel ----
@@ -402,7 +456,9 @@ constexpr int kPatchThreads = 224;       // TMA warp, issuing warp of tile 0, fo
 __global__ void __launch_bounds__(kPatchThreads, 1)
 conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      ConvTcParams p, __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ res,
-                     const __nv_bfloat16* __restrict__ res_mask, int* __restrict__ error_word) {
+                     const __nv_bfloat16* __restrict__ res_mask, float* __restrict__ stat_partial, int* __restrict__ error_word) {
+  __shared__ float stat_run[kStatFloats];
+  if (stat_partial) for (int i = threadIdx.x; i < kStatFloats; i += blockDim.x) stat_run[i] = 0.f;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* b_smem = smem + 2 * (size_t)p.halo_bytes;
@@ -411,17 +467,16 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   uint64_t* a_empty = a_full + 2;              // [2]         MMA -> TMA
   uint64_t* full = a_empty + 2;                // [b_stages]  TMA -> MMA, weight tiles
   uint64_t* empty = full + p.b_stages;         // [b_stages]  MMA -> TMA
-  uint64_t* acc_full = empty + p.b_stages;     // [1]         MMA -> epilogue
-  uint64_t* acc_empty = acc_full + 1;          // [1]         epilogue -> MMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+  uint64_t* acc_full = empty + p.b_stages;     // [3]         MMA -> epilogue, one per accumulator slot
+  uint64_t* acc_empty = acc_full + 3;          // [3]         epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 3);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) { mbar_init(&a_full[s], 1); mbar_init(&a_empty[s], 2); }
     for (int s = 0; s < p.b_stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 2); }
-    mbar_init(acc_full, 2);
-    mbar_init(acc_empty, 4);
+    for (int a = 0; a < 3; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -488,14 +543,17 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 #pragma unroll
       for (int tap = 0; tap < 9; ++tap) tap_off[tap] = (uint64_t)(((tap / 3) * kPatchHalo + (tap % 3)) * row_bytes) >> 4;
       const uint64_t g_off = (uint64_t)(8 * g * row_bytes) >> 4;
-      const uint32_t d_tmem = tmem_base + (uint32_t)(g * p.n_tile);
+      // The 128-row tiles of this CTA, numbered 2 * (patch count) + g, rotate over the accumulator slots.
       uint32_t q = 0, itb = 0, tcount = 0;
       int s = 0;
       uint32_t ph = 0;                                         // itb % b_stages and that stage's phase, kept incrementally
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles && !*abort_flag; tile += gridDim.x, ++tcount) {
-        if (!mbar_wait(acc_empty, (tcount & 1) ^ 1, abort_flag)) break;
+        const uint32_t half = 2 * tcount + (uint32_t)g;
+        const uint32_t slot = half % (uint32_t)p.acc_slots, use = half / (uint32_t)p.acc_slots;
+        if (!mbar_wait(&acc_empty[slot], (use & 1) ^ 1, abort_flag)) break;
         tc_fence_after();
+        const uint32_t d_tmem = tmem_base + slot * (uint32_t)p.n_tile;
         for (int cc = 0; ok && cc < chunks; ++cc, ++q) {
           const int sa = q & 1;
           if (!mbar_wait(&a_full[sa], (q >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -514,7 +572,7 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           }
           if (ok) tc_commit(&a_empty[sa]);
         }
-        if (ok) tc_commit(acc_full);
+        if (ok) tc_commit(&acc_full[slot]);
       }
     }
   } else if (warp >= 2 && warp <= 5) {
@@ -524,10 +582,13 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       const int pt = tile / p.n_tiles, nt = tile - pt * p.n_tiles;
       const int n = pt / (ph_cnt * pw_cnt), rem = pt - n * ph_cnt * pw_cnt;
       const int ph = rem / pw_cnt, pw = rem - ph * pw_cnt;
-      if (!mbar_wait(acc_full, tcount & 1, abort_flag)) break;
-      tc_fence_after();
       const int i = lane_grp * 32 + lane;                       // accumulator row of this thread
+      bool live = true;
       for (int g = 0; g < 2; ++g) {
+        const uint32_t half = 2 * tcount + (uint32_t)g;
+        const uint32_t slot = half % (uint32_t)p.acc_slots, use = half / (uint32_t)p.acc_slots;
+        if (!mbar_wait(&acc_full[slot], use & 1, abort_flag)) { live = false; break; }
+        tc_fence_after();
         const int h = ph * kPatch + (i >> 3), w = pw * kPatch + 8 * g + (i & 7);
         size_t base;
         bool keep = true;
@@ -537,16 +598,16 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           keep = ((h | w) & 1) == 0;
           base = (((size_t)n * (p.H >> 1) + (h >> 1)) * (p.W >> 1) + (w >> 1)) * p.Co + (size_t)nt * p.n_tile;
         }
-        const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)g * p.n_tile;
+        const uint32_t taddr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + slot * (uint32_t)p.n_tile;
         for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
           uint32_t v[16];
           tmem_ld16(taddr + c0, v);
           tmem_ld_wait();
-          if (!keep) continue;
+          if (!keep && !stat_partial) continue;
           float f[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]);
-          if (res) {
+          if (res && keep) {
             uint4 r0 = *reinterpret_cast<const uint4*>(res + base + c0);
             uint4 r1 = *reinterpret_cast<const uint4*>(res + base + c0 + 8);
             const __nv_bfloat16* rb0 = reinterpret_cast<const __nv_bfloat16*>(&r0);
@@ -576,13 +637,19 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             ob0[e] = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
             ob1[e] = __floats2bfloat162_rn(f[8 + 2 * e], f[8 + 2 * e + 1]);
           }
-          *reinterpret_cast<uint4*>(out + base + c0) = o0;
-          *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+          if (keep) {
+            *reinterpret_cast<uint4*>(out + base + c0) = o0;
+            *reinterpret_cast<uint4*>(out + base + c0 + 8) = o1;
+          } else {
+            o0 = o1 = make_uint4(0, 0, 0, 0);
+          }
+          if (stat_partial) stat_add(stat_run, warp - 2, (nt * p.n_tile + c0) >> 4, o0, o1, lane);
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[slot]);            // this tile's accumulator may be overwritten
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty);
+      if (!live) break;
     }
   }
 
@@ -603,6 +670,7 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     tc_fence_after();
     tmem_dealloc(tmem_base, p.tmem_cols);
   }
+  if (stat_partial && !*abort_flag) stat_flush(stat_run, stat_partial, p.Co);
 }
 
 // ----------------------------------------------------------------- host side ---
@@ -677,14 +745,15 @@ inline ConvTcParams conv_tc_params(int N, int H, int W, int Ci, int Co, int taps
   if (p.b_stages < 2) p.patch = 0;
   int stages = (int)(160 * 1024 / p.stage_bytes);
   p.stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
+  p.acc_slots = (p.patch && 3 * nt <= 512) ? 3 : 2;
   uint32_t cols = 32;
-  while (cols < 2u * nt) cols <<= 1;
+  while (cols < (uint32_t)(p.patch ? p.acc_slots : 2) * nt) cols <<= 1;
   p.tmem_cols = cols;
   return p;
 }
 
 inline size_t conv_tc_smem_bytes(const ConvTcParams& p) {
-  if (p.patch) return 2 * (size_t)p.halo_bytes + (size_t)p.b_stages * p.b_bytes + 1024 + 256;
+  if (p.patch) return 2 * (size_t)p.halo_bytes + (size_t)p.b_stages * p.b_bytes + 1024 + 256 + 64;
   return (size_t)p.stages * p.stage_bytes + 1024 + 256;
 }
 
@@ -732,9 +801,11 @@ inline cudaError_t conv_tc_set_attrs() {
   return e;
 }
 
+// `stat_partial` (nullable): room for one row of 2 * Co floats per CTA (at most sm_count rows); *ctas_out = rows written.
 inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const CUtensorMap& map_a,
                                   const CUtensorMap& map_b, __nv_bfloat16* out, const __nv_bfloat16* res,
-                                  const __nv_bfloat16* res_mask, int* error_word, int sm_count) {
+                                  const __nv_bfloat16* res_mask, int* error_word, int sm_count,
+                                  float* stat_partial = nullptr, int* ctas_out = nullptr) {
   const size_t smem = conv_tc_smem_bytes(p);
   {
     cudaError_t e = conv_tc_set_attrs();
@@ -743,12 +814,14 @@ inline cudaError_t conv_tc_launch(cudaStream_t st, const ConvTcParams& p, const 
   if (p.patch) {
     const int tiles = p.N * (p.H / kPatch) * (p.W / kPatch) * p.n_tiles;
     const int grid = tiles < sm_count ? tiles : sm_count;
-    conv3x3_patch_kernel<<<grid, kPatchThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, error_word);
+    if (ctas_out) *ctas_out = grid;
+    conv3x3_patch_kernel<<<grid, kPatchThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, stat_partial, error_word);
     return cudaGetLastError();
   }
   const int tiles = ((p.m_tiles + p.mpair - 1) / p.mpair) * p.n_tiles;
   const int grid = tiles < sm_count ? tiles : sm_count;
-  conv3x3_tc_kernel<<<grid, kThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, error_word);
+  if (ctas_out) *ctas_out = grid;
+  conv3x3_tc_kernel<<<grid, kThreads, smem, st>>>(map_a, map_b, p, out, res, res_mask, stat_partial, error_word);
   return cudaGetLastError();
 }
 

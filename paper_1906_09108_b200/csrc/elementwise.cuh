@@ -244,6 +244,36 @@ bn_stats_kernel(const T* __restrict__ x, RedGeom g, float eps, float* __restrict
       });
 }
 
+// Statistics from the rows of partial sums a wide convolution's epilogue left: partial[nparts][2][C] (sum, sum of
+// squares per CTA) -> stats[0..C) = mean, stats[C..2C) = 1/sqrt(var + eps), and the running statistics.  A block
+// takes 32 channels; its 8 warps take every 8th row, their sums are added in warp order (fp64).
+__global__ void __launch_bounds__(256) stats_finalize_kernel(const float* __restrict__ partial, int nparts, int C, double inv_count,
+                                                             float eps, float* __restrict__ stats, RunningStats run) {
+  grid_dependency_wait();                   // launched ahead of the end of the convolution that writes `partial`
+  __shared__ double fin[2][8][32];
+  const int lane = threadIdx.x & 31, seg = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
+  double s = 0.0, ss = 0.0;
+  if (c < C)
+    for (int r = seg; r < nparts; r += 8) {
+      s += (double)partial[(size_t)r * 2 * C + c];
+      ss += (double)partial[(size_t)r * 2 * C + C + c];
+    }
+  fin[0][seg][lane] = s; fin[1][seg][lane] = ss;
+  __syncthreads();
+  if (seg == 0 && c < C) {
+    double a = 0.0, b = 0.0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) { a += fin[0][q][lane]; b += fin[1][q][lane]; }
+    const double mean = a * inv_count;
+    double var = b * inv_count - mean * mean;
+    if (var < 0.0) var = 0.0;
+    stats[c] = (float)mean;
+    stats[C + c] = (float)(1.0 / sqrt(var + (double)eps));
+    if (run.running) update_running(run, C, c, (float)mean, (float)var);
+  }
+}
+
 // Per-CTA partial sums left by a convolution epilogue, partial[nparts][2*C], to be added up by
 // the kernel that consumes the totals (every block does it for itself: the partials are a few KB
 // and sit in L2).  Fixed order: kEwThreads / (2C) threads share a (sum, channel) pair, each taking

@@ -105,6 +105,7 @@ struct Module {
   char* up = nullptr;                      // dy of a stride-2 convolution spread onto the input's pixel grid
   size_t up_elems = 0;
   float* red_partial = nullptr;            // per-CTA partial sums of the reductions fused into convolution epilogues
+  size_t red_partial_floats = 0;
   unsigned int* red_counter = nullptr;
   float *pooled = nullptr, *dlogits = nullptr, *loss_n = nullptr, *loss = nullptr;   // head
   // host state
@@ -513,7 +514,12 @@ static size_t carve(fdg_ctx* c, char* base) {
     m.bnsums = cv.take<float>((size_t)kRedMaxSums * maxc * 4);
     m.counter = cv.take<unsigned int>(256);
     m.up = m.up_elems ? cv.take<char>(align_up(m.up_elems, 128) * es) : nullptr;
-    m.red_partial = cv.take<float>((size_t)kRedPartialCtas * 2 * 64 * 4);
+    {
+      int widest = 64;                        // rows of 2 * C floats: narrow layers up to 64 channels, wide ones up to 640
+      for (const Unit& u : m.units) if (u.type != U_HEAD && u.co <= tc::kStatChunks * 16) widest = std::max(widest, u.co);
+      m.red_partial_floats = (size_t)kRedPartialCtas * 2 * widest;
+      m.red_partial = cv.take<float>(m.red_partial_floats * 4);
+    }
     m.red_counter = cv.take<unsigned int>(256);
     if (m.k == c->K) {
       const Unit& h = m.units.back();
@@ -576,6 +582,7 @@ template <typename T>
 static void bn_apply(Launch& L, Module& m, const T* x, float* stats, const float* gamma, const float* beta, const T* res,
                      const float* res_stats, const float* res_gamma, const float* res_beta, bool relu, T* y,
                      size_t rows, int C, int nparts = 0, long long run = -1) {
+  if (nparts < 0) nparts = 0;               // the statistics were finalised behind the convolution
   const size_t n = rows * C;
   L.begin(KC_BN_APPLY, (double)n * sizeof(T) * (res ? 3 : 2), 6.0 * n);
   L.note(launch_bn_apply<T>(L.st, x, stats, gamma, beta, res, res_stats, res_gamma, res_beta, relu, y, rows, C,
@@ -630,14 +637,20 @@ static double w_elems(const ConvGeom& g) { return (double)g.Co * g.R * g.S * g.C
 // sums (sum y, sum y^2) the convolution kernel left in m.red_partial from its epilogue, or 0 when it
 // left none and the caller has to run bn_stats.
 template <typename T>
+// Returns the rows of partial sums the kernel left in m.red_partial for the batch norm that follows (`want_stats`;
+// a narrow layer), 0 when it formed none, or -1 when the statistics are already in `stats` (a wide layer, whose
+// totals are finalised right behind the convolution; needs `stats`, with `run` the running statistics' offset or -1).
 static int conv_fprop(Launch& L, Module& m, const ConvGeom& g, const T* x, const T* w, T* y, const T* res,
-                      bool want_stats = false) {
+                      bool want_stats = false, float* stats = nullptr, long long run = -1) {
   L.begin(KC_CONV_FPROP, (in_elems(g) + w_elems(g) + out_elems(g) * (res ? 2 : 1)) * sizeof(T), conv_flops(g));
   int nparts = 0;
   if constexpr (std::is_same<T, bf16>::value) {
     halo::EpiReduce r{};
     r.mode = 1; r.partial = m.red_partial;
-    L.note(bf16_conv_fprop(L.st, &L.c->tmaps, g, x, w, y, res, want_stats ? &r : nullptr, &nparts, L.c->tc_error, &L.c->launches));
+    const WideStats ws{m.red_partial, m.red_partial_floats, stats, (size_t)g.N * g.P * g.Q, L.c->arch.bn_eps,
+                       run >= 0 ? m.running + run : nullptr, kBnMomentum};
+    L.note(bf16_conv_fprop(L.st, &L.c->tmaps, g, x, w, y, res, want_stats ? &r : nullptr, &nparts, L.c->tc_error, &L.c->launches,
+                           (want_stats && stats) ? &ws : nullptr));
   } else {
     L.note(launch_conv_simt<T, CONV_FPROP>(L.st, g, x, w, y, nullptr, nullptr, res, (const T*)nullptr, &L.c->launches));
   }
@@ -723,7 +736,7 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
   T* tmp = reinterpret_cast<T*>(m.temps[2]);
   // statistics of a convolution output y that left `np` rows of partial sums (0: reduce y now)
   auto stats_of = [&](int np, const T* y, size_t rows, int C, float* stats, long long run) {
-    if (!eval && !np) bn_stats<T>(L, m, y, rows, C, eps, stats, run);
+    if (!eval && np == 0) bn_stats<T>(L, m, y, rows, C, eps, stats, run);
   };
   for (const Unit& u : m.units) {
     const size_t rows_in = (size_t)B * u.H * u.W, rows_out = (size_t)B * u.P * u.Q;
@@ -731,7 +744,7 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
       case U_STEM: {
         ConvGeom g = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, 1, 1);
         if (u.bn) {
-          const int np = conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_a, nullptr, !eval);
+          const int np = conv_fprop<T>(L, m, g, x, wt + u.w1, S + u.t_a, nullptr, !eval, F + u.st1, u.r1);
           stats_of(np, S + u.t_a, rows_out, u.co, F + u.st1, u.r1);
           bn_apply<T>(L, m, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_y, rows_out, u.co, np, u.r1);
         } else {
@@ -742,15 +755,15 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
       case U_BASIC: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
-        const int np1 = conv_fprop<T>(L, m, g1, x, wt + u.w1, S + u.t_a, nullptr, !eval);               // c1
+        const int np1 = conv_fprop<T>(L, m, g1, x, wt + u.w1, S + u.t_a, nullptr, !eval, F + u.st1, u.r1);   // c1
         stats_of(np1, S + u.t_a, rows_out, u.co, F + u.st1, u.r1);
         bn_apply<T>(L, m, S + u.t_a, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_b, rows_out, u.co, np1, u.r1);  // a1
         if (u.proj) {          // shortcut first: its statistics must not disturb the partial sums conv2 leaves for BN2
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
-          conv_fprop<T>(L, m, gs, x, wt + u.ws, S + u.t_s, nullptr);                                   // cs
-          stats_of(0, S + u.t_s, rows_out, u.co, F + u.sts, u.rs);
+          const int nps = conv_fprop<T>(L, m, gs, x, wt + u.ws, S + u.t_s, nullptr, !eval, F + u.sts, u.rs);   // cs
+          stats_of(nps < 0 ? nps : 0, S + u.t_s, rows_out, u.co, F + u.sts, u.rs);
         }
-        const int np2 = conv_fprop<T>(L, m, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr, !eval);       // c2
+        const int np2 = conv_fprop<T>(L, m, g2, S + u.t_b, wt + u.w2, S + u.t_c, nullptr, !eval, F + u.st2, u.r2);   // c2
         stats_of(np2, S + u.t_c, rows_out, u.co, F + u.st2, u.r2);
         if (u.proj) {
           bn_apply<T>(L, m, S + u.t_c, F + u.st2, wf + u.g2, wf + u.b2, S + u.t_s, F + u.sts, wf + u.gs, wf + u.bs, true, S + u.t_y, rows_out, u.co, np2, u.r2);
@@ -769,7 +782,7 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
         stats_of(0, x, rows_in, u.ci, F + u.st1, u.r1);
         bn_apply<T>(L, m, x, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows_in, u.ci);   // o
-        const int np = conv_fprop<T>(L, m, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr, !eval);        // c1
+        const int np = conv_fprop<T>(L, m, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr, !eval, F + u.st2, u.r2);   // c1
         stats_of(np, S + u.t_b, rows_out, u.co, F + u.st2, u.r2);
         bn_apply<T>(L, m, S + u.t_b, F + u.st2, wf + u.g2, wf + u.b2, nullptr, nullptr, nullptr, nullptr, true, S + u.t_c, rows_out, u.co, np, u.r2); // a2
         if (u.proj) {

@@ -148,6 +148,43 @@ def test_conv_forward_with_fused_statistics(shape, with_res):
     assert _rel(a, L.relu_forward(L.batchnorm_forward(ys, gam, beta, EPS)[0])) <= 1e-2
 
 
+# (N, H, W, Ci, Co, R, stride): the wide layers' kernels -- patch tiles (16x16 and 32x32 images), per-tap tiles (8x8, also
+# with narrowed column tiles), a strided 3x3 layer computed at full resolution, 1x1 shortcuts of both strides
+WIDE_FUSED_SHAPES = [(6, 16, 16, 320, 320, 3, 1), (3, 32, 32, 160, 160, 3, 1), (16, 8, 8, 640, 640, 3, 1),
+                     (4, 32, 32, 160, 320, 3, 2), (32, 8, 8, 256, 256, 3, 1), (4, 32, 32, 160, 320, 1, 2),
+                     (2, 32, 32, 16, 160, 1, 1)]
+
+
+@pytest.mark.parametrize("shape", WIDE_FUSED_SHAPES)
+@pytest.mark.parametrize("with_res", [False, True])
+def test_wide_conv_forward_with_fused_statistics(shape, with_res):
+    """fdg_conv_forward with reduce = 1 on the wide layers' kernels, then fdg_bn_stats_from_partials: the
+    convolution output, the summed rows against the stored output, and the statistics derived from them."""
+    from paper_1906_09108_b200 import binding as B
+    n, h, w, ci, co, r, stride = shape
+    ops = B.ConvOps(B.FDG_BF16_TC)
+    s = B.fdg_conv_shape(n, h, w, ci, co, r, stride, 1 if r == 3 else 0)
+    p, q = ops.out_hw(s)
+    x, xo = _mk((n, h, w, ci), 41, ops.dtype)
+    wt, wo = _mk((co, r, r, ci), 42, ops.dtype, scale=(2.0 / (r * r * ci)) ** 0.5)
+    res, reso = _mk((n, p, q, co), 43, ops.dtype)
+    y, part = ops.forward(s, x, wt, res=res if with_res else None, reduce=True)
+    assert part.shape[0] >= 1 and not ops.timed_out()
+    yo = L.conv2d_forward(xo, wo, stride, 1 if r == 3 else 0) + (reso if with_res else 0.0)
+    assert _rel(y, yo) <= 1e-2
+    ys = y.float().cpu().numpy().astype(np.float64)                 # the sums are taken over the stored values
+    tot = part.double().sum(dim=0).cpu().numpy()
+    assert np.abs(tot[:co] - ys.sum(axis=(0, 1, 2))).max() <= 1e-4 * np.abs(ys).sum(axis=(0, 1, 2)).max()
+    assert _rel(tot[co:], (ys * ys).sum(axis=(0, 1, 2))) <= 1e-5
+    stats = torch.full((2 * co,), float("nan"), dtype=torch.float32, device="cuda")
+    rc = ops.lib.fdg_bn_stats_from_partials(part.data_ptr(), part.shape[0], n * p * q, co, EPS, stats.data_ptr(),
+                                            torch.cuda.current_stream().cuda_stream)
+    assert rc == B.FDG_OK
+    mean, invstd = _stats_ref(ys)
+    assert np.abs(stats[:co].cpu().numpy() - mean).max() <= 1e-5 * max(np.abs(ys).max(), 1.0)
+    assert _rel(stats[co:], invstd) <= 1e-5
+
+
 @pytest.mark.parametrize("shape", FUSED_SHAPES)
 @pytest.mark.parametrize("with_res", [False, True])
 def test_conv_dgrad_with_fused_bn_backward_sums(shape, with_res):
