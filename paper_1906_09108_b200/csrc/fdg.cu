@@ -738,7 +738,11 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
   auto stats_of = [&](int np, const T* y, size_t rows, int C, float* stats, long long run) {
     if (!eval && np == 0) bn_stats<T>(L, m, y, rows, C, eps, stats, run);
   };
-  for (const Unit& u : m.units) {
+  int x_np = 0;     // -1: the statistics of x (the next pre-activation block's first batch norm) are already in place
+  for (size_t ui = 0; ui < m.units.size(); ++ui) {
+    const Unit& u = m.units[ui];
+    // the pre-activation block that normalises this unit's output first, if it is in this module
+    const Unit* nxt = (ui + 1 < m.units.size() && m.units[ui + 1].type == U_PREACT) ? &m.units[ui + 1] : nullptr;
     const size_t rows_in = (size_t)B * u.H * u.W, rows_out = (size_t)B * u.P * u.Q;
     switch (u.type) {
       case U_STEM: {
@@ -780,7 +784,8 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
       case U_PREACT: {
         ConvGeom g1 = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 3, u.stride, 1);
         ConvGeom g2 = geom(B, u.P, u.Q, u.co, u.P, u.Q, u.co, 3, 1, 1);
-        stats_of(0, x, rows_in, u.ci, F + u.st1, u.r1);
+        stats_of(x_np, x, rows_in, u.ci, F + u.st1, u.r1);
+        x_np = 0;
         bn_apply<T>(L, m, x, F + u.st1, wf + u.g1, wf + u.b1, nullptr, nullptr, nullptr, nullptr, true, S + u.t_a, rows_in, u.ci);   // o
         const int np = conv_fprop<T>(L, m, g1, S + u.t_a, wt + u.w1, S + u.t_b, nullptr, !eval, F + u.st2, u.r2);   // c1
         stats_of(np, S + u.t_b, rows_out, u.co, F + u.st2, u.r2);
@@ -788,10 +793,11 @@ static void forward_module(fdg_ctx* c, Module& m, Launch& L, int64_t tau, int sl
         if (u.proj) {
           ConvGeom gs = geom(B, u.H, u.W, u.ci, u.P, u.Q, u.co, 1, u.stride, 0);
           conv_fprop<T>(L, m, gs, S + u.t_a, wt + u.ws, tmp, nullptr);
-          conv_fprop<T>(L, m, g2, S + u.t_c, wt + u.w2, S + u.t_y, tmp);
+          x_np = conv_fprop<T>(L, m, g2, S + u.t_c, wt + u.w2, S + u.t_y, tmp, !eval && nxt, nxt ? F + nxt->st1 : nullptr, nxt ? nxt->r1 : -1);
         } else {
-          conv_fprop<T>(L, m, g2, S + u.t_c, wt + u.w2, S + u.t_y, x);
+          x_np = conv_fprop<T>(L, m, g2, S + u.t_c, wt + u.w2, S + u.t_y, x, !eval && nxt, nxt ? F + nxt->st1 : nullptr, nxt ? nxt->r1 : -1);
         }
+        if (x_np > 0) x_np = 0;     // rows for a narrow layer's apply kernel: not used here, the block's input is reduced as before
         break;
       }
       case U_HEAD:
