@@ -593,6 +593,9 @@ def run_gpu(args):
             u2, b2, f2 = kernel_bench(B, "fprop", "wrn_stage2", launches=16)
             iso["fprop_wrn_stage2"] = dict(us=u2, tflops=f2 / u2 / 1e6, frac_tensor=f2 / u2 / 1e6 / peaks["bf16_tflops"],
                                            kernel="conv3x3_patch_kernel, [128,16,16,320] -> 320 channels")
+            u2, b2, f2 = kernel_bench(B, "wgrad", "wrn_stage2", launches=16)
+            iso["wgrad_wrn_stage2"] = dict(us=u2, tflops=f2 / u2 / 1e6, frac_tensor=f2 / u2 / 1e6 / peaks["bf16_tflops"],
+                                           kernel="wgrad_wide_kernel + wgrad_wide_sum_kernel, x and dy [128,16,16,320]")
             roof["isolated"] = iso
         elif top["name"].startswith("conv"):
             # fp32 FMA peak: 148 SMs x 128 lanes x 2 flop x max SM clock

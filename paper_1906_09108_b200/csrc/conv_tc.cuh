@@ -558,6 +558,8 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           const int sa = q & 1;
           if (!mbar_wait(&a_full[sa], (q >> 1) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
+          // the last chunk of a 160-channel layer holds 32 channels (the rest of its 64 is the zero fill): two K steps
+          const bool short_chunk = cc == chunks - 1 && (p.Ci & 63) != 0 && (p.Ci & 63) <= 32;
 #pragma unroll
           for (int tap = 0; tap < 9; ++tap, ++itb) {
             if (!mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
@@ -565,8 +567,10 @@ conv3x3_patch_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const uint64_t a0 = halo_desc[sa] + tap_off[tap] + g_off, b0 = b_desc[s];
             tc_mma_bf16(d_tmem, a0, b0, idesc, (uint32_t)(cc | tap));
             tc_mma_bf16(d_tmem, a0 + 2, b0 + 2, idesc, 1);
-            tc_mma_bf16(d_tmem, a0 + 4, b0 + 4, idesc, 1);
-            tc_mma_bf16(d_tmem, a0 + 6, b0 + 6, idesc, 1);
+            if (!short_chunk) {
+              tc_mma_bf16(d_tmem, a0 + 4, b0 + 4, idesc, 1);
+              tc_mma_bf16(d_tmem, a0 + 6, b0 + 6, idesc, 1);
+            }
             tc_commit(&empty[s]);
             if (++s == p.b_stages) { s = 0; ph ^= 1; }
           }
