@@ -26,6 +26,8 @@
  *     fdg_destroy().
  *   - Activations are NHWC; convolution weights are [C_out][R][S][C_in].
  *   - Modules and blocks are numbered from 1 as in the paper.
+ *   - Threading: a context is used by one host thread at a time (its calls enqueue work on its streams and
+ *     update host-side bookkeeping without a lock); different contexts may be used from different threads.
  *
  * Flat parameter layout of a module (fp32), the order fdg_param_layout() reports:
  *   units in network order: stem (module 1), residual blocks, head (module K);
