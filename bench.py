@@ -145,6 +145,23 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------- GPU arm --
+def max_over_ranks(ms, world, device="cuda"):
+    """The slowest rank's time: what a job of `world` independent replicas takes (all-reduce MAX over the process group;
+    `device` is where the group's backend wants its tensors: cuda for NCCL, cpu for gloo)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    tm = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+    return float(tm.item())
+
+
+def whole_job_value(world, batch, steps, ms):
+    """Images per second of the whole job: every rank processed batch * steps images within `ms` (the slowest rank's)."""
+    return world * batch * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -508,12 +525,7 @@ def run_gpu(args):
         g.sync()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            tm = torch.tensor([ms], device="cuda")
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            ms = float(tm.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), world)
 
     dev_step = lambda i: g.step(pool_x[i % POOL], pool_y[i % POOL], loss_dev)
     for i in range(2 * K_MODULES + 2 + (0 if args.no_graphs else 8) + warmup):   # pipeline fill (+ graph recording) + warm-up, untimed
@@ -524,7 +536,7 @@ def run_gpu(args):
     ms = timed(steps, dev_step)
     launches = g.launch_count() - n0
     clocks = sampler.stop() if sampler else None
-    value = world * b * steps / (ms * 1e-3)
+    value = whole_job_value(world, b, steps, ms)
 
     if args.device_arm_only:
         g.close()
@@ -544,7 +556,7 @@ def run_gpu(args):
         host_step(i)
     g.sync()
     ms_e2e = timed(steps, host_step)
-    e2e_value = world * b * steps / (ms_e2e * 1e-3)
+    e2e_value = whole_job_value(world, b, steps, ms_e2e)
     h2d = host_x[0].numel() * 4 + host_y[0].numel() * 4
     final_loss = float(loss_host.item())
     g.close()
