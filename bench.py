@@ -528,10 +528,11 @@ def run_gpu(args):
         return max_over_ranks(e0.elapsed_time(e1), world)
 
     dev_step = lambda i: g.step(pool_x[i % POOL], pool_y[i % POOL], loss_dev)
+    # the clock sampler needs a moment to start: it runs from before the warm-up, so that its samples cover the timed region
+    sampler = ClockSampler(local) if rank == 0 else None
     for i in range(2 * K_MODULES + 2 + (0 if args.no_graphs else 8) + warmup):   # pipeline fill (+ graph recording) + warm-up, untimed
         dev_step(i)
     g.sync()
-    sampler = ClockSampler(local) if rank == 0 else None
     n0 = g.launch_count()
     ms = timed(steps, dev_step)
     launches = g.launch_count() - n0
