@@ -242,3 +242,61 @@ def _check_preact(k, u, ent, flat, grads, saved, cap, cmp, q, g, b, where, _unit
     cmp("dx", cap(u, 4, x_in.shape), q(dx_o), where)
     cmp("bn1.dgamma", _take(grads, ent[0]), dg1_o, where)
     cmp("bn1.dbeta", _take(grads, ent[1]), db1_o, where)
+
+
+def check_forward_layerwise_preact(g, params, arch, K, seed=0, tol=1e-2):
+    """Forward twin for the pre-activation family: after K iterations every module has forwarded one batch (module k
+    batch 1 at iteration k).  Every layer of every block -- batch norm + ReLU, the 3x3 convolutions, the shortcut and
+    the residual sum -- is recomputed by the oracle from what the library saved as that layer's input and compared
+    with what it saved as the layer's output.  Returns (blocks checked, worst error per kind of tensor)."""
+    import torch
+    b, hw0, classes = arch["batch"], arch["in_h"], arch["num_classes"]
+    for t in range(1, K + 1):
+        g.step(torch.from_numpy(S.images(seed, t, b, hw0, hw0, 3)).cuda(), torch.from_numpy(S.labels(seed, t, b, classes)).cuda())
+    g.sync()
+    q = L.round_bf16
+    worst, checked = {}, 0
+
+    def cmp(key, got, want, where):
+        err = _relmax(np.asarray(got, dtype=np.float64).reshape(-1), np.asarray(want, dtype=np.float64).reshape(-1))
+        worst[key] = max(worst.get(key, 0.0), err)
+        assert err <= tol, (where, key, err)
+
+    x_prev = None                                                    # output of the unit before, as the library saved it
+    for k in range(1, K + 1):
+        units = units_of(g.param_layout(k))
+        flat = params[k]
+        for u, (name, ent) in enumerate(units):
+            if name == "head":
+                continue
+            if name == "stem":
+                w1 = q(take(flat, ent[0]))
+                x_in = q(S.images(seed, 1, b, hw0, hw0, 3).astype(np.float64))
+                y = g.saved_tensor_of(k, u, 3, 1)[1].reshape(b, hw0, hw0, w1.shape[0]).astype(np.float64)
+                cmp("stem.y", y, q(L.conv2d_forward(x_in, w1, 1, 1)), (k, name))
+                x_prev = y
+                continue
+            g1, b1 = take(flat, ent[0]), take(flat, ent[1])
+            w1 = q(take(flat, ent[2]))
+            g2, b2 = take(flat, ent[3]), take(flat, ent[4])
+            w2 = q(take(flat, ent[5]))
+            proj = len(ent) > 6
+            co, ci = w1.shape[0], w1.shape[3]
+            hw_in = int(round((x_prev.size / (b * ci)) ** 0.5))
+            x_in = x_prev.reshape(b, hw_in, hw_in, ci)
+            o = g.saved_tensor_of(k, u, 0, 1)[1].reshape(x_in.shape).astype(np.float64)
+            ysz = g.saved_tensor_of(k, u, 3, 1)[1]
+            hw = int(round((ysz.size / (b * co)) ** 0.5))
+            stride = hw_in // hw
+            shp = (b, hw, hw, co)
+            c1, a2 = (g.saved_tensor_of(k, u, i, 1)[1].reshape(shp).astype(np.float64) for i in (1, 2))
+            y = ysz.reshape(shp).astype(np.float64)
+            where = (k, name)
+            cmp("o", o, q(L.relu_forward(L.batchnorm_forward(x_in, g1, b1, EPS)[0])), where)
+            cmp("c1", c1, q(L.conv2d_forward(o, w1, stride, 1)), where)
+            cmp("a2", a2, q(L.relu_forward(L.batchnorm_forward(c1, g2, b2, EPS)[0])), where)
+            sc = q(L.conv2d_forward(o, q(take(flat, ent[6])), stride, 0)) if proj else x_in
+            cmp("y", y, q(L.conv2d_forward(a2, w2, 1, 1) + sc), where)
+            x_prev = y
+            checked += 1
+    return checked, worst

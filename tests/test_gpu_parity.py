@@ -344,3 +344,13 @@ def test_wrn_widths_bf16_layer_by_layer():
     g.close()
     assert checked == 6, worst
     print("worst relative errors:", {k: float("%.2g" % v) for k, v in worst.items()})
+    # and the forward pass, layer by layer (the statistics of these layers come from the convolutions' epilogues)
+    from tests.layerwise import check_forward_layerwise_preact
+    g = B.FDG(B.make_arch(**arch), K=2, split_after_block=(3,), beta=0.5, lr=0.0, weight_decay=0.0, precision=B.FDG_BF16_TC)
+    for k in (1, 2):
+        g.set_params(k, params[k])
+    checked, worst = check_forward_layerwise_preact(g, params, arch, 2)
+    assert g.check_guards() == -1
+    g.close()
+    assert checked == 6, worst
+    print("forward, worst relative errors:", {k: float("%.2g" % v) for k, v in worst.items()})
