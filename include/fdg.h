@@ -242,11 +242,15 @@ fdg_status fdg_step(fdg_ctx* ctx, fdg_stream stream, const float* images_dev, co
                     float* loss_dev);
 
 /* The same iteration fed from host memory: copies `images_host` (fp32, same layout) and
- * `labels_host` to a staging area of the workspace with cudaMemcpyAsync on `stream`, runs
- * fdg_step on them, and enqueues a device-to-host copy of the loss of batch t-K+1 into
- * `loss_host` (nullable; untouched while t < K).  Pinned host buffers keep the call
- * asynchronous; pageable ones make the copies block.  The host buffers may be reused once
- * `stream` has passed the copies; read *loss_host after fdg_sync.  Errors as fdg_step. */
+ * `labels_host` to a staging area of the workspace with cudaMemcpyAsync, runs fdg_step on
+ * them, and enqueues a device-to-host copy of the loss of batch t-K+1 into `loss_host`
+ * (nullable; untouched while t < K).  The two copies go on a stream of the context, ordered
+ * only behind the previous call's read of the staging area, so that from pinned memory they
+ * run beside the previous iteration's module-steps; `stream` waits for them before the step.
+ * They are NOT ordered behind earlier work on `stream`: the host buffers must hold the batch
+ * when the call is made.  Pinned host buffers keep the call asynchronous; pageable ones make
+ * the copies block.  The host buffers may be reused once `stream` has passed the step; read
+ * *loss_host after fdg_sync.  Errors as fdg_step. */
 fdg_status fdg_step_host(fdg_ctx* ctx, fdg_stream stream, const float* images_host, const int32_t* labels_host,
                          float* loss_host);
 

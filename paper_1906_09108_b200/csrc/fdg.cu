@@ -180,6 +180,11 @@ struct fdg_ctx {
   cudaStream_t cap_stream = nullptr;  // origin stream of the recordings (the caller's stream may be the legacy
                                       // default stream, which cannot be captured); graphs are launched on the caller's
   cudaEvent_t ev_fork = nullptr;
+  // fdg_step_host: the host-to-device copy of a call runs on its own stream, beside the step of the call before;
+  // ev_staged = the copy has landed, ev_ingested = the ingest kernel has read the staging buffers (they may be refilled)
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_staged = nullptr, ev_ingested = nullptr;
+  bool record_ingested = false;
   std::vector<cudaEvent_t> ev_cjoin;
   float* lr_dev = nullptr;
   float lr_on_device = -1.f;
@@ -1274,6 +1279,9 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   for (int i = 0; i < kEventRing && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_staged, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_ingested, cudaEventDisableTiming);
   if (e == cudaSuccess && c->use_graphs) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
   c->ev_cjoin.assign(c->K, nullptr);
   for (int k = 0; k < c->K && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&c->ev_cjoin[k], cudaEventDisableTiming);
@@ -1310,6 +1318,9 @@ fdg_status fdg_destroy(fdg_ctx* c) {
   for (int i = 0; i < kEventRing; ++i) cudaEventDestroy(c->ev_in[i]);
   cudaEventDestroy(c->ev_join);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_staged) cudaEventDestroy(c->ev_staged);
+  if (c->ev_ingested) cudaEventDestroy(c->ev_ingested);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
   for (cudaEvent_t ev : c->ev_cjoin) if (ev) cudaEventDestroy(ev);
   for (cudaGraphExec_t g : c->graph_exec) if (g) cudaGraphExecDestroy(g);
@@ -1535,6 +1546,7 @@ fdg_status fdg_step(fdg_ctx* c, fdg_stream stream, const float* images_dev, cons
     ++c->launches;
     e = L.err;
     if (e == cudaSuccess && !serial && !graph) e = cudaEventRecord(c->ev_in[t % kEventRing], cs);
+    if (e == cudaSuccess && c->record_ingested) e = cudaEventRecord(c->ev_ingested, cs);
     if (e != cudaSuccess) return cuda_fail(c, e, "ingest");
   }
   if (graph) e = graph_step(c, cs, loss_dev);
@@ -1550,10 +1562,17 @@ fdg_status fdg_step_host(fdg_ctx* c, fdg_stream stream, const float* images_host
   if (c->latched != FDG_OK) return c->latched;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   const size_t img_bytes = (size_t)c->arch.batch * c->arch.in_h * c->arch.in_w * c->arch.in_c * 4;
-  cudaError_t e = cudaMemcpyAsync(c->host_images, images_host, img_bytes, cudaMemcpyHostToDevice, cs);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(c->host_labels, labels_host, (size_t)c->arch.batch * 4, cudaMemcpyHostToDevice, cs);
+  // The copy waits only for the ingest of the call before (which read the staging buffers), not for that call's
+  // module-steps: from pinned memory it runs beside them.  (An event that was never recorded does not block.)
+  cudaError_t e = cudaStreamWaitEvent(c->copy_stream, c->ev_ingested, 0);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->host_images, images_host, img_bytes, cudaMemcpyHostToDevice, c->copy_stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->host_labels, labels_host, (size_t)c->arch.batch * 4, cudaMemcpyHostToDevice, c->copy_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(c->ev_staged, c->copy_stream);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, c->ev_staged, 0);
   if (e != cudaSuccess) return cuda_fail(c, e, "host to device copy");
+  c->record_ingested = true;
   fdg_status s = fdg_step(c, stream, c->host_images, c->host_labels, nullptr);
+  c->record_ingested = false;
   if (s != FDG_OK) return s;
   if (loss_host && c->t >= c->K) {
     Module& mk = c->mods[c->K - 1];

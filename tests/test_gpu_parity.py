@@ -115,6 +115,48 @@ def test_graph_replay_is_bitwise_identical_to_streams(precision):
         assert np.array_equal(a, b)
 
 
+@pytest.mark.parametrize("graphs", [False, True])
+def test_host_fed_steps_are_bitwise_identical_to_device_fed(graphs):
+    """fdg_step_host copies each batch on a stream of the context, beside the iteration before, and hands it to
+    the same step: 30 iterations enqueued back to back from pinned buffers, none of them waited for, must leave
+    the parameters and every loss of a run fed from device tensors (a copy that overtook the previous ingest,
+    or a step that overtook its copy, would not)."""
+    import torch
+    import fdg_synth as S
+    from paper_1906_09108_b200 import binding as B
+    arch = dict(CFG1, n_per_stage=2, batch=16, in_h=32, in_w=32)
+    steps = 30
+    outs, losses = [], []
+    for host in (False, True):
+        g = B.FDG(B.make_arch(**arch), K=4, split_after_block=(1, 3, 5), beta=0.5, lr=0.05, graphs=graphs)
+        for k in range(1, 5):
+            g.set_params(k, S.init_params(3, k, g.param_layout(k), jitter=True))
+        ls = []
+        if host:
+            hx = [torch.from_numpy(S.images(3, t, 16, 32, 32, 3)).pin_memory() for t in range(1, steps + 1)]
+            hy = [torch.from_numpy(S.labels(3, t, 16, 10)).pin_memory() for t in range(1, steps + 1)]
+            hl = torch.zeros(steps + 1).pin_memory()
+            for t in range(1, steps + 1):      # enqueued back to back, the host never waits
+                g.step_host(hx[t - 1], hy[t - 1], hl[t:])
+            g.sync()
+            ls = [float(v) for v in hl[4:]]
+        else:
+            loss = torch.zeros(steps + 1, device="cuda")
+            for t in range(1, steps + 1):
+                x = torch.from_numpy(S.images(3, t, 16, 32, 32, 3)).cuda()
+                y = torch.from_numpy(S.labels(3, t, 16, 10)).cuda()
+                g.step(x, y, loss[t:])
+            g.sync()
+            ls = [float(v) for v in loss[4:].cpu()]
+        outs.append([g.get_params(k) for k in range(1, 5)])
+        losses.append(ls)
+        assert g.check_guards() == -1
+        g.close()
+    assert losses[0] == losses[1] and all(np.isfinite(losses[0])) and min(losses[0]) > 0
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+
+
 @pytest.mark.parametrize("K,splits,order,steps", [(1, (), "backward_first", 11), (2, (2,), "forward_first", 14),
                                                   (3, (1, 3), "backward_first", 20)])
 def test_graph_replay_fp32_against_oracle(K, splits, order, steps):
