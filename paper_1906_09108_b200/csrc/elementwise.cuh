@@ -632,24 +632,56 @@ __global__ void export_kernel(const T* __restrict__ in, float* __restrict__ out,
 //   pooled [B][F], dlogits [B][classes], loss_n [B] (fp32 scratch for head_param_grad)
 //   dx [B][HW][F] (T) = dpooled[f] / HW
 // A label outside [0, classes) sets *bad_label and is treated as class 0.
+// `groups` > 0 (F a multiple of the 16-byte vector, see head_groups): the sample is read and its gradient written in
+// 16-byte vectors; `groups` sets of threads take every groups-th pixel and their partial sums are added in group
+// order.  `groups` == 0: element by element, for any F.
 template <typename T>
 __global__ void head_fwd_bwd_kernel(const T* __restrict__ x, const float* __restrict__ w, const float* __restrict__ b,
-                                    const int32_t* __restrict__ labels, int HW, int F, int classes, int batch,
+                                    const int32_t* __restrict__ labels, int HW, int F, int classes, int batch, int groups,
                                     float* __restrict__ pooled, float* __restrict__ dlogits,
                                     float* __restrict__ loss_n, T* __restrict__ dx, int* __restrict__ bad_label) {
-  extern __shared__ float hs[];            // pooled[F] | logits[classes] | dpooled[F]
+  constexpr int V = 16 / (int)sizeof(T);
+  extern __shared__ __align__(16) float hs[];   // pooled[F] | dpooled[F] | partial[groups][F] | logits[classes]
   float* s_pool = hs;
-  float* s_logit = hs + F;
-  float* s_dpool = s_logit + classes;
+  float* s_dpool = hs + F;
+  float* s_part = s_dpool + F;
+  float* s_logit = s_part + (size_t)groups * F;
   const int n = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
   const T* xn = x + (size_t)n * HW * F;
-  for (int f = tid; f < F; f += nt) {
-    float a = 0.f;
+  if (groups > 0) {
+    const int cols = F / V;
+    for (int item = tid; item < groups * cols; item += nt) {
+      const int g = item / cols, col = item - g * cols;
+      float acc[V];
+#pragma unroll
+      for (int j = 0; j < V; ++j) acc[j] = 0.f;
+#pragma unroll 4
+      for (int p = g; p < HW; p += groups) {
+        float v[V];
+        load_vec<T, V>(xn + (size_t)p * F + col * V, v);
+#pragma unroll
+        for (int j = 0; j < V; ++j) acc[j] += v[j];
+      }
+#pragma unroll
+      for (int j = 0; j < V; ++j) s_part[(size_t)g * F + col * V + j] = acc[j];
+    }
+    __syncthreads();
+    for (int f = tid; f < F; f += nt) {
+      float a = 0.f;
+      for (int g = 0; g < groups; ++g) a += s_part[(size_t)g * F + f];
+      a /= (float)HW;
+      s_pool[f] = a;
+      pooled[(size_t)n * F + f] = a;
+    }
+  } else {
+    for (int f = tid; f < F; f += nt) {
+      float a = 0.f;
 #pragma unroll 8
-    for (int p = 0; p < HW; ++p) a += to_f(xn[(size_t)p * F + f]);
-    a /= (float)HW;
-    s_pool[f] = a;
-    pooled[(size_t)n * F + f] = a;
+      for (int p = 0; p < HW; ++p) a += to_f(xn[(size_t)p * F + f]);
+      a /= (float)HW;
+      s_pool[f] = a;
+      pooled[(size_t)n * F + f] = a;
+    }
   }
   __syncthreads();
   const int warp = tid >> 5, lane = tid & 31, nwarps = nt >> 5;
@@ -694,31 +726,64 @@ __global__ void head_fwd_bwd_kernel(const T* __restrict__ x, const float* __rest
   }
   __syncthreads();
   T* dxn = dx + (size_t)n * HW * F;
-  for (int i = tid; i < HW * F; i += nt) dxn[i] = from_f<T>(s_dpool[i % F]);
+  if (groups > 0) {
+    // the row of F gradients, packed once as T into the (now free) partial-sum area, then copied to every pixel
+    T* s_row = reinterpret_cast<T*>(s_part);
+    for (int f = tid; f < F; f += nt) s_row[f] = from_f<T>(s_dpool[f]);
+    __syncthreads();
+    const int cols = F / V;
+    const uint4* row4 = reinterpret_cast<const uint4*>(s_row);
+    uint4* dx4 = reinterpret_cast<uint4*>(dxn);
+    for (int i = tid; i < HW * cols; i += nt) dx4[i] = row4[i % cols];
+  } else {
+    for (int i = tid; i < HW * F; i += nt) dxn[i] = from_f<T>(s_dpool[i % F]);
+  }
 }
 
-// One block per class: dW[c][f] = sum_n dlogits[n][c]*pooled[n][f], db[c] = sum_n dlogits[n][c];
-// block 0 also reduces the loss (mean over the batch) and raises *nonfinite if it is NaN/Inf.
+constexpr int kHeadThreads = 256;
+// Pixel groups of head_fwd_bwd_kernel for F features of `elem_bytes` each: 0 when F is not a whole number of
+// 16-byte vectors, otherwise as many as fill the block (at most 8, and within the default shared-memory limit).
+inline int head_groups(int F, int classes, int HW, size_t elem_bytes) {
+  const int V = (int)(16 / elem_bytes);
+  if (F % V != 0) return 0;
+  int g = kHeadThreads / (F / V);
+  if (g > 8) g = 8;
+  if (g > HW) g = HW;
+  if (g < 1) g = 1;
+  while (g > 1 && ((size_t)(2 + g) * F + classes) * 4 > 40 * 1024) --g;
+  return g;
+}
+inline size_t head_smem_bytes(int F, int classes, int groups) { return ((size_t)(2 + groups) * F + classes) * 4; }
+
+// dW[c][f] = sum_n dlogits[n][c]*pooled[n][f], db[c] = sum_n dlogits[n][c].  Grid (classes, ceil(F / 32)), 128
+// threads: a lane owns a feature, the four warps take every fourth sample and their partial sums are added in warp
+// order.  Blocks (c, 0) also form db[c]; block (0, 0) reduces the loss (mean over the batch) and raises *nonfinite if
+// it is NaN/Inf.
 __global__ void head_param_grad_kernel(const float* __restrict__ pooled, const float* __restrict__ dlogits,
                                        const float* __restrict__ loss_n, int F, int classes, int batch,
                                        float* __restrict__ dW, float* __restrict__ db, float* __restrict__ loss,
                                        int* __restrict__ nonfinite) {
+  __shared__ float s_part[4][32];
   const int c = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int f = threadIdx.x; f < F; f += blockDim.x) {
-    float a = 0.f;
+  const int f = blockIdx.y * 32 + lane;
+  float a = 0.f;
+  if (f < F) {
 #pragma unroll 8
-    for (int n = 0; n < batch; ++n) a += dlogits[(size_t)n * classes + c] * pooled[(size_t)n * F + f];
-    dW[(size_t)c * F + f] = a;
+    for (int n = warp; n < batch; n += 4) a += dlogits[(size_t)n * classes + c] * pooled[(size_t)n * F + f];
   }
+  s_part[warp][lane] = a;
+  __syncthreads();
+  if (warp == 0 && f < F) dW[(size_t)c * F + f] = ((s_part[0][lane] + s_part[1][lane]) + s_part[2][lane]) + s_part[3][lane];
+  if (blockIdx.y != 0) return;
   // the sums over the batch: lanes take every 32nd sample, the partial sums meet in a fixed butterfly
-  if (warp == 0) {
-    float a = 0.f;
-    for (int n = lane; n < batch; n += 32) a += dlogits[(size_t)n * classes + c];
+  if (warp == 1) {
+    float s = 0.f;
+    for (int n = lane; n < batch; n += 32) s += dlogits[(size_t)n * classes + c];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-    if (lane == 0) db[c] = a;
-  } else if (warp == 1 && c == 0) {
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) db[c] = s;
+  } else if (warp == 2 && c == 0) {
     double l = 0.0;
     for (int n = lane; n < batch; n += 32) l += (double)loss_n[n];
 #pragma unroll
@@ -729,6 +794,27 @@ __global__ void head_param_grad_kernel(const float* __restrict__ pooled, const f
       if (!isfinite(lf)) atomicExch(nonfinite, 1);
     }
   }
+}
+
+// The two launches of the head on stream `st` (arguments as the kernels').
+template <typename T>
+inline cudaError_t launch_head(cudaStream_t st, const T* x, const float* w, const float* b, const int32_t* labels, int HW,
+                               int F, int classes, int batch, float* pooled, float* dlogits, float* loss_n, T* dx,
+                               float* dW, float* db, float* loss, int* flags, bool second = true, bool first = true) {
+  if (first) {
+    int groups = head_groups(F, classes, HW, sizeof(T));
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(dx)) & 15) groups = 0;   // vectors need 16-byte alignment
+    head_fwd_bwd_kernel<T><<<batch, kHeadThreads, head_smem_bytes(F, classes, groups), st>>>(
+        x, w, b, labels, HW, F, classes, batch, groups, pooled, dlogits, loss_n, dx, flags + 1);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  if (second) {
+    head_param_grad_kernel<<<dim3(classes, (F + 31) / 32), 128, 0, st>>>(pooled, dlogits, loss_n, F, classes, batch, dW, db,
+                                                                          loss, flags);
+    return cudaGetLastError();
+  }
+  return cudaSuccess;
 }
 
 // ------------------------------------------------------------------- SGD ----

@@ -852,15 +852,14 @@ static void head_forward_backward(fdg_ctx* c, Module& m, Launch& L, int64_t tau,
   }
   const int32_t* labels = c->labels + (size_t)(tau % c->label_ring) * B;
   T* dfeat = u.bn ? reinterpret_cast<T*>(m.temps[2]) : gout;
-  const size_t smem = (size_t)(2 * F + classes) * 4;
   L.begin(KC_HEAD, 2.0 * rows * F * sizeof(T), 4.0 * B * F * classes);
-  head_fwd_bwd_kernel<T><<<B, 128, smem, L.st>>>(feat, wf + u.w1, wf + u.w2, labels, HW, F, classes, B, m.pooled,
-                                                  m.dlogits, m.loss_n, dfeat, c->flags + 1);
-  L.check();
+  L.note(launch_head<T>(L.st, feat, wf + u.w1, wf + u.w2, labels, HW, F, classes, B, m.pooled, m.dlogits, m.loss_n, dfeat,
+                        m.grad + u.w1, m.grad + u.w2, m.loss, c->flags, false, true));
+  ++c->launches;
   L.begin(KC_HEAD, 4.0 * B * (F + classes) + 4.0 * classes * F, 2.0 * B * F * classes);
-  head_param_grad_kernel<<<classes, 128, 0, L.st>>>(m.pooled, m.dlogits, m.loss_n, F, classes, B, m.grad + u.w1,
-                                                     m.grad + u.w2, m.loss, c->flags);
-  L.check();
+  L.note(launch_head<T>(L.st, feat, wf + u.w1, wf + u.w2, labels, HW, F, classes, B, m.pooled, m.dlogits, m.loss_n, dfeat,
+                        m.grad + u.w1, m.grad + u.w2, m.loss, c->flags, true, false));
+  ++c->launches;
   if (u.bn)
     bn_backward<T>(L, m, dfeat, feat, x, Fs + u.st1, wf + u.g1, m.grad + u.g1, m.grad + u.b1, nullptr, nullptr, nullptr,
                    nullptr, nullptr, nullptr, gout, nullptr, rows, F);

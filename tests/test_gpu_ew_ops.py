@@ -253,7 +253,8 @@ def test_shrink_ingest_and_update(prec_name):
 
 
 @pytest.mark.parametrize("prec_name", ["fp32", "bf16"])
-@pytest.mark.parametrize("bhwfc", [(8, 8, 8, 64, 10), (5, 4, 4, 32, 7), (6, 8, 8, 640, 100)])
+@pytest.mark.parametrize("bhwfc", [(8, 8, 8, 64, 10), (5, 4, 4, 32, 7), (6, 8, 8, 640, 100), (7, 3, 5, 18, 7),
+                                   (4, 8, 8, 2056, 5), (9, 2, 2, 48, 3), (130, 4, 4, 512, 10)])
 def test_head(prec_name, bhwfc):
     B, ew, tol = _ops(prec_name)
     b, h, w, f, classes = bhwfc
