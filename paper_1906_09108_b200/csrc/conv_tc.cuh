@@ -897,13 +897,48 @@ __global__ void __launch_bounds__(128, 1) mma_rate_kernel(int n, int accs, int r
 // dst[ci][2-r][2-s][co] = src[co][r][s][ci]; taps = 1: the transpose of a 1x1 filter.  One block row per entry of
 // `table` (src offset, dst offset, Co, Ci, taps), all offsets in elements from the two base pointers.
 struct FlipEntry { unsigned long long src, dst; int Co, Ci, taps; };
-__global__ void __launch_bounds__(256) wflip_kernel(const __nv_bfloat16* __restrict__ src_base, __nv_bfloat16* __restrict__ dst_base,
-                                                    const FlipEntry* __restrict__ table) {
-  // 32 x 32 tiles of one tap's [Co][Ci] matrix go through shared memory, so that both the reads (along ci) and
-  // the writes (along co) are contiguous.  256 threads = 32 columns x 8 rows.
-  __shared__ __nv_bfloat16 tile[32][34];
-  const FlipEntry e = table[blockIdx.y];
+// The copy of one entry by the blocks blockIdx.x = 0 .. gridDim.x-1 (256 threads each).  Tiles of one tap's [Co][Ci]
+// matrix go through shared memory, so that both the reads (along ci) and the writes (along co) are contiguous.
+__device__ __forceinline__ void wflip_entry(const __nv_bfloat16* __restrict__ src_base, __nv_bfloat16* __restrict__ dst_base,
+                                            const FlipEntry& e, __nv_bfloat16 (&tile)[64][66]) {
   const int T = e.taps;                                                       // 9, or 1: the plain transpose of a 1x1 filter
+  if (((e.Co | e.Ci) & 7) == 0 &&
+      ((reinterpret_cast<uintptr_t>(src_base + e.src) | reinterpret_cast<uintptr_t>(dst_base + e.dst)) & 15) == 0) {
+    // 64 x 64 tiles moved as 16-byte vectors (8 channels): a thread reads two vectors along ci, then writes two along co
+    // that it gathers from eight rows of the tile.  Rows are 66 elements = 33 words apart: the word-wise stores of a
+    // warp (4 rows x 8 vectors) fall on 32 different banks, the gathers (rows 8 apart) meet two by two.
+    const int tco = (e.Co + 63) / 64, tci = (e.Ci + 63) / 64;
+    const int total = T * tco * tci;
+    const int vr = threadIdx.x >> 3, vc = (threadIdx.x & 7) * 8;                // vector slot: row 0..31 (+32), column 0,8,..56
+    for (int id = blockIdx.x; id < total; id += gridDim.x) {
+      const int t = id / (tco * tci), rem = id - t * tco * tci;
+      const int co0 = (rem / tci) * 64, ci0 = (rem - (rem / tci) * tci) * 64;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int co = co0 + vr + 32 * h, ci = ci0 + vc;
+        if (co < e.Co && ci < e.Ci) {
+          const uint4 v = *reinterpret_cast<const uint4*>(src_base + e.src + ((size_t)co * T + t) * e.Ci + ci);
+          uint32_t* d = reinterpret_cast<uint32_t*>(&tile[vr + 32 * h][vc]);
+          d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+        }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int ci = ci0 + vr + 32 * h, co = co0 + vc;
+        if (co < e.Co && ci < e.Ci) {
+          uint4 v;
+          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(&v);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) o[j] = tile[vc + j][vr + 32 * h];
+          *reinterpret_cast<uint4*>(dst_base + e.dst + ((size_t)ci * T + (T - 1 - t)) * e.Co + co) = v;
+        }
+      }
+      __syncthreads();
+    }
+    return;
+  }
+  // any channel counts and offsets: 32 x 32 tiles, element by element; 256 threads = 32 columns x 8 rows
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int tco = (e.Co + 31) / 32, tci = (e.Ci + 31) / 32;
   const int total = T * tco * tci;
@@ -921,6 +956,16 @@ __global__ void __launch_bounds__(256) wflip_kernel(const __nv_bfloat16* __restr
     }
     __syncthreads();
   }
+}
+__global__ void __launch_bounds__(256) wflip_kernel(const __nv_bfloat16* __restrict__ src_base, __nv_bfloat16* __restrict__ dst_base,
+                                                    const FlipEntry* __restrict__ table) {
+  __shared__ __align__(16) __nv_bfloat16 tile[64][66];
+  wflip_entry(src_base, dst_base, table[blockIdx.y], tile);
+}
+// One filter, its entry passed by value.
+__global__ void __launch_bounds__(256) wflip_one_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, FlipEntry e) {
+  __shared__ __align__(16) __nv_bfloat16 tile[64][66];
+  wflip_entry(src, dst, e, tile);
 }
 
 }  // namespace tc

@@ -133,3 +133,18 @@ def test_conv_ops_bf16_cuda_core_shapes(shape):
 @pytest.mark.parametrize("shape", SHAPES_TC)
 def test_conv_ops_bf16_tensor_core_shapes(shape):
     _run("bf16", shape, True)
+
+
+@pytest.mark.parametrize("co,ci,r", [(16, 16, 3), (64, 160, 3), (320, 160, 1), (24, 20, 3), (10, 6, 1), (200, 72, 3),
+                                     (640, 640, 3), (65, 64, 3)])
+def test_flipped_weight_copy_is_the_index_permutation(co, ci, r):
+    """dst[ci][R-1-r][R-1-s][co] = src[co][r][s][ci], bit for bit: channel counts that take the 16-byte vector
+    tiles (multiples of 8), ragged last tiles (200, 72), and counts that take the element-wise tiles."""
+    from paper_1906_09108_b200 import binding as B
+    ops = B.ConvOps(B.FDG_BF16_TC)
+    s = B.fdg_conv_shape(1, 8, 8, ci, co, r, 1, r // 2)
+    rng = np.random.default_rng(7)
+    w = torch.from_numpy(rng.standard_normal((co, r, r, ci)).astype(np.float32)).to(torch.bfloat16).cuda()
+    got = ops.flip_weights(s, w).view(ci, r, r, co).float().cpu().numpy()
+    want = w.float().cpu().numpy()[:, ::-1, ::-1, :].transpose(3, 1, 2, 0)
+    assert np.array_equal(got, want)
