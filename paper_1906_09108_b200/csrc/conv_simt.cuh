@@ -218,6 +218,39 @@ __global__ void wgrad_reduce_kernel(const float* __restrict__ partial, float* __
   }
 }
 
+// The same sum for many partial rows of a short vector (one row per image): a block takes 32 consecutive outputs,
+// its 16 warps every 16th row (a warp reads 128 contiguous bytes of a row), and the 16 partial sums of an output are
+// added in warp order, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(512) wgrad_reduce_tall_kernel(const float* __restrict__ partial, float* __restrict__ grad,
+                                                                size_t n, int splits) {
+  __shared__ float part[16][33];
+  const int col = threadIdx.x & 31, rg = threadIdx.x >> 5;
+  const size_t i = (size_t)blockIdx.x * 32 + col;
+  float a = 0.f;
+  if (i < n) {
+#pragma unroll 4
+    for (int z = rg; z < splits; z += 16) a += partial[(size_t)z * n + i];
+  }
+  part[rg][col] = a;
+  __syncthreads();
+  if (rg == 0 && i < n) {
+    float t = 0.f;
+#pragma unroll
+    for (int r = 0; r < 16; ++r) t += part[r][col];
+    grad[i] = t;
+  }
+}
+// grad = the sum of `splits` partial rows of n floats, on stream st.
+inline cudaError_t launch_wgrad_reduce(cudaStream_t st, const float* partial, float* grad, size_t n, int splits) {
+  if (splits >= 32 && n <= (size_t)1 << 16) {
+    wgrad_reduce_tall_kernel<<<(unsigned)((n + 31) / 32), 512, 0, st>>>(partial, grad, n, splits);
+  } else {
+    int blocks = (int)((n + 255) / 256); if (blocks > 1184) blocks = 1184;
+    wgrad_reduce_kernel<<<blocks, 256, 0, st>>>(partial, grad, n, splits);
+  }
+  return cudaGetLastError();
+}
+
 // Number of pixel slices the weight-gradient GEMM is split into, and the slice length.
 inline void wgrad_split(const ConvGeom& g, int bm, int bn, int* splits, int* k_chunk) {
   const long M = (long)g.R * g.S * g.Ci, N = g.Co, K = (long)g.N * g.P * g.Q;
@@ -259,9 +292,7 @@ inline cudaError_t launch_conv_simt(cudaStream_t st, const ConvGeom& g, const T*
   if (MODE == CONV_WGRAD && splits > 1) {
     ++*launches;
     size_t n = (size_t)Mdim * Ndim;
-    int blocks = (int)((n + 255) / 256); if (blocks > 1184) blocks = 1184;
-    wgrad_reduce_kernel<<<blocks, 256, 0, st>>>(wpartial, wgrad_out, n, splits);
-    e = cudaGetLastError();
+    e = launch_wgrad_reduce(st, wpartial, wgrad_out, n, splits);
   }
   return e;
 }
@@ -321,10 +352,8 @@ inline cudaError_t launch_small_wgrad(cudaStream_t st, const ConvGeom& g, const 
   small_wgrad_kernel<T><<<g.N, threads, smem, st>>>(x, dy, scratch, g.H, g.W, g.Ci, g.Co);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  int blocks = (outs + 255) / 256;
-  wgrad_reduce_kernel<<<blocks, 256, 0, st>>>(scratch, dw, (size_t)outs, g.N);
   *launches += 2;
-  return cudaGetLastError();
+  return launch_wgrad_reduce(st, scratch, dw, (size_t)outs, g.N);
 }
 
 // ---- weight gradient of a 1x1 convolution (projection shortcut), stride 1 or 2, few channels ----
@@ -390,9 +419,8 @@ inline cudaError_t launch_proj_wgrad(cudaStream_t st, const ConvGeom& g, const T
   proj_wgrad_kernel<T><<<g.N, threads, smem, st>>>(x, dy, scratch, g.H, g.W, g.P, g.Q, g.Ci, g.Co, g.stride, strip);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  wgrad_reduce_kernel<<<(outs + 255) / 256, 256, 0, st>>>(scratch, dw, (size_t)outs, g.N);
   *launches += 2;
-  return cudaGetLastError();
+  return launch_wgrad_reduce(st, scratch, dw, (size_t)outs, g.N);
 }
 
 // Upper bound of the fp32 scratch elements a weight-gradient launch may need.

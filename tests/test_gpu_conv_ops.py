@@ -24,7 +24,7 @@ def _rel(a, b):
 
 # (N, H, W, Ci, Co, R, stride, pad)
 SHAPES_ANY = [(3, 12, 20, 5, 7, 3, 1, 1), (2, 16, 16, 8, 16, 3, 2, 1), (2, 16, 16, 16, 24, 1, 2, 0),
-              (5, 8, 8, 3, 8, 3, 1, 1)]
+              (5, 8, 8, 3, 8, 3, 1, 1), (3, 16, 16, 6, 32, 1, 1, 0), (3, 16, 16, 12, 32, 1, 2, 0)]
 SHAPES_TC = [(4, 32, 32, 16, 16, 3, 1, 1),      # 32 tiles of 4 image rows, 32-byte swizzle
              (6, 16, 16, 32, 32, 3, 1, 1),      # 8 rows per tile, 64-byte swizzle
              (10, 8, 8, 64, 64, 3, 1, 1),       # two images per tile, 128-byte swizzle
