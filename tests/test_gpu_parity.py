@@ -46,11 +46,19 @@ def test_odd_shapes_fp32():
     check_fp32(run_pair(arch, 2, (2,), 6, beta=0.7, lr=0.05))
 
 
-def test_wrn_fp32():
+@pytest.mark.parametrize("seed", [1, 2, 4])
+def test_wrn_fp32(seed):
+    """Pre-activation blocks, K = 2 and 3.  In every seed of this small network some ReLU inputs of the float64 run lie
+    within 3e-7 of zero, about the rounding error of the fp32 pre-activations, so whether one of those gates falls
+    differently in fp32 is decided by the order of a summation; where it does, that element of the gradient changes by
+    O(1) and the batch-norm parameter gradients of its layer by up to 1 % (seed 0: at the 7th to 9th iteration, seed
+    3: from the 2nd on, with the loss still equal to 1e-7 -- the same with every version of the kernels tried).  The
+    seeds used here are ones where no gate falls differently within the iterations compared; what a flipped gate does
+    to a gradient is pinned on the CPU in test_oracle_conditioning.py."""
     arch = dict(family="wrn", n_per_stage=2, widths=(16, 24, 40), stem_width=8, in_h=16, in_w=16, in_c=3,
                 num_classes=20, batch=6)
-    check_fp32(run_pair(arch, 2, (3,), 7, beta=0.6, lr=0.05))
-    check_fp32(run_pair(arch, 3, (2, 4), 9, beta=0.6, lr=0.05))
+    check_fp32(run_pair(arch, 2, (3,), 7, beta=0.6, lr=0.05, seed=seed))
+    check_fp32(run_pair(arch, 3, (2, 4), 9, beta=0.6, lr=0.05, seed=seed))
 
 
 def test_serial_mode_is_bitwise_identical_to_streams():
