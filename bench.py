@@ -211,7 +211,7 @@ KERNEL_SHAPES = {     # the 3x3 stride-1 layer shapes of the 6n+2 workloads and 
     "wrn_stage1": (128, 32, 32, 160), "wrn_stage2": (128, 16, 16, 320), "wrn_stage3": (128, 8, 8, 640)}
 
 
-# The convolution launches as the module-step issues them: on a third of the SMs (four modules side by side),
+# The convolution launches as the module-step issues them: on a quarter of the SMs (four modules side by side),
 # several image tiles per CTA, with the reductions fused into their epilogues.
 STEP_VARIANTS = {
     "fprop_stats": "forward + batch-norm statistics of its output (conv1, conv2 of a block)",
@@ -246,7 +246,7 @@ def kernel_bench(B, which="fprop", stage="stage1", launches=64, reps=5, use_grap
     extra = None
     extra_tensors = 0
     if variant:
-        ex, keep = ops._extra(s, share=3, wgrad_cta_cap=16 if variant == "wgrad_side" else 0,
+        ex, keep = ops._extra(s, share=4, wgrad_cta_cap=16 if variant == "wgrad_side" else 0,
                               reduce={"fprop_stats": 1, "dgrad_bn": 2, "dgrad_res_bn": 2, "wgrad_side": 0}[variant],
                               next_mask=xs[0], next_x=xs[0], next_stats=torch.zeros(2 * c, device="cuda") + 1.0, C_red=c)
         extra = B.C.byref(ex)
@@ -593,7 +593,7 @@ def run_gpu(args):
                         # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this shape,
                         # from the committed ncu summary; null once the kernel's source has changed since
                         traffic=profiled_traffic())
-            # The same kernels in the launch shape the module-step issues them in (a third of the SMs, three image
+            # The same kernels in the launch shape the module-step issues them in (a quarter of the SMs, four image
             # tiles per CTA, reductions fused into the epilogue), the two batch-norm apply kernels at the stage-1
             # shape, and the wide-layer convolution against the tensor roofline: each timed alone the same way.
             iso = {}

@@ -1284,10 +1284,11 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   if (e == cudaSuccess && c->use_graphs) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
   c->ev_cjoin.assign(c->K, nullptr);
   for (int k = 0; k < c->K && e == cudaSuccess; ++k) e = cudaEventCreateWithFlags(&c->ev_cjoin[k], cudaEventDisableTiming);
-  // Convolution launches are sized for the module streams running side by side.  With 128 image tiles
-  // per layer, 148 / K SMs each gives 2 tiles per CTA at K = 2 and 4 at K = 4; three per CTA (43 CTAs)
-  // measured faster at K = 4 than both two and four, so one stream's share is left unclaimed there.
-  c->tmaps.share = c->cfg.serial ? 1 : (c->K > 2 ? c->K - 1 : c->K);
+  // Convolution launches are sized for the module streams running side by side: 148 / K SMs each.  With 128
+  // image tiles per layer that is 2 tiles per CTA at K = 2 and 4 at K = 4 (32 CTAs; measured against 3, 5, 6 and
+  // 8 tiles per CTA: the four chains' convolutions then fit the SMs together and a CTA's start-up is paid once
+  // per four tiles).
+  c->tmaps.share = c->cfg.serial ? 1 : c->K;
   c->tmaps.wgrad_side_cap = 16;
   // Blocks of a batch-norm apply kernel that first re-adds a convolution's partial sums: 4 per SM shared
   // between the module streams (measured optimum: 148 blocks at K = 4, 296 at K = 2).

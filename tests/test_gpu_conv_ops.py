@@ -102,15 +102,15 @@ def _run(prec_name, shape, expect_tc):
     dw = ops.wgrad(s, x, dy).cpu().numpy()
     assert _rel(dw, dwo) < (1e-3 if prec_name == "bf16" else 2e-5)
     if expect_tc:
-        # the launch shapes of a module-step: a third of the SMs per kernel (four modules side by side),
+        # the launch shapes of a module-step: a quarter of the SMs per kernel (four modules side by side),
         # the weight gradient's pixel split capped at 16 CTAs (side stream), and, for stride 2, both
         # gradients on the tensor cores through the spread-out dy
         sp = st == 2
         if sp:
             assert ops.path(s, 1)
-        y = ops.forward(s, x, wt, res=resy, share=3).float().cpu().numpy()
+        y = ops.forward(s, x, wt, res=resy, share=4).float().cpu().numpy()
         assert _rel(y, L.conv2d_forward(xo, wo, st, pad) + resyo) < tol
-        dx = ops.dgrad(s, dy, wt, wf, res=res, res_mask=mask, share=3, spread=sp).float().cpu().numpy()
+        dx = ops.dgrad(s, dy, wt, wf, res=res, res_mask=mask, share=4, spread=sp).float().cpu().numpy()
         assert _rel(dx, dxo + reso * (masko > 0)) < tol
         dx = ops.dgrad(s, dy, wt, wf, spread=sp).float().cpu().numpy()
         assert _rel(dx, dxo) < tol

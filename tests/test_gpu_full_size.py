@@ -111,7 +111,7 @@ def test_forward_of_every_block_at_full_size():
 def test_backward_of_every_block_at_full_size():
     """The backward twin of the test above (Eq. 10 with the shrunk gradient of Eq. 15): ResNet-110, K = 4, batch 128,
     one stream per module plus the side stream of the weight gradients, i.e. the kernels and launch shapes the
-    benchmark's graphs replay (a convolution on a third of the SMs, the weight gradients' pixel split capped at
+    benchmark's graphs replay (a convolution on a quarter of the SMs, the weight gradients' pixel split capped at
     16 CTAs).  A capture keeps every gradient tensor of each module's backward pass at iteration 2K - 1, the first
     one in which all four modules back-propagate.  Every layer of every block is then recomputed by the oracle
     from the library's own inputs to that layer -- the incoming gradient it captured and the activations it saved
@@ -132,7 +132,7 @@ def test_backward_of_every_block_at_full_size():
 def test_bench_launch_shapes_against_oracle():
     """Forward, backward and update at the benchmark's layer shapes, batch and launch shapes, end to end
     against the oracle: a 6n+2 network with n = 2 (14 layers) cut into K = 4 modules, batch 128, graphs on.
-    Every convolution launch is then what the benchmark issues (128 image tiles on 32-43 CTAs, 3-4 tiles
+    Every convolution launch is then what the benchmark issues (128 image tiles on 32 CTAs, 4 tiles
     per CTA, per-CTA partial sums for both kinds of fused reduction, the pixel-split weight gradient),
     and the network is shallow enough for the oracle to run and for bfloat16 gate flips not to pile up
     (the comparison of a 110-layer gradient between two launch shapes of this same library differs by
