@@ -1291,8 +1291,9 @@ fdg_status fdg_create(const fdg_arch* arch, const fdg_config* cfg, void* dev_wor
   c->tmaps.share = c->cfg.serial ? 1 : c->K;
   c->tmaps.wgrad_side_cap = 16;
   // Blocks of a batch-norm apply kernel that first re-adds a convolution's partial sums: 4 per SM shared
-  // between the module streams (measured optimum: 148 blocks at K = 4, 296 at K = 2).
-  c->ew_block_cap = c->cfg.serial ? 4 * 148 : std::max(74, 4 * 148 / c->K);
+  // between the module streams, not fewer than 222 (measured: 222 blocks at K = 4 against 74 / 111 / 148 / 185 /
+  // 259 / 296; K = 2 is flat between 222 and 592).
+  c->ew_block_cap = c->cfg.serial ? 4 * 148 : std::max(222, 4 * 148 / c->K);
   c->graph_exec.assign(c->period, nullptr);
   c->graph_sig.assign(c->period, 0);
   c->graph_launches.assign(c->period, 0);
